@@ -1,0 +1,160 @@
+"""CPU oracle for the DCT compression path (test infrastructure, not product code).
+
+Thin ctypes front end of ``dct_oracle.cpp``: it marshals numpy arrays and adds
+no arithmetic of its own.  Only the tests, the smoke check and the benchmark's
+CPU-baseline leg may import this package; the CUDA path never does.
+
+fp32 data are ``numpy.float32`` arrays; bf16 data are ``numpy.uint16`` arrays
+holding the raw bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import NamedTuple, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dct_oracle.cpp")
+_LIB = os.path.join(_HERE, "libdct_oracle.so")
+
+_c_u64 = ctypes.c_uint64
+_c_u32 = ctypes.c_uint32
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no fast-math: denormals and RNE are kept)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(
+            ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-fno-fast-math",
+             "-ffp-contract=off", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        for name in ("oracle_dp_select", "oracle_dp_compress", "oracle_mp_fwd_f32",
+                     "oracle_mp_fwd_bf16", "oracle_mp_bwd_f32", "oracle_mp_bwd_bf16"):
+            getattr(_lib, name).restype = ctypes.c_int
+    return _lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _check(a: np.ndarray, dtype, name: str) -> np.ndarray:
+    if a.dtype != dtype or not a.flags["C_CONTIGUOUS"]:
+        raise TypeError(f"{name}: need C-contiguous {np.dtype(dtype).name}, got {a.dtype}")
+    return a
+
+
+class SelectResult(NamedTuple):
+    tau: np.float32
+    n_gt: int
+    n_eq: int
+
+
+class CompressResult(NamedTuple):
+    idx: np.ndarray      # int32[count], ascending
+    val: np.ndarray      # float32[count]
+    count: int           # survivors written (<= capacity)
+    needed: int          # survivors found
+
+
+def dp_select(grad: np.ndarray, residual: Optional[np.ndarray], k: int,
+              full_sort: bool = False) -> SelectResult:
+    """Algorithm 1, threshold steps: k-th largest |grad + residual| and tie counts."""
+    lib = _load()
+    _check(grad, np.float32, "grad")
+    if residual is not None:
+        _check(residual, np.float32, "residual")
+        assert residual.size == grad.size
+    tau = ctypes.c_float()
+    n_gt, n_eq = _c_u64(), _c_u64()
+    rc = lib.oracle_dp_select(_ptr(grad), _ptr(residual), _c_u64(grad.size), _c_u64(k),
+                              ctypes.c_int(1 if full_sort else 0),
+                              ctypes.byref(tau), ctypes.byref(n_gt), ctypes.byref(n_eq))
+    if rc:
+        raise ValueError(f"oracle_dp_select: invalid argument (rc={rc})")
+    return SelectResult(np.float32(tau.value), n_gt.value, n_eq.value)
+
+
+def dp_compress(grad: np.ndarray, residual: np.ndarray, tau, tie_budget: Optional[int],
+                capacity: int) -> CompressResult:
+    """Algorithm 1, mask / compressed gradient / error steps.  ``residual`` is updated in place."""
+    lib = _load()
+    _check(grad, np.float32, "grad")
+    _check(residual, np.float32, "residual")
+    assert residual.size == grad.size
+    idx = np.empty(capacity, dtype=np.int32)
+    val = np.empty(capacity, dtype=np.float32)
+    count, needed = _c_u64(), _c_u64()
+    rc = lib.oracle_dp_compress(_ptr(grad), _ptr(residual), _c_u64(grad.size),
+                                ctypes.c_float(float(np.float32(tau))),
+                                ctypes.c_int(0 if tie_budget is None else 1),
+                                _c_u64(0 if tie_budget is None else tie_budget),
+                                _ptr(idx), _ptr(val), _c_u64(capacity),
+                                ctypes.byref(count), ctypes.byref(needed))
+    if rc:
+        raise ValueError(f"oracle_dp_compress: invalid argument (rc={rc})")
+    c = count.value
+    return CompressResult(idx[:c].copy(), val[:c].copy(), c, needed.value)
+
+
+class MpFwdResult(NamedTuple):
+    cols: np.ndarray     # int16[rows, k], ascending within a row: the mask M
+    vals: np.ndarray     # [rows, k], dtype of x
+    tau: np.ndarray      # [rows], dtype of x: the row thresholds tau_i
+
+
+def mp_fwd(x: np.ndarray, k: int, d: Optional[int] = None) -> MpFwdResult:
+    """Algorithm 2, forward pass.  ``x`` is [rows, ld]; the first ``d`` columns of each row count."""
+    lib = _load()
+    assert x.ndim == 2
+    rows, ld = x.shape
+    d = ld if d is None else d
+    if x.dtype == np.float32:
+        fn = lib.oracle_mp_fwd_f32
+    elif x.dtype == np.uint16:
+        fn = lib.oracle_mp_fwd_bf16
+    else:
+        raise TypeError("x: float32 or uint16 (bf16 bits)")
+    _check(x, x.dtype, "x")
+    cols = np.empty((rows, k), dtype=np.int16)
+    vals = np.empty((rows, k), dtype=x.dtype)
+    tau = np.empty(rows, dtype=x.dtype)
+    rc = fn(_ptr(x), _c_u32(rows), _c_u32(d), _c_u32(ld), _c_u32(k),
+            _ptr(cols), _ptr(vals), _ptr(tau))
+    if rc:
+        raise ValueError(f"oracle_mp_fwd: invalid argument (rc={rc})")
+    return MpFwdResult(cols, vals, tau)
+
+
+def mp_bwd(gx: np.ndarray, cols: np.ndarray, d: Optional[int] = None) -> np.ndarray:
+    """Algorithm 2, backward pass: gather ``gx`` through the forward mask ``cols``."""
+    lib = _load()
+    assert gx.ndim == 2 and cols.ndim == 2 and gx.shape[0] == cols.shape[0]
+    rows, ld = gx.shape
+    d = ld if d is None else d
+    k = cols.shape[1]
+    if gx.dtype == np.float32:
+        fn = lib.oracle_mp_bwd_f32
+    elif gx.dtype == np.uint16:
+        fn = lib.oracle_mp_bwd_bf16
+    else:
+        raise TypeError("gx: float32 or uint16 (bf16 bits)")
+    _check(gx, gx.dtype, "gx")
+    _check(cols, np.int16, "cols")
+    gvals = np.empty((rows, k), dtype=gx.dtype)
+    rc = fn(_ptr(gx), _c_u32(rows), _c_u32(d), _c_u32(ld), _c_u32(k), _ptr(cols), _ptr(gvals))
+    if rc:
+        raise ValueError(f"oracle_mp_bwd: invalid argument (rc={rc})")
+    return gvals
