@@ -1,0 +1,525 @@
+#!/usr/bin/env python
+"""Benchmark of the DCT compression hot path on B200.
+
+One STEP is one threshold life-span of DCT-DP at the largest data-parallel configuration
+(2^30 fp32 gradients, density 0.01 %: one exact threshold select followed by 20 fixed-threshold
+hard-threshold + error-feedback + compaction iterations, residual resident in HBM) followed by 50
+DCT-MP iterations at production width (16384 x 4096 bf16, per-row top-k = 205: forward pack, then
+backward pack through the same mask).  Every input is synthetic and seeded, larger than L2, and
+resident in HBM before the timed region of the headline number.
+
+Metric: algorithmic GB/s of the whole step (bytes the method itself must move, see
+``algorithmic_bytes``) -- total over all ranks / max-over-ranks device time.  With N > 1 every
+rank runs the same per-GPU workload on its own data (independent layers / samples: weak scaling,
+no collective on the data path).
+
+``python bench.py --gpus N --steps K --warmup W`` prints ONE JSON line on rank 0.
+``--impl reference`` times the CPU oracle (the only reference there is) on host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2010_08899_b200 import inputs  # noqa: E402
+
+METRIC = "DCT compress GB/s (DP threshold+EF+pack; MP row top-k) vs HBM peak"
+UNIT = "GB/s"
+
+WORKLOADS = {
+    # configs[4] (DP large) + configs[3] (MP production width) of the baseline description
+    "dp_2p30_x20+mp_16384x4096_bf16_x50": dict(
+        dp_n=1 << 30, dp_k=107_375, dp_iters=20, dp_capacity=(1 << 30) // 256, dp_bufs=4, dp_slack=1 << 20,
+        mp_rows=16384, mp_d=4096, mp_k=205, mp_iters=50, mp_bufs=4),
+    # a small stand-in with the same structure, for quick functional runs (not a bench line)
+    "small": dict(
+        dp_n=1 << 22, dp_k=420, dp_iters=4, dp_capacity=(1 << 22) // 64, dp_bufs=2, dp_slack=1 << 12,
+        mp_rows=1024, mp_d=4096, mp_k=205, mp_iters=4, mp_bufs=2),
+}
+DEFAULT_WORKLOAD = "dp_2p30_x20+mp_16384x4096_bf16_x50"
+
+# DRAM bytes per element of the dominant kernel from the committed ncu capture
+# (profiles/dp_compress_kernel_*.md); None until a capture exists.
+NCU_DRAM_BYTES_PER_ELEM_COMPRESS = None
+
+
+def algorithmic_bytes(cfg, survivors_per_iter):
+    """Bytes the method must move in one step.
+    select: every element seen once (4 B); compress: read grad, read residual, write residual
+    (12 B/element) + 8 B per survivor; MP forward: read the matrix once, write (int16 col, value) per
+    kept slot; MP backward: read (col, value) per slot through the mask, write the value."""
+    n, rows, d, k = cfg["dp_n"], cfg["mp_rows"], cfg["mp_d"], cfg["mp_k"]
+    s = 2  # bf16
+    sel = 4 * n
+    cmp_ = sum(12 * n + 8 * c for c in survivors_per_iter)
+    fwd = cfg["mp_iters"] * (rows * d * s + rows * k * (2 + s))
+    bwd = cfg["mp_iters"] * (rows * k * (2 + s) + rows * k * s)
+    return dict(select=sel, compress=cmp_, mp_fwd=fwd, mp_bwd=bwd, total=sel + cmp_ + fwd + bwd)
+
+
+# --------------------------------------------------------------------------------------------
+# the CUDA arm
+# --------------------------------------------------------------------------------------------
+
+class HotPath:
+    """Per-rank buffers and the step function.  All kernels are the library's; torch only owns memory."""
+
+    def __init__(self, cfg, device, rank, total_steps):
+        from paper_2010_08899_b200 import binding as B
+        self.B, self.cfg, self.dev = B, cfg, device
+        self.L = B.lib()
+        c = cfg
+        n, seed0 = c["dp_n"], 10_000 * rank
+        self.g_sel = inputs.dp_mixture(n, 500 + seed0, device)
+        self.g = [inputs.dp_mixture(n + c["dp_slack"], 501 + j + seed0, device) for j in range(c["dp_bufs"])]
+        self.residual = torch.zeros(n, device=device)
+        self.tau = torch.zeros(1, device=device)
+        self.idx = torch.empty(c["dp_capacity"], dtype=torch.int32, device=device)
+        self.val = torch.empty(c["dp_capacity"], device=device)
+        self.ws_sel = B.new_workspace(B.dct_threshold_select_workspace_bytes(n), device)
+        self.ws_cmp = B.new_workspace(B.dct_dp_compress_workspace_bytes(n), device)
+        self.res_sel = B.new_result(device)
+        # one result block per compress call of the whole run, so survivor counts can be read afterwards
+        self.res_cmp = torch.zeros(total_steps * c["dp_iters"], 5, dtype=torch.int64, device=device)
+        rows, d, k = c["mp_rows"], c["mp_d"], c["mp_k"]
+        self.x = [inputs.mp_activations(rows, d, 410 + j + seed0, dtype=torch.bfloat16, device=device,
+                                        col_scale_seed=400) for j in range(c["mp_bufs"])]
+        self.gx = [inputs.mp_gradients(rows, d, 420 + j + seed0, dtype=torch.bfloat16, device=device)
+                   for j in range(c["mp_bufs"])]
+        self.cols = torch.empty(rows * k, dtype=torch.int16, device=device)
+        self.vals = torch.empty(rows * k, dtype=torch.bfloat16, device=device)
+        self.gvals = torch.empty(rows * k, dtype=torch.bfloat16, device=device)
+        self.res_mp = B.new_result(device)
+        self.t = 0            # DP iterations done so far (drives the gradient rotation)
+        self.calls = 0        # compress calls issued (indexes res_cmp)
+        self.launches = 0     # kernels of this library launched
+
+    def grad_view(self, t):
+        """Gradient of iteration t: buffer t mod B, shifted by a multiple of 4 elements so that every
+        element meets fresh values each time round (the residual persists across iterations)."""
+        c = self.cfg
+        buf = self.g[t % c["dp_bufs"]]
+        shift = 4 * ((t // c["dp_bufs"]) % (c["dp_slack"] // 4))
+        return buf[shift:shift + c["dp_n"]]
+
+    def step(self, stream, ev=None):
+        """One step on device-resident inputs.  ``ev`` (optional) collects CUDA events:
+        [start, after select, after each compress..., after MP]."""
+        c, L, s = self.cfg, self.L, stream.cuda_stream
+        n, cap = c["dp_n"], c["dp_capacity"]
+        rec = (lambda: ev.append(_record(stream))) if ev is not None else (lambda: None)
+        rec()
+        st = L.dct_threshold_select(self.g_sel.data_ptr(), None, n, c["dp_k"], self.tau.data_ptr(),
+                                    self.res_sel.data_ptr(), self.ws_sel.data_ptr(), self.ws_sel.numel(), s)
+        assert st == 0, st
+        rec()
+        tau_p, e_p, idx_p, val_p = self.tau.data_ptr(), self.residual.data_ptr(), self.idx.data_ptr(), self.val.data_ptr()
+        ws_p, ws_n = self.ws_cmp.data_ptr(), self.ws_cmp.numel()
+        for _ in range(c["dp_iters"]):
+            g = self.grad_view(self.t)
+            st = L.dct_dp_compress(g.data_ptr(), e_p, n, tau_p, None, idx_p, val_p, cap,
+                                   self.res_cmp[self.calls].data_ptr(), ws_p, ws_n, s)
+            assert st == 0, st
+            self.t += 1
+            self.calls += 1
+            rec()
+        rows, d, k = c["mp_rows"], c["mp_d"], c["mp_k"]
+        cols_p, vals_p, gv_p, res_p = self.cols.data_ptr(), self.vals.data_ptr(), self.gvals.data_ptr(), self.res_mp.data_ptr()
+        for i in range(c["mp_iters"]):
+            j = i % c["mp_bufs"]
+            st = L.dct_mp_topk_pack_fwd(self.x[j].data_ptr(), 1, rows, d, d, k, cols_p, vals_p, None, None, res_p, s)
+            assert st == 0, st
+            st = L.dct_mp_pack_bwd(self.gx[j].data_ptr(), 1, rows, d, d, k, cols_p, gv_p, res_p, s)
+            assert st == 0, st
+        rec()
+        self.launches += 4 + 2 * c["dp_iters"] + 2 * c["mp_iters"]
+
+    def time_mp_parts(self, stream, reps):
+        """Forward and backward pack timed on their own (after the main measurement)."""
+        c, L, s = self.cfg, self.L, stream.cuda_stream
+        rows, d, k = c["mp_rows"], c["mp_d"], c["mp_k"]
+        out = {}
+        for name in ("mp_fwd", "mp_bwd"):
+            for phase in range(2):   # warm-up, then timed
+                a = _record(stream)
+                for i in range(reps):
+                    j = i % c["mp_bufs"]
+                    if name == "mp_fwd":
+                        L.dct_mp_topk_pack_fwd(self.x[j].data_ptr(), 1, rows, d, d, k, self.cols.data_ptr(),
+                                               self.vals.data_ptr(), None, None, None, s)
+                    else:
+                        L.dct_mp_pack_bwd(self.gx[j].data_ptr(), 1, rows, d, d, k, self.cols.data_ptr(),
+                                          self.gvals.data_ptr(), None, s)
+                b = _record(stream)
+                b.synchronize()
+                out[name] = a.elapsed_time(b) / reps
+        return out
+
+
+class HostPath:
+    """The same step through the host-buffer entry points: every input crosses PCIe inside the step."""
+
+    def __init__(self, hp: HotPath):
+        c = hp.cfg
+        self.hp = hp
+        n = c["dp_n"]
+        self.g_sel = hp.g_sel.cpu().pin_memory()
+        self.g = [hp.g[j].cpu().pin_memory() for j in range(min(2, c["dp_bufs"]))]
+        self.g_dev = torch.empty(n, device=hp.dev)
+        self.idx_h = torch.empty(c["dp_capacity"], dtype=torch.int32).pin_memory()
+        self.val_h = torch.empty(c["dp_capacity"]).pin_memory()
+        self.res_h = torch.zeros(5, dtype=torch.int64).pin_memory()
+        self.x = [hp.x[j].cpu().pin_memory() for j in range(min(2, c["mp_bufs"]))]
+        self.gx = [hp.gx[j].cpu().pin_memory() for j in range(min(2, c["mp_bufs"]))]
+        self.x_dev, self.gx_dev = torch.empty_like(hp.x[0]), torch.empty_like(hp.gx[0])
+        slots = c["mp_rows"] * c["mp_k"]
+        self.cols_h = torch.empty(slots, dtype=torch.int16).pin_memory()
+        self.vals_h = torch.empty(slots, dtype=torch.bfloat16).pin_memory()
+        self.gv_h = torch.empty(slots, dtype=torch.bfloat16).pin_memory()
+        self.t = 0
+        self.h2d = 0
+        self.d2h = 0
+
+    def step(self, stream):
+        hp, c, L, s = self.hp, self.hp.cfg, self.hp.L, stream.cuda_stream
+        n, cap = c["dp_n"], c["dp_capacity"]
+        st = L.dct_threshold_select_host(self.g_sel.data_ptr(), self.g_dev.data_ptr(), None, n, c["dp_k"],
+                                         hp.tau.data_ptr(), None, hp.res_sel.data_ptr(), self.res_h.data_ptr(),
+                                         hp.ws_sel.data_ptr(), hp.ws_sel.numel(), s)
+        assert st == 0, st
+        self.h2d += 4 * n
+        self.d2h += 40
+        nb = len(self.g)
+        for _ in range(c["dp_iters"]):
+            buf = self.g[self.t % nb]
+            shift = 4 * ((self.t // nb) % (c["dp_slack"] // 4))
+            g = buf[shift:shift + n]
+            st = L.dct_dp_compress_host(g.data_ptr(), self.g_dev.data_ptr(), hp.residual.data_ptr(), n,
+                                        hp.tau.data_ptr(), None, hp.idx.data_ptr(), hp.val.data_ptr(), cap,
+                                        self.idx_h.data_ptr(), self.val_h.data_ptr(), hp.res_mp.data_ptr(),
+                                        self.res_h.data_ptr(), hp.ws_cmp.data_ptr(), hp.ws_cmp.numel(), s)
+            assert st in (0, 5), st
+            self.t += 1
+            self.h2d += 4 * n
+            self.d2h += 40 + 8 * int(self.res_h[1])
+        rows, d, k = c["mp_rows"], c["mp_d"], c["mp_k"]
+        for i in range(c["mp_iters"]):
+            j = i % len(self.x)
+            st = L.dct_mp_pack_host(self.x[j].data_ptr(), self.gx[j].data_ptr(), self.x_dev.data_ptr(),
+                                    self.gx_dev.data_ptr(), 1, rows, d, d, k, hp.cols.data_ptr(), hp.vals.data_ptr(),
+                                    hp.gvals.data_ptr(), self.cols_h.data_ptr(), self.vals_h.data_ptr(),
+                                    self.gv_h.data_ptr(), hp.res_mp.data_ptr(), self.res_h.data_ptr(), s)
+            assert st == 0, st
+            self.h2d += 2 * rows * d * 2
+            self.d2h += rows * k * 6 + 40
+
+
+def _record(stream):
+    e = torch.cuda.Event(enable_timing=True)
+    e.record(stream)
+    return e
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clock and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.proc, self.uuid = None, None
+        try:
+            self.uuid = "GPU-" + str(torch.cuda.get_device_properties(device_index).uuid)
+        except Exception:
+            self.uuid = None
+
+    def start(self):
+        cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+        if self.uuid:
+            cmd += ["-i", self.uuid]
+        try:
+            self.proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            text, _ = self.proc.communicate()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in text.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) != 7:
+                continue
+            try:
+                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[3:]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def reduce_over_ranks(elapsed_ms: float, units: float, device=None):
+    """(max over ranks of elapsed, sum over ranks of units); identity without a process group."""
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return elapsed_ms, units
+    t = torch.tensor([elapsed_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+# --------------------------------------------------------------------------------------------
+# the CPU oracle arm (reference / cpu_baseline)
+# --------------------------------------------------------------------------------------------
+
+def oracle_sample_step(cfg, scale_div, state=None):
+    """One step of the same schedule on a 1/scale_div sample, run by the CPU oracle as it stands.
+    Returns (seconds, algorithmic bytes, state)."""
+    import numpy as np
+    import oracle
+    n = max(cfg["dp_n"] // scale_div, 4096)
+    rows = max(cfg["mp_rows"] // scale_div, 8)
+    k_dp = max(cfg["dp_k"] // scale_div, 1)
+    d, k = cfg["mp_d"], cfg["mp_k"]
+    if state is None:
+        state = dict(
+            g_sel=inputs.dp_mixture(n, 500).numpy(),
+            g=[inputs.dp_mixture(n + cfg["dp_slack"], 501 + j).numpy() for j in range(2)],
+            e=np.zeros(n, np.float32), t=0,
+            x=[inputs.mp_activations(rows, d, 410 + j, dtype=torch.bfloat16, col_scale_seed=400)
+               .view(torch.int16).numpy().view(np.uint16) for j in range(2)],
+            gx=[inputs.mp_gradients(rows, d, 420 + j, dtype=torch.bfloat16)
+                .view(torch.int16).numpy().view(np.uint16) for j in range(2)])
+    sub = dict(cfg, dp_n=n, mp_rows=rows)
+    t0 = time.perf_counter()
+    tau = oracle.dp_select(state["g_sel"], None, k_dp).tau
+    counts = []
+    for _ in range(cfg["dp_iters"]):
+        t = state["t"]
+        shift = 4 * ((t // 2) % (cfg["dp_slack"] // 4))
+        g = state["g"][t % 2][shift:shift + n]
+        r = oracle.dp_compress(g, state["e"], tau, None, max(cfg["dp_capacity"] // scale_div, 1024))
+        counts.append(r.count)
+        state["t"] += 1
+    for i in range(cfg["mp_iters"]):
+        f = oracle.mp_fwd(state["x"][i % 2], k)
+        oracle.mp_bwd(state["gx"][i % 2], f.cols)
+    dt = time.perf_counter() - t0
+    return dt, algorithmic_bytes(sub, counts)["total"], state
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    scale = 64
+    state = None
+    for _ in range(max(args.warmup, 1)):
+        _, _, state = oracle_sample_step(cfg, scale, state)
+    times, nbytes = [], 0
+    for _ in range(args.steps):
+        dt, b, state = oracle_sample_step(cfg, scale, state)
+        times.append(dt)
+        nbytes += b
+    total = sum(times)
+    value = nbytes / total / 1e9
+    sample = (f"each step = the full schedule (1 select + {cfg['dp_iters']} compress + {cfg['mp_iters']} MP fwd+bwd) "
+              f"on a 1/{scale} sample: {cfg['dp_n'] // scale} gradients, {cfg['mp_rows'] // scale} rows")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32+bf16",
+        "data": "synthetic", "config": {"workload": args.workload, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------
+# main
+# --------------------------------------------------------------------------------------------
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=1, help="steps of the host-buffer (end to end) measurement")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = WORKLOADS[args.workload]
+
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the DCT kernels have no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    stream = torch.cuda.current_stream()
+    total_steps = args.warmup + args.steps
+    hp = HotPath(cfg, device, rank, total_steps)
+    torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        hp.step(stream)
+    barrier()
+    launches_before = hp.launches
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    events = []
+    barrier()
+    t_start = _record(stream)
+    for _ in range(args.steps):
+        ev = []
+        hp.step(stream, ev)
+        events.append(ev)
+    t_stop = _record(stream)
+    barrier()
+    clocks = sampler.stop()
+    elapsed_ms = t_start.elapsed_time(t_stop)
+    gpu_launches = hp.launches - launches_before
+
+    # survivor counts of the timed compress calls -> algorithmic bytes
+    res = hp.res_cmp.cpu()
+    timed = res[args.warmup * cfg["dp_iters"]:]
+    statuses = sorted(set((timed[:, 0] & 0xFFFFFFFF).tolist()))
+    counts = timed[:, 1].tolist()
+    per_step = [algorithmic_bytes(cfg, counts[i * cfg["dp_iters"]:(i + 1) * cfg["dp_iters"]]) for i in range(args.steps)]
+    my_bytes = float(sum(p["total"] for p in per_step))
+    max_ms, all_bytes = reduce_over_ranks(elapsed_ms, my_bytes, device)
+    value = all_bytes / (max_ms * 1e-3) / 1e9
+
+    # per-part device times from the events of the timed region
+    n = cfg["dp_n"]
+    sel_ms = [ev[0].elapsed_time(ev[1]) for ev in events]
+    cmp_ms = [ev[1 + i].elapsed_time(ev[2 + i]) for ev in events for i in range(cfg["dp_iters"])]
+    mp_ms = [ev[1 + cfg["dp_iters"]].elapsed_time(ev[2 + cfg["dp_iters"]]) for ev in events]
+    cmp_avg_ms = sum(cmp_ms) / len(cmp_ms)
+    cmp_bytes_avg = sum(12 * n + 8 * c for c in counts) / len(counts)
+    peak, peak_kind = measured_peaks()
+    achieved = cmp_bytes_avg / (cmp_avg_ms * 1e-3) / 1e9
+    mp_parts = hp.time_mp_parts(stream, cfg["mp_iters"])
+    b0 = per_step[0]
+    parts = {
+        "select": {"ms": statistics.mean(sel_ms), "GBps_at_4B_per_elem": 4 * n / (statistics.mean(sel_ms) * 1e-3) / 1e9},
+        "compress": {"ms": cmp_avg_ms, "GBps": achieved, "survivors_first_last": [counts[0], counts[-1]]},
+        "mp_fwd+bwd_block": {"ms": statistics.mean(mp_ms)},
+        "mp_fwd": {"ms": mp_parts["mp_fwd"], "GBps": b0["mp_fwd"] / cfg["mp_iters"] / (mp_parts["mp_fwd"] * 1e-3) / 1e9},
+        "mp_bwd": {"ms": mp_parts["mp_bwd"], "GBps": b0["mp_bwd"] / cfg["mp_iters"] / (mp_parts["mp_bwd"] * 1e-3) / 1e9,
+                   "dense_equiv_GBps": cfg["mp_rows"] * cfg["mp_d"] * 2 / (mp_parts["mp_bwd"] * 1e-3) / 1e9},
+    }
+    roofline = {
+        "kernel": "dp_compress_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_kind": peak_kind,
+        "traffic": None if NCU_DRAM_BYTES_PER_ELEM_COMPRESS is None else NCU_DRAM_BYTES_PER_ELEM_COMPRESS * n,
+        "algorithmic_bytes_per_launch": cmp_bytes_avg,
+        "frac_of_nominal_8TBps": achieved / 8000.0,
+        "note": "duration = CUDA events around each dct_dp_compress call (descriptor-reset kernel included)",
+    }
+
+    # end to end: the same step through the host-buffer entry points
+    e2e = None
+    if not args.no_e2e:
+        host = HostPath(hp)
+        torch.cuda.synchronize()
+        barrier()
+        t0 = time.perf_counter()
+        a = _record(stream)
+        for _ in range(args.e2e_steps):
+            host.step(stream)
+        b = _record(stream)
+        barrier()
+        e2e_ms = max(a.elapsed_time(b), 0.0)
+        wall_ms = (time.perf_counter() - t0) * 1e3
+        e2e_ms = max(e2e_ms, wall_ms)       # the host-buffer calls synchronise, so wall time is the honest one
+        e2e_bytes = float(sum(p["total"] for p in per_step[:1])) * args.e2e_steps
+        m_ms, a_bytes = reduce_over_ranks(e2e_ms, e2e_bytes, device)
+        e2e = {"value": a_bytes / (m_ms * 1e-3) / 1e9, "unit": UNIT, "steps": args.e2e_steps,
+               "ms_per_step": m_ms / args.e2e_steps,
+               "h2d_bytes_per_step": host.h2d // args.e2e_steps, "d2h_bytes_per_step": host.d2h // args.e2e_steps}
+        del host
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        scale = 16 if args.workload == DEFAULT_WORKLOAD else 4
+        dt, nbytes, _ = oracle_sample_step(cfg, scale)
+        cpu_baseline = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
+                        "sample": f"one full-schedule step on a 1/{scale} sample "
+                                  f"({cfg['dp_n'] // scale} gradients, {cfg['mp_rows'] // scale} rows)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": max_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32+bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "l2": "inputs_larger_than_l2",
+                       "dp": {"n": n, "k": cfg["dp_k"], "iters_per_select": cfg["dp_iters"],
+                              "capacity": cfg["dp_capacity"], "rotating_buffers": cfg["dp_bufs"]},
+                       "mp": {"rows": cfg["mp_rows"], "d": cfg["mp_d"], "k": cfg["mp_k"], "dtype": "bf16",
+                              "iters": cfg["mp_iters"], "rotating_buffers": cfg["mp_bufs"]},
+                       "parallelism": f"independent replicas x{world} (no data-path collective)"},
+            "elements_per_s": (n * cfg["dp_iters"] + cfg["mp_rows"] * cfg["mp_d"] * cfg["mp_iters"]) * world
+                              / (max_ms / args.steps * 1e-3),
+            "roofline": roofline, "parts": parts, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": gpu_launches, "clocks": clocks, "device_status_codes": statuses,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

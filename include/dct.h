@@ -1,0 +1,260 @@
+/*
+ * dct.h -- C ABI of the B200 (sm_100a) compression library for Dynamic
+ * Communication Thresholding (DCT).
+ *
+ * The library implements the two compression operators of the paper:
+ *
+ *   DCT-DP (Algorithm 1): error feedback W = W_grad + E_grad; every L
+ *   iterations a threshold tau = order statistic of |W|; mask M = I(|W| >= tau);
+ *   compressed gradient W_hat = W .* M (sent); error E = W - W_hat (kept).
+ *
+ *   DCT-MP (Algorithm 2): per sample i a threshold tau_i = order statistic of
+ *   |X_act,i|; mask m_i = I(|X_act,i| >= tau_i); X_act .* M and M are sent in
+ *   the forward pass, X_grad .* M (same mask) in the backward pass.
+ *
+ * Conventions common to every entry point
+ *   - Unless a parameter says "host", every pointer is a DEVICE pointer that
+ *     the caller owns.  The library allocates nothing and keeps no state
+ *     between calls.
+ *   - Every call is asynchronous on `stream` (a cudaStream_t passed as an
+ *     opaque pointer; NULL is the legacy default stream).  No call
+ *     synchronises with the host, except the *_host convenience calls.
+ *   - The return value reports what the host can see before launching
+ *     (arguments, workspace size, launch errors).  Conditions only the device
+ *     can see (output capacity exceeded, a bounded device-side wait giving up,
+ *     an out-of-range mask column) are written to `result->status` once the
+ *     stream reaches that point.
+ *   - Magnitudes are ordered by key(x) = bit pattern of x with the sign bit
+ *     cleared, compared as an unsigned integer (uint32 for fp32, uint16 for
+ *     bf16).  For non-NaN x this is the order of |x| with -0 == +0.  Ties in
+ *     key are broken by the lower index / column.
+ *   - Inputs are expected to be finite.  NaN/Inf do not trap and are handled
+ *     deterministically (they order above every finite magnitude), but are
+ *     outside the bit-exactness contract.
+ */
+#ifndef DCT_H_
+#define DCT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(_WIN32)
+#define DCT_API
+#else
+#define DCT_API __attribute__((visibility("default")))
+#endif
+
+typedef enum {
+  DCT_OK              = 0,
+  DCT_ERR_INVALID_ARG = 1, /* host: null pointer, k == 0, k > n, d > 32768, n > 2^31-1, aliasing */
+  DCT_ERR_WORKSPACE   = 2, /* host: workspace_bytes below dct_*_workspace_bytes(n), or misaligned */
+  DCT_ERR_UNSUPPORTED = 3, /* host: dtype or shape outside the supported set */
+  DCT_ERR_CUDA        = 4, /* host: a CUDA runtime call failed (see dct_last_cuda_error) */
+  DCT_ERR_CAPACITY    = 5, /* device: survivors > capacity; output truncated, the rest kept in the residual */
+  DCT_ERR_TIMEOUT     = 6, /* device: a bounded device-side wait gave up; outputs are incomplete */
+  DCT_ERR_BAD_MASK    = 7  /* device: a mask column >= d was met in dct_mp_pack_bwd; that slot was skipped */
+} dct_status_t;
+
+typedef enum { DCT_F32 = 0, DCT_BF16 = 1 } dct_dtype_t;
+
+/* cudaStream_t, passed opaquely so that this header needs no CUDA header. */
+typedef void* dct_stream_t;
+
+/* Result block in DEVICE memory, written by the kernels of one call. */
+typedef struct {
+  uint32_t status;   /* DCT_OK, DCT_ERR_CAPACITY, DCT_ERR_TIMEOUT or DCT_ERR_BAD_MASK */
+  uint32_t reserved;
+  uint64_t count;    /* compress: survivors written (<= capacity) */
+  uint64_t needed;   /* compress: survivors found (may exceed capacity) */
+  uint64_t n_gt;     /* select: #{ |w| >  tau } */
+  uint64_t n_eq;     /* select: #{ |w| == tau };  n_gt < k <= n_gt + n_eq */
+} dct_result_t;
+
+/* Human-readable name of a status code (static storage, never NULL). */
+DCT_API const char* dct_status_string(dct_status_t s);
+
+/* Text of the last CUDA runtime error seen by this thread inside the library. */
+DCT_API const char* dct_last_cuda_error(void);
+
+/* Bytes of device workspace the calls below need for a vector of n elements.
+ * The workspace must be 256-byte aligned; its contents need not be preserved
+ * between calls and two calls that may overlap on the GPU need separate ones. */
+DCT_API size_t dct_threshold_select_workspace_bytes(uint64_t n);
+DCT_API size_t dct_dp_compress_workspace_bytes(uint64_t n);
+
+/*
+ * dct_threshold_select -- Algorithm 1, "Error Feedback", "Sort(|W_grad|)" and
+ * "Assign tau" steps (the branch taken when L divides the iteration number).
+ *
+ * Computes tau = the k-th LARGEST value of |fl32(grad[i] + residual[i])|,
+ * i.e. the order statistic that leaves exactly k survivors when there are no
+ * ties.  (The paper's tau = w_floor(N*eta) of the ascending sort with eta the
+ * fraction dropped corresponds to k = N - floor(N*eta).)  Nothing is modified
+ * except the outputs.
+ *
+ *   grad      [n] fp32, read-only.
+ *   residual  [n] fp32, read-only, or NULL for E_grad = 0.
+ *   n, k      1 <= k <= n <= 2^31-1.
+ *   tau_out   1 fp32 (device): the threshold, sign bit clear.
+ *   result    device block; n_gt, n_eq and status are written.
+ *   workspace >= dct_threshold_select_workspace_bytes(n), 256-byte aligned.
+ *
+ * Returns DCT_OK after enqueueing; DCT_ERR_INVALID_ARG / DCT_ERR_WORKSPACE /
+ * DCT_ERR_CUDA without having launched anything.
+ */
+DCT_API dct_status_t dct_threshold_select(
+    const float* grad, const float* residual, uint64_t n, uint64_t k,
+    float* tau_out, dct_result_t* result,
+    void* workspace, size_t workspace_bytes, dct_stream_t stream);
+
+/*
+ * dct_dp_compress -- Algorithm 1, "Error Feedback", "Compute mask", "Compute
+ * compressed gradient", "Compute error" and the payload of "Send" for a fixed
+ * threshold (the branch that reuses tau from an earlier iteration, or the one
+ * that follows dct_threshold_select on the same stream).
+ *
+ * For every i:  w = fl32(grad[i] + residual[i]);
+ *   pass(i) = key(w) > key(*tau)  ||  (key(w) == key(*tau) && fewer than
+ *             *tie_budget earlier elements had key == key(*tau));
+ *   with tie_budget == NULL the second clause is simply key(w) == key(*tau),
+ *   which is the paper's M = I(|W| >= tau).
+ * Survivors are written in ascending i as (idx_out[j], val_out[j]) = (i, w)
+ * while j < capacity; residual[i] becomes +0.0 for an element that was written
+ * and w for every other element, so  sent + residual == grad + old residual
+ * holds for every i even when the capacity is exceeded.
+ *
+ *   grad       [n] fp32, read-only; must not overlap residual.
+ *   residual   [n] fp32, in/out.
+ *   n          1 <= n <= 2^31-1.
+ *   tau        1 fp32 (device); its magnitude is used.
+ *   tie_budget 1 uint64 (device) or NULL.  Passing k - n_gt from a select on
+ *              the same vector yields exactly k survivors.
+ *   idx_out    [capacity] int32;  val_out [capacity] fp32.  Entries at and
+ *              beyond result->count are left untouched.
+ *   result     device block; count, needed and status (DCT_OK,
+ *              DCT_ERR_CAPACITY or DCT_ERR_TIMEOUT) are written.
+ *   workspace  >= dct_dp_compress_workspace_bytes(n), 256-byte aligned.
+ *
+ * grad and residual should be 16-byte aligned; other alignments are accepted
+ * and take a slower scalar path.
+ */
+DCT_API dct_status_t dct_dp_compress(
+    const float* grad, float* residual, uint64_t n,
+    const float* tau, const uint64_t* tie_budget,
+    int32_t* idx_out, float* val_out, uint64_t capacity,
+    dct_result_t* result,
+    void* workspace, size_t workspace_bytes, dct_stream_t stream);
+
+/*
+ * dct_mp_topk_pack_fwd -- Algorithm 2, forward pass: for every sample (row) i
+ * sort |X_act,i|, take tau_i, build m_i, and pack X_act .* M together with M.
+ *
+ * Keeps exactly k columns per row: every column whose key exceeds key(tau_i),
+ * then the lowest columns with key == key(tau_i) until k are kept, where tau_i
+ * is the k-th largest magnitude of the row.
+ *
+ *   x_act    [rows, ld] row-major, dtype fp32 or bf16, read-only; only the
+ *            first d columns of a row are looked at.
+ *   rows     >= 1;  1 <= k <= d <= 32768;  ld >= d (elements).
+ *   cols_out [rows*k] int16: kept columns, ascending within a row.  This IS
+ *            the mask M; hand it unchanged to dct_mp_pack_bwd.
+ *   vals_out [rows*k] dtype of x_act: x_act[i, cols_out[i*k+s]] (bit copies).
+ *   rows_out [rows*k] int32 or NULL: explicit row id of each slot for callers
+ *            that want (row, col, val) triples; the row is otherwise slot / k.
+ *   tau_out  [rows] dtype of x_act or NULL: the thresholds tau_i (sign clear).
+ *   result   device block or NULL; status is written (always DCT_OK).
+ *
+ * x_act rows should start on 16-byte boundaries (base aligned and ld*size a
+ * multiple of 16); other layouts are accepted and take a slower scalar load.
+ */
+DCT_API dct_status_t dct_mp_topk_pack_fwd(
+    const void* x_act, dct_dtype_t dtype,
+    uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+    int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+    dct_result_t* result, dct_stream_t stream);
+
+/*
+ * dct_mp_pack_bwd -- Algorithm 2, backward pass: X_grad .* M packed through
+ * the mask of the forward pass:  gvals_out[i*k+s] = x_grad[i, cols[i*k+s]].
+ *
+ *   x_grad    [rows, ld] row-major, dtype fp32 or bf16, read-only.
+ *   cols      [rows*k] int16 from dct_mp_topk_pack_fwd, read-only.
+ *   gvals_out [rows*k] dtype of x_grad.
+ *   result    device block or NULL; status is DCT_OK, or DCT_ERR_BAD_MASK if
+ *             some column was outside [0, d) (that slot is written as zero and
+ *             nothing out of bounds is read).
+ */
+DCT_API dct_status_t dct_mp_pack_bwd(
+    const void* x_grad, dct_dtype_t dtype,
+    uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+    const int16_t* cols, void* gvals_out,
+    dct_result_t* result, dct_stream_t stream);
+
+/*
+ * Host-buffer convenience calls: the same operators for a caller whose data
+ * lives in HOST memory (pinned memory gives full copy speed; pageable memory
+ * works).  Each call copies its inputs to the caller-provided device staging
+ * buffers, runs the device entry point above, copies the packed result back
+ * and waits for the stream before returning.
+ *
+ * dct_dp_compress_host: one DCT-DP iteration for a host gradient.  The
+ * residual stays resident on the device (it is state carried across
+ * iterations).
+ *   grad_host        [n] fp32, host.
+ *   grad_dev         [n] fp32 device staging buffer.
+ *   residual_dev, tau_dev, tie_budget_dev, idx_dev, val_dev, result_dev,
+ *   workspace        as in dct_dp_compress (device).
+ *   idx_host/val_host [capacity] host buffers receiving the first count pairs.
+ *   result_host      host copy of the result block.
+ * Returns the host-visible status, or the device-reported status of the call.
+ */
+DCT_API dct_status_t dct_dp_compress_host(
+    const float* grad_host, float* grad_dev, float* residual_dev, uint64_t n,
+    const float* tau_dev, const uint64_t* tie_budget_dev,
+    int32_t* idx_dev, float* val_dev, uint64_t capacity,
+    int32_t* idx_host, float* val_host,
+    dct_result_t* result_dev, dct_result_t* result_host,
+    void* workspace, size_t workspace_bytes, dct_stream_t stream);
+
+/*
+ * dct_threshold_select_host: threshold select for a host gradient (residual,
+ * if any, resident on the device).  tau stays on the device for the compress
+ * calls that follow; tau_host (optional) and result_host receive copies.
+ */
+DCT_API dct_status_t dct_threshold_select_host(
+    const float* grad_host, float* grad_dev, const float* residual_dev, uint64_t n, uint64_t k,
+    float* tau_dev, float* tau_host, dct_result_t* result_dev, dct_result_t* result_host,
+    void* workspace, size_t workspace_bytes, dct_stream_t stream);
+
+/*
+ * dct_mp_pack_host: forward top-k pack of a host activation matrix followed by
+ * the backward pack of a host gradient matrix through the same mask.
+ *   x_act_host/x_grad_host [rows, ld] host; x_act_dev/x_grad_dev device staging.
+ *   cols_dev/vals_dev/gvals_dev [rows*k] device; cols_host/vals_host/gvals_host
+ *   [rows*k] host buffers receiving the packed results.
+ */
+DCT_API dct_status_t dct_mp_pack_host(
+    const void* x_act_host, const void* x_grad_host, void* x_act_dev, void* x_grad_dev,
+    dct_dtype_t dtype, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+    int16_t* cols_dev, void* vals_dev, void* gvals_dev,
+    int16_t* cols_host, void* vals_host, void* gvals_host,
+    dct_result_t* result_dev, dct_result_t* result_host, dct_stream_t stream);
+
+/*
+ * Testing knobs (process-wide, not for production use).  spin_limit is the
+ * number of polls a device-side wait may take before it gives up with
+ * DCT_ERR_TIMEOUT (default 2^21, about a second).  first_ticket is the id of
+ * the first tile dct_dp_compress hands out (default 0); with 1, tile 0 is never
+ * processed, so its successor's bounded wait can be observed to run out without
+ * wedging the GPU.  The paper has no counterpart for this call.
+ */
+DCT_API void dct_debug_configure(uint32_t spin_limit, uint32_t first_ticket);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DCT_H_ */

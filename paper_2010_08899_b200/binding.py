@@ -1,0 +1,311 @@
+"""Python binding of the C ABI in ``include/dct.h``: argument marshalling only.
+
+Every function here has the name and the argument order of its C counterpart,
+takes torch tensors (used purely as device or host buffers), checks dtype and
+contiguity, and passes raw pointers to ``libdct_b200.so``.  No step of the
+method runs in Python or in PyTorch.  If the shared library cannot be loaded
+the import of a symbol fails loudly: there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import NamedTuple, Optional
+
+import torch
+
+from . import build as _build
+
+DCT_OK, DCT_ERR_INVALID_ARG, DCT_ERR_WORKSPACE, DCT_ERR_UNSUPPORTED = 0, 1, 2, 3
+DCT_ERR_CUDA, DCT_ERR_CAPACITY, DCT_ERR_TIMEOUT, DCT_ERR_BAD_MASK = 4, 5, 6, 7
+DCT_F32, DCT_BF16 = 0, 1
+
+RESULT_BYTES = 40          # sizeof(dct_result_t)
+
+# every symbol include/dct.h declares
+EXPORTED_SYMBOLS = (
+    "dct_status_string", "dct_last_cuda_error",
+    "dct_threshold_select_workspace_bytes", "dct_dp_compress_workspace_bytes",
+    "dct_threshold_select", "dct_dp_compress", "dct_mp_topk_pack_fwd", "dct_mp_pack_bwd",
+    "dct_dp_compress_host", "dct_mp_pack_host", "dct_threshold_select_host", "dct_debug_configure",
+)
+
+_vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
+_lib = None
+
+
+class DctError(RuntimeError):
+    def __init__(self, where: str, status: int):
+        self.status = status
+        name = lib().dct_status_string(status).decode()
+        extra = ""
+        if status == DCT_ERR_CUDA:
+            extra = ": " + lib().dct_last_cuda_error().decode()
+        super().__init__(f"{where}: {name}{extra}")
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib() -> ctypes.CDLL:
+    """Load (building first if the sources are newer) the CUDA library.  Raises if that fails."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build()
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing and could not be built: the DCT kernels have no fallback")
+    L = ctypes.CDLL(path)
+    L.dct_status_string.restype = ctypes.c_char_p
+    L.dct_status_string.argtypes = [_int]
+    L.dct_last_cuda_error.restype = ctypes.c_char_p
+    L.dct_last_cuda_error.argtypes = []
+    for f in (L.dct_threshold_select_workspace_bytes, L.dct_dp_compress_workspace_bytes):
+        f.restype = _sz
+        f.argtypes = [_u64]
+    L.dct_threshold_select.restype = _int
+    L.dct_threshold_select.argtypes = [_vp, _vp, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
+    L.dct_dp_compress.restype = _int
+    L.dct_dp_compress.argtypes = [_vp, _vp, _u64, _vp, _vp, _vp, _vp, _u64, _vp, _vp, _sz, _vp]
+    L.dct_mp_topk_pack_fwd.restype = _int
+    L.dct_mp_topk_pack_fwd.argtypes = [_vp, _int, _u32, _u32, _u32, _u32, _vp, _vp, _vp, _vp, _vp, _vp]
+    L.dct_mp_pack_bwd.restype = _int
+    L.dct_mp_pack_bwd.argtypes = [_vp, _int, _u32, _u32, _u32, _u32, _vp, _vp, _vp, _vp]
+    L.dct_dp_compress_host.restype = _int
+    L.dct_dp_compress_host.argtypes = [_vp, _vp, _vp, _u64, _vp, _vp, _vp, _vp, _u64, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+    L.dct_threshold_select_host.restype = _int
+    L.dct_threshold_select_host.argtypes = [_vp, _vp, _vp, _u64, _u64, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+    L.dct_mp_pack_host.restype = _int
+    L.dct_mp_pack_host.argtypes = [_vp, _vp, _vp, _vp, _int, _u32, _u32, _u32, _u32,
+                                   _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+    L.dct_debug_configure.restype = None
+    L.dct_debug_configure.argtypes = [_u32, _u32]
+    _lib = L
+    return L
+
+
+# ----------------------------------------------------------------------------
+# marshalling helpers
+# ----------------------------------------------------------------------------
+
+def _p(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _need(t: torch.Tensor, dtype, name: str, cuda: bool = True):
+    if t.dtype != dtype:
+        raise TypeError(f"{name}: expected {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous")
+    if cuda and not t.is_cuda:
+        raise ValueError(f"{name}: must be a CUDA tensor")
+    if not cuda and t.is_cuda:
+        raise ValueError(f"{name}: must be a host tensor")
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DCT_F32
+    if t.dtype == torch.bfloat16:
+        return DCT_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}: float32 or bfloat16")
+
+
+def _check(where: str, status: int):
+    if status != DCT_OK:
+        raise DctError(where, status)
+
+
+class Result(NamedTuple):
+    status: int
+    count: int
+    needed: int
+    n_gt: int
+    n_eq: int
+
+
+def new_result(device="cuda") -> torch.Tensor:
+    """A device buffer holding one dct_result_t."""
+    return torch.zeros(RESULT_BYTES // 8, dtype=torch.int64, device=device)
+
+
+def read_result(result: torch.Tensor) -> Result:
+    """Copy a result block to the host (synchronises) and decode it."""
+    r = result.cpu().tolist()
+    return Result(r[0] & 0xFFFFFFFF, r[1], r[2], r[3], r[4])
+
+
+def new_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A 256-byte aligned device workspace of at least ``nbytes`` bytes."""
+    t = torch.empty(max(nbytes, 256) + 256, dtype=torch.uint8, device=device)
+    off = (-t.data_ptr()) % 256
+    return t[off:off + max(nbytes, 256)]
+
+
+def k_from_sparsity(n: int, eta_num: int, eta_den: int) -> int:
+    """Survivor target for a sparsity factor eta = eta_num/eta_den (fraction dropped):
+    k = n - floor(n * eta), in exact integer arithmetic (Algorithm 1 / 2, threshold index)."""
+    if not (0 <= eta_num <= eta_den and eta_den > 0):
+        raise ValueError("need 0 <= eta <= 1")
+    return n - (n * eta_num) // eta_den
+
+
+def k_from_density(n: int, den_num: int, den_den: int) -> int:
+    """Survivor target for a kept fraction den_num/den_den: k = ceil(n * density)."""
+    return -((-n * den_num) // den_den)
+
+
+# ----------------------------------------------------------------------------
+# the C entry points
+# ----------------------------------------------------------------------------
+
+def dct_threshold_select_workspace_bytes(n: int) -> int:
+    return lib().dct_threshold_select_workspace_bytes(n)
+
+
+def dct_dp_compress_workspace_bytes(n: int) -> int:
+    return lib().dct_dp_compress_workspace_bytes(n)
+
+
+def dct_threshold_select(grad, residual, n, k, tau_out, result, workspace, stream=None) -> None:
+    _need(grad, torch.float32, "grad")
+    if residual is not None:
+        _need(residual, torch.float32, "residual")
+    _need(tau_out, torch.float32, "tau_out")
+    _need(result, torch.int64, "result")
+    _need(workspace, torch.uint8, "workspace")
+    if grad.numel() < n or (residual is not None and residual.numel() < n) or result.numel() * 8 < RESULT_BYTES:
+        raise ValueError("buffer smaller than n")
+    _check("dct_threshold_select",
+           lib().dct_threshold_select(_p(grad), _p(residual), n, k, _p(tau_out), _p(result),
+                                      _p(workspace), workspace.numel(), _stream(stream)))
+
+
+def dct_dp_compress(grad, residual, n, tau, tie_budget, idx_out, val_out, capacity, result, workspace,
+                    stream=None) -> None:
+    _need(grad, torch.float32, "grad")
+    _need(residual, torch.float32, "residual")
+    _need(tau, torch.float32, "tau")
+    if tie_budget is not None:
+        _need(tie_budget, torch.int64, "tie_budget")
+    _need(idx_out, torch.int32, "idx_out")
+    _need(val_out, torch.float32, "val_out")
+    _need(result, torch.int64, "result")
+    _need(workspace, torch.uint8, "workspace")
+    if grad.numel() < n or residual.numel() < n or idx_out.numel() < capacity or val_out.numel() < capacity:
+        raise ValueError("buffer smaller than n / capacity")
+    _check("dct_dp_compress",
+           lib().dct_dp_compress(_p(grad), _p(residual), n, _p(tau), _p(tie_budget), _p(idx_out), _p(val_out),
+                                 capacity, _p(result), _p(workspace), workspace.numel(), _stream(stream)))
+
+
+def dct_mp_topk_pack_fwd(x_act, rows, d, ld, k, cols_out, vals_out, rows_out=None, tau_out=None, result=None,
+                         stream=None) -> None:
+    code = _dtype_code(x_act)
+    _need(x_act, x_act.dtype, "x_act")
+    _need(cols_out, torch.int16, "cols_out")
+    _need(vals_out, x_act.dtype, "vals_out")
+    if rows_out is not None:
+        _need(rows_out, torch.int32, "rows_out")
+    if tau_out is not None:
+        _need(tau_out, x_act.dtype, "tau_out")
+    if result is not None:
+        _need(result, torch.int64, "result")
+    if ld >= d and rows >= 1 and k >= 1:
+        if (x_act.numel() < (rows - 1) * ld + d or cols_out.numel() < rows * k or vals_out.numel() < rows * k or
+                (rows_out is not None and rows_out.numel() < rows * k) or
+                (tau_out is not None and tau_out.numel() < rows)):
+            raise ValueError("buffer smaller than rows x ld / rows x k")
+    _check("dct_mp_topk_pack_fwd",
+           lib().dct_mp_topk_pack_fwd(_p(x_act), code, rows, d, ld, k, _p(cols_out), _p(vals_out), _p(rows_out),
+                                      _p(tau_out), _p(result), _stream(stream)))
+
+
+def dct_mp_pack_bwd(x_grad, rows, d, ld, k, cols, gvals_out, result=None, stream=None) -> None:
+    code = _dtype_code(x_grad)
+    _need(x_grad, x_grad.dtype, "x_grad")
+    _need(cols, torch.int16, "cols")
+    _need(gvals_out, x_grad.dtype, "gvals_out")
+    if result is not None:
+        _need(result, torch.int64, "result")
+    if ld >= d and rows >= 1 and k >= 1:
+        if x_grad.numel() < (rows - 1) * ld + d or cols.numel() < rows * k or gvals_out.numel() < rows * k:
+            raise ValueError("buffer smaller than rows x ld / rows x k")
+    _check("dct_mp_pack_bwd",
+           lib().dct_mp_pack_bwd(_p(x_grad), code, rows, d, ld, k, _p(cols), _p(gvals_out), _p(result),
+                                 _stream(stream)))
+
+
+def dct_dp_compress_host(grad_host, grad_dev, residual_dev, n, tau_dev, tie_budget_dev, idx_dev, val_dev, capacity,
+                         idx_host, val_host, result_dev, result_host, workspace, stream=None) -> Result:
+    """Returns the decoded host copy of the result block; DCT_ERR_CAPACITY is reported there, not raised."""
+    _need(grad_host, torch.float32, "grad_host", cuda=False)
+    _need(grad_dev, torch.float32, "grad_dev")
+    _need(residual_dev, torch.float32, "residual_dev")
+    _need(idx_host, torch.int32, "idx_host", cuda=False)
+    _need(val_host, torch.float32, "val_host", cuda=False)
+    _need(result_host, torch.int64, "result_host", cuda=False)
+    _need(idx_dev, torch.int32, "idx_dev")
+    _need(val_dev, torch.float32, "val_dev")
+    if min(grad_host.numel(), grad_dev.numel(), residual_dev.numel()) < n or \
+            min(idx_host.numel(), val_host.numel(), idx_dev.numel(), val_dev.numel()) < capacity:
+        raise ValueError("buffer smaller than n / capacity")
+    st = lib().dct_dp_compress_host(_p(grad_host), _p(grad_dev), _p(residual_dev), n, _p(tau_dev),
+                                    _p(tie_budget_dev), _p(idx_dev), _p(val_dev), capacity, _p(idx_host),
+                                    _p(val_host), _p(result_dev), _p(result_host), _p(workspace),
+                                    workspace.numel(), _stream(stream))
+    if st not in (DCT_OK, DCT_ERR_CAPACITY):
+        raise DctError("dct_dp_compress_host", st)
+    r = result_host.tolist()
+    return Result(r[0] & 0xFFFFFFFF, r[1], r[2], r[3], r[4])
+
+
+def dct_threshold_select_host(grad_host, grad_dev, residual_dev, n, k, tau_dev, tau_host, result_dev, result_host,
+                              workspace, stream=None) -> Result:
+    _need(grad_host, torch.float32, "grad_host", cuda=False)
+    _need(grad_dev, torch.float32, "grad_dev")
+    _need(tau_dev, torch.float32, "tau_dev")
+    _need(result_host, torch.int64, "result_host", cuda=False)
+    if min(grad_host.numel(), grad_dev.numel()) < n:
+        raise ValueError("buffer smaller than n")
+    _check("dct_threshold_select_host",
+           lib().dct_threshold_select_host(_p(grad_host), _p(grad_dev), _p(residual_dev), n, k, _p(tau_dev),
+                                           _p(tau_host), _p(result_dev), _p(result_host), _p(workspace),
+                                           workspace.numel(), _stream(stream)))
+    r = result_host.tolist()
+    return Result(r[0] & 0xFFFFFFFF, r[1], r[2], r[3], r[4])
+
+
+def dct_mp_pack_host(x_act_host, x_grad_host, x_act_dev, x_grad_dev, rows, d, ld, k, cols_dev, vals_dev, gvals_dev,
+                     cols_host, vals_host, gvals_host, result_dev, result_host, stream=None) -> None:
+    code = _dtype_code(x_act_host)
+    for t, nm in ((x_act_host, "x_act_host"), (x_grad_host, "x_grad_host"), (vals_host, "vals_host"),
+                  (gvals_host, "gvals_host")):
+        _need(t, x_act_host.dtype, nm, cuda=False)
+    for t, nm in ((x_act_dev, "x_act_dev"), (x_grad_dev, "x_grad_dev"), (vals_dev, "vals_dev"),
+                  (gvals_dev, "gvals_dev")):
+        _need(t, x_act_host.dtype, nm)
+    _need(cols_dev, torch.int16, "cols_dev")
+    _need(cols_host, torch.int16, "cols_host", cuda=False)
+    _need(result_host, torch.int64, "result_host", cuda=False)
+    if min(x_act_host.numel(), x_grad_host.numel(), x_act_dev.numel(), x_grad_dev.numel()) < rows * ld or \
+            min(cols_dev.numel(), vals_dev.numel(), gvals_dev.numel(), cols_host.numel(), vals_host.numel(),
+                gvals_host.numel()) < rows * k:
+        raise ValueError("buffer smaller than rows x ld / rows x k")
+    _check("dct_mp_pack_host",
+           lib().dct_mp_pack_host(_p(x_act_host), _p(x_grad_host), _p(x_act_dev), _p(x_grad_dev), code, rows, d, ld,
+                                  k, _p(cols_dev), _p(vals_dev), _p(gvals_dev), _p(cols_host), _p(vals_host),
+                                  _p(gvals_host), _p(result_dev), _p(result_host), _stream(stream)))
+
+
+def dct_debug_configure(spin_limit: int = 1 << 21, first_ticket: int = 0) -> None:
+    """Testing knobs: iteration limit of device-side waits, and the first tile ticket of dct_dp_compress
+    (a non-zero value leaves tile 0 unprocessed so that the bounded wait can be seen to give up)."""
+    lib().dct_debug_configure(spin_limit, first_ticket)

@@ -1,0 +1,126 @@
+"""GPU parity of DCT-MP (per-row top-k + forward pack, backward pack through the same mask)
+against the CPU oracle: bit-exact on the same seeded inputs, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2010_08899_b200 import binding as B
+from paper_2010_08899_b200 import inputs
+from tests import _gpu as G
+
+pytestmark = pytest.mark.gpu
+
+
+def _compare_fwd_bwd(x_dev, gx_dev, d, k, want_rows=False):
+    rows = x_dev.shape[0]
+    want = oracle.mp_fwd(G.to_oracle(x_dev), k, d=d)
+    cols, vals, tau, rws = G.mp_fwd(x_dev, d, k, want_rows=want_rows)
+    assert np.array_equal(cols.cpu().numpy(), want.cols)
+    assert np.array_equal(G.as_np_bits(vals), want.vals.view(G.as_np_bits(vals).dtype))
+    assert np.array_equal(G.as_np_bits(tau), want.tau.view(G.as_np_bits(tau).dtype))
+    if want_rows:
+        assert np.array_equal(rws.cpu().numpy(), np.repeat(np.arange(rows, dtype=np.int32)[:, None], k, 1))
+    if gx_dev is not None:
+        cols_before = cols.clone()
+        gv, r = G.mp_bwd(gx_dev, d, cols)
+        assert r.status == B.DCT_OK
+        assert torch.equal(cols, cols_before)                  # the mask is consumed unchanged
+        want_g = oracle.mp_bwd(G.to_oracle(gx_dev), want.cols, d=d)
+        assert np.array_equal(G.as_np_bits(gv), want_g.view(G.as_np_bits(gv).dtype))
+    return cols
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d,ld", [(1, 1), (7, 7), (33, 40), (1000, 1000), (1024, 1024), (4097, 4100),
+                                  (5000, 5000), (32768, 32768)])
+def test_mp_odd_shapes(dtype, d, ld):
+    rows = 37 if d < 8192 else 5
+    x = inputs.mp_activations(rows, d, 50 + d, dtype=dtype, device=G.DEV, col_scale_seed=60 + d, ld=ld)
+    gx = inputs.mp_gradients(rows, d, 70 + d, dtype=dtype, device=G.DEV, ld=ld)
+    for k in sorted({1, min(d, 2), max(1, d // 20), max(1, d // 2), max(1, d - 1), d}):
+        cols = _compare_fwd_bwd(x, gx, d, k, want_rows=(k == 1))
+        assert int(cols.max()) < d
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_mp_misaligned_rows(dtype):
+    rows, d, ld, k = 20, 301, 303, 31
+    x = inputs.mp_activations(rows, d, 5, dtype=dtype, device=G.DEV, ld=ld)
+    gx = inputs.mp_gradients(rows, d, 6, dtype=dtype, device=G.DEV, ld=ld)
+    xo = G.offset_copy(x, 1).view(rows, ld)
+    go = G.offset_copy(gx, 3).view(rows, ld)
+    _compare_fwd_bwd(xo, go, d, k)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_mp_ties_signs_and_degenerate_rows(dtype):
+    rows, d = 64, 2048
+    sign = torch.where(inputs.dp_gaussian(rows * d, 1, G.DEV).view(rows, d) > 0, 1.0, -1.0)
+    x = inputs.quantize_mantissa(inputs.mp_activations(rows, d, 2, device=G.DEV, col_scale_seed=3), 1) * sign
+    x[0] = 0.0                                   # all zero: pure lowest-column rule
+    x[1] = 3.0                                   # all equal
+    x[2] = torch.tensor([1.5, -1.5], device=G.DEV).repeat(d // 2)
+    x[3] = 0.0
+    x[3, 5] = -1e30                              # one outlier, rest zeros
+    x[4] = torch.arange(d, device=G.DEV) * 1e-42   # denormals (fp32) / zeros after bf16 rounding
+    x = x.to(dtype).contiguous()
+    gx = inputs.mp_gradients(rows, d, 4, dtype=dtype, device=G.DEV)
+    for k in (1, 64, 102, 1024, d):
+        _compare_fwd_bwd(x, gx, d, k)
+
+
+def test_config2_mp_small():
+    """2048 x 1024 fp32, ReLU of N(0,1), k = 64; plus a tie-injected copy."""
+    rows, d, k = 2048, 1024, 64
+    x = inputs.mp_activations(rows, d, 100, device=G.DEV)
+    gx = inputs.mp_gradients(rows, d, 101, device=G.DEV)
+    zero_frac = float((x == 0).float().mean())
+    assert 0.45 < zero_frac < 0.55
+    _compare_fwd_bwd(x, gx, d, k, want_rows=True)
+    _compare_fwd_bwd(inputs.quantize_mantissa(x, 4), gx, d, k)
+
+
+def test_config4_mp_production_width():
+    """16384 x 4096 bf16, ReLU of N(0,1) with per-column LogNormal scale, k = 205 (5 %)."""
+    rows, d, k = 16384, 4096, 205
+    assert k == B.k_from_sparsity(d, 95, 100)
+    x = inputs.mp_activations(rows, d, 410, dtype=torch.bfloat16, device=G.DEV, col_scale_seed=400)
+    gx = inputs.mp_gradients(rows, d, 420, dtype=torch.bfloat16, device=G.DEV)
+    cols = _compare_fwd_bwd(x, gx, d, k)
+    # ties at tau_i are the common case in bf16: make sure the input really exercises them
+    keys = (x.view(torch.int16).to(torch.int32) & 0x7FFF)
+    kth = torch.topk(keys, k, dim=1).values[:, -1:]
+    tied_rows = ((keys == kth).sum(1) > 1).float().mean().item()
+    assert tied_rows > 0.2
+    assert cols.shape == (rows, k)
+
+
+def test_bwd_rejects_out_of_range_columns():
+    rows, d, k = 8, 100, 4
+    gx = inputs.mp_gradients(rows, d, 1, device=G.DEV)
+    cols = torch.tensor([[0, 1, 2, 3]] * rows, dtype=torch.int16, device=G.DEV)
+    cols[3, 2] = 100
+    cols[5, 0] = -1
+    gv, r = G.mp_bwd(gx, d, cols)
+    assert r.status == B.DCT_ERR_BAD_MASK
+    want = torch.gather(gx, 1, cols.long().clamp(0, d - 1))
+    want[3, 2] = 0
+    want[5, 0] = 0
+    assert torch.equal(gv, want)
+
+
+def test_mp_host_buffer_entry_point():
+    rows, d, k = 256, 512, 26
+    x = inputs.mp_activations(rows, d, 7, dtype=torch.bfloat16).pin_memory()
+    gx = inputs.mp_gradients(rows, d, 8, dtype=torch.bfloat16).pin_memory()
+    dev = lambda *s, dt=torch.bfloat16: torch.empty(*s, dtype=dt, device=G.DEV)
+    host = lambda *s, dt=torch.bfloat16: torch.empty(*s, dtype=dt).pin_memory()
+    cols_h, vals_h, gv_h = host(rows * k, dt=torch.int16), host(rows * k), host(rows * k)
+    res_h = torch.zeros(5, dtype=torch.int64).pin_memory()
+    B.dct_mp_pack_host(x, gx, dev(rows, d), dev(rows, d), rows, d, d, k, dev(rows * k, dt=torch.int16),
+                       dev(rows * k), dev(rows * k), cols_h, vals_h, gv_h, B.new_result(), res_h)
+    want = oracle.mp_fwd(G.to_oracle(x), k)
+    assert np.array_equal(cols_h.numpy().reshape(rows, k), want.cols)
+    assert np.array_equal(G.as_np_bits(vals_h).reshape(rows, k), want.vals)
+    assert np.array_equal(G.as_np_bits(gv_h).reshape(rows, k), oracle.mp_bwd(G.to_oracle(gx), want.cols))
