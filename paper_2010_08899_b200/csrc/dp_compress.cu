@@ -5,27 +5,50 @@
 //   (idx, val) of survivors       (compressed gradient, ascending index)
 //   residual = w - w .* M         (error)
 //
-// One CTA handles one tile of kTileElems consecutive elements.  Tiles are
-// handed out by an atomic ticket, so a tile's predecessors have always started
-// before it; the global output offset of a tile comes from a decoupled
-// look-back over one 64-bit descriptor per tile (2 status bits + two 31-bit
-// running counts: elements above tau and elements equal to tau).
+// The vector is cut into tiles of kTileElems consecutive elements.  Tiles are
+// handed out by an atomic ticket, so a tile's predecessors have always been
+// taken by a running CTA before it; the global output offset of a tile comes
+// from a decoupled look-back over one 64-bit descriptor per tile (2 status bits
+// + two 31-bit running counts: elements above tau and elements equal to tau).
 //
 // HBM traffic: read grad, read residual, write residual = 12 B per element,
-// plus 8 B per survivor.  The residual is stored before the look-back finishes
-// (assuming every flagged element is sent); the rare elements that turn out not
-// to be sent (capacity exceeded, tie budget used up, wait timed out) are
-// rewritten afterwards by the same thread.
+// plus 8 B per survivor.  The residual of a tile is stored before its look-back
+// finishes, assuming that every flagged element is sent; the rare elements that
+// turn out not to be sent (capacity exceeded, tie budget used up, wait timed
+// out) are rewritten afterwards.
+//
+// Two kernels share the per-tile arithmetic:
+//   * dp_compress_stream_kernel -- the fast path for 16-byte aligned vectors.
+//     Persistent CTAs with three roles.  A load warp takes tickets and streams
+//     tiles into a ring of shared-memory stages with bulk asynchronous copies
+//     (TMA engine, no multicast).  Eight compute warps threshold a stage, store
+//     the new residual with 128-bit stores, publish the tile's counts and push
+//     the tile's survivors, in index order, into a small shared-memory queue.
+//     A scan warp runs the look-back for each tile and then drains that tile's
+//     queue to (idx, val).  Nothing on the compute warps' path waits for another
+//     CTA; a tile with more survivors than a queue slot holds is written by the
+//     compute warps themselves once its prefix is known (dense inputs: slower,
+//     same results).
+//   * dp_compress_tile_kernel -- one CTA per tile with plain loads and stores:
+//     the ragged last tile and vectors that are not 16-byte aligned.
 #include "common.cuh"
 
 namespace dct {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;                           // compute threads per CTA
 constexpr int kWarps = kThreads / 32;
-constexpr int kVecs = 4;                                // 128-bit loads per thread and operand
+constexpr int kVecs = 4;                                // 128-bit vectors per thread and operand
 constexpr uint32_t kWarpElems = 32u * kVecs * 4u;       // 512
 constexpr uint32_t kTileElems = kWarps * kWarpElems;    // 4096
+constexpr uint32_t kTileBytes = kTileElems * 4u;        // 16 KiB per operand
+
+#ifndef DCT_CMP_STAGES
+#define DCT_CMP_STAGES 2
+#endif
+constexpr int kStages = DCT_CMP_STAGES;                 // ring depth of the streaming kernel
+constexpr uint32_t kInvalidTile = 0xFFFFFFFFu;
+constexpr uint32_t kMbarLimit = 1u << 24;               // polls before an mbarrier wait gives up
 
 constexpr uint64_t kStatusAggregate = 1ull << 62;       // descriptor holds the tile's own counts
 constexpr uint64_t kStatusInclusive = 2ull << 62;       // descriptor holds counts of tiles 0..this
@@ -38,10 +61,9 @@ __device__ __forceinline__ uint64_t pack_counts(uint64_t status, uint32_t gt, ui
 __device__ __forceinline__ uint32_t desc_gt(uint64_t d) { return static_cast<uint32_t>((d >> 31) & kCountMask); }
 __device__ __forceinline__ uint32_t desc_eq(uint64_t d) { return static_cast<uint32_t>(d & kCountMask); }
 
-// ctrl[0] = next tile ticket, ctrl[1] = abort flag (a wait gave up somewhere)
 struct CompressCtrl {
-    uint32_t ticket;
-    uint32_t abort;
+    uint32_t ticket;     // next tile to hand out
+    uint32_t abort;      // a bounded wait gave up somewhere: everybody stops waiting
 };
 constexpr size_t kCtrlBytes = 256;
 
@@ -61,185 +83,130 @@ __global__ void dp_compress_init_kernel(CompressCtrl* ctrl, uint64_t* tile_state
     }
 }
 
-// Look-back by one warp: returns the counts of all tiles before `tile`.
-// Every wait is bounded; on expiry *timed_out is set and the result is unusable.
+// Look-back by one warp: counts of all tiles before `tile`.  Each round examines a window of
+// 32 * kLookWide descriptors (all loads of a round are in flight together, so a round costs one
+// L2 round trip): persistent CTAs advance in step, so the nearest descriptor that already holds
+// an inclusive prefix is typically a few hundred tiles back.  Every wait is bounded.
+constexpr int kLookWide = 8;
 __device__ __forceinline__ void lookback(const uint64_t* tile_state, const CompressCtrl* ctrl,
                                          uint32_t tile, uint32_t spin_limit,
                                          uint32_t& excl_gt, uint32_t& excl_eq, bool& timed_out) {
     const uint32_t lane = lane_id();
     uint32_t sum_gt = 0, sum_eq = 0;
-    bool fail = false;
-    int64_t window_end = static_cast<int64_t>(tile);   // tiles [window_end-32, window_end) are examined
+    int64_t window_end = static_cast<int64_t>(tile);   // tiles [window_end - 32 kLookWide, window_end)
+    timed_out = false;
     while (true) {
-        const int64_t t = window_end - 1 - lane;
-        uint64_t d = kStatusInclusive;                   // tiles before the first one: empty prefix
-        if (t >= 0) {
+        uint64_t d[kLookWide];
+#pragma unroll
+        for (int q = 0; q < kLookWide; ++q) {            // distance from the tile: q * 32 + lane + 1
+            const int64_t t = window_end - 1 - (q * 32 + static_cast<int64_t>(lane));
+            d[q] = t >= 0 ? ld_relaxed_u64(tile_state + t) : kStatusInclusive;   // before tile 0: empty prefix
+        }
+        bool done = false;
+#pragma unroll
+        for (int q = 0; q < kLookWide; ++q) {
+            if (done) break;
+            const int64_t t = window_end - 1 - (q * 32 + static_cast<int64_t>(lane));
             uint32_t spins = 0;
-            while (true) {
-                d = ld_relaxed_u64(tile_state + t);
-                if (d & kStatusMask) break;
+            bool fail = false;
+            while ((d[q] & kStatusMask) == 0) {          // not published yet: poll this descriptor
                 if (spins >= spin_limit || ((spins & 31u) == 31u && ld_relaxed_u32(&ctrl->abort))) {
                     fail = true;
                     break;
                 }
                 ++spins;
                 if (spins > 16) __nanosleep(spins > 256 ? 400 : 50);
+                d[q] = ld_relaxed_u64(tile_state + t);
             }
+            if (__any_sync(0xFFFFFFFFu, fail)) {
+                timed_out = true;
+                return;
+            }
+            const uint32_t inclusive = __ballot_sync(0xFFFFFFFFu, (d[q] & kStatusMask) == kStatusInclusive);
+            // lanes 0..first (nearest tiles up to and including the first inclusive one) contribute
+            const uint32_t first = inclusive ? (__ffs(inclusive) - 1) : 31u;
+            const bool use = lane <= first;
+            sum_gt += __reduce_add_sync(0xFFFFFFFFu, use ? desc_gt(d[q]) : 0u);
+            sum_eq += __reduce_add_sync(0xFFFFFFFFu, use ? desc_eq(d[q]) : 0u);
+            if (inclusive) done = true;
         }
-        if (__any_sync(0xFFFFFFFFu, fail)) {
-            timed_out = true;
-            return;
-        }
-        const uint32_t inclusive = __ballot_sync(0xFFFFFFFFu, (d & kStatusMask) == kStatusInclusive);
-        // lanes 0..first (nearest tiles up to and including the first inclusive one) contribute
-        const uint32_t first = inclusive ? (__ffs(inclusive) - 1) : 31u;
-        const bool use = lane <= first;
-        sum_gt += __reduce_add_sync(0xFFFFFFFFu, use ? desc_gt(d) : 0u);
-        sum_eq += __reduce_add_sync(0xFFFFFFFFu, use ? desc_eq(d) : 0u);
-        if (inclusive) break;
-        window_end -= 32;
+        if (done) break;
+        window_end -= 32 * kLookWide;
     }
     excl_gt = sum_gt;
     excl_eq = sum_eq;
-    timed_out = false;
 }
 
-template <bool kVectorised>
-__global__ void __launch_bounds__(kThreads)
-dp_compress_kernel(const float* __restrict__ grad, float* __restrict__ residual, uint32_t n,
-                   const float* __restrict__ tau_p, const uint64_t* __restrict__ budget_p,
-                   int32_t* __restrict__ idx_out, float* __restrict__ val_out, uint64_t capacity,
-                   dct_result_t* __restrict__ result, CompressCtrl* ctrl,
-                   uint64_t* __restrict__ tile_state, uint32_t num_tiles, uint32_t spin_limit) {
-    __shared__ uint32_t s_tile;
-    __shared__ uint32_t s_warp_tot[kWarps];   // (gt << 16) | eq of each warp, each <= 512
-    __shared__ uint32_t s_excl[2];
-    __shared__ uint32_t s_abort;
+// A tile's own counts, visible to every later tile as early as possible.
+__device__ __forceinline__ void publish_tile_aggregate(uint64_t* tile_state, uint32_t tile, uint32_t cta_gt,
+                                                       uint32_t cta_eq) {
+    st_relaxed_u64(tile_state + tile, pack_counts(tile == 0 ? kStatusInclusive : kStatusAggregate, cta_gt, cta_eq));
+}
 
-    if (threadIdx.x == 0) {
-        s_tile = atomicAdd(&ctrl->ticket, 1u);
-        s_abort = 0;
-    }
-    __syncthreads();
-    const uint32_t tile = s_tile;
-    if (tile >= num_tiles) return;            // only reachable with a testing ticket offset
-
+// Publishes the tile's descriptors, runs the look-back and, for the last tile of the vector,
+// writes the result block.  Called by one full warp.  Returns false if the wait gave up.
+__device__ __forceinline__ bool resolve_tile_prefix(uint64_t* tile_state, CompressCtrl* ctrl, dct_result_t* result,
+                                                    uint32_t tile, uint32_t last_tile, uint32_t cta_gt,
+                                                    uint32_t cta_eq, uint64_t budget, uint64_t capacity,
+                                                    uint32_t spin_limit, uint32_t& excl_gt, uint32_t& excl_eq,
+                                                    bool publish_aggregate) {
     const uint32_t lane = lane_id();
-    const uint32_t warp = threadIdx.x >> 5;
-    const uint32_t tile_base = tile * kTileElems;
-    const uint32_t warp_base = tile_base + warp * kWarpElems;
-    const uint32_t tau_key = key_f32(__ldg(tau_p));
-    const uint64_t budget = budget_p ? *budget_p : ~0ull;
-
-    // ---- load, error feedback, flags --------------------------------------------------
-    float w[kVecs * 4];
-    const bool full_tile = kVectorised && (tile_base + kTileElems <= n);
-    if (full_tile) {
-        float4 g4[kVecs], e4[kVecs];
-#pragma unroll
-        for (int j = 0; j < kVecs; ++j) g4[j] = ld_readonly_f4(grad + warp_base + j * 128 + lane * 4);
-#pragma unroll
-        for (int j = 0; j < kVecs; ++j) e4[j] = ld_stream_f4(residual + warp_base + j * 128 + lane * 4);
-#pragma unroll
-        for (int j = 0; j < kVecs; ++j) {
-            w[4 * j + 0] = __fadd_rn(g4[j].x, e4[j].x);
-            w[4 * j + 1] = __fadd_rn(g4[j].y, e4[j].y);
-            w[4 * j + 2] = __fadd_rn(g4[j].z, e4[j].z);
-            w[4 * j + 3] = __fadd_rn(g4[j].w, e4[j].w);
+    if (lane == 0 && publish_aggregate) publish_tile_aggregate(tile_state, tile, cta_gt, cta_eq);
+    bool timed_out = false;
+    excl_gt = 0;
+    excl_eq = 0;
+#ifndef DCT_DBG_NO_LOOKBACK
+    if (tile > 0) lookback(tile_state, ctrl, tile, spin_limit, excl_gt, excl_eq, timed_out);
+#endif
+    if (timed_out) {
+        if (lane == 0) {
+            atomicExch(&ctrl->abort, 1u);
+            atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
         }
-    } else {
-#pragma unroll
-        for (int j = 0; j < kVecs; ++j)
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const uint32_t i = warp_base + j * 128 + lane * 4 + c;
-                w[4 * j + c] = (i < n) ? __fadd_rn(grad[i], residual[i]) : 0.0f;
-            }
+        return false;
     }
+    if (lane == 0) {
+        if (tile > 0)
+            st_relaxed_u64(tile_state + tile, pack_counts(kStatusInclusive, excl_gt + cta_gt, excl_eq + cta_eq));
+        if (tile == last_tile) {
+            const uint64_t total_gt = static_cast<uint64_t>(excl_gt) + cta_gt;
+            const uint64_t total_eq = static_cast<uint64_t>(excl_eq) + cta_eq;
+            const uint64_t needed = total_gt + (total_eq < budget ? total_eq : budget);
+            result->needed = needed;
+            result->count = needed < capacity ? needed : capacity;
+            if (needed > capacity) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_CAPACITY));
+        }
+    }
+    return true;
+}
 
-    uint32_t gt_mask = 0, eq_mask = 0;        // bit 4*j + c
+// Error feedback for 16 elements of one thread: element b = 4 j + c sits at
+// warp_base + j * 128 + lane * 4 + c.  Returns the flag masks (bit b).
+__device__ __forceinline__ void flag_elements(const float (&w)[kVecs * 4], uint32_t tau_key, uint32_t valid_mask,
+                                              uint32_t& gt_mask, uint32_t& eq_mask) {
+    gt_mask = 0;
+    eq_mask = 0;
 #pragma unroll
     for (int b = 0; b < kVecs * 4; ++b) {
-        const uint32_t i = warp_base + (b >> 2) * 128 + lane * 4 + (b & 3);
-        const bool valid = full_tile || (i < n);
         const uint32_t kw = key_f32(w[b]);
-        gt_mask |= (valid && kw > tau_key) ? (1u << b) : 0u;
-        eq_mask |= (valid && kw == tau_key) ? (1u << b) : 0u;
+        gt_mask |= (kw > tau_key) ? (1u << b) : 0u;
+        eq_mask |= (kw == tau_key) ? (1u << b) : 0u;
     }
+    gt_mask &= valid_mask;
+    eq_mask &= valid_mask;
+}
 
-    // ---- tile aggregate, published as early as possible ---------------------------------
-    const uint32_t warp_tot =
-        __reduce_add_sync(0xFFFFFFFFu, (static_cast<uint32_t>(__popc(gt_mask)) << 16) | __popc(eq_mask));
-    if (lane == 0) s_warp_tot[warp] = warp_tot;
-    __syncthreads();
-    uint32_t cta_tot = 0, before_warp = 0;
-#pragma unroll
-    for (int v = 0; v < kWarps; ++v) {
-        const uint32_t t = s_warp_tot[v];
-        cta_tot += t;
-        before_warp += (v < static_cast<int>(warp)) ? t : 0u;
-    }
-    const uint32_t cta_gt = cta_tot >> 16, cta_eq = cta_tot & 0xFFFFu;
-    if (threadIdx.x == 0)
-        st_relaxed_u64(tile_state + tile,
-                       pack_counts(tile == 0 ? kStatusInclusive : kStatusAggregate, cta_gt, cta_eq));
-
-    // ---- residual: +0 where flagged, w elsewhere ----------------------------------------
-    const uint32_t flagged = gt_mask | eq_mask;
-    if (full_tile) {
-#pragma unroll
-        for (int j = 0; j < kVecs; ++j) {
-            float4 e;
-            e.x = (flagged >> (4 * j + 0)) & 1u ? 0.0f : w[4 * j + 0];
-            e.y = (flagged >> (4 * j + 1)) & 1u ? 0.0f : w[4 * j + 1];
-            e.z = (flagged >> (4 * j + 2)) & 1u ? 0.0f : w[4 * j + 2];
-            e.w = (flagged >> (4 * j + 3)) & 1u ? 0.0f : w[4 * j + 3];
-            st_stream_f4(residual + warp_base + j * 128 + lane * 4, e);
-        }
-    } else {
-#pragma unroll
-        for (int b = 0; b < kVecs * 4; ++b) {
-            const uint32_t i = warp_base + (b >> 2) * 128 + lane * 4 + (b & 3);
-            if (i < n) residual[i] = (flagged >> b) & 1u ? 0.0f : w[b];
-        }
-    }
-
-    // ---- look-back for the exclusive prefix (warp 0) --------------------------------------
-    if (warp == 0) {
-        uint32_t excl_gt = 0, excl_eq = 0;
-        bool timed_out = false;
-        if (tile > 0) lookback(tile_state, ctrl, tile, spin_limit, excl_gt, excl_eq, timed_out);
-        if (lane == 0) {
-            if (timed_out) {
-                atomicExch(&ctrl->abort, 1u);
-                atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
-                s_abort = 1;
-            } else {
-                if (tile > 0)
-                    st_relaxed_u64(tile_state + tile,
-                                   pack_counts(kStatusInclusive, excl_gt + cta_gt, excl_eq + cta_eq));
-                s_excl[0] = excl_gt;
-                s_excl[1] = excl_eq;
-                if (tile == num_tiles - 1) {
-                    const uint64_t total_gt = static_cast<uint64_t>(excl_gt) + cta_gt;
-                    const uint64_t total_eq = static_cast<uint64_t>(excl_eq) + cta_eq;
-                    const uint64_t needed = total_gt + (total_eq < budget ? total_eq : budget);
-                    result->needed = needed;
-                    result->count = needed < capacity ? needed : capacity;
-                    if (needed > capacity) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_CAPACITY));
-                }
-            }
-        }
-    }
-    if (cta_tot == 0) return;                  // nothing flagged in this tile: no output, no fix-up
-    __syncthreads();
-    if (warp_tot == 0) return;
-    const bool aborted = s_abort != 0;
-    const uint64_t excl_gt = s_excl[0], excl_eq = s_excl[1];
-
-    // ---- positions of this warp's flagged elements -------------------------------------------
-    // Element order inside a warp's 512-element span is (j, lane, c).  Per-j counts (<= 4 per
-    // lane, <= 128 per warp) are packed one per byte so that one warp scan serves all four j.
+// Visits the flagged elements of one warp's 512-element span in index order:
+//   visit(b, i, local_gt, local_eq, is_eq)
+// with b the register slot, i the element index and local_* the number of flagged elements of
+// each kind that precede it inside the tile (before_warp: packed counts of the lower warps).
+// Must be called by all 32 lanes of the warp.
+template <typename Visit>
+__device__ __forceinline__ void for_each_flagged(uint32_t gt_mask, uint32_t eq_mask, uint32_t warp_base,
+                                                 uint32_t before_warp, Visit&& visit) {
+    const uint32_t lane = lane_id();
+    // Element order inside the span is (j, lane, c).  Per-j counts (<= 4 per lane, <= 128 per
+    // warp) are packed one per byte so that one warp scan serves all four j.
     uint32_t pg = 0, pe = 0;
 #pragma unroll
     for (int j = 0; j < kVecs; ++j) {
@@ -259,34 +226,409 @@ dp_compress_kernel(const float* __restrict__ grad, float* __restrict__ residual,
     const uint32_t tot_g = __shfl_sync(0xFFFFFFFFu, ig, 31), tot_e = __shfl_sync(0xFFFFFFFFu, ie, 31);
     const uint32_t ex_g = ig - pg, ex_e = ie - pe;
     uint32_t base_g = before_warp >> 16, base_e = before_warp & 0xFFFFu;
-    if (flagged) {
+    if ((gt_mask | eq_mask) == 0) return;
+#pragma unroll
+    for (int j = 0; j < kVecs; ++j) {
+        uint32_t g0 = base_g + ((ex_g >> (8 * j)) & 0xFFu);
+        uint32_t e0 = base_e + ((ex_e >> (8 * j)) & 0xFFu);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int b = 4 * j + c;
+            const bool is_gt = (gt_mask >> b) & 1u, is_eq = (eq_mask >> b) & 1u;
+            if (is_gt || is_eq) {
+                visit(b, warp_base + j * 128 + lane * 4 + c, g0, e0, is_eq);
+                g0 += is_gt;
+                e0 += is_eq;
+            }
+        }
+        base_g += (tot_g >> (8 * j)) & 0xFFu;
+        base_e += (tot_e >> (8 * j)) & 0xFFu;
+    }
+}
+
+// One flagged element whose global counts of preceding flagged elements are known: it is either
+// written to the output or, if it is not sent after all, put back into the residual.
+__device__ __forceinline__ void place_survivor(uint32_t i, float w, bool is_eq, uint64_t gt_before,
+                                               uint64_t eq_before, uint64_t budget, uint64_t capacity, bool aborted,
+                                               int32_t* __restrict__ idx_out, float* __restrict__ val_out,
+                                               float* __restrict__ residual) {
+    const bool pass = !is_eq || eq_before < budget;
+    const uint64_t pos = gt_before + (eq_before < budget ? eq_before : budget);
+    if (pass && pos < capacity && !aborted) {
+        idx_out[pos] = static_cast<int32_t>(i);
+        val_out[pos] = w;
+    } else {
+        residual[i] = w;
+    }
+}
+
+// Writes the survivors of one warp's span straight from registers.
+__device__ __forceinline__ void emit_warp(const float (&w)[kVecs * 4], uint32_t gt_mask, uint32_t eq_mask,
+                                          uint32_t warp_base, uint32_t before_warp, uint64_t excl_gt,
+                                          uint64_t excl_eq, uint64_t budget, uint64_t capacity, bool aborted,
+                                          int32_t* __restrict__ idx_out, float* __restrict__ val_out,
+                                          float* __restrict__ residual) {
+    for_each_flagged(gt_mask, eq_mask, warp_base, before_warp,
+                     [&](int b, uint32_t i, uint32_t local_gt, uint32_t local_eq, bool is_eq) {
+                         place_survivor(i, w[b], is_eq, excl_gt + local_gt, excl_eq + local_eq, budget, capacity,
+                                        aborted, idx_out, val_out, residual);
+                     });
+}
+
+// ------------------------------------------------------------------------------------------
+// generic path: one CTA per tile, plain loads/stores, any alignment, ragged tail
+// ------------------------------------------------------------------------------------------
+#ifndef DCT_CMP_MIN_BLOCKS
+#define DCT_CMP_MIN_BLOCKS 4
+#endif
+template <bool kVectorised>
+__global__ void __launch_bounds__(kThreads, DCT_CMP_MIN_BLOCKS)
+dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ residual, uint32_t n,
+                        const float* __restrict__ tau_p, const uint64_t* __restrict__ budget_p,
+                        int32_t* __restrict__ idx_out, float* __restrict__ val_out, uint64_t capacity,
+                        dct_result_t* __restrict__ result, CompressCtrl* ctrl,
+                        uint64_t* __restrict__ tile_state, uint32_t num_tiles, uint32_t fixed_tile,
+                        uint32_t spin_limit) {
+    __shared__ uint32_t s_tile;
+    __shared__ uint32_t s_warp_tot[kWarps];   // (gt << 16) | eq of each warp, each <= 512
+    __shared__ uint32_t s_excl[2];
+    __shared__ uint32_t s_abort;
+
+    if (threadIdx.x == 0) {
+        s_tile = fixed_tile != kInvalidTile ? fixed_tile : atomicAdd(&ctrl->ticket, 1u);
+        s_abort = 0;
+    }
+    __syncthreads();
+    const uint32_t tile = s_tile;
+    if (tile >= num_tiles) return;            // only reachable with a testing ticket offset
+
+    const uint32_t lane = lane_id();
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint32_t tile_base = tile * kTileElems;
+    const uint32_t warp_base = tile_base + warp * kWarpElems;
+    const uint32_t tau_key = key_f32(__ldg(tau_p));
+    const uint64_t budget = budget_p ? *budget_p : ~0ull;
+
+    float w[kVecs * 4];
+    uint32_t valid_mask = 0xFFFFu;
+    const bool full_tile = kVectorised && (tile_base + kTileElems <= n);
+    if (full_tile) {
+        float4 g4[kVecs], e4[kVecs];
+#pragma unroll
+        for (int j = 0; j < kVecs; ++j) g4[j] = ld_readonly_f4(grad + warp_base + j * 128 + lane * 4);
+#pragma unroll
+        for (int j = 0; j < kVecs; ++j) e4[j] = ld_stream_f4(residual + warp_base + j * 128 + lane * 4);
 #pragma unroll
         for (int j = 0; j < kVecs; ++j) {
-            uint32_t g0 = base_g + ((ex_g >> (8 * j)) & 0xFFu);
-            uint32_t e0 = base_e + ((ex_e >> (8 * j)) & 0xFFu);
+            w[4 * j + 0] = __fadd_rn(g4[j].x, e4[j].x);
+            w[4 * j + 1] = __fadd_rn(g4[j].y, e4[j].y);
+            w[4 * j + 2] = __fadd_rn(g4[j].z, e4[j].z);
+            w[4 * j + 3] = __fadd_rn(g4[j].w, e4[j].w);
+        }
+    } else {
+        valid_mask = 0;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                const int b = 4 * j + c;
-                const bool is_gt = (gt_mask >> b) & 1u, is_eq = (eq_mask >> b) & 1u;
-                if (is_gt || is_eq) {
-                    const uint64_t gt_before = excl_gt + g0;
-                    const uint64_t eq_before = excl_eq + e0;
-                    const bool pass = is_gt || eq_before < budget;
-                    const uint64_t pos = gt_before + (eq_before < budget ? eq_before : budget);
-                    const uint32_t i = warp_base + j * 128 + lane * 4 + c;
-                    if (pass && pos < capacity && !aborted) {
-                        idx_out[pos] = static_cast<int32_t>(i);
-                        val_out[pos] = w[b];
-                    } else {
-                        residual[i] = w[b];    // not sent after all: it stays in the error
+        for (int b = 0; b < kVecs * 4; ++b) {
+            const uint32_t i = warp_base + (b >> 2) * 128 + lane * 4 + (b & 3);
+            const bool valid = i < n;
+            w[b] = valid ? __fadd_rn(grad[i], residual[i]) : 0.0f;
+            valid_mask |= valid ? (1u << b) : 0u;
+        }
+    }
+    uint32_t gt_mask, eq_mask;
+    flag_elements(w, tau_key, valid_mask, gt_mask, eq_mask);
+
+    const uint32_t warp_tot =
+        __reduce_add_sync(0xFFFFFFFFu, (static_cast<uint32_t>(__popc(gt_mask)) << 16) | __popc(eq_mask));
+    if (lane == 0) s_warp_tot[warp] = warp_tot;
+    __syncthreads();
+    uint32_t cta_tot = 0, before_warp = 0;
+#pragma unroll
+    for (int v = 0; v < kWarps; ++v) {
+        const uint32_t t = s_warp_tot[v];
+        cta_tot += t;
+        before_warp += (v < static_cast<int>(warp)) ? t : 0u;
+    }
+    const uint32_t cta_gt = cta_tot >> 16, cta_eq = cta_tot & 0xFFFFu;
+
+    // residual: +0 where flagged, w elsewhere (flagged elements are rewritten later if not sent)
+    const uint32_t flagged = gt_mask | eq_mask;
+    if (full_tile) {
+#pragma unroll
+        for (int j = 0; j < kVecs; ++j) {
+            float4 e;
+            e.x = (flagged >> (4 * j + 0)) & 1u ? 0.0f : w[4 * j + 0];
+            e.y = (flagged >> (4 * j + 1)) & 1u ? 0.0f : w[4 * j + 1];
+            e.z = (flagged >> (4 * j + 2)) & 1u ? 0.0f : w[4 * j + 2];
+            e.w = (flagged >> (4 * j + 3)) & 1u ? 0.0f : w[4 * j + 3];
+            st_stream_f4(residual + warp_base + j * 128 + lane * 4, e);
+        }
+    } else {
+#pragma unroll
+        for (int b = 0; b < kVecs * 4; ++b) {
+            const uint32_t i = warp_base + (b >> 2) * 128 + lane * 4 + (b & 3);
+            if ((valid_mask >> b) & 1u) residual[i] = (flagged >> b) & 1u ? 0.0f : w[b];
+        }
+    }
+
+    if (warp == 0) {
+        uint32_t excl_gt, excl_eq;
+        const bool ok = resolve_tile_prefix(tile_state, ctrl, result, tile, num_tiles - 1, cta_gt, cta_eq, budget,
+                                            capacity, spin_limit, excl_gt, excl_eq, true);
+        if (lane == 0) {
+            s_abort = ok ? 0u : 1u;
+            s_excl[0] = excl_gt;
+            s_excl[1] = excl_eq;
+        }
+    }
+    if (cta_tot == 0) return;                  // nothing flagged in this tile: no output, no rewrite
+    __syncthreads();
+    if (warp_tot == 0) return;
+    emit_warp(w, gt_mask, eq_mask, warp_base, before_warp, s_excl[0], s_excl[1], budget, capacity, s_abort != 0,
+              idx_out, val_out, residual);
+}
+
+// ------------------------------------------------------------------------------------------
+// fast path: persistent CTAs; load warp + compute warps + scan warp
+// ------------------------------------------------------------------------------------------
+#ifndef DCT_CMP_QUEUE_SLOTS
+#define DCT_CMP_QUEUE_SLOTS 8
+#endif
+#ifndef DCT_CMP_QUEUE_ENTRIES
+#define DCT_CMP_QUEUE_ENTRIES 512
+#endif
+constexpr int kSlots = DCT_CMP_QUEUE_SLOTS;              // tiles a CTA may be ahead of its scan warp
+constexpr uint32_t kQueueEntries = DCT_CMP_QUEUE_ENTRIES;  // survivors of one tile that fit a slot
+constexpr uint32_t kEqBit = 0x80000000u;                 // queue entry: index (31 bits) | "equal to tau"
+constexpr int kLoadWarp = kWarps, kScanWarp = kWarps + 1;
+constexpr int kStreamThreads = kThreads + 64;
+
+struct __align__(128) StreamSmem {
+    float g[kStages][kTileElems];
+    float e[kStages][kTileElems];
+    uint2 queue[kSlots][kQueueEntries];  // (index | kEqBit, value bits) in index order
+    uint64_t full[kStages];              // load -> compute: stage holds a tile (bulk loads landed)
+    uint64_t empty[kStages];             // compute -> load: stage may be refilled
+    uint64_t agg_ready[kSlots];          // compute (8 warps) -> scan: counts and queue of the slot are written
+    uint64_t prefix_ready[kSlots];       // scan -> compute: exclusive prefix of the slot's tile is in prefix[]
+    uint64_t slot_free[kSlots];          // scan -> compute: the slot may be reused
+    uint32_t tile[kStages];
+    uint32_t warp_tot[2][kWarps];
+    uint32_t slot_tile[kSlots];
+    uint32_t slot_agg[kSlots];           // (gt << 16) | eq of the tile
+    uint32_t slot_direct[kSlots];        // 1: the compute warps write this tile's output themselves
+    uint32_t prefix[kSlots][2];
+    uint32_t aborted[kSlots];
+    volatile uint32_t stop;              // a bounded wait gave up inside this CTA
+};
+
+__global__ void __launch_bounds__(kStreamThreads, 2)
+dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ residual, uint32_t num_full_tiles,
+                          uint32_t last_tile, const float* __restrict__ tau_p,
+                          const uint64_t* __restrict__ budget_p, int32_t* __restrict__ idx_out,
+                          float* __restrict__ val_out, uint64_t capacity, dct_result_t* __restrict__ result,
+                          CompressCtrl* ctrl, uint64_t* __restrict__ tile_state, uint32_t spin_limit) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
+    const uint32_t tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
+
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(&sm.full[s], 1);
+            mbar_init(&sm.empty[s], 1);
+        }
+        for (int r = 0; r < kSlots; ++r) {
+            mbar_init(&sm.agg_ready[r], kWarps);
+            mbar_init(&sm.prefix_ready[r], 1);
+            mbar_init(&sm.slot_free[r], 1);
+        }
+        sm.stop = 0;
+        mbar_init_fence();
+        fence_proxy_async_all();
+    }
+    __syncthreads();
+    const uint64_t budget = budget_p ? *budget_p : ~0ull;
+
+    if (warp == kLoadWarp) {
+        // ================= load warp (one lane): tickets and bulk loads ====================
+        if (lane != 0) return;
+        uint32_t ticket = atomicAdd(&ctrl->ticket, 1u);
+        for (uint32_t it = 0;; ++it) {
+            const int s = it % kStages;
+            const uint32_t tile = ticket < num_full_tiles ? ticket : kInvalidTile;
+            // the next ticket is requested now; its latency overlaps the wait below
+            if (tile != kInvalidTile) ticket = atomicAdd(&ctrl->ticket, 1u);
+            if (it >= static_cast<uint32_t>(kStages) &&
+                !mbar_wait_bounded(&sm.empty[s], ((it / kStages) - 1u) & 1u, kMbarLimit, &sm.stop)) {
+                sm.stop = 1;
+                return;
+            }
+            sm.tile[s] = tile;
+            if (tile == kInvalidTile) {
+                mbar_arrive(&sm.full[s]);
+                return;
+            }
+            mbar_arrive_expect_tx(&sm.full[s], 2u * kTileBytes);
+            bulk_load(sm.g[s], grad + static_cast<size_t>(tile) * kTileElems, kTileBytes, &sm.full[s]);
+            bulk_load(sm.e[s], residual + static_cast<size_t>(tile) * kTileElems, kTileBytes, &sm.full[s]);
+        }
+    }
+
+    if (warp == kScanWarp) {
+        // ================= scan warp: look-back, then drain the tile's queue ==================
+        for (uint32_t it = 0;; ++it) {
+            const int r = it % kSlots;
+            const uint32_t parity = (it / kSlots) & 1u;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&sm.agg_ready[r], parity, kMbarLimit, &sm.stop))) {
+                sm.stop = 1;
+                return;
+            }
+            const uint32_t tile = sm.slot_tile[r];
+            if (tile == kInvalidTile) return;
+            const uint32_t tot = sm.slot_agg[r];
+            const uint32_t cta_gt = tot >> 16, cta_eq = tot & 0xFFFFu;
+            uint32_t excl_gt, excl_eq;
+            const bool ok = resolve_tile_prefix(tile_state, ctrl, result, tile, last_tile, cta_gt, cta_eq, budget,
+                                                capacity, spin_limit, excl_gt, excl_eq, false);
+            if (sm.slot_direct[r]) {
+                if (lane == 0) {
+                    sm.prefix[r][0] = excl_gt;
+                    sm.prefix[r][1] = excl_eq;
+                    sm.aborted[r] = ok ? 0u : 1u;
+                }
+            } else {
+                // entries are in index order; eq entries are counted on the fly
+                const uint32_t cnt = cta_gt + cta_eq;
+                uint32_t eq_run = 0;
+                for (uint32_t base = 0; base < cnt; base += 32) {
+                    const uint32_t q = base + lane;
+                    const uint2 ent = q < cnt ? sm.queue[r][q] : make_uint2(0u, 0u);
+                    const bool is_eq = q < cnt && (ent.x & kEqBit);
+                    const uint32_t eq_bal = __ballot_sync(0xFFFFFFFFu, is_eq);
+                    if (q < cnt) {
+                        const uint32_t local_eq = eq_run + __popc(eq_bal & lanemask_lt());
+                        const uint32_t local_gt = q - local_eq;
+                        place_survivor(ent.x & ~kEqBit, __uint_as_float(ent.y), is_eq, uint64_t(excl_gt) + local_gt,
+                                       uint64_t(excl_eq) + local_eq, budget, capacity, !ok, idx_out, val_out,
+                                       residual);
                     }
-                    g0 += is_gt;
-                    e0 += is_eq;
+                    eq_run += __popc(eq_bal);
                 }
             }
-            base_g += (tot_g >> (8 * j)) & 0xFFu;
-            base_e += (tot_e >> (8 * j)) & 0xFFu;
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&sm.prefix_ready[r]);
+                mbar_arrive(&sm.slot_free[r]);
+            }
         }
+    }
+
+    // ===================== compute warps =================================================
+    const uint32_t tau_key = key_f32(__ldg(tau_p));
+    bool healthy = true;
+    uint32_t it = 0;
+    for (;; ++it) {
+        const int s = it % kStages;
+        const int r = it % kSlots;
+        const uint32_t slot_use = it / kSlots;
+        if (!named_barrier_all(1, kThreads,
+                               mbar_wait_bounded(&sm.full[s], (it / kStages) & 1u, kMbarLimit, &sm.stop) &&
+                                   !sm.stop)) {
+            healthy = false;
+            break;
+        }
+        const uint32_t tile = sm.tile[s];
+        if (tile == kInvalidTile) break;
+        const uint32_t warp_base = tile * kTileElems + warp * kWarpElems;
+
+        float w[kVecs * 4];
+        {
+            const float4* gs = reinterpret_cast<const float4*>(sm.g[s]) + warp * (kWarpElems / 4) + lane;
+            const float4* es = reinterpret_cast<const float4*>(sm.e[s]) + warp * (kWarpElems / 4) + lane;
+#pragma unroll
+            for (int j = 0; j < kVecs; ++j) {
+                const float4 g4 = gs[j * 32], e4 = es[j * 32];
+                w[4 * j + 0] = __fadd_rn(g4.x, e4.x);
+                w[4 * j + 1] = __fadd_rn(g4.y, e4.y);
+                w[4 * j + 2] = __fadd_rn(g4.z, e4.z);
+                w[4 * j + 3] = __fadd_rn(g4.w, e4.w);
+            }
+        }
+        uint32_t gt_mask, eq_mask;
+        flag_elements(w, tau_key, 0xFFFFu, gt_mask, eq_mask);
+        const uint32_t flagged = gt_mask | eq_mask;
+#pragma unroll
+        for (int j = 0; j < kVecs; ++j) {
+            float4 e;
+            e.x = (flagged >> (4 * j + 0)) & 1u ? 0.0f : w[4 * j + 0];
+            e.y = (flagged >> (4 * j + 1)) & 1u ? 0.0f : w[4 * j + 1];
+            e.z = (flagged >> (4 * j + 2)) & 1u ? 0.0f : w[4 * j + 2];
+            e.w = (flagged >> (4 * j + 3)) & 1u ? 0.0f : w[4 * j + 3];
+            st_stream_f4(residual + warp_base + j * 128 + lane * 4, e);
+        }
+        const uint32_t warp_tot =
+            __reduce_add_sync(0xFFFFFFFFu, (static_cast<uint32_t>(__popc(gt_mask)) << 16) | __popc(eq_mask));
+        if (lane == 0) sm.warp_tot[it & 1u][warp] = warp_tot;
+        named_barrier_sync(1, kThreads);          // every warp has read the stage and posted its counts
+        uint32_t cta_tot = 0, before_warp = 0;
+#pragma unroll
+        for (int v = 0; v < kWarps; ++v) {
+            const uint32_t t = sm.warp_tot[it & 1u][v];
+            cta_tot += t;
+            before_warp += (v < static_cast<int>(warp)) ? t : 0u;
+        }
+        const uint32_t cta_gt = cta_tot >> 16, cta_eq = cta_tot & 0xFFFFu;
+        const bool direct = cta_gt + cta_eq > kQueueEntries;
+        if (tid == 0) {
+            mbar_arrive(&sm.empty[s]);
+            // later tiles may need these counts right now; the scan warp adds the prefix when it gets here
+            publish_tile_aggregate(tile_state, tile, cta_gt, cta_eq);
+        }
+        // the slot must have been drained by the scan warp (it normally was, long ago)
+        bool slot_ok = true;
+        if (slot_use > 0)
+            slot_ok = mbar_wait_bounded(&sm.slot_free[r], (slot_use - 1u) & 1u, kMbarLimit, &sm.stop);
+        if (!__all_sync(0xFFFFFFFFu, slot_ok)) sm.stop = 1;   // seen by everybody at the next vote
+        if (tid == 0) {
+            sm.slot_tile[r] = tile;
+            sm.slot_agg[r] = cta_tot;
+            sm.slot_direct[r] = direct ? 1u : 0u;
+        }
+        if (!direct && warp_tot != 0 && slot_ok) {
+            uint2* q = sm.queue[r];
+            for_each_flagged(gt_mask, eq_mask, warp_base, before_warp,
+                             [&](int b, uint32_t i, uint32_t local_gt, uint32_t local_eq, bool is_eq) {
+                                 q[local_gt + local_eq] = make_uint2(i | (is_eq ? kEqBit : 0u), __float_as_uint(w[b]));
+                             });
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.agg_ready[r]);
+        if (direct) {
+            // dense tile: wait for its prefix and write the output straight from registers
+            if (!named_barrier_all(1, kThreads,
+                                   mbar_wait_bounded(&sm.prefix_ready[r], slot_use & 1u, kMbarLimit, &sm.stop))) {
+                healthy = false;
+                break;
+            }
+            if (warp_tot != 0)
+                emit_warp(w, gt_mask, eq_mask, warp_base, before_warp, sm.prefix[r][0], sm.prefix[r][1], budget,
+                          capacity, sm.aborted[r] != 0, idx_out, val_out, residual);
+        }
+    }
+    if (healthy) {
+        // tell the scan warp that no more tiles follow
+        const int r = it % kSlots;
+        const uint32_t slot_use = it / kSlots;
+        bool slot_ok = true;
+        if (slot_use > 0)
+            slot_ok = mbar_wait_bounded(&sm.slot_free[r], (slot_use - 1u) & 1u, kMbarLimit, &sm.stop);
+        if (tid == 0) sm.slot_tile[r] = kInvalidTile;
+        __syncwarp();
+        if (lane == 0 && slot_ok) mbar_arrive(&sm.agg_ready[r]);
+    } else if (tid == 0) {
+        sm.stop = 1;
+        atomicExch(&ctrl->abort, 1u);
+        atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
     }
 }
 
@@ -326,21 +668,46 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     auto* ctrl = static_cast<CompressCtrl*>(workspace);
     auto* tile_state = reinterpret_cast<uint64_t*>(static_cast<char*>(workspace) + kCtrlBytes);
+    const uint32_t n32 = static_cast<uint32_t>(n);
     const uint32_t num_tiles = dp_compress_num_tiles(n);
+    const uint32_t num_full = n32 / kTileElems;
     const DebugConfig& dbg = debug_config();
 
     dp_compress_init_kernel<<<(num_tiles + 1023) / 1024, 1024, 0, stream>>>(ctrl, tile_state, num_tiles, result,
                                                                             dbg.first_ticket);
     DCT_CUDA_TRY(cudaGetLastError());
     const bool vec = aligned_to(grad, 16) && aligned_to(residual, 16);
-    if (vec)
-        dp_compress_kernel<true><<<num_tiles, kThreads, 0, stream>>>(
-            grad, residual, static_cast<uint32_t>(n), tau, tie_budget, idx_out, val_out, capacity, result, ctrl,
-            tile_state, num_tiles, dbg.spin_limit);
-    else
-        dp_compress_kernel<false><<<num_tiles, kThreads, 0, stream>>>(
-            grad, residual, static_cast<uint32_t>(n), tau, tie_budget, idx_out, val_out, capacity, result, ctrl,
-            tile_state, num_tiles, dbg.spin_limit);
-    DCT_CUDA_TRY(cudaGetLastError());
+    if (!vec) {
+        dp_compress_tile_kernel<false><<<num_tiles, kThreads, 0, stream>>>(
+            grad, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
+            kInvalidTile, dbg.spin_limit);
+        DCT_CUDA_TRY(cudaGetLastError());
+        return DCT_OK;
+    }
+    if (num_full > 0) {
+        static thread_local int configured_device = -1;
+        int dev = 0;
+        DCT_CUDA_TRY(cudaGetDevice(&dev));
+        if (configured_device != dev) {
+            DCT_CUDA_TRY(cudaFuncSetAttribute(dp_compress_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              static_cast<int>(sizeof(StreamSmem))));
+            configured_device = dev;
+        }
+        const int sms = sm_count();
+        if (sms <= 0) return DCT_ERR_CUDA;
+        const uint32_t ctas_per_sm = sizeof(StreamSmem) <= 110 * 1024 ? 2 : 1;
+        const uint32_t max_grid = static_cast<uint32_t>(sms) * ctas_per_sm;
+        const uint32_t grid = num_full < max_grid ? num_full : max_grid;
+        dp_compress_stream_kernel<<<grid, kStreamThreads, sizeof(StreamSmem), stream>>>(
+            grad, residual, num_full, num_tiles - 1, tau, tie_budget, idx_out, val_out, capacity, result, ctrl,
+            tile_state, dbg.spin_limit);
+        DCT_CUDA_TRY(cudaGetLastError());
+    }
+    if (num_tiles > num_full) {   // ragged last tile
+        dp_compress_tile_kernel<true><<<1, kThreads, 0, stream>>>(
+            grad, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
+            num_full, dbg.spin_limit);
+        DCT_CUDA_TRY(cudaGetLastError());
+    }
     return DCT_OK;
 }

@@ -1,0 +1,97 @@
+"""Run one entry point of the library a few times on seeded synthetic data.
+
+A small command-line driver for profiling and quick timing of a single kernel at a chosen size:
+
+    python -m paper_2010_08899_b200.run_case compress --n 268435456 --iters 3
+    python -m paper_2010_08899_b200.run_case select   --n 268435456 --k 26844
+    python -m paper_2010_08899_b200.run_case mp_fwd   --rows 16384 --d 4096 --k 205 --dtype bf16
+    python -m paper_2010_08899_b200.run_case mp_bwd   --rows 16384 --d 4096 --k 205 --dtype bf16
+
+It prints the mean device time per call (CUDA events) and the algorithmic GB/s.
+"""
+from __future__ import annotations
+
+import argparse
+
+import torch
+
+from . import binding as B
+from . import inputs
+
+
+def main():
+    ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
+    ap.add_argument("entry", choices=["select", "compress", "mp_fwd", "mp_bwd"])
+    ap.add_argument("--n", type=int, default=1 << 28)
+    ap.add_argument("--k", type=int, default=0, help="survivor target (default: 0.01 %% of n, or 5 %% of d)")
+    ap.add_argument("--rows", type=int, default=16384)
+    ap.add_argument("--d", type=int, default=4096)
+    ap.add_argument("--dtype", choices=["f32", "bf16"], default="bf16")
+    ap.add_argument("--dist", choices=["mixture", "gaussian", "dlrm"], default="mixture")
+    ap.add_argument("--iters", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=1)
+    args = ap.parse_args()
+
+    dev = "cuda"
+    stream = torch.cuda.current_stream()
+    reset = lambda: None
+    gen = {"mixture": inputs.dp_mixture, "gaussian": inputs.dp_gaussian, "dlrm": inputs.dp_dlrm_like}[args.dist]
+
+    if args.entry in ("select", "compress"):
+        n = args.n
+        k = args.k or B.k_from_density(n, 1, 10_000)
+        g = [gen(n, 501 + j, dev) for j in range(2)]
+        tau = torch.zeros(1, device=dev)
+        res = B.new_result(dev)
+        ws_s = B.new_workspace(B.dct_threshold_select_workspace_bytes(n), dev)
+        B.dct_threshold_select(g[0], None, n, k, tau, res, ws_s)
+        if args.entry == "select":
+            call = lambda i: B.dct_threshold_select(g[i % 2], None, n, k, tau, res, ws_s)
+            nbytes = 4 * n
+        else:
+            e = torch.zeros(n, device=dev)
+            cap = max(n // 64, 1024)
+            idx = torch.empty(cap, dtype=torch.int32, device=dev)
+            val = torch.empty(cap, device=dev)
+            ws_c = B.new_workspace(B.dct_dp_compress_workspace_bytes(n), dev)
+            call = lambda i: B.dct_dp_compress(g[i % 2], e, n, tau, None, idx, val, cap, res, ws_c)
+            reset = e.zero_          # every timed call starts from a zero residual (same survivor density)
+            nbytes = 12 * n
+    else:
+        rows, d = args.rows, args.d
+        k = args.k or B.k_from_sparsity(d, 95, 100)
+        dt = torch.float32 if args.dtype == "f32" else torch.bfloat16
+        es = 4 if args.dtype == "f32" else 2
+        x = [inputs.mp_activations(rows, d, 410 + j, dtype=dt, device=dev, col_scale_seed=400) for j in range(2)]
+        cols = torch.empty(rows * k, dtype=torch.int16, device=dev)
+        vals = torch.empty(rows * k, dtype=dt, device=dev)
+        B.dct_mp_topk_pack_fwd(x[0], rows, d, d, k, cols, vals)
+        if args.entry == "mp_fwd":
+            call = lambda i: B.dct_mp_topk_pack_fwd(x[i % 2], rows, d, d, k, cols, vals)
+            nbytes = rows * d * es + rows * k * (2 + es)
+        else:
+            gx = [inputs.mp_gradients(rows, d, 420 + j, dtype=dt, device=dev) for j in range(2)]
+            gv = torch.empty(rows * k, dtype=dt, device=dev)
+            call = lambda i: B.dct_mp_pack_bwd(gx[i % 2], rows, d, d, k, cols, gv)
+            nbytes = rows * k * (2 + es) + rows * k * es
+
+    for i in range(args.warmup):
+        reset()
+        call(i)
+    torch.cuda.synchronize()
+    pairs = []
+    for i in range(args.iters):
+        reset()
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        call(i)
+        b.record(stream)
+        pairs.append((a, b))
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in pairs) / args.iters
+    print(f"{args.entry}: {ms:.4f} ms per call, {nbytes / ms / 1e6:.1f} GB/s algorithmic ({nbytes} B per call)")
+
+
+if __name__ == "__main__":
+    main()
