@@ -38,7 +38,7 @@ __global__ void mp_topk_pack_fwd_kernel(const T* __restrict__ x, uint32_t rows, 
                                         int32_t* __restrict__ rows_out, T* __restrict__ tau_out,
                                         dct_result_t* __restrict__ result, bool rows_aligned16) {
     using Tr = ElemTraits<T>;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     T* row_s = reinterpret_cast<T*>(smem_raw);
     __shared__ uint32_t s_hist[256];
     __shared__ uint32_t s_prefix, s_krem;
@@ -204,6 +204,368 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
     if (bad && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
 }
 
+// ------------------------------------------------------------------------------------------
+// bf16 fast path: one warp per row, d = 256 * E8 <= 4096, rows on 16-byte boundaries
+// ------------------------------------------------------------------------------------------
+// Lane l owns the E = d/32 consecutive columns [l E, (l+1) E): every "how many before me" question
+// is then one warp scan.  The row is brought in by 32 bulk asynchronous copies (one span per lane,
+// spans padded by 16 bytes in shared memory so that 128-bit reads of different lanes fall into
+// different banks); the next row is requested as soon as the current one has been filtered.
+//   A  lower bound `low` for tau_i: the k-th largest of the maxima of the d/8 aligned 8-element
+//      leaves.  At least k elements are >= low, and fewer than k leaves hold anything above it.
+//   B  candidates (key >= low; typically ~1.2 k of them) are compacted, in column order, into a list.
+//   C  exact k-th largest of the candidates: radix select, exponent byte then mantissa.
+//   D  the kept columns (key > tau_i, then the lowest-column ties) leave the list in order.
+// If the candidates do not fit the list, at least cap - 8 (k - 1) elements tie at `low`: the list is
+// rebuilt from the elements strictly above `low` (always < 8 k of them); if fewer than k of those
+// exist, tau_i = low and the output is written straight from the row.
+#ifndef DCT_FWD_MAX_WARPS
+#define DCT_FWD_MAX_WARPS 16
+#endif
+constexpr int kFwdMaxWarps = DCT_FWD_MAX_WARPS;   // rows in flight per CTA (one CTA per SM; shared memory bounds it)
+constexpr uint32_t kAbsMask2 = 0x7FFF7FFFu;
+constexpr uint32_t kHistWords = 4u * 256u;  // 4 lane-interleaved copies of 256 bins
+
+template <int E8> struct WarpRowLayout {
+    static constexpr uint32_t E = E8 * 8u, D = E * 32u;
+    static constexpr uint32_t kSpanBytes = E * 2u + 16u;
+    static constexpr uint32_t kRowBytes = 32u * kSpanBytes;
+    // list capacity: every element above `low` always fits (< 8 k); rounded up, at most d
+    __host__ __device__ static constexpr uint32_t list_cap(uint32_t k) {
+        return (8u * k + 64u) < D ? ((8u * k + 64u) & ~31u) : D;
+    }
+    __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) {
+        return kRowBytes + list_cap(k) * 4u + kHistWords * 4u + 16u;
+    }
+};
+
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) { return *reinterpret_cast<__nv_bfloat162*>(&u); }
+__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
+
+// bit j set iff |element j| >= low, for the 8 bf16 of one int4.  Floating-point compare: exact for
+// normal numbers; may also admit a few denormals/zeros if the hardware flushes (a superset is fine
+// for a candidate filter); NaN always passes.
+__device__ __forceinline__ uint32_t mask8_ge_filter(uint4 v, __nv_bfloat162 low2) {
+    const uint32_t r0 = __hgeu2_mask(__habs2(as_bf162(v.x)), low2);
+    const uint32_t r1 = __hgeu2_mask(__habs2(as_bf162(v.y)), low2);
+    const uint32_t r2 = __hgeu2_mask(__habs2(as_bf162(v.z)), low2);
+    const uint32_t r3 = __hgeu2_mask(__habs2(as_bf162(v.w)), low2);
+    const uint32_t m = (r0 & 0x00020001u) | (r1 & 0x00080004u) | (r2 & 0x00200010u) | (r3 & 0x00800040u);
+    return (m | (m >> 16)) & 0xFFu;
+}
+// the same on the integer keys, exact for every bit pattern (low <= 0x8000)
+__device__ __forceinline__ uint32_t mask8_ge_exact(uint4 v, uint32_t low) {
+    const uint32_t low2 = low | (low << 16);
+    // per 16-bit half: bit 15 of ((key | 0x8000) - low) is set iff key >= low (no borrow crosses halves)
+    const uint32_t t0 = (((v.x & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
+    const uint32_t t1 = (((v.y & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
+    const uint32_t t2 = (((v.z & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
+    const uint32_t t3 = (((v.w & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
+    uint32_t m = (t0 >> 15) | (t1 >> 13) | (t2 >> 11) | (t3 >> 9);   // halves at bits {0,16},{2,18},{4,20},{6,22}
+    return (m | (m >> 15)) & 0xFFu;
+}
+
+__device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v) {
+    const uint32_t lane = lane_id();
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, v, o);
+        if (lane >= static_cast<uint32_t>(o)) v += t;
+    }
+    return v;
+}
+
+// hist holds 4 interleaved copies of 256 exponent bins.  Returns the exponent that holds rank k_rem
+// (counting from exponent `top_exp` downwards) and reduces k_rem to the rank inside that exponent.
+__device__ __forceinline__ uint32_t pick_exponent(const uint32_t* hist, uint32_t top_exp, uint32_t& k_rem) {
+    const uint32_t lane = lane_id();
+    for (int top = static_cast<int>(top_exp); top >= 0; top -= 32) {   // 32 exponents per step, highest first
+        const int eb = top - static_cast<int>(lane);
+        uint32_t c = 0;
+        if (eb >= 0) {
+            const uint4 h = reinterpret_cast<const uint4*>(hist)[eb];
+            c = h.x + h.y + h.z + h.w;
+        }
+        const uint32_t inc = warp_inclusive_sum(c);
+        const uint32_t hit = __ballot_sync(0xFFFFFFFFu, inc >= k_rem);
+        if (hit) {
+            const int src = __ffs(hit) - 1;
+            k_rem -= __shfl_sync(0xFFFFFFFFu, inc - c, src);
+            return static_cast<uint32_t>(top - src);
+        }
+        k_rem -= __shfl_sync(0xFFFFFFFFu, inc, 31);
+    }
+    return 0;
+}
+// hist[0..127] holds mantissa counts.  Returns the mantissa that holds rank k_rem from the top and the
+// rank inside it (1-based: how many elements of that bin are still needed).
+__device__ __forceinline__ uint32_t pick_mantissa(const uint32_t* hist, uint32_t k_rem, uint32_t& take) {
+    const uint32_t lane = lane_id();
+    // lane owns 4 bins, top-down: bin(lane, q) = 127 - (4 lane + q)
+    const uint4 h = reinterpret_cast<const uint4*>(hist)[31 - lane];
+    const uint32_t c[4] = {h.w, h.z, h.y, h.x};
+    const uint32_t own = c[0] + c[1] + c[2] + c[3];
+    uint32_t above = warp_inclusive_sum(own) - own, found = 0xFFFFFFFFu, found_take = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if (above < k_rem && k_rem <= above + c[q]) {
+            found = 127u - (4u * lane + q);
+            found_take = k_rem - above;
+        }
+        above += c[q];
+    }
+    const uint32_t who = __ballot_sync(0xFFFFFFFFu, found != 0xFFFFFFFFu);
+    const int src = who ? __ffs(who) - 1 : 0;
+    take = __shfl_sync(0xFFFFFFFFu, found_take, src);
+    return __shfl_sync(0xFFFFFFFFu, found, src) & 0x7Fu;
+}
+
+template <int E8>
+__global__ void __launch_bounds__(kFwdMaxWarps * 32)
+mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
+                             int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
+                             int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
+                             dct_result_t* __restrict__ result) {
+    using Lay = WarpRowLayout<E8>;
+    constexpr uint32_t E = Lay::E;
+    constexpr int kMaskWords = (E8 + 3) / 4;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    const uint32_t cap = Lay::list_cap(k);
+    unsigned char* base = smem_raw + warp * Lay::warp_bytes(k);
+    unsigned char* span = base + lane * Lay::kSpanBytes;
+    uint32_t* list = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
+    uint32_t* hist = list + cap;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(hist + kHistWords);
+    __shared__ uint32_t s_stop;
+
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+    if (threadIdx.x == 0) s_stop = 0;
+    if (lane == 0) {
+        mbar_init(bar, 1);
+        mbar_init_fence();
+        fence_proxy_async_all();
+    }
+    __syncthreads();
+
+    const uint32_t warp_global = blockIdx.x * (blockDim.x >> 5) + warp;
+    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
+    auto request_row = [&](uint32_t r) {
+        if (lane == 0) mbar_arrive_expect_tx(bar, Lay::D * 2u);
+        __syncwarp();
+        bulk_load(span, x + static_cast<size_t>(r) * ld + lane * E, E * 2u, bar);
+    };
+    auto release_row = [&](uint32_t row) {   // the row buffer is no longer needed: request the next row
+        __syncwarp();
+        fence_proxy_async_smem();
+        if (row + total_warps < rows) request_row(row + total_warps);
+    };
+    if (warp_global < rows) request_row(warp_global);
+
+    uint32_t use = 0;
+    for (uint32_t row = warp_global; row < rows; row += total_warps, ++use) {
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
+            s_stop = 1;
+            if (lane == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
+            return;
+        }
+        const size_t out_base = static_cast<size_t>(row) * k;
+
+        // ---- A: leaf maxima, then their k-th largest as the lower bound ---------------------------
+        uint32_t leaf[E8];
+        uint32_t row_max = 0;
+#pragma unroll
+        for (int c = 0; c < E8; ++c) {
+            const uint4 v = *reinterpret_cast<const uint4*>(span + c * 16);
+            const __nv_bfloat162 m2 = __hmax2(__hmax2(__habs2(as_bf162(v.x)), __habs2(as_bf162(v.y))),
+                                              __hmax2(__habs2(as_bf162(v.z)), __habs2(as_bf162(v.w))));
+            const uint32_t m = as_u32(m2);
+            leaf[c] = max(m & 0xFFFFu, m >> 16);
+            row_max = max(row_max, leaf[c]);
+        }
+        row_max = __reduce_max_sync(0xFFFFFFFFu, row_max);
+        uint32_t low = 0;
+        if (k <= 32u * E8) {       // otherwise there are fewer leaves than k: no bound, everything is a candidate
+            uint32_t k_rem = k, unused;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < E8; ++c) atomicAdd(&hist[(leaf[c] >> 7) * 4u + (lane & 3u)], 1u);
+            __syncwarp();
+            const uint32_t eb = pick_exponent(hist, row_max >> 7, k_rem);
+            __syncwarp();
+            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < E8; ++c)
+                if ((leaf[c] >> 7) == eb) atomicAdd(&hist[leaf[c] & 0x7Fu], 1u);
+            __syncwarp();
+            low = (eb << 7) | pick_mantissa(hist, k_rem, unused);
+            __syncwarp();
+        }
+
+        // ---- B: ordered compaction of the candidates ---------------------------------------------
+        uint32_t masks[kMaskWords];
+#pragma unroll
+        for (int i = 0; i < kMaskWords; ++i) masks[i] = 0;
+        uint32_t n_mine = 0;
+        {
+            const __nv_bfloat162 low2 = as_bf162(low | (low << 16));
+#pragma unroll
+            for (int c = 0; c < E8; ++c) {
+                const uint32_t m = mask8_ge_filter(*reinterpret_cast<const uint4*>(span + c * 16), low2);
+                masks[c / 4] |= m << (8 * (c % 4));
+                n_mine += __popc(m);
+            }
+        }
+        uint32_t incl = warp_inclusive_sum(n_mine);
+        uint32_t n_cand = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        if (n_cand > cap) {
+            // many elements tie at `low`: keep only what lies strictly above it (exact integer compare)
+            uint32_t eq_masks[kMaskWords];
+            n_mine = 0;
+            uint32_t n_eq_mine = 0;
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) masks[i] = eq_masks[i] = 0;
+#pragma unroll
+            for (int c = 0; c < E8; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4*>(span + c * 16);
+                const uint32_t gt = mask8_ge_exact(v, low + 1u);
+                const uint32_t eq = mask8_ge_exact(v, low) & ~gt;
+                masks[c / 4] |= gt << (8 * (c % 4));
+                eq_masks[c / 4] |= eq << (8 * (c % 4));
+                n_mine += __popc(gt);
+                n_eq_mine += __popc(eq);
+            }
+            incl = warp_inclusive_sum(n_mine);
+            n_cand = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            if (n_cand < k) {
+                // tau_i = low; keep everything above it and the first k - n_cand ties, straight from the row
+                const uint32_t take = k - n_cand;
+                uint32_t g_at = incl - n_mine;
+                uint32_t e_at = warp_inclusive_sum(n_eq_mine) - n_eq_mine;
+#pragma unroll
+                for (int c = 0; c < E8; ++c) {
+                    const uint32_t gm = (masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
+                    const uint32_t em = (eq_masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
+                    uint32_t m = gm | em;
+                    while (m) {
+                        const uint32_t bit = __ffs(m) - 1;
+                        m &= m - 1;
+                        const bool is_eq = (em >> bit) & 1u;
+                        if (!is_eq || e_at < take) {
+                            const uint32_t j = c * 8 + bit;
+                            const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
+                            cols_out[pos] = static_cast<int16_t>(lane * E + j);
+                            vals_out[pos] = *reinterpret_cast<const uint16_t*>(span + j * 2);
+                            if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
+                        }
+                        g_at += is_eq ? 0u : 1u;
+                        e_at += is_eq ? 1u : 0u;
+                    }
+                }
+                if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(low);
+                release_row(row);
+                continue;
+            }
+        }
+        {
+            uint32_t at = incl - n_mine;
+#pragma unroll
+            for (int c = 0; c < E8; ++c) {
+                uint32_t m = (masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
+                while (m) {
+                    const uint32_t j = c * 8 + (__ffs(m) - 1);
+                    m &= m - 1;
+                    const uint32_t raw = *reinterpret_cast<const uint16_t*>(span + j * 2);
+                    list[at++] = raw | ((lane * E + j) << 16);
+                }
+            }
+        }
+        release_row(row);
+
+        // ---- C: k-th largest of the candidates --------------------------------------------------
+        uint32_t k_rem = k, take;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
+        __syncwarp();
+        for (uint32_t q = lane; q < n_cand; q += 32)
+            atomicAdd(&hist[((list[q] & 0x7FFFu) >> 7) * 4u + (lane & 3u)], 1u);
+        __syncwarp();
+        const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
+        __syncwarp();
+        reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+        __syncwarp();
+        for (uint32_t q = lane; q < n_cand; q += 32) {
+            const uint32_t key = list[q] & 0x7FFFu;
+            if ((key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
+        }
+        __syncwarp();
+        const uint32_t tau_key = (exp_bin << 7) | pick_mantissa(hist, k_rem, take);
+        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+
+        // ---- D: ordered emit from the candidate list ---------------------------------------------------
+        uint32_t g_run = 0, e_run = 0;
+        for (uint32_t q0 = 0; q0 < n_cand; q0 += 32) {
+            if (g_run + (e_run < take ? e_run : take) >= k) break;
+            const uint32_t q = q0 + lane;
+            const uint32_t ent = q < n_cand ? list[q] : 0u;
+            const uint32_t key = ent & 0x7FFFu;
+            const bool is_gt = q < n_cand && key > tau_key, is_eq = q < n_cand && key == tau_key;
+            const uint32_t bg = __ballot_sync(0xFFFFFFFFu, is_gt), be = __ballot_sync(0xFFFFFFFFu, is_eq);
+            const uint32_t lt = lanemask_lt();
+            const uint32_t eq_before = e_run + __popc(be & lt);
+            if (is_gt || (is_eq && eq_before < take)) {
+                const uint32_t pos = g_run + __popc(bg & lt) + (eq_before < take ? eq_before : take);
+                cols_out[out_base + pos] = static_cast<int16_t>(ent >> 16);
+                vals_out[out_base + pos] = static_cast<uint16_t>(ent & 0xFFFFu);
+                if (rows_out) rows_out[out_base + pos] = static_cast<int32_t>(row);
+            }
+            g_run += __popc(bg);
+            e_run += __popc(be);
+        }
+        __syncwarp();
+    }
+}
+
+template <int E8>
+dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+                                  void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
+                                  cudaStream_t stream) {
+    using Lay = WarpRowLayout<E8>;
+    auto kernel = mp_topk_fwd_bf16_warp_kernel<E8>;
+    constexpr size_t kSmemBudget = 220 * 1024;            // of the 227 KiB a CTA may use
+    static thread_local int configured_device = -1;
+    int dev = 0;
+    DCT_CUDA_TRY(cudaGetDevice(&dev));
+    if (configured_device != dev) {
+        DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kSmemBudget)));
+        configured_device = dev;
+    }
+    const size_t per_warp = Lay::warp_bytes(k);
+    size_t warps = kSmemBudget / per_warp;                 // one CTA per SM with as many row slots as fit
+    if (warps > static_cast<size_t>(kFwdMaxWarps)) warps = kFwdMaxWarps;
+    if (warps < 1) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
+    const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
+    kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
+        static_cast<const uint16_t*>(x_act), rows, ld, k, cols_out, static_cast<uint16_t*>(vals_out), rows_out,
+        static_cast<uint16_t*>(tau_out), result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}
+
 int fwd_threads_for(uint32_t d) {
     if (d <= 4096) return 128;
     if (d <= 8192) return 256;
@@ -277,6 +639,16 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (dtype == DCT_F32)
         return launch_fwd<float>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0) {
+        switch (d) {   // warp-per-row path: d = 256 * 2^j
+            case 256: return launch_fwd_bf16_warp<1>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 512: return launch_fwd_bf16_warp<2>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 1024: return launch_fwd_bf16_warp<4>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 2048: return launch_fwd_bf16_warp<8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 4096: return launch_fwd_bf16_warp<16>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            default: break;
+        }
+    }
     return launch_fwd<uint16_t>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
 }
 
