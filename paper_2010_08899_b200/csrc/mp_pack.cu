@@ -232,7 +232,7 @@ template <int E8> struct WarpRowLayout {
     static constexpr uint32_t kRowBytes = 32u * kSpanBytes;
     // list capacity: every element above `low` always fits (< 8 k); rounded up, at most d
     __host__ __device__ static constexpr uint32_t list_cap(uint32_t k) {
-        return (8u * k + 64u) < D ? ((8u * k + 64u) & ~31u) : D;
+        return (8u * k + 255u) < D ? ((8u * k + 255u) & ~255u) : D;   // multiple of 256
     }
     __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) {
         return kRowBytes + list_cap(k) * 4u + kHistWords * 4u + 16u;
@@ -412,6 +412,11 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             __syncwarp();
         }
 
+#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 1
+        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(low);
+        release_row(row);
+        continue;
+#endif
         // ---- B: ordered compaction of the candidates ---------------------------------------------
         uint32_t masks[kMaskWords];
 #pragma unroll
@@ -428,6 +433,11 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         }
         uint32_t incl = warp_inclusive_sum(n_mine);
         uint32_t n_cand = __shfl_sync(0xFFFFFFFFu, incl, 31);
+#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 2
+        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(n_cand);
+        release_row(row);
+        continue;
+#endif
         if (n_cand > cap) {
             // many elements tie at `low`: keep only what lies strictly above it (exact integer compare)
             uint32_t eq_masks[kMaskWords];
@@ -480,10 +490,10 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         {
             uint32_t at = incl - n_mine;
 #pragma unroll
-            for (int c = 0; c < E8; ++c) {
-                uint32_t m = (masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
+            for (int wd = 0; wd < kMaskWords; ++wd) {     // bit b of word wd is element 32 wd + b of the lane's span
+                uint32_t m = masks[wd];
                 while (m) {
-                    const uint32_t j = c * 8 + (__ffs(m) - 1);
+                    const uint32_t j = wd * 32 + (__ffs(m) - 1);
                     m &= m - 1;
                     const uint32_t raw = *reinterpret_cast<const uint16_t*>(span + j * 2);
                     list[at++] = raw | ((lane * E + j) << 16);
@@ -491,46 +501,87 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             }
         }
         release_row(row);
+#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 3
+        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(list[0]);
+        continue;
+#endif
 
         // ---- C: k-th largest of the candidates --------------------------------------------------
+        // The list is consumed in rounds of 256 entries, 8 consecutive entries per lane (two 128-bit
+        // reads); with the usual ~1.2 k candidates there is one round and the entries stay in registers
+        // from the first histogram to the final write.
+        uint32_t ent[8];
+        auto load_round = [&](uint32_t q0) -> uint32_t {      // returns how many of the lane's 8 entries exist
+            const uint32_t first = q0 + lane * 8u;
+            const uint4 a = *reinterpret_cast<const uint4*>(list + first);
+            const uint4 b = *reinterpret_cast<const uint4*>(list + first + 4);
+            ent[0] = a.x; ent[1] = a.y; ent[2] = a.z; ent[3] = a.w;
+            ent[4] = b.x; ent[5] = b.y; ent[6] = b.z; ent[7] = b.w;
+            return first >= n_cand ? 0u : (n_cand - first < 8u ? n_cand - first : 8u);
+        };
+        const bool one_round = n_cand <= 256u;
+        __syncwarp();
+        uint32_t nvalid = load_round(0);
         uint32_t k_rem = k, take;
 #pragma unroll
         for (int i = 0; i < 8; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
         __syncwarp();
-        for (uint32_t q = lane; q < n_cand; q += 32)
-            atomicAdd(&hist[((list[q] & 0x7FFFu) >> 7) * 4u + (lane & 3u)], 1u);
+        for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
+            if (q0) nvalid = load_round(q0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if (static_cast<uint32_t>(i) < nvalid)
+                    atomicAdd(&hist[((ent[i] & 0x7FFFu) >> 7) * 4u + (lane & 3u)], 1u);
+        }
         __syncwarp();
         const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
         __syncwarp();
         reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
         __syncwarp();
-        for (uint32_t q = lane; q < n_cand; q += 32) {
-            const uint32_t key = list[q] & 0x7FFFu;
-            if ((key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
+        for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
+            if (!one_round) nvalid = load_round(q0);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t key = ent[i] & 0x7FFFu;
+                if (static_cast<uint32_t>(i) < nvalid && (key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
+            }
         }
         __syncwarp();
         const uint32_t tau_key = (exp_bin << 7) | pick_mantissa(hist, k_rem, take);
         if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 4
+        continue;
+#endif
 
         // ---- D: ordered emit from the candidate list ---------------------------------------------------
         uint32_t g_run = 0, e_run = 0;
-        for (uint32_t q0 = 0; q0 < n_cand; q0 += 32) {
-            if (g_run + (e_run < take ? e_run : take) >= k) break;
-            const uint32_t q = q0 + lane;
-            const uint32_t ent = q < n_cand ? list[q] : 0u;
-            const uint32_t key = ent & 0x7FFFu;
-            const bool is_gt = q < n_cand && key > tau_key, is_eq = q < n_cand && key == tau_key;
-            const uint32_t bg = __ballot_sync(0xFFFFFFFFu, is_gt), be = __ballot_sync(0xFFFFFFFFu, is_eq);
-            const uint32_t lt = lanemask_lt();
-            const uint32_t eq_before = e_run + __popc(be & lt);
-            if (is_gt || (is_eq && eq_before < take)) {
-                const uint32_t pos = g_run + __popc(bg & lt) + (eq_before < take ? eq_before : take);
-                cols_out[out_base + pos] = static_cast<int16_t>(ent >> 16);
-                vals_out[out_base + pos] = static_cast<uint16_t>(ent & 0xFFFFu);
-                if (rows_out) rows_out[out_base + pos] = static_cast<int32_t>(row);
+        for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
+            if (!one_round) nvalid = load_round(q0);
+            uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t key = ent[i] & 0x7FFFu;
+                if (static_cast<uint32_t>(i) < nvalid) counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
             }
-            g_run += __popc(bg);
-            e_run += __popc(be);
+            const uint32_t inc = warp_inclusive_sum(counts);
+            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);
+            uint32_t g_at = g_run + ((inc - counts) >> 16), e_at = e_run + ((inc - counts) & 0xFFFFu);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t key = ent[i] & 0x7FFFu;
+                const bool live = static_cast<uint32_t>(i) < nvalid;
+                const bool is_gt = live && key > tau_key, is_eq = live && key == tau_key;
+                if (is_gt || (is_eq && e_at < take)) {
+                    const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
+                    cols_out[pos] = static_cast<int16_t>(ent[i] >> 16);
+                    vals_out[pos] = static_cast<uint16_t>(ent[i] & 0xFFFFu);
+                    if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
+                }
+                g_at += is_gt ? 1u : 0u;
+                e_at += is_eq ? 1u : 0u;
+            }
+            g_run += tot >> 16;
+            e_run += tot & 0xFFFFu;
         }
         __syncwarp();
     }

@@ -65,9 +65,10 @@ def main():
         x = [inputs.mp_activations(rows, d, 410 + j, dtype=dt, device=dev, col_scale_seed=400) for j in range(2)]
         cols = torch.empty(rows * k, dtype=torch.int16, device=dev)
         vals = torch.empty(rows * k, dtype=dt, device=dev)
+        tau_i = torch.empty(rows, dtype=dt, device=dev)
         B.dct_mp_topk_pack_fwd(x[0], rows, d, d, k, cols, vals)
         if args.entry == "mp_fwd":
-            call = lambda i: B.dct_mp_topk_pack_fwd(x[i % 2], rows, d, d, k, cols, vals)
+            call = lambda i: B.dct_mp_topk_pack_fwd(x[i % 2], rows, d, d, k, cols, vals, None, tau_i)
             nbytes = rows * d * es + rows * k * (2 + es)
         else:
             gx = [inputs.mp_gradients(rows, d, 420 + j, dtype=dt, device=dev) for j in range(2)]
