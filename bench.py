@@ -49,9 +49,10 @@ WORKLOADS = {
 }
 DEFAULT_WORKLOAD = "dp_2p30_x20+mp_16384x4096_bf16_x50"
 
-# DRAM bytes per element of the dominant kernel from the committed ncu capture
-# (profiles/dp_compress_kernel_*.md); None until a capture exists.
-NCU_DRAM_BYTES_PER_ELEM_COMPRESS = None
+# DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum) of the dominant kernel, from the
+# ncu capture at N = 2^28 summarised in profiles/dp_compress_stream_kernel_n2p28.md; traffic grows in
+# proportion to N, so it is scaled to the launch's element count.
+NCU_DRAM_BYTES_PER_ELEM_COMPRESS = 11.816
 
 
 def algorithmic_bytes(cfg, survivors_per_iter):
@@ -232,8 +233,9 @@ def _record(stream):
 
 
 class ClockSampler:
-    """nvidia-smi sampling of SM clock and throttle reasons while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    """nvidia-smi sampling of SM clock and throttle reasons.  Started before the warm-up so that it is
+    running when the timed region begins; only samples stamped inside the timed window are used."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -245,7 +247,7 @@ class ClockSampler:
             self.uuid = None
 
     def start(self):
-        cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"]
+        cmd = ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"]
         if self.uuid:
             cmd += ["-i", self.uuid]
         try:
@@ -253,31 +255,42 @@ class ClockSampler:
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin: float, t_end: float):
+        """t_begin / t_end: time.time() around the timed region."""
+        import datetime
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             text, _ = self.proc.communicate(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
             text, _ = self.proc.communicate()
-        sm, smax, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        rows = []
         for line in text.strip().splitlines():
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) != 7:
+            if len(parts) != 8:
                 continue
             try:
-                sm.append(float(parts[0])); smax.append(float(parts[1])); power.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]), parts[4:]))
             except ValueError:
                 continue
-            for nm, v in zip(names, parts[3:]):
+        inside = [r for r in rows if t_begin - 0.02 <= r[0] <= t_end + 0.02]
+        window = "timed region"
+        if not inside:                      # clock skew or a very short region: fall back to the busiest samples
+            inside, window = sorted(rows, key=lambda r: -r[3])[:max(1, len(rows) // 4)], "highest-power samples of the run"
+        reasons = set()
+        for r in inside:
+            for nm, v in zip(names, r[4]):
                 if v.lower().startswith("active"):
                     reasons.add(nm)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+        return {"sm_mhz": statistics.median(r[1] for r in inside) if inside else None,
+                "sm_max_mhz": max(r[2] for r in inside) if inside else None,
+                "power_w_max": max(r[3] for r in inside) if inside else None,
+                "samples": len(inside), "window": window, "reasons": sorted(reasons)}
 
 
 def reduce_over_ranks(elapsed_ms: float, units: float, device=None):
@@ -413,14 +426,15 @@ def main():
     hp = HotPath(cfg, device, rank, total_steps)
     torch.cuda.synchronize()
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
     for _ in range(args.warmup):
         hp.step(stream)
     barrier()
     launches_before = hp.launches
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     events = []
     barrier()
+    wall_begin = time.time()
     t_start = _record(stream)
     for _ in range(args.steps):
         ev = []
@@ -428,7 +442,7 @@ def main():
         events.append(ev)
     t_stop = _record(stream)
     barrier()
-    clocks = sampler.stop()
+    clocks = sampler.stop(wall_begin, time.time())
     elapsed_ms = t_start.elapsed_time(t_stop)
     gpu_launches = hp.launches - launches_before
 
@@ -462,7 +476,7 @@ def main():
                    "dense_equiv_GBps": cfg["mp_rows"] * cfg["mp_d"] * 2 / (mp_parts["mp_bwd"] * 1e-3) / 1e9},
     }
     roofline = {
-        "kernel": "dp_compress_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "kernel": "dp_compress_stream_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_kind": peak_kind,
         "traffic": None if NCU_DRAM_BYTES_PER_ELEM_COMPRESS is None else NCU_DRAM_BYTES_PER_ELEM_COMPRESS * n,
         "algorithmic_bytes_per_launch": cmp_bytes_avg,
