@@ -245,6 +245,35 @@ DCT_API dct_status_t dct_mp_pack_host(
     dct_result_t* result_dev, dct_result_t* result_host, dct_stream_t stream);
 
 /*
+ * dct_dp_compress_static -- dct_dp_compress without a workspace argument.
+ * (The paper has no counterpart for this call; it exists for integration reasons only.)
+ *
+ * Some callers have no device memory of their own to offer as a workspace and may not obtain any:
+ * a gradient hook that runs inside a framework whose caching allocator already owns the whole GPU
+ * (a raw cudaMalloc there can fail outright, and it stalls every stream of the device while it
+ * runs), or a plug-in that is only ever handed the tensors it must transform.  For them the tile
+ * descriptors live in an array that is part of the library image itself: 262,400 bytes of device
+ * memory on every GPU that loads the library, held until the process exits.  The call allocates
+ * nothing -- no cudaMalloc, no cudaFree, no library routine that allocates.
+ *
+ * Arguments, outputs, result codes and semantics are exactly those of dct_dp_compress, with
+ *   n <= DCT_DP_COMPRESS_STATIC_MAX_N (2^27 elements); a larger n returns DCT_ERR_UNSUPPORTED
+ *   before anything is launched.
+ * The first call on each device looks up the device address of the built-in array (with that
+ * device current) and remembers it; make that first call outside any stream capture.
+ * All calls on one device share the one array.  Each call re-initialises the part it uses, so
+ * calls that follow one another on a stream are independent of what the previous one left
+ * behind; two calls that may run on the GPU at the same time (different streams, no ordering)
+ * would overwrite each other's descriptors -- use dct_dp_compress with separate workspaces then.
+ */
+#define DCT_DP_COMPRESS_STATIC_MAX_N (1u << 27)
+DCT_API dct_status_t dct_dp_compress_static(
+    const float* grad, float* residual, uint64_t n,
+    const float* tau, const uint64_t* tie_budget,
+    int32_t* idx_out, float* val_out, uint64_t capacity,
+    dct_result_t* result, dct_stream_t stream);
+
+/*
  * Testing knobs (process-wide, not for production use).  spin_limit is the
  * number of polls a device-side wait may take before it gives up with
  * DCT_ERR_TIMEOUT (default 2^21, about a second).  first_ticket is the id of

@@ -28,6 +28,7 @@ EXPORTED_SYMBOLS = (
     "dct_threshold_select_workspace_bytes", "dct_dp_compress_workspace_bytes",
     "dct_threshold_select", "dct_dp_compress", "dct_mp_topk_pack_fwd", "dct_mp_pack_bwd",
     "dct_dp_compress_host", "dct_mp_pack_host", "dct_threshold_select_host", "dct_debug_configure",
+    "dct_dp_compress_static",
 )
 
 _vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
@@ -68,6 +69,8 @@ def lib() -> ctypes.CDLL:
     L.dct_threshold_select.argtypes = [_vp, _vp, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
     L.dct_dp_compress.restype = _int
     L.dct_dp_compress.argtypes = [_vp, _vp, _u64, _vp, _vp, _vp, _vp, _u64, _vp, _vp, _sz, _vp]
+    L.dct_dp_compress_static.restype = _int
+    L.dct_dp_compress_static.argtypes = [_vp, _vp, _u64, _vp, _vp, _vp, _vp, _u64, _vp, _vp]
     L.dct_mp_topk_pack_fwd.restype = _int
     L.dct_mp_topk_pack_fwd.argtypes = [_vp, _int, _u32, _u32, _u32, _u32, _vp, _vp, _vp, _vp, _vp, _vp]
     L.dct_mp_pack_bwd.restype = _int
@@ -204,6 +207,29 @@ def dct_dp_compress(grad, residual, n, tau, tie_budget, idx_out, val_out, capaci
     _check("dct_dp_compress",
            lib().dct_dp_compress(_p(grad), _p(residual), n, _p(tau), _p(tie_budget), _p(idx_out), _p(val_out),
                                  capacity, _p(result), _p(workspace), workspace.numel(), _stream(stream)))
+
+
+DCT_DP_COMPRESS_STATIC_MAX_N = 1 << 27
+
+
+def dct_dp_compress_static(grad, residual, n, tau, tie_budget, idx_out, val_out, capacity, result, stream=None) -> None:
+    """dct_dp_compress for callers that have no workspace to give: the scratch is an array built into the
+    library (n <= DCT_DP_COMPRESS_STATIC_MAX_N).  Calls on one device share that array, so do not let two
+    of them overlap on the GPU; the first call per device should happen outside stream capture."""
+    _need(grad, torch.float32, "grad")
+    _need(residual, torch.float32, "residual")
+    _need(tau, torch.float32, "tau")
+    if tie_budget is not None:
+        _need(tie_budget, torch.int64, "tie_budget")
+    _need(idx_out, torch.int32, "idx_out")
+    _need(val_out, torch.float32, "val_out")
+    _need(result, torch.int64, "result")
+    if n <= DCT_DP_COMPRESS_STATIC_MAX_N and (grad.numel() < n or residual.numel() < n or
+                                              idx_out.numel() < capacity or val_out.numel() < capacity):
+        raise ValueError("buffer smaller than n / capacity")
+    _check("dct_dp_compress_static",
+           lib().dct_dp_compress_static(_p(grad), _p(residual), n, _p(tau), _p(tie_budget), _p(idx_out),
+                                        _p(val_out), capacity, _p(result), _stream(stream)))
 
 
 def dct_mp_topk_pack_fwd(x_act, rows, d, ld, k, cols_out, vals_out, rows_out=None, tau_out=None, result=None,

@@ -31,6 +31,8 @@
 //     same results).
 //   * dp_compress_tile_kernel -- one CTA per tile with plain loads and stores:
 //     the ragged last tile and vectors that are not 16-byte aligned.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace dct {
@@ -710,4 +712,54 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         DCT_CUDA_TRY(cudaGetLastError());
     }
     return DCT_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// dct_dp_compress_static: the same operator for callers that cannot hand over a workspace
+// ------------------------------------------------------------------------------------------
+// The tile descriptors and the ticket live in this file-scope device array instead of a caller
+// buffer.  Every GPU that loads the library carries these 256.25 KiB until the process exits.
+// In host code the array's name is only a stand-in: the device address is fetched once per device
+// with cudaGetSymbolAddress (that device being current) and handed to the kernels like any workspace.
+namespace {
+
+constexpr uint64_t kStaticMaxElems = DCT_DP_COMPRESS_STATIC_MAX_N;
+constexpr size_t kStaticScratchBytes = kCtrlBytes + sizeof(uint64_t) * (kStaticMaxElems / kTileElems);
+static_assert(kStaticMaxElems % kTileElems == 0, "the static scratch is sized in whole tiles");
+
+static __device__ __align__(256) unsigned char dct_static_scratch[kStaticScratchBytes];
+
+// Device address of dct_static_scratch on the current device, looked up on first use.
+cudaError_t static_scratch_address(void** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static void* address[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(mu);
+    if (address[dev] == nullptr) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, dct_static_scratch);   // resolves the symbol in the current device's copy
+        if (e != cudaSuccess) return e;
+        address[dev] = p;
+    }
+    *out = address[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" dct_status_t dct_dp_compress_static(const float* grad, float* residual, uint64_t n, const float* tau,
+                                               const uint64_t* tie_budget, int32_t* idx_out, float* val_out,
+                                               uint64_t capacity, dct_result_t* result, dct_stream_t stream) {
+    if (n == 0) return DCT_ERR_INVALID_ARG;
+    if (n > kStaticMaxElems) return DCT_ERR_UNSUPPORTED;   // the built-in scratch only covers DCT_DP_COMPRESS_STATIC_MAX_N
+    void* scratch = nullptr;
+    DCT_CUDA_TRY(static_scratch_address(&scratch));
+    // dct_dp_compress resets the ticket and every descriptor it is going to use before the main
+    // kernel runs, so whatever the previous call left in the array does not matter.
+    return dct_dp_compress(grad, residual, n, tau, tie_budget, idx_out, val_out, capacity, result, scratch,
+                           kStaticScratchBytes, stream);
 }
