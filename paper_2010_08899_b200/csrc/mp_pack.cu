@@ -216,23 +216,27 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 //   B  candidates (key >= low; typically ~1.2 k of them) are compacted, in column order, into a list.
 //   C  exact k-th largest of the candidates: radix select, exponent byte then mantissa.
 //   D  the kept columns (key > tau_i, then the lowest-column ties) leave the list in order.
-// If the candidates do not fit the list, at least cap - 8 (k - 1) elements tie at `low`: the list is
-// rebuilt from the elements strictly above `low` (always < 8 k of them); if fewer than k of those
-// exist, tau_i = low and the output is written straight from the row.
+// If the candidates do not fit the list (heavy ties at the bound, or k larger than the number of leaves
+// and a short list), the row takes a slow general path: tau_i is found bit by bit by counting over the
+// row, and the output is written straight from the row.
 #ifndef DCT_FWD_MAX_WARPS
-#define DCT_FWD_MAX_WARPS 16
+#define DCT_FWD_MAX_WARPS 20
 #endif
 constexpr int kFwdMaxWarps = DCT_FWD_MAX_WARPS;   // rows in flight per CTA (one CTA per SM; shared memory bounds it)
 constexpr uint32_t kAbsMask2 = 0x7FFF7FFFu;
-constexpr uint32_t kHistWords = 4u * 256u;  // 4 lane-interleaved copies of 256 bins
+constexpr uint32_t kHistWords = 2u * 256u;  // 2 lane-interleaved copies of 256 bins
 
 template <int E8> struct WarpRowLayout {
     static constexpr uint32_t E = E8 * 8u, D = E * 32u;
-    static constexpr uint32_t kSpanBytes = E * 2u + 16u;
+    static constexpr uint32_t kSpanBytes = E * 2u;           // the row lies in shared memory as it does in HBM
     static constexpr uint32_t kRowBytes = 32u * kSpanBytes;
-    // list capacity: every element above `low` always fits (< 8 k); rounded up, at most d
+    // Lane l reads its 16-byte units in the rotated order (c + l) mod E8: with spans of 256 bytes the
+    // eight lanes of a quarter-warp then hit eight different bank groups instead of one.
+    static constexpr bool kRotate = (E8 == 16);
+    // list capacity (a multiple of 256): room for twice the usual ~1.2 k candidates when the leaf bound
+    // exists (k <= number of leaves); the whole row otherwise
     __host__ __device__ static constexpr uint32_t list_cap(uint32_t k) {
-        return (8u * k + 255u) < D ? ((8u * k + 255u) & ~255u) : D;   // multiple of 256
+        return k > 32u * E8 ? D : (((2u * k + 255u) & ~255u) < D ? ((2u * k + 255u) & ~255u) : D);
     }
     __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) {
         return kRowBytes + list_cap(k) * 4u + kHistWords * 4u + 16u;
@@ -275,7 +279,7 @@ __device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v) {
     return v;
 }
 
-// hist holds 4 interleaved copies of 256 exponent bins.  Returns the exponent that holds rank k_rem
+// hist holds 2 interleaved copies of 256 exponent bins.  Returns the exponent that holds rank k_rem
 // (counting from exponent `top_exp` downwards) and reduces k_rem to the rank inside that exponent.
 __device__ __forceinline__ uint32_t pick_exponent(const uint32_t* hist, uint32_t top_exp, uint32_t& k_rem) {
     const uint32_t lane = lane_id();
@@ -283,8 +287,8 @@ __device__ __forceinline__ uint32_t pick_exponent(const uint32_t* hist, uint32_t
         const int eb = top - static_cast<int>(lane);
         uint32_t c = 0;
         if (eb >= 0) {
-            const uint4 h = reinterpret_cast<const uint4*>(hist)[eb];
-            c = h.x + h.y + h.z + h.w;
+            const uint2 h = reinterpret_cast<const uint2*>(hist)[eb];
+            c = h.x + h.y;
         }
         const uint32_t inc = warp_inclusive_sum(c);
         const uint32_t hit = __ballot_sync(0xFFFFFFFFu, inc >= k_rem);
@@ -357,11 +361,14 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 
     const uint32_t warp_global = blockIdx.x * (blockDim.x >> 5) + warp;
     const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
-    auto request_row = [&](uint32_t r) {
-        if (lane == 0) mbar_arrive_expect_tx(bar, Lay::D * 2u);
-        __syncwarp();
-        bulk_load(span, x + static_cast<size_t>(r) * ld + lane * E, E * 2u, bar);
+    auto request_row = [&](uint32_t r) {          // one bulk copy brings the whole row
+        if (lane == 0) {
+            mbar_arrive_expect_tx(bar, Lay::D * 2u);
+            bulk_load(base, x + static_cast<size_t>(r) * ld, Lay::D * 2u, bar);
+        }
     };
+    // the lane's c-th read of a pass: unit (c + lane) mod E8 of its span when rotating, unit c otherwise
+    auto unit_of = [&](int c) -> uint32_t { return Lay::kRotate ? ((c + lane) & (E8 - 1)) : static_cast<uint32_t>(c); };
     auto release_row = [&](uint32_t row) {   // the row buffer is no longer needed: request the next row
         __syncwarp();
         fence_proxy_async_smem();
@@ -383,7 +390,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         uint32_t row_max = 0;
 #pragma unroll
         for (int c = 0; c < E8; ++c) {
-            const uint4 v = *reinterpret_cast<const uint4*>(span + c * 16);
+            const uint4 v = *reinterpret_cast<const uint4*>(span + unit_of(c) * 16);
             const __nv_bfloat162 m2 = __hmax2(__hmax2(__habs2(as_bf162(v.x)), __habs2(as_bf162(v.y))),
                                               __hmax2(__habs2(as_bf162(v.z)), __habs2(as_bf162(v.w))));
             const uint32_t m = as_u32(m2);
@@ -391,24 +398,41 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             row_max = max(row_max, leaf[c]);
         }
         row_max = __reduce_max_sync(0xFFFFFFFFu, row_max);
+#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 0
+        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(row_max + leaf[3]);
+        release_row(row);
+        continue;
+#endif
         uint32_t low = 0;
-        if (k <= 32u * E8) {       // otherwise there are fewer leaves than k: no bound, everything is a candidate
-            uint32_t k_rem = k, unused;
+        const bool have_bound = k <= 32u * E8;   // otherwise there are fewer leaves than k: everything is a candidate
+        if (have_bound) {
+            // One histogram pass over the leaf maxima in bins of 8 keys counted down from the row maximum
+            // (bin 255 collects everything further away).  The bound is the lowest key of the bin in which
+            // the count reaches k: at least k leaves, hence k elements, lie at or above it.
 #pragma unroll
-            for (int i = 0; i < 8; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
-            __syncwarp();
-#pragma unroll
-            for (int c = 0; c < E8; ++c) atomicAdd(&hist[(leaf[c] >> 7) * 4u + (lane & 3u)], 1u);
-            __syncwarp();
-            const uint32_t eb = pick_exponent(hist, row_max >> 7, k_rem);
-            __syncwarp();
-            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+            for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
             __syncwarp();
 #pragma unroll
-            for (int c = 0; c < E8; ++c)
-                if ((leaf[c] >> 7) == eb) atomicAdd(&hist[leaf[c] & 0x7Fu], 1u);
+            for (int c = 0; c < E8; ++c) {
+                const uint32_t rel = (row_max - leaf[c]) >> 3;
+                atomicAdd(&hist[(rel < 255u ? rel : 255u) * 2u + (lane & 1u)], 1u);
+            }
             __syncwarp();
-            low = (eb << 7) | pick_mantissa(hist, k_rem, unused);
+            uint32_t need = k, bin = 255;
+#pragma unroll 1
+            for (uint32_t first = 0; first < 256; first += 32) {
+                const uint2 h = reinterpret_cast<const uint2*>(hist)[first + lane];
+                const uint32_t c = h.x + h.y;
+                const uint32_t inc = warp_inclusive_sum(c);
+                const uint32_t hit = __ballot_sync(0xFFFFFFFFu, inc >= need);
+                if (hit) {
+                    bin = first + (__ffs(hit) - 1);
+                    break;
+                }
+                need -= __shfl_sync(0xFFFFFFFFu, inc, 31);
+            }
+            const uint32_t span_keys = bin * 8u + 7u;
+            low = (bin < 255u && row_max > span_keys) ? row_max - span_keys : 0u;
             __syncwarp();
         }
 
@@ -426,9 +450,21 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             const __nv_bfloat162 low2 = as_bf162(low | (low << 16));
 #pragma unroll
             for (int c = 0; c < E8; ++c) {
-                const uint32_t m = mask8_ge_filter(*reinterpret_cast<const uint4*>(span + c * 16), low2);
+                const uint32_t m = mask8_ge_filter(*reinterpret_cast<const uint4*>(span + unit_of(c) * 16), low2);
                 masks[c / 4] |= m << (8 * (c % 4));
                 n_mine += __popc(m);
+            }
+            if (Lay::kRotate) {
+                // byte c of the 128-bit mask belongs to unit (c + lane) mod 16: rotate left by 8 * (lane mod 16)
+                // bits so that byte u belongs to unit u (column order)
+                const uint32_t words = (lane >> 2) & 3u, bits = (lane & 3u) * 8u;
+                uint32_t w0 = masks[0], w1 = masks[1 % kMaskWords], w2 = masks[2 % kMaskWords], w3 = masks[3 % kMaskWords];
+                if (words & 1u) { const uint32_t t = w3; w3 = w2; w2 = w1; w1 = w0; w0 = t; }
+                if (words & 2u) { uint32_t t = w0; w0 = w2; w2 = t; t = w1; w1 = w3; w3 = t; }
+                masks[0] = __funnelshift_l(w3, w0, bits);
+                masks[1 % kMaskWords] = __funnelshift_l(w0, w1, bits);
+                masks[2 % kMaskWords] = __funnelshift_l(w1, w2, bits);
+                masks[3 % kMaskWords] = __funnelshift_l(w2, w3, bits);
             }
         }
         uint32_t incl = warp_inclusive_sum(n_mine);
@@ -439,7 +475,19 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         continue;
 #endif
         if (n_cand > cap) {
-            // many elements tie at `low`: keep only what lies strictly above it (exact integer compare)
+            // Rare: the candidates do not fit the list (heavy ties at the bound, or no usable bound).
+            // General slow path on the row itself: tau_i bit by bit, most significant first (the largest v
+            // with #{key >= v} >= k), then everything above tau_i and the first ties, in column order.
+            uint32_t tau_key = 0;
+#pragma unroll 1
+            for (int bit = 14; bit >= 0; --bit) {
+                const uint32_t trial = tau_key | (1u << bit);
+                uint32_t cnt = 0;
+#pragma unroll
+                for (int c = 0; c < E8; ++c)
+                    cnt += __popc(mask8_ge_exact(*reinterpret_cast<const uint4*>(span + c * 16), trial));
+                if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= k) tau_key = trial;
+            }
             uint32_t eq_masks[kMaskWords];
             n_mine = 0;
             uint32_t n_eq_mine = 0;
@@ -448,44 +496,40 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 #pragma unroll
             for (int c = 0; c < E8; ++c) {
                 const uint4 v = *reinterpret_cast<const uint4*>(span + c * 16);
-                const uint32_t gt = mask8_ge_exact(v, low + 1u);
-                const uint32_t eq = mask8_ge_exact(v, low) & ~gt;
+                const uint32_t gt = mask8_ge_exact(v, tau_key + 1u);
+                const uint32_t eq = mask8_ge_exact(v, tau_key) & ~gt;
                 masks[c / 4] |= gt << (8 * (c % 4));
                 eq_masks[c / 4] |= eq << (8 * (c % 4));
                 n_mine += __popc(gt);
                 n_eq_mine += __popc(eq);
             }
             incl = warp_inclusive_sum(n_mine);
-            n_cand = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            if (n_cand < k) {
-                // tau_i = low; keep everything above it and the first k - n_cand ties, straight from the row
-                const uint32_t take = k - n_cand;
-                uint32_t g_at = incl - n_mine;
-                uint32_t e_at = warp_inclusive_sum(n_eq_mine) - n_eq_mine;
+            const uint32_t take = k - __shfl_sync(0xFFFFFFFFu, incl, 31);   // ties to keep, lowest columns first
+            uint32_t g_at = incl - n_mine;
+            uint32_t e_at = warp_inclusive_sum(n_eq_mine) - n_eq_mine;
 #pragma unroll
-                for (int c = 0; c < E8; ++c) {
-                    const uint32_t gm = (masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
-                    const uint32_t em = (eq_masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
-                    uint32_t m = gm | em;
-                    while (m) {
-                        const uint32_t bit = __ffs(m) - 1;
-                        m &= m - 1;
-                        const bool is_eq = (em >> bit) & 1u;
-                        if (!is_eq || e_at < take) {
-                            const uint32_t j = c * 8 + bit;
-                            const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
-                            cols_out[pos] = static_cast<int16_t>(lane * E + j);
-                            vals_out[pos] = *reinterpret_cast<const uint16_t*>(span + j * 2);
-                            if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
-                        }
-                        g_at += is_eq ? 0u : 1u;
-                        e_at += is_eq ? 1u : 0u;
+            for (int c = 0; c < E8; ++c) {
+                const uint32_t gm = (masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
+                const uint32_t em = (eq_masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
+                uint32_t m = gm | em;
+                while (m) {
+                    const uint32_t bit = __ffs(m) - 1;
+                    m &= m - 1;
+                    const bool is_eq = (em >> bit) & 1u;
+                    if (!is_eq || e_at < take) {
+                        const uint32_t j = c * 8 + bit;
+                        const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
+                        cols_out[pos] = static_cast<int16_t>(lane * E + j);
+                        vals_out[pos] = *reinterpret_cast<const uint16_t*>(span + j * 2);
+                        if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
                     }
+                    g_at += is_eq ? 0u : 1u;
+                    e_at += is_eq ? 1u : 0u;
                 }
-                if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(low);
-                release_row(row);
-                continue;
             }
+            if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+            release_row(row);
+            continue;
         }
         {
             uint32_t at = incl - n_mine;
@@ -522,38 +566,82 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         const bool one_round = n_cand <= 256u;
         __syncwarp();
         uint32_t nvalid = load_round(0);
-        uint32_t k_rem = k, take;
+        uint32_t tau_key = 0, take = 0;
+        bool found = false;
+        if (have_bound && low != 0) {
+            // tau_i is the (n_cand - k + 1)-th smallest candidate.  Usually it lies within 64 keys of the
+            // bound: a 64-bin histogram of the candidates in [low, low + 64), walked from the bottom, finds it.
+            const uint32_t drop = n_cand - k;                 // candidates to discard, smallest first
+            hist[lane] = 0;
+            hist[lane + 32] = 0;
+            __syncwarp();
+            for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
+                if (q0) nvalid = load_round(q0);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
-        __syncwarp();
-        for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
-            if (q0) nvalid = load_round(q0);
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if (static_cast<uint32_t>(i) < nvalid)
-                    atomicAdd(&hist[((ent[i] & 0x7FFFu) >> 7) * 4u + (lane & 3u)], 1u);
-        }
-        __syncwarp();
-        const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
-        __syncwarp();
-        reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
-        __syncwarp();
-        for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
-            if (!one_round) nvalid = load_round(q0);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const uint32_t key = ent[i] & 0x7FFFu;
-                if (static_cast<uint32_t>(i) < nvalid && (key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t rel = (ent[i] & 0x7FFFu) - low;
+                    if (static_cast<uint32_t>(i) < nvalid && rel < 64u) atomicAdd(&hist[rel], 1u);
+                }
             }
+            __syncwarp();
+            const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
+            const uint32_t own = h.x + h.y;
+            const uint32_t before = warp_inclusive_sum(own) - own;
+            uint32_t my_tau = 0xFFFFFFFFu, my_take = 0;
+            if (before <= drop && drop < before + h.x) {
+                my_tau = low + 2u * lane;
+                my_take = h.x - (drop - before);
+            } else if (before + h.x <= drop && drop < before + own) {
+                my_tau = low + 2u * lane + 1u;
+                my_take = h.y - (drop - before - h.x);
+            }
+            const uint32_t who = __ballot_sync(0xFFFFFFFFu, my_tau != 0xFFFFFFFFu);
+            if (who) {
+                const int src = __ffs(who) - 1;
+                tau_key = __shfl_sync(0xFFFFFFFFu, my_tau, src);
+                take = __shfl_sync(0xFFFFFFFFu, my_take, src);
+                found = true;
+            }
+            __syncwarp();
+            if (!found && !one_round) nvalid = load_round(0);
         }
-        __syncwarp();
-        const uint32_t tau_key = (exp_bin << 7) | pick_mantissa(hist, k_rem, take);
+        if (!found) {
+            // general case: radix select over the candidates, exponent byte then mantissa
+            uint32_t k_rem = k;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
+            __syncwarp();
+            for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
+                if (q0) nvalid = load_round(q0);
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    if (static_cast<uint32_t>(i) < nvalid)
+                        atomicAdd(&hist[((ent[i] & 0x7FFFu) >> 7) * 2u + (lane & 1u)], 1u);
+            }
+            __syncwarp();
+            const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
+            __syncwarp();
+            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+            __syncwarp();
+            for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
+                if (!one_round) nvalid = load_round(q0);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t key = ent[i] & 0x7FFFu;
+                    if (static_cast<uint32_t>(i) < nvalid && (key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
+                }
+            }
+            __syncwarp();
+            tau_key = (exp_bin << 7) | pick_mantissa(hist, k_rem, take);
+        }
         if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
 #if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 4
         continue;
 #endif
 
-        // ---- D: ordered emit from the candidate list ---------------------------------------------------
+        // ---- D: ordered emit ------------------------------------------------------------------------
+        // The kept entries are first compacted in place at the front of the list (a kept entry never moves
+        // to a higher position), then the k entries leave with coalesced stores.
         uint32_t g_run = 0, e_run = 0;
         for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
             if (!one_round) nvalid = load_round(q0);
@@ -566,22 +654,25 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             const uint32_t inc = warp_inclusive_sum(counts);
             const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);
             uint32_t g_at = g_run + ((inc - counts) >> 16), e_at = e_run + ((inc - counts) & 0xFFFFu);
+            __syncwarp();                                     // every lane holds its entries in registers
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint32_t key = ent[i] & 0x7FFFu;
                 const bool live = static_cast<uint32_t>(i) < nvalid;
                 const bool is_gt = live && key > tau_key, is_eq = live && key == tau_key;
-                if (is_gt || (is_eq && e_at < take)) {
-                    const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
-                    cols_out[pos] = static_cast<int16_t>(ent[i] >> 16);
-                    vals_out[pos] = static_cast<uint16_t>(ent[i] & 0xFFFFu);
-                    if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
-                }
+                if (is_gt || (is_eq && e_at < take)) list[g_at + (e_at < take ? e_at : take)] = ent[i];
                 g_at += is_gt ? 1u : 0u;
                 e_at += is_eq ? 1u : 0u;
             }
             g_run += tot >> 16;
             e_run += tot & 0xFFFFu;
+        }
+        __syncwarp();
+        for (uint32_t p = lane; p < k; p += 32) {
+            const uint32_t e = list[p];
+            cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
+            vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
+            if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
         }
         __syncwarp();
     }
