@@ -224,7 +224,7 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 #endif
 constexpr int kFwdMaxWarps = DCT_FWD_MAX_WARPS;   // rows in flight per CTA (one CTA per SM; shared memory bounds it)
 constexpr uint32_t kAbsMask2 = 0x7FFF7FFFu;
-constexpr uint32_t kHistWords = 2u * 256u;  // 2 lane-interleaved copies of 256 bins
+constexpr uint32_t kHistWords = 256u;       // one histogram of up to 256 bins per warp
 
 template <int E8> struct WarpRowLayout {
     static constexpr uint32_t E = E8 * 8u, D = E * 32u;
@@ -279,7 +279,7 @@ __device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v) {
     return v;
 }
 
-// hist holds 2 interleaved copies of 256 exponent bins.  Returns the exponent that holds rank k_rem
+// hist holds 256 exponent bins.  Returns the exponent that holds rank k_rem
 // (counting from exponent `top_exp` downwards) and reduces k_rem to the rank inside that exponent.
 __device__ __forceinline__ uint32_t pick_exponent(const uint32_t* hist, uint32_t top_exp, uint32_t& k_rem) {
     const uint32_t lane = lane_id();
@@ -287,8 +287,7 @@ __device__ __forceinline__ uint32_t pick_exponent(const uint32_t* hist, uint32_t
         const int eb = top - static_cast<int>(lane);
         uint32_t c = 0;
         if (eb >= 0) {
-            const uint2 h = reinterpret_cast<const uint2*>(hist)[eb];
-            c = h.x + h.y;
+            c = hist[eb];
         }
         const uint32_t inc = warp_inclusive_sum(c);
         const uint32_t hit = __ballot_sync(0xFFFFFFFFu, inc >= k_rem);
@@ -409,20 +408,19 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             // One histogram pass over the leaf maxima in bins of 8 keys counted down from the row maximum
             // (bin 255 collects everything further away).  The bound is the lowest key of the bin in which
             // the count reaches k: at least k leaves, hence k elements, lie at or above it.
-#pragma unroll
-            for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
+            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+            reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
             __syncwarp();
 #pragma unroll
             for (int c = 0; c < E8; ++c) {
                 const uint32_t rel = (row_max - leaf[c]) >> 3;
-                atomicAdd(&hist[(rel < 255u ? rel : 255u) * 2u + (lane & 1u)], 1u);
+                atomicAdd(&hist[rel < 255u ? rel : 255u], 1u);
             }
             __syncwarp();
             uint32_t need = k, bin = 255;
 #pragma unroll 1
             for (uint32_t first = 0; first < 256; first += 32) {
-                const uint2 h = reinterpret_cast<const uint2*>(hist)[first + lane];
-                const uint32_t c = h.x + h.y;
+                const uint32_t c = hist[first + lane];
                 const uint32_t inc = warp_inclusive_sum(c);
                 const uint32_t hit = __ballot_sync(0xFFFFFFFFu, inc >= need);
                 if (hit) {
@@ -533,6 +531,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         }
         {
             uint32_t at = incl - n_mine;
+            const uint32_t col0 = (lane * E) << 16;
 #pragma unroll
             for (int wd = 0; wd < kMaskWords; ++wd) {     // bit b of word wd is element 32 wd + b of the lane's span
                 uint32_t m = masks[wd];
@@ -540,7 +539,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                     const uint32_t j = wd * 32 + (__ffs(m) - 1);
                     m &= m - 1;
                     const uint32_t raw = *reinterpret_cast<const uint16_t*>(span + j * 2);
-                    list[at++] = raw | ((lane * E + j) << 16);
+                    list[at++] = (raw | col0) + (j << 16);
                 }
             }
         }
@@ -608,15 +607,14 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         if (!found) {
             // general case: radix select over the candidates, exponent byte then mantissa
             uint32_t k_rem = k;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(hist)[i * 32 + lane] = make_uint4(0, 0, 0, 0);
+            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+            reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
             __syncwarp();
             for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
                 if (q0) nvalid = load_round(q0);
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
-                    if (static_cast<uint32_t>(i) < nvalid)
-                        atomicAdd(&hist[((ent[i] & 0x7FFFu) >> 7) * 2u + (lane & 1u)], 1u);
+                    if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent[i] & 0x7FFFu) >> 7], 1u);
             }
             __syncwarp();
             const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
