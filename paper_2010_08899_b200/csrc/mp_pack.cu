@@ -88,10 +88,18 @@ __global__ void mp_topk_pack_fwd_kernel(const T* __restrict__ x, uint32_t rows, 
             for (uint32_t b = tid; b < 256; b += nt) s_hist[b] = 0;
             __syncthreads();
             const uint32_t prefix = s_prefix;
+            // Exact zeros are the common value after a ReLU: in the first pass they are counted in a register
+            // and added to bin 0 once per thread instead of colliding on one shared-memory word.
+            uint32_t zeros = 0;
             for (uint32_t j = tid; j < d; j += nt) {
                 const uint32_t key = Tr::key(row_s[j]);
-                if (p == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&s_hist[(key >> shift) & (nbins - 1u)], 1u);
+                if (p == 0 && key == 0) {
+                    ++zeros;
+                } else if (p == 0 || (key >> (shift + bits)) == prefix) {
+                    atomicAdd(&s_hist[(key >> shift) & (nbins - 1u)], 1u);
+                }
             }
+            if (zeros) atomicAdd(&s_hist[0], zeros);
             __syncthreads();
             if (warp == 0) {
                 // lane owns 8 bins, top-down: bin(lane, q) = 255 - (8 lane + q); bins >= nbins are empty

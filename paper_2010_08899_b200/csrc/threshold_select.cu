@@ -1,14 +1,25 @@
 // dct_threshold_select: Algorithm 1 (DCT-DP), threshold steps.
 //
-// tau = k-th largest |grad + residual|, found exactly by a most-significant-
-// digit-first radix select on key(w) (31 magnitude bits) instead of the
-// copy-and-sort the paper describes: three passes over the data with digits of
-// 11, 10 and 10 bits.  Each pass builds a histogram of the current digit over
-// the elements whose higher bits equal the prefix chosen so far (per-CTA
-// histogram in shared memory, merged into global memory); the last CTA to
-// finish a pass scans the histogram from the top, picks the digit that holds
-// rank k and extends the prefix.  Nothing is copied, nothing is sorted, and the
-// input is never modified.
+// tau = k-th largest |grad + residual|, found exactly by a most-significant-digit-first radix
+// select on key(w) (31 magnitude bits, digits of 11/10/10 bits) instead of the copy-and-sort the
+// paper describes.  One radix pass streams its source once, builds the histogram of the current
+// digit over the elements whose higher bits equal the prefix chosen so far (per-CTA histogram in
+// shared memory, merged into global memory); the last CTA to finish the pass scans the histogram
+// from the top, picks the digit that holds rank k and extends the prefix.  Nothing is copied,
+// nothing is sorted, and the input is never modified.
+//
+// Three radix passes over the whole vector cost 12 B per element against a floor of 4 B.  When k is
+// small against n (the method's regime) the vector is therefore read only ONCE:
+//   1. a strided sample of 2^20 elements is radix-selected (it lives in L2) for a rank chosen so that,
+//      with overwhelming probability, between k and a few k elements of the whole vector lie at or
+//      above the sampled value `lo`;
+//   2. one streaming pass over the vector appends every key >= key(lo) to a candidate buffer in the
+//      workspace and counts them;
+//   3. if the count c satisfies k <= c <= capacity, tau is the k-th largest candidate (radix select
+//      over the small buffer) and n_gt, n_eq follow from the candidates, since every element >= tau
+//      is one of them.  Otherwise -- the sample misjudged the vector -- the three full passes run.
+// Every decision is taken on the device; all kernels are enqueued up front and the ones that are
+// not needed return at once.  The result is exact in every case.
 #include "common.cuh"
 
 namespace dct {
@@ -19,90 +30,100 @@ constexpr int kSelVecs = 4;
 constexpr uint32_t kSelChunk = kSelThreads * kSelVecs * 4;   // 8192 elements per CTA iteration
 constexpr int kBins = 2048;
 constexpr int kPasses = 3;
+constexpr uint32_t kSampleSize = 1u << 20;                   // elements in the strided sample
+constexpr uint32_t kMaxCandidates = 1u << 22;                // candidate buffer: at most 16 MiB
+#ifndef DCT_SEL_MIN_SAMPLED_N
+#define DCT_SEL_MIN_SAMPLED_N (1u << 27)
+#endif
+constexpr uint32_t kMinSampledN = DCT_SEL_MIN_SAMPLED_N;     // below this the three plain passes are cheaper
 
 __host__ __device__ constexpr int pass_shift(int p) { return p == 0 ? 20 : (p == 1 ? 10 : 0); }
 __host__ __device__ constexpr int pass_bits(int p) { return p == 0 ? 11 : 10; }
 
+// One radix select in flight.
 struct SelectState {
     uint32_t prefix;      // digits chosen so far (right-aligned)
     uint32_t k_rem;       // rank still to be located inside the prefix bucket
     uint64_t n_gt;        // elements known to be above the bucket
     uint32_t done[kPasses];
+    uint32_t enabled;     // 0: every kernel of this select returns at once
+    uint32_t n;           // elements of the source (written on the device for the candidate buffer)
+    uint32_t key_out;     // the selected key (the sample select hands `lo` to the filter this way)
+    uint32_t hist[kPasses * kBins];
 };
-constexpr size_t kSelStateBytes = 256;
 
-__global__ void select_init_kernel(SelectState* st, uint32_t* hist, uint32_t k) {
-    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < kPasses * kBins) hist[i] = 0;
+// Workspace layout: three select states (whole vector, sample, candidates), the candidate counter,
+// the candidate keys.
+struct SelectWorkspace {
+    SelectState full, sample, cand;
+    uint32_t cand_count;      // keys >= lo met by the filter pass (may exceed the capacity)
+    uint32_t cand_capacity;
+    uint32_t pad[62];
+};
+
+constexpr int kInitThreads = 1024;
+__device__ __forceinline__ void reset_state(SelectState* st, uint32_t k, uint32_t n, uint32_t enabled, uint32_t i,
+                                            uint32_t stride) {
+    for (uint32_t b = i; b < kPasses * kBins; b += stride) st->hist[b] = 0;
     if (i == 0) {
         st->prefix = 0;
         st->k_rem = k;
         st->n_gt = 0;
         for (int p = 0; p < kPasses; ++p) st->done[p] = 0;
+        st->enabled = enabled;
+        st->n = n;
+        st->key_out = 0;
     }
 }
 
-template <int kPass, bool kHasResidual, bool kVectorised>
-__global__ void __launch_bounds__(kSelThreads)
-select_pass_kernel(const float* __restrict__ grad, const float* __restrict__ residual, uint32_t n,
-                   SelectState* st, uint32_t* __restrict__ hist_all, float* __restrict__ tau_out,
-                   dct_result_t* __restrict__ result) {
-    constexpr int shift = pass_shift(kPass);
+__global__ void select_init_kernel(SelectWorkspace* ws, uint32_t n, uint32_t k, uint32_t sample_n, uint32_t sample_k,
+                                   uint32_t cand_capacity, dct_result_t* result) {
+    const uint32_t i = threadIdx.x;
+    const bool sampled = sample_n != 0;
+    reset_state(&ws->full, k, n, sampled ? 0u : 1u, i, kInitThreads);
+    reset_state(&ws->sample, sample_k, sample_n, sampled ? 1u : 0u, i, kInitThreads);
+    reset_state(&ws->cand, k, 0u, 0u, i, kInitThreads);
+    if (i == 0) {
+        ws->cand_count = 0;
+        ws->cand_capacity = cand_capacity;
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+}
+
+// Where a pass reads its keys from.
+struct VectorSource {        // key(fl32(grad[i] + residual[i])), i < n
+    const float* grad;
+    const float* residual;   // may be null
+};
+struct StridedSource {       // the same at i * stride
+    const float* grad;
+    const float* residual;
+    uint32_t stride;
+};
+struct KeySource {           // keys stored in the workspace
+    const uint32_t* keys;
+};
+
+__device__ __forceinline__ uint32_t key_at(const VectorSource& s, uint32_t i) {
+    return key_f32(s.residual ? __fadd_rn(s.grad[i], s.residual[i]) : s.grad[i]);
+}
+__device__ __forceinline__ uint32_t key_at(const StridedSource& s, uint32_t i) {
+    const size_t j = static_cast<size_t>(i) * s.stride;
+    return key_f32(s.residual ? __fadd_rn(s.grad[j], s.residual[j]) : s.grad[j]);
+}
+__device__ __forceinline__ uint32_t key_at(const KeySource& s, uint32_t i) { return s.keys[i]; }
+
+// Scan of one pass's histogram by the last CTA: the digit that holds rank k_rem, counted from the top.
+template <int kPass>
+__device__ __forceinline__ void finish_pass(SelectState* st, uint32_t prefix, uint32_t* s_scan, float* tau_out,
+                                            dct_result_t* result) {
     constexpr int bits = pass_bits(kPass);
-    constexpr uint32_t digit_mask = (1u << bits) - 1u;
-    __shared__ uint32_t sh[kBins];
-    __shared__ uint32_t s_scan[kSelThreads / 32];
-    __shared__ uint32_t s_last;
-
-    for (int b = threadIdx.x; b < kBins; b += kSelThreads) sh[b] = 0;
-    const uint32_t prefix = kPass == 0 ? 0u : st->prefix;   // written by the previous launch
-    __syncthreads();
-
-    auto consume = [&](float g, float e) {
-        const float w = kHasResidual ? __fadd_rn(g, e) : g;
-        const uint32_t key = key_f32(w);
-        if (kPass == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&sh[(key >> shift) & digit_mask], 1u);
-    };
-
-    const uint32_t num_chunks = (n + kSelChunk - 1) / kSelChunk;
-    for (uint32_t chunk = blockIdx.x; chunk < num_chunks; chunk += gridDim.x) {
-        const uint32_t base = chunk * kSelChunk;
-        if (kVectorised && base + kSelChunk <= n) {
-            float4 g4[kSelVecs], e4[kSelVecs];
-#pragma unroll
-            for (int j = 0; j < kSelVecs; ++j) {
-                const uint32_t off = base + (j * kSelThreads + threadIdx.x) * 4;
-                g4[j] = ld_readonly_f4(grad + off);
-                if (kHasResidual) e4[j] = ld_readonly_f4(residual + off);
-                else e4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-            for (int j = 0; j < kSelVecs; ++j) {
-                consume(g4[j].x, e4[j].x);
-                consume(g4[j].y, e4[j].y);
-                consume(g4[j].z, e4[j].z);
-                consume(g4[j].w, e4[j].w);
-            }
-        } else {
-            for (uint32_t i = base + threadIdx.x; i < n && i < base + kSelChunk; i += kSelThreads)
-                consume(grad[i], kHasResidual ? residual[i] : 0.0f);
-        }
-    }
-    __syncthreads();
-
-    uint32_t* hist = hist_all + kPass * kBins;
-    for (int b = threadIdx.x; b < kBins; b += kSelThreads) {
-        const uint32_t c = sh[b];
-        if (c) atomicAdd(&hist[b], c);
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) s_last = (atomicAdd(&st->done[kPass], 1u) == gridDim.x - 1) ? 1u : 0u;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-
-    // ---- last CTA: locate the digit that holds rank k_rem, counting from the top ----------
+    const uint32_t* hist = st->hist + kPass * kBins;
     // thread t owns bins top-down: bin(t, q) = kBins-1 - (4t + q), q = 0..3
     const uint32_t k_rem = st->k_rem;
     uint32_t c[4], own = 0;
@@ -111,7 +132,6 @@ select_pass_kernel(const float* __restrict__ grad, const float* __restrict__ res
         c[q] = __ldcg(&hist[kBins - 1 - (4 * threadIdx.x + q)]);
         own += c[q];
     }
-    // exclusive prefix (over threads, i.e. over higher bins) of `own`
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
     uint32_t incl = own;
 #pragma unroll
@@ -123,7 +143,6 @@ select_pass_kernel(const float* __restrict__ grad, const float* __restrict__ res
     __syncthreads();
     uint32_t above = incl - own;
     for (uint32_t v = 0; v < warp; ++v) above += s_scan[v];
-    // `above` = elements in bins higher than this thread's first bin
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         if (above < k_rem && k_rem <= above + c[q]) {
@@ -134,32 +153,184 @@ select_pass_kernel(const float* __restrict__ grad, const float* __restrict__ res
             const uint64_t n_gt = st->n_gt + above;
             st->n_gt = n_gt;
             if (kPass == kPasses - 1) {
-                *tau_out = __uint_as_float(new_prefix);
-                result->status = DCT_OK;
-                result->reserved = 0;
-                result->count = 0;
-                result->needed = 0;
-                result->n_gt = n_gt;
-                result->n_eq = c[q];
+                st->key_out = new_prefix;
+                if (tau_out) {           // this select produces the call's answer
+                    *tau_out = __uint_as_float(new_prefix);
+                    result->n_gt = n_gt;
+                    result->n_eq = c[q];
+                }
             }
         }
         above += c[q];
     }
 }
 
-template <int kPass>
-cudaError_t launch_pass(int grid, cudaStream_t stream, bool has_res, bool vec, const float* grad,
-                        const float* residual, uint32_t n, SelectState* st, uint32_t* hist, float* tau_out,
-                        dct_result_t* result) {
-#define DCT_SEL_LAUNCH(R, V) \
-    select_pass_kernel<kPass, R, V><<<grid, kSelThreads, 0, stream>>>(grad, residual, n, st, hist, tau_out, result)
-    if (has_res) {
-        if (vec) DCT_SEL_LAUNCH(true, true); else DCT_SEL_LAUNCH(true, false);
-    } else {
-        if (vec) DCT_SEL_LAUNCH(false, true); else DCT_SEL_LAUNCH(false, false);
+template <int kPass, typename Source, bool kVectorised>
+__global__ void __launch_bounds__(kSelThreads)
+select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct_result_t* __restrict__ result) {
+    if (!st->enabled) return;
+    constexpr int shift = pass_shift(kPass);
+    constexpr int bits = pass_bits(kPass);
+    constexpr uint32_t digit_mask = (1u << bits) - 1u;
+    __shared__ uint32_t sh[kBins];
+    __shared__ uint32_t s_scan[kSelThreads / 32];
+    __shared__ uint32_t s_last;
+
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) sh[b] = 0;
+    const uint32_t prefix = kPass == 0 ? 0u : st->prefix;   // written by the previous launch
+    const uint32_t n = st->n;
+    __syncthreads();
+
+    auto consume = [&](uint32_t key) {
+        if (kPass == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&sh[(key >> shift) & digit_mask], 1u);
+    };
+
+    const uint32_t num_chunks = (n + kSelChunk - 1) / kSelChunk;
+    for (uint32_t chunk = blockIdx.x; chunk < num_chunks; chunk += gridDim.x) {
+        const uint32_t base = chunk * kSelChunk;
+        bool done = false;
+        if constexpr (kVectorised) {      // VectorSource with 16-byte aligned pointers
+            if (base + kSelChunk <= n) {
+                float4 g4[kSelVecs], e4[kSelVecs];
+#pragma unroll
+                for (int j = 0; j < kSelVecs; ++j) {
+                    const uint32_t off = base + (j * kSelThreads + threadIdx.x) * 4;
+                    g4[j] = ld_readonly_f4(src.grad + off);
+                    e4[j] = src.residual ? ld_readonly_f4(src.residual + off) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                const bool add = src.residual != nullptr;
+#pragma unroll
+                for (int j = 0; j < kSelVecs; ++j) {
+                    consume(key_f32(add ? __fadd_rn(g4[j].x, e4[j].x) : g4[j].x));
+                    consume(key_f32(add ? __fadd_rn(g4[j].y, e4[j].y) : g4[j].y));
+                    consume(key_f32(add ? __fadd_rn(g4[j].z, e4[j].z) : g4[j].z));
+                    consume(key_f32(add ? __fadd_rn(g4[j].w, e4[j].w) : g4[j].w));
+                }
+                done = true;
+            }
+        }
+        if (!done)
+            for (uint32_t i = base + threadIdx.x; i < n && i < base + kSelChunk; i += kSelThreads)
+                consume(key_at(src, i));
     }
-#undef DCT_SEL_LAUNCH
+    __syncthreads();
+
+    uint32_t* hist = st->hist + kPass * kBins;
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) {
+        const uint32_t c = sh[b];
+        if (c) atomicAdd(&hist[b], c);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(&st->done[kPass], 1u) == gridDim.x - 1) ? 1u : 0u;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    finish_pass<kPass>(st, prefix, s_scan, tau_out, result);
+}
+
+// The single streaming pass of the sampled path: every key >= key(lo) goes to the candidate buffer.
+template <bool kVectorised>
+__global__ void __launch_bounds__(kSelThreads)
+select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t* __restrict__ cand_keys) {
+    if (!ws->sample.enabled) return;
+    const uint32_t lo = ws->sample.key_out;
+    const uint32_t capacity = ws->cand_capacity;
+    // Each warp collects its survivors in a small shared-memory buffer and moves them to the candidate
+    // buffer 64 or more at a time, so the global counter sees one atomic per flush, not one per survivor.
+    constexpr uint32_t kWarpBuf = 96, kFlushAt = 64;
+    __shared__ uint32_t s_buf[kSelThreads / 32][kWarpBuf];
+    uint32_t* wbuf = s_buf[threadIdx.x >> 5];
+    uint32_t held = 0;                              // warp-uniform
+    auto flush = [&]() {
+        __syncwarp();
+        uint32_t base = 0;
+        if (lane_id() == 0) base = atomicAdd(&ws->cand_count, held);
+        base = __shfl_sync(0xFFFFFFFFu, base, 0);
+        for (uint32_t i = lane_id(); i < held; i += 32)
+            if (base + i < capacity) cand_keys[base + i] = wbuf[i];
+        __syncwarp();
+        held = 0;
+    };
+    auto keep = [&](bool pred, uint32_t key) {      // called by whole warps
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, pred);
+        if (bal == 0) return;
+        if (pred) wbuf[held + __popc(bal & lanemask_lt())] = key;
+        held += __popc(bal);
+        if (held >= kFlushAt) flush();
+    };
+    const uint32_t num_chunks = (n + kSelChunk - 1) / kSelChunk;
+    for (uint32_t chunk = blockIdx.x; chunk < num_chunks; chunk += gridDim.x) {
+        const uint32_t base = chunk * kSelChunk;
+        if (kVectorised && base + kSelChunk <= n) {
+            float4 g4[kSelVecs], e4[kSelVecs];
+#pragma unroll
+            for (int j = 0; j < kSelVecs; ++j) {
+                const uint32_t off = base + (j * kSelThreads + threadIdx.x) * 4;
+                g4[j] = ld_readonly_f4(src.grad + off);
+                e4[j] = src.residual ? ld_readonly_f4(src.residual + off) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            const bool add = src.residual != nullptr;
+#pragma unroll
+            for (int j = 0; j < kSelVecs; ++j) {
+                const uint32_t k0 = key_f32(add ? __fadd_rn(g4[j].x, e4[j].x) : g4[j].x);
+                const uint32_t k1 = key_f32(add ? __fadd_rn(g4[j].y, e4[j].y) : g4[j].y);
+                const uint32_t k2 = key_f32(add ? __fadd_rn(g4[j].z, e4[j].z) : g4[j].z);
+                const uint32_t k3 = key_f32(add ? __fadd_rn(g4[j].w, e4[j].w) : g4[j].w);
+                const uint32_t top = max(max(k0, k1), max(k2, k3));
+                if (__any_sync(0xFFFFFFFFu, top >= lo)) {
+                    keep(k0 >= lo, k0);
+                    keep(k1 >= lo, k1);
+                    keep(k2 >= lo, k2);
+                    keep(k3 >= lo, k3);
+                }
+            }
+        } else {
+            // whole warps stay together so that the ballots above see every lane
+            for (uint32_t i0 = base + (threadIdx.x & ~31u); i0 < n && i0 < base + kSelChunk; i0 += kSelThreads) {
+                const uint32_t i = i0 + lane_id();
+                const bool in = i < n && i < base + kSelChunk;
+                const uint32_t key = in ? key_at(src, i) : 0u;
+                keep(in && key >= lo, key);
+            }
+        }
+    }
+    if (held) flush();
+}
+
+// After the filter: decide which select produces the answer.
+__global__ void select_decide_kernel(SelectWorkspace* ws, uint32_t k) {
+    if (!ws->sample.enabled) return;
+    const uint32_t c = ws->cand_count;
+    if (c >= k && c <= ws->cand_capacity) {
+        ws->cand.n = c;
+        ws->cand.enabled = 1;
+    } else {
+        ws->full.enabled = 1;      // the sample misjudged the vector: do it the plain way
+    }
+}
+
+template <typename Source, bool kVectorised>
+cudaError_t launch_three_passes(int grid, cudaStream_t stream, Source src, SelectState* st, float* tau_out,
+                                dct_result_t* result) {
+    select_pass_kernel<0, Source, kVectorised><<<grid, kSelThreads, 0, stream>>>(src, st, tau_out, result);
+    select_pass_kernel<1, Source, kVectorised><<<grid, kSelThreads, 0, stream>>>(src, st, tau_out, result);
+    select_pass_kernel<2, Source, kVectorised><<<grid, kSelThreads, 0, stream>>>(src, st, tau_out, result);
     return cudaGetLastError();
+}
+
+// Rank to select in the sample so that the number of vector elements at or above the sampled value is,
+// six standard deviations out, still at least k: returns 0 if that would overflow the candidate buffer.
+uint32_t sample_rank(uint64_t n, uint64_t k, uint32_t sample_n, uint32_t capacity) {
+    const double m = static_cast<double>(k) * sample_n / static_cast<double>(n);   // expected sample rank of tau
+    const double r = m + 6.0 * __builtin_sqrt(m + 1.0) + 20.0;
+    const double expected_max = (r + 6.0 * __builtin_sqrt(r)) * static_cast<double>(n) / sample_n;
+    if (r >= sample_n / 4.0 || expected_max > capacity) return 0;
+    return static_cast<uint32_t>(r);
+}
+
+uint32_t candidate_capacity(uint64_t n) {
+    return static_cast<uint32_t>(n < kMaxCandidates ? n : kMaxCandidates);
 }
 
 }  // namespace
@@ -169,7 +340,9 @@ using namespace dct;
 
 extern "C" size_t dct_threshold_select_workspace_bytes(uint64_t n) {
     if (n == 0 || n > 0x7FFFFFFFull) return 0;
-    return kSelStateBytes + sizeof(uint32_t) * kPasses * kBins;
+    size_t bytes = sizeof(SelectWorkspace);
+    if (n >= kMinSampledN) bytes += sizeof(uint32_t) * static_cast<size_t>(candidate_capacity(n));
+    return (bytes + 255) & ~static_cast<size_t>(255);
 }
 
 extern "C" dct_status_t dct_threshold_select(const float* grad, const float* residual, uint64_t n, uint64_t k,
@@ -183,19 +356,49 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
         return DCT_ERR_WORKSPACE;
 
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    auto* st = static_cast<SelectState*>(workspace);
-    auto* hist = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + kSelStateBytes);
-    const uint32_t n32 = static_cast<uint32_t>(n);
-    const uint32_t num_chunks = (n32 + kSelChunk - 1) / kSelChunk;
+    auto* ws = static_cast<SelectWorkspace*>(workspace);
+    auto* cand_keys = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + sizeof(SelectWorkspace));
+    const uint32_t n32 = static_cast<uint32_t>(n), k32 = static_cast<uint32_t>(k);
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
-    const int grid = static_cast<int>(num_chunks < static_cast<uint32_t>(sms * 4) ? num_chunks : sms * 4);
+    auto grid_for = [&](uint64_t elems) {
+        const uint64_t chunks = (elems + kSelChunk - 1) / kSelChunk;
+        return static_cast<int>(chunks < static_cast<uint64_t>(sms) * 4 ? (chunks ? chunks : 1) : sms * 4);
+    };
     const bool vec = aligned_to(grad, 16) && (!residual || aligned_to(residual, 16));
+    const VectorSource vsrc{grad, residual};
 
-    select_init_kernel<<<(kPasses * kBins + 1023) / 1024, 1024, 0, stream>>>(st, hist, static_cast<uint32_t>(k));
+    // sampled single-pass path?
+    uint32_t sample_n = 0, sample_k = 0, stride = 0, capacity = 0;
+    if (n >= kMinSampledN) {
+        capacity = candidate_capacity(n);
+        stride = n32 / kSampleSize;
+        sample_n = kSampleSize;
+        sample_k = sample_rank(n, k, sample_n, capacity);
+        if (sample_k == 0) sample_n = 0;
+    }
+
+    select_init_kernel<<<1, kInitThreads, 0, stream>>>(ws, n32, k32, sample_n, sample_k, capacity, result);
     DCT_CUDA_TRY(cudaGetLastError());
-    DCT_CUDA_TRY(launch_pass<0>(grid, stream, residual != nullptr, vec, grad, residual, n32, st, hist, tau_out, result));
-    DCT_CUDA_TRY(launch_pass<1>(grid, stream, residual != nullptr, vec, grad, residual, n32, st, hist, tau_out, result));
-    DCT_CUDA_TRY(launch_pass<2>(grid, stream, residual != nullptr, vec, grad, residual, n32, st, hist, tau_out, result));
+    if (sample_n) {
+        const StridedSource ssrc{grad, residual, stride};
+        DCT_CUDA_TRY((launch_three_passes<StridedSource, false>(grid_for(sample_n), stream, ssrc, &ws->sample, nullptr,
+                                                                result)));
+        if (vec)
+            select_filter_kernel<true><<<grid_for(n), kSelThreads, 0, stream>>>(vsrc, n32, ws, cand_keys);
+        else
+            select_filter_kernel<false><<<grid_for(n), kSelThreads, 0, stream>>>(vsrc, n32, ws, cand_keys);
+        DCT_CUDA_TRY(cudaGetLastError());
+        select_decide_kernel<<<1, 1, 0, stream>>>(ws, k32);
+        DCT_CUDA_TRY(cudaGetLastError());
+        const KeySource ksrc{cand_keys};
+        // the candidate count is only known on the device: a fixed modest grid walks whatever is there
+        DCT_CUDA_TRY((launch_three_passes<KeySource, false>(128, stream, ksrc, &ws->cand, tau_out, result)));
+    }
+    // the plain three passes: the only path for small or dense problems, the fall-back otherwise
+    if (vec)
+        DCT_CUDA_TRY((launch_three_passes<VectorSource, true>(grid_for(n), stream, vsrc, &ws->full, tau_out, result)));
+    else
+        DCT_CUDA_TRY((launch_three_passes<VectorSource, false>(grid_for(n), stream, vsrc, &ws->full, tau_out, result)));
     return DCT_OK;
 }
