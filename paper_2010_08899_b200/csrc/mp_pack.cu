@@ -241,13 +241,11 @@ template <int E8> struct WarpRowLayout {
     // Lane l reads its 16-byte units in the rotated order (c + l) mod E8: with spans of 256 bytes the
     // eight lanes of a quarter-warp then hit eight different bank groups instead of one.
     static constexpr bool kRotate = (E8 == 16);
-    // list capacity (a multiple of 256): room for twice the usual ~1.2 k candidates when the leaf bound
-    // exists (k <= number of leaves); the whole row otherwise
-    __host__ __device__ static constexpr uint32_t list_cap(uint32_t k) {
-        return k > 32u * E8 ? D : (((2u * k + 255u) & ~255u) < D ? ((2u * k + 255u) & ~255u) : D);
-    }
+    static constexpr uint32_t kMaskWords = (E8 + 3) / 4;     // 32-bit mask words per lane
+    static constexpr uint32_t kTableWords = 32u * kMaskWords;
+    // per warp: row | candidate-mask table | running-count table | histogram | k output slots | mbarrier
     __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) {
-        return kRowBytes + list_cap(k) * 4u + kHistWords * 4u + 16u;
+        return kRowBytes + 2u * kTableWords * 4u + kHistWords * 4u + ((k + 3u) & ~3u) * 4u + 16u;
     }
 };
 
@@ -331,6 +329,66 @@ __device__ __forceinline__ uint32_t pick_mantissa(const uint32_t* hist, uint32_t
     return __shfl_sync(0xFFFFFFFFu, found, src) & 0x7Fu;
 }
 
+// General slow path for one row (rare): no usable bound, or very many elements tie at it.  tau_i is found
+// bit by bit on the row itself, most significant first (the largest v with #{key >= v} >= k); then
+// everything above tau_i and the first ties are written, in column order, straight from the row.
+// Kept out of line so that the common path stays small in the instruction cache.
+template <int E8>
+__device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_t k, size_t out_base, uint32_t row,
+                                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
+                                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out) {
+    constexpr uint32_t E = E8 * 8u;
+    constexpr int kMaskWords = (E8 + 3) / 4;
+    const uint32_t lane = lane_id();
+    uint32_t tau_key = 0;
+#pragma unroll 1
+    for (int bit = 14; bit >= 0; --bit) {
+        const uint32_t trial = tau_key | (1u << bit);
+        uint32_t cnt = 0;
+#pragma unroll 4
+        for (int c = 0; c < E8; ++c)
+            cnt += __popc(mask8_ge_exact(*reinterpret_cast<const uint4*>(span + c * 16), trial));
+        if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= k) tau_key = trial;
+    }
+    uint32_t gt_masks[kMaskWords], eq_masks[kMaskWords];
+    uint32_t n_gt_mine = 0, n_eq_mine = 0;
+#pragma unroll
+    for (int i = 0; i < kMaskWords; ++i) gt_masks[i] = eq_masks[i] = 0;
+#pragma unroll
+    for (int c = 0; c < E8; ++c) {
+        const uint4 v = *reinterpret_cast<const uint4*>(span + c * 16);
+        const uint32_t gt = mask8_ge_exact(v, tau_key + 1u);
+        const uint32_t eq = mask8_ge_exact(v, tau_key) & ~gt;
+        gt_masks[c / 4] |= gt << (8 * (c % 4));
+        eq_masks[c / 4] |= eq << (8 * (c % 4));
+        n_gt_mine += __popc(gt);
+        n_eq_mine += __popc(eq);
+    }
+    const uint32_t incl = warp_inclusive_sum(n_gt_mine);
+    const uint32_t take = k - __shfl_sync(0xFFFFFFFFu, incl, 31);   // ties to keep, lowest columns first
+    uint32_t g_at = incl - n_gt_mine;
+    uint32_t e_at = warp_inclusive_sum(n_eq_mine) - n_eq_mine;
+#pragma unroll
+    for (int wd = 0; wd < kMaskWords; ++wd) {
+        uint32_t m = gt_masks[wd] | eq_masks[wd];
+        while (m) {
+            const uint32_t bit = __ffs(m) - 1;
+            m &= m - 1;
+            const bool is_eq = (eq_masks[wd] >> bit) & 1u;
+            if (!is_eq || e_at < take) {
+                const uint32_t j = wd * 32 + bit;
+                const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
+                cols_out[pos] = static_cast<int16_t>(lane * E + j);
+                vals_out[pos] = *reinterpret_cast<const uint16_t*>(span + j * 2);
+                if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
+            }
+            g_at += is_eq ? 0u : 1u;
+            e_at += is_eq ? 1u : 0u;
+        }
+    }
+    if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+}
+
 template <int E8>
 __global__ void __launch_bounds__(kFwdMaxWarps * 32)
 mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
@@ -339,15 +397,18 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                              dct_result_t* __restrict__ result) {
     using Lay = WarpRowLayout<E8>;
     constexpr uint32_t E = Lay::E;
-    constexpr int kMaskWords = (E8 + 3) / 4;
+    constexpr int kMaskWords = Lay::kMaskWords;
+    constexpr uint32_t kPerLane = 10, kRound = 32u * kPerLane;   // candidates a lane holds in registers at a time
+    constexpr uint32_t kGuessMargin = 32;                         // keys (a quarter of a binade) below the previous tau_i
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
-    const uint32_t cap = Lay::list_cap(k);
     unsigned char* base = smem_raw + warp * Lay::warp_bytes(k);
     unsigned char* span = base + lane * Lay::kSpanBytes;
-    uint32_t* list = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
-    uint32_t* hist = list + cap;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(hist + kHistWords);
+    uint32_t* mask_tab = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);   // candidate masks, column order
+    uint32_t* count_tab = mask_tab + Lay::kTableWords;                         // candidates before each mask word
+    uint32_t* hist = count_tab + Lay::kTableWords;
+    uint32_t* stage = hist + kHistWords;                                       // the k kept entries, column order
+    uint64_t* bar = reinterpret_cast<uint64_t*>(stage + ((k + 3u) & ~3u));
     __shared__ uint32_t s_stop;
 
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
@@ -384,6 +445,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     if (warp_global < rows) request_row(warp_global);
 
     uint32_t use = 0;
+    uint32_t guess_low = 0;                         // bound guessed from the previous row (0: none)
     for (uint32_t row = warp_global; row < rows; row += total_warps, ++use) {
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
             s_stop = 1;
@@ -392,27 +454,24 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         }
         const size_t out_base = static_cast<size_t>(row) * k;
 
-        // ---- A: leaf maxima, then their k-th largest as the lower bound ---------------------------
-        uint32_t leaf[E8];
-        uint32_t row_max = 0;
+        // ---- A: a lower bound for tau_i --------------------------------------------------------------
+        uint32_t row_max = 0x7FFFu;                  // only the exact bound computes the true maximum
+        const bool have_bound = k <= 32u * E8;       // otherwise there are fewer leaves than k
+        auto exact_bound = [&]() -> uint32_t {
+            // maxima of the aligned 8-element leaves
+            uint32_t leaf[E8];
+            uint32_t top = 0;
 #pragma unroll
-        for (int c = 0; c < E8; ++c) {
-            const uint4 v = *reinterpret_cast<const uint4*>(span + unit_of(c) * 16);
-            const __nv_bfloat162 m2 = __hmax2(__hmax2(__habs2(as_bf162(v.x)), __habs2(as_bf162(v.y))),
-                                              __hmax2(__habs2(as_bf162(v.z)), __habs2(as_bf162(v.w))));
-            const uint32_t m = as_u32(m2);
-            leaf[c] = max(m & 0xFFFFu, m >> 16);
-            row_max = max(row_max, leaf[c]);
-        }
-        row_max = __reduce_max_sync(0xFFFFFFFFu, row_max);
-#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 0
-        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(row_max + leaf[3]);
-        release_row(row);
-        continue;
-#endif
-        uint32_t low = 0;
-        const bool have_bound = k <= 32u * E8;   // otherwise there are fewer leaves than k: everything is a candidate
-        if (have_bound) {
+            for (int c = 0; c < E8; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4*>(span + unit_of(c) * 16);
+                const __nv_bfloat162 m2 = __hmax2(__hmax2(__habs2(as_bf162(v.x)), __habs2(as_bf162(v.y))),
+                                                  __hmax2(__habs2(as_bf162(v.z)), __habs2(as_bf162(v.w))));
+                const uint32_t m = as_u32(m2);
+                leaf[c] = max(m & 0xFFFFu, m >> 16);
+                top = max(top, leaf[c]);
+            }
+            row_max = __reduce_max_sync(0xFFFFFFFFu, top);
+            if (!have_bound) return 0u;
             // One histogram pass over the leaf maxima in bins of 8 keys counted down from the row maximum
             // (bin 255 collects everything further away).  The bound is the lowest key of the bin in which
             // the count reaches k: at least k leaves, hence k elements, lie at or above it.
@@ -437,28 +496,22 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 }
                 need -= __shfl_sync(0xFFFFFFFFu, inc, 31);
             }
-            const uint32_t span_keys = bin * 8u + 7u;
-            low = (bin < 255u && row_max > span_keys) ? row_max - span_keys : 0u;
             __syncwarp();
-        }
+            const uint32_t span_keys = bin * 8u + 7u;
+            return (bin < 255u && row_max > span_keys) ? row_max - span_keys : 0u;
+        };
 
-#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 1
-        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(low);
-        release_row(row);
-        continue;
-#endif
-        // ---- B: ordered compaction of the candidates ---------------------------------------------
+        // ---- B: candidate masks (key >= low), in column order ------------------------------------------
         uint32_t masks[kMaskWords];
+        uint32_t n_mine = 0, incl = 0, n_cand = 0;
+        auto build_masks = [&](uint32_t bound) {
 #pragma unroll
-        for (int i = 0; i < kMaskWords; ++i) masks[i] = 0;
-        uint32_t n_mine = 0;
-        {
-            const __nv_bfloat162 low2 = as_bf162(low | (low << 16));
+            for (int i = 0; i < kMaskWords; ++i) masks[i] = 0;
+            const __nv_bfloat162 low2 = as_bf162(bound | (bound << 16));
 #pragma unroll
             for (int c = 0; c < E8; ++c) {
                 const uint32_t m = mask8_ge_filter(*reinterpret_cast<const uint4*>(span + unit_of(c) * 16), low2);
                 masks[c / 4] |= m << (8 * (c % 4));
-                n_mine += __popc(m);
             }
             if (Lay::kRotate) {
                 // byte c of the 128-bit mask belongs to unit (c + lane) mod 16: rotate left by 8 * (lane mod 16)
@@ -472,123 +525,96 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 masks[2 % kMaskWords] = __funnelshift_l(w1, w2, bits);
                 masks[3 % kMaskWords] = __funnelshift_l(w2, w3, bits);
             }
+            n_mine = 0;
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) n_mine += __popc(masks[i]);
+            incl = warp_inclusive_sum(n_mine);
+            n_cand = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        };
+
+        // Thresholds of neighbouring samples are close (the observation behind the paper's threshold
+        // life-span, applied across rows): first try the previous row's tau_i minus a margin as the bound.
+        // It is only a guess -- it is accepted if it leaves at least k and not too many candidates, and the
+        // exact leaf bound takes over otherwise -- so the result never depends on it.
+        uint32_t low = 0;
+        bool use_guess = have_bound && guess_low != 0;
+#pragma unroll 1
+        while (true) {
+            low = use_guess ? guess_low : exact_bound();
+            build_masks(low);
+            if (!use_guess || (n_cand >= k && n_cand <= kRound)) break;
+            use_guess = false;
         }
-        uint32_t incl = warp_inclusive_sum(n_mine);
-        uint32_t n_cand = __shfl_sync(0xFFFFFFFFu, incl, 31);
 #if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 2
         if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(n_cand);
         release_row(row);
         continue;
 #endif
-        if (n_cand > cap) {
-            // Rare: the candidates do not fit the list (heavy ties at the bound, or no usable bound).
-            // General slow path on the row itself: tau_i bit by bit, most significant first (the largest v
-            // with #{key >= v} >= k), then everything above tau_i and the first ties, in column order.
-            uint32_t tau_key = 0;
-#pragma unroll 1
-            for (int bit = 14; bit >= 0; --bit) {
-                const uint32_t trial = tau_key | (1u << bit);
-                uint32_t cnt = 0;
-#pragma unroll
-                for (int c = 0; c < E8; ++c)
-                    cnt += __popc(mask8_ge_exact(*reinterpret_cast<const uint4*>(span + c * 16), trial));
-                if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= k) tau_key = trial;
-            }
-            uint32_t eq_masks[kMaskWords];
-            n_mine = 0;
-            uint32_t n_eq_mine = 0;
-#pragma unroll
-            for (int i = 0; i < kMaskWords; ++i) masks[i] = eq_masks[i] = 0;
-#pragma unroll
-            for (int c = 0; c < E8; ++c) {
-                const uint4 v = *reinterpret_cast<const uint4*>(span + c * 16);
-                const uint32_t gt = mask8_ge_exact(v, tau_key + 1u);
-                const uint32_t eq = mask8_ge_exact(v, tau_key) & ~gt;
-                masks[c / 4] |= gt << (8 * (c % 4));
-                eq_masks[c / 4] |= eq << (8 * (c % 4));
-                n_mine += __popc(gt);
-                n_eq_mine += __popc(eq);
-            }
-            incl = warp_inclusive_sum(n_mine);
-            const uint32_t take = k - __shfl_sync(0xFFFFFFFFu, incl, 31);   // ties to keep, lowest columns first
-            uint32_t g_at = incl - n_mine;
-            uint32_t e_at = warp_inclusive_sum(n_eq_mine) - n_eq_mine;
-#pragma unroll
-            for (int c = 0; c < E8; ++c) {
-                const uint32_t gm = (masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
-                const uint32_t em = (eq_masks[c / 4] >> (8 * (c % 4))) & 0xFFu;
-                uint32_t m = gm | em;
-                while (m) {
-                    const uint32_t bit = __ffs(m) - 1;
-                    m &= m - 1;
-                    const bool is_eq = (em >> bit) & 1u;
-                    if (!is_eq || e_at < take) {
-                        const uint32_t j = c * 8 + bit;
-                        const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
-                        cols_out[pos] = static_cast<int16_t>(lane * E + j);
-                        vals_out[pos] = *reinterpret_cast<const uint16_t*>(span + j * 2);
-                        if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
-                    }
-                    g_at += is_eq ? 0u : 1u;
-                    e_at += is_eq ? 1u : 0u;
-                }
-            }
-            if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+        if (!have_bound || n_cand > kRound) {
+            mp_row_slow_path<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
             release_row(row);
             continue;
         }
+
+        // ---- candidates into registers, evenly: lane q takes candidates kPerLane q .. kPerLane q + kPerLane - 1 ----
+        // The masks go to a table in column order together with the number of candidates before each mask
+        // word; a lane finds the word that holds its first candidate by bisection and walks on from there.
         {
-            uint32_t at = incl - n_mine;
-            const uint32_t col0 = (lane * E) << 16;
+            uint32_t before = incl - n_mine;
 #pragma unroll
-            for (int wd = 0; wd < kMaskWords; ++wd) {     // bit b of word wd is element 32 wd + b of the lane's span
-                uint32_t m = masks[wd];
-                while (m) {
-                    const uint32_t j = wd * 32 + (__ffs(m) - 1);
+            for (int i = 0; i < kMaskWords; ++i) {
+                mask_tab[lane * kMaskWords + i] = masks[i];
+                count_tab[lane * kMaskWords + i] = before;
+                before += __popc(masks[i]);
+            }
+        }
+        __syncwarp();
+        uint32_t ent[kPerLane];
+        const uint32_t first = lane * kPerLane;                 // rank of the lane's first candidate
+        const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < kPerLane ? n_cand - first : kPerLane);
+        {
+            uint32_t word = 0, m = 0;
+            if (nvalid) {
+                uint32_t lo = 0, hi = Lay::kTableWords - 1;         // largest word with count_tab[word] <= first
+                while (lo < hi) {
+                    const uint32_t mid = (lo + hi + 1) >> 1;
+                    if (count_tab[mid] <= first) lo = mid; else hi = mid - 1;
+                }
+                word = lo;
+                m = mask_tab[word];
+                for (uint32_t skip = first - count_tab[word]; skip; --skip) m &= m - 1;
+            }
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
+                ent[i] = 0;
+                if (static_cast<uint32_t>(i) < nvalid) {
+                    while (m == 0) m = mask_tab[++word];
+                    const uint32_t col = (word / kMaskWords) * E + (word % kMaskWords) * 32u + (__ffs(m) - 1);
                     m &= m - 1;
-                    const uint32_t raw = *reinterpret_cast<const uint16_t*>(span + j * 2);
-                    list[at++] = (raw | col0) + (j << 16);
+                    ent[i] = reinterpret_cast<const uint16_t*>(base)[col] | (col << 16);
                 }
             }
         }
         release_row(row);
 #if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 3
-        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(list[0]);
+        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(ent[0]);
         continue;
 #endif
 
         // ---- C: k-th largest of the candidates --------------------------------------------------
-        // The list is consumed in rounds of 256 entries, 8 consecutive entries per lane (two 128-bit
-        // reads); with the usual ~1.2 k candidates there is one round and the entries stay in registers
-        // from the first histogram to the final write.
-        uint32_t ent[8];
-        auto load_round = [&](uint32_t q0) -> uint32_t {      // returns how many of the lane's 8 entries exist
-            const uint32_t first = q0 + lane * 8u;
-            const uint4 a = *reinterpret_cast<const uint4*>(list + first);
-            const uint4 b = *reinterpret_cast<const uint4*>(list + first + 4);
-            ent[0] = a.x; ent[1] = a.y; ent[2] = a.z; ent[3] = a.w;
-            ent[4] = b.x; ent[5] = b.y; ent[6] = b.z; ent[7] = b.w;
-            return first >= n_cand ? 0u : (n_cand - first < 8u ? n_cand - first : 8u);
-        };
-        const bool one_round = n_cand <= 256u;
-        __syncwarp();
-        uint32_t nvalid = load_round(0);
         uint32_t tau_key = 0, take = 0;
         bool found = false;
-        if (have_bound && low != 0) {
+        if (low != 0) {
             // tau_i is the (n_cand - k + 1)-th smallest candidate.  Usually it lies within 64 keys of the
             // bound: a 64-bin histogram of the candidates in [low, low + 64), walked from the bottom, finds it.
             const uint32_t drop = n_cand - k;                 // candidates to discard, smallest first
             hist[lane] = 0;
             hist[lane + 32] = 0;
             __syncwarp();
-            for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
-                if (q0) nvalid = load_round(q0);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const uint32_t rel = (ent[i] & 0x7FFFu) - low;
-                    if (static_cast<uint32_t>(i) < nvalid && rel < 64u) atomicAdd(&hist[rel], 1u);
-                }
+            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
+                const uint32_t rel = (ent[i] & 0x7FFFu) - low;
+                if (static_cast<uint32_t>(i) < nvalid && rel < 64u) atomicAdd(&hist[rel], 1u);
             }
             __syncwarp();
             const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
@@ -610,7 +636,6 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 found = true;
             }
             __syncwarp();
-            if (!found && !one_round) nvalid = load_round(0);
         }
         if (!found) {
             // general case: radix select over the candidates, exponent byte then mantissa
@@ -618,64 +643,53 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
             reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
             __syncwarp();
-            for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
-                if (q0) nvalid = load_round(q0);
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent[i] & 0x7FFFu) >> 7], 1u);
-            }
+            for (int i = 0; i < static_cast<int>(kPerLane); ++i)
+                if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent[i] & 0x7FFFu) >> 7], 1u);
             __syncwarp();
             const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
             __syncwarp();
             reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
             __syncwarp();
-            for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
-                if (!one_round) nvalid = load_round(q0);
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const uint32_t key = ent[i] & 0x7FFFu;
-                    if (static_cast<uint32_t>(i) < nvalid && (key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
-                }
+            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
+                const uint32_t key = ent[i] & 0x7FFFu;
+                if (static_cast<uint32_t>(i) < nvalid && (key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
             }
             __syncwarp();
             tau_key = (exp_bin << 7) | pick_mantissa(hist, k_rem, take);
         }
         if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+        guess_low = tau_key > kGuessMargin ? tau_key - kGuessMargin : 0u;
 #if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 4
         continue;
 #endif
 
         // ---- D: ordered emit ------------------------------------------------------------------------
-        // The kept entries are first compacted in place at the front of the list (a kept entry never moves
-        // to a higher position), then the k entries leave with coalesced stores.
-        uint32_t g_run = 0, e_run = 0;
-        for (uint32_t q0 = 0; q0 < n_cand; q0 += 256) {
-            if (!one_round) nvalid = load_round(q0);
+        // The kept entries are placed, in column order, into k staging slots; then they leave with
+        // coalesced stores.
+        {
             uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
                 const uint32_t key = ent[i] & 0x7FFFu;
                 if (static_cast<uint32_t>(i) < nvalid) counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
             }
-            const uint32_t inc = warp_inclusive_sum(counts);
-            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, inc, 31);
-            uint32_t g_at = g_run + ((inc - counts) >> 16), e_at = e_run + ((inc - counts) & 0xFFFFu);
-            __syncwarp();                                     // every lane holds its entries in registers
+            const uint32_t before = warp_inclusive_sum(counts) - counts;
+            uint32_t g_at = before >> 16, e_at = before & 0xFFFFu;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
+            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
                 const uint32_t key = ent[i] & 0x7FFFu;
                 const bool live = static_cast<uint32_t>(i) < nvalid;
                 const bool is_gt = live && key > tau_key, is_eq = live && key == tau_key;
-                if (is_gt || (is_eq && e_at < take)) list[g_at + (e_at < take ? e_at : take)] = ent[i];
+                if (is_gt || (is_eq && e_at < take)) stage[g_at + (e_at < take ? e_at : take)] = ent[i];
                 g_at += is_gt ? 1u : 0u;
                 e_at += is_eq ? 1u : 0u;
             }
-            g_run += tot >> 16;
-            e_run += tot & 0xFFFFu;
         }
         __syncwarp();
         for (uint32_t p = lane; p < k; p += 32) {
-            const uint32_t e = list[p];
+            const uint32_t e = stage[p];
             cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
             vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
             if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
@@ -696,7 +710,7 @@ dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t ld,
     DCT_CUDA_TRY(cudaGetDevice(&dev));
     if (configured_device != dev) {
         DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(kSmemBudget)));
+                                          static_cast<int>(kSmemBudget)));   // sized per launch below
         configured_device = dev;
     }
     const size_t per_warp = Lay::warp_bytes(k);
@@ -787,7 +801,9 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (dtype == DCT_F32)
         return launch_fwd<float>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0) {
+    // The warp-per-row kernel holds up to 320 candidates in registers and needs the leaf bound (k <= d/8):
+    // it serves k <= 256 (about 1.25 k candidates); larger k take the general kernel.
+    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && k <= 256 && k <= d / 8) {
         switch (d) {   // warp-per-row path: d = 256 * 2^j
             case 256: return launch_fwd_bf16_warp<1>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             case 512: return launch_fwd_bf16_warp<2>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
