@@ -228,7 +228,7 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 // and a short list), the row takes a slow general path: tau_i is found bit by bit by counting over the
 // row, and the output is written straight from the row.
 #ifndef DCT_FWD_MAX_WARPS
-#define DCT_FWD_MAX_WARPS 20
+#define DCT_FWD_MAX_WARPS 24
 #endif
 constexpr int kFwdMaxWarps = DCT_FWD_MAX_WARPS;   // rows in flight per CTA (one CTA per SM; shared memory bounds it)
 constexpr uint32_t kAbsMask2 = 0x7FFF7FFFu;
@@ -243,9 +243,15 @@ template <int E8> struct WarpRowLayout {
     static constexpr bool kRotate = (E8 == 16);
     static constexpr uint32_t kMaskWords = (E8 + 3) / 4;     // 32-bit mask words per lane
     static constexpr uint32_t kTableWords = 32u * kMaskWords;
-    // per warp: row | candidate-mask table | running-count table | histogram | k output slots | mbarrier
+    // per warp: row | scratch | mbarrier.  The scratch is used in turn, never at the same time, as the
+    // leaf histogram, the candidate-mask and running-count tables, the select histogram and the k
+    // staging slots of the output.
+    __host__ __device__ static constexpr uint32_t scratch_words(uint32_t k) {
+        uint32_t w = 2u * kTableWords > kHistWords ? 2u * kTableWords : kHistWords;
+        return w > ((k + 3u) & ~3u) ? w : ((k + 3u) & ~3u);
+    }
     __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) {
-        return kRowBytes + 2u * kTableWords * 4u + kHistWords * 4u + ((k + 3u) & ~3u) * 4u + 16u;
+        return kRowBytes + scratch_words(k) * 4u + 16u;
     }
 };
 
@@ -404,11 +410,12 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
     unsigned char* base = smem_raw + warp * Lay::warp_bytes(k);
     unsigned char* span = base + lane * Lay::kSpanBytes;
-    uint32_t* mask_tab = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);   // candidate masks, column order
-    uint32_t* count_tab = mask_tab + Lay::kTableWords;                         // candidates before each mask word
-    uint32_t* hist = count_tab + Lay::kTableWords;
-    uint32_t* stage = hist + kHistWords;                                       // the k kept entries, column order
-    uint64_t* bar = reinterpret_cast<uint64_t*>(stage + ((k + 3u) & ~3u));
+    uint32_t* scratch = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
+    uint32_t* mask_tab = scratch;                             // candidate masks, column order
+    uint32_t* count_tab = scratch + Lay::kTableWords;         // candidates before each mask word
+    uint32_t* hist = scratch;                                 // histograms (before / after the tables are in use)
+    uint32_t* stage = scratch;                                // the k kept entries, column order (last use)
+    uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Lay::scratch_words(k));
     __shared__ uint32_t s_stop;
 
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
@@ -668,6 +675,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         // ---- D: ordered emit ------------------------------------------------------------------------
         // The kept entries are placed, in column order, into k staging slots; then they leave with
         // coalesced stores.
+        __syncwarp();                                         // the select histogram is dead: its words become the stage
         {
             uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
 #pragma unroll
