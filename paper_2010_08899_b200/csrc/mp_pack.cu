@@ -395,8 +395,15 @@ __device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_
     if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
 }
 
-template <int E8>
-__global__ void __launch_bounds__(kFwdMaxWarps * 32)
+// PL: candidates a lane holds in registers (10: k <= 224; 20: k <= 448, with 4-element leaves for the
+// exact bound, since 8-element leaves get loose as k approaches their number).
+template <int PL> struct FwdVariant {
+    static constexpr int kMaxWarps = PL <= 10 ? kFwdMaxWarps : 20;    // registers per thread grow with PL
+    static constexpr bool kFineLeaves = PL > 10;
+};
+
+template <int E8, int PL>
+__global__ void __launch_bounds__(FwdVariant<PL>::kMaxWarps * 32)
 mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
@@ -404,7 +411,9 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     using Lay = WarpRowLayout<E8>;
     constexpr uint32_t E = Lay::E;
     constexpr int kMaskWords = Lay::kMaskWords;
-    constexpr uint32_t kPerLane = 10, kRound = 32u * kPerLane;   // candidates a lane holds in registers at a time
+    constexpr uint32_t kPerLane = PL, kRound = 32u * kPerLane;   // candidates a lane holds in registers at a time
+    constexpr bool kFineLeaves = FwdVariant<PL>::kFineLeaves;
+    constexpr int kLeaves = kFineLeaves ? 2 * E8 : E8;           // leaves per lane (4 or 8 elements each)
     constexpr uint32_t kGuessMargin = 32;                         // keys (a quarter of a binade) below the previous tau_i
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
@@ -463,10 +472,11 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 
         // ---- A: a lower bound for tau_i --------------------------------------------------------------
         uint32_t row_max = 0x7FFFu;                  // only the exact bound computes the true maximum
-        const bool have_bound = k <= 32u * E8;       // otherwise there are fewer leaves than k
+        const bool have_bound = k <= 32u * kLeaves;  // otherwise there are fewer leaves than k
         auto exact_bound = [&]() -> uint32_t {
-            // maxima of the aligned 8-element leaves
-            uint32_t leaf[E8];
+            // maxima of the leaves: the 8 elements of a 16-byte unit, or (fine leaves) its even and its odd
+            // elements separately -- any partition of the row into at least k groups will do
+            uint32_t leaf[kLeaves];
             uint32_t top = 0;
 #pragma unroll
             for (int c = 0; c < E8; ++c) {
@@ -474,8 +484,14 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 const __nv_bfloat162 m2 = __hmax2(__hmax2(__habs2(as_bf162(v.x)), __habs2(as_bf162(v.y))),
                                                   __hmax2(__habs2(as_bf162(v.z)), __habs2(as_bf162(v.w))));
                 const uint32_t m = as_u32(m2);
-                leaf[c] = max(m & 0xFFFFu, m >> 16);
-                top = max(top, leaf[c]);
+                if (kFineLeaves) {
+                    leaf[2 * c] = m & 0xFFFFu;
+                    leaf[2 * c + 1] = m >> 16;
+                    top = max(top, max(leaf[2 * c], leaf[2 * c + 1]));
+                } else {
+                    leaf[c] = max(m & 0xFFFFu, m >> 16);
+                    top = max(top, leaf[c]);
+                }
             }
             row_max = __reduce_max_sync(0xFFFFFFFFu, top);
             if (!have_bound) return 0u;
@@ -486,7 +502,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
             __syncwarp();
 #pragma unroll
-            for (int c = 0; c < E8; ++c) {
+            for (int c = 0; c < kLeaves; ++c) {
                 const uint32_t rel = (row_max - leaf[c]) >> 3;
                 atomicAdd(&hist[rel < 255u ? rel : 255u], 1u);
             }
@@ -706,12 +722,13 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     }
 }
 
-template <int E8>
-dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
-                                  void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
-                                  cudaStream_t stream) {
+template <int E8, int PL>
+dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+                                          void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
+                                          cudaStream_t stream) {
     using Lay = WarpRowLayout<E8>;
-    auto kernel = mp_topk_fwd_bf16_warp_kernel<E8>;
+    auto kernel = mp_topk_fwd_bf16_warp_kernel<E8, PL>;
+    constexpr int kMaxWarps = FwdVariant<PL>::kMaxWarps;
     constexpr size_t kSmemBudget = 220 * 1024;            // of the 227 KiB a CTA may use
     static thread_local int configured_device = -1;
     int dev = 0;
@@ -723,7 +740,7 @@ dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t ld,
     }
     const size_t per_warp = Lay::warp_bytes(k);
     size_t warps = kSmemBudget / per_warp;                 // one CTA per SM with as many row slots as fit
-    if (warps > static_cast<size_t>(kFwdMaxWarps)) warps = kFwdMaxWarps;
+    if (warps > static_cast<size_t>(kMaxWarps)) warps = kMaxWarps;
     if (warps < 1) return DCT_ERR_UNSUPPORTED;
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
@@ -734,6 +751,19 @@ dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t ld,
         static_cast<uint16_t*>(tau_out), result);
     DCT_CUDA_TRY(cudaGetLastError());
     return DCT_OK;
+}
+
+// k <= 224: 10 candidates per lane (the exact bound leaves about 1.26 k candidates, 1.4 k at the 99th
+// percentile, which must fit 320); k <= 448: 20 per lane.
+template <int E8>
+dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+                                  void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
+                                  cudaStream_t stream) {
+    if (k <= 224)
+        return launch_fwd_bf16_warp_variant<E8, 10>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result,
+                                                    stream);
+    return launch_fwd_bf16_warp_variant<E8, 20>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result,
+                                                stream);
 }
 
 int fwd_threads_for(uint32_t d) {
@@ -809,9 +839,11 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (dtype == DCT_F32)
         return launch_fwd<float>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-    // The warp-per-row kernel holds up to 320 candidates in registers and needs the leaf bound (k <= d/8):
-    // it serves k <= 256 (about 1.25 k candidates); larger k take the general kernel.
-    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && k <= 256 && k <= d / 8) {
+    // The warp-per-row kernel holds up to 320 (k <= 224) or 640 (k <= 448) candidates in registers and needs
+    // the leaf bound (k <= d/8 with 8-element leaves, k <= d/4 with 4-element ones); larger k take the
+    // general kernel.
+    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 &&
+        ((k <= 224 && k <= d / 8) || (k > 224 && k <= 448 && k <= d / 4))) {
         switch (d) {   // warp-per-row path: d = 256 * 2^j
             case 256: return launch_fwd_bf16_warp<1>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             case 512: return launch_fwd_bf16_warp<2>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);

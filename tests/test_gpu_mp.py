@@ -124,3 +124,20 @@ def test_mp_host_buffer_entry_point():
     assert np.array_equal(cols_h.numpy().reshape(rows, k), want.cols)
     assert np.array_equal(G.as_np_bits(vals_h).reshape(rows, k), want.vals)
     assert np.array_equal(G.as_np_bits(gv_h).reshape(rows, k), oracle.mp_bwd(G.to_oracle(gx), want.cols))
+
+
+def test_mp_bf16_rows_with_wildly_different_scales():
+    """The warp-per-row kernel guesses each row's bound from the previous row's threshold; rows whose
+    scales jump by orders of magnitude make that guess useless in both directions (too few / far too
+    many candidates), which must only cost time, never change the result."""
+    # enough rows that every warp of the persistent grid meets several of them, and a scale pattern whose
+    # period (7) shares no factor with the number of warps, so consecutive rows of a warp differ in scale
+    rows, d, k = 9002, 4096, 205
+    x = inputs.mp_activations(rows, d, 77, dtype=torch.float32, device=G.DEV, col_scale_seed=78)
+    scale = torch.tensor([1.0, 300.0, 0.004, 17.0, 1e-3, 1e4, 1.0], device=G.DEV).repeat(rows // 7)
+    x = (x * scale[:, None]).to(torch.bfloat16).contiguous()
+    x[5] = 0                                    # a dead sample between live ones
+    x[6, ::7] = 2.0                             # heavy ties right after it
+    gx = inputs.mp_gradients(rows, d, 79, dtype=torch.bfloat16, device=G.DEV)
+    for kk in (k, 64, 256):
+        _compare_fwd_bwd(x, gx, d, kk)
