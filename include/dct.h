@@ -195,6 +195,43 @@ DCT_API dct_status_t dct_mp_pack_bwd(
     dct_result_t* result, dct_stream_t stream);
 
 /*
+ * dct_dp_decompress -- the receiving end of Algorithm 1's "Send W_hat": the sparse compressed gradient
+ * goes back into a dense vector (the paper counts this decompression in the overhead of the scheme,
+ * Sec. 2, without prescribing a procedure).
+ *
+ *   idx, val  [capacity] the packed gradient written by dct_dp_compress (ascending, distinct indices).
+ *   packed    the device result block of that dct_dp_compress call; packed->count entries are used
+ *             (at most `capacity`), so no host round trip is needed between the two calls.
+ *   dense     [n] fp32.  accumulate == 0: dense becomes W_hat (zero everywhere else; the call clears
+ *             it).  accumulate != 0: dense[idx[j]] += val[j], for a server that sums the messages
+ *             of several trainers into one vector.
+ *   result    device block; status is DCT_OK, or DCT_ERR_BAD_MASK if an index was outside [0, n)
+ *             or the indices were not ascending (such entries are skipped, nothing out of bounds
+ *             is touched).
+ */
+DCT_API dct_status_t dct_dp_decompress(
+    const int32_t* idx, const float* val, const dct_result_t* packed, uint64_t capacity,
+    float* dense, uint64_t n, int accumulate,
+    dct_result_t* result, dct_stream_t stream);
+
+/*
+ * dct_mp_unpack -- the receiving end of Algorithm 2's two "send" steps: rebuilds the dense
+ * [rows, ld] matrix X .* M from the mask and the packed values (X_act .* M on the next worker in the
+ * forward pass, X_grad .* M on the previous worker in the backward pass).
+ *
+ *   cols      [rows*k] int16: the mask written by dct_mp_topk_pack_fwd.
+ *   vals      [rows*k] packed values (vals_out of the forward call or gvals_out of the backward call).
+ *   dense_out [rows, ld], dtype fp32 or bf16: columns 0..d-1 of every row are written (zero outside the
+ *             mask); columns d..ld-1 are left untouched.
+ *   result    device block or NULL; status is DCT_OK, or DCT_ERR_BAD_MASK if a column was >= d
+ *             (that slot is skipped).
+ */
+DCT_API dct_status_t dct_mp_unpack(
+    const int16_t* cols, const void* vals, dct_dtype_t dtype,
+    uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+    void* dense_out, dct_result_t* result, dct_stream_t stream);
+
+/*
  * Host-buffer convenience calls: the same operators for a caller whose data
  * lives in HOST memory (pinned memory gives full copy speed; pageable memory
  * works).  Each call copies its inputs to the caller-provided device staging

@@ -41,7 +41,8 @@ def _load():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         for name in ("oracle_dp_select", "oracle_dp_compress", "oracle_mp_fwd_f32",
-                     "oracle_mp_fwd_bf16", "oracle_mp_bwd_f32", "oracle_mp_bwd_bf16"):
+                     "oracle_mp_fwd_bf16", "oracle_mp_bwd_f32", "oracle_mp_bwd_bf16",
+                     "oracle_dp_decompress", "oracle_mp_unpack_f32", "oracle_mp_unpack_bf16"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -158,3 +159,39 @@ def mp_bwd(gx: np.ndarray, cols: np.ndarray, d: Optional[int] = None) -> np.ndar
     if rc:
         raise ValueError(f"oracle_mp_bwd: invalid argument (rc={rc})")
     return gvals
+
+
+def dp_decompress(idx: np.ndarray, val: np.ndarray, dense: np.ndarray, accumulate: bool) -> None:
+    """Receiving end of Algorithm 1's send: scatter (idx, val) into ``dense`` (in place); with
+    ``accumulate`` the values are added to what is there, otherwise ``dense`` is cleared first."""
+    lib = _load()
+    _check(idx, np.int32, "idx")
+    _check(val, np.float32, "val")
+    _check(dense, np.float32, "dense")
+    assert idx.size == val.size
+    rc = lib.oracle_dp_decompress(_ptr(idx), _ptr(val), _c_u64(idx.size), _ptr(dense), _c_u64(dense.size),
+                                  ctypes.c_int(1 if accumulate else 0))
+    if rc:
+        raise ValueError(f"oracle_dp_decompress: invalid argument (rc={rc})")
+
+
+def mp_unpack(cols: np.ndarray, vals: np.ndarray, d: int, ld: Optional[int] = None) -> np.ndarray:
+    """Receiving end of Algorithm 2's sends: the dense [rows, ld] matrix that holds ``vals`` at the mask
+    columns and zero at the other columns below d (columns d..ld-1 are returned as zero)."""
+    lib = _load()
+    assert cols.ndim == 2 and vals.shape == cols.shape
+    rows, k = cols.shape
+    ld = d if ld is None else ld
+    if vals.dtype == np.float32:
+        fn = lib.oracle_mp_unpack_f32
+    elif vals.dtype == np.uint16:
+        fn = lib.oracle_mp_unpack_bf16
+    else:
+        raise TypeError("vals: float32 or uint16 (bf16 bits)")
+    _check(cols, np.int16, "cols")
+    _check(vals, vals.dtype, "vals")
+    dense = np.zeros((rows, ld), dtype=vals.dtype)
+    rc = fn(_ptr(cols), _ptr(vals), _c_u32(rows), _c_u32(d), _c_u32(ld), _c_u32(k), _ptr(dense))
+    if rc:
+        raise ValueError(f"oracle_mp_unpack: invalid argument (rc={rc})")
+    return dense

@@ -211,6 +211,55 @@ int mp_backward(const T* gx, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
 
 extern "C" {
 
+// Receiving end of "Send W_hat" (Algorithm 1): the sparse vector goes back into a dense one, either on
+// its own (dense = W_hat) or added to what is already there (a server summing several trainers).
+int oracle_dp_decompress(const int32_t* idx, const float* val, uint64_t count, float* dense, uint64_t n,
+                         int accumulate) {
+    if (dense == nullptr || n == 0) return 1;
+    if (!accumulate)
+        for (uint64_t i = 0; i < n; ++i) dense[i] = 0.0f;
+    for (uint64_t j = 0; j < count; ++j) {
+        if (idx[j] < 0 || static_cast<uint64_t>(idx[j]) >= n) return 2;
+        if (accumulate) {
+            volatile float s = dense[idx[j]] + val[j];
+            dense[idx[j]] = s;
+        } else {
+            dense[idx[j]] = val[j];
+        }
+    }
+    return 0;
+}
+
+}  // extern "C"
+
+namespace {
+// Receiving end of Algorithm 2's sends: X .* M rebuilt from the mask columns and the packed values.
+template <typename T>
+int mp_unpack(const int16_t* cols, const T* vals, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, T* dense) {
+    if (cols == nullptr || vals == nullptr || dense == nullptr || d == 0 || k == 0 || k > d || ld < d) return 1;
+    for (uint32_t i = 0; i < rows; ++i) {
+        for (uint32_t j = 0; j < d; ++j) dense[static_cast<uint64_t>(i) * ld + j] = T(0);
+        for (uint32_t s = 0; s < k; ++s) {
+            const uint32_t c = static_cast<uint16_t>(cols[static_cast<uint64_t>(i) * k + s]);
+            if (c >= d) return 2;
+            dense[static_cast<uint64_t>(i) * ld + c] = vals[static_cast<uint64_t>(i) * k + s];
+        }
+    }
+    return 0;
+}
+}  // namespace
+
+extern "C" {
+
+int oracle_mp_unpack_f32(const int16_t* cols, const float* vals, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                         float* dense) {
+    return mp_unpack<float>(cols, vals, rows, d, ld, k, dense);
+}
+int oracle_mp_unpack_bf16(const int16_t* cols, const uint16_t* vals, uint32_t rows, uint32_t d, uint32_t ld,
+                          uint32_t k, uint16_t* dense) {
+    return mp_unpack<uint16_t>(cols, vals, rows, d, ld, k, dense);
+}
+
 int oracle_mp_fwd_f32(const float* x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                       int16_t* cols, float* vals, float* tau) {
     return mp_forward<float>(x, rows, d, ld, k, [](float v) { return key_f32(v); }, cols, vals, tau);

@@ -28,7 +28,7 @@ EXPORTED_SYMBOLS = (
     "dct_threshold_select_workspace_bytes", "dct_dp_compress_workspace_bytes",
     "dct_threshold_select", "dct_dp_compress", "dct_mp_topk_pack_fwd", "dct_mp_pack_bwd",
     "dct_dp_compress_host", "dct_mp_pack_host", "dct_threshold_select_host", "dct_debug_configure",
-    "dct_dp_compress_static",
+    "dct_dp_compress_static", "dct_dp_decompress", "dct_mp_unpack",
 )
 
 _vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
     L.dct_threshold_select.argtypes = [_vp, _vp, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
     L.dct_dp_compress.restype = _int
     L.dct_dp_compress.argtypes = [_vp, _vp, _u64, _vp, _vp, _vp, _vp, _u64, _vp, _vp, _sz, _vp]
+    L.dct_dp_decompress.restype = _int
+    L.dct_dp_decompress.argtypes = [_vp, _vp, _vp, _u64, _vp, _u64, _int, _vp, _vp]
+    L.dct_mp_unpack.restype = _int
+    L.dct_mp_unpack.argtypes = [_vp, _vp, _int, _u32, _u32, _u32, _u32, _vp, _vp, _vp]
     L.dct_dp_compress_static.restype = _int
     L.dct_dp_compress_static.argtypes = [_vp, _vp, _u64, _vp, _vp, _vp, _vp, _u64, _vp, _vp]
     L.dct_mp_topk_pack_fwd.restype = _int
@@ -267,6 +271,33 @@ def dct_mp_pack_bwd(x_grad, rows, d, ld, k, cols, gvals_out, result=None, stream
     _check("dct_mp_pack_bwd",
            lib().dct_mp_pack_bwd(_p(x_grad), code, rows, d, ld, k, _p(cols), _p(gvals_out), _p(result),
                                  _stream(stream)))
+
+
+def dct_dp_decompress(idx, val, packed, capacity, dense, n, accumulate, result, stream=None) -> None:
+    _need(idx, torch.int32, "idx")
+    _need(val, torch.float32, "val")
+    _need(packed, torch.int64, "packed")
+    _need(dense, torch.float32, "dense")
+    _need(result, torch.int64, "result")
+    if idx.numel() < capacity or val.numel() < capacity or dense.numel() < n:
+        raise ValueError("buffer smaller than capacity / n")
+    _check("dct_dp_decompress",
+           lib().dct_dp_decompress(_p(idx), _p(val), _p(packed), capacity, _p(dense), n, 1 if accumulate else 0,
+                                   _p(result), _stream(stream)))
+
+
+def dct_mp_unpack(cols, vals, rows, d, ld, k, dense_out, result=None, stream=None) -> None:
+    code = _dtype_code(vals)
+    _need(cols, torch.int16, "cols")
+    _need(vals, vals.dtype, "vals")
+    _need(dense_out, vals.dtype, "dense_out")
+    if result is not None:
+        _need(result, torch.int64, "result")
+    if ld >= d and rows >= 1 and k >= 1:
+        if cols.numel() < rows * k or vals.numel() < rows * k or dense_out.numel() < (rows - 1) * ld + d:
+            raise ValueError("buffer smaller than rows x k / rows x ld")
+    _check("dct_mp_unpack",
+           lib().dct_mp_unpack(_p(cols), _p(vals), code, rows, d, ld, k, _p(dense_out), _p(result), _stream(stream)))
 
 
 def dct_dp_compress_host(grad_host, grad_dev, residual_dev, n, tau_dev, tie_budget_dev, idx_dev, val_dev, capacity,

@@ -1,0 +1,207 @@
+// Receiver side of the two "send" steps: turning the packed messages back into dense tensors.
+//
+//   dct_dp_decompress : Algorithm 1, what the parameter server does with the sparse W_hat it receives:
+//                       dense[idx[j]] = val[j] on a zero vector, or dense[idx[j]] += val[j] when the
+//                       messages of several trainers are accumulated.
+//   dct_mp_unpack     : Algorithm 2, what the next worker does with X_act .* M (and the previous worker
+//                       with X_grad .* M): rebuild the [rows, d] matrix that is zero outside the mask.
+//
+// The paper counts decompression in the overhead of the scheme (Sec. 2) but gives no procedure; both
+// are plain scatters.  Indices inside one message are distinct (ascending), so no atomics are needed.
+#include "common.cuh"
+
+namespace dct {
+namespace {
+
+// dense[0..n) = 0 with 128-bit stores, then the scatter, in one kernel: a grid-wide ordering between
+// the two is not needed because every CTA first clears, and then scatters into, ITS OWN range of
+// the dense vector: entries are routed to the CTA that owns idx via a binary search on the ascending idx.
+__global__ void __launch_bounds__(256)
+dp_decompress_kernel(const int32_t* __restrict__ idx, const float* __restrict__ val,
+                     const dct_result_t* __restrict__ packed, uint64_t capacity, float* __restrict__ dense,
+                     uint32_t n, int accumulate, dct_result_t* __restrict__ result) {
+    const uint64_t have = packed->count < capacity ? packed->count : capacity;
+    const uint32_t count = static_cast<uint32_t>(have);
+    // this CTA owns dense[lo, hi): a multiple of 4 elements so that the clearing stores stay aligned
+    const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 3u) & ~3u;
+    const uint64_t lo64 = static_cast<uint64_t>(blockIdx.x) * per;
+    if (lo64 >= n) return;
+    const uint32_t lo = static_cast<uint32_t>(lo64);
+    const uint32_t hi = (n - lo > per) ? lo + per : n;
+    if (!accumulate) {
+        const bool vec = (reinterpret_cast<uintptr_t>(dense) & 15u) == 0;
+        if (vec) {
+            const uint32_t hi4 = lo + ((hi - lo) & ~3u);
+            for (uint32_t i = lo + threadIdx.x * 4; i < hi4; i += blockDim.x * 4)
+                st_stream_f4(dense + i, make_float4(0.f, 0.f, 0.f, 0.f));
+            for (uint32_t i = hi4 + threadIdx.x; i < hi; i += blockDim.x) dense[i] = 0.0f;
+        } else {
+            for (uint32_t i = lo + threadIdx.x; i < hi; i += blockDim.x) dense[i] = 0.0f;
+        }
+        __syncthreads();          // this CTA's range is clear before this CTA writes into it
+    }
+    // first entry with idx >= lo (idx ascending; malformed input only costs misplaced work, never a fault)
+    uint32_t a = 0, b = count;
+    while (a < b) {
+        const uint32_t mid = (a + b) >> 1;
+        if (static_cast<uint32_t>(idx[mid]) < lo) a = mid + 1; else b = mid;
+    }
+    bool bad = false;
+    for (uint32_t j = a + threadIdx.x; j < count; j += blockDim.x) {
+        const uint32_t i = static_cast<uint32_t>(idx[j]);
+        if (i >= hi) break;       // the rest belongs to later CTAs (or is out of range)
+        if (i < lo) { bad = true; continue; }   // not ascending
+        if (accumulate) dense[i] += val[j]; else dense[i] = val[j];
+    }
+    // entries at or beyond n belong to nobody: the last CTA reports them
+    if (hi == n && threadIdx.x == 0 && count > 0 && static_cast<uint32_t>(idx[count - 1]) >= n) bad = true;
+    if (bad) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+mp_unpack_kernel(const int16_t* __restrict__ cols, const T* __restrict__ vals, uint32_t rows, uint32_t d, uint32_t ld,
+                 uint32_t k, T* __restrict__ dense, dct_result_t* __restrict__ result) {
+    const uint32_t lane = lane_id();
+    const uint32_t warps_per_cta = blockDim.x >> 5;
+    bool bad = false;
+    for (uint64_t row = static_cast<uint64_t>(blockIdx.x) * warps_per_cta + (threadIdx.x >> 5); row < rows;
+         row += static_cast<uint64_t>(gridDim.x) * warps_per_cta) {
+        T* out = dense + row * ld;
+        // clear the d columns of the row: 16-byte stores where the row allows it
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(out);
+        constexpr uint32_t per16 = 16 / sizeof(T);
+        uint32_t head = static_cast<uint32_t>(((16 - (addr & 15u)) & 15u) / sizeof(T));
+        if (head > d) head = d;
+        for (uint32_t j = lane; j < head; j += 32) out[j] = T(0);
+        const uint32_t nvec = (d - head) / per16;
+        uint4* out16 = reinterpret_cast<uint4*>(out + head);
+        for (uint32_t v = lane; v < nvec; v += 32) out16[v] = make_uint4(0, 0, 0, 0);
+        for (uint32_t j = head + nvec * per16 + lane; j < d; j += 32) out[j] = T(0);
+        __syncwarp();             // the row is clear before any of its kept entries is written
+        const int16_t* cr = cols + row * k;
+        const T* vr = vals + row * k;
+        for (uint32_t s = lane; s < k; s += 32) {
+            const uint32_t c = static_cast<uint16_t>(__ldg(cr + s));
+            if (c < d) out[c] = __ldg(vr + s); else bad = true;
+        }
+    }
+    if (bad && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
+}
+
+// Fast path for rows that start on 16-byte boundaries and are at most 16 KiB long: every warp builds its
+// row in shared memory (clear, scatter the k kept values) and hands it to one bulk store, so HBM only
+// sees full, sequential 16-byte-aligned writes.
+constexpr int kUnpackWarps = 8;
+template <typename T>
+__global__ void __launch_bounds__(kUnpackWarps * 32)
+mp_unpack_staged_kernel(const int16_t* __restrict__ cols, const T* __restrict__ vals, uint32_t rows, uint32_t d,
+                        uint32_t ld, uint32_t k, T* __restrict__ dense, dct_result_t* __restrict__ result) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    const uint32_t row_bytes = d * static_cast<uint32_t>(sizeof(T));          // a multiple of 16
+    T* buf = reinterpret_cast<T*>(smem_raw + static_cast<size_t>(warp) * row_bytes);
+    bool bad = false;
+    for (uint64_t row = static_cast<uint64_t>(blockIdx.x) * kUnpackWarps + warp; row < rows;
+         row += static_cast<uint64_t>(gridDim.x) * kUnpackWarps) {
+        if (lane == 0) bulk_wait_read<0>();       // the previous row has left the buffer
+        __syncwarp();
+        uint4* b16 = reinterpret_cast<uint4*>(buf);
+        for (uint32_t v = lane; v < row_bytes / 16; v += 32) b16[v] = make_uint4(0, 0, 0, 0);
+        __syncwarp();
+        const int16_t* cr = cols + row * k;
+        const T* vr = vals + row * k;
+        for (uint32_t s = lane; s < k; s += 32) {
+            const uint32_t c = static_cast<uint16_t>(__ldg(cr + s));
+            if (c < d) buf[c] = __ldg(vr + s); else bad = true;
+        }
+        fence_proxy_async_smem();                 // the bulk store reads what the lanes just wrote
+        __syncwarp();
+        if (lane == 0) {
+            bulk_store(dense + row * ld, buf, row_bytes);
+            bulk_commit();
+        }
+    }
+    if (lane == 0) bulk_wait_all<0>();            // nothing may still read this CTA's shared memory
+    if (bad && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
+}
+
+template <typename T>
+cudaError_t launch_unpack(const int16_t* cols, const void* vals, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                          void* dense_out, dct_result_t* result, int sms, cudaStream_t stream) {
+    const size_t row_bytes = static_cast<size_t>(d) * sizeof(T);
+    const bool staged = aligned_to(dense_out, 16) && (static_cast<size_t>(ld) * sizeof(T)) % 16 == 0 &&
+                        row_bytes % 16 == 0 && row_bytes <= 16 * 1024;
+    if (staged) {
+        const size_t smem = kUnpackWarps * row_bytes;
+        auto kernel = mp_unpack_staged_kernel<T>;
+        if (smem > 48 * 1024) {
+            const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                       static_cast<int>(kUnpackWarps * 16 * 1024));
+            if (e != cudaSuccess) return e;
+        }
+        size_t per_sm = (200 * 1024) / (smem + 1024);
+        if (per_sm < 1) per_sm = 1;
+        if (per_sm > 8) per_sm = 8;
+        const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + kUnpackWarps - 1) / kUnpackWarps;
+        const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
+        const unsigned grid = static_cast<unsigned>(ctas_needed < max_grid ? ctas_needed : max_grid);
+        kernel<<<grid, kUnpackWarps * 32, smem, stream>>>(cols, static_cast<const T*>(vals), rows, d, ld, k,
+                                                          static_cast<T*>(dense_out), result);
+    } else {
+        const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + 7) / 8;
+        const uint64_t max_grid = static_cast<uint64_t>(sms) * 8;
+        const unsigned grid = static_cast<unsigned>(ctas_needed < max_grid ? ctas_needed : max_grid);
+        mp_unpack_kernel<T><<<grid, 256, 0, stream>>>(cols, static_cast<const T*>(vals), rows, d, ld, k,
+                                                      static_cast<T*>(dense_out), result);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+}  // namespace dct
+
+using namespace dct;
+
+extern "C" dct_status_t dct_dp_decompress(const int32_t* idx, const float* val, const dct_result_t* packed,
+                                          uint64_t capacity, float* dense, uint64_t n, int accumulate,
+                                          dct_result_t* result, dct_stream_t stream_) {
+    if (!packed || !dense || !result || n == 0 || n > 0x7FFFFFFFull) return DCT_ERR_INVALID_ARG;
+    if (capacity > 0 && (!idx || !val)) return DCT_ERR_INVALID_ARG;
+    if (capacity > 0x7FFFFFFFull) capacity = 0x7FFFFFFFull;
+    if (!aligned_to(idx, 4) || !aligned_to(val, 4) || !aligned_to(dense, 4) || !aligned_to(packed, 8) ||
+        !aligned_to(result, 8) || packed == result)
+        return DCT_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    DCT_CUDA_TRY(cudaMemsetAsync(result, 0, sizeof(dct_result_t), stream));
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    // enough CTAs to fill the machine, but at least 1024 elements of the dense vector each
+    uint64_t grid = static_cast<uint64_t>(sms) * 8;
+    const uint64_t by_size = (n + 1023) / 1024;
+    if (grid > by_size) grid = by_size;
+    dp_decompress_kernel<<<static_cast<unsigned>(grid), 256, 0, stream>>>(idx, val, packed, capacity, dense,
+                                                                         static_cast<uint32_t>(n), accumulate, result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}
+
+extern "C" dct_status_t dct_mp_unpack(const int16_t* cols, const void* vals, dct_dtype_t dtype, uint32_t rows,
+                                      uint32_t d, uint32_t ld, uint32_t k, void* dense_out, dct_result_t* result,
+                                      dct_stream_t stream_) {
+    if (!cols || !vals || !dense_out || rows == 0 || d == 0 || k == 0 || k > d || ld < d || d > 32768u)
+        return DCT_ERR_INVALID_ARG;
+    if (dtype != DCT_F32 && dtype != DCT_BF16) return DCT_ERR_UNSUPPORTED;
+    const size_t es = dtype == DCT_F32 ? 4 : 2;
+    if (!aligned_to(vals, es) || !aligned_to(dense_out, es) || !aligned_to(cols, 2) || (result && !aligned_to(result, 8)))
+        return DCT_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (result) DCT_CUDA_TRY(cudaMemsetAsync(result, 0, sizeof(dct_result_t), stream));
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    if (dtype == DCT_F32)
+        DCT_CUDA_TRY(launch_unpack<float>(cols, vals, rows, d, ld, k, dense_out, result, sms, stream));
+    else
+        DCT_CUDA_TRY(launch_unpack<uint16_t>(cols, vals, rows, d, ld, k, dense_out, result, sms, stream));
+    return DCT_OK;
+}

@@ -6,6 +6,8 @@ A small command-line driver for profiling and quick timing of a single kernel at
     python -m paper_2010_08899_b200.run_case select   --n 268435456 --k 26844
     python -m paper_2010_08899_b200.run_case mp_fwd   --rows 16384 --d 4096 --k 205 --dtype bf16
     python -m paper_2010_08899_b200.run_case mp_bwd   --rows 16384 --d 4096 --k 205 --dtype bf16
+    python -m paper_2010_08899_b200.run_case decompress --n 268435456
+    python -m paper_2010_08899_b200.run_case mp_unpack --rows 16384 --d 4096 --k 205 --dtype bf16
 
 It prints the mean device time per call (CUDA events) and the algorithmic GB/s.
 """
@@ -21,7 +23,7 @@ from . import inputs
 
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("entry", choices=["select", "compress", "mp_fwd", "mp_bwd"])
+    ap.add_argument("entry", choices=["select", "compress", "decompress", "mp_fwd", "mp_bwd", "mp_unpack"])
     ap.add_argument("--n", type=int, default=1 << 28)
     ap.add_argument("--k", type=int, default=0, help="survivor target (default: 0.01 %% of n, or 5 %% of d)")
     ap.add_argument("--rows", type=int, default=16384)
@@ -37,7 +39,7 @@ def main():
     reset = lambda: None
     gen = {"mixture": inputs.dp_mixture, "gaussian": inputs.dp_gaussian, "dlrm": inputs.dp_dlrm_like}[args.dist]
 
-    if args.entry in ("select", "compress"):
+    if args.entry in ("select", "compress", "decompress"):
         n = args.n
         k = args.k or B.k_from_density(n, 1, 10_000)
         g = [gen(n, 501 + j, dev) for j in range(2)]
@@ -57,6 +59,15 @@ def main():
             call = lambda i: B.dct_dp_compress(g[i % 2], e, n, tau, None, idx, val, cap, res, ws_c)
             reset = e.zero_          # every timed call starts from a zero residual (same survivor density)
             nbytes = 12 * n
+            if args.entry == "decompress":
+                call(0)
+                count = B.read_result(res).count
+                packed = res.clone()
+                dense = torch.empty(n, device=dev)
+                res2 = B.new_result(dev)
+                call = lambda i: B.dct_dp_decompress(idx, val, packed, cap, dense, n, False, res2)
+                reset = lambda: None
+                nbytes = 4 * n + 8 * count       # clear the dense vector, read the packed pairs
     else:
         rows, d = args.rows, args.d
         k = args.k or B.k_from_sparsity(d, 95, 100)
@@ -69,6 +80,10 @@ def main():
         B.dct_mp_topk_pack_fwd(x[0], rows, d, d, k, cols, vals)
         if args.entry == "mp_fwd":
             call = lambda i: B.dct_mp_topk_pack_fwd(x[i % 2], rows, d, d, k, cols, vals, None, tau_i)
+            nbytes = rows * d * es + rows * k * (2 + es)
+        elif args.entry == "mp_unpack":
+            dense = [torch.empty(rows, d, dtype=dt, device=dev) for _ in range(2)]
+            call = lambda i: B.dct_mp_unpack(cols, vals, rows, d, d, k, dense[i % 2])
             nbytes = rows * d * es + rows * k * (2 + es)
         else:
             gx = [inputs.mp_gradients(rows, d, 420 + j, dtype=dt, device=dev) for j in range(2)]
