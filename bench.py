@@ -171,6 +171,39 @@ class HotPath:
         return out
 
 
+    def time_extras(self, stream, reps=3):
+        """The entry points beyond the step, timed on their own after the main measurement: threshold
+        life-span L = 1 (select + compress of the same vector), and the two decompression calls."""
+        B, c, s = self.B, self.cfg, stream
+        n, cap = c["dp_n"], c["dp_capacity"]
+        rows, d, k = c["mp_rows"], c["mp_d"], c["mp_k"]
+        out = {}
+        ws = B.new_workspace(B.dct_dp_select_compress_workspace_bytes(n), self.dev)
+        res = B.new_result(self.dev)
+        scratch_e = torch.zeros(n, device=self.dev)
+        dense = torch.empty(n, device=self.dev)
+        dense_mp = torch.empty(rows, d, dtype=torch.bfloat16, device=self.dev)
+        calls = {
+            "dp_select_compress_L1": lambda i: B.dct_dp_select_compress(
+                self.grad_view(i), scratch_e, n, c["dp_k"], self.tau, self.idx, self.val, cap, res, ws, s),
+            "dp_decompress": lambda i: B.dct_dp_decompress(self.idx, self.val, res, cap, dense, n, False,
+                                                           self.res_mp, s),
+            "mp_unpack": lambda i: B.dct_mp_unpack(self.cols, self.vals, rows, d, d, k, dense_mp, None, s),
+        }
+        for name, call in calls.items():
+            call(0)
+            a = _record(stream)
+            for i in range(reps):
+                call(1 + i)
+            b = _record(stream)
+            b.synchronize()
+            out[name] = {"ms": a.elapsed_time(b) / reps}
+        out["dp_select_compress_L1"]["GBps_at_16B_per_elem"] = 16 * n / (out["dp_select_compress_L1"]["ms"] * 1e-3) / 1e9
+        out["dp_decompress"]["GBps_at_4B_per_elem"] = 4 * n / (out["dp_decompress"]["ms"] * 1e-3) / 1e9
+        out["mp_unpack"]["GBps"] = (rows * d * 2 + rows * k * 4) / (out["mp_unpack"]["ms"] * 1e-3) / 1e9
+        return out
+
+
 class HostPath:
     """The same step through the host-buffer entry points: every input crosses PCIe inside the step."""
 
@@ -478,6 +511,7 @@ def main():
         "mp_bwd": {"ms": mp_parts["mp_bwd"], "GBps": b0["mp_bwd"] / cfg["mp_iters"] / (mp_parts["mp_bwd"] * 1e-3) / 1e9,
                    "dense_equiv_GBps": cfg["mp_rows"] * cfg["mp_d"] * 2 / (mp_parts["mp_bwd"] * 1e-3) / 1e9},
     }
+    parts["beyond_the_step"] = hp.time_extras(stream)
     roofline = {
         "kernel": "dp_compress_stream_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_kind": peak_kind,

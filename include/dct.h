@@ -195,6 +195,30 @@ DCT_API dct_status_t dct_mp_pack_bwd(
     dct_result_t* result, dct_stream_t stream);
 
 /*
+ * dct_dp_select_compress -- Algorithm 1 with threshold life-span L = 1: the branch "L divides the
+ * iteration number" taken at every iteration, i.e. top-K sparsification with error feedback where the
+ * threshold comes from the very vector that is compressed (the scheme the paper starts from, and on
+ * its CPUs found 11 % slower end to end than no compression).
+ *
+ * Enqueues dct_threshold_select on fl32(grad + residual), derives the tie budget k - n_gt on the
+ * device, and runs dct_dp_compress with it: exactly min(k, capacity) elements are sent, the lowest
+ * indices first among those equal to the threshold.
+ *
+ *   grad, residual, n, idx_out, val_out, capacity   as in dct_dp_compress.
+ *   k          survivors wanted, 1 <= k <= n.
+ *   tau_out    1 fp32 (device): the threshold that was used.
+ *   result     device block: count (= min(k, capacity)), needed (= k), status as in dct_dp_compress,
+ *              and n_gt, n_eq of the select.
+ *   workspace  >= dct_dp_select_compress_workspace_bytes(n), 256-byte aligned.
+ */
+DCT_API size_t dct_dp_select_compress_workspace_bytes(uint64_t n);
+DCT_API dct_status_t dct_dp_select_compress(
+    const float* grad, float* residual, uint64_t n, uint64_t k,
+    float* tau_out, int32_t* idx_out, float* val_out, uint64_t capacity,
+    dct_result_t* result,
+    void* workspace, size_t workspace_bytes, dct_stream_t stream);
+
+/*
  * dct_dp_decompress -- the receiving end of Algorithm 1's "Send W_hat": the sparse compressed gradient
  * goes back into a dense vector (the paper counts this decompression in the overhead of the scheme,
  * Sec. 2, without prescribing a procedure).

@@ -29,6 +29,7 @@ EXPORTED_SYMBOLS = (
     "dct_threshold_select", "dct_dp_compress", "dct_mp_topk_pack_fwd", "dct_mp_pack_bwd",
     "dct_dp_compress_host", "dct_mp_pack_host", "dct_threshold_select_host", "dct_debug_configure",
     "dct_dp_compress_static", "dct_dp_decompress", "dct_mp_unpack",
+    "dct_dp_select_compress", "dct_dp_select_compress_workspace_bytes",
 )
 
 _vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
@@ -69,6 +70,10 @@ def lib() -> ctypes.CDLL:
     L.dct_threshold_select.argtypes = [_vp, _vp, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
     L.dct_dp_compress.restype = _int
     L.dct_dp_compress.argtypes = [_vp, _vp, _u64, _vp, _vp, _vp, _vp, _u64, _vp, _vp, _sz, _vp]
+    L.dct_dp_select_compress_workspace_bytes.restype = _sz
+    L.dct_dp_select_compress_workspace_bytes.argtypes = [_u64]
+    L.dct_dp_select_compress.restype = _int
+    L.dct_dp_select_compress.argtypes = [_vp, _vp, _u64, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _sz, _vp]
     L.dct_dp_decompress.restype = _int
     L.dct_dp_decompress.argtypes = [_vp, _vp, _vp, _u64, _vp, _u64, _int, _vp, _vp]
     L.dct_mp_unpack.restype = _int
@@ -366,3 +371,25 @@ def dct_debug_configure(spin_limit: int = 1 << 21, first_ticket: int = 0) -> Non
     """Testing knobs: iteration limit of device-side waits, and the first tile ticket of dct_dp_compress
     (a non-zero value leaves tile 0 unprocessed so that the bounded wait can be seen to give up)."""
     lib().dct_debug_configure(spin_limit, first_ticket)
+
+
+def dct_dp_select_compress_workspace_bytes(n: int) -> int:
+    return lib().dct_dp_select_compress_workspace_bytes(n)
+
+
+def dct_dp_select_compress(grad, residual, n, k, tau_out, idx_out, val_out, capacity, result, workspace,
+                           stream=None) -> None:
+    """Threshold life-span L = 1: select on grad + residual, then compress the same vector with the tie
+    budget k - n_gt, all on the stream."""
+    _need(grad, torch.float32, "grad")
+    _need(residual, torch.float32, "residual")
+    _need(tau_out, torch.float32, "tau_out")
+    _need(idx_out, torch.int32, "idx_out")
+    _need(val_out, torch.float32, "val_out")
+    _need(result, torch.int64, "result")
+    _need(workspace, torch.uint8, "workspace")
+    if grad.numel() < n or residual.numel() < n or idx_out.numel() < capacity or val_out.numel() < capacity:
+        raise ValueError("buffer smaller than n / capacity")
+    _check("dct_dp_select_compress",
+           lib().dct_dp_select_compress(_p(grad), _p(residual), n, k, _p(tau_out), _p(idx_out), _p(val_out),
+                                        capacity, _p(result), _p(workspace), workspace.numel(), _stream(stream)))
