@@ -157,9 +157,7 @@ __device__ __forceinline__ bool resolve_tile_prefix(uint64_t* tile_state, Compre
     bool timed_out = false;
     excl_gt = 0;
     excl_eq = 0;
-#ifndef DCT_DBG_NO_LOOKBACK
     if (tile > 0) lookback(tile_state, ctrl, tile, spin_limit, excl_gt, excl_eq, timed_out);
-#endif
     if (timed_out) {
         if (lane == 0) {
             atomicExch(&ctrl->abort, 1u);

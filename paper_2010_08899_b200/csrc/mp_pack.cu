@@ -568,11 +568,6 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             if (!use_guess || (n_cand >= k && n_cand <= kRound)) break;
             use_guess = false;
         }
-#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 2
-        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(n_cand);
-        release_row(row);
-        continue;
-#endif
         if (!have_bound || n_cand > kRound) {
             mp_row_slow_path<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
             release_row(row);
@@ -619,10 +614,6 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             }
         }
         release_row(row);
-#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 3
-        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(ent[0]);
-        continue;
-#endif
 
         // ---- C: k-th largest of the candidates --------------------------------------------------
         uint32_t tau_key = 0, take = 0;
@@ -684,9 +675,6 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         }
         if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
         guess_low = tau_key > kGuessMargin ? tau_key - kGuessMargin : 0u;
-#if defined(DCT_DBG_FWD_STOP) && DCT_DBG_FWD_STOP == 4
-        continue;
-#endif
 
         // ---- D: ordered emit ------------------------------------------------------------------------
         // The kept entries are placed, in column order, into k staging slots; then they leave with
