@@ -28,9 +28,11 @@
  *     cleared, compared as an unsigned integer (uint32 for fp32, uint16 for
  *     bf16).  For non-NaN x this is the order of |x| with -0 == +0.  Ties in
  *     key are broken by the lower index / column.
- *   - Inputs are expected to be finite.  NaN/Inf do not trap and are handled
- *     deterministically (they order above every finite magnitude), but are
- *     outside the bit-exactness contract.
+ *   - Inputs are expected to be finite.  Inf orders above every finite
+ *     magnitude.  NaN never traps and never causes an out-of-bounds access,
+ *     but is outside the contract: the DP calls order it above Inf, while
+ *     dct_mp_topk_pack_fwd may return an arbitrary (valid, k columns) selection
+ *     for a row that contains NaN.
  */
 #ifndef DCT_H_
 #define DCT_H_
@@ -56,7 +58,7 @@ typedef enum {
   DCT_ERR_CUDA        = 4, /* host: a CUDA runtime call failed (see dct_last_cuda_error) */
   DCT_ERR_CAPACITY    = 5, /* device: survivors > capacity; output truncated, the rest kept in the residual */
   DCT_ERR_TIMEOUT     = 6, /* device: a bounded device-side wait gave up; outputs are incomplete */
-  DCT_ERR_BAD_MASK    = 7  /* device: a mask column >= d was met in dct_mp_pack_bwd; that slot was skipped */
+  DCT_ERR_BAD_MASK    = 7  /* device: a mask column >= d (or a packed index outside the vector) was met; that slot was skipped */
 } dct_status_t;
 
 typedef enum { DCT_F32 = 0, DCT_BF16 = 1 } dct_dtype_t;
