@@ -197,6 +197,36 @@ DCT_API dct_status_t dct_mp_pack_bwd(
     dct_result_t* result, dct_stream_t stream);
 
 /*
+ * dct_dp_compress_batched -- dct_dp_compress for all the layers of a model at once.  The paper applies
+ * DCT-DP layer by layer, every layer with its own threshold and its own error (Sec. 2.1); its layers
+ * hold 10^3..10^6 parameters, for which one set of launches per layer costs more than the work itself.
+ * This call runs every layer of `layers` -- each exactly as dct_dp_compress would -- with one reset
+ * kernel, one streaming kernel over all full tiles of all 16-byte aligned layers and one kernel for
+ * the ragged last tiles and the unaligned layers.
+ *
+ *   layers     HOST array of num_layers descriptions; the device pointers inside follow the rules of
+ *              dct_dp_compress.  The array is read before the call returns.  Layers must not share
+ *              residual, output or result buffers.
+ *   workspace  DEVICE, >= dct_dp_compress_batched_workspace_bytes(sizes, num_layers), 256-byte aligned.
+ * Every layer's result block receives its own count / needed / status.
+ */
+typedef struct {
+  const float* grad;           /* [n] device */
+  float* residual;             /* [n] device, in/out */
+  uint64_t n;
+  const float* tau;            /* device scalar */
+  const uint64_t* tie_budget;  /* device scalar or NULL */
+  int32_t* idx_out;            /* [capacity] device */
+  float* val_out;              /* [capacity] device */
+  uint64_t capacity;
+  dct_result_t* result;        /* device */
+} dct_dp_layer_t;
+DCT_API size_t dct_dp_compress_batched_workspace_bytes(const uint64_t* n /* host, per layer */, uint32_t num_layers);
+DCT_API dct_status_t dct_dp_compress_batched(
+    const dct_dp_layer_t* layers /* host */, uint32_t num_layers,
+    void* workspace, size_t workspace_bytes, dct_stream_t stream);
+
+/*
  * dct_dp_select_compress -- Algorithm 1 with threshold life-span L = 1: the branch "L divides the
  * iteration number" taken at every iteration, i.e. top-K sparsification with error feedback where the
  * threshold comes from the very vector that is compressed (the scheme the paper starts from, and on

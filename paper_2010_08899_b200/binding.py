@@ -30,6 +30,7 @@ EXPORTED_SYMBOLS = (
     "dct_dp_compress_host", "dct_mp_pack_host", "dct_threshold_select_host", "dct_debug_configure",
     "dct_dp_compress_static", "dct_dp_decompress", "dct_mp_unpack",
     "dct_dp_select_compress", "dct_dp_select_compress_workspace_bytes",
+    "dct_dp_compress_batched", "dct_dp_compress_batched_workspace_bytes",
 )
 
 _vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
@@ -74,6 +75,10 @@ def lib() -> ctypes.CDLL:
     L.dct_dp_select_compress_workspace_bytes.argtypes = [_u64]
     L.dct_dp_select_compress.restype = _int
     L.dct_dp_select_compress.argtypes = [_vp, _vp, _u64, _u64, _vp, _vp, _vp, _u64, _vp, _vp, _sz, _vp]
+    L.dct_dp_compress_batched_workspace_bytes.restype = _sz
+    L.dct_dp_compress_batched_workspace_bytes.argtypes = [_vp, _u32]
+    L.dct_dp_compress_batched.restype = _int
+    L.dct_dp_compress_batched.argtypes = [_vp, _u32, _vp, _sz, _vp]
     L.dct_dp_decompress.restype = _int
     L.dct_dp_decompress.argtypes = [_vp, _vp, _vp, _u64, _vp, _u64, _int, _vp, _vp]
     L.dct_mp_unpack.restype = _int
@@ -393,3 +398,43 @@ def dct_dp_select_compress(grad, residual, n, k, tau_out, idx_out, val_out, capa
     _check("dct_dp_select_compress",
            lib().dct_dp_select_compress(_p(grad), _p(residual), n, k, _p(tau_out), _p(idx_out), _p(val_out),
                                         capacity, _p(result), _p(workspace), workspace.numel(), _stream(stream)))
+
+
+class _DpLayer(ctypes.Structure):          # dct_dp_layer_t
+    _fields_ = [("grad", _vp), ("residual", _vp), ("n", _u64), ("tau", _vp), ("tie_budget", _vp),
+                ("idx_out", _vp), ("val_out", _vp), ("capacity", _u64), ("result", _vp)]
+
+
+def dct_dp_compress_batched_workspace_bytes(sizes) -> int:
+    arr = (_u64 * len(sizes))(*sizes)
+    return lib().dct_dp_compress_batched_workspace_bytes(arr, len(sizes))
+
+
+def dct_dp_layer_table(layers):
+    """Marshal a sequence of layer dicts (keys of dct_dp_layer_t: grad, residual, n, tau, tie_budget or None,
+    idx_out, val_out, capacity, result) into the host array the C call takes.  Build it once per model."""
+    table = (_DpLayer * len(layers))()
+    for slot, a in zip(table, layers):
+        _need(a["grad"], torch.float32, "grad")
+        _need(a["residual"], torch.float32, "residual")
+        _need(a["tau"], torch.float32, "tau")
+        if a.get("tie_budget") is not None:
+            _need(a["tie_budget"], torch.int64, "tie_budget")
+        _need(a["idx_out"], torch.int32, "idx_out")
+        _need(a["val_out"], torch.float32, "val_out")
+        _need(a["result"], torch.int64, "result")
+        n, cap = a["n"], a["capacity"]
+        if a["grad"].numel() < n or a["residual"].numel() < n or a["idx_out"].numel() < cap or a["val_out"].numel() < cap:
+            raise ValueError("buffer smaller than n / capacity")
+        slot.grad, slot.residual, slot.n, slot.tau = _p(a["grad"]), _p(a["residual"]), n, _p(a["tau"])
+        slot.tie_budget = _p(a.get("tie_budget"))
+        slot.idx_out, slot.val_out, slot.capacity, slot.result = _p(a["idx_out"]), _p(a["val_out"]), cap, _p(a["result"])
+    return table
+
+
+def dct_dp_compress_batched(layers, workspace, stream=None) -> None:
+    """``layers``: a table from dct_dp_layer_table, or the sequence of layer dicts it is built from."""
+    table = layers if isinstance(layers, ctypes.Array) else dct_dp_layer_table(layers)
+    _need(workspace, torch.uint8, "workspace")
+    _check("dct_dp_compress_batched",
+           lib().dct_dp_compress_batched(table, len(table), _p(workspace), workspace.numel(), _stream(stream)))

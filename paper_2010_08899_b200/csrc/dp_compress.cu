@@ -32,6 +32,7 @@
 //   * dp_compress_tile_kernel -- one CTA per tile with plain loads and stores:
 //     the ragged last tile and vectors that are not 16-byte aligned.
 #include <mutex>
+#include <vector>
 
 #include "common.cuh"
 
@@ -64,8 +65,9 @@ __device__ __forceinline__ uint32_t desc_gt(uint64_t d) { return static_cast<uin
 __device__ __forceinline__ uint32_t desc_eq(uint64_t d) { return static_cast<uint32_t>(d & kCountMask); }
 
 struct CompressCtrl {
-    uint32_t ticket;     // next tile to hand out
-    uint32_t abort;      // a bounded wait gave up somewhere: everybody stops waiting
+    uint32_t ticket;       // next tile to hand out
+    uint32_t abort;        // a bounded wait gave up somewhere: everybody stops waiting
+    uint32_t slow_ticket;  // batched calls: next work item of the tile kernel
 };
 constexpr size_t kCtrlBytes = 256;
 
@@ -281,26 +283,18 @@ __device__ __forceinline__ void emit_warp(const float (&w)[kVecs * 4], uint32_t 
 #ifndef DCT_CMP_MIN_BLOCKS
 #define DCT_CMP_MIN_BLOCKS 4
 #endif
+// One tile, by one CTA, with plain loads and stores (every thread of the CTA calls this with the same tile).
 template <bool kVectorised>
-__global__ void __launch_bounds__(kThreads, DCT_CMP_MIN_BLOCKS)
-dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ residual, uint32_t n,
-                        const float* __restrict__ tau_p, const uint64_t* __restrict__ budget_p,
-                        int32_t* __restrict__ idx_out, float* __restrict__ val_out, uint64_t capacity,
-                        dct_result_t* __restrict__ result, CompressCtrl* ctrl,
-                        uint64_t* __restrict__ tile_state, uint32_t num_tiles, uint32_t fixed_tile,
-                        uint32_t spin_limit) {
-    __shared__ uint32_t s_tile;
+__device__ __forceinline__ void compress_tile_body(const float* __restrict__ grad, float* __restrict__ residual,
+                                                   uint32_t n, const float* __restrict__ tau_p,
+                                                   const uint64_t* __restrict__ budget_p,
+                                                   int32_t* __restrict__ idx_out, float* __restrict__ val_out,
+                                                   uint64_t capacity, dct_result_t* __restrict__ result,
+                                                   CompressCtrl* ctrl, uint64_t* __restrict__ tile_state,
+                                                   uint32_t num_tiles, uint32_t tile, uint32_t spin_limit) {
     __shared__ uint32_t s_warp_tot[kWarps];   // (gt << 16) | eq of each warp, each <= 512
     __shared__ uint32_t s_excl[2];
     __shared__ uint32_t s_abort;
-
-    if (threadIdx.x == 0) {
-        s_tile = fixed_tile != kInvalidTile ? fixed_tile : atomicAdd(&ctrl->ticket, 1u);
-        s_abort = 0;
-    }
-    __syncthreads();
-    const uint32_t tile = s_tile;
-    if (tile >= num_tiles) return;            // only reachable with a testing ticket offset
 
     const uint32_t lane = lane_id();
     const uint32_t warp = threadIdx.x >> 5;
@@ -388,6 +382,23 @@ dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ resi
               idx_out, val_out, residual);
 }
 
+template <bool kVectorised>
+__global__ void __launch_bounds__(kThreads, DCT_CMP_MIN_BLOCKS)
+dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ residual, uint32_t n,
+                        const float* __restrict__ tau_p, const uint64_t* __restrict__ budget_p,
+                        int32_t* __restrict__ idx_out, float* __restrict__ val_out, uint64_t capacity,
+                        dct_result_t* __restrict__ result, CompressCtrl* ctrl,
+                        uint64_t* __restrict__ tile_state, uint32_t num_tiles, uint32_t fixed_tile,
+                        uint32_t spin_limit) {
+    __shared__ uint32_t s_tile;
+    if (threadIdx.x == 0) s_tile = fixed_tile != kInvalidTile ? fixed_tile : atomicAdd(&ctrl->ticket, 1u);
+    __syncthreads();
+    const uint32_t tile = s_tile;
+    if (tile >= num_tiles) return;            // only reachable with a testing ticket offset
+    compress_tile_body<kVectorised>(grad, residual, n, tau_p, budget_p, idx_out, val_out, capacity, result, ctrl,
+                                    tile_state, num_tiles, tile, spin_limit);
+}
+
 // ------------------------------------------------------------------------------------------
 // fast path: persistent CTAs; load warp + compute warps + scan warp
 // ------------------------------------------------------------------------------------------
@@ -413,8 +424,10 @@ struct __align__(128) StreamSmem {
     uint64_t prefix_ready[kSlots];       // scan -> compute: exclusive prefix of the slot's tile is in prefix[]
     uint64_t slot_free[kSlots];          // scan -> compute: the slot may be reused
     uint32_t tile[kStages];
+    uint32_t layer[kStages];             // batched calls: which vector the stage's tile belongs to
     uint32_t warp_tot[2][kWarps];
     uint32_t slot_tile[kSlots];
+    uint32_t slot_layer[kSlots];
     uint32_t slot_agg[kSlots];           // (gt << 16) | eq of the tile
     uint32_t slot_direct[kSlots];        // 1: the compute warps write this tile's output themselves
     uint32_t prefix[kSlots][2];
@@ -422,12 +435,60 @@ struct __align__(128) StreamSmem {
     volatile uint32_t stop;              // a bounded wait gave up inside this CTA
 };
 
+// One vector of a call as the kernels see it (a batched call has a table of these in the workspace).
+struct LayerDesc {
+    const float* grad;
+    float* residual;
+    const float* tau;
+    const uint64_t* tie_budget;
+    int32_t* idx_out;
+    float* val_out;
+    dct_result_t* result;
+    uint64_t capacity;
+    uint32_t n;
+    uint32_t first_desc;   // index of the vector's first tile descriptor
+    uint32_t num_full;     // full tiles handled by the streaming kernel (0 for an unaligned vector)
+    uint32_t num_tiles;    // all tiles, a ragged last one included
+};
+struct BatchTable {
+    const LayerDesc* layers;
+    const uint32_t* full_prefix;   // [num_layers + 1] running count of streaming-kernel tiles
+    const uint32_t* slow_prefix;   // [num_layers + 1] running count of tile-kernel tiles
+    uint32_t num_layers;
+};
+// What a role needs to know about the vector it is working on, held in registers.
+struct TileParams {
+    const float* grad;
+    float* residual;
+    int32_t* idx_out;
+    float* val_out;
+    dct_result_t* result;
+    uint64_t* tile_state;          // descriptors of this vector: look-back never leaves them
+    uint64_t capacity, budget;
+    uint32_t tau_key, last_tile;
+};
+__device__ __forceinline__ TileParams load_params(const LayerDesc& d, uint64_t* tile_state_base) {
+    TileParams p;
+    p.grad = d.grad;
+    p.residual = d.residual;
+    p.idx_out = d.idx_out;
+    p.val_out = d.val_out;
+    p.result = d.result;
+    p.tile_state = tile_state_base + d.first_desc;
+    p.capacity = d.capacity;
+    p.budget = d.tie_budget ? *d.tie_budget : ~0ull;
+    p.tau_key = key_f32(*d.tau);
+    p.last_tile = d.num_tiles - 1;
+    return p;
+}
+
+// kBatched == false: one vector, described by `single`, work items are its full tiles.
+// kBatched == true : work items are the full tiles of all vectors of `batch`, in table order; a role
+//                    reloads its TileParams whenever the vector changes under it.
+template <bool kBatched>
 __global__ void __launch_bounds__(kStreamThreads, 2)
-dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ residual, uint32_t num_full_tiles,
-                          uint32_t last_tile, const float* __restrict__ tau_p,
-                          const uint64_t* __restrict__ budget_p, int32_t* __restrict__ idx_out,
-                          float* __restrict__ val_out, uint64_t capacity, dct_result_t* __restrict__ result,
-                          CompressCtrl* ctrl, uint64_t* __restrict__ tile_state, uint32_t spin_limit) {
+dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32_t total_work, CompressCtrl* ctrl,
+                          uint64_t* __restrict__ tile_state_base, uint32_t spin_limit) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
     const uint32_t tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
@@ -447,15 +508,34 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
         fence_proxy_async_all();
     }
     __syncthreads();
-    const uint64_t budget = budget_p ? *budget_p : ~0ull;
 
     if (warp == kLoadWarp) {
         // ================= load warp (one lane): tickets and bulk loads ====================
         if (lane != 0) return;
+        const float* grad = single.grad;
+        const float* residual = single.residual;
+        uint32_t cur_layer = 0, work_lo = 0, work_hi = total_work;     // work items of the current vector
+        if (kBatched) {
+            work_hi = batch.full_prefix[1];
+            grad = batch.layers[0].grad;
+            residual = batch.layers[0].residual;
+        }
         uint32_t ticket = atomicAdd(&ctrl->ticket, 1u);
         for (uint32_t it = 0;; ++it) {
             const int s = it % kStages;
-            const uint32_t tile = ticket < num_full_tiles ? ticket : kInvalidTile;
+            uint32_t tile = ticket < total_work ? ticket : kInvalidTile;
+            if (kBatched && tile != kInvalidTile) {
+                if (tile >= work_hi) {                                 // tickets only grow: walk forward
+                    do {
+                        ++cur_layer;
+                        work_lo = work_hi;
+                        work_hi = batch.full_prefix[cur_layer + 1];
+                    } while (tile >= work_hi);
+                    grad = batch.layers[cur_layer].grad;
+                    residual = batch.layers[cur_layer].residual;
+                }
+                tile -= work_lo;                                       // tile index inside its vector
+            }
             // the next ticket is requested now; its latency overlaps the wait below
             if (tile != kInvalidTile) ticket = atomicAdd(&ctrl->ticket, 1u);
             if (it >= static_cast<uint32_t>(kStages) &&
@@ -464,6 +544,7 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
                 return;
             }
             sm.tile[s] = tile;
+            sm.layer[s] = cur_layer;
             if (tile == kInvalidTile) {
                 mbar_arrive(&sm.full[s]);
                 return;
@@ -476,6 +557,9 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
 
     if (warp == kScanWarp) {
         // ================= scan warp: look-back, then drain the tile's queue ==================
+        TileParams P;
+        uint32_t cur_layer = 0xFFFFFFFFu;
+        if (!kBatched) P = load_params(single, tile_state_base);
         for (uint32_t it = 0;; ++it) {
             const int r = it % kSlots;
             const uint32_t parity = (it / kSlots) & 1u;
@@ -485,11 +569,15 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
             }
             const uint32_t tile = sm.slot_tile[r];
             if (tile == kInvalidTile) return;
+            if (kBatched && sm.slot_layer[r] != cur_layer) {
+                cur_layer = sm.slot_layer[r];
+                P = load_params(batch.layers[cur_layer], tile_state_base);
+            }
             const uint32_t tot = sm.slot_agg[r];
             const uint32_t cta_gt = tot >> 16, cta_eq = tot & 0xFFFFu;
             uint32_t excl_gt, excl_eq;
-            const bool ok = resolve_tile_prefix(tile_state, ctrl, result, tile, last_tile, cta_gt, cta_eq, budget,
-                                                capacity, spin_limit, excl_gt, excl_eq, false);
+            const bool ok = resolve_tile_prefix(P.tile_state, ctrl, P.result, tile, P.last_tile, cta_gt, cta_eq,
+                                                P.budget, P.capacity, spin_limit, excl_gt, excl_eq, false);
             if (sm.slot_direct[r]) {
                 if (lane == 0) {
                     sm.prefix[r][0] = excl_gt;
@@ -509,8 +597,8 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
                         const uint32_t local_eq = eq_run + __popc(eq_bal & lanemask_lt());
                         const uint32_t local_gt = q - local_eq;
                         place_survivor(ent.x & ~kEqBit, __uint_as_float(ent.y), is_eq, uint64_t(excl_gt) + local_gt,
-                                       uint64_t(excl_eq) + local_eq, budget, capacity, !ok, idx_out, val_out,
-                                       residual);
+                                       uint64_t(excl_eq) + local_eq, P.budget, P.capacity, !ok, P.idx_out, P.val_out,
+                                       P.residual);
                     }
                     eq_run += __popc(eq_bal);
                 }
@@ -524,7 +612,9 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
     }
 
     // ===================== compute warps =================================================
-    const uint32_t tau_key = key_f32(__ldg(tau_p));
+    TileParams P;
+    uint32_t cur_layer = 0xFFFFFFFFu;
+    if (!kBatched) P = load_params(single, tile_state_base);
     bool healthy = true;
     uint32_t it = 0;
     for (;; ++it) {
@@ -539,6 +629,10 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
         }
         const uint32_t tile = sm.tile[s];
         if (tile == kInvalidTile) break;
+        if (kBatched && sm.layer[s] != cur_layer) {
+            cur_layer = sm.layer[s];
+            P = load_params(batch.layers[cur_layer], tile_state_base);
+        }
         const uint32_t warp_base = tile * kTileElems + warp * kWarpElems;
 
         float w[kVecs * 4];
@@ -555,7 +649,7 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
             }
         }
         uint32_t gt_mask, eq_mask;
-        flag_elements(w, tau_key, 0xFFFFu, gt_mask, eq_mask);
+        flag_elements(w, P.tau_key, 0xFFFFu, gt_mask, eq_mask);
         const uint32_t flagged = gt_mask | eq_mask;
 #pragma unroll
         for (int j = 0; j < kVecs; ++j) {
@@ -564,7 +658,7 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
             e.y = (flagged >> (4 * j + 1)) & 1u ? 0.0f : w[4 * j + 1];
             e.z = (flagged >> (4 * j + 2)) & 1u ? 0.0f : w[4 * j + 2];
             e.w = (flagged >> (4 * j + 3)) & 1u ? 0.0f : w[4 * j + 3];
-            st_stream_f4(residual + warp_base + j * 128 + lane * 4, e);
+            st_stream_f4(P.residual + warp_base + j * 128 + lane * 4, e);
         }
         const uint32_t warp_tot =
             __reduce_add_sync(0xFFFFFFFFu, (static_cast<uint32_t>(__popc(gt_mask)) << 16) | __popc(eq_mask));
@@ -582,7 +676,7 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
         if (tid == 0) {
             mbar_arrive(&sm.empty[s]);
             // later tiles may need these counts right now; the scan warp adds the prefix when it gets here
-            publish_tile_aggregate(tile_state, tile, cta_gt, cta_eq);
+            publish_tile_aggregate(P.tile_state, tile, cta_gt, cta_eq);
         }
         // the slot must have been drained by the scan warp (it normally was, long ago)
         bool slot_ok = true;
@@ -591,6 +685,7 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
         if (!__all_sync(0xFFFFFFFFu, slot_ok)) sm.stop = 1;   // seen by everybody at the next vote
         if (tid == 0) {
             sm.slot_tile[r] = tile;
+            sm.slot_layer[r] = cur_layer;
             sm.slot_agg[r] = cta_tot;
             sm.slot_direct[r] = direct ? 1u : 0u;
         }
@@ -611,8 +706,8 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
                 break;
             }
             if (warp_tot != 0)
-                emit_warp(w, gt_mask, eq_mask, warp_base, before_warp, sm.prefix[r][0], sm.prefix[r][1], budget,
-                          capacity, sm.aborted[r] != 0, idx_out, val_out, residual);
+                emit_warp(w, gt_mask, eq_mask, warp_base, before_warp, sm.prefix[r][0], sm.prefix[r][1], P.budget,
+                          P.capacity, sm.aborted[r] != 0, P.idx_out, P.val_out, P.residual);
         }
     }
     if (healthy) {
@@ -628,8 +723,54 @@ dp_compress_stream_kernel(const float* __restrict__ grad, float* __restrict__ re
     } else if (tid == 0) {
         sm.stop = 1;
         atomicExch(&ctrl->abort, 1u);
-        atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
+        const LayerDesc& where = kBatched ? batch.layers[cur_layer < batch.num_layers ? cur_layer : 0] : single;
+        atomicMax(&where.result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
     }
+}
+
+// ---- batched calls: many vectors (the layers of a model), one set of launches ------------------------
+__global__ void dp_compress_batched_init_kernel(CompressCtrl* ctrl, uint64_t* tile_state, uint32_t total_tiles,
+                                                const LayerDesc* layers, uint32_t num_layers) {
+    const uint32_t stride = gridDim.x * blockDim.x;
+    const uint32_t i0 = blockIdx.x * blockDim.x + threadIdx.x;
+    for (uint32_t i = i0; i < total_tiles; i += stride) tile_state[i] = 0;
+    for (uint32_t l = i0; l < num_layers; l += stride) {
+        dct_result_t* r = layers[l].result;
+        r->status = DCT_OK;
+        r->reserved = 0;
+        r->count = 0;
+        r->needed = 0;
+        r->n_gt = 0;
+        r->n_eq = 0;
+    }
+    if (i0 == 0) {
+        ctrl->ticket = 0;
+        ctrl->abort = 0;
+        ctrl->slow_ticket = 0;
+    }
+}
+
+// The tiles the streaming kernel does not take: the ragged last tile of every aligned vector and all the
+// tiles of vectors that are not 16-byte aligned.  Work items are handed out in table order by a ticket,
+// so inside an unaligned vector a tile's predecessors have always been taken before it.
+__global__ void __launch_bounds__(kThreads, DCT_CMP_MIN_BLOCKS)
+dp_compress_tile_batched_kernel(const BatchTable batch, uint32_t total_slow, CompressCtrl* ctrl,
+                                uint64_t* __restrict__ tile_state_base, uint32_t spin_limit) {
+    __shared__ uint32_t s_work;
+    if (threadIdx.x == 0) s_work = atomicAdd(&ctrl->slow_ticket, 1u);
+    __syncthreads();
+    const uint32_t work = s_work;
+    if (work >= total_slow) return;
+    uint32_t lo = 0, hi = batch.num_layers;            // the vector l with slow_prefix[l] <= work < slow_prefix[l + 1]
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (batch.slow_prefix[mid] <= work) lo = mid; else hi = mid;
+    }
+    const LayerDesc& d = batch.layers[lo];
+    // an aligned vector contributes only its last tile; an unaligned one all of them
+    const uint32_t tile = d.num_full + (work - batch.slow_prefix[lo]);
+    compress_tile_body<false>(d.grad, d.residual, d.n, d.tau, d.tie_budget, d.idx_out, d.val_out, d.capacity,
+                              d.result, ctrl, tile_state_base + d.first_desc, d.num_tiles, tile, spin_limit);
 }
 
 }  // namespace
@@ -689,7 +830,8 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         int dev = 0;
         DCT_CUDA_TRY(cudaGetDevice(&dev));
         if (configured_device != dev) {
-            DCT_CUDA_TRY(cudaFuncSetAttribute(dp_compress_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            DCT_CUDA_TRY(cudaFuncSetAttribute(dp_compress_stream_kernel<false>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                                               static_cast<int>(sizeof(StreamSmem))));
             configured_device = dev;
         }
@@ -698,15 +840,166 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         const uint32_t ctas_per_sm = sizeof(StreamSmem) <= 110 * 1024 ? 2 : 1;
         const uint32_t max_grid = static_cast<uint32_t>(sms) * ctas_per_sm;
         const uint32_t grid = num_full < max_grid ? num_full : max_grid;
-        dp_compress_stream_kernel<<<grid, kStreamThreads, sizeof(StreamSmem), stream>>>(
-            grad, residual, num_full, num_tiles - 1, tau, tie_budget, idx_out, val_out, capacity, result, ctrl,
-            tile_state, dbg.spin_limit);
+        LayerDesc single{};
+        single.grad = grad;
+        single.residual = residual;
+        single.tau = tau;
+        single.tie_budget = tie_budget;
+        single.idx_out = idx_out;
+        single.val_out = val_out;
+        single.result = result;
+        single.capacity = capacity;
+        single.n = n32;
+        single.first_desc = 0;
+        single.num_full = num_full;
+        single.num_tiles = num_tiles;
+        dp_compress_stream_kernel<false><<<grid, kStreamThreads, sizeof(StreamSmem), stream>>>(
+            single, BatchTable{}, num_full, ctrl, tile_state, dbg.spin_limit);
         DCT_CUDA_TRY(cudaGetLastError());
     }
     if (num_tiles > num_full) {   // ragged last tile
         dp_compress_tile_kernel<true><<<1, kThreads, 0, stream>>>(
             grad, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
             num_full, dbg.spin_limit);
+        DCT_CUDA_TRY(cudaGetLastError());
+    }
+    return DCT_OK;
+}
+
+// ------------------------------------------------------------------------------------------
+// dct_dp_compress_batched: the layers of a model in one set of launches
+// ------------------------------------------------------------------------------------------
+namespace {
+
+struct BatchLayout {
+    size_t layers_off, full_off, slow_off, state_off, bytes;
+    uint64_t total_tiles;
+};
+BatchLayout batch_layout(const uint64_t* n, uint32_t num_layers) {
+    BatchLayout L{};
+    uint64_t tiles = 0;
+    for (uint32_t l = 0; l < num_layers; ++l) tiles += dp_compress_num_tiles(n[l]);
+    L.total_tiles = tiles;
+    size_t off = kCtrlBytes;
+    L.layers_off = off;
+    off += sizeof(LayerDesc) * num_layers;
+    off = (off + 15) & ~static_cast<size_t>(15);
+    L.full_off = off;
+    off += sizeof(uint32_t) * (num_layers + 1);
+    L.slow_off = off;
+    off += sizeof(uint32_t) * (num_layers + 1);
+    off = (off + 255) & ~static_cast<size_t>(255);
+    L.state_off = off;
+    off += sizeof(uint64_t) * tiles;
+    L.bytes = (off + 255) & ~static_cast<size_t>(255);
+    return L;
+}
+
+}  // namespace
+
+extern "C" size_t dct_dp_compress_batched_workspace_bytes(const uint64_t* n, uint32_t num_layers) {
+    if (!n || num_layers == 0) return 0;
+    for (uint32_t l = 0; l < num_layers; ++l)
+        if (n[l] == 0 || n[l] > 0x7FFFFFFFull) return 0;
+    const BatchLayout L = batch_layout(n, num_layers);
+    return L.total_tiles > 0xFFFFFFFFull ? 0 : L.bytes;
+}
+
+extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, uint32_t num_layers, void* workspace,
+                                                size_t workspace_bytes, dct_stream_t stream_) {
+    if (!layers || num_layers == 0) return DCT_ERR_INVALID_ARG;
+    std::vector<uint64_t> sizes(num_layers);
+    for (uint32_t l = 0; l < num_layers; ++l) {
+        const dct_dp_layer_t& a = layers[l];
+        if (!a.grad || !a.residual || !a.tau || !a.result || a.n == 0 || a.n > 0x7FFFFFFFull) return DCT_ERR_INVALID_ARG;
+        if (a.capacity > 0 && (!a.idx_out || !a.val_out)) return DCT_ERR_INVALID_ARG;
+        if (!aligned_to(a.grad, 4) || !aligned_to(a.residual, 4) || !aligned_to(a.tau, 4) || !aligned_to(a.result, 8) ||
+            (a.tie_budget && !aligned_to(a.tie_budget, 8)) || !aligned_to(a.idx_out, 4) || !aligned_to(a.val_out, 4))
+            return DCT_ERR_INVALID_ARG;
+        const uintptr_t g0 = reinterpret_cast<uintptr_t>(a.grad), e0 = reinterpret_cast<uintptr_t>(a.residual);
+        const uintptr_t bytes = static_cast<uintptr_t>(a.n) * 4;
+        if (g0 < e0 + bytes && e0 < g0 + bytes) return DCT_ERR_INVALID_ARG;
+        sizes[l] = a.n;
+    }
+    const BatchLayout L = batch_layout(sizes.data(), num_layers);
+    if (L.total_tiles > 0xFFFFFFFFull) return DCT_ERR_UNSUPPORTED;
+    if (!workspace || !aligned_to(workspace, 256) || workspace_bytes < L.bytes) return DCT_ERR_WORKSPACE;
+
+    // the table the kernels read: descriptors of all vectors, and the two running work counts
+    std::vector<unsigned char> table(L.state_off - L.layers_off);
+    auto* descs = reinterpret_cast<LayerDesc*>(table.data());
+    auto* full_prefix = reinterpret_cast<uint32_t*>(table.data() + (L.full_off - L.layers_off));
+    auto* slow_prefix = reinterpret_cast<uint32_t*>(table.data() + (L.slow_off - L.layers_off));
+    uint32_t first_desc = 0, total_full = 0, total_slow = 0;
+    for (uint32_t l = 0; l < num_layers; ++l) {
+        const dct_dp_layer_t& a = layers[l];
+        LayerDesc& d = descs[l];
+        const uint32_t n32 = static_cast<uint32_t>(a.n);
+        const bool vec = aligned_to(a.grad, 16) && aligned_to(a.residual, 16);
+        d.grad = a.grad;
+        d.residual = a.residual;
+        d.tau = a.tau;
+        d.tie_budget = a.tie_budget;
+        d.idx_out = a.idx_out;
+        d.val_out = a.val_out;
+        d.result = a.result;
+        d.capacity = a.capacity;
+        d.n = n32;
+        d.first_desc = first_desc;
+        d.num_tiles = dp_compress_num_tiles(a.n);
+        d.num_full = vec ? n32 / kTileElems : 0;
+        full_prefix[l] = total_full;
+        slow_prefix[l] = total_slow;
+        total_full += d.num_full;
+        total_slow += d.num_tiles - d.num_full;
+        first_desc += d.num_tiles;
+    }
+    full_prefix[num_layers] = total_full;
+    slow_prefix[num_layers] = total_slow;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    char* ws = static_cast<char*>(workspace);
+    auto* ctrl = reinterpret_cast<CompressCtrl*>(ws);
+    auto* tile_state = reinterpret_cast<uint64_t*>(ws + L.state_off);
+    // pageable source: the runtime has staged the bytes by the time this returns, so `table` may go away
+    DCT_CUDA_TRY(cudaMemcpyAsync(ws + L.layers_off, table.data(), table.size(), cudaMemcpyHostToDevice, stream));
+    BatchTable batch;
+    batch.layers = reinterpret_cast<const LayerDesc*>(ws + L.layers_off);
+    batch.full_prefix = reinterpret_cast<const uint32_t*>(ws + L.full_off);
+    batch.slow_prefix = reinterpret_cast<const uint32_t*>(ws + L.slow_off);
+    batch.num_layers = num_layers;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const DebugConfig& dbg = debug_config();
+    {
+        const uint64_t items = L.total_tiles > num_layers ? L.total_tiles : num_layers;
+        const uint64_t blocks = (items + 1023) / 1024;
+        const unsigned grid = static_cast<unsigned>(blocks < static_cast<uint64_t>(sms) * 4 ? blocks : sms * 4);
+        dp_compress_batched_init_kernel<<<grid, 1024, 0, stream>>>(ctrl, tile_state,
+                                                                   static_cast<uint32_t>(L.total_tiles), batch.layers,
+                                                                   num_layers);
+        DCT_CUDA_TRY(cudaGetLastError());
+    }
+    if (total_full > 0) {
+        static thread_local int configured_device = -1;
+        int dev = 0;
+        DCT_CUDA_TRY(cudaGetDevice(&dev));
+        if (configured_device != dev) {
+            DCT_CUDA_TRY(cudaFuncSetAttribute(dp_compress_stream_kernel<true>,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              static_cast<int>(sizeof(StreamSmem))));
+            configured_device = dev;
+        }
+        const uint32_t ctas_per_sm = sizeof(StreamSmem) <= 110 * 1024 ? 2 : 1;
+        const uint32_t max_grid = static_cast<uint32_t>(sms) * ctas_per_sm;
+        const uint32_t grid = total_full < max_grid ? total_full : max_grid;
+        dp_compress_stream_kernel<true><<<grid, kStreamThreads, sizeof(StreamSmem), stream>>>(
+            LayerDesc{}, batch, total_full, ctrl, tile_state, dbg.spin_limit);
+        DCT_CUDA_TRY(cudaGetLastError());
+    }
+    if (total_slow > 0) {
+        dp_compress_tile_batched_kernel<<<total_slow, kThreads, 0, stream>>>(batch, total_slow, ctrl, tile_state,
+                                                                           dbg.spin_limit);
         DCT_CUDA_TRY(cudaGetLastError());
     }
     return DCT_OK;

@@ -23,7 +23,7 @@ from . import inputs
 
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("entry", choices=["select", "compress", "decompress", "mp_fwd", "mp_bwd", "mp_unpack"])
+    ap.add_argument("entry", choices=["select", "compress", "compress_layers", "decompress", "mp_fwd", "mp_bwd", "mp_unpack"])
     ap.add_argument("--n", type=int, default=1 << 28)
     ap.add_argument("--k", type=int, default=0, help="survivor target (default: 0.01 %% of n, or 5 %% of d)")
     ap.add_argument("--rows", type=int, default=16384)
@@ -38,6 +38,50 @@ def main():
     stream = torch.cuda.current_stream()
     reset = lambda: None
     gen = {"mixture": inputs.dp_mixture, "gaussian": inputs.dp_gaussian, "dlrm": inputs.dp_dlrm_like}[args.dist]
+
+    if args.entry == "compress_layers":
+        # the vector of --n elements cut into DLRM-like dense layers, each with its own threshold and error:
+        # one batched call against one dct_dp_compress call per layer
+        sizes, total = [], 0
+        while total < args.n:
+            for fo, fi in inputs.DLRM_LIKE_LAYERS:
+                if total < args.n:
+                    sizes.append(min(fo * fi, args.n - total))
+                    total += sizes[-1]
+        g_all = inputs.dp_dlrm_like(args.n, 301, dev)
+        e_all = torch.zeros(args.n, device=dev)
+        layers, off = [], 0
+        for m in sizes:
+            cap = max(m // 16, 64)
+            tau = torch.zeros(1, device=dev)
+            r = B.new_result(dev)
+            B.dct_threshold_select(g_all[off:off + m], None, m, B.k_from_density(m, 1, 1000), tau, r,
+                                   B.new_workspace(B.dct_threshold_select_workspace_bytes(m), dev))
+            layers.append(dict(grad=g_all[off:off + m], residual=e_all[off:off + m], n=m, tau=tau, tie_budget=None,
+                               idx_out=torch.empty(cap, dtype=torch.int32, device=dev),
+                               val_out=torch.empty(cap, device=dev), capacity=cap, result=r))
+            off += m
+        ws_b = B.new_workspace(B.dct_dp_compress_batched_workspace_bytes(sizes), dev)
+        ws_1 = B.new_workspace(B.dct_dp_compress_workspace_bytes(max(sizes)), dev)
+        table = B.dct_dp_layer_table(layers)      # marshalled once, as a trainer would
+        variants = {
+            f"batched ({len(sizes)} layers, one call)": lambda: B.dct_dp_compress_batched(table, ws_b),
+            f"one call per layer ({len(sizes)} calls)": lambda: [B.dct_dp_compress(
+                a["grad"], a["residual"], a["n"], a["tau"], None, a["idx_out"], a["val_out"], a["capacity"],
+                a["result"], ws_1) for a in layers],
+        }
+        for name, fn in variants.items():
+            for phase in range(2):
+                e_all.zero_()
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                b.synchronize()
+            ms = a.elapsed_time(b)
+            print(f"compress_layers, {name}: {ms:.4f} ms, {12 * args.n / ms / 1e6:.1f} GB/s algorithmic")
+        return
 
     if args.entry in ("select", "compress", "decompress"):
         n = args.n

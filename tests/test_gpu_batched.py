@@ -1,0 +1,69 @@
+"""dct_dp_compress_batched: every layer of a batched call must come out exactly as the oracle's (and the
+single-vector call's) result for that layer -- own threshold, own error, own output, own counts."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2010_08899_b200 import binding as B
+from paper_2010_08899_b200 import inputs
+from tests import _gpu as G
+from tests._util import bits32
+
+pytestmark = pytest.mark.gpu
+
+
+def _make_layers(sizes, seed, misalign=()):
+    layers = []
+    for j, n in enumerate(sizes):
+        g = inputs.dp_gaussian(n, seed + 3 * j, G.DEV) * (0.1 + j % 5)
+        e = inputs.dp_gaussian(n, seed + 3 * j + 1, G.DEV) * 0.2
+        if j in misalign:
+            g, e = G.offset_copy(g, 1), G.offset_copy(e, 3)
+        k = max(1, n // (20 + 7 * (j % 4)))
+        tau, sel = G.select(g, e, k)
+        cap = n if j % 3 else max(1, k // 2)                 # every third layer overflows its capacity
+        budget = None if j % 2 else torch.tensor([k - sel.n_gt], dtype=torch.int64, device=G.DEV)
+        layers.append(dict(grad=g, residual=e, n=n, tau=tau.clone(), tie_budget=budget, capacity=cap,
+                           idx_out=torch.full((cap + 8,), -7, dtype=torch.int32, device=G.DEV),
+                           val_out=torch.full((cap + 8,), -7.0, device=G.DEV), result=B.new_result()))
+    return layers
+
+
+@pytest.mark.parametrize("sizes,misalign", [
+    ([1], ()), ([5000], ()), ([4096, 4096], ()),
+    ([131072, 16384, 1048576, 524288, 131072, 256, 3, 8191, 12289], ()),        # DLRM-like mix plus odd sizes
+    ([70001, 4096 * 3, 100, 262144 + 5, 9999], (0, 3)),                         # some layers not 16-byte aligned
+    ([(1 << 20) + 17] * 3 + [64] * 40, (41,)),
+])
+def test_batched_equals_per_layer_oracle(sizes, misalign):
+    layers = _make_layers(sizes, 1000 + len(sizes), misalign)
+    want = []
+    for a in layers:
+        e = a["residual"].cpu().numpy().copy()
+        bud = None if a["tie_budget"] is None else int(a["tie_budget"].item())
+        want.append((oracle.dp_compress(a["grad"].cpu().numpy(), e, a["tau"].cpu().numpy()[0], bud, a["capacity"]), e))
+    ws = B.new_workspace(B.dct_dp_compress_batched_workspace_bytes(sizes))
+    ws.fill_(0xAB)                                            # stale workspace contents must not matter
+    B.dct_dp_compress_batched(layers, ws)
+    for a, (w, e_want) in zip(layers, want):
+        r = B.read_result(a["result"])
+        cap = a["capacity"]
+        assert (r.count, r.needed) == (w.count, w.needed)
+        assert r.status == (B.DCT_ERR_CAPACITY if w.needed > cap else B.DCT_OK)
+        assert np.array_equal(a["idx_out"][:r.count].cpu().numpy(), w.idx)
+        assert np.array_equal(bits32(a["val_out"][:r.count].cpu().numpy()), bits32(w.val))
+        assert bool((a["idx_out"][r.count:] == -7).all()) and bool((a["val_out"][r.count:] == -7.0).all())
+        assert np.array_equal(bits32(a["residual"].cpu().numpy()), bits32(e_want))
+
+
+def test_batched_rejects_bad_layers_on_the_host():
+    layers = _make_layers([5000, 6000], 7)
+    ws = B.new_workspace(B.dct_dp_compress_batched_workspace_bytes([5000, 6000]))
+    with pytest.raises(B.DctError):
+        B.dct_dp_compress_batched(layers, ws[:256])
+    bad = dict(layers[1])
+    bad["residual"] = bad["grad"]                              # aliasing
+    with pytest.raises(B.DctError):
+        B.dct_dp_compress_batched([layers[0], bad], ws)
+    assert B.dct_dp_compress_batched_workspace_bytes([0]) == 0
