@@ -213,7 +213,7 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 }
 
 // ------------------------------------------------------------------------------------------
-// bf16 fast path: one warp per row, d = 256 * E8 <= 4096, rows on 16-byte boundaries
+// bf16 fast path: one warp per row, d = 256 * E8 <= 4096 (common widths are instantiated), rows on 16-byte boundaries
 // ------------------------------------------------------------------------------------------
 // Lane l owns the E = d/32 consecutive columns [l E, (l+1) E): every "how many before me" question
 // is then one warp scan.  The row is brought in by 32 bulk asynchronous copies (one span per lane,
@@ -832,11 +832,18 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
     // general kernel.
     if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 &&
         ((k <= 224 && k <= d / 8) || (k > 224 && k <= 448 && k <= d / 4))) {
-        switch (d) {   // warp-per-row path: d = 256 * 2^j
+        switch (d) {   // warp-per-row path: d = 256 * E8 for the instantiated E8
             case 256: return launch_fwd_bf16_warp<1>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             case 512: return launch_fwd_bf16_warp<2>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 768: return launch_fwd_bf16_warp<3>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             case 1024: return launch_fwd_bf16_warp<4>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 1280: return launch_fwd_bf16_warp<5>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 1536: return launch_fwd_bf16_warp<6>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 1792: return launch_fwd_bf16_warp<7>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             case 2048: return launch_fwd_bf16_warp<8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 2560: return launch_fwd_bf16_warp<10>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 3072: return launch_fwd_bf16_warp<12>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            case 3584: return launch_fwd_bf16_warp<14>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             case 4096: return launch_fwd_bf16_warp<16>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             default: break;
         }

@@ -141,3 +141,14 @@ def test_mp_bf16_rows_with_wildly_different_scales():
     gx = inputs.mp_gradients(rows, d, 79, dtype=torch.bfloat16, device=G.DEV)
     for kk in (k, 64, 256):
         _compare_fwd_bwd(x, gx, d, kk)
+
+
+@pytest.mark.parametrize("d", [768, 1280, 1536, 1792, 2560, 3072, 3584])
+def test_mp_bf16_widths_that_are_not_powers_of_two(d):
+    rows = 300
+    x = inputs.mp_activations(rows, d, 11 + d, dtype=torch.bfloat16, device=G.DEV, col_scale_seed=12 + d)
+    x[7] = 0
+    x[8] = 1.0
+    gx = inputs.mp_gradients(rows, d, 13 + d, dtype=torch.bfloat16, device=G.DEV)
+    for k in (1, d // 20, d // 10, d // 8, d // 5):
+        _compare_fwd_bwd(x, gx, d, k)
