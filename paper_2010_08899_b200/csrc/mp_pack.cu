@@ -215,18 +215,24 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 // ------------------------------------------------------------------------------------------
 // bf16 fast path: one warp per row, d = 256 * E8 <= 4096 (common widths are instantiated), rows on 16-byte boundaries
 // ------------------------------------------------------------------------------------------
-// Lane l owns the E = d/32 consecutive columns [l E, (l+1) E): every "how many before me" question
-// is then one warp scan.  The row is brought in by 32 bulk asynchronous copies (one span per lane,
-// spans padded by 16 bytes in shared memory so that 128-bit reads of different lanes fall into
-// different banks); the next row is requested as soon as the current one has been filtered.
-//   A  lower bound `low` for tau_i: the k-th largest of the maxima of the d/8 aligned 8-element
-//      leaves.  At least k elements are >= low, and fewer than k leaves hold anything above it.
-//   B  candidates (key >= low; typically ~1.2 k of them) are compacted, in column order, into a list.
-//   C  exact k-th largest of the candidates: radix select, exponent byte then mantissa.
-//   D  the kept columns (key > tau_i, then the lowest-column ties) leave the list in order.
-// If the candidates do not fit the list (heavy ties at the bound, or k larger than the number of leaves
-// and a short list), the row takes a slow general path: tau_i is found bit by bit by counting over the
-// row, and the output is written straight from the row.
+// One bulk asynchronous copy brings a row into shared memory exactly as it lies in HBM; the next row is
+// requested as soon as the candidates of the current one sit in registers.
+//   A  a lower bound `low` for tau_i.  First guess: the previous row's tau_i minus a margin (thresholds of
+//      neighbouring samples are close).  If that leaves fewer than k or too many candidates, the exact
+//      bound takes over: the k-th largest of the maxima of the aligned 8-element (or 4-element) leaves --
+//      at least k elements are >= it, and fewer than k leaves hold anything above it.
+//   B  one pass over the row (lane l reads the 16-byte units l, l + 32, ...: conflict-free for every width)
+//      writes one flag per column, key >= low, into a bit table in column order; a warp scan over the
+//      per-lane counts gives the number of candidates before every table word.
+//   C  the candidates (typically ~1.3 k) are dealt out evenly, in column order, ceil(n/32) to a lane, which
+//      finds its first one by bisection over the running counts and walks the table from there.
+//   D  exact k-th largest of the candidates: a 64-bin histogram just above the bound, else a radix select
+//      (exponent byte, then mantissa).
+//   E  the kept entries (key > tau_i, then the lowest-column ties) go, in column order, through k staging
+//      slots to coalesced stores.
+// If the candidates do not fit the registers (heavy ties at the bound, or k larger than the number of
+// leaves), the row takes a slow general path: tau_i is found bit by bit by counting over the row, and the
+// output is written straight from the row.
 #ifndef DCT_FWD_MAX_WARPS
 #define DCT_FWD_MAX_WARPS 24
 #endif
@@ -238,10 +244,8 @@ template <int E8> struct WarpRowLayout {
     static constexpr uint32_t E = E8 * 8u, D = E * 32u;
     static constexpr uint32_t kSpanBytes = E * 2u;           // the row lies in shared memory as it does in HBM
     static constexpr uint32_t kRowBytes = 32u * kSpanBytes;
-    // Lane l reads its 16-byte units in the rotated order (c + l) mod E8: with spans of 256 bytes the
-    // eight lanes of a quarter-warp then hit eight different bank groups instead of one.
-    static constexpr bool kRotate = (E8 == 16);
-    static constexpr uint32_t kMaskWords = (E8 + 3) / 4;     // 32-bit mask words per lane
+    static constexpr uint32_t kRowWords = 8u * E8;           // 32-bit candidate-mask words of a row (one bit per column)
+    static constexpr uint32_t kMaskWords = (E8 + 3) / 4;     // mask words a lane looks after: lane l has words [l kMaskWords, (l+1) kMaskWords)
     static constexpr uint32_t kTableWords = 32u * kMaskWords;
     // per warp: row | scratch | mbarrier.  The scratch is used in turn, never at the same time, as the
     // leaf histogram, the candidate-mask and running-count tables, the select histogram and the k
@@ -409,7 +413,6 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
                              dct_result_t* __restrict__ result) {
     using Lay = WarpRowLayout<E8>;
-    constexpr uint32_t E = Lay::E;
     constexpr int kMaskWords = Lay::kMaskWords;
     constexpr uint32_t kPerLane = PL, kRound = 32u * kPerLane;   // candidates a lane holds in registers at a time
     constexpr bool kFineLeaves = FwdVariant<PL>::kFineLeaves;
@@ -451,8 +454,9 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             bulk_load(base, x + static_cast<size_t>(r) * ld, Lay::D * 2u, bar);
         }
     };
-    // the lane's c-th read of a pass: unit (c + lane) mod E8 of its span when rotating, unit c otherwise
-    auto unit_of = [&](int c) -> uint32_t { return Lay::kRotate ? ((c + lane) & (E8 - 1)) : static_cast<uint32_t>(c); };
+    // In the passes over the whole row lane l reads the 16-byte units l, l + 32, l + 64, ...: the 32 lanes of a
+    // 128-bit load then touch 512 consecutive bytes (no bank conflict for any row width).
+    const unsigned char* unit0 = base + lane * 16u;
     auto release_row = [&](uint32_t row) {   // the row buffer is no longer needed: request the next row
         __syncwarp();
         fence_proxy_async_smem();
@@ -480,7 +484,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             uint32_t top = 0;
 #pragma unroll
             for (int c = 0; c < E8; ++c) {
-                const uint4 v = *reinterpret_cast<const uint4*>(span + unit_of(c) * 16);
+                const uint4 v = *reinterpret_cast<const uint4*>(unit0 + c * 512);
                 const __nv_bfloat162 m2 = __hmax2(__hmax2(__habs2(as_bf162(v.x)), __habs2(as_bf162(v.y))),
                                                   __hmax2(__habs2(as_bf162(v.z)), __habs2(as_bf162(v.w))));
                 const uint32_t m = as_u32(m2);
@@ -528,25 +532,30 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         uint32_t masks[kMaskWords];
         uint32_t n_mine = 0, incl = 0, n_cand = 0;
         auto build_masks = [&](uint32_t bound) {
-#pragma unroll
-            for (int i = 0; i < kMaskWords; ++i) masks[i] = 0;
+            // unit u = 32 c + lane covers columns 8 u .. 8 u + 7: its 8 flags are byte u of the mask table, which
+            // therefore holds one bit per column, in column order
             const __nv_bfloat162 low2 = as_bf162(bound | (bound << 16));
+            unsigned char* tab8 = reinterpret_cast<unsigned char*>(mask_tab) + lane;
 #pragma unroll
-            for (int c = 0; c < E8; ++c) {
-                const uint32_t m = mask8_ge_filter(*reinterpret_cast<const uint4*>(span + unit_of(c) * 16), low2);
-                masks[c / 4] |= m << (8 * (c % 4));
+            for (int c = 0; c < E8; ++c)
+                tab8[c * 32] = static_cast<unsigned char>(
+                    mask8_ge_filter(*reinterpret_cast<const uint4*>(unit0 + c * 512), low2));
+            __syncwarp();
+            // the lane's own words: columns 32 kMaskWords lane onwards (words past the end of the row are empty)
+            if (kMaskWords == 4) {
+                const uint4 t = reinterpret_cast<const uint4*>(mask_tab)[lane];
+                masks[0] = t.x; masks[1 % kMaskWords] = t.y; masks[2 % kMaskWords] = t.z; masks[3 % kMaskWords] = t.w;
+            } else if (kMaskWords == 2) {
+                const uint2 t = reinterpret_cast<const uint2*>(mask_tab)[lane];
+                masks[0] = t.x; masks[1 % kMaskWords] = t.y;
+            } else {
+#pragma unroll
+                for (int i = 0; i < kMaskWords; ++i) masks[i] = mask_tab[lane * kMaskWords + i];
             }
-            if (Lay::kRotate) {
-                // byte c of the 128-bit mask belongs to unit (c + lane) mod 16: rotate left by 8 * (lane mod 16)
-                // bits so that byte u belongs to unit u (column order)
-                const uint32_t words = (lane >> 2) & 3u, bits = (lane & 3u) * 8u;
-                uint32_t w0 = masks[0], w1 = masks[1 % kMaskWords], w2 = masks[2 % kMaskWords], w3 = masks[3 % kMaskWords];
-                if (words & 1u) { const uint32_t t = w3; w3 = w2; w2 = w1; w1 = w0; w0 = t; }
-                if (words & 2u) { uint32_t t = w0; w0 = w2; w2 = t; t = w1; w1 = w3; w3 = t; }
-                masks[0] = __funnelshift_l(w3, w0, bits);
-                masks[1 % kMaskWords] = __funnelshift_l(w0, w1, bits);
-                masks[2 % kMaskWords] = __funnelshift_l(w1, w2, bits);
-                masks[3 % kMaskWords] = __funnelshift_l(w2, w3, bits);
+            if (Lay::kRowWords != Lay::kTableWords) {
+#pragma unroll
+                for (int i = 0; i < kMaskWords; ++i)
+                    if (lane * kMaskWords + i >= Lay::kRowWords) masks[i] = 0u;
             }
             n_mine = 0;
 #pragma unroll
@@ -568,7 +577,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             if (!use_guess || (n_cand >= k && n_cand <= kRound)) break;
             use_guess = false;
         }
-        if (!have_bound || n_cand > kRound) {
+        if (!have_bound || n_cand > kRound || low == 0) {
             mp_row_slow_path<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
             release_row(row);
             continue;
@@ -581,15 +590,18 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             uint32_t before = incl - n_mine;
 #pragma unroll
             for (int i = 0; i < kMaskWords; ++i) {
-                mask_tab[lane * kMaskWords + i] = masks[i];
+                if (Lay::kRowWords != Lay::kTableWords) mask_tab[lane * kMaskWords + i] = masks[i];   // zero the padding words
                 count_tab[lane * kMaskWords + i] = before;
                 before += __popc(masks[i]);
             }
         }
         __syncwarp();
+        // Every lane takes per_lane = ceil(n_cand / 32) consecutive candidates (the last lanes fewer or none).  An unused
+        // slot holds 0: its key is below the bound (low >= 1 here), so the select and the emit skip it unaided.
         uint32_t ent[kPerLane];
-        const uint32_t first = lane * kPerLane;                 // rank of the lane's first candidate
-        const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < kPerLane ? n_cand - first : kPerLane);
+        const uint32_t per_lane = (n_cand + 31u) >> 5;
+        const uint32_t first = lane * per_lane;                 // rank of the lane's first candidate
+        const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < per_lane ? n_cand - first : per_lane);
         {
             uint32_t word = 0, m = 0;
             if (nvalid) {
@@ -607,7 +619,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 ent[i] = 0;
                 if (static_cast<uint32_t>(i) < nvalid) {
                     while (m == 0) m = mask_tab[++word];
-                    const uint32_t col = (word / kMaskWords) * E + (word % kMaskWords) * 32u + (__ffs(m) - 1);
+                    const uint32_t col = word * 32u + (__ffs(m) - 1);
                     m &= m - 1;
                     ent[i] = reinterpret_cast<const uint16_t*>(base)[col] | (col << 16);
                 }
@@ -618,7 +630,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         // ---- C: k-th largest of the candidates --------------------------------------------------
         uint32_t tau_key = 0, take = 0;
         bool found = false;
-        if (low != 0) {
+        {
             // tau_i is the (n_cand - k + 1)-th smallest candidate.  Usually it lies within 64 keys of the
             // bound: a 64-bin histogram of the candidates in [low, low + 64), walked from the bottom, finds it.
             const uint32_t drop = n_cand - k;                 // candidates to discard, smallest first
@@ -628,7 +640,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 #pragma unroll
             for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
                 const uint32_t rel = (ent[i] & 0x7FFFu) - low;
-                if (static_cast<uint32_t>(i) < nvalid && rel < 64u) atomicAdd(&hist[rel], 1u);
+                if (rel < 64u) atomicAdd(&hist[rel], 1u);
             }
             __syncwarp();
             const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
@@ -685,15 +697,14 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 #pragma unroll
             for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
                 const uint32_t key = ent[i] & 0x7FFFu;
-                if (static_cast<uint32_t>(i) < nvalid) counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
+                counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
             }
             const uint32_t before = warp_inclusive_sum(counts) - counts;
             uint32_t g_at = before >> 16, e_at = before & 0xFFFFu;
 #pragma unroll
             for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
                 const uint32_t key = ent[i] & 0x7FFFu;
-                const bool live = static_cast<uint32_t>(i) < nvalid;
-                const bool is_gt = live && key > tau_key, is_eq = live && key == tau_key;
+                const bool is_gt = key > tau_key, is_eq = key == tau_key;
                 if (is_gt || (is_eq && e_at < take)) stage[g_at + (e_at < take ? e_at : take)] = ent[i];
                 g_at += is_gt ? 1u : 0u;
                 e_at += is_eq ? 1u : 0u;
