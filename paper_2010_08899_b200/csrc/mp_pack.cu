@@ -285,6 +285,12 @@ __device__ __forceinline__ uint32_t mask8_ge_exact(uint4 v, uint32_t low) {
     return (m | (m >> 15)) & 0xFFu;
 }
 
+// v = *(uint2*)shared_address if p (a predicated load: no branch)
+__device__ __forceinline__ void lds64_if(uint2& v, uint32_t shared_address, bool p) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %3, 0;\n\t@q ld.shared.v2.u32 {%0, %1}, [%2];\n\t}"
+                 : "+r"(v.x), "+r"(v.y) : "r"(shared_address), "r"(static_cast<uint32_t>(p)));
+}
+
 __device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v) {
     const uint32_t lane = lane_id();
 #pragma unroll
@@ -423,8 +429,8 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     unsigned char* base = smem_raw + warp * Lay::warp_bytes(k);
     unsigned char* span = base + lane * Lay::kSpanBytes;
     uint32_t* scratch = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
-    uint32_t* mask_tab = scratch;                             // candidate masks, column order
-    uint32_t* count_tab = scratch + Lay::kTableWords;         // candidates before each mask word
+    uint32_t* mask_tab = scratch;                             // one bit per column (key >= bound), column order
+    uint2* table = reinterpret_cast<uint2*>(scratch);        // per mask word: {mask, running count and link}, built after the bit table
     uint32_t* hist = scratch;                                 // histograms (before / after the tables are in use)
     uint32_t* stage = scratch;                                // the k kept entries, column order (last use)
     uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Lay::scratch_words(k));
@@ -583,15 +589,34 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             continue;
         }
 
-        // ---- candidates into registers, evenly: lane q takes candidates kPerLane q .. kPerLane q + kPerLane - 1 ----
-        // The masks go to a table in column order together with the number of candidates before each mask
-        // word; a lane finds the word that holds its first candidate by bisection and walks on from there.
+        // ---- candidates into registers, evenly -------------------------------------------------------
+        // Every table word becomes an entry {mask, candidates before it << 16 | index of the next non-empty
+        // word}.  A lane finds the word that holds its first candidate by bisection over the running counts and
+        // walks on from there; the link takes it over any run of empty words in one step.
+        uint32_t first_word;                                    // the row's first non-empty word
         {
+            const uint32_t wbase = lane * kMaskWords;
+            uint32_t my_first = Lay::kTableWords;               // the lane's first non-empty word
+#pragma unroll
+            for (int i = kMaskWords - 1; i >= 0; --i)
+                if (masks[i]) my_first = wbase + i;
+            // after the last non-empty word the link wraps to the first one: a walk that runs past its candidates
+            // (unused slots) then still meets a non-empty word, and its result is discarded
+            const uint32_t holders = __ballot_sync(0xFFFFFFFFu, n_mine != 0);
+            const uint32_t later = holders & (0xFFFFFFFEu << lane);
+            first_word = __shfl_sync(0xFFFFFFFFu, my_first, __ffs(holders) - 1);
+            // (all lanes take part in the shuffle; the source lane is the next holder, or the first one to wrap)
+            uint32_t link = __shfl_sync(0xFFFFFFFFu, my_first, __ffs(later ? later : holders) - 1);
+            uint32_t next_of[kMaskWords];
+#pragma unroll
+            for (int i = kMaskWords - 1; i >= 0; --i) {
+                next_of[i] = link;
+                if (masks[i]) link = wbase + i;
+            }
             uint32_t before = incl - n_mine;
 #pragma unroll
             for (int i = 0; i < kMaskWords; ++i) {
-                if (Lay::kRowWords != Lay::kTableWords) mask_tab[lane * kMaskWords + i] = masks[i];   // zero the padding words
-                count_tab[lane * kMaskWords + i] = before;
+                table[wbase + i] = make_uint2(masks[i], (before << 16) | next_of[i]);
                 before += __popc(masks[i]);
             }
         }
@@ -603,26 +628,35 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         const uint32_t first = lane * per_lane;                 // rank of the lane's first candidate
         const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < per_lane ? n_cand - first : per_lane);
         {
-            uint32_t word = 0, m = 0;
+            uint32_t word = 0, m = 0, link = first_word;
             if (nvalid) {
-                uint32_t lo = 0, hi = Lay::kTableWords - 1;         // largest word with count_tab[word] <= first
+                uint32_t lo = 0, hi = Lay::kTableWords - 1;         // largest word with (candidates before it) <= first
+                const uint32_t limit = (first + 1u) << 16;
                 while (lo < hi) {
                     const uint32_t mid = (lo + hi + 1) >> 1;
-                    if (count_tab[mid] <= first) lo = mid; else hi = mid - 1;
+                    if (table[mid].y < limit) lo = mid; else hi = mid - 1;
                 }
+                const uint2 e = table[lo];
                 word = lo;
-                m = mask_tab[word];
-                for (uint32_t skip = first - count_tab[word]; skip; --skip) m &= m - 1;
+                m = e.x;
+                link = e.y & 0xFFFFu;
+                for (uint32_t skip = first - (e.y >> 16); skip; --skip) m &= m - 1;
             }
+            // `ahead` is the entry the walk moves to when the current word runs out; it is fetched when the walk
+            // arrives at a word, long before it is needed
+            uint2 ahead = table[link];
+            const uint32_t table_addr = smem_addr(table);
 #pragma unroll
             for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                ent[i] = 0;
-                if (static_cast<uint32_t>(i) < nvalid) {
-                    while (m == 0) m = mask_tab[++word];
-                    const uint32_t col = word * 32u + (__ffs(m) - 1);
-                    m &= m - 1;
-                    ent[i] = reinterpret_cast<const uint16_t*>(base)[col] | (col << 16);
-                }
+                const bool advance = (m == 0);
+                m = advance ? ahead.x : m;
+                word = advance ? link : word;
+                link = advance ? (ahead.y & 0xFFFFu) : link;
+                lds64_if(ahead, table_addr + link * 8u, advance);
+                const uint32_t col = word * 32u + (__ffs(m) - 1);
+                m &= m - 1;
+                const uint32_t e = reinterpret_cast<const uint16_t*>(base)[col] | (col << 16);
+                ent[i] = static_cast<uint32_t>(i) < nvalid ? e : 0u;
             }
         }
         release_row(row);
