@@ -668,13 +668,15 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             // tau_i is the (n_cand - k + 1)-th smallest candidate.  Usually it lies within 64 keys of the
             // bound: a 64-bin histogram of the candidates in [low, low + 64), walked from the bottom, finds it.
             const uint32_t drop = n_cand - k;                 // candidates to discard, smallest first
+            // (everything beyond the window, unused slots included, goes to a bin of the lane's own: no branch)
             hist[lane] = 0;
             hist[lane + 32] = 0;
+            hist[lane + 64] = 0;
             __syncwarp();
 #pragma unroll
             for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
                 const uint32_t rel = (ent[i] & 0x7FFFu) - low;
-                if (rel < 64u) atomicAdd(&hist[rel], 1u);
+                atomicAdd(&hist[rel < 64u ? rel : 64u + lane], 1u);
             }
             __syncwarp();
             const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
@@ -734,13 +736,15 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
             }
             const uint32_t before = warp_inclusive_sum(counts) - counts;
-            uint32_t g_at = before >> 16, e_at = before & 0xFFFFu;
+            uint32_t e_at = before & 0xFFFFu;                 // ties before this entry
+            uint32_t pos = (before >> 16) + (e_at < take ? e_at : take);   // kept entries before it
 #pragma unroll
             for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
                 const uint32_t key = ent[i] & 0x7FFFu;
-                const bool is_gt = key > tau_key, is_eq = key == tau_key;
-                if (is_gt || (is_eq && e_at < take)) stage[g_at + (e_at < take ? e_at : take)] = ent[i];
-                g_at += is_gt ? 1u : 0u;
+                const bool is_eq = key == tau_key;
+                const bool keep = key > tau_key || (is_eq && e_at < take);
+                if (keep) stage[pos] = ent[i];
+                pos += keep ? 1u : 0u;
                 e_at += is_eq ? 1u : 0u;
             }
         }
