@@ -366,6 +366,90 @@ DCT_API dct_status_t dct_dp_compress_static(
     int32_t* idx_out, float* val_out, uint64_t capacity,
     dct_result_t* result, dct_stream_t stream);
 
+/* ------------------------------------------------------------------------- *
+ * Threshold diagnostics: the quantities behind the paper's threshold plots.
+ * None of them changes a gradient, a residual or an activation.
+ * ------------------------------------------------------------------------- */
+
+#define DCT_DIAG_MAX_QUANTILES 4u
+
+/*
+ * dct_threshold_select_multi -- the top-k thresholds of one gradient vector at
+ * several sparsity levels at once (Sec. 2.1, the figure that plots the top-K
+ * threshold at 75 / 90 / 95 % sparsity over the iterations and motivates the
+ * threshold life-span L).
+ *
+ * For every q < m:  tau_out[q] = ks[q]-th largest |fl32(grad + residual)|, exactly
+ * as dct_threshold_select would return it for k = ks[q], with
+ * results[q].n_gt / n_eq / status filled the same way.  All m thresholds come
+ * out of the same three streaming passes over the vector (one shared histogram
+ * of the leading digit, then one histogram per threshold), so the cost does not
+ * grow with m and does not depend on how dense the quantiles are.
+ *
+ *   grad, residual  [n] fp32 device, read only; residual may be NULL.
+ *   ks              [m] HOST array of survivor targets, 1 <= ks[q] <= n, any order.
+ *   m               1 .. DCT_DIAG_MAX_QUANTILES.
+ *   tau_out         [m] fp32 device.   results  [m] dct_result_t device.
+ *   workspace       device, 256-byte aligned,
+ *                   >= dct_threshold_select_multi_workspace_bytes(n, m); caller owned.
+ * Errors: as dct_threshold_select (DCT_ERR_INVALID_ARG also for m out of range).
+ */
+DCT_API size_t dct_threshold_select_multi_workspace_bytes(uint64_t n, uint32_t m);
+DCT_API dct_status_t dct_threshold_select_multi(
+    const float* grad, const float* residual, uint64_t n,
+    const uint64_t* ks, uint32_t m,
+    float* tau_out, dct_result_t* results,
+    void* workspace, size_t workspace_bytes, dct_stream_t stream);
+
+/*
+ * dct_mp_threshold_mean -- the mean over the batch of the per-sample top-k
+ * thresholds, (1/B) sum_i tau_i, at several sparsity levels, measured without
+ * sparsifying anything (Sec. 2.2, the figure that plots this mean at 75 / 90 /
+ * 95 % sparsity with and without DCT-MP).
+ *
+ * For every q < m and row i:  tau_out[q*rows + i] = ks[q]-th largest |x[i, :d]|
+ * (the tau_i of dct_mp_topk_pack_fwd for k = ks[q], bit for bit), and
+ * mean_out[q] = (sum_i tau_out[q*rows + i]) / rows in binary64.  The sum is
+ * accumulated in binary64 in a fixed order (the same input always gives the same
+ * bits); it is the exact sum whenever that is representable, which holds for
+ * every batch whose thresholds span fewer than 53 - 24 - log2(rows) binades,
+ * and is otherwise within rows * 2^-53 relative of it.  Each row is read from
+ * HBM once, whatever m is.
+ *
+ *   x_act     [rows, ld] fp32 or bf16 device, read only.
+ *   ks        [m] HOST array, 1 <= ks[q] <= d.   m  1 .. DCT_DIAG_MAX_QUANTILES.
+ *   mean_out  [m] binary64 device.
+ *   tau_out   [m*rows] dtype device (required: it is also the scratch of the mean).
+ * Limits and errors as dct_mp_topk_pack_fwd.
+ */
+DCT_API dct_status_t dct_mp_threshold_mean(
+    const void* x_act, dct_dtype_t dtype, uint32_t rows, uint32_t d, uint32_t ld,
+    const uint32_t* ks, uint32_t m,
+    double* mean_out, void* tau_out, dct_stream_t stream);
+
+/*
+ * dct_dp_drift_check -- has the survivor count of a compress call drifted away
+ * from the target k while the threshold is being reused?  (Sec. 2.1 reuses tau
+ * for L iterations because it moves little around its running mean; this is the
+ * guard for the case where it does move.  The paper states the observation, not
+ * a monitor: the rule below is this library's.)
+ *
+ * Reads compress_result->needed (the true survivor count of the last
+ * dct_dp_compress on this stream) and writes
+ *   *flag_out = 1  if needed * ratio_den > k * ratio_num   (too dense: tau too low),
+ *               2  if needed * ratio_num < k * ratio_den   (too sparse: tau too high),
+ *               0  otherwise,
+ * i.e. 0 while k / ratio <= needed <= k * ratio with ratio = ratio_num / ratio_den >= 1.
+ * Everything stays on the device and on the stream, so a trainer can branch on the
+ * flag (or capture the check in a graph) without a host round trip.
+ *   compress_result  device;  flag_out  device uint32;  k >= 1;
+ *   ratio_num >= ratio_den >= 1 (else DCT_ERR_INVALID_ARG).
+ */
+DCT_API dct_status_t dct_dp_drift_check(
+    const dct_result_t* compress_result, uint64_t k,
+    uint32_t ratio_num, uint32_t ratio_den,
+    uint32_t* flag_out, dct_stream_t stream);
+
 /*
  * Testing knobs (process-wide, not for production use).  spin_limit is the
  * number of polls a device-side wait may take before it gives up with

@@ -42,7 +42,9 @@ def _load():
         _lib = ctypes.CDLL(build())
         for name in ("oracle_dp_select", "oracle_dp_compress", "oracle_mp_fwd_f32",
                      "oracle_mp_fwd_bf16", "oracle_mp_bwd_f32", "oracle_mp_bwd_bf16",
-                     "oracle_dp_decompress", "oracle_mp_unpack_f32", "oracle_mp_unpack_bf16"):
+                     "oracle_dp_decompress", "oracle_mp_unpack_f32", "oracle_mp_unpack_bf16",
+                     "oracle_dp_select_multi", "oracle_mp_threshold_mean_f32", "oracle_mp_threshold_mean_bf16",
+                     "oracle_dp_drift_flag"):
             getattr(_lib, name).restype = ctypes.c_int
     return _lib
 
@@ -195,3 +197,60 @@ def mp_unpack(cols: np.ndarray, vals: np.ndarray, d: int, ld: Optional[int] = No
     if rc:
         raise ValueError(f"oracle_mp_unpack: invalid argument (rc={rc})")
     return dense
+
+
+class SelectMultiResult(NamedTuple):
+    tau: np.ndarray        # float32 [m]
+    n_gt: np.ndarray       # uint64 [m]
+    n_eq: np.ndarray       # uint64 [m]
+
+
+def dp_select_multi(grad: np.ndarray, residual: Optional[np.ndarray], ks) -> SelectMultiResult:
+    """Top-k thresholds of one vector at several survivor targets (Sec. 2.1, threshold plot)."""
+    lib = _load()
+    _check(grad, np.float32, "grad")
+    if residual is not None:
+        _check(residual, np.float32, "residual")
+    m = len(ks)
+    ks_a = np.asarray(ks, dtype=np.uint64)
+    tau = np.zeros(m, dtype=np.float32)
+    n_gt = np.zeros(m, dtype=np.uint64)
+    n_eq = np.zeros(m, dtype=np.uint64)
+    rc = lib.oracle_dp_select_multi(_ptr(grad), _ptr(residual), _c_u64(grad.size), _ptr(ks_a), _c_u32(m),
+                                    _ptr(tau), _ptr(n_gt), _ptr(n_eq))
+    if rc != 0:
+        raise ValueError(f"oracle_dp_select_multi: bad arguments ({rc})")
+    return SelectMultiResult(tau, n_gt, n_eq)
+
+
+class ThresholdMeanResult(NamedTuple):
+    mean: np.ndarray       # float64 [m]
+    tau: np.ndarray        # [m, rows], dtype of x
+
+
+def mp_threshold_mean(x: np.ndarray, ks, d: Optional[int] = None) -> ThresholdMeanResult:
+    """(1/B) sum_i tau_i at several sparsity levels, nothing sparsified (Sec. 2.2, threshold plot)."""
+    lib = _load()
+    rows, ld = x.shape
+    d = ld if d is None else d
+    m = len(ks)
+    ks_a = np.asarray(ks, dtype=np.uint32)
+    mean = np.zeros(m, dtype=np.float64)
+    tau = np.zeros((m, rows), dtype=x.dtype)
+    if x.dtype == np.float32:
+        fn = lib.oracle_mp_threshold_mean_f32
+    elif x.dtype == np.uint16:
+        fn = lib.oracle_mp_threshold_mean_bf16
+    else:
+        raise TypeError("x: float32, or uint16 holding bf16 bit patterns")
+    _check(x, x.dtype, "x")
+    rc = fn(_ptr(x), _c_u32(rows), _c_u32(d), _c_u32(ld), _ptr(ks_a), _c_u32(m), _ptr(mean), _ptr(tau))
+    if rc != 0:
+        raise ValueError(f"oracle_mp_threshold_mean: bad arguments ({rc})")
+    return ThresholdMeanResult(mean, tau)
+
+
+def dp_drift_flag(needed: int, k: int, ratio_num: int, ratio_den: int) -> int:
+    """1: survivors above k * ratio; 2: below k / ratio; 0: inside (ratio = ratio_num / ratio_den >= 1)."""
+    lib = _load()
+    return lib.oracle_dp_drift_flag(_c_u64(needed), _c_u64(k), _c_u32(ratio_num), _c_u32(ratio_den))

@@ -284,3 +284,95 @@ int oracle_mp_bwd_bf16(const uint16_t* gx, uint32_t rows, uint32_t d, uint32_t l
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------
+// Threshold diagnostics (the quantities behind the paper's two threshold plots)
+// ---------------------------------------------------------------------------
+namespace {
+
+// tau_i for one row and one sparsity level: the row's magnitudes sorted in
+// descending order, read at position k (Algorithm 2, threshold step).
+template <typename T, typename KeyFn>
+uint32_t row_threshold_key(const T* x, uint32_t d, uint32_t k, KeyFn key) {
+    std::vector<uint32_t> mags(d);
+    for (uint32_t j = 0; j < d; ++j) mags[j] = key(x[j]);
+    std::sort(mags.begin(), mags.end(), [](uint32_t a, uint32_t b) { return a > b; });
+    return mags[k - 1];
+}
+
+inline double value_of_key(float, uint32_t k) { return static_cast<double>(float_of(k)); }
+inline double value_of_key(uint16_t, uint32_t k) { return static_cast<double>(float_of(k << 16)); }
+
+// Sec. 2.2 (the plot of the mean threshold): mean_out[q] = (1/B) sum_i tau_i at
+// sparsity level q, with tau_i the ks[q]-th largest magnitude of row i.  The
+// sum runs over the rows in order, in binary64; nothing is sparsified.
+template <typename T, typename KeyFn, typename FromKey>
+int mp_threshold_mean(const T* x, uint32_t rows, uint32_t d, uint32_t ld, const uint32_t* ks, uint32_t m,
+                      KeyFn key, FromKey from_key, double* mean_out, T* tau_out) {
+    if (x == nullptr || ks == nullptr || mean_out == nullptr || rows == 0 || d == 0 || ld < d) return 1;
+    for (uint32_t q = 0; q < m; ++q) {
+        if (ks[q] == 0 || ks[q] > d) return 1;
+        double sum = 0.0;
+        for (uint32_t i = 0; i < rows; ++i) {
+            const uint32_t tk = row_threshold_key(x + static_cast<uint64_t>(i) * ld, d, ks[q], key);
+            if (tau_out) tau_out[static_cast<uint64_t>(q) * rows + i] = from_key(tk);
+            volatile double s = sum + value_of_key(T(), tk);
+            sum = s;
+        }
+        mean_out[q] = sum / static_cast<double>(rows);
+    }
+    return 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+// Sec. 2.1 (the plot of the top-K threshold at several sparsity levels): the
+// order statistic of Algorithm 1 read at several positions of ONE sorted copy.
+int oracle_dp_select_multi(const float* grad, const float* residual, uint64_t n, const uint64_t* ks, uint32_t m,
+                           float* tau_out, uint64_t* n_gt_out, uint64_t* n_eq_out) {
+    if (grad == nullptr || ks == nullptr || n == 0) return 1;
+    std::vector<uint32_t> sorted(n);
+    for (uint64_t i = 0; i < n; ++i) sorted[i] = key_f32(error_feedback(grad, residual, i));
+    std::sort(sorted.begin(), sorted.end());      // ascending: w_1 <= ... <= w_n
+    for (uint32_t q = 0; q < m; ++q) {
+        if (ks[q] == 0 || ks[q] > n) return 1;
+        const uint32_t tau_key = sorted[n - ks[q]];
+        uint64_t n_gt = 0, n_eq = 0;
+        for (uint64_t i = 0; i < n; ++i) {
+            if (sorted[i] > tau_key) ++n_gt;
+            else if (sorted[i] == tau_key) ++n_eq;
+        }
+        tau_out[q] = float_of(tau_key);
+        if (n_gt_out) n_gt_out[q] = n_gt;
+        if (n_eq_out) n_eq_out[q] = n_eq;
+    }
+    return 0;
+}
+
+int oracle_mp_threshold_mean_f32(const float* x, uint32_t rows, uint32_t d, uint32_t ld, const uint32_t* ks,
+                                 uint32_t m, double* mean_out, float* tau_out) {
+    return mp_threshold_mean<float>(x, rows, d, ld, ks, m, [](float v) { return key_f32(v); },
+                                    [](uint32_t k) { return float_of(k); }, mean_out, tau_out);
+}
+int oracle_mp_threshold_mean_bf16(const uint16_t* x, uint32_t rows, uint32_t d, uint32_t ld, const uint32_t* ks,
+                                  uint32_t m, double* mean_out, uint16_t* tau_out) {
+    return mp_threshold_mean<uint16_t>(x, rows, d, ld, ks, m,
+                                       [](uint16_t v) { return static_cast<uint32_t>(key_bf16(v)); },
+                                       [](uint32_t k) { return static_cast<uint16_t>(k); }, mean_out, tau_out);
+}
+
+// Guard for a reused threshold (Sec. 2.1, threshold life-span): 1 if the survivor
+// count exceeds k * num / den, 2 if it is below k * den / num, 0 otherwise
+// (num / den >= 1; exact integer comparison).  The rule is the library's, not
+// the paper's; the oracle states it so that the device kernel has a definition.
+int oracle_dp_drift_flag(uint64_t needed, uint64_t k, uint32_t num, uint32_t den) {
+    const unsigned __int128 a = static_cast<unsigned __int128>(needed) * den, b = static_cast<unsigned __int128>(k) * num;
+    const unsigned __int128 c = static_cast<unsigned __int128>(needed) * num, e = static_cast<unsigned __int128>(k) * den;
+    if (a > b) return 1;
+    if (c < e) return 2;
+    return 0;
+}
+
+}  // extern "C"

@@ -31,6 +31,8 @@ EXPORTED_SYMBOLS = (
     "dct_dp_compress_static", "dct_dp_decompress", "dct_mp_unpack",
     "dct_dp_select_compress", "dct_dp_select_compress_workspace_bytes",
     "dct_dp_compress_batched", "dct_dp_compress_batched_workspace_bytes",
+    "dct_threshold_select_multi", "dct_threshold_select_multi_workspace_bytes",
+    "dct_mp_threshold_mean", "dct_dp_drift_check",
 )
 
 _vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
@@ -96,6 +98,14 @@ def lib() -> ctypes.CDLL:
     L.dct_mp_pack_host.restype = _int
     L.dct_mp_pack_host.argtypes = [_vp, _vp, _vp, _vp, _int, _u32, _u32, _u32, _u32,
                                    _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+    L.dct_threshold_select_multi_workspace_bytes.restype = _sz
+    L.dct_threshold_select_multi_workspace_bytes.argtypes = [_u64, _u32]
+    L.dct_threshold_select_multi.restype = _int
+    L.dct_threshold_select_multi.argtypes = [_vp, _vp, _u64, _vp, _u32, _vp, _vp, _vp, _sz, _vp]
+    L.dct_mp_threshold_mean.restype = _int
+    L.dct_mp_threshold_mean.argtypes = [_vp, _int, _u32, _u32, _u32, _vp, _u32, _vp, _vp, _vp]
+    L.dct_dp_drift_check.restype = _int
+    L.dct_dp_drift_check.argtypes = [_vp, _u64, _u32, _u32, _vp, _vp]
     L.dct_debug_configure.restype = None
     L.dct_debug_configure.argtypes = [_u32, _u32]
     _lib = L
@@ -438,3 +448,61 @@ def dct_dp_compress_batched(layers, workspace, stream=None) -> None:
     _need(workspace, torch.uint8, "workspace")
     _check("dct_dp_compress_batched",
            lib().dct_dp_compress_batched(table, len(table), _p(workspace), workspace.numel(), _stream(stream)))
+
+
+# ----------------------------------------------------------------------------
+# threshold diagnostics
+# ----------------------------------------------------------------------------
+
+DCT_DIAG_MAX_QUANTILES = 4
+
+
+def dct_threshold_select_multi_workspace_bytes(n: int, m: int) -> int:
+    return lib().dct_threshold_select_multi_workspace_bytes(n, m)
+
+
+def dct_threshold_select_multi(grad, residual, n, ks, tau_out, results, workspace, stream=None) -> None:
+    """Thresholds of one vector for the survivor targets ``ks`` (a host sequence) out of the same three
+    passes; tau_out [m] fp32 and results [m * 5] int64 (one dct_result_t per rank) are device tensors."""
+    _need(grad, torch.float32, "grad")
+    if residual is not None:
+        _need(residual, torch.float32, "residual")
+    _need(tau_out, torch.float32, "tau_out")
+    _need(results, torch.int64, "results")
+    _need(workspace, torch.uint8, "workspace")
+    m = len(ks)
+    if grad.numel() < n or (residual is not None and residual.numel() < n):
+        raise ValueError("buffer smaller than n")
+    if tau_out.numel() < m or results.numel() * 8 < m * RESULT_BYTES:
+        raise ValueError("tau_out / results smaller than m")
+    arr = (_u64 * max(m, 1))(*ks)
+    _check("dct_threshold_select_multi",
+           lib().dct_threshold_select_multi(_p(grad), _p(residual), n, arr, m, _p(tau_out), _p(results),
+                                            _p(workspace), workspace.numel(), _stream(stream)))
+
+
+def dct_mp_threshold_mean(x_act, rows, d, ld, ks, mean_out, tau_out, stream=None) -> None:
+    """mean_out[q] = mean over the rows of the ks[q]-th largest |x[i, :d]|; tau_out [m * rows] receives the
+    per-row thresholds.  Nothing is sparsified."""
+    code = _dtype_code(x_act)
+    _need(x_act, x_act.dtype, "x_act")
+    _need(mean_out, torch.float64, "mean_out")
+    _need(tau_out, x_act.dtype, "tau_out")
+    m = len(ks)
+    if x_act.numel() < (rows - 1) * ld + d:
+        raise ValueError("x_act smaller than rows x ld")
+    if mean_out.numel() < m or tau_out.numel() < m * rows:
+        raise ValueError("mean_out / tau_out smaller than m / m * rows")
+    arr = (_u32 * max(m, 1))(*ks)
+    _check("dct_mp_threshold_mean",
+           lib().dct_mp_threshold_mean(_p(x_act), code, rows, d, ld, arr, m, _p(mean_out), _p(tau_out),
+                                       _stream(stream)))
+
+
+def dct_dp_drift_check(compress_result, k, ratio_num, ratio_den, flag_out, stream=None) -> None:
+    """flag_out[0] = 1 / 2 / 0: the survivor count of the last compress call is above k * ratio / below
+    k / ratio / inside.  Device to device, on the stream."""
+    _need(compress_result, torch.int64, "compress_result")
+    _need(flag_out, torch.int32, "flag_out")
+    _check("dct_dp_drift_check",
+           lib().dct_dp_drift_check(_p(compress_result), k, ratio_num, ratio_den, _p(flag_out), _stream(stream)))

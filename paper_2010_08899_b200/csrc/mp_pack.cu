@@ -10,25 +10,10 @@
 //
 // Backward: a gather of X_grad through that column list, one warp per row.
 #include "common.cuh"
+#include "row_select.cuh"
 
 namespace dct {
 namespace {
-
-template <typename T> struct ElemTraits;
-template <> struct ElemTraits<float> {
-    static constexpr int kPasses = 4;
-    __device__ static __forceinline__ uint32_t key(float x) { return key_f32(x); }
-    __device__ static __forceinline__ float from_key(uint32_t k) { return __uint_as_float(k); }
-    __host__ __device__ static constexpr int shift(int p) { return p == 0 ? 23 : (p == 1 ? 15 : (p == 2 ? 7 : 0)); }
-    __host__ __device__ static constexpr int bits(int p) { return p == 3 ? 7 : 8; }
-};
-template <> struct ElemTraits<uint16_t> {   // bf16 carried as its bit pattern
-    static constexpr int kPasses = 2;
-    __device__ static __forceinline__ uint32_t key(uint16_t x) { return key_bf16(x); }
-    __device__ static __forceinline__ uint16_t from_key(uint32_t k) { return static_cast<uint16_t>(k); }
-    __host__ __device__ static constexpr int shift(int p) { return p == 0 ? 7 : 0; }
-    __host__ __device__ static constexpr int bits(int p) { return p == 0 ? 8 : 7; }
-};
 
 constexpr int kMaxWarps = 32;
 
@@ -41,7 +26,7 @@ __global__ void mp_topk_pack_fwd_kernel(const T* __restrict__ x, uint32_t rows, 
     extern __shared__ __align__(128) unsigned char smem_raw[];
     T* row_s = reinterpret_cast<T*>(smem_raw);
     __shared__ uint32_t s_hist[256];
-    __shared__ uint32_t s_prefix, s_krem;
+    __shared__ uint32_t s_sel[2];
     __shared__ uint32_t s_wcnt[kMaxWarps];   // (gt << 16) | eq per warp; both <= 32768 / warps... see below
 
     const uint32_t tid = threadIdx.x, nt = blockDim.x;
@@ -75,61 +60,9 @@ __global__ void mp_topk_pack_fwd_kernel(const T* __restrict__ x, uint32_t rows, 
         } else {
             for (uint32_t j = tid; j < d; j += nt) row_s[j] = xr[j];
         }
-        if (tid == 0) {
-            s_prefix = 0;
-            s_krem = k;
-        }
-
         // ---- radix select of the k-th largest key ------------------------------------------
-#pragma unroll
-        for (int p = 0; p < Tr::kPasses; ++p) {
-            const int shift = Tr::shift(p), bits = Tr::bits(p);
-            const uint32_t nbins = 1u << bits;
-            for (uint32_t b = tid; b < 256; b += nt) s_hist[b] = 0;
-            __syncthreads();
-            const uint32_t prefix = s_prefix;
-            // Exact zeros are the common value after a ReLU: in the first pass they are counted in a register
-            // and added to bin 0 once per thread instead of colliding on one shared-memory word.
-            uint32_t zeros = 0;
-            for (uint32_t j = tid; j < d; j += nt) {
-                const uint32_t key = Tr::key(row_s[j]);
-                if (p == 0 && key == 0) {
-                    ++zeros;
-                } else if (p == 0 || (key >> (shift + bits)) == prefix) {
-                    atomicAdd(&s_hist[(key >> shift) & (nbins - 1u)], 1u);
-                }
-            }
-            if (zeros) atomicAdd(&s_hist[0], zeros);
-            __syncthreads();
-            if (warp == 0) {
-                // lane owns 8 bins, top-down: bin(lane, q) = 255 - (8 lane + q); bins >= nbins are empty
-                const uint32_t k_rem = s_krem;
-                uint32_t c[8], own = 0;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    c[q] = s_hist[255 - (8 * lane + q)];
-                    own += c[q];
-                }
-                uint32_t incl = own;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                    if (lane >= static_cast<uint32_t>(o)) incl += t;
-                }
-                uint32_t above = incl - own;
-#pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    if (above < k_rem && k_rem <= above + c[q]) {
-                        s_prefix = (prefix << bits) | (255u - (8u * lane + q));
-                        s_krem = k_rem - above;
-                    }
-                    above += c[q];
-                }
-            }
-            __syncthreads();
-        }
-        const uint32_t tau_key = s_prefix;
-        const uint32_t take = s_krem;          // ties (key == tau_key) to keep, lowest columns first
+        uint32_t tau_key, take;      // take: ties (key == tau_key) to keep, lowest columns first
+        cta_row_select<T>(row_s, d, k, s_hist, s_sel, tau_key, take);
         if (tid == 0 && tau_out) tau_out[row] = Tr::from_key(tau_key);
 
         // ---- ordered emit: count per warp, then write ----------------------------------------

@@ -8,6 +8,8 @@ A small command-line driver for profiling and quick timing of a single kernel at
     python -m paper_2010_08899_b200.run_case mp_bwd   --rows 16384 --d 4096 --k 205 --dtype bf16
     python -m paper_2010_08899_b200.run_case decompress --n 268435456
     python -m paper_2010_08899_b200.run_case mp_unpack --rows 16384 --d 4096 --k 205 --dtype bf16
+    python -m paper_2010_08899_b200.run_case select_multi --n 268435456          (75 / 90 / 95 % sparsity)
+    python -m paper_2010_08899_b200.run_case threshold_mean --rows 16384 --d 4096 --dtype bf16
 
 It prints the mean device time per call (CUDA events) and the algorithmic GB/s.
 """
@@ -23,7 +25,8 @@ from . import inputs
 
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("entry", choices=["select", "compress", "compress_layers", "decompress", "mp_fwd", "mp_bwd", "mp_unpack"])
+    ap.add_argument("entry", choices=["select", "compress", "compress_layers", "decompress", "mp_fwd", "mp_bwd", "mp_unpack",
+                                     "select_multi", "threshold_mean"])
     ap.add_argument("--n", type=int, default=1 << 28)
     ap.add_argument("--k", type=int, default=0, help="survivor target (default: 0.01 %% of n, or 5 %% of d)")
     ap.add_argument("--rows", type=int, default=16384)
@@ -83,7 +86,27 @@ def main():
             print(f"compress_layers, {name}: {ms:.4f} ms, {12 * args.n / ms / 1e6:.1f} GB/s algorithmic")
         return
 
-    if args.entry in ("select", "compress", "decompress"):
+    if args.entry == "select_multi":
+        # the paper's three sparsity levels (75 / 90 / 95 %) out of one set of passes
+        n = args.n
+        ks = [B.k_from_sparsity(n, 75, 100), B.k_from_sparsity(n, 90, 100), B.k_from_sparsity(n, 95, 100)]
+        g = [gen(n, 501 + j, dev) for j in range(2)]
+        taus = torch.zeros(len(ks), device=dev)
+        res = torch.zeros(5 * len(ks), dtype=torch.int64, device=dev)
+        ws = B.new_workspace(B.dct_threshold_select_multi_workspace_bytes(n, len(ks)), dev)
+        call = lambda i: B.dct_threshold_select_multi(g[i % 2], None, n, ks, taus, res, ws)
+        nbytes = 4 * n
+    elif args.entry == "threshold_mean":
+        rows, d = args.rows, args.d
+        dt = torch.float32 if args.dtype == "f32" else torch.bfloat16
+        es = 4 if args.dtype == "f32" else 2
+        ks = [B.k_from_sparsity(d, 75, 100), B.k_from_sparsity(d, 90, 100), B.k_from_sparsity(d, 95, 100)]
+        x = [inputs.mp_activations(rows, d, 410 + j, dtype=dt, device=dev, col_scale_seed=400) for j in range(2)]
+        mean = torch.zeros(len(ks), dtype=torch.float64, device=dev)
+        tau_rows = torch.zeros(len(ks) * rows, dtype=dt, device=dev)
+        call = lambda i: B.dct_mp_threshold_mean(x[i % 2], rows, d, d, ks, mean, tau_rows)
+        nbytes = rows * d * es
+    elif args.entry in ("select", "compress", "decompress"):
         n = args.n
         k = args.k or B.k_from_density(n, 1, 10_000)
         g = [gen(n, 501 + j, dev) for j in range(2)]
