@@ -145,9 +145,9 @@ class HotPath:
             assert st == 0, st
         rec()
         # kernels of this library per step: the select enqueues 12 (reset, 3 sample passes, filter, decide,
-        # 3 candidate passes, 3 full passes that return at once) from n = 2^27 and 4 (reset + 3 passes) below;
+        # 3 candidate passes, 3 full passes that return at once) from n = 2^25 and 4 (reset + 3 passes) below;
         # each compress is a reset kernel + the streaming kernel; each MP iteration a forward and a backward kernel
-        self.launches += (12 if n >= (1 << 27) else 4) + 2 * c["dp_iters"] + 2 * c["mp_iters"]
+        self.launches += (12 if n >= (1 << 25) else 4) + 2 * c["dp_iters"] + 2 * c["mp_iters"]
 
     def time_mp_parts(self, stream, reps):
         """Forward and backward pack timed on their own (after the main measurement)."""

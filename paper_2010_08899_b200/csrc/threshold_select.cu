@@ -10,9 +10,10 @@
 //
 // Three radix passes over the whole vector cost 12 B per element against a floor of 4 B.  When k is
 // small against n (the method's regime) the vector is therefore read only ONCE:
-//   1. a strided sample of 2^20 elements is radix-selected (it lives in L2) for a rank chosen so that,
-//      with overwhelming probability, between k and a few k elements of the whole vector lie at or
-//      above the sampled value `lo`;
+//   1. a sample of 2^20 elements -- 2^17 evenly spaced groups of 8 consecutive elements, i.e. whole
+//      32-byte sectors, so the sample costs 4 MiB of HBM traffic and then lives in L2 -- is
+//      radix-selected for a rank chosen so that, with overwhelming probability, between k and a few k
+//      elements of the whole vector lie at or above the sampled value `lo`;
 //   2. one streaming pass over the vector appends every key >= key(lo) to a candidate buffer in the
 //      workspace and counts them;
 //   3. if the count c satisfies k <= c <= capacity, tau is the k-th largest candidate (radix select
@@ -30,10 +31,11 @@ constexpr int kSelVecs = 4;
 constexpr uint32_t kSelChunk = kSelThreads * kSelVecs * 4;   // 8192 elements per CTA iteration
 constexpr int kBins = 2048;
 constexpr int kPasses = 3;
-constexpr uint32_t kSampleSize = 1u << 20;                   // elements in the strided sample
+constexpr uint32_t kSampleSize = 1u << 20;                   // elements in the sample
+constexpr uint32_t kSampleGroup = 8;                         // consecutive elements taken at each sample position
 constexpr uint32_t kMaxCandidates = 1u << 22;                // candidate buffer: at most 16 MiB
 #ifndef DCT_SEL_MIN_SAMPLED_N
-#define DCT_SEL_MIN_SAMPLED_N (1u << 27)
+#define DCT_SEL_MIN_SAMPLED_N (1u << 25)
 #endif
 constexpr uint32_t kMinSampledN = DCT_SEL_MIN_SAMPLED_N;     // below this the three plain passes are cheaper
 
@@ -100,7 +102,7 @@ struct VectorSource {        // key(fl32(grad[i] + residual[i])), i < n
     const float* grad;
     const float* residual;   // may be null
 };
-struct StridedSource {       // the same at i * stride
+struct StridedSource {       // the same at (i / 8) * stride + i % 8: groups of 8 neighbours, `stride` elements apart
     const float* grad;
     const float* residual;
     uint32_t stride;
@@ -113,7 +115,7 @@ __device__ __forceinline__ uint32_t key_at(const VectorSource& s, uint32_t i) {
     return key_f32(s.residual ? __fadd_rn(s.grad[i], s.residual[i]) : s.grad[i]);
 }
 __device__ __forceinline__ uint32_t key_at(const StridedSource& s, uint32_t i) {
-    const size_t j = static_cast<size_t>(i) * s.stride;
+    const size_t j = static_cast<size_t>(i / kSampleGroup) * s.stride + (i % kSampleGroup);
     return key_f32(s.residual ? __fadd_rn(s.grad[j], s.residual[j]) : s.grad[j]);
 }
 __device__ __forceinline__ uint32_t key_at(const KeySource& s, uint32_t i) { return s.keys[i]; }
@@ -372,7 +374,7 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
     uint32_t sample_n = 0, sample_k = 0, stride = 0, capacity = 0;
     if (n >= kMinSampledN) {
         capacity = candidate_capacity(n);
-        stride = n32 / kSampleSize;
+        stride = (n32 / (kSampleSize / kSampleGroup)) & ~(kSampleGroup - 1u);   // groups start on 32-byte boundaries
         sample_n = kSampleSize;
         sample_k = sample_rank(n, k, sample_n, capacity);
         if (sample_k == 0) sample_n = 0;

@@ -11,7 +11,7 @@ pytestmark = pytest.mark.gpu
 
 
 def test_select_is_deterministic_on_both_paths():
-    for n, k in (((1 << 27) + 12345, 20_000), (3_000_017, 3000)):        # sampled single pass / three plain passes
+    for n, k in (((1 << 25) + 12345, 20_000), (3_000_017, 3000)):        # sampled single pass / three plain passes
         g = inputs.dp_mixture(n, 7, G.DEV)
         e = inputs.dp_gaussian(n, 8, G.DEV) * 0.01
         first = None

@@ -196,3 +196,28 @@ def test_host_buffer_entry_point():
     assert np.array_equal(idx_host.numpy()[:r.count], want.idx)
     assert np.array_equal(bits32(val_host.numpy()[:r.count]), bits32(want.val))
     assert np.array_equal(bits32(e_dev.cpu().numpy()), bits32(e))
+
+
+def test_select_sampled_path_and_its_fallbacks():
+    """From 2^25 elements the select reads the vector once, guided by a sample of 2^17 groups of 8
+    neighbours.  The sample only steers: when it misjudges the vector (too few or far too many
+    candidates) or cannot be used (dense k), the plain passes must give the same exact answer."""
+    n = (1 << 25) + 999
+    stride = (n // (1 << 17)) & ~7
+    sampled = (torch.arange(1 << 17, device=G.DEV)[:, None] * stride + torch.arange(8, device=G.DEV)[None, :]).reshape(-1)
+    assert int(sampled.max()) < n
+    base = inputs.dp_mixture(n, 90, G.DEV)
+    cases = {}
+    cases["iid, sparse k"] = (base, 3356)
+    cases["dense k: no sample"] = (base, n // 4)
+    big_at_sampled = inputs.dp_gaussian(n, 91, G.DEV)
+    big_at_sampled[sampled] = 1000.0 + inputs.dp_gaussian(sampled.numel(), 92, G.DEV)
+    cases["sample overestimates: too few candidates"] = (big_at_sampled, 10_000)
+    zero_at_sampled = inputs.dp_gaussian(n, 93, G.DEV)
+    zero_at_sampled[sampled] = 0.0
+    cases["sample underestimates: candidates overflow"] = (zero_at_sampled, 5_000)
+    for name, (g, k) in cases.items():
+        tau_dev, r = G.select(g, None, k)
+        want = oracle.dp_select(g.cpu().numpy(), None, k)
+        assert bits32(tau_dev.cpu().numpy())[0] == bits32(want.tau)[0], name
+        assert (r.n_gt, r.n_eq) == (want.n_gt, want.n_eq), name
