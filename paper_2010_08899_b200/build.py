@@ -9,9 +9,9 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdct_b200.so")
-SOURCES = ["abi.cu", "dp_compress.cu", "threshold_select.cu", "mp_pack.cu", "decompress.cu", "diagnostics.cu",
+SOURCES = ["abi.cu", "dp_compress.cu", "threshold_select.cu", "mp_pack.cu", "mp_pack_f32.cu", "decompress.cu", "diagnostics.cu",
            "dp_select_compress.cu"]
-HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "row_select.cuh"), os.path.join(ROOT, "include", "dct.h")]
+HEADERS = [os.path.join(CSRC, "common.cuh"), os.path.join(CSRC, "row_select.cuh"), os.path.join(CSRC, "mp_warp.cuh"), os.path.join(ROOT, "include", "dct.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -11,6 +11,7 @@
 // Backward: a gather of X_grad through that column list, one warp per row.
 #include "common.cuh"
 #include "row_select.cuh"
+#include "mp_warp.cuh"
 
 namespace dct {
 namespace {
@@ -166,13 +167,6 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 // If the candidates do not fit the registers (heavy ties at the bound, or k larger than the number of
 // leaves), the row takes a slow general path: tau_i is found bit by bit by counting over the row, and the
 // output is written straight from the row.
-#ifndef DCT_FWD_MAX_WARPS
-#define DCT_FWD_MAX_WARPS 24
-#endif
-constexpr int kFwdMaxWarps = DCT_FWD_MAX_WARPS;   // rows in flight per CTA (one CTA per SM; shared memory bounds it)
-constexpr uint32_t kAbsMask2 = 0x7FFF7FFFu;
-constexpr uint32_t kHistWords = 256u;       // one histogram of up to 256 bins per warp
-
 template <int E8> struct WarpRowLayout {
     static constexpr uint32_t E = E8 * 8u, D = E * 32u;
     static constexpr uint32_t kSpanBytes = E * 2u;           // the row lies in shared memory as it does in HBM
@@ -191,9 +185,6 @@ template <int E8> struct WarpRowLayout {
         return kRowBytes + scratch_words(k) * 4u + 16u;
     }
 };
-
-__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) { return *reinterpret_cast<__nv_bfloat162*>(&u); }
-__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
 
 // bit j set iff |element j| >= low, for the 8 bf16 of one int4.  Floating-point compare: exact for
 // normal numbers; may also admit a few denormals/zeros if the hardware flushes (a superset is fine
@@ -216,66 +207,6 @@ __device__ __forceinline__ uint32_t mask8_ge_exact(uint4 v, uint32_t low) {
     const uint32_t t3 = (((v.w & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
     uint32_t m = (t0 >> 15) | (t1 >> 13) | (t2 >> 11) | (t3 >> 9);   // halves at bits {0,16},{2,18},{4,20},{6,22}
     return (m | (m >> 15)) & 0xFFu;
-}
-
-// v = *(uint2*)shared_address if p (a predicated load: no branch)
-__device__ __forceinline__ void lds64_if(uint2& v, uint32_t shared_address, bool p) {
-    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %3, 0;\n\t@q ld.shared.v2.u32 {%0, %1}, [%2];\n\t}"
-                 : "+r"(v.x), "+r"(v.y) : "r"(shared_address), "r"(static_cast<uint32_t>(p)));
-}
-
-__device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v) {
-    const uint32_t lane = lane_id();
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, v, o);
-        if (lane >= static_cast<uint32_t>(o)) v += t;
-    }
-    return v;
-}
-
-// hist holds 256 exponent bins.  Returns the exponent that holds rank k_rem
-// (counting from exponent `top_exp` downwards) and reduces k_rem to the rank inside that exponent.
-__device__ __forceinline__ uint32_t pick_exponent(const uint32_t* hist, uint32_t top_exp, uint32_t& k_rem) {
-    const uint32_t lane = lane_id();
-    for (int top = static_cast<int>(top_exp); top >= 0; top -= 32) {   // 32 exponents per step, highest first
-        const int eb = top - static_cast<int>(lane);
-        uint32_t c = 0;
-        if (eb >= 0) {
-            c = hist[eb];
-        }
-        const uint32_t inc = warp_inclusive_sum(c);
-        const uint32_t hit = __ballot_sync(0xFFFFFFFFu, inc >= k_rem);
-        if (hit) {
-            const int src = __ffs(hit) - 1;
-            k_rem -= __shfl_sync(0xFFFFFFFFu, inc - c, src);
-            return static_cast<uint32_t>(top - src);
-        }
-        k_rem -= __shfl_sync(0xFFFFFFFFu, inc, 31);
-    }
-    return 0;
-}
-// hist[0..127] holds mantissa counts.  Returns the mantissa that holds rank k_rem from the top and the
-// rank inside it (1-based: how many elements of that bin are still needed).
-__device__ __forceinline__ uint32_t pick_mantissa(const uint32_t* hist, uint32_t k_rem, uint32_t& take) {
-    const uint32_t lane = lane_id();
-    // lane owns 4 bins, top-down: bin(lane, q) = 127 - (4 lane + q)
-    const uint4 h = reinterpret_cast<const uint4*>(hist)[31 - lane];
-    const uint32_t c[4] = {h.w, h.z, h.y, h.x};
-    const uint32_t own = c[0] + c[1] + c[2] + c[3];
-    uint32_t above = warp_inclusive_sum(own) - own, found = 0xFFFFFFFFu, found_take = 0;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        if (above < k_rem && k_rem <= above + c[q]) {
-            found = 127u - (4u * lane + q);
-            found_take = k_rem - above;
-        }
-        above += c[q];
-    }
-    const uint32_t who = __ballot_sync(0xFFFFFFFFu, found != 0xFFFFFFFFu);
-    const int src = who ? __ffs(who) - 1 : 0;
-    take = __shfl_sync(0xFFFFFFFFu, found_take, src);
-    return __shfl_sync(0xFFFFFFFFu, found, src) & 0x7Fu;
 }
 
 // General slow path for one row (rare): no usable bound, or very many elements tie at it.  tau_i is found
@@ -337,13 +268,6 @@ __device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_
     }
     if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
 }
-
-// PL: candidates a lane holds in registers (10: k <= 224; 20: k <= 448, with 4-element leaves for the
-// exact bound, since 8-element leaves get loose as k approaches their number).
-template <int PL> struct FwdVariant {
-    static constexpr int kMaxWarps = PL <= 10 ? kFwdMaxWarps : 20;    // registers per thread grow with PL
-    static constexpr bool kFineLeaves = PL > 10;
-};
 
 template <int E8, int PL>
 __global__ void __launch_bounds__(FwdVariant<PL>::kMaxWarps * 32)
@@ -807,8 +731,13 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
     const size_t es = dtype == DCT_F32 ? 4 : 2;
     if ((rows_out && !aligned_to(rows_out, 4)) || (tau_out && !aligned_to(tau_out, es))) return DCT_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    if (dtype == DCT_F32)
+    if (dtype == DCT_F32) {
+        bool handled = false;       // the warp-per-row fp32 kernel takes the same shapes as the bf16 one below
+        const dct_status_t fast = launch_fwd_f32_warp(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
+                                                      result, stream, &handled);
+        if (fast != DCT_OK || handled) return fast;
         return launch_fwd<float>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    }
     // The warp-per-row kernel holds up to 320 (k <= 224) or 640 (k <= 448) candidates in registers and needs
     // the leaf bound (k <= d/8 with 8-element leaves, k <= d/4 with 4-element ones); larger k take the
     // general kernel.

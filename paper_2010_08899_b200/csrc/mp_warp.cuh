@@ -1,0 +1,93 @@
+// Pieces shared by the warp-per-row forward kernels of DCT-MP (Algorithm 2): one warp finds the row
+// threshold tau_i and packs the row (bf16: mp_pack.cu; fp32: mp_pack_f32.cu).
+#pragma once
+#include "common.cuh"
+
+namespace dct {
+
+#ifndef DCT_FWD_MAX_WARPS
+#define DCT_FWD_MAX_WARPS 24
+#endif
+constexpr int kFwdMaxWarps = DCT_FWD_MAX_WARPS;   // rows in flight per CTA (one CTA per SM; shared memory bounds it)
+constexpr uint32_t kAbsMask2 = 0x7FFF7FFFu;
+constexpr uint32_t kHistWords = 256u;       // one histogram of up to 256 bins per warp
+
+
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) { return *reinterpret_cast<__nv_bfloat162*>(&u); }
+__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
+
+
+// v = *(uint2*)shared_address if p (a predicated load: no branch)
+__device__ __forceinline__ void lds64_if(uint2& v, uint32_t shared_address, bool p) {
+    asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %3, 0;\n\t@q ld.shared.v2.u32 {%0, %1}, [%2];\n\t}"
+                 : "+r"(v.x), "+r"(v.y) : "r"(shared_address), "r"(static_cast<uint32_t>(p)));
+}
+
+__device__ __forceinline__ uint32_t warp_inclusive_sum(uint32_t v) {
+    const uint32_t lane = lane_id();
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, v, o);
+        if (lane >= static_cast<uint32_t>(o)) v += t;
+    }
+    return v;
+}
+
+// hist holds 256 exponent bins.  Returns the exponent that holds rank k_rem
+// (counting from exponent `top_exp` downwards) and reduces k_rem to the rank inside that exponent.
+__device__ __forceinline__ uint32_t pick_exponent(const uint32_t* hist, uint32_t top_exp, uint32_t& k_rem) {
+    const uint32_t lane = lane_id();
+    for (int top = static_cast<int>(top_exp); top >= 0; top -= 32) {   // 32 exponents per step, highest first
+        const int eb = top - static_cast<int>(lane);
+        uint32_t c = 0;
+        if (eb >= 0) {
+            c = hist[eb];
+        }
+        const uint32_t inc = warp_inclusive_sum(c);
+        const uint32_t hit = __ballot_sync(0xFFFFFFFFu, inc >= k_rem);
+        if (hit) {
+            const int src = __ffs(hit) - 1;
+            k_rem -= __shfl_sync(0xFFFFFFFFu, inc - c, src);
+            return static_cast<uint32_t>(top - src);
+        }
+        k_rem -= __shfl_sync(0xFFFFFFFFu, inc, 31);
+    }
+    return 0;
+}
+// hist[0..127] holds mantissa counts.  Returns the mantissa that holds rank k_rem from the top and the
+// rank inside it (1-based: how many elements of that bin are still needed).
+__device__ __forceinline__ uint32_t pick_mantissa(const uint32_t* hist, uint32_t k_rem, uint32_t& take) {
+    const uint32_t lane = lane_id();
+    // lane owns 4 bins, top-down: bin(lane, q) = 127 - (4 lane + q)
+    const uint4 h = reinterpret_cast<const uint4*>(hist)[31 - lane];
+    const uint32_t c[4] = {h.w, h.z, h.y, h.x};
+    const uint32_t own = c[0] + c[1] + c[2] + c[3];
+    uint32_t above = warp_inclusive_sum(own) - own, found = 0xFFFFFFFFu, found_take = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        if (above < k_rem && k_rem <= above + c[q]) {
+            found = 127u - (4u * lane + q);
+            found_take = k_rem - above;
+        }
+        above += c[q];
+    }
+    const uint32_t who = __ballot_sync(0xFFFFFFFFu, found != 0xFFFFFFFFu);
+    const int src = who ? __ffs(who) - 1 : 0;
+    take = __shfl_sync(0xFFFFFFFFu, found_take, src);
+    return __shfl_sync(0xFFFFFFFFu, found, src) & 0x7Fu;
+}
+
+// PL: candidates a lane holds in registers (10: k <= 224; 20: k <= 448, with 4-element leaves for the
+// exact bound, since 8-element leaves get loose as k approaches their number).
+template <int PL> struct FwdVariant {
+    static constexpr int kMaxWarps = PL <= 10 ? kFwdMaxWarps : 20;    // registers per thread grow with PL
+    static constexpr bool kFineLeaves = PL > 10;
+};
+
+
+// The fp32 kernels live in their own translation unit.
+dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                 int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                 dct_result_t* result, cudaStream_t stream, bool* handled);
+
+}  // namespace dct

@@ -126,8 +126,9 @@ def test_mp_host_buffer_entry_point():
     assert np.array_equal(G.as_np_bits(gv_h).reshape(rows, k), oracle.mp_bwd(G.to_oracle(gx), want.cols))
 
 
-def test_mp_bf16_rows_with_wildly_different_scales():
-    """The warp-per-row kernel guesses each row's bound from the previous row's threshold; rows whose
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_mp_rows_with_wildly_different_scales(dtype):
+    """The warp-per-row kernels guess each row's bound from the previous row's threshold; rows whose
     scales jump by orders of magnitude make that guess useless in both directions (too few / far too
     many candidates), which must only cost time, never change the result."""
     # enough rows that every warp of the persistent grid meets several of them, and a scale pattern whose
@@ -135,20 +136,42 @@ def test_mp_bf16_rows_with_wildly_different_scales():
     rows, d, k = 9002, 4096, 205
     x = inputs.mp_activations(rows, d, 77, dtype=torch.float32, device=G.DEV, col_scale_seed=78)
     scale = torch.tensor([1.0, 300.0, 0.004, 17.0, 1e-3, 1e4, 1.0], device=G.DEV).repeat(rows // 7)
-    x = (x * scale[:, None]).to(torch.bfloat16).contiguous()
+    x = (x * scale[:, None]).to(dtype).contiguous()
     x[5] = 0                                    # a dead sample between live ones
     x[6, ::7] = 2.0                             # heavy ties right after it
-    gx = inputs.mp_gradients(rows, d, 79, dtype=torch.bfloat16, device=G.DEV)
+    gx = inputs.mp_gradients(rows, d, 79, dtype=dtype, device=G.DEV)
     for kk in (k, 64, 256):
         _compare_fwd_bwd(x, gx, d, kk)
 
 
-@pytest.mark.parametrize("d", [768, 1280, 1536, 1792, 2560, 3072, 3584])
-def test_mp_bf16_widths_that_are_not_powers_of_two(d):
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [256, 512, 768, 1280, 1536, 1792, 2560, 3072, 3584, 4096])
+def test_mp_warp_per_row_widths(dtype, d):
+    """Every row width the warp-per-row kernels are instantiated for, both dtypes, with k on both sides of
+    their limits (k <= d/8 and 224, k <= d/4 and 448)."""
     rows = 300
-    x = inputs.mp_activations(rows, d, 11 + d, dtype=torch.bfloat16, device=G.DEV, col_scale_seed=12 + d)
+    x = inputs.mp_activations(rows, d, 11 + d, dtype=dtype, device=G.DEV, col_scale_seed=12 + d)
     x[7] = 0
     x[8] = 1.0
-    gx = inputs.mp_gradients(rows, d, 13 + d, dtype=torch.bfloat16, device=G.DEV)
-    for k in (1, d // 20, d // 10, d // 8, d // 5):
+    x[9, ::3] = -2.5
+    gx = inputs.mp_gradients(rows, d, 13 + d, dtype=dtype, device=G.DEV)
+    for k in sorted({1, max(1, d // 20), d // 10, d // 8, d // 5, min(d // 4, 448), min(d // 4, 448) + 1}):
         _compare_fwd_bwd(x, gx, d, k)
+
+
+def test_mp_f32_keys_that_differ_only_in_the_low_bits():
+    """fp32 rows whose magnitudes share their upper 16 bits in large groups: the 15-bit bucket of tau_i
+    then holds many members, and the order inside it is decided by the lower 16 bits alone (few members:
+    ranked through the list; more than 64: bit by bit), with exact ties on top."""
+    rows, d, k = 600, 4096, 205
+    g = torch.Generator(device=G.DEV).manual_seed(5)
+    hi = torch.randint(0x3F00, 0x3F10, (rows, d), generator=g, device=G.DEV, dtype=torch.int32)       # 16 buckets only
+    lo = torch.randint(0, 1 << 16, (rows, d), generator=g, device=G.DEV, dtype=torch.int32)
+    lo[100:200] &= 0xFF00                                   # coarse lower bits: exact ties inside the bucket
+    lo[200:300] = 0                                         # bf16-valued fp32: every member of a bucket ties
+    sign = torch.randint(0, 2, (rows, d), generator=g, device=G.DEV, dtype=torch.int32) << 31
+    x = ((hi << 16) | lo | sign).view(torch.float32).contiguous()
+    x[300:400, 1000:] = 0.0                                 # ~1000 live columns: buckets of ~60 members
+    gx = inputs.mp_gradients(rows, d, 6, device=G.DEV)
+    for kk in (k, 17, 448):
+        _compare_fwd_bwd(x, gx, d, kk)
