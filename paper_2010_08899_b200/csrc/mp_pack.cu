@@ -309,7 +309,9 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     }
     __syncthreads();
 
-    const uint32_t warp_global = blockIdx.x * (blockDim.x >> 5) + warp;
+    // rows are dealt out CTA by CTA (row mod grid = CTA), then warp by warp: every SM gets the same number of
+    // rows to within one, and the last, partly filled round is spread over all SMs
+    const uint32_t warp_global = blockIdx.x + gridDim.x * warp;             // this warp's first row
     const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
     auto request_row = [&](uint32_t r) {          // one bulk copy brings the whole row
         if (lane == 0) {
