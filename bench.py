@@ -173,7 +173,8 @@ class HotPath:
 
     def time_extras(self, stream, reps=3):
         """The entry points beyond the step, timed on their own after the main measurement: threshold
-        life-span L = 1 (select + compress of the same vector), and the two decompression calls."""
+        life-span L = 1 (select + compress of the same vector), the two decompression calls, the threshold
+        diagnostics and the fp32 forward pack."""
         B, c, s = self.B, self.cfg, stream
         n, cap = c["dp_n"], c["dp_capacity"]
         rows, d, k = c["mp_rows"], c["mp_d"], c["mp_k"]
@@ -190,6 +191,22 @@ class HotPath:
                                                            self.res_mp, s),
             "mp_unpack": lambda i: B.dct_mp_unpack(self.cols, self.vals, rows, d, d, k, dense_mp, None, s),
         }
+        # threshold diagnostics at the paper's three sparsity levels (75 / 90 / 95 %), and the fp32 forward pack
+        ks_dp = [B.k_from_sparsity(n, q, 100) for q in (75, 90, 95)]
+        ks_mp = [B.k_from_sparsity(d, q, 100) for q in (75, 90, 95)]
+        taus3 = torch.zeros(3, device=self.dev)
+        res3 = torch.zeros(15, dtype=torch.int64, device=self.dev)
+        ws3 = B.new_workspace(B.dct_threshold_select_multi_workspace_bytes(n, 3), self.dev)
+        mean3 = torch.zeros(3, dtype=torch.float64, device=self.dev)
+        tau_rows = torch.zeros(3 * rows, dtype=torch.bfloat16, device=self.dev)
+        x32 = [self.x[j % len(self.x)].float() for j in range(2)]
+        vals32 = torch.empty(rows * k, device=self.dev)
+        calls["threshold_select_multi_3_levels"] = lambda i: B.dct_threshold_select_multi(
+            self.grad_view(i), None, n, ks_dp, taus3, res3, ws3, s)
+        calls["mp_threshold_mean_3_levels"] = lambda i: B.dct_mp_threshold_mean(
+            self.x[i % len(self.x)], rows, d, d, ks_mp, mean3, tau_rows, s)
+        calls["mp_fwd_fp32"] = lambda i: B.dct_mp_topk_pack_fwd(x32[i % 2], rows, d, d, k, self.cols, vals32, None,
+                                                                 None, None, s)
         for name, call in calls.items():
             call(0)
             a = _record(stream)
@@ -198,6 +215,9 @@ class HotPath:
             b = _record(stream)
             b.synchronize()
             out[name] = {"ms": a.elapsed_time(b) / reps}
+        out["mp_fwd_fp32"]["GBps"] = (rows * d * 4 + rows * k * 6) / (out["mp_fwd_fp32"]["ms"] * 1e-3) / 1e9
+        out["threshold_select_multi_3_levels"]["GBps_at_4B_per_elem"] = \
+            4 * n / (out["threshold_select_multi_3_levels"]["ms"] * 1e-3) / 1e9
         out["dp_select_compress_L1"]["GBps_at_16B_per_elem"] = 16 * n / (out["dp_select_compress_L1"]["ms"] * 1e-3) / 1e9
         out["dp_decompress"]["GBps_at_4B_per_elem"] = 4 * n / (out["dp_decompress"]["ms"] * 1e-3) / 1e9
         out["mp_unpack"]["GBps"] = (rows * d * 2 + rows * k * 4) / (out["mp_unpack"]["ms"] * 1e-3) / 1e9

@@ -46,10 +46,7 @@ constexpr uint32_t kWarpElems = 32u * kVecs * 4u;       // 512
 constexpr uint32_t kTileElems = kWarps * kWarpElems;    // 4096
 constexpr uint32_t kTileBytes = kTileElems * 4u;        // 16 KiB per operand
 
-#ifndef DCT_CMP_STAGES
-#define DCT_CMP_STAGES 2
-#endif
-constexpr int kStages = DCT_CMP_STAGES;                 // ring depth of the streaming kernel
+constexpr int kStages = 2;                              // ring depth of the streaming kernel
 constexpr uint32_t kInvalidTile = 0xFFFFFFFFu;
 constexpr uint32_t kMbarLimit = 1u << 24;               // polls before an mbarrier wait gives up
 
@@ -280,9 +277,7 @@ __device__ __forceinline__ void emit_warp(const float (&w)[kVecs * 4], uint32_t 
 // ------------------------------------------------------------------------------------------
 // generic path: one CTA per tile, plain loads/stores, any alignment, ragged tail
 // ------------------------------------------------------------------------------------------
-#ifndef DCT_CMP_MIN_BLOCKS
-#define DCT_CMP_MIN_BLOCKS 4
-#endif
+constexpr int kTileKernelMinBlocks = 4;                 // CTAs of the tile kernel the register budget must allow per SM
 // One tile, by one CTA, with plain loads and stores (every thread of the CTA calls this with the same tile).
 template <bool kVectorised>
 __device__ __forceinline__ void compress_tile_body(const float* __restrict__ grad, float* __restrict__ residual,
@@ -383,7 +378,7 @@ __device__ __forceinline__ void compress_tile_body(const float* __restrict__ gra
 }
 
 template <bool kVectorised>
-__global__ void __launch_bounds__(kThreads, DCT_CMP_MIN_BLOCKS)
+__global__ void __launch_bounds__(kThreads, kTileKernelMinBlocks)
 dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ residual, uint32_t n,
                         const float* __restrict__ tau_p, const uint64_t* __restrict__ budget_p,
                         int32_t* __restrict__ idx_out, float* __restrict__ val_out, uint64_t capacity,
@@ -402,14 +397,8 @@ dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ resi
 // ------------------------------------------------------------------------------------------
 // fast path: persistent CTAs; load warp + compute warps + scan warp
 // ------------------------------------------------------------------------------------------
-#ifndef DCT_CMP_QUEUE_SLOTS
-#define DCT_CMP_QUEUE_SLOTS 8
-#endif
-#ifndef DCT_CMP_QUEUE_ENTRIES
-#define DCT_CMP_QUEUE_ENTRIES 512
-#endif
-constexpr int kSlots = DCT_CMP_QUEUE_SLOTS;              // tiles a CTA may be ahead of its scan warp
-constexpr uint32_t kQueueEntries = DCT_CMP_QUEUE_ENTRIES;  // survivors of one tile that fit a slot
+constexpr int kSlots = 8;                                // tiles a CTA may be ahead of its scan warp
+constexpr uint32_t kQueueEntries = 512;                  // survivors of one tile that fit a slot
 constexpr uint32_t kEqBit = 0x80000000u;                 // queue entry: index (31 bits) | "equal to tau"
 constexpr int kLoadWarp = kWarps, kScanWarp = kWarps + 1;
 constexpr int kStreamThreads = kThreads + 64;
@@ -753,7 +742,7 @@ __global__ void dp_compress_batched_init_kernel(CompressCtrl* ctrl, uint64_t* ti
 // The tiles the streaming kernel does not take: the ragged last tile of every aligned vector and all the
 // tiles of vectors that are not 16-byte aligned.  Work items are handed out in table order by a ticket,
 // so inside an unaligned vector a tile's predecessors have always been taken before it.
-__global__ void __launch_bounds__(kThreads, DCT_CMP_MIN_BLOCKS)
+__global__ void __launch_bounds__(kThreads, kTileKernelMinBlocks)
 dp_compress_tile_batched_kernel(const BatchTable batch, uint32_t total_slow, CompressCtrl* ctrl,
                                 uint64_t* __restrict__ tile_state_base, uint32_t spin_limit) {
     __shared__ uint32_t s_work;

@@ -5,10 +5,7 @@
 
 namespace dct {
 
-#ifndef DCT_FWD_MAX_WARPS
-#define DCT_FWD_MAX_WARPS 24
-#endif
-constexpr int kFwdMaxWarps = DCT_FWD_MAX_WARPS;   // rows in flight per CTA (one CTA per SM; shared memory bounds it)
+constexpr int kFwdMaxWarps = 24;   // rows in flight per CTA (one CTA per SM; shared memory bounds it)
 constexpr uint32_t kAbsMask2 = 0x7FFF7FFFu;
 constexpr uint32_t kHistWords = 256u;       // one histogram of up to 256 bins per warp
 

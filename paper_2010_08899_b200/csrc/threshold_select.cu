@@ -34,10 +34,7 @@ constexpr int kPasses = 3;
 constexpr uint32_t kSampleSize = 1u << 20;                   // elements in the sample
 constexpr uint32_t kSampleGroup = 8;                         // consecutive elements taken at each sample position
 constexpr uint32_t kMaxCandidates = 1u << 22;                // candidate buffer: at most 16 MiB
-#ifndef DCT_SEL_MIN_SAMPLED_N
-#define DCT_SEL_MIN_SAMPLED_N (1u << 25)
-#endif
-constexpr uint32_t kMinSampledN = DCT_SEL_MIN_SAMPLED_N;     // below this the three plain passes are cheaper
+constexpr uint32_t kMinSampledN = 1u << 25;                  // below this the three plain passes are cheaper
 
 __host__ __device__ constexpr int pass_shift(int p) { return p == 0 ? 20 : (p == 1 ? 10 : 0); }
 __host__ __device__ constexpr int pass_bits(int p) { return p == 0 ? 11 : 10; }
