@@ -525,7 +525,8 @@ def main():
     b0 = per_step[0]
     parts = {
         "select": {"ms": statistics.mean(sel_ms), "GBps_at_4B_per_elem": 4 * n / (statistics.mean(sel_ms) * 1e-3) / 1e9},
-        "compress": {"ms": cmp_avg_ms, "GBps": achieved, "survivors_first_last": [counts[0], counts[-1]]},
+        "compress": {"ms": cmp_avg_ms, "ms_median": statistics.median(cmp_ms), "ms_best": min(cmp_ms), "GBps": achieved,
+                     "survivors_first_last": [counts[0], counts[-1]]},
         "mp_fwd+bwd_block": {"ms": statistics.mean(mp_ms)},
         "mp_fwd": {"ms": mp_parts["mp_fwd"], "GBps": b0["mp_fwd"] / cfg["mp_iters"] / (mp_parts["mp_fwd"] * 1e-3) / 1e9},
         "mp_bwd": {"ms": mp_parts["mp_bwd"], "GBps": b0["mp_bwd"] / cfg["mp_iters"] / (mp_parts["mp_bwd"] * 1e-3) / 1e9,
