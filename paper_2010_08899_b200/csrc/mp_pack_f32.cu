@@ -551,6 +551,10 @@ dct_status_t launch_variant(const void* x_act, uint32_t rows, uint32_t ld, uint3
 template <int E8>
 dct_status_t launch_width(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out, void* vals_out,
                           int32_t* rows_out, void* tau_out, dct_result_t* result, cudaStream_t stream) {
+    if constexpr (E8 <= 4) {        // narrow rows: k <= 112 needs 5 candidates per lane, not 10
+        if (k <= 112)
+            return launch_variant<E8, 5>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    }
     if (k <= 224)
         return launch_variant<E8, 10>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     return launch_variant<E8, 20>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);

@@ -74,7 +74,7 @@ __device__ __forceinline__ uint32_t pick_mantissa(const uint32_t* hist, uint32_t
     return __shfl_sync(0xFFFFFFFFu, found, src) & 0x7Fu;
 }
 
-// PL: candidates a lane holds in registers (10: k <= 224; 20: k <= 448, with 4-element leaves for the
+// PL: candidates a lane holds in registers (5: k <= 112, rows of at most 1024 columns; 10: k <= 224; 20: k <= 448, with 4-element leaves for the
 // exact bound, since 8-element leaves get loose as k approaches their number).
 template <int PL> struct FwdVariant {
     static constexpr int kMaxWarps = PL <= 10 ? kFwdMaxWarps : 20;    // registers per thread grow with PL
