@@ -186,29 +186,6 @@ template <int E8> struct WarpRowLayout {
     }
 };
 
-// bit j set iff |element j| >= low, for the 8 bf16 of one int4.  Floating-point compare: exact for
-// normal numbers; may also admit a few denormals/zeros if the hardware flushes (a superset is fine
-// for a candidate filter); NaN always passes.
-__device__ __forceinline__ uint32_t mask8_ge_filter(uint4 v, __nv_bfloat162 low2) {
-    const uint32_t r0 = __hgeu2_mask(__habs2(as_bf162(v.x)), low2);
-    const uint32_t r1 = __hgeu2_mask(__habs2(as_bf162(v.y)), low2);
-    const uint32_t r2 = __hgeu2_mask(__habs2(as_bf162(v.z)), low2);
-    const uint32_t r3 = __hgeu2_mask(__habs2(as_bf162(v.w)), low2);
-    const uint32_t m = (r0 & 0x00020001u) | (r1 & 0x00080004u) | (r2 & 0x00200010u) | (r3 & 0x00800040u);
-    return (m | (m >> 16)) & 0xFFu;
-}
-// the same on the integer keys, exact for every bit pattern (low <= 0x8000)
-__device__ __forceinline__ uint32_t mask8_ge_exact(uint4 v, uint32_t low) {
-    const uint32_t low2 = low | (low << 16);
-    // per 16-bit half: bit 15 of ((key | 0x8000) - low) is set iff key >= low (no borrow crosses halves)
-    const uint32_t t0 = (((v.x & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
-    const uint32_t t1 = (((v.y & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
-    const uint32_t t2 = (((v.z & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
-    const uint32_t t3 = (((v.w & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
-    uint32_t m = (t0 >> 15) | (t1 >> 13) | (t2 >> 11) | (t3 >> 9);   // halves at bits {0,16},{2,18},{4,20},{6,22}
-    return (m | (m >> 15)) & 0xFFu;
-}
-
 // General slow path for one row (rare): no usable bound, or very many elements tie at it.  tau_i is found
 // bit by bit on the row itself, most significant first (the largest v with #{key >= v} >= k); then
 // everything above tau_i and the first ties are written, in column order, straight from the row.
@@ -744,6 +721,12 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
                                                       result, stream, &handled);
         if (fast != DCT_OK || handled) return fast;
         return launch_fwd<float>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    }
+    {   // narrow rows (256 or 512 columns, small k): the row stays in registers, several rows per warp
+        bool handled = false;
+        const dct_status_t narrow = launch_fwd_bf16_narrow(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
+                                                           result, stream, &handled);
+        if (narrow != DCT_OK || handled) return narrow;
     }
     // The warp-per-row kernel holds up to 320 (k <= 224) or 640 (k <= 448) candidates in registers and needs
     // the leaf bound (k <= d/8 with 8-element leaves, k <= d/4 with 4-element ones); larger k take the

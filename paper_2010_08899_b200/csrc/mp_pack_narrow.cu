@@ -1,0 +1,372 @@
+// dct_mp_topk_pack_fwd, bf16 rows of 256 or 512 columns: Algorithm 2 (DCT-MP) with the row held in
+// registers and several samples per warp.
+//
+// For narrow rows the fixed cost per row of the shared-memory kernel (mp_pack.cu: bulk copy, barrier, bit
+// table, bisection, linked walk) outweighs the work on the row itself, and so do the warp scans and votes
+// when a whole warp serves one short row.  Here a row belongs to a group of G lanes (G = 8 or 16, so a
+// warp works on 4 or 2 rows at once, every scan and vote serving all of them; G = 32 works too but is
+// no faster than the shared-memory kernel and is not used); lane l of the group
+// loads its E consecutive columns (E <= 32: at most four 16-byte loads) straight into registers, and the
+// next rows are fetched while the current ones are worked on.  The candidate bits of a lane are one
+// register word in column order, so one segmented scan ranks every candidate.  Steps per row:
+//   A  bound: the previous row's tau_i minus a margin; if that leaves fewer than k or too many candidates,
+//      the exact bound (the k-th largest maximum of the aligned 8-element leaves, found bit by bit) -- the
+//      row is still in registers, so trying again costs no memory traffic.
+//   B  candidates (key >= bound, ~1.3 k of them) go, in column order, to the group's list in shared memory;
+//      their values are re-read from the row in global memory, which the loads above left in L1.
+//   C  the list is dealt out evenly, at most 5 candidates to a lane; tau_i comes from a 64-bin histogram
+//      just above the bound (else bit by bit over the candidates), and the ordered emit is that of the
+//      wide kernel.
+// Decisions that change the control flow (bound rejected, window missed, candidates do not fit) are taken
+// for the warp as a whole, so all its lanes stay together; the slow path works on the rows in global memory.
+#include "common.cuh"
+#include "mp_warp.cuh"
+
+namespace dct {
+namespace {
+
+constexpr int kNarrowWarps = 16;                 // warps per CTA
+constexpr uint32_t kNarrowPerLane = 5;           // candidates a lane holds in registers
+constexpr uint32_t kNarrowScratchWords = 320;    // per warp; a group's share holds its list / histogram / stage
+
+template <int G> struct Group {
+    static constexpr uint32_t kRows = 32u / G;                       // rows a warp works on at once
+    static constexpr uint32_t kList = kNarrowPerLane * G;            // candidates of a row that fit
+    static constexpr uint32_t kShare = kNarrowScratchWords / kRows;  // scratch words of one group: >= 64 + G, >= kList
+    static constexpr uint32_t kBins = 64u / G;                       // window bins a lane looks after
+    static_assert(kShare >= 64u + G && kShare >= kList, "scratch share too small");
+
+    __device__ static __forceinline__ uint32_t inclusive_sum(uint32_t v, uint32_t gl) {
+#pragma unroll
+        for (int o = 1; o < G; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, v, o, G);
+            if (gl >= static_cast<uint32_t>(o)) v += t;
+        }
+        return v;
+    }
+    __device__ static __forceinline__ uint32_t last(uint32_t v) { return __shfl_sync(0xFFFFFFFFu, v, G - 1, G); }
+    __device__ static __forceinline__ uint32_t from(uint32_t v, uint32_t src) { return __shfl_sync(0xFFFFFFFFu, v, src, G); }
+    __device__ static __forceinline__ uint32_t sum(uint32_t v) {
+#pragma unroll
+        for (int o = G / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o, G);
+        return v;
+    }
+    // votes of the group's lanes, bit i = lane i of the group
+    __device__ static __forceinline__ uint32_t ballot(bool p, uint32_t group_base) {
+        const uint32_t all = __ballot_sync(0xFFFFFFFFu, p);
+        return G == 32 ? all : (all >> group_base) & ((1u << (G & 31)) - 1u);
+    }
+};
+
+// Slow path for the rows a warp holds: tau_i bit by bit by counting over the row (read again from global
+// memory), then the ordered emit straight from the row.  Called by the whole warp; groups without a row
+// (valid == false) run along on a row of their own that exists and store nothing.
+template <int E8, int G>
+__device__ __noinline__ void narrow_slow_path(const uint16_t* __restrict__ xr, bool valid, uint32_t k, size_t out_base,
+                                              uint32_t row, int16_t* __restrict__ cols_out,
+                                              uint16_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
+                                              uint16_t* __restrict__ tau_out) {
+    using Gr = Group<G>;
+    constexpr uint32_t E = E8 * 8u;
+    const uint32_t gl = lane_id() & (G - 1);
+    const uint4* mine = reinterpret_cast<const uint4*>(xr + gl * E);
+    uint4 v[E8];
+#pragma unroll
+    for (int c = 0; c < E8; ++c) v[c] = __ldg(mine + c);
+    uint32_t tau_key = 0;
+#pragma unroll 1
+    for (int bit = 14; bit >= 0; --bit) {
+        const uint32_t trial = tau_key | (1u << bit);
+        uint32_t cnt = 0;
+#pragma unroll
+        for (int c = 0; c < E8; ++c) cnt += __popc(mask8_ge_exact(v[c], trial));
+        if (Gr::sum(cnt) >= k) tau_key = trial;
+    }
+    uint32_t gt_mask = 0, eq_mask = 0;
+#pragma unroll
+    for (int c = 0; c < E8; ++c) {
+        const uint32_t gt = mask8_ge_exact(v[c], tau_key + 1u);
+        const uint32_t eq = mask8_ge_exact(v[c], tau_key) & ~gt;
+        gt_mask |= gt << (8 * c);
+        eq_mask |= eq << (8 * c);
+    }
+    const uint32_t n_gt_mine = __popc(gt_mask), n_eq_mine = __popc(eq_mask);
+    const uint32_t incl = Gr::inclusive_sum(n_gt_mine, gl);
+    const uint32_t take = k - Gr::last(incl);       // ties to keep, lowest columns first
+    uint32_t g_at = incl - n_gt_mine;
+    uint32_t e_at = Gr::inclusive_sum(n_eq_mine, gl) - n_eq_mine;
+    uint32_t m = valid ? (gt_mask | eq_mask) : 0u;
+    while (m) {
+        const uint32_t j = __ffs(m) - 1;
+        m &= m - 1;
+        const bool is_eq = (eq_mask >> j) & 1u;
+        if (!is_eq || e_at < take) {
+            const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
+            cols_out[pos] = static_cast<int16_t>(gl * E + j);
+            vals_out[pos] = xr[gl * E + j];
+            if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
+        }
+        g_at += is_eq ? 0u : 1u;
+        e_at += is_eq ? 1u : 0u;
+    }
+    if (valid && gl == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+}
+
+template <int E8, int G>
+__global__ void __launch_bounds__(kNarrowWarps * 32)
+mp_topk_fwd_bf16_narrow_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
+                               int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
+                               int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
+                               dct_result_t* __restrict__ result) {
+    using Gr = Group<G>;
+    constexpr uint32_t E = E8 * 8u;                // columns per lane; the lane's candidate bits are one word
+    constexpr uint32_t kRows = Gr::kRows;
+    constexpr uint32_t kGuessMargin = 32;
+    __shared__ uint32_t s_scratch[kNarrowWarps][kNarrowScratchWords];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    const uint32_t gl = lane & (G - 1), group = lane / G, group_base = group * G;
+    uint32_t* share = s_scratch[warp] + group * Gr::kShare;   // this group's list / histogram / stage, in turn
+
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+    // Row bundles (kRows consecutive rows) are dealt out CTA by CTA, then warp by warp.
+    const uint32_t warps = blockDim.x >> 5;
+    const uint64_t bundles = (static_cast<uint64_t>(rows) + kRows - 1) / kRows;
+    const uint64_t first_bundle = blockIdx.x + static_cast<uint64_t>(gridDim.x) * warp;
+    const uint64_t bundle_step = static_cast<uint64_t>(gridDim.x) * warps;
+    // a group past the last row reads the last row instead (and stores nothing)
+    auto row_of = [&](uint64_t bundle) -> uint64_t {
+        const uint64_t r = bundle * kRows + group;
+        return r < rows ? r : rows - 1;
+    };
+    auto load_row = [&](uint64_t r, uint4 (&v)[E8]) {
+        const uint4* src = reinterpret_cast<const uint4*>(x + r * ld + gl * E);
+#pragma unroll
+        for (int c = 0; c < E8; ++c) v[c] = __ldg(src + c);
+    };
+    uint4 cur[E8], nxt[E8];
+    if (first_bundle < bundles) load_row(row_of(first_bundle), nxt);
+
+    uint32_t guess_low = 0;                         // bound guessed from the group's previous row (0: none)
+    const bool have_bound = k <= G * E8;            // at least k leaves in a row
+    for (uint64_t bundle = first_bundle; bundle < bundles; bundle += bundle_step) {
+        const bool valid = bundle * kRows + group < rows;
+        const uint64_t row64 = row_of(bundle);
+        const uint32_t row = static_cast<uint32_t>(row64);
+#pragma unroll
+        for (int c = 0; c < E8; ++c) cur[c] = nxt[c];
+        if (bundle + bundle_step < bundles) load_row(row_of(bundle + bundle_step), nxt);   // in flight meanwhile
+        const uint16_t* xr = x + row64 * ld;
+        const size_t out_base = static_cast<size_t>(row) * k;
+
+        // ---- B (with A): candidate bits of the lane, one word in column order -------------------------
+        uint32_t mask = 0, incl = 0, n_cand = 0;
+        auto build_mask = [&](uint32_t bound) {
+            const __nv_bfloat162 low2 = as_bf162(bound | (bound << 16));
+            mask = 0;
+#pragma unroll
+            for (int c = 0; c < E8; ++c) mask |= mask8_ge_filter(cur[c], low2) << (8 * c);
+            incl = Gr::inclusive_sum(__popc(mask), gl);
+            n_cand = Gr::last(incl);
+        };
+        uint32_t low = guess_low;
+        bool settled = false;
+        if (have_bound && __all_sync(0xFFFFFFFFu, guess_low != 0)) {
+            build_mask(low);
+            settled = __all_sync(0xFFFFFFFFu, n_cand >= k && n_cand <= Gr::kList);
+        }
+        if (!settled) {
+            // exact bound: the k-th largest of the row's leaf maxima, bit by bit
+            uint32_t leaf[E8];
+#pragma unroll
+            for (int c = 0; c < E8; ++c) {
+                const __nv_bfloat162 m2 = __hmax2(__hmax2(__habs2(as_bf162(cur[c].x)), __habs2(as_bf162(cur[c].y))),
+                                                  __hmax2(__habs2(as_bf162(cur[c].z)), __habs2(as_bf162(cur[c].w))));
+                const uint32_t m = as_u32(m2);
+                leaf[c] = max(m & 0xFFFFu, m >> 16);
+            }
+            low = 0;
+            if (have_bound) {
+#pragma unroll 1
+                for (int bit = 14; bit >= 0; --bit) {
+                    const uint32_t trial = low | (1u << bit);
+                    uint32_t cnt = 0;
+#pragma unroll
+                    for (int c = 0; c < E8; ++c) cnt += leaf[c] >= trial ? 1u : 0u;
+                    if (Gr::sum(cnt) >= k) low = trial;
+                }
+            }
+            build_mask(low);
+        }
+        if (!have_bound || __any_sync(0xFFFFFFFFu, n_cand > Gr::kList || low == 0)) {
+            narrow_slow_path<E8, G>(xr, valid, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
+            continue;
+        }
+
+        // candidates into the group's list, column order: entry = value | column << 16
+        __syncwarp();                                   // whatever used the scratch before is done
+        {
+            uint32_t at = incl - __popc(mask);
+            uint32_t m = mask;
+            while (m) {
+                const uint32_t col = gl * E + (__ffs(m) - 1);
+                m &= m - 1;
+                share[at++] = __ldg(xr + col) | (col << 16);
+            }
+        }
+        __syncwarp();
+        uint32_t ent[kNarrowPerLane];                   // 0: unused slot (a key below the bound, which is >= 1)
+        const uint32_t per_lane = (n_cand + G - 1) / G;
+#pragma unroll
+        for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+            const uint32_t r = gl * per_lane + i;
+            ent[i] = (static_cast<uint32_t>(i) < per_lane && r < n_cand) ? share[r] : 0u;
+        }
+        __syncwarp();                                   // the list is in registers: its words become the histogram
+
+        // ---- C: k-th largest of the candidates --------------------------------------------------
+        uint32_t tau_key = 0, take = 0;
+        bool found = false;
+        {
+            // 64 bins just above the bound, G private overflow bins behind them
+            const uint32_t drop = n_cand - k;
+            for (uint32_t b = gl; b < 64u + G; b += G) share[b] = 0;
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+                const uint32_t rel = (ent[i] & 0x7FFFu) - low;
+                atomicAdd(&share[rel < 64u ? rel : 64u + gl], 1u);
+            }
+            __syncwarp();
+            uint32_t h[Gr::kBins], own = 0;             // the lane looks after bins gl kBins .. gl kBins + kBins - 1
+#pragma unroll
+            for (int j = 0; j < static_cast<int>(Gr::kBins); ++j) {
+                h[j] = share[gl * Gr::kBins + j];
+                own += h[j];
+            }
+            uint32_t before = Gr::inclusive_sum(own, gl) - own;
+            uint32_t my_tau = 0, my_take = 0;
+            bool mine = false;
+#pragma unroll
+            for (int j = 0; j < static_cast<int>(Gr::kBins); ++j) {
+                if (before <= drop && drop < before + h[j]) {
+                    mine = true;
+                    my_tau = low + gl * Gr::kBins + j;
+                    my_take = h[j] - (drop - before);
+                }
+                before += h[j];
+            }
+            const uint32_t who = Gr::ballot(mine, group_base);
+            const uint32_t src = who ? __ffs(who) - 1 : 0u;
+            tau_key = Gr::from(my_tau, src);
+            take = Gr::from(my_take, src);
+            found = who != 0;
+            __syncwarp();
+        }
+        if (__any_sync(0xFFFFFFFFu, !found)) {
+            // tau_i beyond the window for some row: the k-th largest candidate key, bit by bit (every group
+            // recomputes; where the window had the answer this gives the same one)
+            uint32_t t = 0;
+#pragma unroll 1
+            for (int bit = 14; bit >= 0; --bit) {
+                const uint32_t trial = t | (1u << bit);
+                uint32_t cnt = 0;
+#pragma unroll
+                for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) cnt += (ent[i] & 0x7FFFu) >= trial ? 1u : 0u;
+                if (Gr::sum(cnt) >= k) t = trial;
+            }
+            uint32_t above = 0;
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) above += (ent[i] & 0x7FFFu) > t ? 1u : 0u;
+            tau_key = t;
+            take = k - Gr::sum(above);
+        }
+        if (valid && gl == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+        guess_low = tau_key > kGuessMargin ? tau_key - kGuessMargin : 0u;
+
+        // ---- D: ordered emit ------------------------------------------------------------------------
+        {
+            uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+                const uint32_t key = ent[i] & 0x7FFFu;
+                counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
+            }
+            const uint32_t before = Gr::inclusive_sum(counts, gl) - counts;
+            uint32_t e_at = before & 0xFFFFu;
+            uint32_t pos = (before >> 16) + (e_at < take ? e_at : take);
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+                const uint32_t key = ent[i] & 0x7FFFu;
+                const bool is_eq = key == tau_key;
+                const bool keep = key > tau_key || (is_eq && e_at < take);
+                if (keep) share[pos] = ent[i];
+                pos += keep ? 1u : 0u;
+                e_at += is_eq ? 1u : 0u;
+            }
+        }
+        __syncwarp();
+        if (valid) {
+            for (uint32_t p = gl; p < k; p += G) {
+                const uint32_t e = share[p];
+                cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
+                vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
+                if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
+            }
+        }
+        __syncwarp();
+    }
+}
+
+template <int E8, int G>
+dct_status_t launch_narrow(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+                           void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
+                           cudaStream_t stream) {
+    auto kernel = mp_topk_fwd_bf16_narrow_kernel<E8, G>;
+    int per_sm = 0;
+    DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kNarrowWarps * 32, 0));
+    if (per_sm < 1) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint64_t bundles = (static_cast<uint64_t>(rows) + Group<G>::kRows - 1) / Group<G>::kRows;
+    const uint64_t ctas_needed = (bundles + kNarrowWarps - 1) / kNarrowWarps;
+    const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
+    const uint32_t grid = static_cast<uint32_t>(ctas_needed < max_grid ? ctas_needed : max_grid);
+    kernel<<<grid, kNarrowWarps * 32, 0, stream>>>(static_cast<const uint16_t*>(x_act), rows, ld, k, cols_out,
+                                                   static_cast<uint16_t*>(vals_out), rows_out,
+                                                   static_cast<uint16_t*>(tau_out), result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}
+
+}  // namespace
+
+// *handled = false: not a shape of this path; the caller goes on to the other kernels.
+// The list of a row holds 5 candidates per lane of its group and must take the ~1.3 k candidates (1.45 k at
+// the 99th percentile) the bound leaves: k <= 3.4 lanes.
+dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                    int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                    dct_result_t* result, cudaStream_t stream, bool* handled) {
+    *handled = false;
+    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0 || k > d / 8) return DCT_OK;
+    *handled = true;
+    switch (d) {
+        case 256:
+            if (k <= 27) return launch_narrow<4, 8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            break;
+        case 512:
+            if (k <= 54) return launch_narrow<4, 16>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            break;
+        default: break;
+    }
+    *handled = false;
+    return DCT_OK;
+}
+
+}  // namespace dct

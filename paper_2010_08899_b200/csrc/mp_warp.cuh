@@ -14,6 +14,29 @@ __device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) { return *reinter
 __device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
 
 
+// bit j set iff |element j| >= low, for the 8 bf16 of one int4.  Floating-point compare: exact for
+// normal numbers; may also admit a few denormals/zeros if the hardware flushes (a superset is fine
+// for a candidate filter); NaN always passes.
+__device__ __forceinline__ uint32_t mask8_ge_filter(uint4 v, __nv_bfloat162 low2) {
+    const uint32_t r0 = __hgeu2_mask(__habs2(as_bf162(v.x)), low2);
+    const uint32_t r1 = __hgeu2_mask(__habs2(as_bf162(v.y)), low2);
+    const uint32_t r2 = __hgeu2_mask(__habs2(as_bf162(v.z)), low2);
+    const uint32_t r3 = __hgeu2_mask(__habs2(as_bf162(v.w)), low2);
+    const uint32_t m = (r0 & 0x00020001u) | (r1 & 0x00080004u) | (r2 & 0x00200010u) | (r3 & 0x00800040u);
+    return (m | (m >> 16)) & 0xFFu;
+}
+// the same on the integer keys, exact for every bit pattern (low <= 0x8000)
+__device__ __forceinline__ uint32_t mask8_ge_exact(uint4 v, uint32_t low) {
+    const uint32_t low2 = low | (low << 16);
+    // per 16-bit half: bit 15 of ((key | 0x8000) - low) is set iff key >= low (no borrow crosses halves)
+    const uint32_t t0 = (((v.x & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
+    const uint32_t t1 = (((v.y & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
+    const uint32_t t2 = (((v.z & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
+    const uint32_t t3 = (((v.w & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
+    uint32_t m = (t0 >> 15) | (t1 >> 13) | (t2 >> 11) | (t3 >> 9);   // halves at bits {0,16},{2,18},{4,20},{6,22}
+    return (m | (m >> 15)) & 0xFFu;
+}
+
 // v = *(uint2*)shared_address if p (a predicated load: no branch)
 __device__ __forceinline__ void lds64_if(uint2& v, uint32_t shared_address, bool p) {
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %3, 0;\n\t@q ld.shared.v2.u32 {%0, %1}, [%2];\n\t}"
@@ -81,6 +104,11 @@ template <int PL> struct FwdVariant {
     static constexpr bool kFineLeaves = PL > 10;
 };
 
+
+// Rows of 256 or 512 bf16 columns: the row stays in registers, several rows per warp (mp_pack_narrow.cu).
+dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                    int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                    dct_result_t* result, cudaStream_t stream, bool* handled);
 
 // The fp32 kernels live in their own translation unit.
 dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,

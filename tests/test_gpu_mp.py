@@ -175,3 +175,24 @@ def test_mp_f32_keys_that_differ_only_in_the_low_bits():
     gx = inputs.mp_gradients(rows, d, 6, device=G.DEV)
     for kk in (k, 17, 448):
         _compare_fwd_bwd(x, gx, d, kk)
+
+
+@pytest.mark.parametrize("d,k_limit", [(256, 27), (512, 54), (768, 96), (1024, 96)])
+def test_mp_bf16_narrow_rows_several_per_warp(d, k_limit):
+    """Rows of at most 1024 bf16 columns stay in registers, 4 / 2 / 1 of them per warp: row counts that leave
+    the last warp partly filled, k on both sides of the path's limit, and rows that force each of its
+    fall-backs (no previous threshold, threshold far from the previous one, ties that overflow the list,
+    dead rows) next to ordinary ones in the same warp."""
+    for rows in (1, 3, 37, 1001):
+        x = inputs.mp_activations(rows, d, 21 + d + rows, dtype=torch.float32, device=G.DEV, col_scale_seed=22 + d)
+        scale = torch.tensor([1.0, 250.0, 0.01, 1.0, 3.0], device=G.DEV).repeat(rows // 5 + 1)[:rows]
+        x = x * scale[:, None]
+        if rows > 30:
+            x[4] = 0.0                                  # dead row
+            x[9] = 1.5                                  # every element ties
+            x[10, ::2] = -7.0                           # half the row ties above everything else
+            x[17] = inputs.quantize_mantissa(x[17], 1)  # coarse values
+        x = x.to(torch.bfloat16).contiguous()
+        gx = inputs.mp_gradients(rows, d, 23 + d, dtype=torch.bfloat16, device=G.DEV)
+        for k in sorted({1, max(1, d // 20), k_limit, k_limit + 1}):
+            _compare_fwd_bwd(x, gx, d, k)
