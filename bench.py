@@ -106,6 +106,15 @@ class HotPath:
         self.calls = 0        # compress calls issued (indexes res_cmp)
         self.launches = 0     # kernels of this library launched
 
+    def input_checksums(self):
+        """64-bit sums of the bit patterns of one buffer of every kind of input (so that two runs can be seen
+        to have worked on the same data)."""
+        def bits_sum(t):
+            w = t.view(torch.int32) if t.element_size() == 4 else t.view(torch.int16)
+            return int(w.sum(dtype=torch.int64).item()) & 0xFFFFFFFFFFFFFFFF
+        return {"g_select": bits_sum(self.g_sel[: self.cfg["dp_n"]]), "g_0": bits_sum(self.g[0]),
+                "x_act_0": bits_sum(self.x[0]), "x_grad_0": bits_sum(self.gx[0])}
+
     def grad_view(self, t):
         """Gradient of iteration t: buffer t mod B, shifted by a multiple of 4 elements so that every
         element meets fresh values each time round (the residual persists across iterations)."""
@@ -587,6 +596,7 @@ def main():
                               / (max_ms / args.steps * 1e-3),
             "roofline": roofline, "parts": parts, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": gpu_launches, "clocks": clocks, "device_status_codes": statuses,
+            "input_checksums": hp.input_checksums(),
         }
         print(json.dumps(line), flush=True)
     if world > 1:
