@@ -147,7 +147,7 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 }
 
 // ------------------------------------------------------------------------------------------
-// bf16 fast path: one warp per row, d = 256 * E8 <= 4096 (common widths are instantiated), rows on 16-byte boundaries
+// bf16 fast path: one warp per row, d <= 4096 a multiple of 8 (held in a buffer of 256 * E8 columns), rows on 16-byte boundaries
 // ------------------------------------------------------------------------------------------
 // One bulk asynchronous copy brings a row into shared memory exactly as it lies in HBM; the next row is
 // requested as soon as the candidates of the current one sit in registers.
@@ -168,7 +168,7 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 // leaves), the row takes a slow general path: tau_i is found bit by bit by counting over the row, and the
 // output is written straight from the row.
 template <int E8> struct WarpRowLayout {
-    static constexpr uint32_t E = E8 * 8u, D = E * 32u;
+    static constexpr uint32_t E = E8 * 8u;                   // columns per lane of the buffer (256 * E8 columns in all)
     static constexpr uint32_t kSpanBytes = E * 2u;           // the row lies in shared memory as it does in HBM
     static constexpr uint32_t kRowBytes = 32u * kSpanBytes;
     static constexpr uint32_t kRowWords = 8u * E8;           // 32-bit candidate-mask words of a row (one bit per column)
@@ -248,7 +248,7 @@ __device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_
 
 template <int E8, int PL>
 __global__ void __launch_bounds__(FwdVariant<PL>::kMaxWarps * 32)
-mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
+mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
                              dct_result_t* __restrict__ result) {
@@ -284,6 +284,11 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         mbar_init_fence();
         fence_proxy_async_all();
     }
+    // A row of d <= D columns (d a multiple of 8) fills the first d columns of the buffer; the rest is zeroed
+    // once and never written again: zeros lie below every bound and, being the last columns, lose every tie.
+    const uint32_t row_bytes = d * 2u;
+    for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
+        *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
     // rows are dealt out CTA by CTA (row mod grid = CTA), then warp by warp: every SM gets the same number of
@@ -292,8 +297,8 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
     auto request_row = [&](uint32_t r) {          // one bulk copy brings the whole row
         if (lane == 0) {
-            mbar_arrive_expect_tx(bar, Lay::D * 2u);
-            bulk_load(base, x + static_cast<size_t>(r) * ld, Lay::D * 2u, bar);
+            mbar_arrive_expect_tx(bar, row_bytes);
+            bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, bar);
         }
     };
     // In the passes over the whole row lane l reads the 16-byte units l, l + 32, l + 64, ...: the 32 lanes of a
@@ -596,7 +601,8 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 }
 
 template <int E8, int PL>
-dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                          int16_t* cols_out,
                                           void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
                                           cudaStream_t stream) {
     using Lay = WarpRowLayout<E8>;
@@ -620,7 +626,7 @@ dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
     kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
-        static_cast<const uint16_t*>(x_act), rows, ld, k, cols_out, static_cast<uint16_t*>(vals_out), rows_out,
+        static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out, static_cast<uint16_t*>(vals_out), rows_out,
         static_cast<uint16_t*>(tau_out), result);
     DCT_CUDA_TRY(cudaGetLastError());
     return DCT_OK;
@@ -629,18 +635,18 @@ dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint
 // k <= 224: 10 candidates per lane (the exact bound leaves about 1.26 k candidates, 1.4 k at the 99th
 // percentile, which must fit 320); k <= 448: 20 per lane.
 template <int E8>
-dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
                                   void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
                                   cudaStream_t stream) {
     if constexpr (E8 <= 4) {        // narrow rows: k <= 112 needs 5 candidates per lane, not 10
         if (k <= 112)
-            return launch_fwd_bf16_warp_variant<E8, 5>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out,
+            return launch_fwd_bf16_warp_variant<E8, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
                                                        result, stream);
     }
     if (k <= 224)
-        return launch_fwd_bf16_warp_variant<E8, 10>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result,
+        return launch_fwd_bf16_warp_variant<E8, 10>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result,
                                                     stream);
-    return launch_fwd_bf16_warp_variant<E8, 20>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result,
+    return launch_fwd_bf16_warp_variant<E8, 20>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result,
                                                 stream);
 }
 
@@ -731,23 +737,25 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
     // The warp-per-row kernel holds up to 320 (k <= 224) or 640 (k <= 448) candidates in registers and needs
     // the leaf bound (k <= d/8 with 8-element leaves, k <= d/4 with 4-element ones); larger k take the
     // general kernel.
-    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 &&
+    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && d % 8 == 0 && d <= 4096 &&
         ((k <= 224 && k <= d / 8) || (k > 224 && k <= 448 && k <= d / 4))) {
-        switch (d) {   // warp-per-row path: d = 256 * E8 for the instantiated E8
-            case 256: return launch_fwd_bf16_warp<1>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 512: return launch_fwd_bf16_warp<2>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 768: return launch_fwd_bf16_warp<3>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 1024: return launch_fwd_bf16_warp<4>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 1280: return launch_fwd_bf16_warp<5>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 1536: return launch_fwd_bf16_warp<6>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 1792: return launch_fwd_bf16_warp<7>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 2048: return launch_fwd_bf16_warp<8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 2560: return launch_fwd_bf16_warp<10>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 3072: return launch_fwd_bf16_warp<12>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 3584: return launch_fwd_bf16_warp<14>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            case 4096: return launch_fwd_bf16_warp<16>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-            default: break;
-        }
+        // warp-per-row path: the smallest instantiated buffer of 256 * E8 columns that holds the row
+#define DCT_BF16_WIDTH(E8) \
+    if (d <= 256u * E8)    \
+        return launch_fwd_bf16_warp<E8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+        DCT_BF16_WIDTH(1);
+        DCT_BF16_WIDTH(2);
+        DCT_BF16_WIDTH(3);
+        DCT_BF16_WIDTH(4);
+        DCT_BF16_WIDTH(5);
+        DCT_BF16_WIDTH(6);
+        DCT_BF16_WIDTH(7);
+        DCT_BF16_WIDTH(8);
+        DCT_BF16_WIDTH(10);
+        DCT_BF16_WIDTH(12);
+        DCT_BF16_WIDTH(14);
+        DCT_BF16_WIDTH(16);
+#undef DCT_BF16_WIDTH
     }
     return launch_fwd<uint16_t>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
 }

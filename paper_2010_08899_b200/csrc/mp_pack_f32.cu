@@ -9,7 +9,8 @@
 //     top k.  The members (a handful: the candidates are about two per bucket near the threshold) are
 //     then ranked by their full keys, which gives the exact 31-bit tau_i and the number of ties to keep.
 //   * the candidates carry their full 32-bit value from the row buffer, so the emit needs nothing else.
-// Rows are 16-byte aligned, d = 256 * E8 with the instantiated E8, k <= 224 and k <= d/8 (10
+// Rows are 16-byte aligned, d <= 4096 a multiple of 4 (held zero-padded in a buffer of 256 * E8 columns),
+// k <= 224 and k <= d/8 (10
 // candidates per lane) or k <= 448 and k <= d/4 (20 per lane); everything else takes the general kernel.
 #include "common.cuh"
 #include "mp_warp.cuh"
@@ -107,7 +108,7 @@ __device__ __noinline__ void mp_row_slow_path_f32(const unsigned char* span, uin
 
 template <int E8, int PL>
 __global__ void __launch_bounds__(FwdVariant<PL>::kMaxWarps * 32)
-mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
+mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                             int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
                             int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
                             dct_result_t* __restrict__ result) {
@@ -144,6 +145,11 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
         mbar_init_fence();
         fence_proxy_async_all();
     }
+    // A row of d <= D columns (d a multiple of 4) fills the first d columns of the buffer; the rest is zeroed
+    // once and never written again: zeros lie below every bound and, being the last columns, lose every tie.
+    const uint32_t row_bytes = d * 4u;
+    for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
+        *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
     // rows are dealt out CTA by CTA (row mod grid = CTA), then warp by warp: every SM gets the same number of
@@ -152,8 +158,8 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
     const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
     auto request_row = [&](uint32_t r) {          // one bulk copy brings the whole row
         if (lane == 0) {
-            mbar_arrive_expect_tx(bar, Lay::kRowBytes);
-            bulk_load(base, x + static_cast<size_t>(r) * ld, Lay::kRowBytes, bar);
+            mbar_arrive_expect_tx(bar, row_bytes);
+            bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, bar);
         }
     };
     auto release_row = [&](uint32_t row) {   // the row buffer is no longer needed: request the next row
@@ -518,7 +524,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
 }
 
 template <int E8, int PL>
-dct_status_t launch_variant(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+dct_status_t launch_variant(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
                             void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
                             cudaStream_t stream) {
     using Lay = RowLayoutF32<E8>;
@@ -542,22 +548,23 @@ dct_status_t launch_variant(const void* x_act, uint32_t rows, uint32_t ld, uint3
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
     kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
-        static_cast<const uint32_t*>(x_act), rows, ld, k, cols_out, static_cast<uint32_t*>(vals_out), rows_out,
+        static_cast<const uint32_t*>(x_act), rows, d, ld, k, cols_out, static_cast<uint32_t*>(vals_out), rows_out,
         static_cast<uint32_t*>(tau_out), result);
     DCT_CUDA_TRY(cudaGetLastError());
     return DCT_OK;
 }
 
 template <int E8>
-dct_status_t launch_width(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out, void* vals_out,
+dct_status_t launch_width(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
+                          void* vals_out,
                           int32_t* rows_out, void* tau_out, dct_result_t* result, cudaStream_t stream) {
     if constexpr (E8 <= 4) {        // narrow rows: k <= 112 needs 5 candidates per lane, not 10
         if (k <= 112)
-            return launch_variant<E8, 5>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            return launch_variant<E8, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     }
     if (k <= 224)
-        return launch_variant<E8, 10>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-    return launch_variant<E8, 20>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        return launch_variant<E8, 10>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    return launch_variant<E8, 20>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
 }
 
 }  // namespace
@@ -567,26 +574,25 @@ dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, u
                                  int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                  dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
-    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0) return DCT_OK;
+    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 4 != 0 || d > 4096) return DCT_OK;
     if (!((k <= 224 && k <= d / 8) || (k > 224 && k <= 448 && k <= d / 4))) return DCT_OK;
     *handled = true;
 #define DCT_F32_WIDTH(E8) \
-    case 256 * E8: return launch_width<E8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
-    switch (d) {
-        DCT_F32_WIDTH(1);
-        DCT_F32_WIDTH(2);
-        DCT_F32_WIDTH(3);
-        DCT_F32_WIDTH(4);
-        DCT_F32_WIDTH(5);
-        DCT_F32_WIDTH(6);
-        DCT_F32_WIDTH(7);
-        DCT_F32_WIDTH(8);
-        DCT_F32_WIDTH(10);
-        DCT_F32_WIDTH(12);
-        DCT_F32_WIDTH(14);
-        DCT_F32_WIDTH(16);
-        default: break;
-    }
+    if (d <= 256u * E8)   \
+        return launch_width<E8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+    // the smallest instantiated buffer of 256 * E8 columns that holds the row
+    DCT_F32_WIDTH(1);
+    DCT_F32_WIDTH(2);
+    DCT_F32_WIDTH(3);
+    DCT_F32_WIDTH(4);
+    DCT_F32_WIDTH(5);
+    DCT_F32_WIDTH(6);
+    DCT_F32_WIDTH(7);
+    DCT_F32_WIDTH(8);
+    DCT_F32_WIDTH(10);
+    DCT_F32_WIDTH(12);
+    DCT_F32_WIDTH(14);
+    DCT_F32_WIDTH(16);
 #undef DCT_F32_WIDTH
     *handled = false;
     return DCT_OK;

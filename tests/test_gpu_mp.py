@@ -196,3 +196,22 @@ def test_mp_bf16_narrow_rows_several_per_warp(d, k_limit):
         gx = inputs.mp_gradients(rows, d, 23 + d, dtype=torch.bfloat16, device=G.DEV)
         for k in sorted({1, max(1, d // 20), k_limit, k_limit + 1}):
             _compare_fwd_bwd(x, gx, d, k)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("d", [264, 1000, 2000, 3000, 4000, 4088])
+def test_mp_warp_per_row_widths_between_the_buffer_sizes(dtype, d):
+    """Rows whose width is a multiple of 16 bytes but not of 256 columns sit zero-padded in the next larger
+    buffer of the warp-per-row kernels: the padding must never be selected, not even by rows with fewer than
+    k non-zeros (ties at zero go to the lowest columns) or rows of equal values."""
+    rows = 203
+    x = inputs.mp_activations(rows, d, 31 + d, dtype=dtype, device=G.DEV, col_scale_seed=32 + d)
+    x[5] = 0.0                                   # dead row: the first k columns
+    x[6] = -0.75                                 # all equal
+    x[7] = 0.0
+    x[7, d - 3:] = 1.0                           # three non-zeros at the very end, zeros elsewhere
+    x[8, : d - 8] = 0.0                          # only the last 8 columns alive
+    gx = inputs.mp_gradients(rows, d, 33 + d, dtype=dtype, device=G.DEV)
+    for k in sorted({1, 7, d // 20, d // 8, min(d // 4, 448)}):
+        cols = _compare_fwd_bwd(x, gx, d, k)
+        assert int(cols.max()) < d
