@@ -632,22 +632,329 @@ dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint
     return DCT_OK;
 }
 
-// k <= 224: 10 candidates per lane (the exact bound leaves about 1.26 k candidates, 1.4 k at the 99th
-// percentile, which must fit 320); k <= 448: 20 per lane.
+// 5, 10 or 20 candidates per lane: see fwd_candidates_per_lane.
 template <int E8>
 dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
                                   void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
                                   cudaStream_t stream) {
-    if constexpr (E8 <= 4) {        // narrow rows: k <= 112 needs 5 candidates per lane, not 10
-        if (k <= 112)
+    const int per_lane = fwd_candidates_per_lane(d, k);
+    if constexpr (E8 <= 4) {
+        if (per_lane == 5)
             return launch_fwd_bf16_warp_variant<E8, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
                                                        result, stream);
     }
-    if (k <= 224)
+    if (per_lane == 10)
         return launch_fwd_bf16_warp_variant<E8, 10>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result,
                                                     stream);
     return launch_fwd_bf16_warp_variant<E8, 20>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result,
                                                 stream);
+}
+
+// ------------------------------------------------------------------------------------------
+// bf16, dense k (up to a quarter of the row and more): one warp per row
+// ------------------------------------------------------------------------------------------
+// With k in the hundreds or thousands the candidates no longer fit registers, but they need not: tau_i
+// is pinned between two bounds and everything is emitted straight from the candidate bits.
+//   A  `low`: the previous row's tau_i minus a margin (first row of a warp: a quantile of 128 samples of
+//      the row).  One pass over the row builds two bit tables, key >= low and key >= low + 64.  If their
+//      counts n_low, n_high satisfy n_high < k <= n_low, tau_i lies in the 64-key window between them;
+//      otherwise low moves (by 64, 128, ... keys) and the pass is repeated, a few times at most.
+//   B  the elements inside the window (in the low table, not in the high one: a handful per lane) are
+//      read and counted into a 64-bin histogram; a scan over it gives tau_i and the number of ties kept.
+//   C  every lane walks its candidate bits in column order: elements of the high table are kept as they
+//      are, window elements are compared with tau_i; kept entries go to k staging slots and leave with
+//      coalesced stores.
+// A row for which this fails (tau_i = 0, bounds that do not converge) takes the bit-serial slow path.
+constexpr uint32_t kDenseWindow = 64;
+constexpr uint32_t kDenseMaxK = 1280;                 // staging slots per warp (5 KiB)
+constexpr int kDenseMaxWarps = 24;
+constexpr int kDenseRetries = 6;
+
+template <int E8> struct DenseLayout {
+    using Row = WarpRowLayout<E8>;
+    // per warp: row | low table (128 words) | high table (128 words) | histogram (64 words) | stage (k words) | mbarrier
+    static constexpr uint32_t kTabWords = 128;
+    __host__ __device__ static constexpr uint32_t scratch_words(uint32_t k) { return 2u * kTabWords + 64u + ((k + 3u) & ~3u); }
+    __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) { return Row::kRowBytes + scratch_words(k) * 4u + 16u; }
+};
+
+template <int E8>
+__global__ void __launch_bounds__(kDenseMaxWarps * 32)
+mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
+                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
+                              dct_result_t* __restrict__ result) {
+    using Lay = WarpRowLayout<E8>;
+    using Den = DenseLayout<E8>;
+    constexpr int kMaskWords = Lay::kMaskWords;
+    constexpr uint32_t kGuessMargin = 32;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    unsigned char* base = smem_raw + warp * Den::warp_bytes(k);
+    unsigned char* span = base + lane * Lay::kSpanBytes;
+    uint32_t* scratch = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
+    uint32_t* tab_low = scratch;                               // one bit per column: key >= low
+    uint32_t* tab_high = scratch + Den::kTabWords;             // one bit per column: key >= low + window
+    uint32_t* hist = scratch + 2u * Den::kTabWords;
+    uint32_t* stage = hist + 64;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Den::scratch_words(k));
+    const uint16_t* row16 = reinterpret_cast<const uint16_t*>(base);
+    __shared__ uint32_t s_stop;
+
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+    if (threadIdx.x == 0) s_stop = 0;
+    if (lane == 0) {
+        mbar_init(bar, 1);
+        mbar_init_fence();
+        fence_proxy_async_all();
+    }
+    const uint32_t row_bytes = d * 2u;                         // the tail of the buffer stays zero (see the sparse kernel)
+    for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
+        *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+
+    const uint32_t warp_global = blockIdx.x + gridDim.x * warp;
+    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
+    auto request_row = [&](uint32_t r) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(bar, row_bytes);
+            bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, bar);
+        }
+    };
+    auto release_row = [&](uint32_t row) {
+        __syncwarp();
+        fence_proxy_async_smem();
+        if (row + total_warps < rows) request_row(row + total_warps);
+    };
+    const unsigned char* unit0 = base + lane * 16u;
+    if (warp_global < rows) request_row(warp_global);
+
+    uint32_t use = 0;
+    uint32_t guess_low = 0;
+    for (uint32_t row = warp_global; row < rows; row += total_warps, ++use) {
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
+            s_stop = 1;
+            if (lane == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
+            return;
+        }
+        const size_t out_base = static_cast<size_t>(row) * k;
+
+        // ---- A: bounds around tau_i ------------------------------------------------------------------
+        uint32_t low = guess_low;
+        if (low == 0) {
+            // no previous row: the (k/d)-quantile of up to 128 samples (element 0 of up to four units of every
+            // lane), taken a little low, found bit by bit
+            constexpr int kSamples = E8 < 4 ? E8 : 4;
+            uint32_t sample[kSamples];
+#pragma unroll
+            for (int c = 0; c < kSamples; ++c) sample[c] = *reinterpret_cast<const uint16_t*>(unit0 + c * 512) & 0x7FFFu;
+            const uint32_t n_samples = 32u * kSamples;
+            uint32_t rank = (n_samples * k + d - 1) / d;                   // expected rank of tau_i among the samples
+            rank += 2u * static_cast<uint32_t>(__fsqrt_rn(static_cast<float>(rank))) + 2u;
+            if (rank > n_samples) rank = n_samples;
+#pragma unroll 1
+            for (int bit = 14; bit >= 0; --bit) {
+                const uint32_t trial = low | (1u << bit);
+                uint32_t cnt = 0;
+#pragma unroll
+                for (int c = 0; c < kSamples; ++c) cnt += sample[c] >= trial ? 1u : 0u;
+                if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= rank) low = trial;
+            }
+            if (low == 0) low = 1;
+        }
+        uint32_t geL[kMaskWords], geH[kMaskWords];
+        uint32_t n_low = 0, n_high = 0, before_packed = 0;
+        bool pinned = false;
+        uint32_t step = kDenseWindow;
+        int last_move = 0;
+#pragma unroll 1
+        for (int attempt = 0; attempt < kDenseRetries; ++attempt) {
+            // exact integer compares (the tables decide what is kept, so "a superset" is not enough here);
+            // low <= 0x7F80 keeps low + window within their 2^15 range
+            const uint32_t high = low + kDenseWindow;
+            unsigned char* tl = reinterpret_cast<unsigned char*>(tab_low) + lane;
+            unsigned char* th = reinterpret_cast<unsigned char*>(tab_high) + lane;
+            __syncwarp();
+            if (low >= 0x0080u && high <= 0x7F80u) {
+                // both bounds are normal numbers (or infinity): the packed floating-point compare is exact for
+                // every element that is not a NaN, and a NaN lands in both tables, i.e. outside the window
+                const __nv_bfloat162 low2 = as_bf162(low * 0x10001u), high2 = as_bf162(high * 0x10001u);
+#pragma unroll
+                for (int c = 0; c < E8; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(unit0 + c * 512);
+                    tl[c * 32] = static_cast<unsigned char>(mask8_ge_filter(v, low2));
+                    th[c * 32] = static_cast<unsigned char>(mask8_ge_filter(v, high2));
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < E8; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(unit0 + c * 512);
+                    tl[c * 32] = static_cast<unsigned char>(mask8_ge_exact(v, low));
+                    th[c * 32] = static_cast<unsigned char>(mask8_ge_exact(v, high));
+                }
+            }
+            __syncwarp();
+            uint32_t mine = 0;
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) {
+                const uint32_t w = lane * kMaskWords + i;
+                const bool real = Lay::kRowWords == Lay::kTableWords || w < Lay::kRowWords;
+                geL[i] = real ? tab_low[w] : 0u;
+                geH[i] = real ? tab_high[w] : 0u;
+                mine += (__popc(geL[i]) << 16) | __popc(geH[i]);
+            }
+            const uint32_t incl = warp_inclusive_sum(mine);        // both counts stay below 2^16
+            const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            n_low = total >> 16;
+            n_high = total & 0xFFFFu;
+            before_packed = incl - mine;
+            if (n_high < k && k <= n_low) {
+                pinned = true;
+                break;
+            }
+            // move the window: down if too few elements lie above low, up if too many lie above low + window;
+            // the step doubles while the direction stays the same and halves when it turns
+            const int move = n_low < k ? -1 : 1;
+            if (attempt > 0) step = (move == last_move) ? step * 2u : (step > kDenseWindow ? step / 2u : kDenseWindow);
+            last_move = move;
+            if (move < 0) {
+                if (low == 1) break;                               // tau_i = 0: fewer than k non-zeros
+                low = low > step ? low - step : 1u;
+            } else {
+                low = low + step < 0x7F80u ? low + step : 0x7F80u;
+            }
+        }
+        if (!pinned) {
+            mp_row_slow_path<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
+            release_row(row);
+            continue;
+        }
+
+        // ---- B: tau_i from the elements inside the window ----------------------------------------------
+        hist[lane] = 0;
+        hist[lane + 32] = 0;
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < kMaskWords; ++i) {
+            uint32_t m = geL[i] & ~geH[i];
+            const uint32_t col0 = (lane * kMaskWords + i) * 32u;
+            while (m) {
+                const uint32_t col = col0 + (__ffs(m) - 1);
+                m &= m - 1;
+                atomicAdd(&hist[((row16[col] & 0x7FFFu) - low) & 63u], 1u);
+            }
+        }
+        __syncwarp();
+        uint32_t tau_key, take;
+        {
+            const uint32_t drop = n_low - k;                       // window elements to discard, smallest first
+            const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
+            const uint32_t own = h.x + h.y;
+            const uint32_t before = warp_inclusive_sum(own) - own;
+            uint32_t my_tau = 0, my_take = 0;
+            bool mine = false;
+            if (before <= drop && drop < before + h.x) {
+                mine = true;
+                my_tau = low + 2u * lane;
+                my_take = h.x - (drop - before);
+            } else if (before + h.x <= drop && drop < before + own) {
+                mine = true;
+                my_tau = low + 2u * lane + 1u;
+                my_take = h.y - (drop - before - h.x);
+            }
+            const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);   // exactly one lane: n_high < k <= n_low
+            const int src = who ? __ffs(who) - 1 : 0;
+            tau_key = __shfl_sync(0xFFFFFFFFu, my_tau, src);
+            take = __shfl_sync(0xFFFFFFFFu, my_take, src);
+        }
+        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+        guess_low = tau_key > kGuessMargin ? tau_key - kGuessMargin : 1u;
+
+        // ---- C: ordered emit ------------------------------------------------------------------------
+        // kept entries before this lane: everything in the high table, plus the window elements above tau_i,
+        // plus the first `take` ties
+        uint32_t counts = (before_packed & 0xFFFFu) << 16;         // (kept for sure << 16) | ties, of the lanes before: high part
+        {
+            uint32_t mine = 0;                                     // (window elements > tau << 16) | window elements == tau
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) {
+                uint32_t m = geL[i] & ~geH[i];
+                const uint32_t col0 = (lane * kMaskWords + i) * 32u;
+                while (m) {
+                    const uint32_t col = col0 + (__ffs(m) - 1);
+                    m &= m - 1;
+                    const uint32_t key = row16[col] & 0x7FFFu;
+                    mine += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
+                }
+            }
+            counts += warp_inclusive_sum(mine) - mine;
+        }
+        {
+            uint32_t e_at = counts & 0xFFFFu;                      // ties before this lane
+            uint32_t pos = (counts >> 16) + (e_at < take ? e_at : take);
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) {
+                uint32_t m = geL[i];
+                const uint32_t col0 = (lane * kMaskWords + i) * 32u;
+                while (m) {
+                    const uint32_t col = col0 + (__ffs(m) - 1);
+                    m &= m - 1;
+                    const uint32_t v = row16[col];
+                    const uint32_t key = v & 0x7FFFu;              // >= low; the elements of the high table are > tau_i
+                    const bool is_eq = key == tau_key;
+                    const bool keep = key > tau_key || (is_eq && e_at < take);
+                    if (keep) stage[pos] = v | (col << 16);
+                    pos += keep ? 1u : 0u;
+                    e_at += is_eq ? 1u : 0u;
+                }
+            }
+        }
+        release_row(row);
+        for (uint32_t p = lane; p < k; p += 32) {
+            const uint32_t e = stage[p];
+            cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
+            vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
+            if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
+        }
+        __syncwarp();
+    }
+}
+
+template <int E8>
+dct_status_t launch_fwd_bf16_dense(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
+                                   void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
+                                   cudaStream_t stream) {
+    using Den = DenseLayout<E8>;
+    auto kernel = mp_topk_fwd_bf16_dense_kernel<E8>;
+    constexpr size_t kSmemBudget = 220 * 1024;
+    static thread_local int configured_device = -1;
+    int dev = 0;
+    DCT_CUDA_TRY(cudaGetDevice(&dev));
+    if (configured_device != dev) {
+        DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kSmemBudget)));
+        configured_device = dev;
+    }
+    const size_t per_warp = Den::warp_bytes(k);
+    size_t warps = kSmemBudget / per_warp;
+    if (warps > static_cast<size_t>(kDenseMaxWarps)) warps = kDenseMaxWarps;
+    if (warps < 1) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
+    const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
+    kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
+        static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out, static_cast<uint16_t*>(vals_out), rows_out,
+        static_cast<uint16_t*>(tau_out), result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
 }
 
 int fwd_threads_for(uint32_t d) {
@@ -734,11 +1041,9 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
                                                            result, stream, &handled);
         if (narrow != DCT_OK || handled) return narrow;
     }
-    // The warp-per-row kernel holds up to 320 (k <= 224) or 640 (k <= 448) candidates in registers and needs
-    // the leaf bound (k <= d/8 with 8-element leaves, k <= d/4 with 4-element ones); larger k take the
-    // general kernel.
+    // The sparse warp-per-row kernel holds up to 320 or 640 candidates in registers and needs a tight leaf bound.
     if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && d % 8 == 0 && d <= 4096 &&
-        ((k <= 224 && k <= d / 8) || (k > 224 && k <= 448 && k <= d / 4))) {
+        fwd_candidates_per_lane(d, k) != 0) {
         // warp-per-row path: the smallest instantiated buffer of 256 * E8 columns that holds the row
 #define DCT_BF16_WIDTH(E8) \
     if (d <= 256u * E8)    \
@@ -756,6 +1061,20 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
         DCT_BF16_WIDTH(14);
         DCT_BF16_WIDTH(16);
 #undef DCT_BF16_WIDTH
+    }
+    // dense k (beyond the candidate registers of the kernels above, up to half the row): bounds + bit tables
+    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && d % 8 == 0 && d <= 4096 && k <= kDenseMaxK &&
+        k <= d / 2) {
+#define DCT_BF16_DENSE(E8) \
+    if (d <= 256u * E8)    \
+        return launch_fwd_bf16_dense<E8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+        DCT_BF16_DENSE(1);
+        DCT_BF16_DENSE(2);
+        DCT_BF16_DENSE(4);
+        DCT_BF16_DENSE(8);
+        DCT_BF16_DENSE(12);
+        DCT_BF16_DENSE(16);
+#undef DCT_BF16_DENSE
     }
     return launch_fwd<uint16_t>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
 }

@@ -556,13 +556,13 @@ dct_status_t launch_variant(const void* x_act, uint32_t rows, uint32_t d, uint32
 
 template <int E8>
 dct_status_t launch_width(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
-                          void* vals_out,
-                          int32_t* rows_out, void* tau_out, dct_result_t* result, cudaStream_t stream) {
-    if constexpr (E8 <= 4) {        // narrow rows: k <= 112 needs 5 candidates per lane, not 10
-        if (k <= 112)
+                          void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result, cudaStream_t stream) {
+    const int per_lane = fwd_candidates_per_lane(d, k);
+    if constexpr (E8 <= 4) {
+        if (per_lane == 5)
             return launch_variant<E8, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     }
-    if (k <= 224)
+    if (per_lane == 10)
         return launch_variant<E8, 10>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     return launch_variant<E8, 20>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
 }
@@ -575,7 +575,7 @@ dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, u
                                  dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
     if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 4 != 0 || d > 4096) return DCT_OK;
-    if (!((k <= 224 && k <= d / 8) || (k > 224 && k <= 448 && k <= d / 4))) return DCT_OK;
+    if (fwd_candidates_per_lane(d, k) == 0) return DCT_OK;
     *handled = true;
 #define DCT_F32_WIDTH(E8) \
     if (d <= 256u * E8)   \

@@ -358,10 +358,10 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
     *handled = true;
     switch (d) {
         case 256:
-            if (k <= 27) return launch_narrow<4, 8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            if (k <= 20) return launch_narrow<4, 8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             break;
         case 512:
-            if (k <= 54) return launch_narrow<4, 16>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            if (k <= 40) return launch_narrow<4, 16>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             break;
         default: break;
     }

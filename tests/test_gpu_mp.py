@@ -177,7 +177,7 @@ def test_mp_f32_keys_that_differ_only_in_the_low_bits():
         _compare_fwd_bwd(x, gx, d, kk)
 
 
-@pytest.mark.parametrize("d,k_limit", [(256, 27), (512, 54), (768, 96), (1024, 96)])
+@pytest.mark.parametrize("d,k_limit", [(256, 20), (512, 40), (768, 48), (1024, 64)])
 def test_mp_bf16_narrow_rows_several_per_warp(d, k_limit):
     """Rows of at most 1024 bf16 columns stay in registers, 4 / 2 / 1 of them per warp: row counts that leave
     the last warp partly filled, k on both sides of the path's limit, and rows that force each of its
@@ -215,3 +215,24 @@ def test_mp_warp_per_row_widths_between_the_buffer_sizes(dtype, d):
     for k in sorted({1, 7, d // 20, d // 8, min(d // 4, 448)}):
         cols = _compare_fwd_bwd(x, gx, d, k)
         assert int(cols.max()) < d
+
+
+@pytest.mark.parametrize("d", [512, 1024, 2000, 4096])
+def test_mp_bf16_dense_k(d):
+    """k from a quarter to half of the row (75 % sparsity and below): tau_i is pinned between two bit tables
+    64 keys apart.  Rows whose scale jumps by orders of magnitude make the window move several times;
+    ties, dead rows and rows with fewer than k non-zeros take the remaining branches."""
+    rows = 2500
+    x = inputs.mp_activations(rows, d, 51 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=52 + d)
+    sign = torch.where(inputs.dp_gaussian(rows * d, 53 + d, G.DEV).view(rows, d) > 0, 1.0, -1.0)
+    scale = torch.tensor([1.0, 40.0, 1.0, 1e-3, 1e4, 1.0, 1.0], device=G.DEV).repeat(rows // 7 + 1)[:rows]
+    x = x * sign * scale[:, None]
+    x[3] = 0.0                                      # dead row
+    x[4] = 2.0                                      # every element ties
+    x[5, d // 3:] = 0.0                             # fewer than d/2 non-zeros
+    x[6] = inputs.quantize_mantissa(x[6], 1)        # few distinct values
+    x[7] = 3.0e38                                   # the top of the bf16 range
+    x = x.to(torch.bfloat16).contiguous()
+    gx = inputs.mp_gradients(rows, d, 54 + d, dtype=torch.bfloat16, device=G.DEV)
+    for k in sorted({d // 4 + 1, d // 3, d // 2, min(d // 2, 1280)}):
+        _compare_fwd_bwd(x, gx, d, k)
