@@ -1,14 +1,18 @@
 // dct_mp_topk_pack_fwd / dct_mp_pack_bwd: Algorithm 2 (DCT-MP).
 //
-// Forward: one CTA per sample (row).  The row is read from HBM exactly once
-// into shared memory; the row threshold tau_i (k-th largest magnitude) is found
-// on chip by a most-significant-digit-first radix select over key(x) with 8-bit
-// digits (4 passes for fp32's 31 key bits, 2 for bf16's 15); then the kept
-// columns -- every key above tau_i plus the lowest-column ties -- are written
-// in ascending column order together with their values.  The int16 column list
-// is the mask M.
+// Forward.  Every kernel reads a row from HBM exactly once, finds the row threshold tau_i (k-th largest
+// magnitude) on chip and writes the kept columns -- every key above tau_i plus the lowest-column ties --
+// in ascending column order together with their values.  The int16 column list is the mask M.
+//   * general kernel (this file): one CTA per row, any dtype / width / stride / k; tau_i by a radix select
+//     over the row in shared memory (row_select.cuh).
+//   * bf16, sparse k, rows up to 4096 columns on 16-byte boundaries (this file): one warp per row, the
+//     candidates above a bound in registers.
+//   * bf16, dense k (this file): one warp per row, tau_i pinned between two bit tables.
+//   * bf16, rows of 256 / 512 columns: several rows per warp, rows in registers (mp_pack_narrow.cu).
+//   * fp32, sparse k: one warp per row (mp_pack_f32.cu).
+// dct_mp_topk_pack_fwd (end of this file) picks among them.
 //
-// Backward: a gather of X_grad through that column list, one warp per row.
+// Backward: a gather of X_grad through the column list, one warp per row.
 #include "common.cuh"
 #include "row_select.cuh"
 #include "mp_warp.cuh"
