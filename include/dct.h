@@ -227,6 +227,35 @@ DCT_API dct_status_t dct_dp_compress_batched(
     void* workspace, size_t workspace_bytes, dct_stream_t stream);
 
 /*
+ * dct_threshold_select_batched -- dct_threshold_select for all the layers of a model at once: the other
+ * half of the layer-wise scheme of Sec. 2.1 (every L iterations each layer gets a new threshold of its
+ * own).  Three streaming passes over all layers together -- every CTA works through a contiguous run of
+ * 8192-element chunks and keeps the digit histogram of the layer it is in -- each followed by one small
+ * kernel that scans every layer's histogram: seven launches whatever the number of layers.
+ *
+ * For every layer l:  *layers[l].tau_out = layers[l].k-th largest |fl32(grad + residual)| of that layer,
+ * and layers[l].result->n_gt / n_eq / status are filled as by dct_threshold_select.
+ *
+ *   layers     HOST array of num_layers descriptions (device pointers inside; residual may be NULL;
+ *              1 <= k <= n <= 2^31-1 per layer, and the sizes must add up to less than 2^44).  Read before the
+ *              call returns.  Layers must not share tau_out or result.
+ *   workspace  DEVICE, >= dct_threshold_select_batched_workspace_bytes(num_layers), 256-byte aligned.
+ * Errors: DCT_ERR_INVALID_ARG / DCT_ERR_WORKSPACE as for dct_threshold_select, before anything is launched.
+ */
+typedef struct {
+  const float* grad;           /* [n] device, read only */
+  const float* residual;       /* [n] device, read only, or NULL */
+  uint64_t n;
+  uint64_t k;
+  float* tau_out;              /* device scalar */
+  dct_result_t* result;        /* device */
+} dct_select_layer_t;
+DCT_API size_t dct_threshold_select_batched_workspace_bytes(uint32_t num_layers);
+DCT_API dct_status_t dct_threshold_select_batched(
+    const dct_select_layer_t* layers /* host */, uint32_t num_layers,
+    void* workspace, size_t workspace_bytes, dct_stream_t stream);
+
+/*
  * dct_dp_select_compress -- Algorithm 1 with threshold life-span L = 1: the branch "L divides the
  * iteration number" taken at every iteration, i.e. top-K sparsification with error feedback where the
  * threshold comes from the very vector that is compressed (the scheme the paper starts from, and on

@@ -33,6 +33,7 @@ EXPORTED_SYMBOLS = (
     "dct_dp_compress_batched", "dct_dp_compress_batched_workspace_bytes",
     "dct_threshold_select_multi", "dct_threshold_select_multi_workspace_bytes",
     "dct_mp_threshold_mean", "dct_dp_drift_check",
+    "dct_threshold_select_batched", "dct_threshold_select_batched_workspace_bytes",
 )
 
 _vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
@@ -106,6 +107,10 @@ def lib() -> ctypes.CDLL:
     L.dct_mp_threshold_mean.argtypes = [_vp, _int, _u32, _u32, _u32, _vp, _u32, _vp, _vp, _vp]
     L.dct_dp_drift_check.restype = _int
     L.dct_dp_drift_check.argtypes = [_vp, _u64, _u32, _u32, _vp, _vp]
+    L.dct_threshold_select_batched_workspace_bytes.restype = _sz
+    L.dct_threshold_select_batched_workspace_bytes.argtypes = [_u32]
+    L.dct_threshold_select_batched.restype = _int
+    L.dct_threshold_select_batched.argtypes = [_vp, _u32, _vp, _sz, _vp]
     L.dct_debug_configure.restype = None
     L.dct_debug_configure.argtypes = [_u32, _u32]
     _lib = L
@@ -506,3 +511,40 @@ def dct_dp_drift_check(compress_result, k, ratio_num, ratio_den, flag_out, strea
     _need(flag_out, torch.int32, "flag_out")
     _check("dct_dp_drift_check",
            lib().dct_dp_drift_check(_p(compress_result), k, ratio_num, ratio_den, _p(flag_out), _stream(stream)))
+
+
+# ----------------------------------------------------------------------------
+# thresholds of all layers at once
+# ----------------------------------------------------------------------------
+
+class _SelectLayer(ctypes.Structure):      # dct_select_layer_t
+    _fields_ = [("grad", _vp), ("residual", _vp), ("n", _u64), ("k", _u64), ("tau_out", _vp), ("result", _vp)]
+
+
+def dct_threshold_select_batched_workspace_bytes(num_layers: int) -> int:
+    return lib().dct_threshold_select_batched_workspace_bytes(num_layers)
+
+
+def dct_select_layer_table(layers):
+    """Marshal a sequence of layer dicts (keys of dct_select_layer_t: grad, residual or None, n, k, tau_out,
+    result) into the host array the C call takes."""
+    table = (_SelectLayer * len(layers))()
+    for slot, a in zip(table, layers):
+        _need(a["grad"], torch.float32, "grad")
+        if a.get("residual") is not None:
+            _need(a["residual"], torch.float32, "residual")
+        _need(a["tau_out"], torch.float32, "tau_out")
+        _need(a["result"], torch.int64, "result")
+        if a["grad"].numel() < a["n"] or (a.get("residual") is not None and a["residual"].numel() < a["n"]):
+            raise ValueError("buffer smaller than n")
+        slot.grad, slot.residual, slot.n, slot.k = _p(a["grad"]), _p(a.get("residual")), a["n"], a["k"]
+        slot.tau_out, slot.result = _p(a["tau_out"]), _p(a["result"])
+    return table
+
+
+def dct_threshold_select_batched(layers, workspace, stream=None) -> None:
+    """``layers``: a table from dct_select_layer_table, or the sequence of layer dicts it is built from."""
+    table = layers if isinstance(layers, ctypes.Array) else dct_select_layer_table(layers)
+    _need(workspace, torch.uint8, "workspace")
+    _check("dct_threshold_select_batched",
+           lib().dct_threshold_select_batched(table, len(table), _p(workspace), workspace.numel(), _stream(stream)))

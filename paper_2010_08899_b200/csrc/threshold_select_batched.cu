@@ -1,0 +1,258 @@
+// dct_threshold_select_batched: Algorithm 1 (DCT-DP), threshold steps, for all the layers of a model at
+// once (Sec. 2.1: each layer has a threshold of its own, renewed every L iterations).
+//
+// The same most-significant-digit-first radix select as dct_threshold_select (digits of 11/10/10 bits
+// over the 31 magnitude bits), carried out for every layer in the same three passes.  The elements of all
+// layers are cut into chunks of 8192; every CTA takes a contiguous run of chunks, so it changes layer
+// rarely, keeps the digit histogram of the layer it is in in shared memory and merges it into that
+// layer's histogram in global memory when it moves on.  After each pass one CTA per layer scans the
+// layer's histogram from the top, picks the digit that holds rank k and extends the layer's prefix.
+#include <cstddef>
+#include <vector>
+
+#include "common.cuh"
+
+namespace dct {
+namespace {
+
+constexpr int kThreads = 512;
+constexpr int kVecs = 4;
+constexpr uint32_t kChunk = kThreads * kVecs * 4;            // 8192 elements
+constexpr int kBins = 2048;
+constexpr int kPasses = 3;
+
+__host__ __device__ constexpr int pass_shift(int p) { return p == 0 ? 20 : (p == 1 ? 10 : 0); }
+__host__ __device__ constexpr int pass_bits(int p) { return p == 0 ? 11 : 10; }
+
+struct LayerState {                 // device copy of a layer's description + its select in flight
+    const float* grad;
+    const float* residual;
+    float* tau_out;
+    dct_result_t* result;
+    uint64_t first_chunk;           // index of the layer's first chunk among all chunks
+    uint64_t n_gt;                  // elements known to be above the prefix bucket
+    uint32_t n, k;
+    uint32_t prefix, k_rem;
+    uint32_t hist[kPasses][kBins];
+};
+
+// chunk -> layer: the last layer whose first chunk is <= chunk
+__device__ __forceinline__ uint32_t layer_of_chunk(const LayerState* layers, uint32_t num_layers, uint64_t chunk) {
+    uint32_t lo = 0, hi = num_layers - 1;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi + 1) >> 1;
+        if (layers[mid].first_chunk <= chunk) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+__global__ void batched_init_kernel(LayerState* layers, uint32_t num_layers) {
+    // the description part has been copied in; clear the select state, the histograms and the result
+    for (uint32_t l = blockIdx.x; l < num_layers; l += gridDim.x) {
+        LayerState* st = layers + l;
+        uint32_t* h = &st->hist[0][0];
+        for (uint32_t b = threadIdx.x; b < kPasses * kBins; b += blockDim.x) h[b] = 0;
+        if (threadIdx.x == 0) {
+            st->n_gt = 0;
+            st->prefix = 0;
+            st->k_rem = st->k;
+            dct_result_t* r = st->result;
+            r->status = DCT_OK;
+            r->reserved = 0;
+            r->count = 0;
+            r->needed = 0;
+            r->n_gt = 0;
+            r->n_eq = 0;
+        }
+    }
+}
+
+template <int kPass>
+__global__ void __launch_bounds__(kThreads)
+batched_pass_kernel(LayerState* layers, uint32_t num_layers, uint64_t total_chunks) {
+    constexpr int shift = pass_shift(kPass);
+    constexpr int bits = pass_bits(kPass);
+    constexpr uint32_t digit_mask = (1u << bits) - 1u;
+    __shared__ uint32_t sh[kBins];
+
+    // this CTA's contiguous run of chunks
+    const uint64_t per_cta = (total_chunks + gridDim.x - 1) / gridDim.x;
+    const uint64_t c_begin = static_cast<uint64_t>(blockIdx.x) * per_cta;
+    const uint64_t c_end = c_begin + per_cta < total_chunks ? c_begin + per_cta : total_chunks;
+    if (c_begin >= c_end) return;
+
+    for (int b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0;
+    uint32_t layer = layer_of_chunk(layers, num_layers, c_begin);
+    __syncthreads();
+
+    auto flush = [&](uint32_t l) {          // merge the shared histogram into layer l's and clear it
+        __syncthreads();
+        uint32_t* hist = layers[l].hist[kPass];
+        for (int b = threadIdx.x; b < kBins; b += kThreads) {
+            const uint32_t c = sh[b];
+            if (c) {
+                atomicAdd(&hist[b], c);
+                sh[b] = 0;
+            }
+        }
+        __syncthreads();
+    };
+
+    for (uint64_t chunk = c_begin; chunk < c_end; ++chunk) {
+        while (layer + 1 < num_layers && layers[layer + 1].first_chunk <= chunk) {     // the run has entered the next layer
+            flush(layer);
+            ++layer;
+        }
+        const LayerState& st = layers[layer];
+        const float* __restrict__ grad = st.grad;
+        const float* __restrict__ residual = st.residual;
+        const uint32_t n = st.n;
+        const uint32_t prefix = kPass == 0 ? 0u : st.prefix;      // written by the scan kernel of the previous pass
+        const uint32_t base = static_cast<uint32_t>(chunk - st.first_chunk) * kChunk;
+        auto consume = [&](uint32_t key) {
+            if (kPass == 0 || (key >> (shift + bits)) == prefix) atomicAdd(&sh[(key >> shift) & digit_mask], 1u);
+        };
+        const bool vec = (reinterpret_cast<uintptr_t>(grad) & 15u) == 0 &&
+                         (residual == nullptr || (reinterpret_cast<uintptr_t>(residual) & 15u) == 0);
+        if (vec && base + kChunk <= n) {
+            float4 g4[kVecs], e4[kVecs];
+#pragma unroll
+            for (int j = 0; j < kVecs; ++j) {
+                const uint32_t off = base + (j * kThreads + threadIdx.x) * 4;
+                g4[j] = ld_readonly_f4(grad + off);
+                e4[j] = residual ? ld_readonly_f4(residual + off) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            const bool add = residual != nullptr;
+#pragma unroll
+            for (int j = 0; j < kVecs; ++j) {
+                consume(key_f32(add ? __fadd_rn(g4[j].x, e4[j].x) : g4[j].x));
+                consume(key_f32(add ? __fadd_rn(g4[j].y, e4[j].y) : g4[j].y));
+                consume(key_f32(add ? __fadd_rn(g4[j].z, e4[j].z) : g4[j].z));
+                consume(key_f32(add ? __fadd_rn(g4[j].w, e4[j].w) : g4[j].w));
+            }
+        } else {
+            for (uint32_t i = base + threadIdx.x; i < n && i < base + kChunk; i += kThreads)
+                consume(key_f32(residual ? __fadd_rn(grad[i], residual[i]) : grad[i]));
+        }
+    }
+    flush(layer);
+}
+
+// One CTA per layer: the digit that holds rank k_rem, counted from the top of the layer's histogram.
+template <int kPass>
+__global__ void __launch_bounds__(kThreads)
+batched_scan_kernel(LayerState* layers, uint32_t num_layers) {
+    constexpr int bits = pass_bits(kPass);
+    __shared__ uint32_t s_scan[kThreads / 32];
+    for (uint32_t l = blockIdx.x; l < num_layers; l += gridDim.x) {
+        LayerState* st = layers + l;
+        const uint32_t* hist = st->hist[kPass];
+        const uint32_t prefix = kPass == 0 ? 0u : st->prefix;
+        const uint32_t k_rem = st->k_rem;
+        // thread t owns bins top-down: bin(t, q) = kBins-1 - (4t + q), q = 0..3
+        uint32_t c[4], own = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            c[q] = hist[kBins - 1 - (4 * threadIdx.x + q)];
+            own += c[q];
+        }
+        const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+        uint32_t incl = own;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= static_cast<uint32_t>(o)) incl += t;
+        }
+        if (lane == 31) s_scan[warp] = incl;
+        __syncthreads();                       // also: every thread has read prefix and k_rem
+        uint32_t above = incl - own;
+        for (uint32_t v = 0; v < warp; ++v) above += s_scan[v];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (above < k_rem && k_rem <= above + c[q]) {
+                const uint32_t digit = kBins - 1 - (4 * threadIdx.x + q);
+                const uint32_t new_prefix = (prefix << bits) | digit;
+                const uint64_t n_gt = st->n_gt + above;
+                st->prefix = new_prefix;
+                st->k_rem = k_rem - above;
+                st->n_gt = n_gt;
+                if (kPass == kPasses - 1) {
+                    *st->tau_out = __uint_as_float(new_prefix);
+                    st->result->n_gt = n_gt;
+                    st->result->n_eq = c[q];
+                }
+            }
+            above += c[q];
+        }
+        __syncthreads();                       // s_scan is reused for the next layer
+    }
+}
+
+}  // namespace
+}  // namespace dct
+
+using namespace dct;
+
+extern "C" size_t dct_threshold_select_batched_workspace_bytes(uint32_t num_layers) {
+    if (num_layers == 0) return 0;
+    return (static_cast<size_t>(num_layers) * sizeof(LayerState) + 255) & ~static_cast<size_t>(255);
+}
+
+extern "C" dct_status_t dct_threshold_select_batched(const dct_select_layer_t* layers, uint32_t num_layers,
+                                                     void* workspace, size_t workspace_bytes, dct_stream_t stream_) {
+    if (!layers || num_layers == 0) return DCT_ERR_INVALID_ARG;
+    uint64_t total_chunks = 0, total_elems = 0;
+    for (uint32_t l = 0; l < num_layers; ++l) {
+        const dct_select_layer_t& a = layers[l];
+        if (!a.grad || !a.tau_out || !a.result || a.n == 0 || a.n > 0x7FFFFFFFull || a.k == 0 || a.k > a.n)
+            return DCT_ERR_INVALID_ARG;
+        if (!aligned_to(a.grad, 4) || (a.residual && !aligned_to(a.residual, 4)) || !aligned_to(a.tau_out, 4) ||
+            !aligned_to(a.result, 8))
+            return DCT_ERR_INVALID_ARG;
+        total_elems += a.n;
+    }
+    if (total_elems >= (1ull << 44)) return DCT_ERR_INVALID_ARG;
+    if (!workspace || !aligned_to(workspace, 256) ||
+        workspace_bytes < dct_threshold_select_batched_workspace_bytes(num_layers))
+        return DCT_ERR_WORKSPACE;
+
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    auto* dev_layers = static_cast<LayerState*>(workspace);
+    // Only the description (the head of every LayerState) travels; the histograms are cleared on the device.
+    struct Head {
+        const float* grad;
+        const float* residual;
+        float* tau_out;
+        dct_result_t* result;
+        uint64_t first_chunk;
+        uint64_t n_gt;
+        uint32_t n, k;
+    };
+    static_assert(sizeof(Head) <= offsetof(LayerState, prefix), "head must not reach into the select state");
+    std::vector<Head> heads(num_layers);
+    for (uint32_t l = 0; l < num_layers; ++l) {
+        const dct_select_layer_t& a = layers[l];
+        heads[l] = Head{a.grad, a.residual, a.tau_out, a.result, total_chunks, 0, static_cast<uint32_t>(a.n),
+                        static_cast<uint32_t>(a.k)};
+        total_chunks += (a.n + kChunk - 1) / kChunk;
+    }
+    // pageable source: the runtime has staged the bytes by the time each call returns, so `heads` may go away
+    DCT_CUDA_TRY(cudaMemcpy2DAsync(dev_layers, sizeof(LayerState), heads.data(), sizeof(Head), sizeof(Head), num_layers,
+                                   cudaMemcpyHostToDevice, stream));
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint32_t init_grid = num_layers < 1024u ? num_layers : 1024u;
+    batched_init_kernel<<<init_grid, kThreads, 0, stream>>>(dev_layers, num_layers);
+    DCT_CUDA_TRY(cudaGetLastError());
+    const uint64_t want = static_cast<uint64_t>(sms) * 4;
+    const uint32_t grid = static_cast<uint32_t>(total_chunks < want ? total_chunks : want);
+    const uint32_t scan_grid = num_layers < static_cast<uint32_t>(sms) * 4u ? num_layers : static_cast<uint32_t>(sms) * 4u;
+    batched_pass_kernel<0><<<grid, kThreads, 0, stream>>>(dev_layers, num_layers, total_chunks);
+    batched_scan_kernel<0><<<scan_grid, kThreads, 0, stream>>>(dev_layers, num_layers);
+    batched_pass_kernel<1><<<grid, kThreads, 0, stream>>>(dev_layers, num_layers, total_chunks);
+    batched_scan_kernel<1><<<scan_grid, kThreads, 0, stream>>>(dev_layers, num_layers);
+    batched_pass_kernel<2><<<grid, kThreads, 0, stream>>>(dev_layers, num_layers, total_chunks);
+    batched_scan_kernel<2><<<scan_grid, kThreads, 0, stream>>>(dev_layers, num_layers);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}

@@ -53,17 +53,35 @@ def main():
                     total += sizes[-1]
         g_all = inputs.dp_dlrm_like(args.n, 301, dev)
         e_all = torch.zeros(args.n, device=dev)
-        layers, off = [], 0
+        layers, sel_layers, off = [], [], 0
         for m in sizes:
             cap = max(m // 16, 64)
             tau = torch.zeros(1, device=dev)
-            r = B.new_result(dev)
-            B.dct_threshold_select(g_all[off:off + m], None, m, B.k_from_density(m, 1, 1000), tau, r,
-                                   B.new_workspace(B.dct_threshold_select_workspace_bytes(m), dev))
+            sel_layers.append(dict(grad=g_all[off:off + m], residual=None, n=m, k=B.k_from_density(m, 1, 1000),
+                                   tau_out=tau, result=B.new_result(dev)))
             layers.append(dict(grad=g_all[off:off + m], residual=e_all[off:off + m], n=m, tau=tau, tie_budget=None,
                                idx_out=torch.empty(cap, dtype=torch.int32, device=dev),
-                               val_out=torch.empty(cap, device=dev), capacity=cap, result=r))
+                               val_out=torch.empty(cap, device=dev), capacity=cap, result=B.new_result(dev)))
             off += m
+        # the thresholds of all layers: one batched call against one dct_threshold_select call per layer
+        ws_sb = B.new_workspace(B.dct_threshold_select_batched_workspace_bytes(len(sizes)), dev)
+        ws_s1 = B.new_workspace(B.dct_threshold_select_workspace_bytes(max(sizes)), dev)
+        sel_table = B.dct_select_layer_table(sel_layers)
+        sel_variants = {
+            f"select, batched ({len(sizes)} layers, one call)": lambda: B.dct_threshold_select_batched(sel_table, ws_sb),
+            f"select, one call per layer ({len(sizes)} calls)": lambda: [B.dct_threshold_select(
+                a["grad"], None, a["n"], a["k"], a["tau_out"], a["result"], ws_s1) for a in sel_layers],
+        }
+        for name, fn in sel_variants.items():
+            for phase in range(2):
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                fn()
+                b.record(stream)
+                b.synchronize()
+            ms = a.elapsed_time(b)
+            print(f"compress_layers, {name}: {ms:.4f} ms, {4 * args.n / ms / 1e6:.1f} GB/s at the 4 B floor")
         ws_b = B.new_workspace(B.dct_dp_compress_batched_workspace_bytes(sizes), dev)
         ws_1 = B.new_workspace(B.dct_dp_compress_workspace_bytes(max(sizes)), dev)
         table = B.dct_dp_layer_table(layers)      # marshalled once, as a trainer would

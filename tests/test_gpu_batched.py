@@ -67,3 +67,81 @@ def test_batched_rejects_bad_layers_on_the_host():
     with pytest.raises(B.DctError):
         B.dct_dp_compress_batched([layers[0], bad], ws)
     assert B.dct_dp_compress_batched_workspace_bytes([0]) == 0
+
+
+def _select_layers(sizes, seed, misalign=(), with_residual=True):
+    layers = []
+    for j, n in enumerate(sizes):
+        g = inputs.dp_dlrm_like(n, seed + 3 * j, G.DEV) * (0.1 + j % 5) if n > 64 else inputs.dp_gaussian(n, seed + 3 * j, G.DEV)
+        e = inputs.dp_gaussian(n, seed + 3 * j + 1, G.DEV) * 0.05 if (with_residual and j % 3 != 2) else None
+        if j % 4 == 1:
+            g = inputs.quantize_mantissa(g, 3)                  # heavy ties in some layers
+        if j in misalign:
+            g = G.offset_copy(g, 1)
+            e = None if e is None else G.offset_copy(e, 3)
+        k = [1, max(1, n // 1000), max(1, n // 20), max(1, n // 4), n][j % 5]
+        layers.append(dict(grad=g, residual=e, n=n, k=k, tau_out=torch.full((3,), -7.0, device=G.DEV),
+                           result=B.new_result()))
+    return layers
+
+
+@pytest.mark.parametrize("sizes,misalign", [
+    ([1], ()), ([8192], ()), ([8193, 1, 8191], ()),
+    ([131072, 16384, 1048576, 524288, 131072, 256, 3, 8191, 12289], ()),        # DLRM-like mix plus odd sizes
+    ([70001, 4096 * 3, 100, 262144 + 5, 9999], (0, 3)),                         # some layers not 16-byte aligned
+    ([(1 << 21) + 17] * 2 + [64] * 300, (41,)),                                 # more layers than CTAs, tiny ones
+])
+def test_batched_select_equals_per_layer_oracle(sizes, misalign):
+    """dct_threshold_select_batched: every layer's threshold and counts as the oracle (and the single-vector
+    select) give them for that layer alone."""
+    layers = _select_layers(sizes, 3000 + len(sizes), misalign)
+    ws = B.new_workspace(B.dct_threshold_select_batched_workspace_bytes(len(sizes)))
+    ws.fill_(0xCD)                                            # stale workspace contents must not matter
+    B.dct_threshold_select_batched(layers, ws)
+    for j, a in enumerate(layers):
+        e = None if a["residual"] is None else a["residual"].cpu().numpy()
+        want = oracle.dp_select(a["grad"].cpu().numpy(), e, a["k"])
+        r = B.read_result(a["result"])
+        assert r.status == B.DCT_OK, j
+        assert bits32(a["tau_out"][:1].cpu().numpy())[0] == bits32(want.tau)[0], j
+        assert (r.n_gt, r.n_eq) == (want.n_gt, want.n_eq), j
+        assert bool((a["tau_out"][1:] == -7.0).all()), j
+    # the same call again on the same workspace gives the same answer
+    first = [a["tau_out"][:1].clone() for a in layers]
+    B.dct_threshold_select_batched(layers, ws)
+    assert all(torch.equal(a["tau_out"][:1], t) for a, t in zip(layers, first))
+
+
+def test_batched_select_feeds_batched_compress():
+    """The layer-wise scheme end to end: thresholds of all layers in one call, then all layers compressed in
+    one call with the tie budgets k - n_gt: exactly k survivors per layer."""
+    sizes = [131072, 16384, 262144, 65536, 131072, 256]
+    sel = _select_layers(sizes, 4000, with_residual=True)
+    for a in sel:
+        a["k"] = max(1, a["n"] // 100)
+        if a["residual"] is None:
+            a["residual"] = torch.zeros(a["n"], device=G.DEV)
+    B.dct_threshold_select_batched(sel, B.new_workspace(B.dct_threshold_select_batched_workspace_bytes(len(sizes))))
+    layers = []
+    for a in sel:
+        r = B.read_result(a["result"])
+        budget = torch.tensor([a["k"] - r.n_gt], dtype=torch.int64, device=G.DEV)
+        layers.append(dict(grad=a["grad"], residual=a["residual"], n=a["n"], tau=a["tau_out"][:1].clone(),
+                           tie_budget=budget, capacity=a["n"],
+                           idx_out=torch.empty(a["n"], dtype=torch.int32, device=G.DEV),
+                           val_out=torch.empty(a["n"], device=G.DEV), result=B.new_result()))
+    B.dct_dp_compress_batched(layers, B.new_workspace(B.dct_dp_compress_batched_workspace_bytes(sizes)))
+    for a, s in zip(layers, sel):
+        r = B.read_result(a["result"])
+        assert (r.status, r.count, r.needed) == (B.DCT_OK, s["k"], s["k"])
+
+
+def test_batched_select_rejects_bad_layers_on_the_host():
+    g = inputs.dp_gaussian(100, 1, G.DEV)
+    ok = dict(grad=g, residual=None, n=100, k=5, tau_out=torch.zeros(1, device=G.DEV), result=B.new_result())
+    ws = B.new_workspace(B.dct_threshold_select_batched_workspace_bytes(2))
+    for bad in (dict(ok, k=0), dict(ok, k=101), dict(ok, n=0)):
+        with pytest.raises(B.DctError):
+            B.dct_threshold_select_batched([ok, bad], ws)
+    with pytest.raises(B.DctError):
+        B.dct_threshold_select_batched([ok, ok], ws[:256])
