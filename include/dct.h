@@ -168,10 +168,17 @@ DCT_API dct_status_t dct_dp_compress(
  *   rows_out [rows*k] int32 or NULL: explicit row id of each slot for callers
  *            that want (row, col, val) triples; the row is otherwise slot / k.
  *   tau_out  [rows] dtype of x_act or NULL: the thresholds tau_i (sign clear).
- *   result   device block or NULL; status is written (always DCT_OK).
+ *   result   device block or NULL; status is written (DCT_OK; see below).
  *
  * x_act rows should start on 16-byte boundaries (base aligned and ld*size a
  * multiple of 16); other layouts are accepted and take a slower scalar load.
+ * Every shape gives the same result; the time does depend on it.  Rows on
+ * 16-byte boundaries with d <= 4096 and d*size a multiple of 16 are packed by
+ * one warp per row (bf16: any k up to d/2 and 1280; fp32: k up to about d/10
+ * and 441); everything else (wider rows, denser k, odd strides) takes a general
+ * kernel that is several times slower.  status may also be DCT_ERR_TIMEOUT if a
+ * bounded wait for an asynchronous copy gave up (not seen in practice; the
+ * outputs are then incomplete).
  */
 DCT_API dct_status_t dct_mp_topk_pack_fwd(
     const void* x_act, dct_dtype_t dtype,
