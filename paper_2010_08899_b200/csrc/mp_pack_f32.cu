@@ -567,6 +567,370 @@ dct_status_t launch_width(const void* x_act, uint32_t rows, uint32_t d, uint32_t
     return launch_variant<E8, 20>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
 }
 
+// ------------------------------------------------------------------------------------------
+// fp32, dense k (up to half the row): one warp per row
+// ------------------------------------------------------------------------------------------
+// As the dense bf16 kernel (mp_pack.cu), on the upper 15 key bits: two bit tables, upper bits >= low and
+// >= low + 64, pin the 15-bit bucket of tau_i inside a 64-bucket window; a 64-bin histogram of the window
+// elements gives the bucket and how many of its members are kept; the members (a handful) are ranked by
+// their full keys, which gives the exact 31-bit tau_i and the ties to keep; then every lane walks its
+// candidate bits in column order and keeps what the full key says.  Kept entries go through staging slots
+// (16-bit column, 32-bit value) to coalesced stores.
+constexpr uint32_t kDenseWindowF32 = 64;
+constexpr uint32_t kDenseMaxKF32 = 1280;
+constexpr int kDenseMaxWarpsF32 = 24;
+constexpr int kDenseRetriesF32 = 6;
+
+template <int E8> struct DenseLayoutF32 {
+    using Row = RowLayoutF32<E8>;
+    static constexpr uint32_t kTabWords = 128;
+    // per warp: row | low table | high table | histogram (64) + member list (1 + 64) | staged values (k) | staged columns (k/2) | mbarrier
+    __host__ __device__ static constexpr uint32_t kpad(uint32_t k) { return (k + 7u) & ~7u; }   // keeps every part a multiple of 16 bytes
+    __host__ __device__ static constexpr uint32_t scratch_words(uint32_t k) {
+        return 2u * kTabWords + 64u + 68u + kpad(k) + kpad(k) / 2u;
+    }
+    __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) { return Row::kRowBytes + scratch_words(k) * 4u + 16u; }
+};
+
+// flags of 8 consecutive fp32: upper 15 key bits >= low, exact for every bit pattern
+__device__ __forceinline__ uint32_t mask8_upper_ge_exact(uint4 a, uint4 b, uint32_t low) {
+    auto ge = [low](uint32_t v) -> uint32_t { return ((v >> 16) & 0x7FFFu) >= low ? 1u : 0u; };
+    return ge(a.x) | (ge(a.y) << 1) | (ge(a.z) << 2) | (ge(a.w) << 3) | (ge(b.x) << 4) | (ge(b.y) << 5) | (ge(b.z) << 6) |
+           (ge(b.w) << 7);
+}
+
+template <int E8>
+__global__ void __launch_bounds__(kDenseMaxWarpsF32 * 32)
+mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                             int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
+                             int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
+                             dct_result_t* __restrict__ result) {
+    using Lay = RowLayoutF32<E8>;
+    using Den = DenseLayoutF32<E8>;
+    constexpr int kMaskWords = Lay::kMaskWords;
+    constexpr uint32_t kGuessMargin = 32;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    unsigned char* base = smem_raw + warp * Den::warp_bytes(k);
+    unsigned char* span = base + lane * (Lay::E * 4u);
+    uint32_t* scratch = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
+    uint32_t* tab_low = scratch;
+    uint32_t* tab_high = scratch + Den::kTabWords;
+    uint32_t* hist = scratch + 2u * Den::kTabWords;            // 64 bins
+    uint32_t* n_members = hist + 64;                           // 1 word, then up to 64 member keys
+    uint32_t* members = n_members + 1;
+    uint32_t* stage_val = hist + 64 + 68;
+    uint16_t* stage_col = reinterpret_cast<uint16_t*>(stage_val + Den::kpad(k));
+    uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Den::scratch_words(k));
+    const uint32_t* row32 = reinterpret_cast<const uint32_t*>(base);
+    __shared__ uint32_t s_stop;
+
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+    if (threadIdx.x == 0) s_stop = 0;
+    if (lane == 0) {
+        mbar_init(bar, 1);
+        mbar_init_fence();
+        fence_proxy_async_all();
+    }
+    const uint32_t row_bytes = d * 4u;                         // the tail of the buffer stays zero
+    for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
+        *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+
+    const uint32_t warp_global = blockIdx.x + gridDim.x * warp;
+    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
+    auto request_row = [&](uint32_t r) {
+        if (lane == 0) {
+            mbar_arrive_expect_tx(bar, row_bytes);
+            bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, bar);
+        }
+    };
+    auto release_row = [&](uint32_t row) {
+        __syncwarp();
+        fence_proxy_async_smem();
+        if (row + total_warps < rows) request_row(row + total_warps);
+    };
+    // 32-byte pieces (8 columns, one table byte), halves read in a lane-dependent order: see the sparse kernel
+    const uint32_t swap = (lane >> 2) & 1u;
+    const unsigned char* piece_first = base + lane * 32u + swap * 16u;
+    const unsigned char* piece_second = base + lane * 32u + (swap ^ 1u) * 16u;
+    const uint32_t e_first = swap * 4u, e_second = (swap ^ 1u) * 4u;
+    const uint32_t c_first_01 = (1u << e_first) | (1u << (17u + e_first));
+    const uint32_t c_first_23 = (4u << e_first) | (4u << (17u + e_first));
+    const uint32_t c_second_01 = (1u << e_second) | (1u << (17u + e_second));
+    const uint32_t c_second_23 = (4u << e_second) | (4u << (17u + e_second));
+    if (warp_global < rows) request_row(warp_global);
+
+    uint32_t use = 0;
+    uint32_t guess_low = 0;
+    for (uint32_t row = warp_global; row < rows; row += total_warps, ++use) {
+        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
+            s_stop = 1;
+            if (lane == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
+            return;
+        }
+        const size_t out_base = static_cast<size_t>(row) * k;
+
+        // ---- A: bounds around the upper 15 bits of tau_i ------------------------------------------------
+        uint32_t low = guess_low;
+        if (low == 0) {
+            // no previous row: a conservative (k/d)-quantile of up to 128 samples (column 0 of up to four pieces)
+            constexpr int kSamples = E8 < 4 ? E8 : 4;
+            uint32_t sample[kSamples];
+#pragma unroll
+            for (int c = 0; c < kSamples; ++c)
+                sample[c] = (*reinterpret_cast<const uint32_t*>(base + lane * 32u + c * 1024) >> 16) & 0x7FFFu;
+            const uint32_t n_samples = 32u * kSamples;
+            uint32_t rank = (n_samples * k + d - 1) / d;
+            rank += 2u * static_cast<uint32_t>(__fsqrt_rn(static_cast<float>(rank))) + 2u;
+            if (rank > n_samples) rank = n_samples;
+#pragma unroll 1
+            for (int bit = 14; bit >= 0; --bit) {
+                const uint32_t trial = low | (1u << bit);
+                uint32_t cnt = 0;
+#pragma unroll
+                for (int c = 0; c < kSamples; ++c) cnt += sample[c] >= trial ? 1u : 0u;
+                if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= rank) low = trial;
+            }
+            if (low == 0) low = 1;
+        }
+        uint32_t geL[kMaskWords], geH[kMaskWords];
+        uint32_t n_low = 0, n_high = 0, before_packed = 0;
+        bool pinned = false;
+        uint32_t step = kDenseWindowF32;
+        int last_move = 0;
+#pragma unroll 1
+        for (int attempt = 0; attempt < kDenseRetriesF32; ++attempt) {
+            const uint32_t high = low + kDenseWindowF32;
+            unsigned char* tl = reinterpret_cast<unsigned char*>(tab_low) + lane;
+            unsigned char* th = reinterpret_cast<unsigned char*>(tab_high) + lane;
+            __syncwarp();
+            if (low >= 0x0080u && high <= 0x7F80u) {
+                // normal bounds: the packed compare on the upper halves is exact (a NaN lands in both tables)
+                const __nv_bfloat162 low2 = as_bf162(low * 0x10001u), high2 = as_bf162(high * 0x10001u);
+#pragma unroll
+                for (int c = 0; c < E8; ++c) {
+                    const uint4 a = *reinterpret_cast<const uint4*>(piece_first + c * 1024);
+                    const uint4 b = *reinterpret_cast<const uint4*>(piece_second + c * 1024);
+                    const __nv_bfloat162 h0 = __habs2(as_bf162(upper_halves(a.x, a.y))), h1 = __habs2(as_bf162(upper_halves(a.z, a.w)));
+                    const __nv_bfloat162 h2 = __habs2(as_bf162(upper_halves(b.x, b.y))), h3 = __habs2(as_bf162(upper_halves(b.z, b.w)));
+                    const uint32_t ml = (__hgeu2_mask(h0, low2) & c_first_01) | (__hgeu2_mask(h1, low2) & c_first_23) |
+                                        (__hgeu2_mask(h2, low2) & c_second_01) | (__hgeu2_mask(h3, low2) & c_second_23);
+                    const uint32_t mh = (__hgeu2_mask(h0, high2) & c_first_01) | (__hgeu2_mask(h1, high2) & c_first_23) |
+                                        (__hgeu2_mask(h2, high2) & c_second_01) | (__hgeu2_mask(h3, high2) & c_second_23);
+                    tl[c * 32] = static_cast<unsigned char>(ml | (ml >> 16));
+                    th[c * 32] = static_cast<unsigned char>(mh | (mh >> 16));
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < E8; ++c) {
+                    const uint4 a = *reinterpret_cast<const uint4*>(base + lane * 32u + c * 1024);
+                    const uint4 b = *reinterpret_cast<const uint4*>(base + lane * 32u + c * 1024 + 16);
+                    tl[c * 32] = static_cast<unsigned char>(mask8_upper_ge_exact(a, b, low));
+                    th[c * 32] = static_cast<unsigned char>(mask8_upper_ge_exact(a, b, high));
+                }
+            }
+            __syncwarp();
+            uint32_t mine = 0;
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) {
+                const uint32_t w = lane * kMaskWords + i;
+                const bool real = Lay::kRowWords == Lay::kTableWords || w < Lay::kRowWords;
+                geL[i] = real ? tab_low[w] : 0u;
+                geH[i] = real ? tab_high[w] : 0u;
+                mine += (__popc(geL[i]) << 16) | __popc(geH[i]);
+            }
+            const uint32_t incl = warp_inclusive_sum(mine);
+            const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            n_low = total >> 16;
+            n_high = total & 0xFFFFu;
+            before_packed = incl - mine;
+            if (n_high < k && k <= n_low) {
+                pinned = true;
+                break;
+            }
+            const int move = n_low < k ? -1 : 1;
+            if (attempt > 0) step = (move == last_move) ? step * 2u : (step > kDenseWindowF32 ? step / 2u : kDenseWindowF32);
+            last_move = move;
+            if (move < 0) {
+                if (low == 1) break;
+                low = low > step ? low - step : 1u;
+            } else {
+                low = low + step < 0x7F80u ? low + step : 0x7F80u;
+            }
+        }
+        if (!pinned) {
+            mp_row_slow_path_f32<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
+            release_row(row);
+            continue;
+        }
+
+        // ---- B: the bucket of tau_i, then tau_i among its members ------------------------------------------
+        hist[lane] = 0;
+        hist[lane + 32] = 0;
+        if (lane == 0) *n_members = 0;
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < kMaskWords; ++i) {
+            uint32_t m = geL[i] & ~geH[i];
+            const uint32_t col0 = (lane * kMaskWords + i) * 32u;
+            while (m) {
+                const uint32_t col = col0 + (__ffs(m) - 1);
+                m &= m - 1;
+                atomicAdd(&hist[(((row32[col] >> 16) & 0x7FFFu) - low) & 63u], 1u);
+            }
+        }
+        __syncwarp();
+        uint32_t tau15, take15;
+        {
+            const uint32_t drop = n_low - k;
+            const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];
+            const uint32_t own = h.x + h.y;
+            const uint32_t before = warp_inclusive_sum(own) - own;
+            uint32_t my_tau = 0, my_take = 0;
+            bool mine = false;
+            if (before <= drop && drop < before + h.x) {
+                mine = true;
+                my_tau = low + 2u * lane;
+                my_take = h.x - (drop - before);
+            } else if (before + h.x <= drop && drop < before + own) {
+                mine = true;
+                my_tau = low + 2u * lane + 1u;
+                my_take = h.y - (drop - before - h.x);
+            }
+            const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
+            const int src = who ? __ffs(who) - 1 : 0;
+            tau15 = __shfl_sync(0xFFFFFFFFu, my_tau, src);
+            take15 = __shfl_sync(0xFFFFFFFFu, my_take, src);
+        }
+        guess_low = tau15 > kGuessMargin ? tau15 - kGuessMargin : 1u;
+        // members of the bucket: full keys into the list
+#pragma unroll
+        for (int i = 0; i < kMaskWords; ++i) {
+            uint32_t m = geL[i] & ~geH[i];
+            const uint32_t col0 = (lane * kMaskWords + i) * 32u;
+            while (m) {
+                const uint32_t col = col0 + (__ffs(m) - 1);
+                m &= m - 1;
+                const uint32_t key = row32[col] & 0x7FFFFFFFu;
+                if ((key >> 16) == tau15) {
+                    const uint32_t slot = atomicAdd(n_members, 1u);
+                    if (slot < 64u) members[slot] = key;
+                }
+            }
+        }
+        __syncwarp();
+        const uint32_t n_mem = *n_members;
+        if (n_mem > 64u) {                                     // too many to rank here (coarse or tied data)
+            mp_row_slow_path_f32<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
+            release_row(row);
+            continue;
+        }
+        uint32_t tau_key = 0, take = 0;
+        for (uint32_t j = lane; j < ((n_mem + 31u) & ~31u); j += 32) {
+            const bool have = j < n_mem;
+            const uint32_t mine = have ? members[j] : 0u;
+            uint32_t greater = 0, equal = 0;
+            for (uint32_t i = 0; i < n_mem; ++i) {
+                const uint32_t other = members[i];
+                greater += other > mine ? 1u : 0u;
+                equal += other == mine ? 1u : 0u;
+            }
+            const uint32_t hit = __ballot_sync(0xFFFFFFFFu, have && greater < take15 && take15 <= greater + equal);
+            if (hit) {
+                const int src = __ffs(hit) - 1;
+                tau_key = __shfl_sync(0xFFFFFFFFu, mine, src);
+                take = take15 - __shfl_sync(0xFFFFFFFFu, greater, src);
+            }
+        }
+        if (lane == 0 && tau_out) tau_out[row] = tau_key;
+
+        // ---- C: ordered emit ------------------------------------------------------------------------
+        uint32_t counts = (before_packed & 0xFFFFu) << 16;         // kept for sure (high table) before this lane
+        {
+            uint32_t mine = 0;                                     // (window elements > tau << 16) | window elements == tau
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) {
+                uint32_t m = geL[i] & ~geH[i];
+                const uint32_t col0 = (lane * kMaskWords + i) * 32u;
+                while (m) {
+                    const uint32_t col = col0 + (__ffs(m) - 1);
+                    m &= m - 1;
+                    const uint32_t key = row32[col] & 0x7FFFFFFFu;
+                    mine += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
+                }
+            }
+            counts += warp_inclusive_sum(mine) - mine;
+        }
+        {
+            uint32_t e_at = counts & 0xFFFFu;
+            uint32_t pos = (counts >> 16) + (e_at < take ? e_at : take);
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) {
+                uint32_t m = geL[i];
+                const uint32_t col0 = (lane * kMaskWords + i) * 32u;
+                while (m) {
+                    const uint32_t col = col0 + (__ffs(m) - 1);
+                    m &= m - 1;
+                    const uint32_t v = row32[col];
+                    const uint32_t key = v & 0x7FFFFFFFu;
+                    const bool is_eq = key == tau_key;
+                    const bool keep = key > tau_key || (is_eq && e_at < take);
+                    if (keep) {
+                        stage_val[pos] = v;
+                        stage_col[pos] = static_cast<uint16_t>(col);
+                    }
+                    pos += keep ? 1u : 0u;
+                    e_at += is_eq ? 1u : 0u;
+                }
+            }
+        }
+        release_row(row);
+        for (uint32_t p = lane; p < k; p += 32) {
+            cols_out[out_base + p] = static_cast<int16_t>(stage_col[p]);
+            vals_out[out_base + p] = stage_val[p];
+            if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
+        }
+        __syncwarp();
+    }
+}
+
+template <int E8>
+dct_status_t launch_dense(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
+                          void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result, cudaStream_t stream) {
+    using Den = DenseLayoutF32<E8>;
+    auto kernel = mp_topk_fwd_f32_dense_kernel<E8>;
+    constexpr size_t kSmemBudget = 220 * 1024;
+    static thread_local int configured_device = -1;
+    int dev = 0;
+    DCT_CUDA_TRY(cudaGetDevice(&dev));
+    if (configured_device != dev) {
+        DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(kSmemBudget)));
+        configured_device = dev;
+    }
+    const size_t per_warp = Den::warp_bytes(k);
+    size_t warps = kSmemBudget / per_warp;
+    if (warps > static_cast<size_t>(kDenseMaxWarpsF32)) warps = kDenseMaxWarpsF32;
+    if (warps < 1) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
+    const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
+    kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
+        static_cast<const uint32_t*>(x_act), rows, d, ld, k, cols_out, static_cast<uint32_t*>(vals_out), rows_out,
+        static_cast<uint32_t*>(tau_out), result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}
+
 }  // namespace
 
 // *handled = false: the shape is not one of the fast path's; the caller runs the general kernel.
@@ -575,7 +939,22 @@ dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, u
                                  dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
     if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 4 != 0 || d > 4096) return DCT_OK;
-    if (fwd_candidates_per_lane(d, k) == 0) return DCT_OK;
+    if (fwd_candidates_per_lane(d, k) == 0) {
+        // dense k (beyond the candidate registers, up to half the row): bounds + bit tables
+        // (rows of more than 2048 columns leave too few warps per SM for it: the general kernel is as fast there)
+        if (k > kDenseMaxKF32 || k > d / 2 || d > 2048) return DCT_OK;
+        *handled = true;
+#define DCT_F32_DENSE(E8) \
+    if (d <= 256u * E8)   \
+        return launch_dense<E8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+        DCT_F32_DENSE(1);
+        DCT_F32_DENSE(2);
+        DCT_F32_DENSE(4);
+        DCT_F32_DENSE(8);
+#undef DCT_F32_DENSE
+        *handled = false;
+        return DCT_OK;
+    }
     *handled = true;
 #define DCT_F32_WIDTH(E8) \
     if (d <= 256u * E8)   \

@@ -173,7 +173,7 @@ def test_mp_f32_keys_that_differ_only_in_the_low_bits():
     x = ((hi << 16) | lo | sign).view(torch.float32).contiguous()
     x[300:400, 1000:] = 0.0                                 # ~1000 live columns: buckets of ~60 members
     gx = inputs.mp_gradients(rows, d, 6, device=G.DEV)
-    for kk in (k, 17, 448):
+    for kk in (k, 17, 448, 1024, 2048):
         _compare_fwd_bwd(x, gx, d, kk)
 
 
@@ -217,8 +217,9 @@ def test_mp_warp_per_row_widths_between_the_buffer_sizes(dtype, d):
         assert int(cols.max()) < d
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("d", [512, 1024, 2000, 4096])
-def test_mp_bf16_dense_k(d):
+def test_mp_dense_k(dtype, d):
     """k from a quarter to half of the row (75 % sparsity and below): tau_i is pinned between two bit tables
     64 keys apart.  Rows whose scale jumps by orders of magnitude make the window move several times;
     ties, dead rows and rows with fewer than k non-zeros take the remaining branches."""
@@ -231,8 +232,8 @@ def test_mp_bf16_dense_k(d):
     x[4] = 2.0                                      # every element ties
     x[5, d // 3:] = 0.0                             # fewer than d/2 non-zeros
     x[6] = inputs.quantize_mantissa(x[6], 1)        # few distinct values
-    x[7] = 3.0e38                                   # the top of the bf16 range
-    x = x.to(torch.bfloat16).contiguous()
-    gx = inputs.mp_gradients(rows, d, 54 + d, dtype=torch.bfloat16, device=G.DEV)
+    x[7] = 3.0e38                                   # the top of the range
+    x = x.to(dtype).contiguous()
+    gx = inputs.mp_gradients(rows, d, 54 + d, dtype=dtype, device=G.DEV)
     for k in sorted({d // 4 + 1, d // 3, d // 2, min(d // 2, 1280)}):
         _compare_fwd_bwd(x, gx, d, k)
