@@ -2,6 +2,8 @@
 every case is compared with the oracle bit for bit.  The fixed cases of the other test files aim at
 known corners; this file looks for the unknown ones (a shape that straddles two code paths, an odd
 combination of stride and width, a value pattern nobody thought of)."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -13,6 +15,9 @@ from tests import _gpu as G
 from tests._util import bits32
 
 pytestmark = pytest.mark.gpu
+
+# DCT_SWEEP_SEED=<int> in the environment runs the sweep on another set of cases
+SEED = int(os.environ.get("DCT_SWEEP_SEED", "0"))
 
 
 def _mp_case(rng: np.random.Generator, case: int):
@@ -55,8 +60,8 @@ def _mp_case(rng: np.random.Generator, case: int):
 
 @pytest.mark.parametrize("chunk", range(16))
 def test_mp_random_cases(chunk):
-    rng = np.random.default_rng(100 + chunk)
-    for case in range(chunk * 12, chunk * 12 + 12):
+    rng = np.random.default_rng(100 + chunk + 1000 * SEED)
+    for case in range(chunk * 12 + 10000 * SEED, chunk * 12 + 12 + 10000 * SEED):
         x, gx, d, k = _mp_case(rng, case)
         what = f"case {case}: {tuple(x.shape)} d={d} k={k} {x.dtype}"
         want = oracle.mp_fwd(G.to_oracle(x), k, d=d)
@@ -72,8 +77,8 @@ def test_mp_random_cases(chunk):
 
 @pytest.mark.parametrize("chunk", range(10))
 def test_dp_random_cases(chunk):
-    rng = np.random.default_rng(200 + chunk)
-    for case in range(chunk * 6, chunk * 6 + 6):
+    rng = np.random.default_rng(200 + chunk + 1000 * SEED)
+    for case in range(chunk * 6 + 10000 * SEED, chunk * 6 + 6 + 10000 * SEED):
         n = int(rng.choice([int(rng.integers(1, 5000)), int(rng.integers(5000, 200_000)),
                             4096 * int(rng.integers(1, 300)) + int(rng.integers(-2, 3)),
                             int(rng.integers(200_000, 3_000_000))]))
