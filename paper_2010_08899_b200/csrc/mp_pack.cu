@@ -151,7 +151,7 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
 }
 
 // ------------------------------------------------------------------------------------------
-// bf16 fast path: one warp per row, d <= 4096 a multiple of 8 (held in a buffer of 256 * E8 columns), rows on 16-byte boundaries
+// bf16 fast path: one warp per row, d <= 8192 a multiple of 8 (held in a buffer of 256 * E8 columns), rows on 16-byte boundaries
 // ------------------------------------------------------------------------------------------
 // One bulk asynchronous copy brings a row into shared memory exactly as it lies in HBM; the next row is
 // requested as soon as the candidates of the current one sit in registers.
@@ -250,8 +250,15 @@ __device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_
     if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
 }
 
+// Warps of a CTA: as many row buffers as shared memory holds, at most FwdVariant<PL>::kMaxWarps (wide rows leave
+// fewer warps and therefore more registers for each of them).
+template <int E8, int PL> constexpr int fwd_bf16_max_warps() {
+    constexpr int by_smem = static_cast<int>((220u * 1024u) / WarpRowLayout<E8>::warp_bytes(1));
+    return by_smem < FwdVariant<PL>::kMaxWarps ? by_smem : FwdVariant<PL>::kMaxWarps;
+}
+
 template <int E8, int PL>
-__global__ void __launch_bounds__(FwdVariant<PL>::kMaxWarps * 32)
+__global__ void __launch_bounds__(fwd_bf16_max_warps<E8, PL>() * 32)
 mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
@@ -611,7 +618,7 @@ dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint
                                           cudaStream_t stream) {
     using Lay = WarpRowLayout<E8>;
     auto kernel = mp_topk_fwd_bf16_warp_kernel<E8, PL>;
-    constexpr int kMaxWarps = FwdVariant<PL>::kMaxWarps;
+    constexpr int kMaxWarps = fwd_bf16_max_warps<E8, PL>();
     constexpr size_t kSmemBudget = 220 * 1024;            // of the 227 KiB a CTA may use
     static thread_local int configured_device = -1;
     int dev = 0;
@@ -677,7 +684,7 @@ constexpr int kDenseRetries = 6;
 template <int E8> struct DenseLayout {
     using Row = WarpRowLayout<E8>;
     // per warp: row | low table (128 words) | high table (128 words) | histogram (64 words) | stage (k words) | mbarrier
-    static constexpr uint32_t kTabWords = 128;
+    static constexpr uint32_t kTabWords = Row::kTableWords > 128u ? Row::kTableWords : 128u;
     __host__ __device__ static constexpr uint32_t scratch_words(uint32_t k) { return 2u * kTabWords + 64u + ((k + 3u) & ~3u); }
     __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) { return Row::kRowBytes + scratch_words(k) * 4u + 16u; }
 };
@@ -1046,7 +1053,7 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
         if (narrow != DCT_OK || handled) return narrow;
     }
     // The sparse warp-per-row kernel holds up to 320 or 640 candidates in registers and needs a tight leaf bound.
-    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && d % 8 == 0 && d <= 4096 &&
+    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && d % 8 == 0 && d <= 8192 &&
         fwd_candidates_per_lane(d, k) != 0) {
         // warp-per-row path: the smallest instantiated buffer of 256 * E8 columns that holds the row
 #define DCT_BF16_WIDTH(E8) \
@@ -1064,10 +1071,12 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
         DCT_BF16_WIDTH(12);
         DCT_BF16_WIDTH(14);
         DCT_BF16_WIDTH(16);
+        DCT_BF16_WIDTH(24);
+        DCT_BF16_WIDTH(32);
 #undef DCT_BF16_WIDTH
     }
     // dense k (beyond the candidate registers of the kernels above, up to half the row): bounds + bit tables
-    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && d % 8 == 0 && d <= 4096 && k <= kDenseMaxK &&
+    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && d % 8 == 0 && d <= 8192 && k <= kDenseMaxK &&
         k <= d / 2) {
 #define DCT_BF16_DENSE(E8) \
     if (d <= 256u * E8)    \
@@ -1078,6 +1087,7 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
         DCT_BF16_DENSE(8);
         DCT_BF16_DENSE(12);
         DCT_BF16_DENSE(16);
+        DCT_BF16_DENSE(32);
 #undef DCT_BF16_DENSE
     }
     return launch_fwd<uint16_t>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);

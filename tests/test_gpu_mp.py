@@ -237,3 +237,22 @@ def test_mp_dense_k(dtype, d):
     gx = inputs.mp_gradients(rows, d, 54 + d, dtype=dtype, device=G.DEV)
     for k in sorted({d // 4 + 1, d // 3, d // 2, min(d // 2, 1280)}):
         _compare_fwd_bwd(x, gx, d, k)
+
+
+@pytest.mark.parametrize("d", [5000, 6144, 8000, 8192])
+def test_mp_bf16_wide_rows(d):
+    """bf16 rows of more than 4096 and up to 8192 columns take the warp-per-row kernels too (buffers of 6144
+    and 8192 columns): sparse k with 10 and 20 candidates per lane, dense k, and the degenerate rows."""
+    rows = 700
+    x = inputs.mp_activations(rows, d, 61 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=62 + d)
+    scale = torch.tensor([1.0, 30.0, 1e-2, 1.0, 1.0], device=G.DEV).repeat(rows // 5 + 1)[:rows]
+    x = x * scale[:, None]
+    x[3] = 0.0
+    x[4] = -1.25
+    x[5, 100:] = 0.0
+    x[6] = inputs.quantize_mantissa(x[6], 2)
+    x = x.to(torch.bfloat16).contiguous()
+    gx = inputs.mp_gradients(rows, d, 63 + d, dtype=torch.bfloat16, device=G.DEV)
+    for k in sorted({1, d // 40, d // 20, d // 10, 1000, 1280}):
+        cols = _compare_fwd_bwd(x, gx, d, k)
+        assert int(cols.max()) < d
