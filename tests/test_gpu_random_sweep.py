@@ -35,6 +35,8 @@ def _mp_case(rng: np.random.Generator, case: int):
     d = max(1, d)
     ld = d + (int(rng.integers(0, 3)) * int(rng.choice([1, 4, 8])) if rng.integers(2) else 0)
     rows = int(rng.integers(1, 700)) if d <= 4096 else int(rng.integers(1, 40))
+    if d <= 2048 and rng.integers(6) == 0:              # enough rows that every warp meets several in a row
+        rows = int(rng.integers(4000, 12000))
     kmode = rng.integers(5)
     k = [1, max(1, d // 20), max(1, d // 8), max(1, d // 4), int(rng.integers(1, d + 1))][kmode]
     k = min(k + int(rng.integers(0, 2)), d)
