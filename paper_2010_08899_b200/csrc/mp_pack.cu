@@ -466,10 +466,22 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 if (masks[i]) link = wbase + i;
             }
             uint32_t before = incl - n_mine;
+            if (kMaskWords == 4) {
+                uint32_t y[4];
 #pragma unroll
-            for (int i = 0; i < kMaskWords; ++i) {
-                table[wbase + i] = make_uint2(masks[i], (before << 16) | next_of[i]);
-                before += __popc(masks[i]);
+                for (int i = 0; i < 4; ++i) {
+                    y[i] = (before << 16) | next_of[i % kMaskWords];
+                    before += __popc(masks[i % kMaskWords]);
+                }
+                uint4* t4 = reinterpret_cast<uint4*>(table + wbase);
+                t4[0] = make_uint4(masks[0], y[0], masks[1 % kMaskWords], y[1]);
+                t4[1] = make_uint4(masks[2 % kMaskWords], y[2], masks[3 % kMaskWords], y[3]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < kMaskWords; ++i) {
+                    table[wbase + i] = make_uint2(masks[i], (before << 16) | next_of[i]);
+                    before += __popc(masks[i]);
+                }
             }
         }
         __syncwarp();
@@ -481,7 +493,32 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < per_lane ? n_cand - first : per_lane);
         {
             uint32_t word = 0, m = 0, link = first_word;
-            if (nvalid) {
+            if (kMaskWords == 4) {
+                // the lane whose words hold rank `first`: the last one with (candidates before it) <= first, found
+                // by a binary search over the lanes' running counts (every lane takes part in the shuffles)
+                const uint32_t excl = incl - n_mine;
+                const uint32_t pc = __popc(masks[0]) | (__popc(masks[1 % kMaskWords]) << 8) | (__popc(masks[2 % kMaskWords]) << 16);
+                uint32_t owner = 0, owner_excl = 0;
+#pragma unroll
+                for (int step = 16; step > 0; step >>= 1) {
+                    const uint32_t v = __shfl_sync(0xFFFFFFFFu, excl, owner + step);
+                    if (v <= first) {
+                        owner += step;
+                        owner_excl = v;
+                    }
+                }
+                const uint32_t opc = __shfl_sync(0xFFFFFFFFu, pc, owner);
+                if (nvalid) {
+                    const uint32_t r = first - owner_excl;          // rank inside the owner's four words
+                    const uint32_t p0 = opc & 0xFFu, p01 = p0 + ((opc >> 8) & 0xFFu), p012 = p01 + (opc >> 16);
+                    const uint32_t i = (r >= p0 ? 1u : 0u) + (r >= p01 ? 1u : 0u) + (r >= p012 ? 1u : 0u);
+                    const uint2 e = table[owner * 4u + i];
+                    word = owner * 4u + i;
+                    m = e.x;
+                    link = e.y & 0xFFFFu;
+                    for (uint32_t skip = r - (i == 0 ? 0u : (i == 1 ? p0 : (i == 2 ? p01 : p012))); skip; --skip) m &= m - 1;
+                }
+            } else if (nvalid) {
                 uint32_t lo = 0, hi = Lay::kTableWords - 1;         // largest word with (candidates before it) <= first
                 const uint32_t limit = (first + 1u) << 16;
                 while (lo < hi) {
