@@ -250,11 +250,13 @@ __device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_
     if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
 }
 
-// Warps of a CTA: as many row buffers as shared memory holds, at most FwdVariant<PL>::kMaxWarps (wide rows leave
-// fewer warps and therefore more registers for each of them).
+// Warps of a CTA: as many row buffers as shared memory holds (wide rows leave fewer warps and therefore more
+// registers for each of them), at most 32 with up to 10 candidates per lane (the kernel then fits 64 registers;
+// 32 warps against 24 are worth 7 to 11 % on rows of 2048 and 1024 columns) and 20 with 20 per lane.
 template <int E8, int PL> constexpr int fwd_bf16_max_warps() {
     constexpr int by_smem = static_cast<int>((220u * 1024u) / WarpRowLayout<E8>::warp_bytes(1));
-    return by_smem < FwdVariant<PL>::kMaxWarps ? by_smem : FwdVariant<PL>::kMaxWarps;
+    constexpr int by_regs = PL <= 10 ? 32 : 20;
+    return by_smem < by_regs ? by_smem : by_regs;
 }
 
 template <int E8, int PL>
@@ -565,7 +567,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 #pragma unroll
             for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
                 const uint32_t rel = (ent[i] & 0x7FFFu) - low;
-                atomicAdd(&hist[rel < 64u ? rel : 64u + lane], 1u);
+                atomicAdd(&hist[min(rel, 64u + lane)], 1u);
             }
             __syncwarp();
             const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
@@ -638,11 +640,25 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             }
         }
         __syncwarp();
-        for (uint32_t p = lane; p < k; p += 32) {
-            const uint32_t e = stage[p];
-            cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
-            vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
-            if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
+        {
+            // the first 256 slots with constant offsets from one pointer each, any further ones in a loop
+            int16_t* cp = cols_out + out_base + lane;
+            uint16_t* vp = vals_out + out_base + lane;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                if (lane + 32u * j < k) {
+                    const uint32_t e = stage[lane + 32 * j];
+                    cp[32 * j] = static_cast<int16_t>(e >> 16);
+                    vp[32 * j] = static_cast<uint16_t>(e & 0xFFFFu);
+                }
+            }
+            for (uint32_t p = lane + 256u; p < k; p += 32) {
+                const uint32_t e = stage[p];
+                cp[p - lane] = static_cast<int16_t>(e >> 16);
+                vp[p - lane] = static_cast<uint16_t>(e & 0xFFFFu);
+            }
+            if (rows_out)
+                for (uint32_t p = lane; p < k; p += 32) rows_out[out_base + p] = static_cast<int32_t>(row);
         }
         __syncwarp();
     }
