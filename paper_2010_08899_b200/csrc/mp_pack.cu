@@ -282,6 +282,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     uint32_t* stage = scratch;                                // the k kept entries, column order (last use)
     uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Lay::scratch_words(k));
     __shared__ uint32_t s_stop;
+    __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
 
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
         result->status = DCT_OK;
@@ -291,7 +292,10 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         result->n_gt = 0;
         result->n_eq = 0;
     }
-    if (threadIdx.x == 0) s_stop = 0;
+    if (threadIdx.x == 0) {
+        s_stop = 0;
+        s_next = blockDim.x >> 5;
+    }
     if (lane == 0) {
         mbar_init(bar, 1);
         mbar_init_fence();
@@ -304,10 +308,11 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
-    // rows are dealt out CTA by CTA (row mod grid = CTA), then warp by warp: every SM gets the same number of
-    // rows to within one, and the last, partly filled round is spread over all SMs
+    // Rows are dealt out CTA by CTA (row mod grid = CTA): every SM gets the same number of rows to within one.
+    // Inside the CTA a warp takes the CTA's next row whenever it lets go of one (a counter in shared memory): the
+    // warps drift apart by up to a row's time, and the rows of the last, partly filled round go to the warps that
+    // are ahead instead of to fixed ones.
     const uint32_t warp_global = blockIdx.x + gridDim.x * warp;             // this warp's first row
-    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
     auto request_row = [&](uint32_t r) {          // one bulk copy brings the whole row
         if (lane == 0) {
             mbar_arrive_expect_tx(bar, row_bytes);
@@ -317,16 +322,22 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     // In the passes over the whole row lane l reads the 16-byte units l, l + 32, l + 64, ...: the 32 lanes of a
     // 128-bit load then touch 512 consecutive bytes (no bank conflict for any row width).
     const unsigned char* unit0 = base + lane * 16u;
-    auto release_row = [&](uint32_t row) {   // the row buffer is no longer needed: request the next row
+    uint64_t next_row = 0;
+    auto release_row = [&]() {               // the row buffer is no longer needed: request the next row
         __syncwarp();
         fence_proxy_async_smem();
-        if (row + total_warps < rows) request_row(row + total_warps);
+        uint32_t j = 0;
+        if (lane == 0) j = atomicAdd(&s_next, 1u);
+        j = __shfl_sync(0xFFFFFFFFu, j, 0);
+        next_row = blockIdx.x + static_cast<uint64_t>(gridDim.x) * j;
+        if (next_row < rows) request_row(static_cast<uint32_t>(next_row));
     };
     if (warp_global < rows) request_row(warp_global);
 
     uint32_t use = 0;
     uint32_t guess_low = 0;                         // bound guessed from the previous row (0: none)
-    for (uint32_t row = warp_global; row < rows; row += total_warps, ++use) {
+    for (uint64_t row64 = warp_global; row64 < rows; row64 = next_row, ++use) {
+        const uint32_t row = static_cast<uint32_t>(row64);
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
             s_stop = 1;
             if (lane == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
@@ -439,7 +450,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         }
         if (!have_bound || n_cand > kRound || low == 0) {
             mp_row_slow_path<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
-            release_row(row);
+            release_row();
             continue;
         }
 
@@ -550,7 +561,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 ent[i] = static_cast<uint32_t>(i) < nvalid ? e : 0u;
             }
         }
-        release_row(row);
+        release_row();
 
         // ---- C: k-th largest of the candidates --------------------------------------------------
         uint32_t tau_key = 0, take = 0;
@@ -764,6 +775,7 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
     uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Den::scratch_words(k));
     const uint16_t* row16 = reinterpret_cast<const uint16_t*>(base);
     __shared__ uint32_t s_stop;
+    __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
 
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
         result->status = DCT_OK;
@@ -773,7 +785,10 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
         result->n_gt = 0;
         result->n_eq = 0;
     }
-    if (threadIdx.x == 0) s_stop = 0;
+    if (threadIdx.x == 0) {
+        s_stop = 0;
+        s_next = blockDim.x >> 5;
+    }
     if (lane == 0) {
         mbar_init(bar, 1);
         mbar_init_fence();
@@ -785,24 +800,29 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
     __syncthreads();
 
     const uint32_t warp_global = blockIdx.x + gridDim.x * warp;
-    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
     auto request_row = [&](uint32_t r) {
         if (lane == 0) {
             mbar_arrive_expect_tx(bar, row_bytes);
             bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, bar);
         }
     };
-    auto release_row = [&](uint32_t row) {
+    uint64_t next_row = 0;
+    auto release_row = [&]() {               // the row buffer is no longer needed: request the CTA's next row
         __syncwarp();
         fence_proxy_async_smem();
-        if (row + total_warps < rows) request_row(row + total_warps);
+        uint32_t j = 0;
+        if (lane == 0) j = atomicAdd(&s_next, 1u);
+        j = __shfl_sync(0xFFFFFFFFu, j, 0);
+        next_row = blockIdx.x + static_cast<uint64_t>(gridDim.x) * j;
+        if (next_row < rows) request_row(static_cast<uint32_t>(next_row));
     };
     const unsigned char* unit0 = base + lane * 16u;
     if (warp_global < rows) request_row(warp_global);
 
     uint32_t use = 0;
     uint32_t guess_low = 0;
-    for (uint32_t row = warp_global; row < rows; row += total_warps, ++use) {
+    for (uint64_t row64 = warp_global; row64 < rows; row64 = next_row, ++use) {
+        const uint32_t row = static_cast<uint32_t>(row64);
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
             s_stop = 1;
             if (lane == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
@@ -897,7 +917,7 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
         }
         if (!pinned) {
             mp_row_slow_path<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
-            release_row(row);
+            release_row();
             continue;
         }
 
@@ -980,7 +1000,7 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
                 }
             }
         }
-        release_row(row);
+        release_row();
         for (uint32_t p = lane; p < k; p += 32) {
             const uint32_t e = stage[p];
             cols_out[out_base + p] = static_cast<int16_t>(e >> 16);

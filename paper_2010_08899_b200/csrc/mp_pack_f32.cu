@@ -130,6 +130,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
     uint32_t* stage_val = scratch + Lay::kpad(k);
     uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Lay::scratch_words(k));
     __shared__ uint32_t s_stop;
+    __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
 
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
         result->status = DCT_OK;
@@ -139,7 +140,10 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
         result->n_gt = 0;
         result->n_eq = 0;
     }
-    if (threadIdx.x == 0) s_stop = 0;
+    if (threadIdx.x == 0) {
+        s_stop = 0;
+        s_next = blockDim.x >> 5;
+    }
     if (lane == 0) {
         mbar_init(bar, 1);
         mbar_init_fence();
@@ -152,20 +156,24 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
         *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
 
-    // rows are dealt out CTA by CTA (row mod grid = CTA), then warp by warp: every SM gets the same number of
-    // rows to within one, and the last, partly filled round is spread over all SMs
+    // rows are dealt out CTA by CTA (row mod grid = CTA); inside the CTA a warp takes the CTA's next row whenever
+    // it lets go of one (see the bf16 kernel in mp_pack.cu)
     const uint32_t warp_global = blockIdx.x + gridDim.x * warp;             // this warp's first row
-    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
     auto request_row = [&](uint32_t r) {          // one bulk copy brings the whole row
         if (lane == 0) {
             mbar_arrive_expect_tx(bar, row_bytes);
             bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, bar);
         }
     };
-    auto release_row = [&](uint32_t row) {   // the row buffer is no longer needed: request the next row
+    uint64_t next_row = 0;
+    auto release_row = [&]() {               // the row buffer is no longer needed: request the CTA's next row
         __syncwarp();
         fence_proxy_async_smem();
-        if (row + total_warps < rows) request_row(row + total_warps);
+        uint32_t j = 0;
+        if (lane == 0) j = atomicAdd(&s_next, 1u);
+        j = __shfl_sync(0xFFFFFFFFu, j, 0);
+        next_row = blockIdx.x + static_cast<uint64_t>(gridDim.x) * j;
+        if (next_row < rows) request_row(static_cast<uint32_t>(next_row));
     };
     // In the passes over the whole row lane l reads the 32-byte pieces l, l + 32, ... (8 columns each, one byte
     // of the bit table).  The two 16-byte halves of a piece are read in an order that depends on the lane, so
@@ -184,7 +192,8 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
 
     uint32_t use = 0;
     uint32_t guess_low = 0;                         // 15-bit bound guessed from the previous row (0: none)
-    for (uint32_t row = warp_global; row < rows; row += total_warps, ++use) {
+    for (uint64_t row64 = warp_global; row64 < rows; row64 = next_row, ++use) {
+        const uint32_t row = static_cast<uint32_t>(row64);
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
             s_stop = 1;
             if (lane == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
@@ -298,7 +307,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
         }
         if (!have_bound || n_cand > kRound || low == 0) {
             mp_row_slow_path_f32<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
-            release_row(row);
+            release_row();
             continue;
         }
 
@@ -402,7 +411,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 ent_col[i] = live ? col : 0u;
             }
         }
-        release_row(row);
+        release_row();
 
         // ---- D: the 15-bit bucket of tau_i and how many of its members are kept -------------------------
         uint32_t tau15 = 0, take15 = 0;
@@ -661,6 +670,7 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
     uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Den::scratch_words(k));
     const uint32_t* row32 = reinterpret_cast<const uint32_t*>(base);
     __shared__ uint32_t s_stop;
+    __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
 
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
         result->status = DCT_OK;
@@ -670,7 +680,10 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
         result->n_gt = 0;
         result->n_eq = 0;
     }
-    if (threadIdx.x == 0) s_stop = 0;
+    if (threadIdx.x == 0) {
+        s_stop = 0;
+        s_next = blockDim.x >> 5;
+    }
     if (lane == 0) {
         mbar_init(bar, 1);
         mbar_init_fence();
@@ -682,17 +695,21 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
     __syncthreads();
 
     const uint32_t warp_global = blockIdx.x + gridDim.x * warp;
-    const uint32_t total_warps = gridDim.x * (blockDim.x >> 5);
     auto request_row = [&](uint32_t r) {
         if (lane == 0) {
             mbar_arrive_expect_tx(bar, row_bytes);
             bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, bar);
         }
     };
-    auto release_row = [&](uint32_t row) {
+    uint64_t next_row = 0;
+    auto release_row = [&]() {               // the row buffer is no longer needed: request the CTA's next row
         __syncwarp();
         fence_proxy_async_smem();
-        if (row + total_warps < rows) request_row(row + total_warps);
+        uint32_t j = 0;
+        if (lane == 0) j = atomicAdd(&s_next, 1u);
+        j = __shfl_sync(0xFFFFFFFFu, j, 0);
+        next_row = blockIdx.x + static_cast<uint64_t>(gridDim.x) * j;
+        if (next_row < rows) request_row(static_cast<uint32_t>(next_row));
     };
     // 32-byte pieces (8 columns, one table byte), halves read in a lane-dependent order: see the sparse kernel
     const uint32_t swap = (lane >> 2) & 1u;
@@ -707,7 +724,8 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
 
     uint32_t use = 0;
     uint32_t guess_low = 0;
-    for (uint32_t row = warp_global; row < rows; row += total_warps, ++use) {
+    for (uint64_t row64 = warp_global; row64 < rows; row64 = next_row, ++use) {
+        const uint32_t row = static_cast<uint32_t>(row64);
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
             s_stop = 1;
             if (lane == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
@@ -805,7 +823,7 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
         }
         if (!pinned) {
             mp_row_slow_path_f32<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
-            release_row(row);
+            release_row();
             continue;
         }
 
@@ -867,7 +885,7 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
         const uint32_t n_mem = *n_members;
         if (n_mem > 64u) {                                     // too many to rank here (coarse or tied data)
             mp_row_slow_path_f32<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
-            release_row(row);
+            release_row();
             continue;
         }
         uint32_t tau_key = 0, take = 0;
@@ -929,7 +947,7 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
                 }
             }
         }
-        release_row(row);
+        release_row();
         for (uint32_t p = lane; p < k; p += 32) {
             cols_out[out_base + p] = static_cast<int16_t>(stage_col[p]);
             vals_out[out_base + p] = stage_val[p];
