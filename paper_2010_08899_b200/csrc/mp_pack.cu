@@ -698,6 +698,7 @@ dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint
     if (warps < 1) return DCT_ERR_UNSUPPORTED;
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
+    warps = warps_for_rows(warps, rows, sms);
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
     kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
@@ -1032,6 +1033,7 @@ dct_status_t launch_fwd_bf16_dense(const void* x_act, uint32_t rows, uint32_t d,
     if (warps < 1) return DCT_ERR_UNSUPPORTED;
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
+    warps = warps_for_rows(warps, rows, sms);
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
     kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(

@@ -105,6 +105,13 @@ template <int PL> struct FwdVariant {
 };
 
 
+// Warps per CTA when there are fewer rows than row slots on the device: the rows are spread over all SMs (fewer
+// warps per CTA) instead of filling some SMs and leaving the others idle.
+inline size_t warps_for_rows(size_t max_warps, uint32_t rows, int sms) {
+    const size_t per_sm = (static_cast<size_t>(rows) + static_cast<size_t>(sms) - 1) / static_cast<size_t>(sms);
+    return per_sm >= max_warps ? max_warps : (per_sm < 1 ? 1 : per_sm);
+}
+
 // Which sparse warp-per-row variant fits a shape: candidates per lane (5, 10 or 20), or 0 if none does.
 // The exact bound (k-th largest leaf maximum) leaves k * r candidates, where r grows as k approaches the
 // number of leaves L: measured 99th percentiles on post-ReLU rows with log-normal column scales are
