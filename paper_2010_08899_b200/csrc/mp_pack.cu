@@ -15,6 +15,8 @@
 // Backward: a gather of X_grad through the column list, one warp per row.
 #include "common.cuh"
 #include "row_select.cuh"
+#include <type_traits>
+
 #include "mp_warp.cuh"
 
 namespace dct {
@@ -250,12 +252,19 @@ __device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_
     if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
 }
 
+// Slot counts the tail of the sparse kernel is instantiated for besides PL itself: what rows mostly need when
+// the guessed bound is accepted (k + a few dozen candidates rather than the k * 1.45 the exact bound may leave).
+template <int PL> struct FwdTrips;
+template <> struct FwdTrips<5> { static constexpr uint32_t kFew = 3, kSome = 4; };
+template <> struct FwdTrips<10> { static constexpr uint32_t kFew = 8, kSome = 9; };
+template <> struct FwdTrips<20> { static constexpr uint32_t kFew = 15, kSome = 17; };
+
 // Warps of a CTA: as many row buffers as shared memory holds (wide rows leave fewer warps and therefore more
 // registers for each of them), at most 32 with up to 10 candidates per lane (the kernel then fits 64 registers;
-// 32 warps against 24 are worth 7 to 11 % on rows of 2048 and 1024 columns) and 20 with 20 per lane.
+// 32 warps against 24 are worth 7 to 11 % on rows of 2048 and 1024 columns) and 24 with 20 per lane.
 template <int E8, int PL> constexpr int fwd_bf16_max_warps() {
     constexpr int by_smem = static_cast<int>((220u * 1024u) / WarpRowLayout<E8>::warp_bytes(1));
-    constexpr int by_regs = PL <= 10 ? 32 : 20;
+    constexpr int by_regs = PL <= 10 ? 32 : 24;
     return by_smem < by_regs ? by_smem : by_regs;
 }
 
@@ -498,180 +507,198 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             }
         }
         __syncwarp();
-        // Every lane takes per_lane = ceil(n_cand / 32) consecutive candidates (the last lanes fewer or none).  An unused
-        // slot holds 0: its key is below the bound (low >= 1 here), so the select and the emit skip it unaided.
-        uint32_t ent[kPerLane];
+        // The rest of the row's work runs over the slots a lane holds.  per_lane varies from row to row (2 or 3 for
+        // k = 52 of 1024 columns, 4 or 5 for k = 102 of 2048), so for rows of up to 3072 columns the code is
+        // instantiated for three slot counts and the row takes the smallest that fits: the loops below are unrolled
+        // over exactly that many slots (4 to 11 % faster there).  The kernels for wider rows are larger and lose
+        // more to the extra code than they gain (4096 columns: 16 % slower with three copies, 3 % with two).
         const uint32_t per_lane = (n_cand + 31u) >> 5;
-        const uint32_t first = lane * per_lane;                 // rank of the lane's first candidate
-        const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < per_lane ? n_cand - first : per_lane);
-        {
-            uint32_t word = 0, m = 0, link = first_word;
-            if (kMaskWords == 4) {
-                // the lane whose words hold rank `first`: the last one with (candidates before it) <= first, found
-                // by a binary search over the lanes' running counts (every lane takes part in the shuffles)
-                const uint32_t excl = incl - n_mine;
-                const uint32_t pc = __popc(masks[0]) | (__popc(masks[1 % kMaskWords]) << 8) | (__popc(masks[2 % kMaskWords]) << 16);
-                uint32_t owner = 0, owner_excl = 0;
-#pragma unroll
-                for (int step = 16; step > 0; step >>= 1) {
-                    const uint32_t v = __shfl_sync(0xFFFFFFFFu, excl, owner + step);
-                    if (v <= first) {
-                        owner += step;
-                        owner_excl = v;
+        auto finish_row = [&](auto trips_tag) {
+            constexpr uint32_t kTrips = decltype(trips_tag)::value;
+            // Every lane takes per_lane = ceil(n_cand / 32) consecutive candidates (the last lanes fewer or none).  An unused
+            // slot holds 0: its key is below the bound (low >= 1 here), so the select and the emit skip it unaided.
+            uint32_t ent[kTrips];
+            const uint32_t first = lane * per_lane;                 // rank of the lane's first candidate
+            const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < per_lane ? n_cand - first : per_lane);
+            {
+                uint32_t word = 0, m = 0, link = first_word;
+                if (kMaskWords == 4) {
+                    // the lane whose words hold rank `first`: the last one with (candidates before it) <= first, found
+                    // by a binary search over the lanes' running counts (every lane takes part in the shuffles)
+                    const uint32_t excl = incl - n_mine;
+                    const uint32_t pc = __popc(masks[0]) | (__popc(masks[1 % kMaskWords]) << 8) | (__popc(masks[2 % kMaskWords]) << 16);
+                    uint32_t owner = 0, owner_excl = 0;
+    #pragma unroll
+                    for (int step = 16; step > 0; step >>= 1) {
+                        const uint32_t v = __shfl_sync(0xFFFFFFFFu, excl, owner + step);
+                        if (v <= first) {
+                            owner += step;
+                            owner_excl = v;
+                        }
                     }
-                }
-                const uint32_t opc = __shfl_sync(0xFFFFFFFFu, pc, owner);
-                if (nvalid) {
-                    const uint32_t r = first - owner_excl;          // rank inside the owner's four words
-                    const uint32_t p0 = opc & 0xFFu, p01 = p0 + ((opc >> 8) & 0xFFu), p012 = p01 + (opc >> 16);
-                    const uint32_t i = (r >= p0 ? 1u : 0u) + (r >= p01 ? 1u : 0u) + (r >= p012 ? 1u : 0u);
-                    const uint2 e = table[owner * 4u + i];
-                    word = owner * 4u + i;
+                    const uint32_t opc = __shfl_sync(0xFFFFFFFFu, pc, owner);
+                    if (nvalid) {
+                        const uint32_t r = first - owner_excl;          // rank inside the owner's four words
+                        const uint32_t p0 = opc & 0xFFu, p01 = p0 + ((opc >> 8) & 0xFFu), p012 = p01 + (opc >> 16);
+                        const uint32_t i = (r >= p0 ? 1u : 0u) + (r >= p01 ? 1u : 0u) + (r >= p012 ? 1u : 0u);
+                        const uint2 e = table[owner * 4u + i];
+                        word = owner * 4u + i;
+                        m = e.x;
+                        link = e.y & 0xFFFFu;
+                        for (uint32_t skip = r - (i == 0 ? 0u : (i == 1 ? p0 : (i == 2 ? p01 : p012))); skip; --skip) m &= m - 1;
+                    }
+                } else if (nvalid) {
+                    uint32_t lo = 0, hi = Lay::kTableWords - 1;         // largest word with (candidates before it) <= first
+                    const uint32_t limit = (first + 1u) << 16;
+                    while (lo < hi) {
+                        const uint32_t mid = (lo + hi + 1) >> 1;
+                        if (table[mid].y < limit) lo = mid; else hi = mid - 1;
+                    }
+                    const uint2 e = table[lo];
+                    word = lo;
                     m = e.x;
                     link = e.y & 0xFFFFu;
-                    for (uint32_t skip = r - (i == 0 ? 0u : (i == 1 ? p0 : (i == 2 ? p01 : p012))); skip; --skip) m &= m - 1;
+                    for (uint32_t skip = first - (e.y >> 16); skip; --skip) m &= m - 1;
                 }
-            } else if (nvalid) {
-                uint32_t lo = 0, hi = Lay::kTableWords - 1;         // largest word with (candidates before it) <= first
-                const uint32_t limit = (first + 1u) << 16;
-                while (lo < hi) {
-                    const uint32_t mid = (lo + hi + 1) >> 1;
-                    if (table[mid].y < limit) lo = mid; else hi = mid - 1;
+                // `ahead` is the entry the walk moves to when the current word runs out; it is fetched when the walk
+                // arrives at a word, long before it is needed
+                uint2 ahead = table[link];
+                const uint32_t table_addr = smem_addr(table);
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const bool advance = (m == 0);
+                    m = advance ? ahead.x : m;
+                    word = advance ? link : word;
+                    link = advance ? (ahead.y & 0xFFFFu) : link;
+                    lds64_if(ahead, table_addr + link * 8u, advance);
+                    const uint32_t col = word * 32u + (__ffs(m) - 1);
+                    m &= m - 1;
+                    const uint32_t e = reinterpret_cast<const uint16_t*>(base)[col] | (col << 16);
+                    ent[i] = static_cast<uint32_t>(i) < nvalid ? e : 0u;
                 }
-                const uint2 e = table[lo];
-                word = lo;
-                m = e.x;
-                link = e.y & 0xFFFFu;
-                for (uint32_t skip = first - (e.y >> 16); skip; --skip) m &= m - 1;
             }
-            // `ahead` is the entry the walk moves to when the current word runs out; it is fetched when the walk
-            // arrives at a word, long before it is needed
-            uint2 ahead = table[link];
-            const uint32_t table_addr = smem_addr(table);
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const bool advance = (m == 0);
-                m = advance ? ahead.x : m;
-                word = advance ? link : word;
-                link = advance ? (ahead.y & 0xFFFFu) : link;
-                lds64_if(ahead, table_addr + link * 8u, advance);
-                const uint32_t col = word * 32u + (__ffs(m) - 1);
-                m &= m - 1;
-                const uint32_t e = reinterpret_cast<const uint16_t*>(base)[col] | (col << 16);
-                ent[i] = static_cast<uint32_t>(i) < nvalid ? e : 0u;
-            }
-        }
-        release_row();
+            release_row();
 
-        // ---- C: k-th largest of the candidates --------------------------------------------------
-        uint32_t tau_key = 0, take = 0;
-        bool found = false;
-        {
-            // tau_i is the (n_cand - k + 1)-th smallest candidate.  Usually it lies within 64 keys of the
-            // bound: a 64-bin histogram of the candidates in [low, low + 64), walked from the bottom, finds it.
-            const uint32_t drop = n_cand - k;                 // candidates to discard, smallest first
-            // (everything beyond the window, unused slots included, goes to a bin of the lane's own: no branch)
-            hist[lane] = 0;
-            hist[lane + 32] = 0;
-            hist[lane + 64] = 0;
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t rel = (ent[i] & 0x7FFFu) - low;
-                atomicAdd(&hist[min(rel, 64u + lane)], 1u);
+            // ---- C: k-th largest of the candidates --------------------------------------------------
+            uint32_t tau_key = 0, take = 0;
+            bool found = false;
+            {
+                // tau_i is the (n_cand - k + 1)-th smallest candidate.  Usually it lies within 64 keys of the
+                // bound: a 64-bin histogram of the candidates in [low, low + 64), walked from the bottom, finds it.
+                const uint32_t drop = n_cand - k;                 // candidates to discard, smallest first
+                // (everything beyond the window, unused slots included, goes to a bin of the lane's own: no branch)
+                hist[lane] = 0;
+                hist[lane + 32] = 0;
+                hist[lane + 64] = 0;
+                __syncwarp();
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const uint32_t rel = (ent[i] & 0x7FFFu) - low;
+                    atomicAdd(&hist[min(rel, 64u + lane)], 1u);
+                }
+                __syncwarp();
+                const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
+                const uint32_t own = h.x + h.y;
+                const uint32_t before = warp_inclusive_sum(own) - own;
+                uint32_t my_tau = 0xFFFFFFFFu, my_take = 0;
+                if (before <= drop && drop < before + h.x) {
+                    my_tau = low + 2u * lane;
+                    my_take = h.x - (drop - before);
+                } else if (before + h.x <= drop && drop < before + own) {
+                    my_tau = low + 2u * lane + 1u;
+                    my_take = h.y - (drop - before - h.x);
+                }
+                const uint32_t who = __ballot_sync(0xFFFFFFFFu, my_tau != 0xFFFFFFFFu);
+                if (who) {
+                    const int src = __ffs(who) - 1;
+                    tau_key = __shfl_sync(0xFFFFFFFFu, my_tau, src);
+                    take = __shfl_sync(0xFFFFFFFFu, my_take, src);
+                    found = true;
+                }
+                __syncwarp();
             }
-            __syncwarp();
-            const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
-            const uint32_t own = h.x + h.y;
-            const uint32_t before = warp_inclusive_sum(own) - own;
-            uint32_t my_tau = 0xFFFFFFFFu, my_take = 0;
-            if (before <= drop && drop < before + h.x) {
-                my_tau = low + 2u * lane;
-                my_take = h.x - (drop - before);
-            } else if (before + h.x <= drop && drop < before + own) {
-                my_tau = low + 2u * lane + 1u;
-                my_take = h.y - (drop - before - h.x);
+            if (!found) {
+                // general case: radix select over the candidates, exponent byte then mantissa
+                uint32_t k_rem = k;
+                reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+                reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
+                __syncwarp();
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i)
+                    if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent[i] & 0x7FFFu) >> 7], 1u);
+                __syncwarp();
+                const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
+                __syncwarp();
+                reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+                __syncwarp();
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const uint32_t key = ent[i] & 0x7FFFu;
+                    if (static_cast<uint32_t>(i) < nvalid && (key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
+                }
+                __syncwarp();
+                tau_key = (exp_bin << 7) | pick_mantissa(hist, k_rem, take);
             }
-            const uint32_t who = __ballot_sync(0xFFFFFFFFu, my_tau != 0xFFFFFFFFu);
-            if (who) {
-                const int src = __ffs(who) - 1;
-                tau_key = __shfl_sync(0xFFFFFFFFu, my_tau, src);
-                take = __shfl_sync(0xFFFFFFFFu, my_take, src);
-                found = true;
-            }
-            __syncwarp();
-        }
-        if (!found) {
-            // general case: radix select over the candidates, exponent byte then mantissa
-            uint32_t k_rem = k;
-            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
-            reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i)
-                if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent[i] & 0x7FFFu) >> 7], 1u);
-            __syncwarp();
-            const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
-            __syncwarp();
-            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t key = ent[i] & 0x7FFFu;
-                if (static_cast<uint32_t>(i) < nvalid && (key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
-            }
-            __syncwarp();
-            tau_key = (exp_bin << 7) | pick_mantissa(hist, k_rem, take);
-        }
-        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
-        guess_low = tau_key > kGuessMargin ? tau_key - kGuessMargin : 0u;
+            if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+            guess_low = tau_key > kGuessMargin ? tau_key - kGuessMargin : 0u;
 
-        // ---- D: ordered emit ------------------------------------------------------------------------
-        // The kept entries are placed, in column order, into k staging slots; then they leave with
-        // coalesced stores.
-        __syncwarp();                                         // the select histogram is dead: its words become the stage
-        {
-            uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t key = ent[i] & 0x7FFFu;
-                counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
-            }
-            const uint32_t before = warp_inclusive_sum(counts) - counts;
-            uint32_t e_at = before & 0xFFFFu;                 // ties before this entry
-            uint32_t pos = (before >> 16) + (e_at < take ? e_at : take);   // kept entries before it
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t key = ent[i] & 0x7FFFu;
-                const bool is_eq = key == tau_key;
-                const bool keep = key > tau_key || (is_eq && e_at < take);
-                if (keep) stage[pos] = ent[i];
-                pos += keep ? 1u : 0u;
-                e_at += is_eq ? 1u : 0u;
-            }
-        }
-        __syncwarp();
-        {
-            // the first 256 slots with constant offsets from one pointer each, any further ones in a loop
-            int16_t* cp = cols_out + out_base + lane;
-            uint16_t* vp = vals_out + out_base + lane;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                if (lane + 32u * j < k) {
-                    const uint32_t e = stage[lane + 32 * j];
-                    cp[32 * j] = static_cast<int16_t>(e >> 16);
-                    vp[32 * j] = static_cast<uint16_t>(e & 0xFFFFu);
+            // ---- D: ordered emit ------------------------------------------------------------------------
+            // The kept entries are placed, in column order, into k staging slots; then they leave with
+            // coalesced stores.
+            __syncwarp();                                         // the select histogram is dead: its words become the stage
+            {
+                uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const uint32_t key = ent[i] & 0x7FFFu;
+                    counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
+                }
+                const uint32_t before = warp_inclusive_sum(counts) - counts;
+                uint32_t e_at = before & 0xFFFFu;                 // ties before this entry
+                uint32_t pos = (before >> 16) + (e_at < take ? e_at : take);   // kept entries before it
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const uint32_t key = ent[i] & 0x7FFFu;
+                    const bool is_eq = key == tau_key;
+                    const bool keep = key > tau_key || (is_eq && e_at < take);
+                    if (keep) stage[pos] = ent[i];
+                    pos += keep ? 1u : 0u;
+                    e_at += is_eq ? 1u : 0u;
                 }
             }
-            for (uint32_t p = lane + 256u; p < k; p += 32) {
-                const uint32_t e = stage[p];
-                cp[p - lane] = static_cast<int16_t>(e >> 16);
-                vp[p - lane] = static_cast<uint16_t>(e & 0xFFFFu);
+            __syncwarp();
+            {
+                // the first 256 slots with constant offsets from one pointer each, any further ones in a loop
+                int16_t* cp = cols_out + out_base + lane;
+                uint16_t* vp = vals_out + out_base + lane;
+    #pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (lane + 32u * j < k) {
+                        const uint32_t e = stage[lane + 32 * j];
+                        cp[32 * j] = static_cast<int16_t>(e >> 16);
+                        vp[32 * j] = static_cast<uint16_t>(e & 0xFFFFu);
+                    }
+                }
+                for (uint32_t p = lane + 256u; p < k; p += 32) {
+                    const uint32_t e = stage[p];
+                    cp[p - lane] = static_cast<int16_t>(e >> 16);
+                    vp[p - lane] = static_cast<uint16_t>(e & 0xFFFFu);
+                }
+                if (rows_out)
+                    for (uint32_t p = lane; p < k; p += 32) rows_out[out_base + p] = static_cast<int32_t>(row);
             }
-            if (rows_out)
-                for (uint32_t p = lane; p < k; p += 32) rows_out[out_base + p] = static_cast<int32_t>(row);
+            __syncwarp();
+        };
+        if constexpr (E8 <= 12) {
+            if (per_lane <= FwdTrips<PL>::kFew)
+                finish_row(std::integral_constant<uint32_t, FwdTrips<PL>::kFew>{});
+            else if (per_lane <= FwdTrips<PL>::kSome)
+                finish_row(std::integral_constant<uint32_t, FwdTrips<PL>::kSome>{});
+            else
+                finish_row(std::integral_constant<uint32_t, PL>{});
+        } else {
+            finish_row(std::integral_constant<uint32_t, PL>{});
         }
-        __syncwarp();
     }
 }
 
