@@ -15,8 +15,6 @@
 // Backward: a gather of X_grad through the column list, one warp per row.
 #include "common.cuh"
 #include "row_select.cuh"
-#include <type_traits>
-
 #include "mp_warp.cuh"
 
 namespace dct {
@@ -251,13 +249,6 @@ __device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_
     }
     if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
 }
-
-// Slot counts the tail of the sparse kernel is instantiated for besides PL itself: what rows mostly need when
-// the guessed bound is accepted (k + a few dozen candidates rather than the k * 1.45 the exact bound may leave).
-template <int PL> struct FwdTrips;
-template <> struct FwdTrips<5> { static constexpr uint32_t kFew = 3, kSome = 4; };
-template <> struct FwdTrips<10> { static constexpr uint32_t kFew = 8, kSome = 9; };
-template <> struct FwdTrips<20> { static constexpr uint32_t kFew = 15, kSome = 17; };
 
 // Warps of a CTA: as many row buffers as shared memory holds (wide rows leave fewer warps and therefore more
 // registers for each of them), at most 32 with up to 10 candidates per lane (the kernel then fits 64 registers;

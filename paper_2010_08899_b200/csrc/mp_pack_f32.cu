@@ -349,223 +349,239 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
             }
         }
         __syncwarp();
-        uint32_t ent_val[kPerLane];      // the candidate's 32 bits (0: unused slot, a key below every bound)
-        uint32_t ent_col[kPerLane];
+        // the rest runs over the slots a lane holds, instantiated for the slot counts rows mostly need (see the bf16
+        // kernel in mp_pack.cu); only for rows of up to 2048 columns (4 to 8 % faster there; at 4096 columns the
+        // three copies made the kernel 70 % slower)
         const uint32_t per_lane = (n_cand + 31u) >> 5;
-        const uint32_t first = lane * per_lane;
-        const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < per_lane ? n_cand - first : per_lane);
-        {
-            uint32_t word = 0, m = 0, link = first_word;
-            if (kMaskWords == 4) {
-                // the lane whose words hold rank `first`: the last one with (candidates before it) <= first, found
-                // by a binary search over the lanes' running counts (every lane takes part in the shuffles)
-                const uint32_t excl = incl - n_mine;
-                const uint32_t pc = __popc(masks[0]) | (__popc(masks[1 % kMaskWords]) << 8) | (__popc(masks[2 % kMaskWords]) << 16);
-                uint32_t owner = 0, owner_excl = 0;
-#pragma unroll
-                for (int step = 16; step > 0; step >>= 1) {
-                    const uint32_t v = __shfl_sync(0xFFFFFFFFu, excl, owner + step);
-                    if (v <= first) {
-                        owner += step;
-                        owner_excl = v;
+        auto finish_row = [&](auto trips_tag) {
+            constexpr uint32_t kTrips = decltype(trips_tag)::value;
+            uint32_t ent_val[kTrips];      // the candidate's 32 bits (0: unused slot, a key below every bound)
+            uint32_t ent_col[kTrips];
+            const uint32_t first = lane * per_lane;
+            const uint32_t nvalid = first >= n_cand ? 0u : (n_cand - first < per_lane ? n_cand - first : per_lane);
+            {
+                uint32_t word = 0, m = 0, link = first_word;
+                if (kMaskWords == 4) {
+                    // the lane whose words hold rank `first`: the last one with (candidates before it) <= first, found
+                    // by a binary search over the lanes' running counts (every lane takes part in the shuffles)
+                    const uint32_t excl = incl - n_mine;
+                    const uint32_t pc = __popc(masks[0]) | (__popc(masks[1 % kMaskWords]) << 8) | (__popc(masks[2 % kMaskWords]) << 16);
+                    uint32_t owner = 0, owner_excl = 0;
+    #pragma unroll
+                    for (int step = 16; step > 0; step >>= 1) {
+                        const uint32_t v = __shfl_sync(0xFFFFFFFFu, excl, owner + step);
+                        if (v <= first) {
+                            owner += step;
+                            owner_excl = v;
+                        }
                     }
-                }
-                const uint32_t opc = __shfl_sync(0xFFFFFFFFu, pc, owner);
-                if (nvalid) {
-                    const uint32_t r = first - owner_excl;          // rank inside the owner's four words
-                    const uint32_t p0 = opc & 0xFFu, p01 = p0 + ((opc >> 8) & 0xFFu), p012 = p01 + (opc >> 16);
-                    const uint32_t i = (r >= p0 ? 1u : 0u) + (r >= p01 ? 1u : 0u) + (r >= p012 ? 1u : 0u);
-                    const uint2 e = table[owner * 4u + i];
-                    word = owner * 4u + i;
+                    const uint32_t opc = __shfl_sync(0xFFFFFFFFu, pc, owner);
+                    if (nvalid) {
+                        const uint32_t r = first - owner_excl;          // rank inside the owner's four words
+                        const uint32_t p0 = opc & 0xFFu, p01 = p0 + ((opc >> 8) & 0xFFu), p012 = p01 + (opc >> 16);
+                        const uint32_t i = (r >= p0 ? 1u : 0u) + (r >= p01 ? 1u : 0u) + (r >= p012 ? 1u : 0u);
+                        const uint2 e = table[owner * 4u + i];
+                        word = owner * 4u + i;
+                        m = e.x;
+                        link = e.y & 0xFFFFu;
+                        for (uint32_t skip = r - (i == 0 ? 0u : (i == 1 ? p0 : (i == 2 ? p01 : p012))); skip; --skip) m &= m - 1;
+                    }
+                } else if (nvalid) {
+                    uint32_t lo = 0, hi = Lay::kTableWords - 1;
+                    const uint32_t limit = (first + 1u) << 16;
+                    while (lo < hi) {
+                        const uint32_t mid = (lo + hi + 1) >> 1;
+                        if (table[mid].y < limit) lo = mid; else hi = mid - 1;
+                    }
+                    const uint2 e = table[lo];
+                    word = lo;
                     m = e.x;
                     link = e.y & 0xFFFFu;
-                    for (uint32_t skip = r - (i == 0 ? 0u : (i == 1 ? p0 : (i == 2 ? p01 : p012))); skip; --skip) m &= m - 1;
+                    for (uint32_t skip = first - (e.y >> 16); skip; --skip) m &= m - 1;
                 }
-            } else if (nvalid) {
-                uint32_t lo = 0, hi = Lay::kTableWords - 1;
-                const uint32_t limit = (first + 1u) << 16;
-                while (lo < hi) {
-                    const uint32_t mid = (lo + hi + 1) >> 1;
-                    if (table[mid].y < limit) lo = mid; else hi = mid - 1;
+                uint2 ahead = table[link];
+                const uint32_t table_addr = smem_addr(table);
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const bool advance = (m == 0);
+                    m = advance ? ahead.x : m;
+                    word = advance ? link : word;
+                    link = advance ? (ahead.y & 0xFFFFu) : link;
+                    lds64_if(ahead, table_addr + link * 8u, advance);
+                    const uint32_t col = word * 32u + (__ffs(m) - 1);
+                    m &= m - 1;
+                    const uint32_t v = reinterpret_cast<const uint32_t*>(base)[col];
+                    const bool live = static_cast<uint32_t>(i) < nvalid;
+                    ent_val[i] = live ? v : 0u;
+                    ent_col[i] = live ? col : 0u;
                 }
-                const uint2 e = table[lo];
-                word = lo;
-                m = e.x;
-                link = e.y & 0xFFFFu;
-                for (uint32_t skip = first - (e.y >> 16); skip; --skip) m &= m - 1;
             }
-            uint2 ahead = table[link];
-            const uint32_t table_addr = smem_addr(table);
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const bool advance = (m == 0);
-                m = advance ? ahead.x : m;
-                word = advance ? link : word;
-                link = advance ? (ahead.y & 0xFFFFu) : link;
-                lds64_if(ahead, table_addr + link * 8u, advance);
-                const uint32_t col = word * 32u + (__ffs(m) - 1);
-                m &= m - 1;
-                const uint32_t v = reinterpret_cast<const uint32_t*>(base)[col];
-                const bool live = static_cast<uint32_t>(i) < nvalid;
-                ent_val[i] = live ? v : 0u;
-                ent_col[i] = live ? col : 0u;
-            }
-        }
-        release_row();
+            release_row();
 
-        // ---- D: the 15-bit bucket of tau_i and how many of its members are kept -------------------------
-        uint32_t tau15 = 0, take15 = 0;
-        bool found = false;
-        {
-            const uint32_t drop = n_cand - k;                 // candidates to discard, smallest first
-            hist[lane] = 0;
-            hist[lane + 32] = 0;
-            hist[lane + 64] = 0;
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t rel = ((ent_val[i] >> 16) & 0x7FFFu) - low;
-                atomicAdd(&hist[rel < 64u ? rel : 64u + lane], 1u);
+            // ---- D: the 15-bit bucket of tau_i and how many of its members are kept -------------------------
+            uint32_t tau15 = 0, take15 = 0;
+            bool found = false;
+            {
+                const uint32_t drop = n_cand - k;                 // candidates to discard, smallest first
+                hist[lane] = 0;
+                hist[lane + 32] = 0;
+                hist[lane + 64] = 0;
+                __syncwarp();
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const uint32_t rel = ((ent_val[i] >> 16) & 0x7FFFu) - low;
+                    atomicAdd(&hist[rel < 64u ? rel : 64u + lane], 1u);
+                }
+                __syncwarp();
+                const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
+                const uint32_t own = h.x + h.y;
+                const uint32_t before = warp_inclusive_sum(own) - own;
+                uint32_t my_tau = 0xFFFFFFFFu, my_take = 0;
+                if (before <= drop && drop < before + h.x) {
+                    my_tau = low + 2u * lane;
+                    my_take = h.x - (drop - before);
+                } else if (before + h.x <= drop && drop < before + own) {
+                    my_tau = low + 2u * lane + 1u;
+                    my_take = h.y - (drop - before - h.x);
+                }
+                const uint32_t who = __ballot_sync(0xFFFFFFFFu, my_tau != 0xFFFFFFFFu);
+                if (who) {
+                    const int src = __ffs(who) - 1;
+                    tau15 = __shfl_sync(0xFFFFFFFFu, my_tau, src);
+                    take15 = __shfl_sync(0xFFFFFFFFu, my_take, src);
+                    found = true;
+                }
+                __syncwarp();
             }
-            __syncwarp();
-            const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
-            const uint32_t own = h.x + h.y;
-            const uint32_t before = warp_inclusive_sum(own) - own;
-            uint32_t my_tau = 0xFFFFFFFFu, my_take = 0;
-            if (before <= drop && drop < before + h.x) {
-                my_tau = low + 2u * lane;
-                my_take = h.x - (drop - before);
-            } else if (before + h.x <= drop && drop < before + own) {
-                my_tau = low + 2u * lane + 1u;
-                my_take = h.y - (drop - before - h.x);
+            if (!found) {
+                // general case: radix select over the candidates' upper 15 bits, exponent byte then mantissa
+                uint32_t k_rem = k;
+                reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+                reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
+                __syncwarp();
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i)
+                    if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent_val[i] >> 23) & 0xFFu], 1u);
+                __syncwarp();
+                const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
+                __syncwarp();
+                reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
+                __syncwarp();
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const uint32_t key15 = (ent_val[i] >> 16) & 0x7FFFu;
+                    if (static_cast<uint32_t>(i) < nvalid && (key15 >> 7) == exp_bin) atomicAdd(&hist[key15 & 0x7Fu], 1u);
+                }
+                __syncwarp();
+                tau15 = (exp_bin << 7) | pick_mantissa(hist, k_rem, take15);
+                __syncwarp();
             }
-            const uint32_t who = __ballot_sync(0xFFFFFFFFu, my_tau != 0xFFFFFFFFu);
-            if (who) {
-                const int src = __ffs(who) - 1;
-                tau15 = __shfl_sync(0xFFFFFFFFu, my_tau, src);
-                take15 = __shfl_sync(0xFFFFFFFFu, my_take, src);
-                found = true;
-            }
-            __syncwarp();
-        }
-        if (!found) {
-            // general case: radix select over the candidates' upper 15 bits, exponent byte then mantissa
-            uint32_t k_rem = k;
-            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
-            reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i)
-                if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent_val[i] >> 23) & 0xFFu], 1u);
-            __syncwarp();
-            const uint32_t exp_bin = pick_exponent(hist, row_max >> 7, k_rem);
-            __syncwarp();
-            reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t key15 = (ent_val[i] >> 16) & 0x7FFFu;
-                if (static_cast<uint32_t>(i) < nvalid && (key15 >> 7) == exp_bin) atomicAdd(&hist[key15 & 0x7Fu], 1u);
-            }
-            __syncwarp();
-            tau15 = (exp_bin << 7) | pick_mantissa(hist, k_rem, take15);
-            __syncwarp();
-        }
-        guess_low = tau15 > kGuessMargin ? tau15 - kGuessMargin : 0u;
+            guess_low = tau15 > kGuessMargin ? tau15 - kGuessMargin : 0u;
 
-        // ---- D': exact tau_i among the members of that bucket: the take15-th largest full key ------------
-        uint32_t tau_key = 0, take = 0;
-        {
-            uint32_t* n_members = scratch;                 // the histogram is dead
-            uint32_t* members = scratch + 1;
-            if (lane == 0) *n_members = 0;
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
-                if ((key >> 16) == tau15) {
-                    const uint32_t slot = atomicAdd(n_members, 1u);
-                    if (slot < kMaxMembers) members[slot] = key;
-                }
-            }
-            __syncwarp();
-            const uint32_t n_mem = *n_members;             // >= take15 >= 1
-            if (n_mem <= kMaxMembers) {
-                // lane j ranks members j and j + 32 among all of them
-                for (uint32_t j = lane; j < ((n_mem + 31u) & ~31u); j += 32) {
-                    const bool have = j < n_mem;
-                    const uint32_t mine = have ? members[j] : 0u;
-                    uint32_t greater = 0, equal = 0;
-                    for (uint32_t i = 0; i < n_mem; ++i) {
-                        const uint32_t other = members[i];
-                        greater += other > mine ? 1u : 0u;
-                        equal += other == mine ? 1u : 0u;
-                    }
-                    const uint32_t hit = __ballot_sync(0xFFFFFFFFu, have && greater < take15 && take15 <= greater + equal);
-                    if (hit) {
-                        const int src = __ffs(hit) - 1;
-                        tau_key = __shfl_sync(0xFFFFFFFFu, mine, src);
-                        take = take15 - __shfl_sync(0xFFFFFFFFu, greater, src);
-                    }
-                }
-            } else {
-                // many members (ties, coarse data): the take15-th largest, bit by bit over the lower 16 bits
-                uint32_t prefix = tau15 << 16;
-#pragma unroll 1
-                for (int bit = 15; bit >= 0; --bit) {
-                    const uint32_t trial = prefix | (1u << bit);
-                    uint32_t cnt = 0;
-#pragma unroll
-                    for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                        const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
-                        cnt += ((key >> 16) == tau15 && key >= trial) ? 1u : 0u;
-                    }
-                    if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= take15) prefix = trial;
-                }
-                tau_key = prefix;
-                uint32_t above = 0;
-#pragma unroll
-                for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
+            // ---- D': exact tau_i among the members of that bucket: the take15-th largest full key ------------
+            uint32_t tau_key = 0, take = 0;
+            {
+                uint32_t* n_members = scratch;                 // the histogram is dead
+                uint32_t* members = scratch + 1;
+                if (lane == 0) *n_members = 0;
+                __syncwarp();
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
-                    above += ((key >> 16) == tau15 && key > tau_key) ? 1u : 0u;
+                    if ((key >> 16) == tau15) {
+                        const uint32_t slot = atomicAdd(n_members, 1u);
+                        if (slot < kMaxMembers) members[slot] = key;
+                    }
                 }
-                take = take15 - __reduce_add_sync(0xFFFFFFFFu, above);
+                __syncwarp();
+                const uint32_t n_mem = *n_members;             // >= take15 >= 1
+                if (n_mem <= kMaxMembers) {
+                    // lane j ranks members j and j + 32 among all of them
+                    for (uint32_t j = lane; j < ((n_mem + 31u) & ~31u); j += 32) {
+                        const bool have = j < n_mem;
+                        const uint32_t mine = have ? members[j] : 0u;
+                        uint32_t greater = 0, equal = 0;
+                        for (uint32_t i = 0; i < n_mem; ++i) {
+                            const uint32_t other = members[i];
+                            greater += other > mine ? 1u : 0u;
+                            equal += other == mine ? 1u : 0u;
+                        }
+                        const uint32_t hit = __ballot_sync(0xFFFFFFFFu, have && greater < take15 && take15 <= greater + equal);
+                        if (hit) {
+                            const int src = __ffs(hit) - 1;
+                            tau_key = __shfl_sync(0xFFFFFFFFu, mine, src);
+                            take = take15 - __shfl_sync(0xFFFFFFFFu, greater, src);
+                        }
+                    }
+                } else {
+                    // many members (ties, coarse data): the take15-th largest, bit by bit over the lower 16 bits
+                    uint32_t prefix = tau15 << 16;
+    #pragma unroll 1
+                    for (int bit = 15; bit >= 0; --bit) {
+                        const uint32_t trial = prefix | (1u << bit);
+                        uint32_t cnt = 0;
+    #pragma unroll
+                        for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                            const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
+                            cnt += ((key >> 16) == tau15 && key >= trial) ? 1u : 0u;
+                        }
+                        if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= take15) prefix = trial;
+                    }
+                    tau_key = prefix;
+                    uint32_t above = 0;
+    #pragma unroll
+                    for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                        const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
+                        above += ((key >> 16) == tau15 && key > tau_key) ? 1u : 0u;
+                    }
+                    take = take15 - __reduce_add_sync(0xFFFFFFFFu, above);
+                }
             }
-        }
-        if (lane == 0 && tau_out) tau_out[row] = tau_key;
+            if (lane == 0 && tau_out) tau_out[row] = tau_key;
 
-        // ---- E: ordered emit ------------------------------------------------------------------------
-        __syncwarp();                                         // the member list is dead: its words become the stage
-        {
-            uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
-                counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
-            }
-            const uint32_t before = warp_inclusive_sum(counts) - counts;
-            uint32_t e_at = before & 0xFFFFu;                 // ties before this entry
-            uint32_t pos = (before >> 16) + (e_at < take ? e_at : take);   // kept entries before it
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kPerLane); ++i) {
-                const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
-                const bool is_eq = key == tau_key;
-                const bool keep = key > tau_key || (is_eq && e_at < take);
-                if (keep) {
-                    stage_col[pos] = ent_col[i];
-                    stage_val[pos] = ent_val[i];
+            // ---- E: ordered emit ------------------------------------------------------------------------
+            __syncwarp();                                         // the member list is dead: its words become the stage
+            {
+                uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
+                    counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
                 }
-                pos += keep ? 1u : 0u;
-                e_at += is_eq ? 1u : 0u;
+                const uint32_t before = warp_inclusive_sum(counts) - counts;
+                uint32_t e_at = before & 0xFFFFu;                 // ties before this entry
+                uint32_t pos = (before >> 16) + (e_at < take ? e_at : take);   // kept entries before it
+    #pragma unroll
+                for (int i = 0; i < static_cast<int>(kTrips); ++i) {
+                    const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
+                    const bool is_eq = key == tau_key;
+                    const bool keep = key > tau_key || (is_eq && e_at < take);
+                    if (keep) {
+                        stage_col[pos] = ent_col[i];
+                        stage_val[pos] = ent_val[i];
+                    }
+                    pos += keep ? 1u : 0u;
+                    e_at += is_eq ? 1u : 0u;
+                }
             }
+            __syncwarp();
+            for (uint32_t p = lane; p < k; p += 32) {
+                cols_out[out_base + p] = static_cast<int16_t>(stage_col[p]);
+                vals_out[out_base + p] = stage_val[p];
+                if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
+            }
+            __syncwarp();
+        };
+        if constexpr (E8 <= 8) {
+            if (per_lane <= FwdTrips<PL>::kFew)
+                finish_row(std::integral_constant<uint32_t, FwdTrips<PL>::kFew>{});
+            else if (per_lane <= FwdTrips<PL>::kSome)
+                finish_row(std::integral_constant<uint32_t, FwdTrips<PL>::kSome>{});
+            else
+                finish_row(std::integral_constant<uint32_t, PL>{});
+        } else {
+            finish_row(std::integral_constant<uint32_t, PL>{});
         }
-        __syncwarp();
-        for (uint32_t p = lane; p < k; p += 32) {
-            cols_out[out_base + p] = static_cast<int16_t>(stage_col[p]);
-            vals_out[out_base + p] = stage_val[p];
-            if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
-        }
-        __syncwarp();
     }
 }
 

@@ -1,6 +1,8 @@
 // Pieces shared by the warp-per-row forward kernels of DCT-MP (Algorithm 2): one warp finds the row
 // threshold tau_i and packs the row (bf16: mp_pack.cu; fp32: mp_pack_f32.cu).
 #pragma once
+#include <type_traits>
+
 #include "common.cuh"
 
 namespace dct {
@@ -104,6 +106,13 @@ template <int PL> struct FwdVariant {
     static constexpr bool kFineLeaves = PL > 10;
 };
 
+
+// Slot counts the tail of the sparse kernel is instantiated for besides PL itself: what rows mostly need when
+// the guessed bound is accepted (k + a few dozen candidates rather than the k * 1.45 the exact bound may leave).
+template <int PL> struct FwdTrips;
+template <> struct FwdTrips<5> { static constexpr uint32_t kFew = 3, kSome = 4; };
+template <> struct FwdTrips<10> { static constexpr uint32_t kFew = 8, kSome = 9; };
+template <> struct FwdTrips<20> { static constexpr uint32_t kFew = 15, kSome = 17; };
 
 // Warps per CTA when there are fewer rows than row slots on the device: the rows are spread over all SMs (fewer
 // warps per CTA) instead of filling some SMs and leaving the others idle.
