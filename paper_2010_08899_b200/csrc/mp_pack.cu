@@ -755,9 +755,12 @@ dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t d, 
 //      otherwise low moves (by 64, 128, ... keys) and the pass is repeated, a few times at most.
 //   B  the elements inside the window (in the low table, not in the high one: a handful per lane) are
 //      read and counted into a 64-bin histogram; a scan over it gives tau_i and the number of ties kept.
-//   C  every lane walks its candidate bits in column order: elements of the high table are kept as they
-//      are, window elements are compared with tau_i; kept entries go to k staging slots and leave with
-//      coalesced stores.
+//   C  the kept columns become a third bit table: the high table, plus the window elements above tau_i, plus the
+//      first ties; every table word gets the number of kept entries before it.
+//   D  the k output slots are dealt out evenly, ceil(k / 32) consecutive ones to a lane, which finds the word of
+//      its first slot by bisection over the running counts and walks the kept bits from there; the entries go
+//      through k staging slots to coalesced stores.  (With the columns instead of the slots dealt out evenly the
+//      warp waits for the lane with the most kept columns: 1.4 times the mean for k = 1024 of 4096.)
 // A row for which this fails (tau_i = 0, bounds that do not converge) takes the bit-serial slow path.
 constexpr uint32_t kDenseWindow = 64;
 constexpr uint32_t kDenseMaxK = 1280;                 // staging slots per warp (5 KiB)
@@ -768,7 +771,7 @@ template <int E8> struct DenseLayout {
     using Row = WarpRowLayout<E8>;
     // per warp: row | low table (128 words) | high table (128 words) | histogram (64 words) | stage (k words) | mbarrier
     static constexpr uint32_t kTabWords = Row::kTableWords > 128u ? Row::kTableWords : 128u;
-    __host__ __device__ static constexpr uint32_t scratch_words(uint32_t k) { return 2u * kTabWords + 64u + ((k + 3u) & ~3u); }
+    __host__ __device__ static constexpr uint32_t scratch_words(uint32_t k) { return 2u * kTabWords + 64u + ((k + (k >> 5) + 4u) & ~3u); }
     __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) { return Row::kRowBytes + scratch_words(k) * 4u + 16u; }
 };
 
@@ -781,7 +784,6 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
     using Lay = WarpRowLayout<E8>;
     using Den = DenseLayout<E8>;
     constexpr int kMaskWords = Lay::kMaskWords;
-    constexpr uint32_t kGuessMargin = 32;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
     unsigned char* base = smem_raw + warp * Den::warp_bytes(k);
@@ -840,6 +842,12 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
 
     uint32_t use = 0;
     uint32_t guess_low = 0;
+    // Width of the window in keys.  A wide window rarely misses tau_i, but every element inside it is looked at
+    // one by one, in loops whose length is that of the lane with the most of them (k = 1024 of 4096 post-ReLU
+    // columns: 220 elements in 64 keys, 44 % of the row's time).  The width is halved, down to 16 keys, while a
+    // row finds more than 96 elements in it, and doubled again when a row needs a second pass: a second pass over
+    // the row is cheaper than a crowded window (9 % faster at k = 1024, 11 % at k = 600).
+    uint32_t window = kDenseWindow;
     for (uint64_t row64 = warp_global; row64 < rows; row64 = next_row, ++use) {
         const uint32_t row = static_cast<uint32_t>(row64);
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
@@ -873,15 +881,16 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
             if (low == 0) low = 1;
         }
         uint32_t geL[kMaskWords], geH[kMaskWords];
-        uint32_t n_low = 0, n_high = 0, before_packed = 0;
+        uint32_t n_low = 0, n_high = 0;
         bool pinned = false;
-        uint32_t step = kDenseWindow;
+        uint32_t step = window;
+        bool moved = false;
         int last_move = 0;
 #pragma unroll 1
         for (int attempt = 0; attempt < kDenseRetries; ++attempt) {
             // exact integer compares (the tables decide what is kept, so "a superset" is not enough here);
             // low <= 0x7F80 keeps low + window within their 2^15 range
-            const uint32_t high = low + kDenseWindow;
+            const uint32_t high = low + window;
             unsigned char* tl = reinterpret_cast<unsigned char*>(tab_low) + lane;
             unsigned char* th = reinterpret_cast<unsigned char*>(tab_high) + lane;
             __syncwarp();
@@ -917,7 +926,6 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
             const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
             n_low = total >> 16;
             n_high = total & 0xFFFFu;
-            before_packed = incl - mine;
             if (n_high < k && k <= n_low) {
                 pinned = true;
                 break;
@@ -925,7 +933,8 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
             // move the window: down if too few elements lie above low, up if too many lie above low + window;
             // the step doubles while the direction stays the same and halves when it turns
             const int move = n_low < k ? -1 : 1;
-            if (attempt > 0) step = (move == last_move) ? step * 2u : (step > kDenseWindow ? step / 2u : kDenseWindow);
+            if (attempt > 0) step = (move == last_move) ? step * 2u : (step > window ? step / 2u : window);
+            moved = true;
             last_move = move;
             if (move < 0) {
                 if (low == 1) break;                               // tau_i = 0: fewer than k non-zeros
@@ -978,50 +987,112 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
             take = __shfl_sync(0xFFFFFFFFu, my_take, src);
         }
         if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
-        guess_low = tau_key > kGuessMargin ? tau_key - kGuessMargin : 1u;
+        if (moved)
+            window = window < kDenseWindow ? window * 2u : kDenseWindow;
+        else if (n_low - n_high > 96u && window > 16u)
+            window >>= 1;
+        guess_low = tau_key > window / 2u ? tau_key - window / 2u : 1u;
 
-        // ---- C: ordered emit ------------------------------------------------------------------------
-        // kept entries before this lane: everything in the high table, plus the window elements above tau_i,
-        // plus the first `take` ties
-        uint32_t counts = (before_packed & 0xFFFFu) << 16;         // (kept for sure << 16) | ties, of the lanes before: high part
+        // ---- C: the kept columns as a bit table -------------------------------------------------------------
+        // everything in the high table, plus the window elements above tau_i, plus the first `take` ties
+        uint32_t keep[kMaskWords];
         {
-            uint32_t mine = 0;                                     // (window elements > tau << 16) | window elements == tau
+            uint32_t ties[kMaskWords];
+            uint32_t n_ties = 0;
 #pragma unroll
             for (int i = 0; i < kMaskWords; ++i) {
-                uint32_t m = geL[i] & ~geH[i];
+                uint32_t m = geL[i] & ~geH[i], gt = 0, eq = 0;
                 const uint32_t col0 = (lane * kMaskWords + i) * 32u;
                 while (m) {
-                    const uint32_t col = col0 + (__ffs(m) - 1);
+                    const uint32_t b = __ffs(m) - 1;
                     m &= m - 1;
-                    const uint32_t key = row16[col] & 0x7FFFu;
-                    mine += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
+                    const uint32_t key = row16[col0 + b] & 0x7FFFu;
+                    gt |= (key > tau_key ? 1u : 0u) << b;
+                    eq |= (key == tau_key ? 1u : 0u) << b;
                 }
+                keep[i] = geH[i] | gt;
+                ties[i] = eq;
+                n_ties += __popc(eq);
             }
-            counts += warp_inclusive_sum(mine) - mine;
-        }
-        {
-            uint32_t e_at = counts & 0xFFFFu;                      // ties before this lane
-            uint32_t pos = (counts >> 16) + (e_at < take ? e_at : take);
+            const uint32_t ties_before = warp_inclusive_sum(n_ties) - n_ties;
+            uint32_t room = ties_before < take ? take - ties_before : 0u;   // ties this lane may still keep
 #pragma unroll
             for (int i = 0; i < kMaskWords; ++i) {
-                uint32_t m = geL[i];
-                const uint32_t col0 = (lane * kMaskWords + i) * 32u;
-                while (m) {
-                    const uint32_t col = col0 + (__ffs(m) - 1);
-                    m &= m - 1;
-                    const uint32_t v = row16[col];
-                    const uint32_t key = v & 0x7FFFu;              // >= low; the elements of the high table are > tau_i
-                    const bool is_eq = key == tau_key;
-                    const bool keep = key > tau_key || (is_eq && e_at < take);
-                    if (keep) stage[pos] = v | (col << 16);
-                    pos += keep ? 1u : 0u;
-                    e_at += is_eq ? 1u : 0u;
+                uint32_t e = ties[i];
+                const uint32_t n = __popc(e);
+                if (n > room) {
+                    for (uint32_t extra = n - room; extra; --extra) e &= ~(0x80000000u >> __clz(e));   // highest columns go
+                    room = 0;
+                } else {
+                    room -= n;
+                }
+                keep[i] |= e;
+            }
+        }
+        // the two bit tables make room for one entry per word: {kept columns, kept entries before the word}
+        uint2* ktab = reinterpret_cast<uint2*>(tab_low);
+        {
+            uint32_t mine = 0;
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) mine += __popc(keep[i]);
+            uint32_t before = warp_inclusive_sum(mine) - mine;
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < kMaskWords; ++i) {
+                ktab[lane * kMaskWords + i] = make_uint2(keep[i], before);
+                before += __popc(keep[i]);
+            }
+        }
+        __syncwarp();
+
+        // ---- D: ordered emit, evenly -------------------------------------------------------------------------
+        // Lane l produces the output slots l * per .. l * per + per - 1 (per = ceil(k / 32)): it finds the word that
+        // holds its first slot by bisection over the running counts and walks the kept bits from there.  The entries
+        // pass through a staging area (slot p at word p + p / 32: neither the lanes' writes, 32 slots apart, nor the
+        // coalesced reads meet in a bank).
+        {
+            const uint32_t per = (k + 31u) >> 5;
+            const uint32_t first = lane * per;
+            const uint32_t nvalid = first >= k ? 0u : (k - first < per ? k - first : per);
+            if (nvalid) {
+                uint32_t lo = 0, hi = Lay::kTableWords - 1;           // largest word with (entries before it) <= first
+                while (lo < hi) {
+                    const uint32_t mid = (lo + hi + 1) >> 1;
+                    if (ktab[mid].y <= first) lo = mid; else hi = mid - 1;
+                }
+                const uint2 e = ktab[lo];
+                uint32_t word = lo, m = e.x;
+                for (uint32_t skip = first - e.y; skip; --skip) m &= m - 1;
+                // `ahead` is the next word's bits, fetched when the walk arrives at a word; eight columns are found
+                // first, then their values are read together and staged
+                uint32_t ahead = word + 1 < Lay::kTableWords ? ktab[word + 1].x : 0u;
+                for (uint32_t j0 = 0; j0 < nvalid; j0 += 8) {
+                    uint32_t col[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (m == 0) {
+                            m = ahead;
+                            ++word;
+                            while (m == 0) m = ktab[++word].x;     // an empty word (ends: kept bits lie ahead)
+                            ahead = word + 1 < Lay::kTableWords ? ktab[word + 1].x : 0u;
+                        }
+                        col[u] = word * 32u + (__ffs(m) - 1);
+                        if (j0 + u + 1 < nvalid) m &= m - 1;       // the last slot's bit stays: m != 0 or none is needed
+                    }
+                    uint32_t v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = row16[col[u]];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const uint32_t p = first + j0 + u;
+                        if (j0 + u < nvalid) stage[p + (p >> 5)] = v[u] | (col[u] << 16);
+                    }
                 }
             }
         }
         release_row();
         for (uint32_t p = lane; p < k; p += 32) {
-            const uint32_t e = stage[p];
+            const uint32_t e = stage[p + (p >> 5)];
             cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
             vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
             if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
