@@ -208,9 +208,22 @@ select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct
                 done = true;
             }
         }
-        if (!done)
-            for (uint32_t i = base + threadIdx.x; i < n && i < base + kSelChunk; i += kSelThreads)
-                consume(key_at(src, i));
+        if (!done) {
+            // scalar loads, eight per thread in flight before their histogram updates
+            const uint32_t lim = n - base < kSelChunk ? n : base + kSelChunk;
+            constexpr int kBatch = 8;
+            for (uint32_t i0 = base + threadIdx.x; i0 < lim; i0 += kSelThreads * kBatch) {
+                uint32_t key[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const uint32_t i = i0 + u * kSelThreads;
+                    key[u] = i < lim ? key_at(src, i) : 0u;
+                }
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u)
+                    if (i0 + u * kSelThreads < lim) consume(key[u]);
+            }
+        }
     }
     __syncthreads();
 
