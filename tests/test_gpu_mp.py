@@ -239,6 +239,27 @@ def test_mp_dense_k(dtype, d):
         _compare_fwd_bwd(x, gx, d, k)
 
 
+@pytest.mark.parametrize("d", [1024, 4096])
+def test_mp_dense_k_clustered_columns_and_many_ties(d):
+    """The dense bf16 kernel deals the k output slots out evenly and walks a bit table of the kept columns: rows whose
+    kept columns sit in one part of the row (long runs of empty table words before, between and after them), rows
+    of a few distinct values (every row has many ties at tau_i, spread over the lanes, of which only some are
+    kept), and k that is not a multiple of 32."""
+    rows = 900
+    x = inputs.mp_activations(rows, d, 71 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=72 + d)
+    third = d // 3
+    x[0::6, third:] = 0.0                            # only the first third is alive
+    x[1::6, :d - third] = 0.0                        # only the last third
+    x[2::6, third // 2:d - third // 2] = 0.0         # both ends, nothing in the middle
+    x[3::6] = inputs.quantize_mantissa(x[3::6], 2)   # a handful of distinct values per binade: ties everywhere
+    x[4::6] = torch.round(x[4::6] * 4.0) / 4.0       # multiples of 0.25, most of them 0
+    x = x.to(torch.bfloat16).contiguous()
+    gx = inputs.mp_gradients(rows, d, 73 + d, dtype=torch.bfloat16, device=G.DEV)
+    for k in sorted({d // 4 + 3, third - 5, third, third + 1, min(d // 2 - 1, 1279), min(d // 2, 1280)}):
+        cols = _compare_fwd_bwd(x, gx, d, k)
+        assert int(cols.max()) < d
+
+
 @pytest.mark.parametrize("d", [5000, 6144, 8000, 8192])
 def test_mp_bf16_wide_rows(d):
     """bf16 rows of more than 4096 and up to 8192 columns take the warp-per-row kernels too (buffers of 6144
