@@ -764,7 +764,7 @@ dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t d, 
 // A row for which this fails (tau_i = 0, bounds that do not converge) takes the bit-serial slow path.
 constexpr uint32_t kDenseWindow = 64;
 constexpr uint32_t kDenseMaxK = 1280;                 // staging slots per warp (5 KiB)
-constexpr int kDenseMaxWarps = 24;
+constexpr int kDenseMaxWarps = 32;
 constexpr int kDenseRetries = 6;
 
 template <int E8> struct DenseLayout {

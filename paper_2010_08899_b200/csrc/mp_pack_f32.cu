@@ -647,7 +647,7 @@ dct_status_t launch_width(const void* x_act, uint32_t rows, uint32_t d, uint32_t
 // (16-bit column, 32-bit value) to coalesced stores.
 constexpr uint32_t kDenseWindowF32 = 64;
 constexpr uint32_t kDenseMaxKF32 = 1280;
-constexpr int kDenseMaxWarpsF32 = 24;
+constexpr int kDenseMaxWarpsF32 = 32;
 constexpr int kDenseRetriesF32 = 6;
 
 template <int E8> struct DenseLayoutF32 {
