@@ -519,7 +519,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                     const uint32_t excl = incl - n_mine;
                     const uint32_t pc = __popc(masks[0]) | (__popc(masks[1 % kMaskWords]) << 8) | (__popc(masks[2 % kMaskWords]) << 16);
                     uint32_t owner = 0, owner_excl = 0;
-    #pragma unroll
+#pragma unroll
                     for (int step = 16; step > 0; step >>= 1) {
                         const uint32_t v = __shfl_sync(0xFFFFFFFFu, excl, owner + step);
                         if (v <= first) {
@@ -555,7 +555,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 // arrives at a word, long before it is needed
                 uint2 ahead = table[link];
                 const uint32_t table_addr = smem_addr(table);
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const bool advance = (m == 0);
                     m = advance ? ahead.x : m;
@@ -582,7 +582,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 hist[lane + 32] = 0;
                 hist[lane + 64] = 0;
                 __syncwarp();
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t rel = (ent[i] & 0x7FFFu) - low;
                     atomicAdd(&hist[min(rel, 64u + lane)], 1u);
@@ -614,7 +614,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
                 reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
                 __syncwarp();
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i)
                     if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent[i] & 0x7FFFu) >> 7], 1u);
                 __syncwarp();
@@ -622,7 +622,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 __syncwarp();
                 reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
                 __syncwarp();
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t key = ent[i] & 0x7FFFu;
                     if (static_cast<uint32_t>(i) < nvalid && (key >> 7) == exp_bin) atomicAdd(&hist[key & 0x7Fu], 1u);
@@ -639,7 +639,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             __syncwarp();                                         // the select histogram is dead: its words become the stage
             {
                 uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t key = ent[i] & 0x7FFFu;
                     counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
@@ -647,7 +647,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 const uint32_t before = warp_inclusive_sum(counts) - counts;
                 uint32_t e_at = before & 0xFFFFu;                 // ties before this entry
                 uint32_t pos = (before >> 16) + (e_at < take ? e_at : take);   // kept entries before it
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t key = ent[i] & 0x7FFFu;
                     const bool is_eq = key == tau_key;
@@ -662,7 +662,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 // the first 256 slots with constant offsets from one pointer each, any further ones in a loop
                 int16_t* cp = cols_out + out_base + lane;
                 uint16_t* vp = vals_out + out_base + lane;
-    #pragma unroll
+#pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     if (lane + 32u * j < k) {
                         const uint32_t e = stage[lane + 32 * j];

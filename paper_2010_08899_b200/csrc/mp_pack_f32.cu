@@ -373,7 +373,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                     const uint32_t excl = incl - n_mine;
                     const uint32_t pc = __popc(masks[0]) | (__popc(masks[1 % kMaskWords]) << 8) | (__popc(masks[2 % kMaskWords]) << 16);
                     uint32_t owner = 0, owner_excl = 0;
-    #pragma unroll
+#pragma unroll
                     for (int step = 16; step > 0; step >>= 1) {
                         const uint32_t v = __shfl_sync(0xFFFFFFFFu, excl, owner + step);
                         if (v <= first) {
@@ -407,7 +407,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 }
                 uint2 ahead = table[link];
                 const uint32_t table_addr = smem_addr(table);
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const bool advance = (m == 0);
                     m = advance ? ahead.x : m;
@@ -433,7 +433,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 hist[lane + 32] = 0;
                 hist[lane + 64] = 0;
                 __syncwarp();
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t rel = ((ent_val[i] >> 16) & 0x7FFFu) - low;
                     atomicAdd(&hist[rel < 64u ? rel : 64u + lane], 1u);
@@ -465,7 +465,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
                 reinterpret_cast<uint4*>(hist)[lane + 32] = make_uint4(0, 0, 0, 0);
                 __syncwarp();
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i)
                     if (static_cast<uint32_t>(i) < nvalid) atomicAdd(&hist[(ent_val[i] >> 23) & 0xFFu], 1u);
                 __syncwarp();
@@ -473,7 +473,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 __syncwarp();
                 reinterpret_cast<uint4*>(hist)[lane] = make_uint4(0, 0, 0, 0);
                 __syncwarp();
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t key15 = (ent_val[i] >> 16) & 0x7FFFu;
                     if (static_cast<uint32_t>(i) < nvalid && (key15 >> 7) == exp_bin) atomicAdd(&hist[key15 & 0x7Fu], 1u);
@@ -491,7 +491,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 uint32_t* members = scratch + 1;
                 if (lane == 0) *n_members = 0;
                 __syncwarp();
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
                     if ((key >> 16) == tau15) {
@@ -522,11 +522,11 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 } else {
                     // many members (ties, coarse data): the take15-th largest, bit by bit over the lower 16 bits
                     uint32_t prefix = tau15 << 16;
-    #pragma unroll 1
+#pragma unroll 1
                     for (int bit = 15; bit >= 0; --bit) {
                         const uint32_t trial = prefix | (1u << bit);
                         uint32_t cnt = 0;
-    #pragma unroll
+#pragma unroll
                         for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                             const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
                             cnt += ((key >> 16) == tau15 && key >= trial) ? 1u : 0u;
@@ -535,7 +535,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                     }
                     tau_key = prefix;
                     uint32_t above = 0;
-    #pragma unroll
+#pragma unroll
                     for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                         const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
                         above += ((key >> 16) == tau15 && key > tau_key) ? 1u : 0u;
@@ -549,7 +549,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
             __syncwarp();                                         // the member list is dead: its words become the stage
             {
                 uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
                     counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
@@ -557,7 +557,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 const uint32_t before = warp_inclusive_sum(counts) - counts;
                 uint32_t e_at = before & 0xFFFFu;                 // ties before this entry
                 uint32_t pos = (before >> 16) + (e_at < take ? e_at : take);   // kept entries before it
-    #pragma unroll
+#pragma unroll
                 for (int i = 0; i < static_cast<int>(kTrips); ++i) {
                     const uint32_t key = ent_val[i] & 0x7FFFFFFFu;
                     const bool is_eq = key == tau_key;
