@@ -70,6 +70,9 @@ constexpr size_t kCtrlBytes = 256;
 
 __global__ void dp_compress_init_kernel(CompressCtrl* ctrl, uint64_t* tile_state, uint32_t num_tiles,
                                         dct_result_t* result, uint32_t first_ticket) {
+    // the streaming kernel that follows may be scheduled already (it waits for this grid before it touches the
+    // control block): its launch latency and set-up then overlap this kernel
+    asm volatile("griddepcontrol.launch_dependents;");
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < num_tiles) tile_state[i] = 0;
     if (i == 0) {
@@ -497,6 +500,9 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
         fence_proxy_async_all();
     }
     __syncthreads();
+    // launched as a programmatic dependent of the kernel that resets the control block: everything above ran
+    // while that kernel was still at work, nothing below may (a no-op under an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == kLoadWarp) {
         // ================= load warp (one lane): tickets and bulk loads ====================
@@ -842,9 +848,18 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         single.first_desc = 0;
         single.num_full = num_full;
         single.num_tiles = num_tiles;
-        dp_compress_stream_kernel<false><<<grid, kStreamThreads, sizeof(StreamSmem), stream>>>(
-            single, BatchTable{}, num_full, ctrl, tile_state, dbg.spin_limit);
-        DCT_CUDA_TRY(cudaGetLastError());
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(kStreamThreads);
+        cfg.dynamicSmemBytes = sizeof(StreamSmem);
+        cfg.stream = stream;
+        cudaLaunchAttribute overlap = {};
+        overlap.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        overlap.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &overlap;
+        cfg.numAttrs = 1;
+        DCT_CUDA_TRY(cudaLaunchKernelEx(&cfg, dp_compress_stream_kernel<false>, single, BatchTable{}, num_full, ctrl,
+                                        tile_state, dbg.spin_limit));
     }
     if (num_tiles > num_full) {   // ragged last tile
         dp_compress_tile_kernel<true><<<1, kThreads, 0, stream>>>(
