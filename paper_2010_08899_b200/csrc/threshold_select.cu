@@ -75,8 +75,32 @@ __device__ __forceinline__ void reset_state(SelectState* st, uint32_t k, uint32_
     }
 }
 
+// The kernels of one select call form a chain in which each reads what the one before wrote.  From the second on
+// they are launched as programmatic dependents: a kernel lets the next one be scheduled at once (its launch
+// latency and set-up overlap this kernel) and waits for the one before it to finish, memory included, before it
+// touches the workspace.  Under an ordinary launch both calls do nothing.
+__device__ __forceinline__ void chain_release_next() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void chain_wait_previous() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// (host side) launches `kernel` as a programmatic dependent of the kernel launched before it on the stream
+template <typename... Params, typename... Args>
+cudaError_t launch_chained(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute overlap = {};
+    overlap.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    overlap.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &overlap;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 __global__ void select_init_kernel(SelectWorkspace* ws, uint32_t n, uint32_t k, uint32_t sample_n, uint32_t sample_k,
                                    uint32_t cand_capacity, dct_result_t* result) {
+    chain_release_next();
     const uint32_t i = threadIdx.x;
     const bool sampled = sample_n != 0;
     reset_state(&ws->full, k, n, sampled ? 0u : 1u, i, kInitThreads);
@@ -167,7 +191,6 @@ __device__ __forceinline__ void finish_pass(SelectState* st, uint32_t prefix, ui
 template <int kPass, typename Source, bool kVectorised>
 __global__ void __launch_bounds__(kSelThreads)
 select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct_result_t* __restrict__ result) {
-    if (!st->enabled) return;
     constexpr int shift = pass_shift(kPass);
     constexpr int bits = pass_bits(kPass);
     constexpr uint32_t digit_mask = (1u << bits) - 1u;
@@ -176,6 +199,8 @@ select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct
     __shared__ uint32_t s_last;
 
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) sh[b] = 0;
+    chain_wait_previous();
+    if (!st->enabled) return;
     const uint32_t prefix = kPass == 0 ? 0u : st->prefix;   // written by the previous launch
     const uint32_t n = st->n;
     __syncthreads();
@@ -225,6 +250,9 @@ select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct
             }
         }
     }
+    // this CTA's share of the pass is read: once every CTA is here the next kernel of the chain may be scheduled
+    // (not earlier: the kernels after it would follow one by one and sit on the SMs while this one still works)
+    chain_release_next();
     __syncthreads();
 
     uint32_t* hist = st->hist + kPass * kBins;
@@ -245,6 +273,7 @@ select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct
 template <bool kVectorised>
 __global__ void __launch_bounds__(kSelThreads)
 select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t* __restrict__ cand_keys) {
+    chain_wait_previous();
     if (!ws->sample.enabled) return;
     const uint32_t lo = ws->sample.key_out;
     const uint32_t capacity = ws->cand_capacity;
@@ -307,11 +336,14 @@ select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t
             }
         }
     }
+    chain_release_next();
     if (held) flush();
 }
 
 // After the filter: decide which select produces the answer.
 __global__ void select_decide_kernel(SelectWorkspace* ws, uint32_t k) {
+    chain_release_next();
+    chain_wait_previous();
     if (!ws->sample.enabled) return;
     const uint32_t c = ws->cand_count;
     if (c >= k && c <= ws->cand_capacity) {
@@ -325,10 +357,12 @@ __global__ void select_decide_kernel(SelectWorkspace* ws, uint32_t k) {
 template <typename Source, bool kVectorised>
 cudaError_t launch_three_passes(int grid, cudaStream_t stream, Source src, SelectState* st, float* tau_out,
                                 dct_result_t* result) {
-    select_pass_kernel<0, Source, kVectorised><<<grid, kSelThreads, 0, stream>>>(src, st, tau_out, result);
-    select_pass_kernel<1, Source, kVectorised><<<grid, kSelThreads, 0, stream>>>(src, st, tau_out, result);
-    select_pass_kernel<2, Source, kVectorised><<<grid, kSelThreads, 0, stream>>>(src, st, tau_out, result);
-    return cudaGetLastError();
+    cudaError_t e = launch_chained(select_pass_kernel<0, Source, kVectorised>, grid, kSelThreads, stream, src, st, tau_out, result);
+    if (e == cudaSuccess)
+        e = launch_chained(select_pass_kernel<1, Source, kVectorised>, grid, kSelThreads, stream, src, st, tau_out, result);
+    if (e == cudaSuccess)
+        e = launch_chained(select_pass_kernel<2, Source, kVectorised>, grid, kSelThreads, stream, src, st, tau_out, result);
+    return e;
 }
 
 // Rank to select in the sample so that the number of vector elements at or above the sampled value is,
@@ -397,12 +431,10 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
         DCT_CUDA_TRY((launch_three_passes<StridedSource, false>(grid_for(sample_n), stream, ssrc, &ws->sample, nullptr,
                                                                 result)));
         if (vec)
-            select_filter_kernel<true><<<grid_for(n), kSelThreads, 0, stream>>>(vsrc, n32, ws, cand_keys);
+            DCT_CUDA_TRY(launch_chained(select_filter_kernel<true>, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
         else
-            select_filter_kernel<false><<<grid_for(n), kSelThreads, 0, stream>>>(vsrc, n32, ws, cand_keys);
-        DCT_CUDA_TRY(cudaGetLastError());
-        select_decide_kernel<<<1, 1, 0, stream>>>(ws, k32);
-        DCT_CUDA_TRY(cudaGetLastError());
+            DCT_CUDA_TRY(launch_chained(select_filter_kernel<false>, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
+        DCT_CUDA_TRY(launch_chained(select_decide_kernel, 1, 1, stream, ws, k32));
         const KeySource ksrc{cand_keys};
         // the candidate count is only known on the device: a fixed modest grid walks whatever is there
         DCT_CUDA_TRY((launch_three_passes<KeySource, false>(128, stream, ksrc, &ws->cand, tau_out, result)));
