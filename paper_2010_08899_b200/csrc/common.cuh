@@ -148,4 +148,27 @@ DebugConfig& debug_config();
 
 int sm_count();              // multiprocessors of the current device (cached per device)
 
+// The kernels of one call often form a chain in which each reads what the one before wrote.  From the second on
+// they are launched as programmatic dependents: a kernel lets the next one be scheduled at once (its launch
+// latency and set-up overlap this kernel) and waits for the one before it to finish, memory included, before it
+// touches the workspace.  Under an ordinary launch both calls do nothing.
+__device__ __forceinline__ void chain_release_next() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void chain_wait_previous() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// (host side) launches `kernel` as a programmatic dependent of the kernel launched before it on the stream
+template <typename... Params, typename... Args>
+cudaError_t launch_chained(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t stream, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute overlap = {};
+    overlap.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    overlap.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &overlap;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 }  // namespace dct

@@ -75,29 +75,6 @@ __device__ __forceinline__ void reset_state(SelectState* st, uint32_t k, uint32_
     }
 }
 
-// The kernels of one select call form a chain in which each reads what the one before wrote.  From the second on
-// they are launched as programmatic dependents: a kernel lets the next one be scheduled at once (its launch
-// latency and set-up overlap this kernel) and waits for the one before it to finish, memory included, before it
-// touches the workspace.  Under an ordinary launch both calls do nothing.
-__device__ __forceinline__ void chain_release_next() { asm volatile("griddepcontrol.launch_dependents;"); }
-__device__ __forceinline__ void chain_wait_previous() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-// (host side) launches `kernel` as a programmatic dependent of the kernel launched before it on the stream
-template <typename... Params, typename... Args>
-cudaError_t launch_chained(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t stream, Args... args) {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = stream;
-    cudaLaunchAttribute overlap = {};
-    overlap.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    overlap.val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = &overlap;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
-}
-
 __global__ void select_init_kernel(SelectWorkspace* ws, uint32_t n, uint32_t k, uint32_t sample_n, uint32_t sample_k,
                                    uint32_t cand_capacity, dct_result_t* result) {
     chain_release_next();

@@ -47,6 +47,7 @@ __device__ __forceinline__ uint32_t layer_of_chunk(const LayerState* layers, uin
 }
 
 __global__ void batched_init_kernel(LayerState* layers, uint32_t num_layers) {
+    chain_release_next();
     // the description part has been copied in; clear the select state, the histograms and the result
     for (uint32_t l = blockIdx.x; l < num_layers; l += gridDim.x) {
         LayerState* st = layers + l;
@@ -82,6 +83,7 @@ batched_pass_kernel(LayerState* layers, uint32_t num_layers, uint64_t total_chun
     if (c_begin >= c_end) return;
 
     for (int b = threadIdx.x; b < kBins; b += kThreads) sh[b] = 0;
+    chain_wait_previous();
     uint32_t layer = layer_of_chunk(layers, num_layers, c_begin);
     __syncthreads();
 
@@ -135,6 +137,7 @@ batched_pass_kernel(LayerState* layers, uint32_t num_layers, uint64_t total_chun
                 consume(key_f32(residual ? __fadd_rn(grad[i], residual[i]) : grad[i]));
         }
     }
+    chain_release_next();
     flush(layer);
 }
 
@@ -144,6 +147,8 @@ __global__ void __launch_bounds__(kThreads)
 batched_scan_kernel(LayerState* layers, uint32_t num_layers) {
     constexpr int bits = pass_bits(kPass);
     __shared__ uint32_t s_scan[kThreads / 32];
+    chain_release_next();
+    chain_wait_previous();
     for (uint32_t l = blockIdx.x; l < num_layers; l += gridDim.x) {
         LayerState* st = layers + l;
         const uint32_t* hist = st->hist[kPass];
@@ -247,12 +252,12 @@ extern "C" dct_status_t dct_threshold_select_batched(const dct_select_layer_t* l
     const uint64_t want = static_cast<uint64_t>(sms) * 4;
     const uint32_t grid = static_cast<uint32_t>(total_chunks < want ? total_chunks : want);
     const uint32_t scan_grid = num_layers < static_cast<uint32_t>(sms) * 4u ? num_layers : static_cast<uint32_t>(sms) * 4u;
-    batched_pass_kernel<0><<<grid, kThreads, 0, stream>>>(dev_layers, num_layers, total_chunks);
-    batched_scan_kernel<0><<<scan_grid, kThreads, 0, stream>>>(dev_layers, num_layers);
-    batched_pass_kernel<1><<<grid, kThreads, 0, stream>>>(dev_layers, num_layers, total_chunks);
-    batched_scan_kernel<1><<<scan_grid, kThreads, 0, stream>>>(dev_layers, num_layers);
-    batched_pass_kernel<2><<<grid, kThreads, 0, stream>>>(dev_layers, num_layers, total_chunks);
-    batched_scan_kernel<2><<<scan_grid, kThreads, 0, stream>>>(dev_layers, num_layers);
-    DCT_CUDA_TRY(cudaGetLastError());
+    // each kernel from here on is a programmatic dependent of the one before it (common.cuh)
+    DCT_CUDA_TRY(launch_chained(batched_pass_kernel<0>, grid, kThreads, stream, dev_layers, num_layers, total_chunks));
+    DCT_CUDA_TRY(launch_chained(batched_scan_kernel<0>, scan_grid, kThreads, stream, dev_layers, num_layers));
+    DCT_CUDA_TRY(launch_chained(batched_pass_kernel<1>, grid, kThreads, stream, dev_layers, num_layers, total_chunks));
+    DCT_CUDA_TRY(launch_chained(batched_scan_kernel<1>, scan_grid, kThreads, stream, dev_layers, num_layers));
+    DCT_CUDA_TRY(launch_chained(batched_pass_kernel<2>, grid, kThreads, stream, dev_layers, num_layers, total_chunks));
+    DCT_CUDA_TRY(launch_chained(batched_scan_kernel<2>, scan_grid, kThreads, stream, dev_layers, num_layers));
     return DCT_OK;
 }
