@@ -157,11 +157,12 @@ __device__ __forceinline__ void chain_wait_previous() { asm volatile("griddepcon
 
 // (host side) launches `kernel` as a programmatic dependent of the kernel launched before it on the stream
 template <typename... Params, typename... Args>
-cudaError_t launch_chained(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t stream, Args... args) {
+cudaError_t launch_chained_smem(void (*kernel)(Params...), unsigned grid, unsigned block, size_t dynamic_smem,
+                                cudaStream_t stream, Args... args) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(block);
-    cfg.dynamicSmemBytes = 0;
+    cfg.dynamicSmemBytes = dynamic_smem;
     cfg.stream = stream;
     cudaLaunchAttribute overlap = {};
     overlap.id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -169,6 +170,10 @@ cudaError_t launch_chained(void (*kernel)(Params...), unsigned grid, unsigned bl
     cfg.attrs = &overlap;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+template <typename... Params, typename... Args>
+cudaError_t launch_chained(void (*kernel)(Params...), unsigned grid, unsigned block, cudaStream_t stream, Args... args) {
+    return launch_chained_smem(kernel, grid, block, 0, stream, args...);
 }
 
 }  // namespace dct

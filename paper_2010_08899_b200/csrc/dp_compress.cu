@@ -72,7 +72,7 @@ __global__ void dp_compress_init_kernel(CompressCtrl* ctrl, uint64_t* tile_state
                                         dct_result_t* result, uint32_t first_ticket) {
     // the streaming kernel that follows may be scheduled already (it waits for this grid before it touches the
     // control block): its launch latency and set-up then overlap this kernel
-    asm volatile("griddepcontrol.launch_dependents;");
+    chain_release_next();
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < num_tiles) tile_state[i] = 0;
     if (i == 0) {
@@ -502,7 +502,7 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
     __syncthreads();
     // launched as a programmatic dependent of the kernel that resets the control block: everything above ran
     // while that kernel was still at work, nothing below may (a no-op under an ordinary launch)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    chain_wait_previous();
 
     if (warp == kLoadWarp) {
         // ================= load warp (one lane): tickets and bulk loads ====================
@@ -726,6 +726,7 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
 // ---- batched calls: many vectors (the layers of a model), one set of launches ------------------------
 __global__ void dp_compress_batched_init_kernel(CompressCtrl* ctrl, uint64_t* tile_state, uint32_t total_tiles,
                                                 const LayerDesc* layers, uint32_t num_layers) {
+    chain_release_next();     // the streaming kernel may be scheduled; it waits for this grid (see dp_compress_init_kernel)
     const uint32_t stride = gridDim.x * blockDim.x;
     const uint32_t i0 = blockIdx.x * blockDim.x + threadIdx.x;
     for (uint32_t i = i0; i < total_tiles; i += stride) tile_state[i] = 0;
@@ -848,18 +849,8 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         single.first_desc = 0;
         single.num_full = num_full;
         single.num_tiles = num_tiles;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(grid);
-        cfg.blockDim = dim3(kStreamThreads);
-        cfg.dynamicSmemBytes = sizeof(StreamSmem);
-        cfg.stream = stream;
-        cudaLaunchAttribute overlap = {};
-        overlap.id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        overlap.val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = &overlap;
-        cfg.numAttrs = 1;
-        DCT_CUDA_TRY(cudaLaunchKernelEx(&cfg, dp_compress_stream_kernel<false>, single, BatchTable{}, num_full, ctrl,
-                                        tile_state, dbg.spin_limit));
+        DCT_CUDA_TRY(launch_chained_smem(dp_compress_stream_kernel<false>, grid, kStreamThreads, sizeof(StreamSmem), stream,
+                                         single, BatchTable{}, num_full, ctrl, tile_state, dbg.spin_limit));
     }
     if (num_tiles > num_full) {   // ragged last tile
         dp_compress_tile_kernel<true><<<1, kThreads, 0, stream>>>(
@@ -997,9 +988,8 @@ extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, ui
         const uint32_t ctas_per_sm = sizeof(StreamSmem) <= 110 * 1024 ? 2 : 1;
         const uint32_t max_grid = static_cast<uint32_t>(sms) * ctas_per_sm;
         const uint32_t grid = total_full < max_grid ? total_full : max_grid;
-        dp_compress_stream_kernel<true><<<grid, kStreamThreads, sizeof(StreamSmem), stream>>>(
-            LayerDesc{}, batch, total_full, ctrl, tile_state, dbg.spin_limit);
-        DCT_CUDA_TRY(cudaGetLastError());
+        DCT_CUDA_TRY(launch_chained_smem(dp_compress_stream_kernel<true>, grid, kStreamThreads, sizeof(StreamSmem), stream,
+                                         LayerDesc{}, batch, total_full, ctrl, tile_state, dbg.spin_limit));
     }
     if (total_slow > 0) {
         dp_compress_tile_batched_kernel<<<total_slow, kThreads, 0, stream>>>(batch, total_slow, ctrl, tile_state,
