@@ -848,6 +848,10 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
     // row finds more than 96 elements in it, and doubled again when a row needs a second pass: a second pass over
     // the row is cheaper than a crowded window (9 % faster at k = 1024, 11 % at k = 600).
     uint32_t window = kDenseWindow;
+    // k a multiple of 256 (every lane has a multiple of 8 output slots) and 16-byte aligned outputs: the emit writes
+    // 128-bit words straight to global memory
+    const bool direct = (k & 255u) == 0 && ((reinterpret_cast<uintptr_t>(cols_out) | reinterpret_cast<uintptr_t>(vals_out)) & 15u) == 0 &&
+                        (rows_out == nullptr || (reinterpret_cast<uintptr_t>(rows_out) & 15u) == 0);
     for (uint64_t row64 = warp_global; row64 < rows; row64 = next_row, ++use) {
         const uint32_t row = static_cast<uint32_t>(row64);
         if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
@@ -1082,20 +1086,36 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
                     uint32_t v[8];
 #pragma unroll
                     for (int u = 0; u < 8; ++u) v[u] = row16[col[u]];
+                    if (direct) {
+                        // eight consecutive slots of this lane are 16 aligned bytes of either output: no staging
+                        const size_t at = out_base + first + j0;
+                        *reinterpret_cast<uint4*>(cols_out + at) = make_uint4(col[0] | (col[1] << 16), col[2] | (col[3] << 16),
+                                                                              col[4] | (col[5] << 16), col[6] | (col[7] << 16));
+                        *reinterpret_cast<uint4*>(vals_out + at) = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16),
+                                                                              v[4] | (v[5] << 16), v[6] | (v[7] << 16));
+                        if (rows_out) {
+                            const uint4 r4 = make_uint4(row, row, row, row);
+                            reinterpret_cast<uint4*>(rows_out + at)[0] = r4;
+                            reinterpret_cast<uint4*>(rows_out + at)[1] = r4;
+                        }
+                    } else {
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const uint32_t p = first + j0 + u;
-                        if (j0 + u < nvalid) stage[p + (p >> 5)] = v[u] | (col[u] << 16);
+                        for (int u = 0; u < 8; ++u) {
+                            const uint32_t p = first + j0 + u;
+                            if (j0 + u < nvalid) stage[p + (p >> 5)] = v[u] | (col[u] << 16);
+                        }
                     }
                 }
             }
         }
         release_row();
-        for (uint32_t p = lane; p < k; p += 32) {
-            const uint32_t e = stage[p + (p >> 5)];
-            cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
-            vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
-            if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
+        if (!direct) {
+            for (uint32_t p = lane; p < k; p += 32) {
+                const uint32_t e = stage[p + (p >> 5)];
+                cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
+                vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
+                if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
+            }
         }
         __syncwarp();
     }

@@ -260,6 +260,31 @@ def test_mp_dense_k_clustered_columns_and_many_ties(d):
         assert int(cols.max()) < d
 
 
+@pytest.mark.parametrize("d,k", [(1024, 256), (2048, 512), (4096, 1024), (4096, 1280)])
+def test_mp_dense_k_multiple_of_256_writes_whole_words(d, k):
+    """With k a multiple of 256 and 16-byte aligned outputs the dense bf16 kernel writes 128-bit words straight
+    from the emit (cols, vals and the optional row ids); with an output that starts 2 bytes off it must fall back to
+    the staged stores.  Both give the oracle's result, and neither writes outside its rows * k slots."""
+    rows = 333
+    x = inputs.mp_activations(rows, d, 81 + d, dtype=torch.bfloat16, device=G.DEV, col_scale_seed=82 + d)
+    x[5] = 0.5                                       # every element ties: the first k columns win
+    want = oracle.mp_fwd(G.to_oracle(x), k, d=d)
+    cols, vals, tau, rws = G.mp_fwd(x, d, k, want_rows=True)
+    assert np.array_equal(cols.cpu().numpy(), want.cols)
+    assert np.array_equal(G.as_np_bits(vals), want.vals.view(np.uint16))
+    assert np.array_equal(rws.cpu().numpy(), np.repeat(np.arange(rows, dtype=np.int32)[:, None], k, 1))
+    # outputs one element (2 bytes) off a 16-byte boundary
+    cols_buf = torch.full((rows * k + 9,), -1, dtype=torch.int16, device=G.DEV)
+    vals_buf = torch.full((rows * k + 9,), 99.0, dtype=torch.bfloat16, device=G.DEV)
+    res = B.new_result()
+    B.dct_mp_topk_pack_fwd(x, rows, d, d, k, cols_buf[1:], vals_buf[1:], None, None, res)
+    assert B.read_result(res).status == B.DCT_OK
+    assert np.array_equal(cols_buf[1:1 + rows * k].view(rows, k).cpu().numpy(), want.cols)
+    assert np.array_equal(G.as_np_bits(vals_buf[1:1 + rows * k].view(rows, k)), want.vals.view(np.uint16))
+    assert int(cols_buf[0]) == -1 and bool((cols_buf[1 + rows * k:] == -1).all())
+    assert float(vals_buf[0]) == 99.0 and bool((vals_buf[1 + rows * k:] == 99.0).all())
+
+
 @pytest.mark.parametrize("d", [5000, 6144, 8000, 8192])
 def test_mp_bf16_wide_rows(d):
     """bf16 rows of more than 4096 and up to 8192 columns take the warp-per-row kernels too (buffers of 6144
