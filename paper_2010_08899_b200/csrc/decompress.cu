@@ -180,6 +180,10 @@ extern "C" dct_status_t dct_dp_decompress(const int32_t* idx, const float* val, 
     uint64_t grid = static_cast<uint64_t>(sms) * 8;
     const uint64_t by_size = (n + 1023) / 1024;
     if (grid > by_size) grid = by_size;
+    // ... and at most 16384 elements (64 KB) each: the CTAs at work then write neighbouring ranges instead of 1184
+    // streams spread over the whole vector (2^30 elements: 0.749 -> 0.620 ms; ranges of 8192 or 32768 are slower)
+    const uint64_t by_range = (n + 16383) / 16384;
+    if (grid < by_range) grid = by_range;
     dp_decompress_kernel<<<static_cast<unsigned>(grid), 256, 0, stream>>>(idx, val, packed, capacity, dense,
                                                                          static_cast<uint32_t>(n), accumulate, result);
     DCT_CUDA_TRY(cudaGetLastError());
