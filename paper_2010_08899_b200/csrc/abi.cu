@@ -1,5 +1,6 @@
 // Host-side pieces of the C ABI that are not tied to one kernel: status names,
 // error text, device queries, the testing knobs and the host-buffer wrappers.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
@@ -35,6 +36,12 @@ int sm_count() {
         cached[dev] = v;
     }
     return cached[dev];
+}
+
+uint32_t next_launch_ticket() {
+    static std::atomic<uint32_t> counter{0x5EED0000u};
+    uint32_t t = counter.fetch_add(1u, std::memory_order_relaxed) + 1u;
+    return t != 0u ? t : counter.fetch_add(1u, std::memory_order_relaxed) + 1u;
 }
 
 }  // namespace dct

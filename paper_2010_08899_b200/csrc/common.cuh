@@ -147,6 +147,7 @@ struct DebugConfig {
 DebugConfig& debug_config();
 
 int sm_count();              // multiprocessors of the current device (cached per device)
+uint32_t next_launch_ticket();   // a process-wide, never-zero, ever-changing number that marks one launch
 
 // The kernels of one call often form a chain in which each reads what the one before wrote.  From the second on
 // they are launched as programmatic dependents: a kernel lets the next one be scheduled at once (its launch

@@ -113,13 +113,25 @@ __global__ void mp_topk_pack_fwd_kernel(const T* __restrict__ x, uint32_t rows, 
     }
 }
 
+// The result block is reset inside the kernel (no memset node, no reset kernel on the stream).  Thread 0 of CTA 0
+// clears it and then publishes the launch's ticket in `reserved` (release); a warp that has met a bad column
+// waits (bounded) for that ticket before it raises the status, so the reset can never wipe a report.
 template <typename T>
 __global__ void __launch_bounds__(256)
 mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
-                   const int16_t* __restrict__ cols, T* __restrict__ gvals, dct_result_t* __restrict__ result) {
+                   const int16_t* __restrict__ cols, T* __restrict__ gvals, dct_result_t* __restrict__ result,
+                   uint32_t ticket) {
     const uint32_t lane = lane_id();
     const uint32_t warps_per_cta = blockDim.x >> 5;
     bool bad = false;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&result->reserved), "r"(ticket) : "memory");
+    }
     for (uint64_t row = static_cast<uint64_t>(blockIdx.x) * warps_per_cta + (threadIdx.x >> 5); row < rows;
          row += static_cast<uint64_t>(gridDim.x) * warps_per_cta) {
         const T* gr = gx + row * ld;
@@ -147,7 +159,14 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
             }
         }
     }
-    if (bad && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
+    if (bad && result) {
+        for (uint32_t spin = 0; spin < (1u << 20); ++spin) {          // CTA 0 is dispatched first: normally no wait at all
+            uint32_t seen;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&result->reserved) : "memory");
+            if (seen == ticket) break;
+        }
+        atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -190,66 +209,6 @@ template <int E8> struct WarpRowLayout {
     }
 };
 
-// General slow path for one row (rare): no usable bound, or very many elements tie at it.  tau_i is found
-// bit by bit on the row itself, most significant first (the largest v with #{key >= v} >= k); then
-// everything above tau_i and the first ties are written, in column order, straight from the row.
-// Kept out of line so that the common path stays small in the instruction cache.
-template <int E8>
-__device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_t k, size_t out_base, uint32_t row,
-                                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
-                                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out) {
-    constexpr uint32_t E = E8 * 8u;
-    constexpr int kMaskWords = (E8 + 3) / 4;
-    const uint32_t lane = lane_id();
-    uint32_t tau_key = 0;
-#pragma unroll 1
-    for (int bit = 14; bit >= 0; --bit) {
-        const uint32_t trial = tau_key | (1u << bit);
-        uint32_t cnt = 0;
-#pragma unroll 4
-        for (int c = 0; c < E8; ++c)
-            cnt += __popc(mask8_ge_exact(*reinterpret_cast<const uint4*>(span + c * 16), trial));
-        if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= k) tau_key = trial;
-    }
-    uint32_t gt_masks[kMaskWords], eq_masks[kMaskWords];
-    uint32_t n_gt_mine = 0, n_eq_mine = 0;
-#pragma unroll
-    for (int i = 0; i < kMaskWords; ++i) gt_masks[i] = eq_masks[i] = 0;
-#pragma unroll
-    for (int c = 0; c < E8; ++c) {
-        const uint4 v = *reinterpret_cast<const uint4*>(span + c * 16);
-        const uint32_t gt = mask8_ge_exact(v, tau_key + 1u);
-        const uint32_t eq = mask8_ge_exact(v, tau_key) & ~gt;
-        gt_masks[c / 4] |= gt << (8 * (c % 4));
-        eq_masks[c / 4] |= eq << (8 * (c % 4));
-        n_gt_mine += __popc(gt);
-        n_eq_mine += __popc(eq);
-    }
-    const uint32_t incl = warp_inclusive_sum(n_gt_mine);
-    const uint32_t take = k - __shfl_sync(0xFFFFFFFFu, incl, 31);   // ties to keep, lowest columns first
-    uint32_t g_at = incl - n_gt_mine;
-    uint32_t e_at = warp_inclusive_sum(n_eq_mine) - n_eq_mine;
-#pragma unroll
-    for (int wd = 0; wd < kMaskWords; ++wd) {
-        uint32_t m = gt_masks[wd] | eq_masks[wd];
-        while (m) {
-            const uint32_t bit = __ffs(m) - 1;
-            m &= m - 1;
-            const bool is_eq = (eq_masks[wd] >> bit) & 1u;
-            if (!is_eq || e_at < take) {
-                const uint32_t j = wd * 32 + bit;
-                const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
-                cols_out[pos] = static_cast<int16_t>(lane * E + j);
-                vals_out[pos] = *reinterpret_cast<const uint16_t*>(span + j * 2);
-                if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
-            }
-            g_at += is_eq ? 0u : 1u;
-            e_at += is_eq ? 1u : 0u;
-        }
-    }
-    if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
-}
-
 // Warps of a CTA: as many row buffers as shared memory holds (wide rows leave fewer warps and therefore more
 // registers for each of them), at most 32 with up to 10 candidates per lane (the kernel then fits 64 registers;
 // 32 warps against 24 are worth 7 to 11 % on rows of 2048 and 1024 columns) and 24 with 20 per lane.
@@ -283,18 +242,12 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Lay::scratch_words(k));
     __shared__ uint32_t s_stop;
     __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
+    __shared__ uint32_t s_hint;                               // the latest bound any warp of this CTA guessed from a tau_i
 
-    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
-        result->status = DCT_OK;
-        result->reserved = 0;
-        result->count = 0;
-        result->needed = 0;
-        result->n_gt = 0;
-        result->n_eq = 0;
-    }
     if (threadIdx.x == 0) {
         s_stop = 0;
         s_next = blockDim.x >> 5;
+        s_hint = 0;
     }
     if (lane == 0) {
         mbar_init(bar, 1);
@@ -307,6 +260,17 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
         *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
+    // Everything above is set-up in shared memory; the kernel before this one on the stream (which may have
+    // produced x or may still read the outputs) must have finished before anything below.
+    chain_wait_previous();
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
 
     // Rows are dealt out CTA by CTA (row mod grid = CTA): every SM gets the same number of rows to within one.
     // Inside the CTA a warp takes the CTA's next row whenever it lets go of one (a counter in shared memory): the
@@ -440,6 +404,8 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         // It is only a guess -- it is accepted if it leaves at least k and not too many candidates, and the
         // exact leaf bound takes over otherwise -- so the result never depends on it.
         uint32_t low = 0;
+        // a warp that has no row behind it borrows the latest guess of its CTA
+        if (guess_low == 0) guess_low = *reinterpret_cast<volatile uint32_t*>(&s_hint);
         bool use_guess = have_bound && guess_low != 0;
 #pragma unroll 1
         while (true) {
@@ -632,6 +598,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             }
             if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
             guess_low = tau_key > kGuessMargin ? tau_key - kGuessMargin : 0u;
+            if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&s_hint) = guess_low;
 
             // ---- D: ordered emit ------------------------------------------------------------------------
             // The kept entries are placed, in column order, into k staging slots; then they leave with
@@ -691,6 +658,9 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             finish_row(std::integral_constant<uint32_t, PL>{});
         }
     }
+    // This warp has no row left: the next kernel on the stream may be scheduled as the CTAs of this one retire
+    // (its set-up then overlaps the tail of this kernel; it still waits for this kernel's end before it works).
+    chain_release_next();
 }
 
 template <int E8, int PL>
@@ -719,10 +689,9 @@ dct_status_t launch_fwd_bf16_warp_variant(const void* x_act, uint32_t rows, uint
     warps = warps_for_rows(warps, rows, sms);
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
-    kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
-        static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out, static_cast<uint16_t*>(vals_out), rows_out,
-        static_cast<uint16_t*>(tau_out), result);
-    DCT_CUDA_TRY(cudaGetLastError());
+    DCT_CUDA_TRY(launch_chained_smem(kernel, grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream,
+                                     static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out,
+                                     static_cast<uint16_t*>(vals_out), rows_out, static_cast<uint16_t*>(tau_out), result));
     return DCT_OK;
 }
 
@@ -798,14 +767,6 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
     __shared__ uint32_t s_stop;
     __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
 
-    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
-        result->status = DCT_OK;
-        result->reserved = 0;
-        result->count = 0;
-        result->needed = 0;
-        result->n_gt = 0;
-        result->n_eq = 0;
-    }
     if (threadIdx.x == 0) {
         s_stop = 0;
         s_next = blockDim.x >> 5;
@@ -819,6 +780,15 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
     for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
         *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
+    chain_wait_previous();                                     // set-up above, inputs and outputs only below (see the sparse kernel)
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
 
     const uint32_t warp_global = blockIdx.x + gridDim.x * warp;
     auto request_row = [&](uint32_t r) {
@@ -1119,6 +1089,7 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
         }
         __syncwarp();
     }
+    chain_release_next();                                      // no row left for this warp (see the sparse kernel)
 }
 
 template <int E8>
@@ -1145,10 +1116,9 @@ dct_status_t launch_fwd_bf16_dense(const void* x_act, uint32_t rows, uint32_t d,
     warps = warps_for_rows(warps, rows, sms);
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
-    kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
-        static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out, static_cast<uint16_t*>(vals_out), rows_out,
-        static_cast<uint16_t*>(tau_out), result);
-    DCT_CUDA_TRY(cudaGetLastError());
+    DCT_CUDA_TRY(launch_chained_smem(kernel, grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream,
+                                     static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out,
+                                     static_cast<uint16_t*>(vals_out), rows_out, static_cast<uint16_t*>(tau_out), result));
     return DCT_OK;
 }
 
@@ -1186,7 +1156,6 @@ dct_status_t launch_fwd(const void* x_act, uint32_t rows, uint32_t d, uint32_t l
 template <typename T>
 dct_status_t launch_bwd(const void* x_grad, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, const int16_t* cols,
                         void* gvals_out, dct_result_t* result, cudaStream_t stream) {
-    if (result) DCT_CUDA_TRY(cudaMemsetAsync(result, 0, sizeof(dct_result_t), stream));
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + 7) / 8;
@@ -1195,7 +1164,7 @@ dct_status_t launch_bwd(const void* x_grad, uint32_t rows, uint32_t d, uint32_t 
     const uint64_t max_grid = static_cast<uint64_t>(sms) * 32;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < max_grid ? ctas_needed : max_grid);
     mp_pack_bwd_kernel<T><<<grid, 256, 0, stream>>>(static_cast<const T*>(x_grad), rows, d, ld, k, cols,
-                                                    static_cast<T*>(gvals_out), result);
+                                                    static_cast<T*>(gvals_out), result, next_launch_ticket());
     DCT_CUDA_TRY(cudaGetLastError());
     return DCT_OK;
 }

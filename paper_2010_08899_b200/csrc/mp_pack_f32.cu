@@ -137,18 +137,12 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
     uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Lay::scratch_words(k));
     __shared__ uint32_t s_stop;
     __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
+    __shared__ uint32_t s_hint;                               // the latest bound any warp of this CTA guessed from a tau_i
 
-    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
-        result->status = DCT_OK;
-        result->reserved = 0;
-        result->count = 0;
-        result->needed = 0;
-        result->n_gt = 0;
-        result->n_eq = 0;
-    }
     if (threadIdx.x == 0) {
         s_stop = 0;
         s_next = blockDim.x >> 5;
+        s_hint = 0;
     }
     if (lane == 0) {
         mbar_init(bar, 1);
@@ -161,6 +155,15 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
     for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
         *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
+    chain_wait_previous();          // set-up above; inputs and outputs only below (see the bf16 kernel in mp_pack.cu)
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
 
     // rows are dealt out CTA by CTA (row mod grid = CTA); inside the CTA a warp takes the CTA's next row whenever
     // it lets go of one (see the bf16 kernel in mp_pack.cu)
@@ -303,6 +306,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
         };
 
         uint32_t low = 0;
+        if (guess_low == 0) guess_low = *reinterpret_cast<volatile uint32_t*>(&s_hint);   // none of its own: the CTA's latest
         bool use_guess = have_bound && guess_low != 0;
 #pragma unroll 1
         while (true) {
@@ -483,6 +487,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
                 __syncwarp();
             }
             guess_low = tau15 > kGuessMargin ? tau15 - kGuessMargin : 0u;
+            if (lane == 0) *reinterpret_cast<volatile uint32_t*>(&s_hint) = guess_low;
 
             // ---- D': exact tau_i among the members of that bucket: the take15-th largest full key ------------
             uint32_t tau_key = 0, take = 0;
@@ -589,6 +594,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
             finish_row(std::integral_constant<uint32_t, PL>{});
         }
     }
+    chain_release_next();           // no row left for this warp: the next kernel may be scheduled as this one's CTAs retire
 }
 
 template <int E8, int PL>
@@ -616,10 +622,9 @@ dct_status_t launch_variant(const void* x_act, uint32_t rows, uint32_t d, uint32
     warps = warps_for_rows(warps, rows, sms);
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
-    kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
-        static_cast<const uint32_t*>(x_act), rows, d, ld, k, cols_out, static_cast<uint32_t*>(vals_out), rows_out,
-        static_cast<uint32_t*>(tau_out), result);
-    DCT_CUDA_TRY(cudaGetLastError());
+    DCT_CUDA_TRY(launch_chained_smem(kernel, grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream,
+                                     static_cast<const uint32_t*>(x_act), rows, d, ld, k, cols_out,
+                                     static_cast<uint32_t*>(vals_out), rows_out, static_cast<uint32_t*>(tau_out), result));
     return DCT_OK;
 }
 
@@ -695,14 +700,6 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
     __shared__ uint32_t s_stop;
     __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
 
-    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
-        result->status = DCT_OK;
-        result->reserved = 0;
-        result->count = 0;
-        result->needed = 0;
-        result->n_gt = 0;
-        result->n_eq = 0;
-    }
     if (threadIdx.x == 0) {
         s_stop = 0;
         s_next = blockDim.x >> 5;
@@ -716,6 +713,15 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
     for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
         *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
+    chain_wait_previous();          // set-up above; inputs and outputs only below (see the bf16 kernel in mp_pack.cu)
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
 
     const uint32_t warp_global = blockIdx.x + gridDim.x * warp;
     auto request_row = [&](uint32_t r) {
@@ -978,6 +984,7 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
         }
         __syncwarp();
     }
+    chain_release_next();           // no row left for this warp
 }
 
 template <int E8>
@@ -1003,10 +1010,9 @@ dct_status_t launch_dense(const void* x_act, uint32_t rows, uint32_t d, uint32_t
     warps = warps_for_rows(warps, rows, sms);
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
-    kernel<<<grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream>>>(
-        static_cast<const uint32_t*>(x_act), rows, d, ld, k, cols_out, static_cast<uint32_t*>(vals_out), rows_out,
-        static_cast<uint32_t*>(tau_out), result);
-    DCT_CUDA_TRY(cudaGetLastError());
+    DCT_CUDA_TRY(launch_chained_smem(kernel, grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream,
+                                     static_cast<const uint32_t*>(x_act), rows, d, ld, k, cols_out,
+                                     static_cast<uint32_t*>(vals_out), rows_out, static_cast<uint32_t*>(tau_out), result));
     return DCT_OK;
 }
 

@@ -99,6 +99,66 @@ __device__ __forceinline__ uint32_t pick_mantissa(const uint32_t* hist, uint32_t
     return __shfl_sync(0xFFFFFFFFu, found, src) & 0x7Fu;
 }
 
+// General slow path for one row (rare): no usable bound, or very many elements tie at it.  tau_i is found
+// bit by bit on the row itself, most significant first (the largest v with #{key >= v} >= k); then
+// everything above tau_i and the first ties are written, in column order, straight from the row.
+// Kept out of line so that the common path stays small in the instruction cache.
+template <int E8>
+__device__ __noinline__ void mp_row_slow_path(const unsigned char* span, uint32_t k, size_t out_base, uint32_t row,
+                                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
+                                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out) {
+    constexpr uint32_t E = E8 * 8u;
+    constexpr int kMaskWords = (E8 + 3) / 4;
+    const uint32_t lane = lane_id();
+    uint32_t tau_key = 0;
+#pragma unroll 1
+    for (int bit = 14; bit >= 0; --bit) {
+        const uint32_t trial = tau_key | (1u << bit);
+        uint32_t cnt = 0;
+#pragma unroll 4
+        for (int c = 0; c < E8; ++c)
+            cnt += __popc(mask8_ge_exact(*reinterpret_cast<const uint4*>(span + c * 16), trial));
+        if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= k) tau_key = trial;
+    }
+    uint32_t gt_masks[kMaskWords], eq_masks[kMaskWords];
+    uint32_t n_gt_mine = 0, n_eq_mine = 0;
+#pragma unroll
+    for (int i = 0; i < kMaskWords; ++i) gt_masks[i] = eq_masks[i] = 0;
+#pragma unroll
+    for (int c = 0; c < E8; ++c) {
+        const uint4 v = *reinterpret_cast<const uint4*>(span + c * 16);
+        const uint32_t gt = mask8_ge_exact(v, tau_key + 1u);
+        const uint32_t eq = mask8_ge_exact(v, tau_key) & ~gt;
+        gt_masks[c / 4] |= gt << (8 * (c % 4));
+        eq_masks[c / 4] |= eq << (8 * (c % 4));
+        n_gt_mine += __popc(gt);
+        n_eq_mine += __popc(eq);
+    }
+    const uint32_t incl = warp_inclusive_sum(n_gt_mine);
+    const uint32_t take = k - __shfl_sync(0xFFFFFFFFu, incl, 31);   // ties to keep, lowest columns first
+    uint32_t g_at = incl - n_gt_mine;
+    uint32_t e_at = warp_inclusive_sum(n_eq_mine) - n_eq_mine;
+#pragma unroll
+    for (int wd = 0; wd < kMaskWords; ++wd) {
+        uint32_t m = gt_masks[wd] | eq_masks[wd];
+        while (m) {
+            const uint32_t bit = __ffs(m) - 1;
+            m &= m - 1;
+            const bool is_eq = (eq_masks[wd] >> bit) & 1u;
+            if (!is_eq || e_at < take) {
+                const uint32_t j = wd * 32 + bit;
+                const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
+                cols_out[pos] = static_cast<int16_t>(lane * E + j);
+                vals_out[pos] = *reinterpret_cast<const uint16_t*>(span + j * 2);
+                if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
+            }
+            g_at += is_eq ? 0u : 1u;
+            e_at += is_eq ? 1u : 0u;
+        }
+    }
+    if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+}
+
 // PL: candidates a lane holds in registers (5: k <= 112, rows of at most 1024 columns; 10: k <= 224; 20: k <= 448, with 4-element leaves for the
 // exact bound, since 8-element leaves get loose as k approaches their number).
 template <int PL> struct FwdVariant {

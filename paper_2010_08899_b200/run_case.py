@@ -35,6 +35,8 @@ def main():
     ap.add_argument("--dist", choices=["mixture", "gaussian", "dlrm"], default="mixture")
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
+    ap.add_argument("--back-to-back", action="store_true",
+                    help="time all iterations between one pair of events (launch gaps overlap, as in a training loop)")
     args = ap.parse_args()
 
     dev = "cuda"
@@ -180,6 +182,17 @@ def main():
         reset()
         call(i)
     torch.cuda.synchronize()
+    if args.back_to_back:
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for i in range(args.iters):
+            call(i)
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / args.iters
+        print(f"{args.entry}: {ms:.4f} ms per call back to back, {nbytes / ms / 1e6:.1f} GB/s algorithmic ({nbytes} B per call)")
+        return
     pairs = []
     for i in range(args.iters):
         reset()
