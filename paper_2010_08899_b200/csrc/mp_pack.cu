@@ -369,12 +369,11 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         auto build_masks = [&](uint32_t bound) {
             // unit u = 32 c + lane covers columns 8 u .. 8 u + 7: its 8 flags are byte u of the mask table, which
             // therefore holds one bit per column, in column order
-            const __nv_bfloat162 low2 = as_bf162(bound | (bound << 16));
             unsigned char* tab8 = reinterpret_cast<unsigned char*>(mask_tab) + lane;
 #pragma unroll
             for (int c = 0; c < E8; ++c)
                 tab8[c * 32] = static_cast<unsigned char>(
-                    mask8_ge_filter(*reinterpret_cast<const uint4*>(unit0 + c * 512), low2));
+                    mask8_ge_exact(*reinterpret_cast<const uint4*>(unit0 + c * 512), bound));
             __syncwarp();
             // the lane's own words: columns 32 kMaskWords lane onwards (words past the end of the row are empty)
             if (kMaskWords == 4) {
@@ -862,29 +861,16 @@ mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uin
         int last_move = 0;
 #pragma unroll 1
         for (int attempt = 0; attempt < kDenseRetries; ++attempt) {
-            // exact integer compares (the tables decide what is kept, so "a superset" is not enough here);
-            // low <= 0x7F80 keeps low + window within their 2^15 range
+            // exact compares (the tables decide what is kept); low <= 0x7F80 keeps low + window within the 2^15 keys
             const uint32_t high = low + window;
             unsigned char* tl = reinterpret_cast<unsigned char*>(tab_low) + lane;
             unsigned char* th = reinterpret_cast<unsigned char*>(tab_high) + lane;
             __syncwarp();
-            if (low >= 0x0080u && high <= 0x7F80u) {
-                // both bounds are normal numbers (or infinity): the packed floating-point compare is exact for
-                // every element that is not a NaN, and a NaN lands in both tables, i.e. outside the window
-                const __nv_bfloat162 low2 = as_bf162(low * 0x10001u), high2 = as_bf162(high * 0x10001u);
 #pragma unroll
-                for (int c = 0; c < E8; ++c) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(unit0 + c * 512);
-                    tl[c * 32] = static_cast<unsigned char>(mask8_ge_filter(v, low2));
-                    th[c * 32] = static_cast<unsigned char>(mask8_ge_filter(v, high2));
-                }
-            } else {
-#pragma unroll
-                for (int c = 0; c < E8; ++c) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(unit0 + c * 512);
-                    tl[c * 32] = static_cast<unsigned char>(mask8_ge_exact(v, low));
-                    th[c * 32] = static_cast<unsigned char>(mask8_ge_exact(v, high));
-                }
+            for (int c = 0; c < E8; ++c) {
+                const uint4 v = *reinterpret_cast<const uint4*>(unit0 + c * 512);
+                tl[c * 32] = static_cast<unsigned char>(mask8_ge_exact(v, low));
+                th[c * 32] = static_cast<unsigned char>(mask8_ge_exact(v, high));
             }
             __syncwarp();
             uint32_t mine = 0;

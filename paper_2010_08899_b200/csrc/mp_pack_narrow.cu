@@ -168,10 +168,9 @@ mp_topk_fwd_bf16_narrow_kernel(const uint16_t* __restrict__ x, uint32_t rows, ui
         // ---- B (with A): candidate bits of the lane, one word in column order -------------------------
         uint32_t mask = 0, incl = 0, n_cand = 0;
         auto build_mask = [&](uint32_t bound) {
-            const __nv_bfloat162 low2 = as_bf162(bound | (bound << 16));
             mask = 0;
 #pragma unroll
-            for (int c = 0; c < E8; ++c) mask |= mask8_ge_filter(cur[c], low2) << (8 * c);
+            for (int c = 0; c < E8; ++c) mask |= mask8_ge_exact(cur[c], bound) << (8 * c);
             incl = Gr::inclusive_sum(__popc(mask), gl);
             n_cand = Gr::last(incl);
         };

@@ -16,27 +16,29 @@ __device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u) { return *reinter
 __device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 h) { return *reinterpret_cast<uint32_t*>(&h); }
 
 
-// bit j set iff |element j| >= low, for the 8 bf16 of one int4.  Floating-point compare: exact for
-// normal numbers; may also admit a few denormals/zeros if the hardware flushes (a superset is fine
-// for a candidate filter); NaN always passes.
-__device__ __forceinline__ uint32_t mask8_ge_filter(uint4 v, __nv_bfloat162 low2) {
-    const uint32_t r0 = __hgeu2_mask(__habs2(as_bf162(v.x)), low2);
-    const uint32_t r1 = __hgeu2_mask(__habs2(as_bf162(v.y)), low2);
-    const uint32_t r2 = __hgeu2_mask(__habs2(as_bf162(v.z)), low2);
-    const uint32_t r3 = __hgeu2_mask(__habs2(as_bf162(v.w)), low2);
-    const uint32_t m = (r0 & 0x00020001u) | (r1 & 0x00080004u) | (r2 & 0x00200010u) | (r3 & 0x00800040u);
-    return (m | (m >> 16)) & 0xFFu;
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
 }
-// the same on the integer keys, exact for every bit pattern (low <= 0x8000)
+__device__ __forceinline__ int dp4a_ss(uint32_t a, uint32_t b, int c) {     // signed 8-bit dot product + c
+    int d;
+    asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+// bit j set iff key(element j) >= low, for the 8 bf16 of one int4; exact for every bit pattern (low <= 0x8000).
+// Per 16-bit half, bit 15 of ((x | 0x8000) - low) is set iff key(x) >= low, and no borrow crosses the halves.  A
+// byte permutation picks the upper byte of every half with its sign bit replicated (0xFF = -1 or 0), and two
+// signed dot products with the weights -2^j turn the eight bytes into the eight flags: 12 instructions.
 __device__ __forceinline__ uint32_t mask8_ge_exact(uint4 v, uint32_t low) {
     const uint32_t low2 = low | (low << 16);
-    // per 16-bit half: bit 15 of ((key | 0x8000) - low) is set iff key >= low (no borrow crosses halves)
-    const uint32_t t0 = (((v.x & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
-    const uint32_t t1 = (((v.y & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
-    const uint32_t t2 = (((v.z & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
-    const uint32_t t3 = (((v.w & kAbsMask2) | 0x80008000u) - low2) & 0x80008000u;
-    uint32_t m = (t0 >> 15) | (t1 >> 13) | (t2 >> 11) | (t3 >> 9);   // halves at bits {0,16},{2,18},{4,20},{6,22}
-    return (m | (m >> 15)) & 0xFFu;
+    const uint32_t t0 = (v.x | 0x80008000u) - low2;
+    const uint32_t t1 = (v.y | 0x80008000u) - low2;
+    const uint32_t t2 = (v.z | 0x80008000u) - low2;
+    const uint32_t t3 = (v.w | 0x80008000u) - low2;
+    const uint32_t a = prmt(t0, t1, 0xFDB9u);              // elements 0..3
+    const uint32_t b = prmt(t2, t3, 0xFDB9u);              // elements 4..7
+    return static_cast<uint32_t>(dp4a_ss(b, 0x80C0E0F0u, dp4a_ss(a, 0xF8FCFEFFu, 0)));
 }
 
 // v = *(uint2*)shared_address if p (a predicated load: no branch)
