@@ -268,16 +268,22 @@ DCT_API dct_status_t dct_threshold_select_batched(
  * threshold comes from the very vector that is compressed (the scheme the paper starts from, and on
  * its CPUs found 11 % slower end to end than no compression).
  *
- * Enqueues dct_threshold_select on fl32(grad + residual), derives the tie budget k - n_gt on the
- * device, and runs dct_dp_compress with it: exactly min(k, capacity) elements are sent, the lowest
- * indices first among those equal to the threshold.
+ * The result is that of dct_threshold_select on fl32(grad + residual) followed by dct_dp_compress with the
+ * tie budget k - n_gt: exactly min(k, capacity) elements are sent, the lowest indices first among those
+ * equal to the threshold.  From 2^25 elements, with k small against n, the vector is streamed only once
+ * (12 bytes per element, the cost of an iteration with a fixed threshold): a bound from a sector-wise
+ * sample, one compress pass that leaves w in the residual and packs the elements above the bound, the
+ * exact select over those, and a pass over them that sends the survivors and puts the others back; should
+ * the sample misjudge the vector, the plain select and compress run on w instead (same result, decided on
+ * the device).  Smaller vectors and dense k take the two operators back to back (20 bytes per element).
  *
  *   grad, residual, n, idx_out, val_out, capacity   as in dct_dp_compress.
  *   k          survivors wanted, 1 <= k <= n.
  *   tau_out    1 fp32 (device): the threshold that was used.
  *   result     device block: count (= min(k, capacity)), needed (= k), status as in dct_dp_compress,
  *              and n_gt, n_eq of the select.
- *   workspace  >= dct_dp_select_compress_workspace_bytes(n), 256-byte aligned.
+ *   workspace  >= dct_dp_select_compress_workspace_bytes(n), 256-byte aligned (from 2^25 elements it includes
+ *              32 MiB for the packed elements above the bound).
  */
 DCT_API size_t dct_dp_select_compress_workspace_bytes(uint64_t n);
 DCT_API dct_status_t dct_dp_select_compress(

@@ -35,6 +35,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "dp_chain.cuh"
 
 namespace dct {
 namespace {
@@ -69,10 +70,12 @@ struct CompressCtrl {
 constexpr size_t kCtrlBytes = 256;
 
 __global__ void dp_compress_init_kernel(CompressCtrl* ctrl, uint64_t* tile_state, uint32_t num_tiles,
-                                        dct_result_t* result, uint32_t first_ticket) {
+                                        dct_result_t* result, uint32_t first_ticket,
+                                        const uint32_t* __restrict__ enabled = nullptr) {
     // the streaming kernel that follows may be scheduled already (it waits for this grid before it touches the
     // control block): its launch latency and set-up then overlap this kernel
     chain_release_next();
+    if (enabled && *enabled == 0) return;     // a conditional call that is not needed: nothing is touched
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < num_tiles) tile_state[i] = 0;
     if (i == 0) {
@@ -307,15 +310,17 @@ __device__ __forceinline__ void compress_tile_body(const float* __restrict__ gra
     if (full_tile) {
         float4 g4[kVecs], e4[kVecs];
 #pragma unroll
-        for (int j = 0; j < kVecs; ++j) g4[j] = ld_readonly_f4(grad + warp_base + j * 128 + lane * 4);
+        for (int j = 0; j < kVecs; ++j)
+            g4[j] = grad ? ld_readonly_f4(grad + warp_base + j * 128 + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int j = 0; j < kVecs; ++j) e4[j] = ld_stream_f4(residual + warp_base + j * 128 + lane * 4);
 #pragma unroll
         for (int j = 0; j < kVecs; ++j) {
-            w[4 * j + 0] = __fadd_rn(g4[j].x, e4[j].x);
-            w[4 * j + 1] = __fadd_rn(g4[j].y, e4[j].y);
-            w[4 * j + 2] = __fadd_rn(g4[j].z, e4[j].z);
-            w[4 * j + 3] = __fadd_rn(g4[j].w, e4[j].w);
+            // (no gradient: w is the stored value itself, bit for bit -- adding +0 would turn -0 into +0)
+            w[4 * j + 0] = grad ? __fadd_rn(g4[j].x, e4[j].x) : e4[j].x;
+            w[4 * j + 1] = grad ? __fadd_rn(g4[j].y, e4[j].y) : e4[j].y;
+            w[4 * j + 2] = grad ? __fadd_rn(g4[j].z, e4[j].z) : e4[j].z;
+            w[4 * j + 3] = grad ? __fadd_rn(g4[j].w, e4[j].w) : e4[j].w;
         }
     } else {
         valid_mask = 0;
@@ -323,7 +328,7 @@ __device__ __forceinline__ void compress_tile_body(const float* __restrict__ gra
         for (int b = 0; b < kVecs * 4; ++b) {
             const uint32_t i = warp_base + (b >> 2) * 128 + lane * 4 + (b & 3);
             const bool valid = i < n;
-            w[b] = valid ? __fadd_rn(grad[i], residual[i]) : 0.0f;
+            w[b] = valid ? (grad ? __fadd_rn(grad[i], residual[i]) : residual[i]) : 0.0f;
             valid_mask |= valid ? (1u << b) : 0u;
         }
     }
@@ -387,8 +392,9 @@ dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ resi
                         int32_t* __restrict__ idx_out, float* __restrict__ val_out, uint64_t capacity,
                         dct_result_t* __restrict__ result, CompressCtrl* ctrl,
                         uint64_t* __restrict__ tile_state, uint32_t num_tiles, uint32_t fixed_tile,
-                        uint32_t spin_limit) {
+                        uint32_t spin_limit, const uint32_t* __restrict__ enabled = nullptr) {
     __shared__ uint32_t s_tile;
+    if (enabled && *enabled == 0) return;     // a conditional call that is not needed
     if (threadIdx.x == 0) s_tile = fixed_tile != kInvalidTile ? fixed_tile : atomicAdd(&ctrl->ticket, 1u);
     __syncthreads();
     const uint32_t tile = s_tile;
@@ -858,6 +864,35 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
             num_full, dbg.spin_limit);
         DCT_CUDA_TRY(cudaGetLastError());
     }
+    return DCT_OK;
+}
+
+// Algorithm 1, mask / compressed gradient / error steps on a vector that is already summed (w = g + e lies in
+// `residual`), enqueued unconditionally but run only if *enabled != 0: the plain way of dct_dp_select_compress when
+// its sample has misjudged the vector.  One CTA per tile with plain loads (the rare path need not be the fast one).
+dct_status_t dct::compress_presummed_if(const uint32_t* enabled, float* residual, uint64_t n, const float* tau,
+                                        const uint64_t* tie_budget, int32_t* idx_out, float* val_out, uint64_t capacity,
+                                        dct_result_t* result, void* workspace, size_t workspace_bytes,
+                                        cudaStream_t stream) {
+    if (!workspace || !aligned_to(workspace, 256) || workspace_bytes < dct_dp_compress_workspace_bytes(n))
+        return DCT_ERR_WORKSPACE;
+    auto* ctrl = static_cast<CompressCtrl*>(workspace);
+    auto* tile_state = reinterpret_cast<uint64_t*>(static_cast<char*>(workspace) + kCtrlBytes);
+    const uint32_t n32 = static_cast<uint32_t>(n);
+    const uint32_t num_tiles = dp_compress_num_tiles(n);
+    const DebugConfig& dbg = debug_config();
+    dp_compress_init_kernel<<<(num_tiles + 1023) / 1024, 1024, 0, stream>>>(ctrl, tile_state, num_tiles, result, 0u,
+                                                                            enabled);
+    DCT_CUDA_TRY(cudaGetLastError());
+    if (aligned_to(residual, 16))
+        dp_compress_tile_kernel<true><<<num_tiles, kThreads, 0, stream>>>(
+            nullptr, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
+            kInvalidTile, dbg.spin_limit, enabled);
+    else
+        dp_compress_tile_kernel<false><<<num_tiles, kThreads, 0, stream>>>(
+            nullptr, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
+            kInvalidTile, dbg.spin_limit, enabled);
+    DCT_CUDA_TRY(cudaGetLastError());
     return DCT_OK;
 }
 

@@ -22,6 +22,7 @@
 // Every decision is taken on the device; all kernels are enqueued up front and the ones that are
 // not needed return at once.  The result is exact in every case.
 #include "common.cuh"
+#include "dp_chain.cuh"
 
 namespace dct {
 namespace {
@@ -108,6 +109,9 @@ struct StridedSource {       // the same at (i / 8) * stride + i % 8: groups of 
 struct KeySource {           // keys stored in the workspace
     const uint32_t* keys;
 };
+struct ValueSource {         // key(values[i]): a list of packed values
+    const float* values;
+};
 
 __device__ __forceinline__ uint32_t key_at(const VectorSource& s, uint32_t i) {
     return key_f32(s.residual ? __fadd_rn(s.grad[i], s.residual[i]) : s.grad[i]);
@@ -117,6 +121,7 @@ __device__ __forceinline__ uint32_t key_at(const StridedSource& s, uint32_t i) {
     return key_f32(s.residual ? __fadd_rn(s.grad[j], s.residual[j]) : s.grad[j]);
 }
 __device__ __forceinline__ uint32_t key_at(const KeySource& s, uint32_t i) { return s.keys[i]; }
+__device__ __forceinline__ uint32_t key_at(const ValueSource& s, uint32_t i) { return key_f32(s.values[i]); }
 
 // Scan of one pass's histogram by the last CTA: the digit that holds rank k_rem, counted from the top.
 template <int kPass>
@@ -356,7 +361,89 @@ uint32_t candidate_capacity(uint64_t n) {
     return static_cast<uint32_t>(n < kMaxCandidates ? n : kMaxCandidates);
 }
 
+// L = 1: after the compress pass that extracted the candidates.  The list is usable if it holds at least k
+// elements and nothing was cut off; otherwise the plain select runs on w.
+__global__ void l1_decide_kernel(SelectWorkspace* ws, L1Block* block, uint32_t k, uint32_t cand_capacity) {
+    chain_release_next();
+    chain_wait_previous();
+    const uint64_t found = block->cand_result.needed;
+    const bool ok = block->cand_result.status == DCT_OK && found >= k && found <= cand_capacity;
+    block->use_candidates = ok ? 1u : 0u;
+    block->fallback = ok ? 0u : 1u;
+    block->cand_count = static_cast<uint32_t>(block->cand_result.count);
+    ws->cand.n = static_cast<uint32_t>(found);
+    ws->cand.enabled = ok ? 1u : 0u;
+    ws->full.enabled = ok ? 0u : 1u;
+}
+// the candidates go back into the residual, which then holds w = g + e everywhere
+__global__ void l1_restore_kernel(const int32_t* __restrict__ cand_idx, const float* __restrict__ cand_val,
+                                  float* __restrict__ residual, const L1Block* block) {
+    chain_release_next();
+    chain_wait_previous();
+    if (!block->fallback) return;
+    const uint32_t c = block->cand_count;
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < c; i += gridDim.x * blockDim.x)
+        residual[cand_idx[i]] = cand_val[i];
+}
+__global__ void l1_budget_kernel(L1Block* block, const dct_result_t* sel, uint64_t k) {
+    chain_release_next();
+    chain_wait_previous();
+    block->n_gt = sel->n_gt;
+    block->n_eq = sel->n_eq;
+    block->tie_budget = k > sel->n_gt ? k - sel->n_gt : 0;
+}
+
 }  // namespace
+
+bool l1_sampled_path_applies(uint64_t n, uint64_t k, uint64_t cand_capacity) {
+    if (n < kMinSampledN || n > 0x7FFFFFFFull || cand_capacity == 0) return false;
+    const uint64_t cap = cand_capacity < 0xFFFFFFFFull ? cand_capacity : 0xFFFFFFFFull;
+    return sample_rank(n, k, kSampleSize, static_cast<uint32_t>(cap)) != 0;
+}
+
+dct_status_t l1_sample_bound(const float* grad, const float* residual, uint64_t n, uint64_t k, uint64_t cand_capacity,
+                             L1Block* block, void* select_ws, cudaStream_t stream) {
+    auto* ws = static_cast<SelectWorkspace*>(select_ws);
+    const uint32_t n32 = static_cast<uint32_t>(n), k32 = static_cast<uint32_t>(k);
+    const uint32_t cap = static_cast<uint32_t>(cand_capacity < 0xFFFFFFFFull ? cand_capacity : 0xFFFFFFFFull);
+    const uint32_t sample_k = sample_rank(n, k, kSampleSize, cap);
+    if (sample_k == 0) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint32_t stride = (n32 / (kSampleSize / kSampleGroup)) & ~(kSampleGroup - 1u);
+    select_init_kernel<<<1, kInitThreads, 0, stream>>>(ws, n32, k32, kSampleSize, sample_k, cap, &block->scratch);
+    DCT_CUDA_TRY(cudaGetLastError());
+    const StridedSource ssrc{grad, residual, stride};
+    const uint64_t chunks = (kSampleSize + kSelChunk - 1) / kSelChunk;
+    const int grid = static_cast<int>(chunks < static_cast<uint64_t>(sms) * 4 ? chunks : sms * 4);
+    DCT_CUDA_TRY((launch_three_passes<StridedSource, false>(grid, stream, ssrc, &ws->sample, &block->lo, &block->scratch)));
+    return DCT_OK;
+}
+
+dct_status_t l1_exact_threshold(const int32_t* cand_idx, const float* cand_val, uint64_t cand_capacity, float* residual,
+                                uint64_t n, uint64_t k, float* tau_out, L1Block* block, void* select_ws,
+                                cudaStream_t stream) {
+    auto* ws = static_cast<SelectWorkspace*>(select_ws);
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint32_t cap = static_cast<uint32_t>(cand_capacity < 0xFFFFFFFFull ? cand_capacity : 0xFFFFFFFFull);
+    DCT_CUDA_TRY(launch_chained(l1_decide_kernel, 1, 1, stream, ws, block, static_cast<uint32_t>(k), cap));
+    DCT_CUDA_TRY(launch_chained(l1_restore_kernel, sms * 2, 256, stream, cand_idx, cand_val, residual,
+                                static_cast<const L1Block*>(block)));
+    // the exact select: over the candidates (normally), or over w (the kernels that are not needed return at once)
+    const ValueSource csrc{cand_val};
+    DCT_CUDA_TRY((launch_three_passes<ValueSource, false>(128, stream, csrc, &ws->cand, tau_out, &block->scratch)));
+    const VectorSource wsrc{residual, nullptr};
+    const uint64_t chunks = (n + kSelChunk - 1) / kSelChunk;
+    const int grid = static_cast<int>(chunks < static_cast<uint64_t>(sms) * 4 ? (chunks ? chunks : 1) : sms * 4);
+    if (aligned_to(residual, 16))
+        DCT_CUDA_TRY((launch_three_passes<VectorSource, true>(grid, stream, wsrc, &ws->full, tau_out, &block->scratch)));
+    else
+        DCT_CUDA_TRY((launch_three_passes<VectorSource, false>(grid, stream, wsrc, &ws->full, tau_out, &block->scratch)));
+    DCT_CUDA_TRY(launch_chained(l1_budget_kernel, 1, 1, stream, block, static_cast<const dct_result_t*>(&block->scratch), k));
+    return DCT_OK;
+}
+
 }  // namespace dct
 
 using namespace dct;
