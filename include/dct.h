@@ -15,7 +15,8 @@
  * Conventions common to every entry point
  *   - Unless a parameter says "host", every pointer is a DEVICE pointer that
  *     the caller owns.  The library allocates nothing and keeps no state
- *     between calls.
+ *     between calls -- with one exception, dct_dp_compress_static, whose scratch
+ *     is an array built into the library (see there).
  *   - Every call is asynchronous on `stream` (a cudaStream_t passed as an
  *     opaque pointer; NULL is the legacy default stream).  No call
  *     synchronises with the host, except the *_host convenience calls.
@@ -216,6 +217,8 @@ DCT_API dct_status_t dct_mp_pack_bwd(
  *              residual, output or result buffers.
  *   workspace  DEVICE, >= dct_dp_compress_batched_workspace_bytes(sizes, num_layers), 256-byte aligned.
  * Every layer's result block receives its own count / needed / status.
+ * Returns DCT_ERR_UNSUPPORTED while `stream` is being captured into a CUDA graph (the call uploads a table it
+ * builds from `layers` on the host, which a graph would outlive).
  */
 typedef struct {
   const float* grad;           /* [n] device */
@@ -247,7 +250,9 @@ DCT_API dct_status_t dct_dp_compress_batched(
  *              1 <= k <= n <= 2^31-1 per layer, and the sizes must add up to less than 2^44).  Read before the
  *              call returns.  Layers must not share tau_out or result.
  *   workspace  DEVICE, >= dct_threshold_select_batched_workspace_bytes(num_layers), 256-byte aligned.
- * Errors: DCT_ERR_INVALID_ARG / DCT_ERR_WORKSPACE as for dct_threshold_select, before anything is launched.
+ * Errors: DCT_ERR_INVALID_ARG / DCT_ERR_WORKSPACE as for dct_threshold_select, before anything is launched;
+ * DCT_ERR_UNSUPPORTED while `stream` is being captured into a CUDA graph (the call uploads a table it builds
+ * from `layers` on the host, which a graph would outlive).
  */
 typedef struct {
   const float* grad;           /* [n] device, read only */
@@ -493,7 +498,9 @@ DCT_API dct_status_t dct_dp_drift_check(
     uint32_t* flag_out, dct_stream_t stream);
 
 /*
- * Testing knobs (process-wide, not for production use).  spin_limit is the
+ * TEST-ONLY knobs, exported for the library's own test-suite and not part of the production interface: two
+ * process-wide words (atomics) that every later call reads once.  A build with -DDCT_NO_TEST_HOOKS turns the
+ * call into a no-op.  spin_limit is the
  * number of polls a device-side wait may take before it gives up with
  * DCT_ERR_TIMEOUT (default 2^21, about a second).  first_ticket is the id of
  * the first tile dct_dp_compress hands out (default 0); with 1, tile 0 is never

@@ -18,10 +18,14 @@ void note_cuda_error(cudaError_t e) {
     (void)cudaGetLastError();   // clear the sticky-free error state
 }
 
-DebugConfig& debug_config() {
-    // about one second of waiting at the back-off the look-back uses
-    static DebugConfig cfg = {1u << 21, 0u};
-    return cfg;
+namespace {
+// about one second of waiting at the back-off the look-back uses; tile ids start at 0
+std::atomic<uint32_t> g_spin_limit{1u << 21};
+std::atomic<uint32_t> g_first_ticket{0u};
+}  // namespace
+
+DebugConfig debug_config() {
+    return DebugConfig{g_spin_limit.load(std::memory_order_relaxed), g_first_ticket.load(std::memory_order_relaxed)};
 }
 
 int sm_count() {
@@ -65,9 +69,13 @@ extern "C" const char* dct_status_string(dct_status_t s) {
 extern "C" const char* dct_last_cuda_error(void) { return g_last_error; }
 
 extern "C" void dct_debug_configure(uint32_t spin_limit, uint32_t first_ticket) {
-    DebugConfig& c = debug_config();
-    c.spin_limit = spin_limit;
-    c.first_ticket = first_ticket;
+#ifndef DCT_NO_TEST_HOOKS
+    g_spin_limit.store(spin_limit, std::memory_order_relaxed);
+    g_first_ticket.store(first_ticket, std::memory_order_relaxed);
+#else
+    (void)spin_limit;
+    (void)first_ticket;
+#endif
 }
 
 extern "C" dct_status_t dct_dp_compress_host(const float* grad_host, float* grad_dev, float* residual_dev, uint64_t n,

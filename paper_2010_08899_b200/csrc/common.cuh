@@ -138,13 +138,20 @@ void note_cuda_error(cudaError_t e);          // remembers the text for dct_last
         }                                                    \
     } while (0)
 
+// true while `stream` is being captured into a CUDA graph (calls that upload a host-built table from a
+// temporary refuse to run then: the graph would keep a pointer to freed host memory)
+inline bool stream_is_capturing(cudaStream_t stream) {
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    return cudaStreamIsCapturing(stream, &st) == cudaSuccess && st != cudaStreamCaptureStatusNone;
+}
+
 inline bool aligned_to(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 struct DebugConfig {
     uint32_t spin_limit;     // iterations a device-side wait may take before it gives up
     uint32_t first_ticket;   // first tile id handed out by dct_dp_compress (testing: 0 in production)
 };
-DebugConfig& debug_config();
+DebugConfig debug_config();    // a snapshot of the two testing knobs (atomics inside)
 
 int sm_count();              // multiprocessors of the current device (cached per device)
 uint32_t next_launch_ticket();   // a process-wide, never-zero, ever-changing number that marks one launch

@@ -25,7 +25,8 @@ dp_decompress_kernel(const int32_t* __restrict__ idx, const float* __restrict__ 
     // this CTA owns dense[lo, hi): a multiple of 4 elements so that the clearing stores stay aligned
     const uint32_t per = ((n + gridDim.x - 1) / gridDim.x + 3u) & ~3u;
     const uint64_t lo64 = static_cast<uint64_t>(blockIdx.x) * per;
-    if (lo64 >= n) return;
+    bool bad = false;
+    if (lo64 < n) {               // (CTAs past the end of the vector only help to check the list)
     const uint32_t lo = static_cast<uint32_t>(lo64);
     const uint32_t hi = (n - lo > per) ? lo + per : n;
     if (!accumulate) {
@@ -46,15 +47,21 @@ dp_decompress_kernel(const int32_t* __restrict__ idx, const float* __restrict__ 
         const uint32_t mid = (a + b) >> 1;
         if (static_cast<uint32_t>(idx[mid]) < lo) a = mid + 1; else b = mid;
     }
-    bool bad = false;
     for (uint32_t j = a + threadIdx.x; j < count; j += blockDim.x) {
         const uint32_t i = static_cast<uint32_t>(idx[j]);
         if (i >= hi) break;       // the rest belongs to later CTAs (or is out of range)
         if (i < lo) { bad = true; continue; }   // not ascending
         if (accumulate) dense[i] += val[j]; else dense[i] = val[j];
     }
-    // entries at or beyond n belong to nobody: the last CTA reports them
-    if (hi == n && threadIdx.x == 0 && count > 0 && static_cast<uint32_t>(idx[count - 1]) >= n) bad = true;
+    }
+    // The list itself is checked once, by all CTAs together: every index inside [0, n), every index above the one
+    // before it.  (An index that fails is never written outside the vector -- the loop above only writes inside this
+    // CTA's range -- but the dense vector is then not what the sender meant: DCT_ERR_BAD_MASK.)
+    for (uint64_t j = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < count;
+         j += static_cast<uint64_t>(gridDim.x) * blockDim.x) {
+        const int32_t i = idx[j];
+        if (static_cast<uint32_t>(i) >= n || (j > 0 && i <= idx[j - 1])) bad = true;
+    }
     if (bad) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
 }
 

@@ -938,6 +938,7 @@ extern "C" size_t dct_dp_compress_batched_workspace_bytes(const uint64_t* n, uin
 extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, uint32_t num_layers, void* workspace,
                                                 size_t workspace_bytes, dct_stream_t stream_) {
     if (!layers || num_layers == 0) return DCT_ERR_INVALID_ARG;
+    if (stream_is_capturing(static_cast<cudaStream_t>(stream_))) return DCT_ERR_UNSUPPORTED;   // uploads a temporary table
     std::vector<uint64_t> sizes(num_layers);
     for (uint32_t l = 0; l < num_layers; ++l) {
         const dct_dp_layer_t& a = layers[l];

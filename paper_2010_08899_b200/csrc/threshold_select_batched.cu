@@ -206,6 +206,7 @@ extern "C" size_t dct_threshold_select_batched_workspace_bytes(uint32_t num_laye
 extern "C" dct_status_t dct_threshold_select_batched(const dct_select_layer_t* layers, uint32_t num_layers,
                                                      void* workspace, size_t workspace_bytes, dct_stream_t stream_) {
     if (!layers || num_layers == 0) return DCT_ERR_INVALID_ARG;
+    if (stream_is_capturing(static_cast<cudaStream_t>(stream_))) return DCT_ERR_UNSUPPORTED;   // uploads a temporary table
     uint64_t total_chunks = 0, total_elems = 0;
     for (uint32_t l = 0; l < num_layers; ++l) {
         const dct_select_layer_t& a = layers[l];

@@ -178,6 +178,34 @@ def test_gpu_mp_unpack_matches_oracle_and_round_trips(dtype, rows, d, ld, k):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("accumulate", [False, True])
+@pytest.mark.parametrize("bad_idx", [[3, -1, 10], [3, 70000, 10], [10, 5], [7, 7], [0, 1, 2, 2, 9]])
+def test_gpu_dp_decompress_checks_the_whole_index_list(bad_idx, accumulate):
+    """A negative or too-large index in the middle of the list, an unsorted pair and a duplicate are all reported,
+    whichever CTA's range they fall into, and nothing outside the vector is touched."""
+    from paper_2010_08899_b200 import binding as B
+    n = 300_000                                     # several CTA ranges
+    filler = list(range(20_000, 20_000 + 40_000, 7))  # a valid ascending run after the bad entries
+    good = [i for i in bad_idx if 0 <= i < n]
+    idx_list = bad_idx + [i for i in filler if i > max(good)]
+    idx = torch.tensor(idx_list, dtype=torch.int32, device="cuda")
+    val = torch.arange(1, len(idx_list) + 1, dtype=torch.float32, device="cuda")
+    packed = torch.tensor([0, len(idx_list), len(idx_list), 0, 0], dtype=torch.int64, device="cuda")
+    buf = torch.full((n + 64,), 9.0, device="cuda")
+    res = B.new_result()
+    B.dct_dp_decompress(idx, val, packed, len(idx_list), buf[:n], n, accumulate, res)
+    assert B.read_result(res).status == B.DCT_ERR_BAD_MASK
+    assert bool((buf[n:] == 9.0).all())
+    # the same list without its faults is accepted
+    ok = sorted(set(good) | {i for i in filler if i > max(good)})
+    idx2 = torch.tensor(ok, dtype=torch.int32, device="cuda")
+    packed2 = torch.tensor([0, len(ok), len(ok), 0, 0], dtype=torch.int64, device="cuda")
+    res2 = B.new_result()
+    B.dct_dp_decompress(idx2, val[:len(ok)].contiguous(), packed2, len(ok), buf[:n], n, accumulate, res2)
+    assert B.read_result(res2).status == B.DCT_OK
+
+
+@pytest.mark.gpu
 def test_gpu_mp_unpack_rejects_out_of_range_columns():
     from paper_2010_08899_b200 import binding as B
     rows, d, k = 4, 50, 3

@@ -370,12 +370,15 @@ def test_mp_bwd_is_a_gather_and_reuses_the_mask():
     assert np.array_equal(f.cols, cols_before)
     want = torch.take_along_dim(torch.from_numpy(gx), torch.from_numpy(f.cols.astype(np.int64)), dim=1).numpy()
     assert np.array_equal(bits32(gv), bits32(want))
-    # dense reconstruction: X_grad .* M and X_act .* M have the same support (the mask)
+    # dense reconstruction: scattering the packed gradients back gives X_grad .* M, whose support lies inside the
+    # mask of X_act .* M and which agrees with X_grad on every kept column
     m_f = np.zeros((rows, d), bool)
-    m_b = np.zeros((rows, d), bool)
     np.put_along_axis(m_f, f.cols.astype(np.int64), True, axis=1)
-    np.put_along_axis(m_b, f.cols.astype(np.int64), True, axis=1)
-    assert np.array_equal(m_f, m_b) and np.all(m_f.sum(1) == k)
+    assert np.all(m_f.sum(1) == k)
+    dense_b = np.zeros((rows, d), np.float32)
+    np.put_along_axis(dense_b, f.cols.astype(np.int64), gv, axis=1)
+    assert np.array_equal(bits32(dense_b), bits32(np.where(m_f, gx, np.float32(0))))
+    assert not np.any((dense_b != 0) & ~m_f)
     # bf16
     gb = bf16_bits(torch.from_numpy(gx).to(torch.bfloat16))
     assert np.array_equal(oracle.mp_bwd(gb, f.cols), np.take_along_axis(gb, f.cols.astype(np.int64), axis=1))
