@@ -53,6 +53,10 @@ DEFAULT_WORKLOAD = "dp_2p30_x20+mp_16384x4096_bf16_x50"
 # ncu capture at N = 2^28 summarised in profiles/dp_compress_stream_kernel_n2p28.md; traffic grows in
 # proportion to N, so it is scaled to the launch's element count.
 NCU_DRAM_BYTES_PER_ELEM_COMPRESS = 11.816
+# DRAM bytes of one forward-pack launch at 16384 x 4096 bf16, k = 205 (134.3 MB read: the matrix once; 5.7 MB
+# written before the kernel ends, the rest of the 13.4 MB of output still in L2), from the ncu capture summarised in
+# profiles/mp_kernels_16384x4096_bf16_k205.md
+NCU_DRAM_BYTES_MP_FWD = 140.0e6
 
 
 def algorithmic_bytes(cfg, survivors_per_iter):
@@ -101,7 +105,8 @@ class HotPath:
         self.cols = torch.empty(rows * k, dtype=torch.int16, device=device)
         self.vals = torch.empty(rows * k, dtype=torch.bfloat16, device=device)
         self.gvals = torch.empty(rows * k, dtype=torch.bfloat16, device=device)
-        self.res_mp = B.new_result(device)
+        self.res_mp = B.new_result(device)        # forward pack
+        self.res_mp_bwd = B.new_result(device)    # backward pack (its own block: neither call wipes the other's status)
         self.t = 0            # DP iterations done so far (drives the gradient rotation)
         self.calls = 0        # compress calls issued (indexes res_cmp)
         self.launches = 0     # kernels of this library launched
@@ -146,16 +151,18 @@ class HotPath:
             rec()
         rows, d, k = c["mp_rows"], c["mp_d"], c["mp_k"]
         cols_p, vals_p, gv_p, res_p = self.cols.data_ptr(), self.vals.data_ptr(), self.gvals.data_ptr(), self.res_mp.data_ptr()
+        res_b = self.res_mp_bwd.data_ptr()
         for i in range(c["mp_iters"]):
             j = i % c["mp_bufs"]
             st = L.dct_mp_topk_pack_fwd(self.x[j].data_ptr(), 1, rows, d, d, k, cols_p, vals_p, None, None, res_p, s)
             assert st == 0, st
-            st = L.dct_mp_pack_bwd(self.gx[j].data_ptr(), 1, rows, d, d, k, cols_p, gv_p, res_p, s)
+            st = L.dct_mp_pack_bwd(self.gx[j].data_ptr(), 1, rows, d, d, k, cols_p, gv_p, res_b, s)
             assert st == 0, st
         rec()
         # kernels of this library per step: the select enqueues 12 (reset, 3 sample passes, filter, decide,
         # 3 candidate passes, 3 full passes that return at once) from n = 2^25 and 4 (reset + 3 passes) below;
         # each compress is a reset kernel + the streaming kernel; each MP iteration a forward and a backward kernel
+        # (the backward pack resets its result block inside the kernel)
         self.launches += (12 if n >= (1 << 25) else 4) + 2 * c["dp_iters"] + 2 * c["mp_iters"]
 
     def time_mp_parts(self, stream, reps):
@@ -179,6 +186,110 @@ class HotPath:
                 out[name] = a.elapsed_time(b) / reps
         return out
 
+
+    def time_mp_variants(self, stream, reps):
+        """The forward pack on the same matrices at the paper's denser sparsity levels (90 % and 75 %: k = 410 and
+        1024 of 4096), and at k = 205 on rows whose scales differ by orders of magnitude from one row to the next
+        (the previous row's threshold is then a useless guess for the next: the worst case for real activations)."""
+        c, L, s = self.cfg, self.L, stream.cuda_stream
+        rows, d = c["mp_rows"], c["mp_d"]
+        out = {}
+        scale = torch.pow(2.0, ((torch.arange(rows, device=self.dev) % 7) * 3 - 9).float())[:, None]
+        varied = [(self.x[j].float() * scale).to(torch.bfloat16) for j in range(2)]
+        for name, mats, k in (("mp_fwd_k410", self.x, 410), ("mp_fwd_k1024", self.x, 1024),
+                              ("mp_fwd_varied_rows", varied, c["mp_k"])):
+            if k > d // 2:
+                continue
+            cols = torch.empty(rows * k, dtype=torch.int16, device=self.dev)
+            vals = torch.empty(rows * k, dtype=torch.bfloat16, device=self.dev)
+            for phase in range(2):
+                a = _record(stream)
+                for i in range(reps):
+                    st = L.dct_mp_topk_pack_fwd(mats[i % len(mats)].data_ptr(), 1, rows, d, d, k, cols.data_ptr(),
+                                                vals.data_ptr(), None, None, None, s)
+                    assert st == 0, st
+                b = _record(stream)
+                b.synchronize()
+            ms = a.elapsed_time(b) / reps
+            out[name] = {"ms": ms, "k": k, "GBps": (rows * d * 2 + rows * k * 4) / (ms * 1e-3) / 1e9}
+        return out
+
+    def time_c3(self, stream, iters=20):
+        """DCT-DP at DLRM-like MLP scale (64 Mi gradients as concatenated dense-layer blocks, Student-t values,
+        density 0.1 %): the select, the fixed-threshold iterations (mean of `iters`, error starting at zero), and
+        the same vector cut into its 219 layers, each with its own threshold and error, in one batched call."""
+        B = self.B
+        n, dev = 64 << 20, self.dev
+        k = B.k_from_density(n, 1, 1000)
+        cap = n // 32
+        slack = 1 << 12
+        g_raw = [inputs.dp_dlrm_like(n + slack, 300 + j, dev) for j in range(3)]
+        g = [t[:n] for t in g_raw]
+        # iteration i: buffer 1 + i mod 2, shifted by 4 (i div 2) elements, so that every element meets fresh values
+        # each iteration while the error persists (as with a new mini-batch per iteration)
+        fresh = lambda i: g_raw[1 + i % 2][4 * (i // 2): 4 * (i // 2) + n]
+        e = torch.zeros(n, device=dev)
+        tau = torch.zeros(1, device=dev)
+        idx = torch.empty(cap, dtype=torch.int32, device=dev)
+        val = torch.empty(cap, device=dev)
+        res = torch.zeros(iters, 5, dtype=torch.int64, device=dev)
+        res_s = B.new_result(dev)
+        ws_s = B.new_workspace(B.dct_threshold_select_workspace_bytes(n), dev)
+        ws_c = B.new_workspace(B.dct_dp_compress_workspace_bytes(n), dev)
+        out = {"n": n, "k": k}
+        for phase in range(2):
+            a = _record(stream)
+            for i in range(4):
+                B.dct_threshold_select(g[i % 3], None, n, k, tau, res_s, ws_s, stream)
+            b = _record(stream)
+            b.synchronize()
+        ms = a.elapsed_time(b) / 4
+        out["select"] = {"ms": ms, "GBps_at_4B_per_elem": 4 * n / (ms * 1e-3) / 1e9}
+        B.dct_threshold_select(g[0], None, n, k, tau, res_s, ws_s, stream)
+        for phase in range(2):
+            e.zero_()
+            a = _record(stream)
+            for i in range(iters):
+                B.dct_dp_compress(fresh(i), e, n, tau, None, idx, val, cap, res[i], ws_c, stream)
+            b = _record(stream)
+            b.synchronize()
+        ms = a.elapsed_time(b) / iters
+        counts = res[:, 1].tolist()
+        nbytes = sum(12 * n + 8 * c for c in counts) / iters
+        out["compress"] = {"ms": ms, "GBps": nbytes / (ms * 1e-3) / 1e9, "survivors_first_last": [counts[0], counts[-1]]}
+        # layer-wise: every layer its own tau, E and output
+        sizes, total = [], 0
+        while total < n:
+            for fo, fi in inputs.DLRM_LIKE_LAYERS:
+                if total < n:
+                    sizes.append(min(fo * fi, n - total))
+                    total += sizes[-1]
+        e.zero_()
+        sel_layers, layers, off = [], [], 0
+        for m in sizes:
+            lcap = max(m // 16, 64)
+            t = torch.zeros(1, device=dev)
+            sel_layers.append(dict(grad=g[0][off:off + m], residual=None, n=m, k=B.k_from_density(m, 1, 1000),
+                                   tau_out=t, result=B.new_result(dev)))
+            layers.append(dict(grad=g[1][off:off + m], residual=e[off:off + m], n=m, tau=t, tie_budget=None,
+                               idx_out=torch.empty(lcap, dtype=torch.int32, device=dev),
+                               val_out=torch.empty(lcap, device=dev), capacity=lcap, result=B.new_result(dev)))
+            off += m
+        ws_sb = B.new_workspace(B.dct_threshold_select_batched_workspace_bytes(len(sizes)), dev)
+        ws_cb = B.new_workspace(B.dct_dp_compress_batched_workspace_bytes(sizes), dev)
+        sel_table, cmp_table = B.dct_select_layer_table(sel_layers), B.dct_dp_layer_table(layers)
+        for name, fn, bytes_per_elem in (("select_batched", lambda: B.dct_threshold_select_batched(sel_table, ws_sb, stream), 4),
+                                         ("compress_batched", lambda: B.dct_dp_compress_batched(cmp_table, ws_cb, stream), 12)):
+            for phase in range(2):
+                e.zero_()
+                a = _record(stream)
+                for i in range(4):
+                    fn()
+                b = _record(stream)
+                b.synchronize()
+            ms = a.elapsed_time(b) / 4
+            out[name] = {"ms": ms, "layers": len(sizes), f"GBps_at_{bytes_per_elem}B_per_elem": bytes_per_elem * n / (ms * 1e-3) / 1e9}
+        return out
 
     def time_extras(self, stream, reps=3):
         """The entry points beyond the step, timed on their own after the main measurement: threshold
@@ -383,6 +494,22 @@ def measured_peaks():
 # the CPU oracle arm (reference / cpu_baseline)
 # --------------------------------------------------------------------------------------------
 
+def oracle_sample_state(cfg, scale_div, seed0=0):
+    """Host inputs of the 1/scale_div sample (numpy views of seeded torch tensors)."""
+    import numpy as np
+    n = max(cfg["dp_n"] // scale_div, 4096)
+    rows = max(cfg["mp_rows"] // scale_div, 8)
+    d = cfg["mp_d"]
+    return dict(
+        g_sel=inputs.dp_mixture(n, 500 + seed0).numpy(),
+        g=[inputs.dp_mixture(n + cfg["dp_slack"], 501 + j + seed0).numpy() for j in range(2)],
+        e=np.zeros(n, np.float32), t=0,
+        x=[inputs.mp_activations(rows, d, 410 + j + seed0, dtype=torch.bfloat16, col_scale_seed=400)
+           .view(torch.int16).numpy().view(np.uint16) for j in range(2)],
+        gx=[inputs.mp_gradients(rows, d, 420 + j + seed0, dtype=torch.bfloat16)
+            .view(torch.int16).numpy().view(np.uint16) for j in range(2)])
+
+
 def oracle_sample_step(cfg, scale_div, state=None):
     """One step of the same schedule on a 1/scale_div sample, run by the CPU oracle as it stands.
     Returns (seconds, algorithmic bytes, state)."""
@@ -393,14 +520,7 @@ def oracle_sample_step(cfg, scale_div, state=None):
     k_dp = max(cfg["dp_k"] // scale_div, 1)
     d, k = cfg["mp_d"], cfg["mp_k"]
     if state is None:
-        state = dict(
-            g_sel=inputs.dp_mixture(n, 500).numpy(),
-            g=[inputs.dp_mixture(n + cfg["dp_slack"], 501 + j).numpy() for j in range(2)],
-            e=np.zeros(n, np.float32), t=0,
-            x=[inputs.mp_activations(rows, d, 410 + j, dtype=torch.bfloat16, col_scale_seed=400)
-               .view(torch.int16).numpy().view(np.uint16) for j in range(2)],
-            gx=[inputs.mp_gradients(rows, d, 420 + j, dtype=torch.bfloat16)
-                .view(torch.int16).numpy().view(np.uint16) for j in range(2)])
+        state = oracle_sample_state(cfg, scale_div)
     sub = dict(cfg, dp_n=n, mp_rows=rows)
     t0 = time.perf_counter()
     tau = oracle.dp_select(state["g_sel"], None, k_dp).tau
@@ -417,6 +537,28 @@ def oracle_sample_step(cfg, scale_div, state=None):
         oracle.mp_bwd(state["gx"][i % 2], f.cols)
     dt = time.perf_counter() - t0
     return dt, algorithmic_bytes(sub, counts)["total"], state
+
+
+def usable_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def oracle_sharded_step(cfg, scale_div, threads):
+    """The same sample cut into `threads` independent shards -- every shard its own gradient slice, threshold,
+    error and rows, the way the paper's workers each compress their own layers and samples -- with one unmodified
+    oracle per thread (the C calls release the interpreter lock).  Returns (seconds, algorithmic bytes)."""
+    import concurrent.futures
+    shard_cfg = dict(cfg, dp_n=max(cfg["dp_n"] // threads, 4096 * scale_div), mp_rows=max(cfg["mp_rows"] // threads, 8 * scale_div),
+                     dp_k=max(cfg["dp_k"] // threads, scale_div), dp_capacity=max(cfg["dp_capacity"] // threads, 1024 * scale_div))
+    states = [oracle_sample_state(shard_cfg, scale_div, seed0=1000 * (t + 1)) for t in range(threads)]
+    with concurrent.futures.ThreadPoolExecutor(max_workers=threads) as pool:
+        t0 = time.perf_counter()
+        results = list(pool.map(lambda st: oracle_sample_step(shard_cfg, scale_div, st), states))
+        dt = time.perf_counter() - t0
+    return dt, sum(r[1] for r in results)
 
 
 def run_reference(args, cfg):
@@ -459,7 +601,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
-    ap.add_argument("--e2e-steps", type=int, default=1, help="steps of the host-buffer (end to end) measurement")
+    ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the host-buffer (end to end) measurement")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -542,7 +684,19 @@ def main():
         "mp_bwd": {"ms": mp_parts["mp_bwd"], "GBps": b0["mp_bwd"] / cfg["mp_iters"] / (mp_parts["mp_bwd"] * 1e-3) / 1e9,
                    "dense_equiv_GBps": cfg["mp_rows"] * cfg["mp_d"] * 2 / (mp_parts["mp_bwd"] * 1e-3) / 1e9},
     }
+    parts.update(hp.time_mp_variants(stream, cfg["mp_iters"]))
     parts["beyond_the_step"] = hp.time_extras(stream)
+    if args.workload == DEFAULT_WORKLOAD:
+        parts["c3"] = hp.time_c3(stream)
+    fwd_bytes = b0["mp_fwd"] / cfg["mp_iters"]
+    roofline_mp = {
+        "kernel": "mp_topk_fwd_bf16_warp_kernel<16,10>", "bound": "hbm", "achieved": parts["mp_fwd"]["GBps"], "peak": peak,
+        "unit": "GB/s", "frac": parts["mp_fwd"]["GBps"] / peak, "peak_kind": peak_kind,
+        "traffic": NCU_DRAM_BYTES_MP_FWD if cfg["mp_rows"] * cfg["mp_d"] == 16384 * 4096 else None,
+        "algorithmic_bytes_per_launch": fwd_bytes, "frac_of_nominal_8TBps": parts["mp_fwd"]["GBps"] / 8000.0,
+        "note": "duration = CUDA events around %d forward launches back to back, rotating over %d matrices"
+                % (cfg["mp_iters"], cfg["mp_bufs"]),
+    }
     roofline = {
         "kernel": "dp_compress_stream_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak, "peak_kind": peak_kind,
@@ -556,6 +710,8 @@ def main():
     e2e = None
     if not args.no_e2e:
         host = HostPath(hp)
+        host.step(stream)                   # warm-up: pinned pages touched, first-call set-up done
+        host.h2d = host.d2h = 0
         torch.cuda.synchronize()
         barrier()
         t0 = time.perf_counter()
@@ -569,7 +725,7 @@ def main():
         e2e_ms = max(e2e_ms, wall_ms)       # the host-buffer calls synchronise, so wall time is the honest one
         e2e_bytes = float(sum(p["total"] for p in per_step[:1])) * args.e2e_steps
         m_ms, a_bytes = reduce_over_ranks(e2e_ms, e2e_bytes, device)
-        e2e = {"value": a_bytes / (m_ms * 1e-3) / 1e9, "unit": UNIT, "steps": args.e2e_steps,
+        e2e = {"value": a_bytes / (m_ms * 1e-3) / 1e9, "unit": UNIT, "steps": args.e2e_steps, "warmup": 1,
                "ms_per_step": m_ms / args.e2e_steps,
                "h2d_bytes_per_step": host.h2d // args.e2e_steps, "d2h_bytes_per_step": host.d2h // args.e2e_steps}
         del host
@@ -578,9 +734,17 @@ def main():
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         scale = 16 if args.workload == DEFAULT_WORKLOAD else 4
         dt, nbytes, _ = oracle_sample_step(cfg, scale)
+        sample = (f"one full-schedule step on a 1/{scale} sample "
+                  f"({cfg['dp_n'] // scale} gradients, {cfg['mp_rows'] // scale} rows)")
         cpu_baseline = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "seconds": dt,
-                        "sample": f"one full-schedule step on a 1/{scale} sample "
-                                  f"({cfg['dp_n'] // scale} gradients, {cfg['mp_rows'] // scale} rows)"}
+                        "sample": sample}
+        threads = usable_cores()
+        if threads > 1:
+            dt_t, nbytes_t = oracle_sharded_step(cfg, scale, threads)
+            cpu_baseline["threads"] = {
+                "value": nbytes_t / dt_t / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": dt_t,
+                "sample": sample + f", cut into {threads} independent shards (own threshold, error and rows each, as the "
+                                   "paper's workers have), one oracle per thread"}
 
     if rank == 0:
         line = {
@@ -595,7 +759,7 @@ def main():
                        "parallelism": f"independent replicas x{world} (no data-path collective)"},
             "elements_per_s": (n * cfg["dp_iters"] + cfg["mp_rows"] * cfg["mp_d"] * cfg["mp_iters"]) * world
                               / (max_ms / args.steps * 1e-3),
-            "roofline": roofline, "parts": parts, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "roofline": roofline, "roofline_mp": roofline_mp, "parts": parts, "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": gpu_launches, "clocks": clocks, "device_status_codes": statuses,
             "input_checksums": hp.input_checksums(),
         }

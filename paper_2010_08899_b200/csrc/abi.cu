@@ -89,7 +89,10 @@ extern "C" dct_status_t dct_dp_compress_host(const float* grad_host, float* grad
     DCT_CUDA_TRY(cudaMemcpyAsync(grad_dev, grad_host, n * sizeof(float), cudaMemcpyHostToDevice, stream));
     const dct_status_t st = dct_dp_compress(grad_dev, residual_dev, n, tau_dev, tie_budget_dev, idx_dev, val_dev,
                                             capacity, result_dev, workspace, workspace_bytes, stream_);
-    if (st != DCT_OK) return st;
+    if (st != DCT_OK) {
+        (void)cudaStreamSynchronize(stream);      // the upload above is in flight: the caller's buffers are free on return
+        return st;
+    }
     DCT_CUDA_TRY(cudaMemcpyAsync(result_host, result_dev, sizeof(dct_result_t), cudaMemcpyDeviceToHost, stream));
     DCT_CUDA_TRY(cudaStreamSynchronize(stream));
     const uint64_t count = result_host->count;
@@ -110,7 +113,10 @@ extern "C" dct_status_t dct_threshold_select_host(const float* grad_host, float*
     DCT_CUDA_TRY(cudaMemcpyAsync(grad_dev, grad_host, n * sizeof(float), cudaMemcpyHostToDevice, stream));
     const dct_status_t st = dct_threshold_select(grad_dev, residual_dev, n, k, tau_dev, result_dev, workspace,
                                                  workspace_bytes, stream_);
-    if (st != DCT_OK) return st;
+    if (st != DCT_OK) {
+        (void)cudaStreamSynchronize(stream);
+        return st;
+    }
     if (tau_host) DCT_CUDA_TRY(cudaMemcpyAsync(tau_host, tau_dev, sizeof(float), cudaMemcpyDeviceToHost, stream));
     DCT_CUDA_TRY(cudaMemcpyAsync(result_host, result_dev, sizeof(dct_result_t), cudaMemcpyDeviceToHost, stream));
     DCT_CUDA_TRY(cudaStreamSynchronize(stream));
@@ -133,14 +139,24 @@ extern "C" dct_status_t dct_mp_pack_host(const void* x_act_host, const void* x_g
     DCT_CUDA_TRY(cudaMemcpyAsync(x_act_dev, x_act_host, mat_bytes, cudaMemcpyHostToDevice, stream));
     dct_status_t st = dct_mp_topk_pack_fwd(x_act_dev, dtype, rows, d, ld, k, cols_dev, vals_dev, nullptr, nullptr,
                                            result_dev, stream_);
-    if (st != DCT_OK) return st;
+    if (st != DCT_OK) {
+        (void)cudaStreamSynchronize(stream);
+        return st;
+    }
+    // the forward status leaves the device before the backward call reuses the result block
+    DCT_CUDA_TRY(cudaMemcpyAsync(result_host, result_dev, sizeof(dct_result_t), cudaMemcpyDeviceToHost, stream));
     DCT_CUDA_TRY(cudaMemcpyAsync(cols_host, cols_dev, slots * sizeof(int16_t), cudaMemcpyDeviceToHost, stream));
     DCT_CUDA_TRY(cudaMemcpyAsync(vals_host, vals_dev, slots * es, cudaMemcpyDeviceToHost, stream));
     DCT_CUDA_TRY(cudaMemcpyAsync(x_grad_dev, x_grad_host, mat_bytes, cudaMemcpyHostToDevice, stream));
     st = dct_mp_pack_bwd(x_grad_dev, dtype, rows, d, ld, k, cols_dev, gvals_dev, result_dev, stream_);
-    if (st != DCT_OK) return st;
+    if (st != DCT_OK) {
+        (void)cudaStreamSynchronize(stream);
+        return st;
+    }
     DCT_CUDA_TRY(cudaMemcpyAsync(gvals_host, gvals_dev, slots * es, cudaMemcpyDeviceToHost, stream));
-    DCT_CUDA_TRY(cudaMemcpyAsync(result_host, result_dev, sizeof(dct_result_t), cudaMemcpyDeviceToHost, stream));
+    dct_result_t backward;
+    DCT_CUDA_TRY(cudaMemcpyAsync(&backward, result_dev, sizeof(dct_result_t), cudaMemcpyDeviceToHost, stream));
     DCT_CUDA_TRY(cudaStreamSynchronize(stream));
+    if (backward.status > result_host->status) result_host->status = backward.status;   // the worse of the two
     return static_cast<dct_status_t>(result_host->status);
 }
