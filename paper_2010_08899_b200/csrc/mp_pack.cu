@@ -7,7 +7,8 @@
 //     over the row in shared memory (row_select.cuh).
 //   * bf16, sparse k, rows up to 4096 columns on 16-byte boundaries (this file): one warp per row, the
 //     candidates above a bound in registers.
-//   * bf16, dense k (this file): one warp per row, tau_i pinned between two bit tables.
+//   * bf16, denser k (mp_pack_span.cu): one warp per row, every lane looking after a contiguous span of the row,
+//     tau_i pinned between two bounds.
 //   * bf16, rows of 256 / 512 columns: several rows per warp, rows in registers (mp_pack_narrow.cu).
 //   * fp32, sparse k: one warp per row (mp_pack_f32.cu).
 // dct_mp_topk_pack_fwd (end of this file) picks among them.
@@ -113,6 +114,21 @@ __global__ void mp_topk_pack_fwd_kernel(const T* __restrict__ x, uint32_t rows, 
     }
 }
 
+// One element of the gradient matrix through the read-only path without a line in L1: the kept columns of a row
+// touch every 128-byte line about once, so an L1 line is never hit again (the backward pack alone: 24.8 -> 22.6 us
+// at 16384 x 4096 bf16).  What reaches DRAM is the same with every flavour of load: whole 128-byte lines.
+template <typename T> __device__ __forceinline__ T gather_load(const T* p) {
+    if constexpr (sizeof(T) == 2) {
+        uint16_t v;
+        asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p));
+        return *reinterpret_cast<T*>(&v);
+    } else {
+        uint32_t v;
+        asm volatile("ld.global.nc.L1::no_allocate.u32 %0, [%1];" : "=r"(v) : "l"(p));
+        return *reinterpret_cast<T*>(&v);
+    }
+}
+
 // The result block is reset inside the kernel (no memset node, no reset kernel on the stream).  Thread 0 of CTA 0
 // clears it and then publishes the launch's ticket in `reserved` (release); a warp that has met a bad column
 // waits (bounded) for that ticket before it raises the status, so the reset can never wipe a report.
@@ -150,7 +166,7 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
                 const uint32_t s = s0 + u * 32 + lane;
                 const bool ok = c[u] < d;
                 if (s < k && !ok) bad = true;
-                v[u] = (s < k && ok) ? __ldg(gr + c[u]) : T(0);
+                v[u] = (s < k && ok) ? gather_load(gr + c[u]) : T(0);
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
@@ -712,402 +728,6 @@ dct_status_t launch_fwd_bf16_warp(const void* x_act, uint32_t rows, uint32_t d, 
                                                 stream);
 }
 
-// ------------------------------------------------------------------------------------------
-// bf16, dense k (up to a quarter of the row and more): one warp per row
-// ------------------------------------------------------------------------------------------
-// With k in the hundreds or thousands the candidates no longer fit registers, but they need not: tau_i
-// is pinned between two bounds and everything is emitted straight from the candidate bits.
-//   A  `low`: the previous row's tau_i minus a margin (first row of a warp: a quantile of 128 samples of
-//      the row).  One pass over the row builds two bit tables, key >= low and key >= low + 64.  If their
-//      counts n_low, n_high satisfy n_high < k <= n_low, tau_i lies in the 64-key window between them;
-//      otherwise low moves (by 64, 128, ... keys) and the pass is repeated, a few times at most.
-//   B  the elements inside the window (in the low table, not in the high one: a handful per lane) are
-//      read and counted into a 64-bin histogram; a scan over it gives tau_i and the number of ties kept.
-//   C  the kept columns become a third bit table: the high table, plus the window elements above tau_i, plus the
-//      first ties; every table word gets the number of kept entries before it.
-//   D  the k output slots are dealt out evenly, ceil(k / 32) consecutive ones to a lane, which finds the word of
-//      its first slot by bisection over the running counts and walks the kept bits from there; the entries go
-//      through k staging slots to coalesced stores.  (With the columns instead of the slots dealt out evenly the
-//      warp waits for the lane with the most kept columns: 1.4 times the mean for k = 1024 of 4096.)
-// A row for which this fails (tau_i = 0, bounds that do not converge) takes the bit-serial slow path.
-constexpr uint32_t kDenseWindow = 64;
-constexpr uint32_t kDenseMaxK = 1280;                 // staging slots per warp (5 KiB)
-constexpr int kDenseMaxWarps = 32;
-constexpr int kDenseRetries = 6;
-
-template <int E8> struct DenseLayout {
-    using Row = WarpRowLayout<E8>;
-    // per warp: row | low table (128 words) | high table (128 words) | histogram (64 words) | stage (k words) | mbarrier
-    static constexpr uint32_t kTabWords = Row::kTableWords > 128u ? Row::kTableWords : 128u;
-    __host__ __device__ static constexpr uint32_t scratch_words(uint32_t k) { return 2u * kTabWords + 64u + ((k + (k >> 5) + 4u) & ~3u); }
-    __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) { return Row::kRowBytes + scratch_words(k) * 4u + 16u; }
-};
-
-template <int E8>
-__global__ void __launch_bounds__(kDenseMaxWarps * 32)
-mp_topk_fwd_bf16_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
-                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
-                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
-                              dct_result_t* __restrict__ result) {
-    using Lay = WarpRowLayout<E8>;
-    using Den = DenseLayout<E8>;
-    constexpr int kMaskWords = Lay::kMaskWords;
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
-    unsigned char* base = smem_raw + warp * Den::warp_bytes(k);
-    unsigned char* span = base + lane * Lay::kSpanBytes;
-    uint32_t* scratch = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
-    uint32_t* tab_low = scratch;                               // one bit per column: key >= low
-    uint32_t* tab_high = scratch + Den::kTabWords;             // one bit per column: key >= low + window
-    uint32_t* hist = scratch + 2u * Den::kTabWords;
-    uint32_t* stage = hist + 64;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(scratch + Den::scratch_words(k));
-    const uint16_t* row16 = reinterpret_cast<const uint16_t*>(base);
-    __shared__ uint32_t s_stop;
-    __shared__ uint32_t s_next;                               // rows of this CTA handed out so far
-
-    if (threadIdx.x == 0) {
-        s_stop = 0;
-        s_next = blockDim.x >> 5;
-    }
-    if (lane == 0) {
-        mbar_init(bar, 1);
-        mbar_init_fence();
-        fence_proxy_async_all();
-    }
-    const uint32_t row_bytes = d * 2u;                         // the tail of the buffer stays zero (see the sparse kernel)
-    for (uint32_t b = row_bytes + lane * 16u; b < Lay::kRowBytes; b += 512u)
-        *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
-    __syncthreads();
-    chain_wait_previous();                                     // set-up above, inputs and outputs only below (see the sparse kernel)
-    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
-        result->status = DCT_OK;
-        result->reserved = 0;
-        result->count = 0;
-        result->needed = 0;
-        result->n_gt = 0;
-        result->n_eq = 0;
-    }
-
-    const uint32_t warp_global = blockIdx.x + gridDim.x * warp;
-    auto request_row = [&](uint32_t r) {
-        if (lane == 0) {
-            mbar_arrive_expect_tx(bar, row_bytes);
-            bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, bar);
-        }
-    };
-    uint64_t next_row = 0;
-    auto release_row = [&]() {               // the row buffer is no longer needed: request the CTA's next row
-        __syncwarp();
-        fence_proxy_async_smem();
-        uint32_t j = 0;
-        if (lane == 0) j = atomicAdd(&s_next, 1u);
-        j = __shfl_sync(0xFFFFFFFFu, j, 0);
-        next_row = blockIdx.x + static_cast<uint64_t>(gridDim.x) * j;
-        if (next_row < rows) request_row(static_cast<uint32_t>(next_row));
-    };
-    const unsigned char* unit0 = base + lane * 16u;
-    if (warp_global < rows) request_row(warp_global);
-
-    uint32_t use = 0;
-    uint32_t guess_low = 0;
-    // Width of the window in keys.  A wide window rarely misses tau_i, but every element inside it is looked at
-    // one by one, in loops whose length is that of the lane with the most of them (k = 1024 of 4096 post-ReLU
-    // columns: 220 elements in 64 keys, 44 % of the row's time).  The width is halved, down to 16 keys, while a
-    // row finds more than 96 elements in it, and doubled again when a row needs a second pass: a second pass over
-    // the row is cheaper than a crowded window (9 % faster at k = 1024, 11 % at k = 600).
-    uint32_t window = kDenseWindow;
-    // k a multiple of 256 (every lane has a multiple of 8 output slots) and 16-byte aligned outputs: the emit writes
-    // 128-bit words straight to global memory
-    const bool direct = (k & 255u) == 0 && ((reinterpret_cast<uintptr_t>(cols_out) | reinterpret_cast<uintptr_t>(vals_out)) & 15u) == 0 &&
-                        (rows_out == nullptr || (reinterpret_cast<uintptr_t>(rows_out) & 15u) == 0);
-    for (uint64_t row64 = warp_global; row64 < rows; row64 = next_row, ++use) {
-        const uint32_t row = static_cast<uint32_t>(row64);
-        if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(bar, use & 1u, 1u << 24, &s_stop))) {
-            s_stop = 1;
-            if (lane == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
-            return;
-        }
-        const size_t out_base = static_cast<size_t>(row) * k;
-
-        // ---- A: bounds around tau_i ------------------------------------------------------------------
-        uint32_t low = guess_low;
-        if (low == 0) {
-            // no previous row: the (k/d)-quantile of up to 128 samples (element 0 of up to four units of every
-            // lane), taken a little low, found bit by bit
-            constexpr int kSamples = E8 < 4 ? E8 : 4;
-            uint32_t sample[kSamples];
-#pragma unroll
-            for (int c = 0; c < kSamples; ++c) sample[c] = *reinterpret_cast<const uint16_t*>(unit0 + c * 512) & 0x7FFFu;
-            const uint32_t n_samples = 32u * kSamples;
-            uint32_t rank = (n_samples * k + d - 1) / d;                   // expected rank of tau_i among the samples
-            rank += 2u * static_cast<uint32_t>(__fsqrt_rn(static_cast<float>(rank))) + 2u;
-            if (rank > n_samples) rank = n_samples;
-#pragma unroll 1
-            for (int bit = 14; bit >= 0; --bit) {
-                const uint32_t trial = low | (1u << bit);
-                uint32_t cnt = 0;
-#pragma unroll
-                for (int c = 0; c < kSamples; ++c) cnt += sample[c] >= trial ? 1u : 0u;
-                if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= rank) low = trial;
-            }
-            if (low == 0) low = 1;
-        }
-        uint32_t geL[kMaskWords], geH[kMaskWords];
-        uint32_t n_low = 0, n_high = 0;
-        bool pinned = false;
-        uint32_t step = window;
-        bool moved = false;
-        int last_move = 0;
-#pragma unroll 1
-        for (int attempt = 0; attempt < kDenseRetries; ++attempt) {
-            // exact compares (the tables decide what is kept); low <= 0x7F80 keeps low + window within the 2^15 keys
-            const uint32_t high = low + window;
-            unsigned char* tl = reinterpret_cast<unsigned char*>(tab_low) + lane;
-            unsigned char* th = reinterpret_cast<unsigned char*>(tab_high) + lane;
-            __syncwarp();
-#pragma unroll
-            for (int c = 0; c < E8; ++c) {
-                const uint4 v = *reinterpret_cast<const uint4*>(unit0 + c * 512);
-                tl[c * 32] = static_cast<unsigned char>(mask8_ge_exact(v, low));
-                th[c * 32] = static_cast<unsigned char>(mask8_ge_exact(v, high));
-            }
-            __syncwarp();
-            uint32_t mine = 0;
-#pragma unroll
-            for (int i = 0; i < kMaskWords; ++i) {
-                const uint32_t w = lane * kMaskWords + i;
-                const bool real = Lay::kRowWords == Lay::kTableWords || w < Lay::kRowWords;
-                geL[i] = real ? tab_low[w] : 0u;
-                geH[i] = real ? tab_high[w] : 0u;
-                mine += (__popc(geL[i]) << 16) | __popc(geH[i]);
-            }
-            const uint32_t incl = warp_inclusive_sum(mine);        // both counts stay below 2^16
-            const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            n_low = total >> 16;
-            n_high = total & 0xFFFFu;
-            if (n_high < k && k <= n_low) {
-                pinned = true;
-                break;
-            }
-            // move the window: down if too few elements lie above low, up if too many lie above low + window;
-            // the step doubles while the direction stays the same and halves when it turns
-            const int move = n_low < k ? -1 : 1;
-            if (attempt > 0) step = (move == last_move) ? step * 2u : (step > window ? step / 2u : window);
-            moved = true;
-            last_move = move;
-            if (move < 0) {
-                if (low == 1) break;                               // tau_i = 0: fewer than k non-zeros
-                low = low > step ? low - step : 1u;
-            } else {
-                low = low + step < 0x7F80u ? low + step : 0x7F80u;
-            }
-        }
-        if (!pinned) {
-            mp_row_slow_path<E8>(span, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
-            release_row();
-            continue;
-        }
-
-        // ---- B: tau_i from the elements inside the window ----------------------------------------------
-        hist[lane] = 0;
-        hist[lane + 32] = 0;
-        __syncwarp();
-#pragma unroll
-        for (int i = 0; i < kMaskWords; ++i) {
-            uint32_t m = geL[i] & ~geH[i];
-            const uint32_t col0 = (lane * kMaskWords + i) * 32u;
-            while (m) {
-                const uint32_t col = col0 + (__ffs(m) - 1);
-                m &= m - 1;
-                atomicAdd(&hist[((row16[col] & 0x7FFFu) - low) & 63u], 1u);
-            }
-        }
-        __syncwarp();
-        uint32_t tau_key, take;
-        {
-            const uint32_t drop = n_low - k;                       // window elements to discard, smallest first
-            const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];   // lane owns bins 2 lane, 2 lane + 1
-            const uint32_t own = h.x + h.y;
-            const uint32_t before = warp_inclusive_sum(own) - own;
-            uint32_t my_tau = 0, my_take = 0;
-            bool mine = false;
-            if (before <= drop && drop < before + h.x) {
-                mine = true;
-                my_tau = low + 2u * lane;
-                my_take = h.x - (drop - before);
-            } else if (before + h.x <= drop && drop < before + own) {
-                mine = true;
-                my_tau = low + 2u * lane + 1u;
-                my_take = h.y - (drop - before - h.x);
-            }
-            const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);   // exactly one lane: n_high < k <= n_low
-            const int src = who ? __ffs(who) - 1 : 0;
-            tau_key = __shfl_sync(0xFFFFFFFFu, my_tau, src);
-            take = __shfl_sync(0xFFFFFFFFu, my_take, src);
-        }
-        if (lane == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
-        if (moved)
-            window = window < kDenseWindow ? window * 2u : kDenseWindow;
-        else if (n_low - n_high > 96u && window > 16u)
-            window >>= 1;
-        guess_low = tau_key > window / 2u ? tau_key - window / 2u : 1u;
-
-        // ---- C: the kept columns as a bit table -------------------------------------------------------------
-        // everything in the high table, plus the window elements above tau_i, plus the first `take` ties
-        uint32_t keep[kMaskWords];
-        {
-            uint32_t ties[kMaskWords];
-            uint32_t n_ties = 0;
-#pragma unroll
-            for (int i = 0; i < kMaskWords; ++i) {
-                uint32_t m = geL[i] & ~geH[i], gt = 0, eq = 0;
-                const uint32_t col0 = (lane * kMaskWords + i) * 32u;
-                while (m) {
-                    const uint32_t b = __ffs(m) - 1;
-                    m &= m - 1;
-                    const uint32_t key = row16[col0 + b] & 0x7FFFu;
-                    gt |= (key > tau_key ? 1u : 0u) << b;
-                    eq |= (key == tau_key ? 1u : 0u) << b;
-                }
-                keep[i] = geH[i] | gt;
-                ties[i] = eq;
-                n_ties += __popc(eq);
-            }
-            const uint32_t ties_before = warp_inclusive_sum(n_ties) - n_ties;
-            uint32_t room = ties_before < take ? take - ties_before : 0u;   // ties this lane may still keep
-#pragma unroll
-            for (int i = 0; i < kMaskWords; ++i) {
-                uint32_t e = ties[i];
-                const uint32_t n = __popc(e);
-                if (n > room) {
-                    for (uint32_t extra = n - room; extra; --extra) e &= ~(0x80000000u >> __clz(e));   // highest columns go
-                    room = 0;
-                } else {
-                    room -= n;
-                }
-                keep[i] |= e;
-            }
-        }
-        // the two bit tables make room for one entry per word: {kept columns, kept entries before the word}
-        uint2* ktab = reinterpret_cast<uint2*>(tab_low);
-        {
-            uint32_t mine = 0;
-#pragma unroll
-            for (int i = 0; i < kMaskWords; ++i) mine += __popc(keep[i]);
-            uint32_t before = warp_inclusive_sum(mine) - mine;
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < kMaskWords; ++i) {
-                ktab[lane * kMaskWords + i] = make_uint2(keep[i], before);
-                before += __popc(keep[i]);
-            }
-        }
-        __syncwarp();
-
-        // ---- D: ordered emit, evenly -------------------------------------------------------------------------
-        // Lane l produces the output slots l * per .. l * per + per - 1 (per = ceil(k / 32)): it finds the word that
-        // holds its first slot by bisection over the running counts and walks the kept bits from there.  The entries
-        // pass through a staging area (slot p at word p + p / 32: neither the lanes' writes, 32 slots apart, nor the
-        // coalesced reads meet in a bank).
-        {
-            const uint32_t per = (k + 31u) >> 5;
-            const uint32_t first = lane * per;
-            const uint32_t nvalid = first >= k ? 0u : (k - first < per ? k - first : per);
-            if (nvalid) {
-                uint32_t lo = 0, hi = Lay::kTableWords - 1;           // largest word with (entries before it) <= first
-                while (lo < hi) {
-                    const uint32_t mid = (lo + hi + 1) >> 1;
-                    if (ktab[mid].y <= first) lo = mid; else hi = mid - 1;
-                }
-                const uint2 e = ktab[lo];
-                uint32_t word = lo, m = e.x;
-                for (uint32_t skip = first - e.y; skip; --skip) m &= m - 1;
-                // `ahead` is the next word's bits, fetched when the walk arrives at a word; eight columns are found
-                // first, then their values are read together and staged
-                uint32_t ahead = word + 1 < Lay::kTableWords ? ktab[word + 1].x : 0u;
-                for (uint32_t j0 = 0; j0 < nvalid; j0 += 8) {
-                    uint32_t col[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        if (m == 0) {
-                            m = ahead;
-                            ++word;
-                            while (m == 0) m = ktab[++word].x;     // an empty word (ends: kept bits lie ahead)
-                            ahead = word + 1 < Lay::kTableWords ? ktab[word + 1].x : 0u;
-                        }
-                        col[u] = word * 32u + (__ffs(m) - 1);
-                        if (j0 + u + 1 < nvalid) m &= m - 1;       // the last slot's bit stays: m != 0 or none is needed
-                    }
-                    uint32_t v[8];
-#pragma unroll
-                    for (int u = 0; u < 8; ++u) v[u] = row16[col[u]];
-                    if (direct) {
-                        // eight consecutive slots of this lane are 16 aligned bytes of either output: no staging
-                        const size_t at = out_base + first + j0;
-                        *reinterpret_cast<uint4*>(cols_out + at) = make_uint4(col[0] | (col[1] << 16), col[2] | (col[3] << 16),
-                                                                              col[4] | (col[5] << 16), col[6] | (col[7] << 16));
-                        *reinterpret_cast<uint4*>(vals_out + at) = make_uint4(v[0] | (v[1] << 16), v[2] | (v[3] << 16),
-                                                                              v[4] | (v[5] << 16), v[6] | (v[7] << 16));
-                        if (rows_out) {
-                            const uint4 r4 = make_uint4(row, row, row, row);
-                            reinterpret_cast<uint4*>(rows_out + at)[0] = r4;
-                            reinterpret_cast<uint4*>(rows_out + at)[1] = r4;
-                        }
-                    } else {
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) {
-                            const uint32_t p = first + j0 + u;
-                            if (j0 + u < nvalid) stage[p + (p >> 5)] = v[u] | (col[u] << 16);
-                        }
-                    }
-                }
-            }
-        }
-        release_row();
-        if (!direct) {
-            for (uint32_t p = lane; p < k; p += 32) {
-                const uint32_t e = stage[p + (p >> 5)];
-                cols_out[out_base + p] = static_cast<int16_t>(e >> 16);
-                vals_out[out_base + p] = static_cast<uint16_t>(e & 0xFFFFu);
-                if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
-            }
-        }
-        __syncwarp();
-    }
-    chain_release_next();                                      // no row left for this warp (see the sparse kernel)
-}
-
-template <int E8>
-dct_status_t launch_fwd_bf16_dense(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
-                                   void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
-                                   cudaStream_t stream) {
-    using Den = DenseLayout<E8>;
-    auto kernel = mp_topk_fwd_bf16_dense_kernel<E8>;
-    constexpr size_t kSmemBudget = 220 * 1024;
-    static thread_local int configured_device = -1;
-    int dev = 0;
-    DCT_CUDA_TRY(cudaGetDevice(&dev));
-    if (configured_device != dev) {
-        DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          static_cast<int>(kSmemBudget)));
-        configured_device = dev;
-    }
-    const size_t per_warp = Den::warp_bytes(k);
-    size_t warps = kSmemBudget / per_warp;
-    if (warps > static_cast<size_t>(kDenseMaxWarps)) warps = kDenseMaxWarps;
-    if (warps < 1) return DCT_ERR_UNSUPPORTED;
-    const int sms = sm_count();
-    if (sms <= 0) return DCT_ERR_CUDA;
-    warps = warps_for_rows(warps, rows, sms);
-    const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + warps - 1) / warps;
-    const uint32_t grid = static_cast<uint32_t>(ctas_needed < static_cast<uint64_t>(sms) ? ctas_needed : sms);
-    DCT_CUDA_TRY(launch_chained_smem(kernel, grid, static_cast<unsigned>(warps * 32), warps * per_warp, stream,
-                                     static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out,
-                                     static_cast<uint16_t*>(vals_out), rows_out, static_cast<uint16_t*>(tau_out), result));
-    return DCT_OK;
-}
-
 int fwd_threads_for(uint32_t d) {
     if (d <= 4096) return 128;
     if (d <= 8192) return 256;
@@ -1216,20 +836,13 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
         DCT_BF16_WIDTH(32);
 #undef DCT_BF16_WIDTH
     }
-    // dense k (beyond the candidate registers of the kernels above, up to half the row): bounds + bit tables
-    if (aligned_to(x_act, 16) && (static_cast<size_t>(ld) * 2) % 16 == 0 && d % 8 == 0 && d <= 8192 && k <= kDenseMaxK &&
-        k <= d / 2) {
-#define DCT_BF16_DENSE(E8) \
-    if (d <= 256u * E8)    \
-        return launch_fwd_bf16_dense<E8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
-        DCT_BF16_DENSE(1);
-        DCT_BF16_DENSE(2);
-        DCT_BF16_DENSE(4);
-        DCT_BF16_DENSE(8);
-        DCT_BF16_DENSE(12);
-        DCT_BF16_DENSE(16);
-        DCT_BF16_DENSE(32);
-#undef DCT_BF16_DENSE
+    // denser k (beyond the candidate registers of the kernels above, up to 3/8 of the row): every lane looks after
+    // one contiguous span of the row (mp_pack_span.cu)
+    {
+        bool handled = false;
+        const dct_status_t span = launch_fwd_bf16_span(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
+                                                       result, stream, &handled);
+        if (span != DCT_OK || handled) return span;
     }
     return launch_fwd<uint16_t>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
 }

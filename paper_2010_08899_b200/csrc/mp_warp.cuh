@@ -207,6 +207,11 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
                                     int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                     dct_result_t* result, cudaStream_t stream, bool* handled);
 
+// bf16, every lane looking after one contiguous span of the row (mp_pack_span.cu).
+dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                  int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                  dct_result_t* result, cudaStream_t stream, bool* handled);
+
 // The fp32 kernels live in their own translation unit.
 dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                  int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,

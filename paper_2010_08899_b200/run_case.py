@@ -35,11 +35,26 @@ def main():
     ap.add_argument("--dist", choices=["mixture", "gaussian", "dlrm"], default="mixture")
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
+    ap.add_argument("--l2-fetch", type=int, default=0, choices=[0, 32, 64, 128],
+                    help="set this process's cudaLimitMaxL2FetchGranularity hint (bytes) before anything runs")
     ap.add_argument("--back-to-back", action="store_true",
                     help="time all iterations between one pair of events (launch gaps overlap, as in a training loop)")
     args = ap.parse_args()
 
     dev = "cuda"
+    if args.l2_fetch:
+        # a hint of this process's CUDA context (it dies with the process; no setting of the GPU changes)
+        import ctypes
+        import glob
+        import os
+        torch.cuda.init()
+        torch.zeros(1, device=dev)                                            # the primary context exists
+        found = glob.glob(os.path.join(os.path.dirname(torch.__file__), "..", "nvidia", "cuda_runtime", "lib", "libcudart.so*"))
+        rt = ctypes.CDLL(found[0] if found else "libcudart.so")
+        rc = rt.cudaDeviceSetLimit(5, ctypes.c_size_t(args.l2_fetch))         # 5 = cudaLimitMaxL2FetchGranularity
+        got = ctypes.c_size_t(0)
+        rt.cudaDeviceGetLimit(ctypes.byref(got), 5)
+        print(f"cudaLimitMaxL2FetchGranularity <- {args.l2_fetch} B: return code {rc}, now {got.value} B")
     stream = torch.cuda.current_stream()
     reset = lambda: None
     gen = {"mixture": inputs.dp_mixture, "gaussian": inputs.dp_gaussian, "dlrm": inputs.dp_dlrm_like}[args.dist]

@@ -220,9 +220,10 @@ def test_mp_warp_per_row_widths_between_the_buffer_sizes(dtype, d):
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("d", [512, 1024, 2000, 4096])
 def test_mp_dense_k(dtype, d):
-    """k from a quarter to half of the row (75 % sparsity and below): tau_i is pinned between two bit tables
-    64 keys apart.  Rows whose scale jumps by orders of magnitude make the window move several times;
-    ties, dead rows and rows with fewer than k non-zeros take the remaining branches."""
+    """k from a quarter to half of the row (75 % sparsity and below): up to 3/8 of the row tau_i is pinned between
+    two bounds at most 64 keys apart (beyond, the general kernel serves).  Rows whose scale jumps by orders of
+    magnitude make the window move several times; ties, dead rows and rows with fewer than k non-zeros (tau_i = 0:
+    the first zeros fill the row's slots) take the remaining branches."""
     rows = 2500
     x = inputs.mp_activations(rows, d, 51 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=52 + d)
     sign = torch.where(inputs.dp_gaussian(rows * d, 53 + d, G.DEV).view(rows, d) > 0, 1.0, -1.0)
@@ -241,10 +242,10 @@ def test_mp_dense_k(dtype, d):
 
 @pytest.mark.parametrize("d", [1024, 4096])
 def test_mp_dense_k_clustered_columns_and_many_ties(d):
-    """The dense bf16 kernel deals the k output slots out evenly and walks a bit table of the kept columns: rows whose
-    kept columns sit in one part of the row (long runs of empty table words before, between and after them), rows
-    of a few distinct values (every row has many ties at tau_i, spread over the lanes, of which only some are
-    kept), and k that is not a multiple of 32."""
+    """In the bf16 kernel for denser k every lane walks the kept bits of its own span of the row: rows whose kept
+    columns sit in one part of the row (some lanes hold nearly everything, others nothing), rows of a few distinct
+    values (every row has many ties at tau_i, spread over the lanes, of which only some are kept; windows that
+    have to be narrowed), and k that is not a multiple of 32."""
     rows = 900
     x = inputs.mp_activations(rows, d, 71 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=72 + d)
     third = d // 3
@@ -262,9 +263,9 @@ def test_mp_dense_k_clustered_columns_and_many_ties(d):
 
 @pytest.mark.parametrize("d,k", [(1024, 256), (2048, 512), (4096, 1024), (4096, 1280)])
 def test_mp_dense_k_multiple_of_256_writes_whole_words(d, k):
-    """With k a multiple of 256 and 16-byte aligned outputs the dense bf16 kernel writes 128-bit words straight
-    from the emit (cols, vals and the optional row ids); with an output that starts 2 bytes off it must fall back to
-    the staged stores.  Both give the oracle's result, and neither writes outside its rows * k slots."""
+    """With 4-byte aligned outputs the bf16 kernel for denser k stores its staged entries in pairs (4-byte words of
+    either output, plus the optional row ids); an output that starts 2 bytes off goes to the general kernel.  Both
+    give the oracle's result, and neither writes outside its rows * k slots."""
     rows = 333
     x = inputs.mp_activations(rows, d, 81 + d, dtype=torch.bfloat16, device=G.DEV, col_scale_seed=82 + d)
     x[5] = 0.5                                       # every element ties: the first k columns win
