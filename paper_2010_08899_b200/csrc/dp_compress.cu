@@ -378,11 +378,12 @@ __device__ __forceinline__ void compress_tile_body(const float* __restrict__ gra
             s_excl[1] = excl_eq;
         }
     }
-    if (cta_tot == 0) return;                  // nothing flagged in this tile: no output, no rewrite
-    __syncthreads();
-    if (warp_tot == 0) return;
-    emit_warp(w, gt_mask, eq_mask, warp_base, before_warp, s_excl[0], s_excl[1], budget, capacity, s_abort != 0,
-              idx_out, val_out, residual);
+    if (cta_tot != 0) {                        // (nothing flagged in this tile: no output, no rewrite)
+        __syncthreads();
+        if (warp_tot != 0)
+            emit_warp(w, gt_mask, eq_mask, warp_base, before_warp, s_excl[0], s_excl[1], budget, capacity, s_abort != 0,
+                      idx_out, val_out, residual);
+    }
 }
 
 template <bool kVectorised>
@@ -395,12 +396,18 @@ dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ resi
                         uint32_t spin_limit, const uint32_t* __restrict__ enabled = nullptr) {
     __shared__ uint32_t s_tile;
     if (enabled && *enabled == 0) return;     // a conditional call that is not needed
-    if (threadIdx.x == 0) s_tile = fixed_tile != kInvalidTile ? fixed_tile : atomicAdd(&ctrl->ticket, 1u);
-    __syncthreads();
-    const uint32_t tile = s_tile;
-    if (tile >= num_tiles) return;            // only reachable with a testing ticket offset
-    compress_tile_body<kVectorised>(grad, residual, n, tau_p, budget_p, idx_out, val_out, capacity, result, ctrl,
-                                    tile_state, num_tiles, tile, spin_limit);
+    // A CTA works through tickets until none is left (the grid need not be as large as the number of tiles).  Tiles
+    // are only taken by running CTAs and in order, so the oldest unfinished tile never waits for one not yet taken.
+    for (;;) {
+        if (threadIdx.x == 0) s_tile = fixed_tile != kInvalidTile ? fixed_tile : atomicAdd(&ctrl->ticket, 1u);
+        __syncthreads();
+        const uint32_t tile = s_tile;
+        if (tile >= num_tiles) return;
+        compress_tile_body<kVectorised>(grad, residual, n, tau_p, budget_p, idx_out, val_out, capacity, result, ctrl,
+                                        tile_state, num_tiles, tile, spin_limit);
+        if (fixed_tile != kInvalidTile) return;
+        __syncthreads();                      // the tile's shared-memory words are free for the next one
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -821,7 +828,10 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
     DCT_CUDA_TRY(cudaGetLastError());
     const bool vec = aligned_to(grad, 16) && aligned_to(residual, 16);
     if (!vec) {
-        dp_compress_tile_kernel<false><<<num_tiles, kThreads, 0, stream>>>(
+        const int sms_t = sm_count();
+        if (sms_t <= 0) return DCT_ERR_CUDA;
+        const uint32_t tile_grid = num_tiles < static_cast<uint32_t>(sms_t) * 8u ? num_tiles : static_cast<uint32_t>(sms_t) * 8u;
+        dp_compress_tile_kernel<false><<<tile_grid, kThreads, 0, stream>>>(
             grad, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
             kInvalidTile, dbg.spin_limit);
         DCT_CUDA_TRY(cudaGetLastError());
@@ -884,12 +894,15 @@ dct_status_t dct::compress_presummed_if(const uint32_t* enabled, float* residual
     dp_compress_init_kernel<<<(num_tiles + 1023) / 1024, 1024, 0, stream>>>(ctrl, tile_state, num_tiles, result, 0u,
                                                                             enabled);
     DCT_CUDA_TRY(cudaGetLastError());
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint32_t tile_grid = num_tiles < static_cast<uint32_t>(sms) * 8u ? num_tiles : static_cast<uint32_t>(sms) * 8u;
     if (aligned_to(residual, 16))
-        dp_compress_tile_kernel<true><<<num_tiles, kThreads, 0, stream>>>(
+        dp_compress_tile_kernel<true><<<tile_grid, kThreads, 0, stream>>>(
             nullptr, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
             kInvalidTile, dbg.spin_limit, enabled);
     else
-        dp_compress_tile_kernel<false><<<num_tiles, kThreads, 0, stream>>>(
+        dp_compress_tile_kernel<false><<<tile_grid, kThreads, 0, stream>>>(
             nullptr, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
             kInvalidTile, dbg.spin_limit, enabled);
     DCT_CUDA_TRY(cudaGetLastError());

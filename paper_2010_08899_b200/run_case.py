@@ -6,6 +6,7 @@ A small command-line driver for profiling and quick timing of a single kernel at
     python -m paper_2010_08899_b200.run_case select   --n 268435456 --k 26844
     python -m paper_2010_08899_b200.run_case mp_fwd   --rows 16384 --d 4096 --k 205 --dtype bf16
     python -m paper_2010_08899_b200.run_case mp_bwd   --rows 16384 --d 4096 --k 205 --dtype bf16
+    python -m paper_2010_08899_b200.run_case select_compress --n 268435456   (threshold life-span L = 1)
     python -m paper_2010_08899_b200.run_case decompress --n 268435456
     python -m paper_2010_08899_b200.run_case mp_unpack --rows 16384 --d 4096 --k 205 --dtype bf16
     python -m paper_2010_08899_b200.run_case select_multi --n 268435456          (75 / 90 / 95 % sparsity)
@@ -25,7 +26,7 @@ from . import inputs
 
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
-    ap.add_argument("entry", choices=["select", "compress", "compress_layers", "decompress", "mp_fwd", "mp_bwd", "mp_unpack",
+    ap.add_argument("entry", choices=["select", "compress", "select_compress", "compress_layers", "decompress", "mp_fwd", "mp_bwd", "mp_unpack",
                                      "select_multi", "threshold_mean"])
     ap.add_argument("--n", type=int, default=1 << 28)
     ap.add_argument("--k", type=int, default=0, help="survivor target (default: 0.01 %% of n, or 5 %% of d)")
@@ -141,6 +142,19 @@ def main():
         tau_rows = torch.zeros(len(ks) * rows, dtype=dt, device=dev)
         call = lambda i: B.dct_mp_threshold_mean(x[i % 2], rows, d, d, ks, mean, tau_rows)
         nbytes = rows * d * es
+    elif args.entry == "select_compress":
+        # select and compress the same vector every iteration (exactly k survivors); the error carries over
+        n = args.n
+        k = args.k or B.k_from_density(n, 1, 10_000)
+        g = [gen(n, 501 + j, dev) for j in range(2)]
+        e = torch.zeros(n, device=dev)
+        cap = max(n // 64, 1024)
+        idx = torch.empty(cap, dtype=torch.int32, device=dev)
+        val = torch.empty(cap, device=dev)
+        tau, res = torch.zeros(1, device=dev), B.new_result()
+        ws = B.new_workspace(B.dct_dp_select_compress_workspace_bytes(n), dev)
+        call = lambda i: B.dct_dp_select_compress(g[i % 2], e, n, k, tau, idx, val, cap, res, ws)
+        nbytes = 12 * n
     elif args.entry in ("select", "compress", "decompress"):
         n = args.n
         k = args.k or B.k_from_density(n, 1, 10_000)
