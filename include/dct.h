@@ -175,9 +175,12 @@ DCT_API dct_status_t dct_dp_compress(
  * multiple of 16); other layouts are accepted and take a slower scalar load.
  * Every shape gives the same result; the time does depend on it.  Rows on
  * 16-byte boundaries with d*size a multiple of 16 are packed by one warp per
- * row (bf16: d <= 8192, any k up to d/2 and 1280; fp32: d <= 4096, k up to
- * about d/10 and 441, denser k for d <= 2048); everything else (wider rows, denser k, odd strides) takes a general
- * kernel that is several times slower.  status may also be DCT_ERR_TIMEOUT if a
+ * row (bf16: d <= 8192, k up to 3d/8 and 2048; fp32: d <= 4096, k up to
+ * about d/10 and 441, denser k for d <= 2048) or, bf16 rows of 8193..32768
+ * columns with k up to 3d/8 and 2300, by one CTA per row; everything else
+ * (wider fp32 rows, denser k, odd strides, outputs that are not 4-byte
+ * aligned for the denser bf16 cases) takes a general kernel that is several
+ * times slower.  status may also be DCT_ERR_TIMEOUT if a
  * bounded wait for an asynchronous copy gave up (not seen in practice; the
  * outputs are then incomplete).
  */

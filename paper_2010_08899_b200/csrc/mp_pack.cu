@@ -245,7 +245,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     constexpr uint32_t kPerLane = PL, kRound = 32u * kPerLane;   // candidates a lane holds in registers at a time
     constexpr bool kFineLeaves = FwdVariant<PL>::kFineLeaves;
     constexpr int kLeaves = kFineLeaves ? 2 * E8 : E8;           // leaves per lane (4 or 8 elements each)
-    constexpr uint32_t kGuessMargin = 32;                         // keys (a quarter of a binade) below the previous tau_i
+    constexpr uint32_t kGuessMargin = 32;  // keys (a quarter of a binade) below the previous tau_i
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
     unsigned char* base = smem_raw + warp * Lay::warp_bytes(k);

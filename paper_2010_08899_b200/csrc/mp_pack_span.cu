@@ -481,12 +481,442 @@ dct_status_t launch_span(const void* x_act, uint32_t rows, uint32_t d, uint32_t 
     return DCT_OK;
 }
 
+
+// ------------------------------------------------------------------------------------------
+// rows of more than 8192 columns (up to 32768): W warps per row, one row per CTA at a time
+// ------------------------------------------------------------------------------------------
+// The same steps as above with a CTA in the place of the warp: warp w looks after the columns [4096 w, 4096 w + 4096)
+// of the row (lane l of it after 128 of them), counts and offsets are summed over the warps through shared memory, and
+// the histogram of the window elements is the CTA's.  Several CTAs share an SM, so one CTA's load overlaps another's
+// work.  A row whose window does not settle is not handed to another routine: its threshold is found bit by bit
+// (15 counting passes) and the row is then packed with a window of one key, whose elements -- all ties at tau_i --
+// are taken as bits in column order, without lists.
+constexpr uint32_t kWideListLen = 8;              // window elements a lane can take
+constexpr uint32_t kWideListStride = 9;
+constexpr uint32_t kWideMaxK = 2300;
+constexpr int kWideRetries = 6;
+
+template <int W> struct WideLayout {
+    static constexpr uint32_t kSegBytes = 8192u;             // one warp's 4096 columns
+    static constexpr uint32_t kRowBytes = W * kSegBytes;
+    static constexpr uint32_t kHistBytes = 512u;
+    static constexpr uint32_t kListBytes = W * 32u * kWideListStride * 4u;
+    __host__ __device__ static constexpr uint32_t cta_bytes(uint32_t k) {
+        const uint32_t stage = (4u * (k + 2u) + 15u) & ~15u;
+        return (kRowBytes + kHistBytes + (kListBytes > stage ? kListBytes : stage) + 127u) & ~127u;
+    }
+};
+
+template <int W>
+__global__ void __launch_bounds__(W * 32)
+mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                             int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
+                             int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
+                             dct_result_t* __restrict__ result) {
+    using Lay = WideLayout<W>;
+    constexpr int kWords = 4;                                  // 128 columns per lane
+    constexpr uint32_t kLaneCols = 128u;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    unsigned char* base = smem_raw;
+    const unsigned char* own = base + warp * Lay::kSegBytes + lane * 256u;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
+    uint32_t* lists = hist + Lay::kHistBytes / 4;
+    uint32_t* stage = lists;
+    __shared__ uint64_t s_bar;
+    __shared__ uint32_t s_stop;
+    __shared__ uint32_t s_cnt[2][W];                           // per-warp packed counts (double-buffered across passes)
+    __shared__ uint32_t s_max[2][W];
+    __shared__ uint32_t s_sum[2][W];                           // per-warp totals for the two prefix sums of a row
+    __shared__ uint32_t s_guess;
+
+    if (threadIdx.x == 0) {
+        s_stop = 0;
+        mbar_init(&s_bar, 1);
+        mbar_init_fence();
+        fence_proxy_async_all();
+    }
+    const uint32_t row_bytes = d * 2u;                         // the tail of the buffer stays zero
+    for (uint32_t b = row_bytes + threadIdx.x * 16u; b < Lay::kRowBytes; b += W * 512u)
+        *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+    const uint32_t swz = lane & 7u;
+    const uint32_t fix_sel = 0x3210u ^ (0x1111u * (swz & 3u));
+    uint32_t unit_base[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) unit_base[c] = smem_addr(own) ^ (16u * (swz ^ static_cast<uint32_t>(c)));
+    const uint32_t row_addr = smem_addr(base);
+    const uint32_t col0 = warp * 4096u + lane * kLaneCols;     // first column of the lane's span
+
+    auto request_row = [&](uint64_t r) {
+        if (threadIdx.x == 0) {
+            fence_proxy_async_smem();
+            mbar_arrive_expect_tx(&s_bar, row_bytes);
+            bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, &s_bar);
+        }
+    };
+    // sum of one packed word per warp over the CTA (and optionally the part before this warp)
+    auto cta_sum = [&](uint32_t (*slot)[W], uint32_t parity, uint32_t warp_total, uint32_t& before) -> uint32_t {
+        if (lane == 0) slot[parity][warp] = warp_total;
+        __syncthreads();
+        uint32_t total = 0;
+        before = 0;
+#pragma unroll
+        for (int w = 0; w < W; ++w) {
+            const uint32_t t = slot[parity][w];
+            total += t;
+            before += static_cast<uint32_t>(w) < warp ? t : 0u;
+        }
+        return total;
+    };
+
+    // both flag sets of the lane's span for the bounds (low, high); returns the lane's packed counts
+    uint32_t ge_low[kWords], ge_high[kWords];
+    auto flag_pass = [&](uint32_t low, uint32_t high) -> uint32_t {
+        const uint32_t low2 = low * 0x10001u, high2 = high * 0x10001u;
+#pragma unroll
+        for (int i = 0; i < kWords; ++i) ge_low[i] = ge_high[i] = 0;
+        static_for<16>([&](auto c_tag) {
+            constexpr int c = decltype(c_tag)::value;
+            uint32_t f_low, f_high;
+            flags8_two(lds128<128 * (c / 8)>(unit_base[c % 8]), low2, high2, f_low, f_high);
+            constexpr uint32_t sel = c % 4 == 1 ? 0x3410u : (c % 4 == 2 ? 0x3240u : 0x3214u);
+            ge_low[c / 4] = (c % 4 == 0) ? (f_low << 24) : prmt(ge_low[c / 4], f_low, sel);
+            ge_high[c / 4] = (c % 4 == 0) ? (f_high << 24) : prmt(ge_high[c / 4], f_high, sel);
+        });
+#pragma unroll
+        for (int h = 0; h < kWords; h += 2) {
+            const uint32_t l0 = ge_low[h], l1 = ge_low[h + 1], h0 = ge_high[h], h1 = ge_high[h + 1];
+            ge_low[h] = (swz & 4u) ? l1 : l0;
+            ge_low[h + 1] = (swz & 4u) ? l0 : l1;
+            ge_high[h] = (swz & 4u) ? h1 : h0;
+            ge_high[h + 1] = (swz & 4u) ? h0 : h1;
+        }
+        uint32_t mine = 0;
+#pragma unroll
+        for (int i = 0; i < kWords; ++i) {
+            ge_low[i] = prmt(ge_low[i], 0u, fix_sel);
+            ge_high[i] = prmt(ge_high[i], 0u, fix_sel);
+            mine += (__popc(ge_low[i]) << 16) | __popc(ge_high[i]);
+        }
+        return mine;
+    };
+
+    if (blockIdx.x < rows) request_row(blockIdx.x);
+    uint32_t use = 0, pass_no = 0;
+    uint32_t guess_low = 0;
+    uint32_t window = kSpanWindow;
+    for (uint64_t row64 = blockIdx.x; row64 < rows; row64 += gridDim.x, ++use) {
+        const uint32_t row = static_cast<uint32_t>(row64);
+        if (!__syncthreads_and(mbar_wait_bounded(&s_bar, use & 1u, 1u << 24, &s_stop) ? 1 : 0)) {
+            s_stop = 1;
+            if (threadIdx.x == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
+            return;
+        }
+        const size_t out_base = static_cast<size_t>(row) * k;
+
+        // ---- A: bounds around tau_i ------------------------------------------------------------------
+        uint32_t low = guess_low;
+        if (low == 0) {
+            // the (k/d)-quantile of 128 samples of the first warp's columns, taken a little low, found bit by bit
+            if (warp == 0) {
+                uint32_t sample[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) sample[c] = *reinterpret_cast<const uint16_t*>(own + c * 16) & 0x7FFFu;
+                uint32_t rank = (128u * k + d - 1) / d;
+                rank += 2u * static_cast<uint32_t>(__fsqrt_rn(static_cast<float>(rank))) + 2u;
+                if (rank > 128u) rank = 128u;
+                uint32_t q = 0;
+#pragma unroll 1
+                for (int bit = 14; bit >= 0; --bit) {
+                    const uint32_t trial = q | (1u << bit);
+                    uint32_t cnt = 0;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) cnt += sample[c] >= trial ? 1u : 0u;
+                    if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= rank) q = trial;
+                }
+                if (lane == 0) s_guess = q ? q : 1u;
+            }
+            __syncthreads();
+            low = s_guess;
+        }
+        if (low > 0x7F80u) low = 0x7F80u;
+
+        // ---- B: the window ---------------------------------------------------------------------------
+        uint32_t n_low = 0, n_high = 0;
+        bool pinned = false, moved = false, crowded = false;
+        uint32_t width = window;                                // of the window that is finally used (1: exact mode)
+#pragma unroll 1
+        for (int attempt = 0; attempt < kWideRetries; ++attempt) {
+            const uint32_t mine = flag_pass(low, low + window);
+            uint32_t before;
+            const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, mine), before);
+            const uint32_t in_window = (mine >> 16) - (mine & 0xFFFFu);
+            const uint32_t warp_max = __reduce_max_sync(0xFFFFFFFFu, in_window);
+            if (lane == 0) s_max[pass_no & 1u][warp] = warp_max;   // (read after the next barrier only if needed)
+            ++pass_no;
+            n_low = total >> 16;
+            n_high = total & 0xFFFFu;
+            if (n_high < k && k <= n_low) {
+                __syncthreads();
+                uint32_t cta_max = 0;
+#pragma unroll
+                for (int w = 0; w < W; ++w) cta_max = max(cta_max, s_max[(pass_no - 1u) & 1u][w]);
+                if (cta_max <= kWideListLen) {
+                    pinned = true;
+                    width = window;
+                    break;
+                }
+                if (window <= 4u) break;
+                window >>= 1;
+                crowded = true;
+                continue;
+            }
+            const uint32_t per_key_x16 = max(((n_low - n_high) << 4) / window, 4u);
+            moved = true;
+            if (n_low < k) {
+                if (low == 1) break;                               // tau_i = 0
+                const uint32_t below = max(((k - n_low) << 4) / per_key_x16 + window / 2u, window / 2u);
+                low = low > below ? low - below : 1u;
+            } else {
+                const uint32_t above = ((n_high - k + 1u) << 4) / per_key_x16 + window / 2u;
+                low = low + above < 0x7F80u ? low + above : 0x7F80u;
+            }
+        }
+        uint32_t tau_key = 0, take = 0;
+        if (!pinned) {
+            // exact mode: the largest v with #{key >= v} >= k, bit by bit; then a window of one key at it
+            uint32_t v = 0;
+#pragma unroll 1
+            for (int bit = 14; bit >= 0; --bit) {
+                const uint32_t trial = v | (1u << bit);
+                const uint32_t mine = flag_pass(trial, trial);
+                uint32_t before;
+                const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, mine), before);
+                ++pass_no;
+                if ((total >> 16) >= k) v = trial;
+            }
+            tau_key = v;
+            const uint32_t mine = flag_pass(v, v + 1u);          // v = 0: every column, the padding included, is >= 0
+            uint32_t before;
+            const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, mine), before);
+            ++pass_no;
+            n_low = total >> 16;
+            n_high = total & 0xFFFFu;
+            take = k - n_high;
+            width = 1;
+            guess_low = 0;
+        }
+
+        // ---- C: tau_i and the kept columns as bits --------------------------------------------------------
+        uint32_t keep[kWords];
+        if (width == 1) {
+            // every window element ties at tau_i: the first `take` of them, in column order, are kept
+            uint32_t ties[kWords], n_ties = 0;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                ties[i] = ge_low[i] & ~ge_high[i];
+                n_ties += __popc(ties[i]);
+            }
+            const uint32_t incl = warp_inclusive_sum(n_ties);
+            uint32_t warps_before;
+            cta_sum(s_sum, 0, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
+            const uint32_t ties_before = warps_before + incl - n_ties;
+            uint32_t room = ties_before < take ? take - ties_before : 0u;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t z = ties[i];
+                const uint32_t n = __popc(z);
+                if (n > room) {
+                    for (uint32_t extra = n - room; extra; --extra) z &= z - 1u;   // the highest columns go (lowest bits)
+                    room = 0;
+                } else {
+                    room -= n;
+                }
+                keep[i] = ge_high[i] | z;
+            }
+        } else {
+            if (threadIdx.x < 64) hist[threadIdx.x] = 0;
+            __syncthreads();
+            uint32_t* my_list = lists + threadIdx.x * kWideListStride;
+            uint32_t n_list = 0;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t m = ge_low[i] & ~ge_high[i];
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    const uint32_t col = col0 + 32u * i + 31u - q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 2u * col));
+                    const uint32_t key = v & 0x7FFFu;
+                    atomicAdd(&hist[key - low], 1u);
+                    my_list[n_list++] = ((32u * i + q) << 16) | key;
+                }
+            }
+            __syncthreads();
+            {
+                const uint32_t drop = n_low - k;
+                const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];
+                const uint32_t own_cnt = h.x + h.y;
+                const uint32_t before = warp_inclusive_sum(own_cnt) - own_cnt;
+                uint32_t my_tau = 0, my_take = 0;
+                bool mine = false;
+                if (before <= drop && drop < before + h.x) {
+                    mine = true;
+                    my_tau = low + 2u * lane;
+                    my_take = h.x - (drop - before);
+                } else if (before + h.x <= drop && drop < before + own_cnt) {
+                    mine = true;
+                    my_tau = low + 2u * lane + 1u;
+                    my_take = h.y - (drop - before - h.x);
+                }
+                const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
+                const int src = who ? __ffs(who) - 1 : 0;
+                tau_key = __shfl_sync(0xFFFFFFFFu, my_tau, src);
+                take = __shfl_sync(0xFFFFFFFFu, my_take, src);
+            }
+            if (crowded) {
+            } else if (moved) {
+                window = window < kSpanWindow ? window * 2u : kSpanWindow;
+            } else if (n_low - n_high > 64u * W && window > 16u) {
+                window >>= 1;
+            }
+            guess_low = tau_key > window / 2u ? tau_key - window / 2u : 1u;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) keep[i] = ge_high[i];
+            uint32_t n_ties = 0;
+            for (uint32_t j = 0; j < n_list; ++j) n_ties += (my_list[j] & 0xFFFFu) == tau_key ? 1u : 0u;
+            const uint32_t incl = warp_inclusive_sum(n_ties);
+            uint32_t warps_before;
+            cta_sum(s_sum, 0, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
+            const uint32_t ties_before = warps_before + incl - n_ties;
+            uint32_t room = ties_before < take ? take - ties_before : 0u;
+            for (uint32_t j = 0; j < n_list; ++j) {
+                const uint32_t e = my_list[j];
+                const uint32_t key = e & 0xFFFFu;
+                bool add = key > tau_key;
+                if (key == tau_key && room > 0u) {
+                    add = true;
+                    --room;
+                }
+                const uint32_t bit = add ? 1u << ((e >> 16) & 31u) : 0u;
+                const uint32_t word = e >> 21;
+#pragma unroll
+                for (int i = 0; i < kWords; ++i) keep[i] |= word == static_cast<uint32_t>(i) ? bit : 0u;
+            }
+        }
+        if (threadIdx.x == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+
+        // ---- D: every lane stages its kept entries at its offset of the row's output ----------------------------
+        const uint32_t shift = static_cast<uint32_t>(out_base) & 1u;
+        {
+            uint32_t kept_mine = 0;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) kept_mine += __popc(keep[i]);
+            const uint32_t incl = warp_inclusive_sum(kept_mine);
+            uint32_t warps_before;
+            cta_sum(s_sum, 1, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);   // (the barrier inside: all lists are read)
+            uint32_t at = smem_addr(stage) + 4u * (shift + warps_before + incl - kept_mine);
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t m = keep[i];
+                const uint32_t colb = col0 + 32u * i + 31u;
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    const uint32_t col = colb - q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 2u * col));
+                    asm volatile("st.shared.u32 [%0], %1;" ::"r"(at), "r"(prmt(v, col, 0x5410u)) : "memory");
+                    at += 4u;
+                }
+            }
+        }
+        fence_proxy_async_smem();                              // this thread's reads of the row come before the next bulk copy into it
+        __syncthreads();                                       // the stage is complete, the row buffer free
+        if (row64 + gridDim.x < rows) request_row(row64 + gridDim.x);
+
+        // ---- E: the staged entries leave in pairs ------------------------------------------------------------------
+        {
+            const size_t pair_base = out_base - shift;
+            const uint32_t last = shift + k;
+            for (uint32_t p = 2u * threadIdx.x; p < last; p += 2u * W * 32u) {
+                const uint2 e = *reinterpret_cast<const uint2*>(stage + p);
+                const bool first = p >= shift, second = p + 1u < last;
+                if (first && second) {
+                    *reinterpret_cast<uint32_t*>(cols_out + pair_base + p) = prmt(e.x, e.y, 0x7632u);
+                    *reinterpret_cast<uint32_t*>(vals_out + pair_base + p) = prmt(e.x, e.y, 0x5410u);
+                } else if (first) {
+                    cols_out[pair_base + p] = static_cast<int16_t>(e.x >> 16);
+                    vals_out[pair_base + p] = static_cast<uint16_t>(e.x & 0xFFFFu);
+                } else if (second) {
+                    cols_out[pair_base + p + 1u] = static_cast<int16_t>(e.y >> 16);
+                    vals_out[pair_base + p + 1u] = static_cast<uint16_t>(e.y & 0xFFFFu);
+                }
+            }
+            if (rows_out)
+                for (uint32_t p = threadIdx.x; p < k; p += W * 32u) rows_out[out_base + p] = static_cast<int32_t>(row);
+        }
+        __syncthreads();                                       // the stage has been read: its words may become lists again
+    }
+}
+
+template <int W>
+dct_status_t launch_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
+                         void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result, cudaStream_t stream) {
+    using Lay = WideLayout<W>;
+    auto kernel = mp_topk_fwd_bf16_wide_kernel<W>;
+    const size_t smem = Lay::cta_bytes(k);
+    static thread_local int configured_device = -1;
+    int dev = 0;
+    DCT_CUDA_TRY(cudaGetDevice(&dev));
+    if (configured_device != dev) {
+        DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        configured_device = dev;
+    }
+    int per_sm = 0;
+    DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, W * 32, smem));
+    if (per_sm < 1) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
+    const uint32_t grid = static_cast<uint32_t>(rows < max_grid ? rows : max_grid);
+    kernel<<<grid, W * 32, smem, stream>>>(static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out,
+                                           static_cast<uint16_t*>(vals_out), rows_out, static_cast<uint16_t*>(tau_out),
+                                           result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}
+
 }  // namespace
 
 dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                   int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                   dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
+    if (d > 8192 && d <= 32768 && d % 8 == 0 && k <= kWideMaxK && 8ull * k <= 3ull * d && aligned_to(x_act, 16) &&
+        (static_cast<size_t>(ld) * 2) % 16 == 0 && aligned_to(cols_out, 4) && aligned_to(vals_out, 4)) {
+        *handled = true;
+        // as many warps as the row has segments of 4096 columns (the last one zero-padded)
+#define DCT_WIDE_WARPS(W) \
+    if (d <= 4096u * W) return launch_wide<W>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+        DCT_WIDE_WARPS(3);
+        DCT_WIDE_WARPS(4);
+        DCT_WIDE_WARPS(5);
+        DCT_WIDE_WARPS(6);
+        DCT_WIDE_WARPS(7);
+        DCT_WIDE_WARPS(8);
+#undef DCT_WIDE_WARPS
+    }
     // (beyond 3/8 of the row a post-ReLU row's threshold is next to zero, where keys are sparse and the window
     // rarely settles: the general kernel serves those)
     if (d > 8192 || d % 8 != 0 || k > kSpanMaxK || 8ull * k > 3ull * d) return DCT_OK;

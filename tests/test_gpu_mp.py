@@ -303,3 +303,27 @@ def test_mp_bf16_wide_rows(d):
     for k in sorted({1, d // 40, d // 20, d // 10, 1000, 1280}):
         cols = _compare_fwd_bwd(x, gx, d, k)
         assert int(cols.max()) < d
+
+
+@pytest.mark.parametrize("d", [8200, 12288, 16384, 20000, 32768])
+def test_mp_bf16_rows_wider_than_8192(d):
+    """bf16 rows of more than 8192 columns are packed by a CTA per row (4 or 8 warps, each looking after 4096 columns):
+    sparse and denser k, rows of very different scales (the window has to move), dead rows, rows where everything
+    ties, rows with fewer than k non-zeros, rows of a few distinct values (crowded windows and the exact mode), and
+    more rows than CTAs, so that every CTA works through several rows."""
+    rows = 1500 if d <= 16384 else 700
+    x = inputs.mp_activations(rows, d, 91 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=92 + d)
+    sign = torch.where(inputs.dp_gaussian(rows * d, 93 + d, G.DEV).view(rows, d) > 0, 1.0, -1.0)
+    scale = torch.tensor([1.0, 30.0, 1e-2, 1.0, 1e3, 1.0, 1.0], device=G.DEV).repeat(rows // 7 + 1)[:rows]
+    x = x * sign * scale[:, None]
+    x[3] = 0.0
+    x[4] = -1.25
+    x[5, 300:] = 0.0
+    x[6] = inputs.quantize_mantissa(x[6], 1)
+    x[7::50] = inputs.quantize_mantissa(x[7::50], 2)
+    x[8] = 3.0e38
+    x = x.to(torch.bfloat16).contiguous()
+    gx = inputs.mp_gradients(rows, d, 94 + d, dtype=torch.bfloat16, device=G.DEV)
+    for k in sorted({1, 33, d // 20, min(d // 8, 2300), min(d // 4 + 1, 2299)}):
+        cols = _compare_fwd_bwd(x, gx, d, k, want_rows=(k == 33))
+        assert int(cols.max()) < d
