@@ -75,6 +75,9 @@ __global__ void dp_compress_init_kernel(CompressCtrl* ctrl, uint64_t* tile_state
     // the streaming kernel that follows may be scheduled already (it waits for this grid before it touches the
     // control block): its launch latency and set-up then overlap this kernel
     chain_release_next();
+    // launched as a programmatic dependent itself: the kernel before it on the stream (say, the previous call's
+    // streaming kernel, which still reads these descriptors) has to be finished before anything is reset
+    chain_wait_previous();
     if (enabled && *enabled == 0) return;     // a conditional call that is not needed: nothing is touched
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < num_tiles) tile_state[i] = 0;
@@ -823,9 +826,8 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
     const uint32_t num_full = n32 / kTileElems;
     const DebugConfig& dbg = debug_config();
 
-    dp_compress_init_kernel<<<(num_tiles + 1023) / 1024, 1024, 0, stream>>>(ctrl, tile_state, num_tiles, result,
-                                                                            dbg.first_ticket);
-    DCT_CUDA_TRY(cudaGetLastError());
+    DCT_CUDA_TRY(launch_chained(dp_compress_init_kernel, (num_tiles + 1023) / 1024, 1024, stream, ctrl, tile_state, num_tiles,
+                                result, dbg.first_ticket, static_cast<const uint32_t*>(nullptr)));
     const bool vec = aligned_to(grad, 16) && aligned_to(residual, 16);
     if (!vec) {
         const int sms_t = sm_count();
