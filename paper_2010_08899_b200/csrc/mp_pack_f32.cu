@@ -40,6 +40,18 @@ constexpr uint32_t kMaxMembers = 64;      // bucket members ranked through the l
 
 // upper halves of two fp32 words in one register: (hi16(b) << 16) | hi16(a)
 __device__ __forceinline__ uint32_t upper_halves(uint32_t a, uint32_t b) { return __byte_perm(a, b, 0x7632); }
+// Flags "upper 15 key bits >= low" of the 8 fp32 of one 32-byte piece, read as two 16-byte halves `first` and `second`
+// (a lane reads the halves in either order; w_first / w_second are the dot-product weights -2^j of the four columns
+// each half holds).  Exact for every bit pattern: per 16-bit half, bit 15 of ((x | 0x8000) - low) is set iff the
+// key's upper bits are >= low; a byte permutation with sign replication and two signed dot products collect the
+// eight flags, bit j = column j of the piece (see mask8_ge_exact in mp_warp.cuh).  low2 = low in both halves.
+__device__ __forceinline__ uint32_t piece_flags(uint4 first, uint4 second, uint32_t low2, uint32_t w_first, uint32_t w_second) {
+    const uint32_t t0 = (upper_halves(first.x, first.y) | 0x80008000u) - low2;
+    const uint32_t t1 = (upper_halves(first.z, first.w) | 0x80008000u) - low2;
+    const uint32_t t2 = (upper_halves(second.x, second.y) | 0x80008000u) - low2;
+    const uint32_t t3 = (upper_halves(second.z, second.w) | 0x80008000u) - low2;
+    return static_cast<uint32_t>(dp4a_ss(prmt(t2, t3, 0xFDB9u), w_second, dp4a_ss(prmt(t0, t1, 0xFDB9u), w_first, 0)));
+}
 
 // exact key >= low on 31-bit keys, 4 elements
 __device__ __forceinline__ uint32_t mask4_ge_exact(uint4 v, uint32_t low) {
@@ -190,13 +202,9 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
     const uint32_t swap = (lane >> 2) & 1u;                   // 1: this lane reads columns 4..7 of a piece first
     const unsigned char* piece_first = base + lane * 32u + swap * 16u;
     const unsigned char* piece_second = base + lane * 32u + (swap ^ 1u) * 16u;
-    // where the compare results of the two reads go in the byte of the piece (bit j = column j of the piece);
-    // the low half of a result word is the even element of a pair, the high half (folded down by 16) the odd one
-    const uint32_t e_first = swap * 4u, e_second = (swap ^ 1u) * 4u;
-    const uint32_t c_first_01 = (1u << e_first) | (1u << (17u + e_first));
-    const uint32_t c_first_23 = (4u << e_first) | (4u << (17u + e_first));
-    const uint32_t c_second_01 = (1u << e_second) | (1u << (17u + e_second));
-    const uint32_t c_second_23 = (4u << e_second) | (4u << (17u + e_second));
+    // where the flags of the two reads go in the byte of the piece (bit j = column j of the piece)
+    const uint32_t w_first = swap ? 0x80C0E0F0u : 0xF8FCFEFFu;      // dot-product weights -2^j of the columns a read holds
+    const uint32_t w_second = swap ? 0xF8FCFEFFu : 0x80C0E0F0u;
     if (warp_global < rows) request_row(warp_global);
 
     uint32_t use = 0;
@@ -269,18 +277,13 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
         uint32_t masks[kMaskWords];
         uint32_t n_mine = 0, incl = 0, n_cand = 0;
         auto build_masks = [&](uint32_t bound) {
-            const __nv_bfloat162 low2 = as_bf162(bound | (bound << 16));
+            const uint32_t low2 = bound | (bound << 16);
             unsigned char* tab8 = reinterpret_cast<unsigned char*>(mask_tab) + lane;
 #pragma unroll
             for (int c = 0; c < E8; ++c) {
                 const uint4 a = *reinterpret_cast<const uint4*>(piece_first + c * 1024);
                 const uint4 b = *reinterpret_cast<const uint4*>(piece_second + c * 1024);
-                const uint32_t r0 = __hgeu2_mask(__habs2(as_bf162(upper_halves(a.x, a.y))), low2);
-                const uint32_t r1 = __hgeu2_mask(__habs2(as_bf162(upper_halves(a.z, a.w))), low2);
-                const uint32_t r2 = __hgeu2_mask(__habs2(as_bf162(upper_halves(b.x, b.y))), low2);
-                const uint32_t r3 = __hgeu2_mask(__habs2(as_bf162(upper_halves(b.z, b.w))), low2);
-                const uint32_t m = (r0 & c_first_01) | (r1 & c_first_23) | (r2 & c_second_01) | (r3 & c_second_23);
-                tab8[c * 32] = static_cast<unsigned char>(m | (m >> 16));
+                tab8[c * 32] = static_cast<unsigned char>(piece_flags(a, b, low2, w_first, w_second));
             }
             __syncwarp();
             if (kMaskWords == 4) {
@@ -666,13 +669,6 @@ template <int E8> struct DenseLayoutF32 {
     __host__ __device__ static constexpr uint32_t warp_bytes(uint32_t k) { return Row::kRowBytes + scratch_words(k) * 4u + 16u; }
 };
 
-// flags of 8 consecutive fp32: upper 15 key bits >= low, exact for every bit pattern
-__device__ __forceinline__ uint32_t mask8_upper_ge_exact(uint4 a, uint4 b, uint32_t low) {
-    auto ge = [low](uint32_t v) -> uint32_t { return ((v >> 16) & 0x7FFFu) >= low ? 1u : 0u; };
-    return ge(a.x) | (ge(a.y) << 1) | (ge(a.z) << 2) | (ge(a.w) << 3) | (ge(b.x) << 4) | (ge(b.y) << 5) | (ge(b.z) << 6) |
-           (ge(b.w) << 7);
-}
-
 template <int E8>
 __global__ void __launch_bounds__(kDenseMaxWarpsF32 * 32)
 mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
@@ -744,11 +740,8 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
     const uint32_t swap = (lane >> 2) & 1u;
     const unsigned char* piece_first = base + lane * 32u + swap * 16u;
     const unsigned char* piece_second = base + lane * 32u + (swap ^ 1u) * 16u;
-    const uint32_t e_first = swap * 4u, e_second = (swap ^ 1u) * 4u;
-    const uint32_t c_first_01 = (1u << e_first) | (1u << (17u + e_first));
-    const uint32_t c_first_23 = (4u << e_first) | (4u << (17u + e_first));
-    const uint32_t c_second_01 = (1u << e_second) | (1u << (17u + e_second));
-    const uint32_t c_second_23 = (4u << e_second) | (4u << (17u + e_second));
+    const uint32_t w_first = swap ? 0x80C0E0F0u : 0xF8FCFEFFu;      // dot-product weights -2^j of the columns a read holds
+    const uint32_t w_second = swap ? 0xF8FCFEFFu : 0x80C0E0F0u;
     if (warp_global < rows) request_row(warp_global);
 
     uint32_t use = 0;
@@ -796,29 +789,14 @@ mp_topk_fwd_f32_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint
             unsigned char* tl = reinterpret_cast<unsigned char*>(tab_low) + lane;
             unsigned char* th = reinterpret_cast<unsigned char*>(tab_high) + lane;
             __syncwarp();
-            if (low >= 0x0080u && high <= 0x7F80u) {
-                // normal bounds: the packed compare on the upper halves is exact (a NaN lands in both tables)
-                const __nv_bfloat162 low2 = as_bf162(low * 0x10001u), high2 = as_bf162(high * 0x10001u);
+            {
+                const uint32_t low2 = low * 0x10001u, high2 = high * 0x10001u;
 #pragma unroll
                 for (int c = 0; c < E8; ++c) {
                     const uint4 a = *reinterpret_cast<const uint4*>(piece_first + c * 1024);
                     const uint4 b = *reinterpret_cast<const uint4*>(piece_second + c * 1024);
-                    const __nv_bfloat162 h0 = __habs2(as_bf162(upper_halves(a.x, a.y))), h1 = __habs2(as_bf162(upper_halves(a.z, a.w)));
-                    const __nv_bfloat162 h2 = __habs2(as_bf162(upper_halves(b.x, b.y))), h3 = __habs2(as_bf162(upper_halves(b.z, b.w)));
-                    const uint32_t ml = (__hgeu2_mask(h0, low2) & c_first_01) | (__hgeu2_mask(h1, low2) & c_first_23) |
-                                        (__hgeu2_mask(h2, low2) & c_second_01) | (__hgeu2_mask(h3, low2) & c_second_23);
-                    const uint32_t mh = (__hgeu2_mask(h0, high2) & c_first_01) | (__hgeu2_mask(h1, high2) & c_first_23) |
-                                        (__hgeu2_mask(h2, high2) & c_second_01) | (__hgeu2_mask(h3, high2) & c_second_23);
-                    tl[c * 32] = static_cast<unsigned char>(ml | (ml >> 16));
-                    th[c * 32] = static_cast<unsigned char>(mh | (mh >> 16));
-                }
-            } else {
-#pragma unroll
-                for (int c = 0; c < E8; ++c) {
-                    const uint4 a = *reinterpret_cast<const uint4*>(base + lane * 32u + c * 1024);
-                    const uint4 b = *reinterpret_cast<const uint4*>(base + lane * 32u + c * 1024 + 16);
-                    tl[c * 32] = static_cast<unsigned char>(mask8_upper_ge_exact(a, b, low));
-                    th[c * 32] = static_cast<unsigned char>(mask8_upper_ge_exact(a, b, high));
+                    tl[c * 32] = static_cast<unsigned char>(piece_flags(a, b, low2, w_first, w_second));
+                    th[c * 32] = static_cast<unsigned char>(piece_flags(a, b, high2, w_first, w_second));
                 }
             }
             __syncwarp();
