@@ -325,6 +325,15 @@ class HotPath:
             self.grad_view(i), None, n, ks_dp, taus3, res3, ws3, s)
         calls["mp_threshold_mean_3_levels"] = lambda i: B.dct_mp_threshold_mean(
             self.x[i % len(self.x)], rows, d, d, ks_mp, mean3, tau_rows, s)
+        # the select of ONE vector range-partitioned over the ranks (every rank's vector is a shard of it): three
+        # streaming passes with one all-reduce of 2048 counts each (alone at N = 1)
+        import torch.distributed as dist
+        world = dist.get_world_size() if dist.is_available() and dist.is_initialized() else 1
+        ws_sh = B.new_workspace(B.dct_threshold_select_shard_workspace_bytes(), self.dev)
+        hist_sh = torch.empty(2048, dtype=torch.int64, device=self.dev)
+        res_sh = B.new_result(self.dev)
+        calls["threshold_select_sharded"] = lambda i: B.dct_threshold_select_sharded(
+            self.grad_view(i), None, n, c["dp_k"] * world, taus3[:1], res_sh, ws_sh, hist=hist_sh, stream=s)
         calls["mp_fwd_fp32"] = lambda i: B.dct_mp_topk_pack_fwd(x32[i % 2], rows, d, d, k, self.cols, vals32, None,
                                                                  None, None, s)
         for name, call in calls.items():
@@ -340,6 +349,8 @@ class HotPath:
             4 * n / (out["threshold_select_multi_3_levels"]["ms"] * 1e-3) / 1e9
         # one streaming pass: read g, read e, write e' (the floor of a fixed-threshold iteration)
         out["dp_select_compress_L1"]["GBps_at_12B_per_elem"] = 12 * n / (out["dp_select_compress_L1"]["ms"] * 1e-3) / 1e9
+        out["threshold_select_sharded"]["GBps_at_4B_per_elem"] = 4 * n / (out["threshold_select_sharded"]["ms"] * 1e-3) / 1e9
+        out["threshold_select_sharded"]["ranks"] = world
         out["dp_decompress"]["GBps_at_4B_per_elem"] = 4 * n / (out["dp_decompress"]["ms"] * 1e-3) / 1e9
         out["mp_unpack"]["GBps"] = (rows * d * 2 + rows * k * 4) / (out["mp_unpack"]["ms"] * 1e-3) / 1e9
         return out

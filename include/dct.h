@@ -416,6 +416,42 @@ DCT_API dct_status_t dct_dp_compress_static(
     int32_t* idx_out, float* val_out, uint64_t capacity,
     dct_result_t* result, dct_stream_t stream);
 
+/*
+ * dct_threshold_select_shard_{begin,pass,advance} -- the threshold steps of Algorithm 1 (error feedback, sort,
+ * assign tau) for ONE gradient vector that is range-partitioned over several GPUs: every rank holds a contiguous
+ * shard of W_grad and of E_grad, and all ranks want the k-th largest |fl32(W_grad + E_grad)| of the WHOLE vector.
+ * The paper's trainers each compress their own layers (Sec. 2.1) and need no such exchange; this serves a layer
+ * that is itself split over GPUs.
+ *
+ * The select is a radix select in three passes (11 / 10 / 10 key bits).  Per pass every rank calls `pass`, which
+ * writes the 2048-bin digit histogram of its own shard (restricted to the digits chosen so far) to hist_out; the
+ * caller sums the histograms over the ranks (an all-reduce of 16 KiB by whatever transport it uses: the library
+ * never touches another GPU's memory); every rank then calls `advance` with the summed histogram and arrives at
+ * the same digit.  After advance(pass = 2) every rank's tau_out, result->n_gt and result->n_eq are those of
+ * dct_threshold_select on the concatenated vector.  Compression needs no exchange: each rank runs dct_dp_compress
+ * on its shard with that tau.
+ *
+ *   k_global   1 <= k_global <= total number of elements over all ranks (not checked: the ranks' sizes are not
+ *              known here; with a larger k the outputs are unspecified).
+ *   workspace  DEVICE, >= dct_threshold_select_shard_workspace_bytes(), 256-byte aligned: the state of one select
+ *              (the same on every rank after every advance).  `begin` resets it.
+ *   grad, residual  [n_local] fp32 device, read only; residual may be NULL; n_local may be 0 (an empty shard).
+ *   pass       0, 1, 2, in this order, each followed by its advance.
+ *   hist_out   [2048] uint64 DEVICE: overwritten with this shard's histogram.
+ *   hist_global [2048] uint64 DEVICE: the sum over all ranks.
+ *   tau_out, result  device; written by advance(pass = 2) only (may be NULL for passes 0 and 1).
+ * Errors: DCT_ERR_INVALID_ARG / DCT_ERR_WORKSPACE before anything is launched.
+ */
+DCT_API size_t dct_threshold_select_shard_workspace_bytes(void);
+DCT_API dct_status_t dct_threshold_select_shard_begin(
+    uint64_t k_global, void* workspace, size_t workspace_bytes, dct_stream_t stream);
+DCT_API dct_status_t dct_threshold_select_shard_pass(
+    const float* grad, const float* residual, uint64_t n_local, uint32_t pass,
+    const void* workspace, uint64_t* hist_out, dct_stream_t stream);
+DCT_API dct_status_t dct_threshold_select_shard_advance(
+    const uint64_t* hist_global, uint32_t pass, void* workspace,
+    float* tau_out, dct_result_t* result, dct_stream_t stream);
+
 /* ------------------------------------------------------------------------- *
  * Threshold diagnostics: the quantities behind the paper's threshold plots.
  * None of them changes a gradient, a residual or an activation.

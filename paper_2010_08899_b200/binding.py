@@ -34,6 +34,8 @@ EXPORTED_SYMBOLS = (
     "dct_threshold_select_multi", "dct_threshold_select_multi_workspace_bytes",
     "dct_mp_threshold_mean", "dct_dp_drift_check",
     "dct_threshold_select_batched", "dct_threshold_select_batched_workspace_bytes",
+    "dct_threshold_select_shard_workspace_bytes", "dct_threshold_select_shard_begin",
+    "dct_threshold_select_shard_pass", "dct_threshold_select_shard_advance",
 )
 
 _vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
@@ -111,6 +113,14 @@ def lib() -> ctypes.CDLL:
     L.dct_threshold_select_batched_workspace_bytes.argtypes = [_u32]
     L.dct_threshold_select_batched.restype = _int
     L.dct_threshold_select_batched.argtypes = [_vp, _u32, _vp, _sz, _vp]
+    L.dct_threshold_select_shard_workspace_bytes.restype = _sz
+    L.dct_threshold_select_shard_workspace_bytes.argtypes = []
+    L.dct_threshold_select_shard_begin.restype = _int
+    L.dct_threshold_select_shard_begin.argtypes = [_u64, _vp, _sz, _vp]
+    L.dct_threshold_select_shard_pass.restype = _int
+    L.dct_threshold_select_shard_pass.argtypes = [_vp, _vp, _u64, _u32, _vp, _vp, _vp]
+    L.dct_threshold_select_shard_advance.restype = _int
+    L.dct_threshold_select_shard_advance.argtypes = [_vp, _u32, _vp, _vp, _vp, _vp]
     L.dct_debug_configure.restype = None
     L.dct_debug_configure.argtypes = [_u32, _u32]
     _lib = L
@@ -548,3 +558,64 @@ def dct_threshold_select_batched(layers, workspace, stream=None) -> None:
     _need(workspace, torch.uint8, "workspace")
     _check("dct_threshold_select_batched",
            lib().dct_threshold_select_batched(table, len(table), _p(workspace), workspace.numel(), _stream(stream)))
+
+
+# --------------------------------------------------------------------------------------------
+# one vector range-partitioned over several ranks: the select with one small all-reduce per radix pass
+# --------------------------------------------------------------------------------------------
+
+SHARD_PASSES = 3
+SHARD_BINS = 2048
+
+
+def sharded_select_rounds(local_histogram, advance, all_reduce_sum):
+    """The rounds of the range-partitioned select, free of any device code so that the exchange can be exercised on
+    CPU ranks: per pass ``local_histogram(p)`` returns this rank's 2048 digit counts, ``all_reduce_sum(h)`` returns
+    (or turns ``h`` into) their sum over the ranks, and ``advance(p, h)`` lets the rank pick the digit."""
+    for p in range(SHARD_PASSES):
+        h = local_histogram(p)
+        summed = all_reduce_sum(h)
+        advance(p, h if summed is None else summed)
+
+
+def dct_threshold_select_shard_workspace_bytes() -> int:
+    return lib().dct_threshold_select_shard_workspace_bytes()
+
+
+def dct_threshold_select_sharded(grad, residual, n_local, k_global, tau_out, result, workspace, group=None,
+                                 hist=None, stream=None) -> None:
+    """The k_global-th largest |grad + residual| of a vector whose shards lie on the ranks of ``group`` (the default
+    process group if None; a single process without a group selects over its own shard alone).  Every rank calls
+    this with its own shard; all get the same tau_out / result.  One all-reduce of 2048 int64 counts per pass."""
+    import torch.distributed as dist
+    if n_local:
+        _need(grad, torch.float32, "grad")
+    if residual is not None:
+        _need(residual, torch.float32, "residual")
+    _need(tau_out, torch.float32, "tau_out")
+    _need(result, torch.int64, "result")
+    _need(workspace, torch.uint8, "workspace")
+    if hist is None:
+        hist = torch.empty(SHARD_BINS, dtype=torch.int64, device=tau_out.device)
+    _need(hist, torch.int64, "hist")
+    L, s = lib(), _stream(stream)
+    _check("dct_threshold_select_shard_begin",
+           L.dct_threshold_select_shard_begin(k_global, _p(workspace), workspace.numel(), s))
+    multi = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
+
+    def local_histogram(p):
+        _check("dct_threshold_select_shard_pass",
+               L.dct_threshold_select_shard_pass(_p(grad) if n_local else None, _p(residual), n_local, p, _p(workspace),
+                                                 _p(hist), s))
+        return hist
+
+    def all_reduce_sum(h):
+        if multi:
+            dist.all_reduce(h, op=dist.ReduceOp.SUM, group=group)
+        return None
+
+    def advance(p, h):
+        _check("dct_threshold_select_shard_advance",
+               L.dct_threshold_select_shard_advance(_p(h), p, _p(workspace), _p(tau_out), _p(result), s))
+
+    sharded_select_rounds(local_histogram, advance, all_reduce_sum)
