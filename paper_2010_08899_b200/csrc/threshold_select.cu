@@ -49,6 +49,8 @@ struct SelectState {
     uint32_t enabled;     // 0: every kernel of this select returns at once
     uint32_t n;           // elements of the source (written on the device for the candidate buffer)
     uint32_t key_out;     // the selected key (the sample select hands `lo` to the filter this way)
+    uint32_t last_pass;   // the pass that ends this select: 2, or 1 for a select that only needs a lower bound of the
+                          // rank-th key (its lower 10 bits are then zero)
     uint32_t hist[kPasses * kBins];
 };
 
@@ -63,7 +65,7 @@ struct SelectWorkspace {
 
 constexpr int kInitThreads = 1024;
 __device__ __forceinline__ void reset_state(SelectState* st, uint32_t k, uint32_t n, uint32_t enabled, uint32_t i,
-                                            uint32_t stride) {
+                                            uint32_t stride, uint32_t last_pass = kPasses - 1) {
     for (uint32_t b = i; b < kPasses * kBins; b += stride) st->hist[b] = 0;
     if (i == 0) {
         st->prefix = 0;
@@ -73,6 +75,7 @@ __device__ __forceinline__ void reset_state(SelectState* st, uint32_t k, uint32_
         st->enabled = enabled;
         st->n = n;
         st->key_out = 0;
+        st->last_pass = last_pass;
     }
 }
 
@@ -82,7 +85,8 @@ __global__ void select_init_kernel(SelectWorkspace* ws, uint32_t n, uint32_t k, 
     const uint32_t i = threadIdx.x;
     const bool sampled = sample_n != 0;
     reset_state(&ws->full, k, n, sampled ? 0u : 1u, i, kInitThreads);
-    reset_state(&ws->sample, sample_k, sample_n, sampled ? 1u : 0u, i, kInitThreads);
+    // the sample only has to give a lower bound of its rank-th key: two passes (21 of the 31 key bits) do
+    reset_state(&ws->sample, sample_k, sample_n, sampled ? 1u : 0u, i, kInitThreads, 1u);
     reset_state(&ws->cand, k, 0u, 0u, i, kInitThreads);
     if (i == 0) {
         ws->cand_count = 0;
@@ -157,10 +161,11 @@ __device__ __forceinline__ void finish_pass(SelectState* st, uint32_t prefix, ui
             st->k_rem = k_rem - above;
             const uint64_t n_gt = st->n_gt + above;
             st->n_gt = n_gt;
-            if (kPass == kPasses - 1) {
-                st->key_out = new_prefix;
+            if (kPass == static_cast<int>(st->last_pass)) {
+                const uint32_t key = new_prefix << pass_shift(kPass);      // (the bits no pass has looked at are zero)
+                st->key_out = key;
                 if (tau_out) {           // this select produces the call's answer
-                    *tau_out = __uint_as_float(new_prefix);
+                    *tau_out = __uint_as_float(key);
                     result->n_gt = n_gt;
                     result->n_eq = c[q];
                 }
@@ -170,19 +175,15 @@ __device__ __forceinline__ void finish_pass(SelectState* st, uint32_t prefix, ui
     }
 }
 
+// One radix pass of one select by the whole grid.  sh (kBins words, cleared by the caller), s_scan and s_last are the
+// CTA's shared memory; the caller has waited for the previous kernel of the chain.
 template <int kPass, typename Source, bool kVectorised>
-__global__ void __launch_bounds__(kSelThreads)
-select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct_result_t* __restrict__ result) {
+__device__ __forceinline__ void select_pass_body(const Source& src, SelectState* st, float* __restrict__ tau_out,
+                                                 dct_result_t* __restrict__ result, uint32_t* sh, uint32_t* s_scan,
+                                                 uint32_t& s_last) {
     constexpr int shift = pass_shift(kPass);
     constexpr int bits = pass_bits(kPass);
     constexpr uint32_t digit_mask = (1u << bits) - 1u;
-    __shared__ uint32_t sh[kBins];
-    __shared__ uint32_t s_scan[kSelThreads / 32];
-    __shared__ uint32_t s_last;
-
-    for (int b = threadIdx.x; b < kBins; b += kSelThreads) sh[b] = 0;
-    chain_wait_previous();
-    if (!st->enabled) return;
     const uint32_t prefix = kPass == 0 ? 0u : st->prefix;   // written by the previous launch
     const uint32_t n = st->n;
     __syncthreads();
@@ -249,6 +250,36 @@ select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct
     if (!s_last) return;
     __threadfence();
     finish_pass<kPass>(st, prefix, s_scan, tau_out, result);
+}
+
+template <int kPass, typename Source, bool kVectorised>
+__global__ void __launch_bounds__(kSelThreads)
+select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct_result_t* __restrict__ result) {
+    __shared__ uint32_t sh[kBins];
+    __shared__ uint32_t s_scan[kSelThreads / 32];
+    __shared__ uint32_t s_last;
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) sh[b] = 0;
+    chain_wait_previous();
+    if (!st->enabled) return;
+    select_pass_body<kPass, Source, kVectorised>(src, st, tau_out, result, sh, s_scan, s_last);
+}
+
+// The same pass for whichever of two selects is enabled: the select over the few candidates (the normal case) or,
+// should the sample have misjudged the vector, the plain select over the whole vector -- one launch instead of two,
+// of which one would return at once.
+template <int kPass, typename CandSource, bool kVectorised>
+__global__ void __launch_bounds__(kSelThreads)
+select_pass_either_kernel(CandSource cand_src, SelectState* cand, VectorSource full_src, SelectState* full,
+                          float* __restrict__ tau_out, dct_result_t* __restrict__ result) {
+    __shared__ uint32_t sh[kBins];
+    __shared__ uint32_t s_scan[kSelThreads / 32];
+    __shared__ uint32_t s_last;
+    for (int b = threadIdx.x; b < kBins; b += kSelThreads) sh[b] = 0;
+    chain_wait_previous();
+    if (cand->enabled)
+        select_pass_body<kPass, CandSource, false>(cand_src, cand, tau_out, result, sh, s_scan, s_last);
+    else if (full->enabled)
+        select_pass_body<kPass, VectorSource, kVectorised>(full_src, full, tau_out, result, sh, s_scan, s_last);
 }
 
 // The single streaming pass of the sampled path: every key >= key(lo) goes to the candidate buffer.
@@ -338,12 +369,37 @@ __global__ void select_decide_kernel(SelectWorkspace* ws, uint32_t k) {
 
 template <typename Source, bool kVectorised>
 cudaError_t launch_three_passes(int grid, cudaStream_t stream, Source src, SelectState* st, float* tau_out,
-                                dct_result_t* result) {
+                                dct_result_t* result, int passes = kPasses) {
     cudaError_t e = launch_chained(select_pass_kernel<0, Source, kVectorised>, grid, kSelThreads, stream, src, st, tau_out, result);
-    if (e == cudaSuccess)
+    if (e == cudaSuccess && passes > 1)
         e = launch_chained(select_pass_kernel<1, Source, kVectorised>, grid, kSelThreads, stream, src, st, tau_out, result);
-    if (e == cudaSuccess)
+    if (e == cudaSuccess && passes > 2)
         e = launch_chained(select_pass_kernel<2, Source, kVectorised>, grid, kSelThreads, stream, src, st, tau_out, result);
+    return e;
+}
+
+// The two passes of the sample select (its state says that pass 1 is its last).
+constexpr int kSamplePasses = 2;
+
+// Three launches that run the candidate select or, if that one is disabled and the other enabled, the select over
+// the whole vector.  The grid is the vector's: the few candidates are spread over it.
+template <typename CandSource>
+cudaError_t launch_three_either(int grid, cudaStream_t stream, CandSource csrc, SelectState* cand, VectorSource vsrc,
+                                bool vectorised, SelectState* full, float* tau_out, dct_result_t* result) {
+    cudaError_t e;
+    if (vectorised) {
+        e = launch_chained(select_pass_either_kernel<0, CandSource, true>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+        if (e == cudaSuccess)
+            e = launch_chained(select_pass_either_kernel<1, CandSource, true>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+        if (e == cudaSuccess)
+            e = launch_chained(select_pass_either_kernel<2, CandSource, true>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+    } else {
+        e = launch_chained(select_pass_either_kernel<0, CandSource, false>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+        if (e == cudaSuccess)
+            e = launch_chained(select_pass_either_kernel<1, CandSource, false>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+        if (e == cudaSuccess)
+            e = launch_chained(select_pass_either_kernel<2, CandSource, false>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+    }
     return e;
 }
 
@@ -416,7 +472,8 @@ dct_status_t l1_sample_bound(const float* grad, const float* residual, uint64_t 
     const StridedSource ssrc{grad, residual, stride};
     const uint64_t chunks = (kSampleSize + kSelChunk - 1) / kSelChunk;
     const int grid = static_cast<int>(chunks < static_cast<uint64_t>(sms) * 4 ? chunks : sms * 4);
-    DCT_CUDA_TRY((launch_three_passes<StridedSource, false>(grid, stream, ssrc, &ws->sample, &block->lo, &block->scratch)));
+    DCT_CUDA_TRY((launch_three_passes<StridedSource, false>(grid, stream, ssrc, &ws->sample, &block->lo, &block->scratch,
+                                                            kSamplePasses)));
     return DCT_OK;
 }
 
@@ -430,16 +487,13 @@ dct_status_t l1_exact_threshold(const int32_t* cand_idx, const float* cand_val, 
     DCT_CUDA_TRY(launch_chained(l1_decide_kernel, 1, 1, stream, ws, block, static_cast<uint32_t>(k), cap));
     DCT_CUDA_TRY(launch_chained(l1_restore_kernel, sms * 2, 256, stream, cand_idx, cand_val, residual,
                                 static_cast<const L1Block*>(block)));
-    // the exact select: over the candidates (normally), or over w (the kernels that are not needed return at once)
+    // the exact select: over the candidates (normally), or over w
     const ValueSource csrc{cand_val};
-    DCT_CUDA_TRY((launch_three_passes<ValueSource, false>(128, stream, csrc, &ws->cand, tau_out, &block->scratch)));
     const VectorSource wsrc{residual, nullptr};
     const uint64_t chunks = (n + kSelChunk - 1) / kSelChunk;
     const int grid = static_cast<int>(chunks < static_cast<uint64_t>(sms) * 4 ? (chunks ? chunks : 1) : sms * 4);
-    if (aligned_to(residual, 16))
-        DCT_CUDA_TRY((launch_three_passes<VectorSource, true>(grid, stream, wsrc, &ws->full, tau_out, &block->scratch)));
-    else
-        DCT_CUDA_TRY((launch_three_passes<VectorSource, false>(grid, stream, wsrc, &ws->full, tau_out, &block->scratch)));
+    DCT_CUDA_TRY(launch_three_either(grid, stream, csrc, &ws->cand, wsrc, aligned_to(residual, 16), &ws->full, tau_out,
+                                     &block->scratch));
     DCT_CUDA_TRY(launch_chained(l1_budget_kernel, 1, 1, stream, block, static_cast<const dct_result_t*>(&block->scratch), k));
     return DCT_OK;
 }
@@ -493,17 +547,19 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
     if (sample_n) {
         const StridedSource ssrc{grad, residual, stride};
         DCT_CUDA_TRY((launch_three_passes<StridedSource, false>(grid_for(sample_n), stream, ssrc, &ws->sample, nullptr,
-                                                                result)));
+                                                                result, kSamplePasses)));
         if (vec)
             DCT_CUDA_TRY(launch_chained(select_filter_kernel<true>, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
         else
             DCT_CUDA_TRY(launch_chained(select_filter_kernel<false>, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
         DCT_CUDA_TRY(launch_chained(select_decide_kernel, 1, 1, stream, ws, k32));
+        // the exact select over the candidates (their count is only known on the device) or, should the sample
+        // have misjudged the vector, over the vector itself: the same three launches serve either
         const KeySource ksrc{cand_keys};
-        // the candidate count is only known on the device: a fixed modest grid walks whatever is there
-        DCT_CUDA_TRY((launch_three_passes<KeySource, false>(128, stream, ksrc, &ws->cand, tau_out, result)));
+        DCT_CUDA_TRY(launch_three_either(grid_for(n), stream, ksrc, &ws->cand, vsrc, vec, &ws->full, tau_out, result));
+        return DCT_OK;
     }
-    // the plain three passes: the only path for small or dense problems, the fall-back otherwise
+    // small or dense problems: the plain three passes
     if (vec)
         DCT_CUDA_TRY((launch_three_passes<VectorSource, true>(grid_for(n), stream, vsrc, &ws->full, tau_out, result)));
     else
