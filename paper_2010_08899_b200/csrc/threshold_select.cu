@@ -179,13 +179,12 @@ __device__ __forceinline__ void finish_pass(SelectState* st, uint32_t prefix, ui
 // CTA's shared memory; the caller has waited for the previous kernel of the chain.
 template <int kPass, typename Source, bool kVectorised>
 __device__ __forceinline__ void select_pass_body(const Source& src, SelectState* st, float* __restrict__ tau_out,
-                                                 dct_result_t* __restrict__ result, uint32_t* sh, uint32_t* s_scan,
-                                                 uint32_t& s_last) {
+                                                 dct_result_t* __restrict__ result, uint32_t n, uint32_t* sh,
+                                                 uint32_t* s_scan, uint32_t& s_last) {
     constexpr int shift = pass_shift(kPass);
     constexpr int bits = pass_bits(kPass);
     constexpr uint32_t digit_mask = (1u << bits) - 1u;
     const uint32_t prefix = kPass == 0 ? 0u : st->prefix;   // written by the previous launch
-    const uint32_t n = st->n;
     __syncthreads();
 
     auto consume = [&](uint32_t key) {
@@ -261,25 +260,39 @@ select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) sh[b] = 0;
     chain_wait_previous();
     if (!st->enabled) return;
-    select_pass_body<kPass, Source, kVectorised>(src, st, tau_out, result, sh, s_scan, s_last);
+    select_pass_body<kPass, Source, kVectorised>(src, st, tau_out, result, st->n, sh, s_scan, s_last);
 }
 
-// The same pass for whichever of two selects is enabled: the select over the few candidates (the normal case) or,
-// should the sample have misjudged the vector, the plain select over the whole vector -- one launch instead of two,
-// of which one would return at once.
+// The same pass for one of two selects: the one over the few candidates (the normal case) or, should the sample have
+// misjudged the vector, the plain one over the whole vector -- one launch instead of two, of which one would return
+// at once.  Which one: with k_decide == 0 the enabled flags of the two states say (a kernel before this one set
+// them); otherwise every CTA of every pass decides for itself from the candidate count that the filter left, the
+// same way each time: the candidates if they are at least k_decide and all fitted into their buffer.
 template <int kPass, typename CandSource, bool kVectorised>
 __global__ void __launch_bounds__(kSelThreads)
-select_pass_either_kernel(CandSource cand_src, SelectState* cand, VectorSource full_src, SelectState* full,
+select_pass_either_kernel(CandSource cand_src, VectorSource full_src, SelectWorkspace* ws, uint32_t k_decide,
                           float* __restrict__ tau_out, dct_result_t* __restrict__ result) {
     __shared__ uint32_t sh[kBins];
     __shared__ uint32_t s_scan[kSelThreads / 32];
     __shared__ uint32_t s_last;
     for (int b = threadIdx.x; b < kBins; b += kSelThreads) sh[b] = 0;
     chain_wait_previous();
-    if (cand->enabled)
-        select_pass_body<kPass, CandSource, false>(cand_src, cand, tau_out, result, sh, s_scan, s_last);
-    else if (full->enabled)
-        select_pass_body<kPass, VectorSource, kVectorised>(full_src, full, tau_out, result, sh, s_scan, s_last);
+    bool use_cand, use_full;
+    uint32_t cand_n;
+    if (k_decide) {
+        cand_n = ws->cand_count;
+        use_cand = cand_n >= k_decide && cand_n <= ws->cand_capacity;
+        use_full = !use_cand;
+    } else {
+        cand_n = ws->cand.n;
+        use_cand = ws->cand.enabled != 0;
+        use_full = ws->full.enabled != 0;
+    }
+    if (use_cand)
+        select_pass_body<kPass, CandSource, false>(cand_src, &ws->cand, tau_out, result, cand_n, sh, s_scan, s_last);
+    else if (use_full)
+        select_pass_body<kPass, VectorSource, kVectorised>(full_src, &ws->full, tau_out, result, ws->full.n, sh, s_scan,
+                                                           s_last);
 }
 
 // The single streaming pass of the sampled path: every key >= key(lo) goes to the candidate buffer.
@@ -353,20 +366,6 @@ select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t
     if (held) flush();
 }
 
-// After the filter: decide which select produces the answer.
-__global__ void select_decide_kernel(SelectWorkspace* ws, uint32_t k) {
-    chain_release_next();
-    chain_wait_previous();
-    if (!ws->sample.enabled) return;
-    const uint32_t c = ws->cand_count;
-    if (c >= k && c <= ws->cand_capacity) {
-        ws->cand.n = c;
-        ws->cand.enabled = 1;
-    } else {
-        ws->full.enabled = 1;      // the sample misjudged the vector: do it the plain way
-    }
-}
-
 template <typename Source, bool kVectorised>
 cudaError_t launch_three_passes(int grid, cudaStream_t stream, Source src, SelectState* st, float* tau_out,
                                 dct_result_t* result, int passes = kPasses) {
@@ -381,24 +380,24 @@ cudaError_t launch_three_passes(int grid, cudaStream_t stream, Source src, Selec
 // The two passes of the sample select (its state says that pass 1 is its last).
 constexpr int kSamplePasses = 2;
 
-// Three launches that run the candidate select or, if that one is disabled and the other enabled, the select over
-// the whole vector.  The grid is the vector's: the few candidates are spread over it.
+// Three launches that run the candidate select or the select over the whole vector (k_decide: see the kernel).  The
+// grid is the vector's: the few candidates are spread over it.
 template <typename CandSource>
-cudaError_t launch_three_either(int grid, cudaStream_t stream, CandSource csrc, SelectState* cand, VectorSource vsrc,
-                                bool vectorised, SelectState* full, float* tau_out, dct_result_t* result) {
+cudaError_t launch_three_either(int grid, cudaStream_t stream, CandSource csrc, VectorSource vsrc, bool vectorised,
+                                SelectWorkspace* ws, uint32_t k_decide, float* tau_out, dct_result_t* result) {
     cudaError_t e;
     if (vectorised) {
-        e = launch_chained(select_pass_either_kernel<0, CandSource, true>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+        e = launch_chained(select_pass_either_kernel<0, CandSource, true>, grid, kSelThreads, stream, csrc, vsrc, ws, k_decide, tau_out, result);
         if (e == cudaSuccess)
-            e = launch_chained(select_pass_either_kernel<1, CandSource, true>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+            e = launch_chained(select_pass_either_kernel<1, CandSource, true>, grid, kSelThreads, stream, csrc, vsrc, ws, k_decide, tau_out, result);
         if (e == cudaSuccess)
-            e = launch_chained(select_pass_either_kernel<2, CandSource, true>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+            e = launch_chained(select_pass_either_kernel<2, CandSource, true>, grid, kSelThreads, stream, csrc, vsrc, ws, k_decide, tau_out, result);
     } else {
-        e = launch_chained(select_pass_either_kernel<0, CandSource, false>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+        e = launch_chained(select_pass_either_kernel<0, CandSource, false>, grid, kSelThreads, stream, csrc, vsrc, ws, k_decide, tau_out, result);
         if (e == cudaSuccess)
-            e = launch_chained(select_pass_either_kernel<1, CandSource, false>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+            e = launch_chained(select_pass_either_kernel<1, CandSource, false>, grid, kSelThreads, stream, csrc, vsrc, ws, k_decide, tau_out, result);
         if (e == cudaSuccess)
-            e = launch_chained(select_pass_either_kernel<2, CandSource, false>, grid, kSelThreads, stream, csrc, cand, vsrc, full, tau_out, result);
+            e = launch_chained(select_pass_either_kernel<2, CandSource, false>, grid, kSelThreads, stream, csrc, vsrc, ws, k_decide, tau_out, result);
     }
     return e;
 }
@@ -492,7 +491,7 @@ dct_status_t l1_exact_threshold(const int32_t* cand_idx, const float* cand_val, 
     const VectorSource wsrc{residual, nullptr};
     const uint64_t chunks = (n + kSelChunk - 1) / kSelChunk;
     const int grid = static_cast<int>(chunks < static_cast<uint64_t>(sms) * 4 ? (chunks ? chunks : 1) : sms * 4);
-    DCT_CUDA_TRY(launch_three_either(grid, stream, csrc, &ws->cand, wsrc, aligned_to(residual, 16), &ws->full, tau_out,
+    DCT_CUDA_TRY(launch_three_either(grid, stream, csrc, wsrc, aligned_to(residual, 16), ws, 0u, tau_out,
                                      &block->scratch));
     DCT_CUDA_TRY(launch_chained(l1_budget_kernel, 1, 1, stream, block, static_cast<const dct_result_t*>(&block->scratch), k));
     return DCT_OK;
@@ -552,11 +551,10 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
             DCT_CUDA_TRY(launch_chained(select_filter_kernel<true>, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
         else
             DCT_CUDA_TRY(launch_chained(select_filter_kernel<false>, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
-        DCT_CUDA_TRY(launch_chained(select_decide_kernel, 1, 1, stream, ws, k32));
         // the exact select over the candidates (their count is only known on the device) or, should the sample
         // have misjudged the vector, over the vector itself: the same three launches serve either
         const KeySource ksrc{cand_keys};
-        DCT_CUDA_TRY(launch_three_either(grid_for(n), stream, ksrc, &ws->cand, vsrc, vec, &ws->full, tau_out, result));
+        DCT_CUDA_TRY(launch_three_either(grid_for(n), stream, ksrc, vsrc, vec, ws, k32, tau_out, result));
         return DCT_OK;
     }
     // small or dense problems: the plain three passes
