@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libdct_b200.so")
-SOURCES = ["mp_pack.cu", "mp_pack_span.cu", "mp_pack_f32.cu", "mp_pack_narrow.cu", "dp_compress.cu", "threshold_select.cu", "threshold_select_batched.cu", "threshold_select_sharded.cu", "decompress.cu", "diagnostics.cu",
+SOURCES = ["mp_pack.cu", "mp_pack_span.cu", "mp_pack_f32_wide.cu", "mp_pack_f32.cu", "mp_pack_narrow.cu", "dp_compress.cu", "threshold_select.cu", "threshold_select_batched.cu", "threshold_select_sharded.cu", "decompress.cu", "diagnostics.cu",
            "dp_select_compress.cu", "abi.cu"]          # the slowest to compile first
 HEADERS = [os.path.join(CSRC, h) for h in ("common.cuh", "row_select.cuh", "mp_warp.cuh", "dp_chain.cuh")] + \
           [os.path.join(ROOT, "include", "dct.h")]

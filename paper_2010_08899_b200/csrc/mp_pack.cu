@@ -810,6 +810,10 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
         const dct_status_t fast = launch_fwd_f32_warp(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
                                                       result, stream, &handled);
         if (fast != DCT_OK || handled) return fast;
+        // rows of more than 2048 columns that the warp-per-row kernels leave out: one CTA per row
+        const dct_status_t wide = launch_fwd_f32_wide(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
+                                                      result, stream, &handled);
+        if (wide != DCT_OK || handled) return wide;
         return launch_fwd<float>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     }
     {   // narrow rows (256 or 512 columns, small k): the row stays in registers, several rows per warp

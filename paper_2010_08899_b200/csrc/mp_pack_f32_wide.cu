@@ -1,0 +1,463 @@
+// dct_mp_topk_pack_fwd, fp32, rows of more than 2048 columns (up to 32768) that the warp-per-row kernels do not serve:
+// Algorithm 2 (DCT-MP), forward pass -- one CTA of W warps per row, warp w looking after the columns
+// [2048 w, 2048 w + 2048) and lane l of it after 64 of them.
+//
+// The row arrives by one bulk copy (TMA engine) into shared memory as it lies in HBM.  The steps are those of the
+// bf16 kernel for wide rows (mp_pack_span.cu), on two levels, because a key has 31 bits and the packed compares 15:
+//   A  two bounds around the *bucket* of tau_i (a bucket = the upper 15 bits of the key, the bf16 truncation of |x|):
+//      the previous row's bucket minus half a window, or a quantile of 128 samples of the row.
+//   B  one pass over the lane's sixteen 16-byte units gives two flags per column (bucket >= low, bucket >= high) as
+//      bits in registers: the upper halves of the fp32 words are gathered by byte permutes, the compares are integer
+//      subtractions on the packed halves, and a byte permutation plus two dot-product instructions collect 8 flags.
+//      The units are read in an XOR-swizzled order (no bank conflicts although the lanes' spans are 256 bytes
+//      apart); a byte permutation puts the flags back in column order.  Counts are summed over the CTA; the window
+//      moves until n_high < k <= n_low.
+//   C  the buckets of the window elements go into a 64-bin histogram, which gives the bucket of tau_i and how many of
+//      its members belong to the top k.  A second flag pass at that bucket marks the members; their lower 16 key bits
+//      are then searched bit by bit (16 counting rounds over the few members, summed over the CTA), which gives the
+//      exact 31-bit tau_i; members above it and the first ties, in column order, join the columns above the bucket.
+//   D  a scan over the kept counts gives every lane its offset in the row's output; it stages column and value.
+//   E  the staged entries leave as coalesced stores while the row buffer already receives the CTA's next row.
+// A row whose window does not settle finds its bucket bit by bit (15 counting passes) and goes on from C's second
+// half; a row with fewer than k elements outside bucket 0 starts there.  The result never depends on the guesses.
+#include "common.cuh"
+#include "mp_warp.cuh"
+
+namespace dct {
+namespace {
+
+constexpr uint32_t kWideWindowF32 = 64;           // widest window, in buckets (= histogram bins)
+constexpr uint32_t kWideMaxKF32 = 4096;
+constexpr int kWideRetriesF32 = 6;
+
+template <int W> struct WideLayoutF32 {
+    static constexpr uint32_t kSegBytes = 8192u;             // one warp's 2048 columns
+    static constexpr uint32_t kRowBytes = W * kSegBytes;
+    static constexpr uint32_t kHistBytes = 256u;
+    __host__ __device__ static constexpr uint32_t vals_bytes(uint32_t k) { return 4u * k; }
+    __host__ __device__ static constexpr uint32_t cta_bytes(uint32_t k) {
+        return (kRowBytes + kHistBytes + vals_bytes(k) + 2u * (k + 2u) + 127u) & ~127u;
+    }
+};
+
+// upper halves of two fp32 words in one register, with bit 15 of either half set: (hi16(b) << 16) | hi16(a) | 0x80008000
+__device__ __forceinline__ uint32_t upper_halves_set(uint32_t a, uint32_t b) {
+    return prmt(a, b, 0x7632u) | 0x80008000u;
+}
+
+template <int W>
+__global__ void __launch_bounds__(W * 32)
+mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                            int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
+                            int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
+                            dct_result_t* __restrict__ result) {
+    using Lay = WideLayoutF32<W>;
+    constexpr int kWords = 2;                                  // 64 columns per lane
+    constexpr uint32_t kLaneCols = 64u;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    unsigned char* base = smem_raw;
+    const unsigned char* own = base + warp * Lay::kSegBytes + lane * 256u;
+    uint32_t* hist = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
+    uint32_t* stage_vals = hist + Lay::kHistBytes / 4;
+    uint16_t* stage_cols = reinterpret_cast<uint16_t*>(stage_vals + k);
+    __shared__ uint64_t s_bar;
+    __shared__ uint32_t s_stop;
+    __shared__ uint32_t s_cnt[2][W];                           // per-warp packed counts (double-buffered across passes)
+    __shared__ uint32_t s_sum[2][W];                           // per-warp totals for the two prefix sums of a row
+    __shared__ uint32_t s_guess;
+
+    if (threadIdx.x == 0) {
+        s_stop = 0;
+        mbar_init(&s_bar, 1);
+        mbar_init_fence();
+        fence_proxy_async_all();
+    }
+    const uint32_t row_bytes = d * 4u;                         // the tail of the buffer stays zero
+    for (uint32_t b = row_bytes + threadIdx.x * 16u; b < Lay::kRowBytes; b += W * 512u)
+        *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+    // Step c of a pass reads the unit (swz ^ c % 8) + 8 (c / 8) of the lane's sixteen; steps 2p and 2p + 1 make up the
+    // 32-byte piece (p % 4 ^ swz / 2) + 4 (p / 4), its upper half first if swz is odd.
+    const uint32_t swz = lane & 7u;
+    const uint32_t fix_sel = 0x3210u ^ (0x1111u * (swz >> 1));
+    const uint32_t w_first = (swz & 1u) ? 0xFFFEFCF8u : 0xF0E0C080u;     // column j of a piece at bit 7 - j
+    const uint32_t w_second = (swz & 1u) ? 0xF0E0C080u : 0xFFFEFCF8u;
+    uint32_t unit_base[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) unit_base[c] = smem_addr(own) ^ (16u * (swz ^ static_cast<uint32_t>(c)));
+    const uint32_t row_addr = smem_addr(base);
+    const uint32_t col0 = warp * 2048u + lane * kLaneCols;     // first column of the lane's span
+
+    auto request_row = [&](uint64_t r) {
+        if (threadIdx.x == 0) {
+            fence_proxy_async_smem();
+            mbar_arrive_expect_tx(&s_bar, row_bytes);
+            bulk_load(base, x + static_cast<size_t>(r) * ld, row_bytes, &s_bar);
+        }
+    };
+    // sum of one packed word per warp over the CTA, and the part of it that belongs to the warps before this one
+    auto cta_sum = [&](uint32_t (*slot)[W], uint32_t parity, uint32_t warp_total, uint32_t& before) -> uint32_t {
+        if (lane == 0) slot[parity][warp] = warp_total;
+        __syncthreads();
+        uint32_t total = 0;
+        before = 0;
+#pragma unroll
+        for (int w = 0; w < W; ++w) {
+            const uint32_t t = slot[parity][w];
+            total += t;
+            before += static_cast<uint32_t>(w) < warp ? t : 0u;
+        }
+        return total;
+    };
+
+    // Both flag sets of the lane's span for the bucket bounds (low, high): column 32 i + j of the span at bit 31 - j of
+    // word i.  Returns the lane's counts, (#low << 16) | #high.  Exact for every bit pattern: per 16-bit half, bit 15
+    // of ((bucket | 0x8000) - bound) is set iff bucket >= bound, and no borrow crosses the halves (bound <= 0x8000).
+    uint32_t ge_low[kWords], ge_high[kWords];
+    auto flag_pass = [&](uint32_t low, uint32_t high) -> uint32_t {
+        const uint32_t low2 = low * 0x10001u, high2 = high * 0x10001u;
+#pragma unroll
+        for (int i = 0; i < kWords; ++i) ge_low[i] = ge_high[i] = 0;
+        static_for<8>([&](auto p_tag) {
+            constexpr int p = decltype(p_tag)::value;
+            const uint4 a = lds128<128 * (p / 4)>(unit_base[(2 * p) % 8]);
+            const uint4 b = lds128<128 * (p / 4)>(unit_base[(2 * p + 1) % 8]);
+            const uint32_t u0 = upper_halves_set(a.x, a.y), u1 = upper_halves_set(a.z, a.w);
+            const uint32_t u2 = upper_halves_set(b.x, b.y), u3 = upper_halves_set(b.z, b.w);
+            const uint32_t f_low = static_cast<uint32_t>(
+                dp4a_ss(prmt(u2 - low2, u3 - low2, 0xFDB9u), w_second, dp4a_ss(prmt(u0 - low2, u1 - low2, 0xFDB9u), w_first, 0)));
+            const uint32_t f_high = static_cast<uint32_t>(
+                dp4a_ss(prmt(u2 - high2, u3 - high2, 0xFDB9u), w_second, dp4a_ss(prmt(u0 - high2, u1 - high2, 0xFDB9u), w_first, 0)));
+            // piece p (in read order) is byte 3 - p % 4 of word p / 4
+            constexpr uint32_t sel = p % 4 == 1 ? 0x3410u : (p % 4 == 2 ? 0x3240u : 0x3214u);
+            ge_low[p / 4] = (p % 4 == 0) ? (f_low << 24) : prmt(ge_low[p / 4], f_low, sel);
+            ge_high[p / 4] = (p % 4 == 0) ? (f_high << 24) : prmt(ge_high[p / 4], f_high, sel);
+        });
+        uint32_t mine = 0;
+#pragma unroll
+        for (int i = 0; i < kWords; ++i) {
+            ge_low[i] = prmt(ge_low[i], 0u, fix_sel);
+            ge_high[i] = prmt(ge_high[i], 0u, fix_sel);
+            mine += (__popc(ge_low[i]) << 16) | __popc(ge_high[i]);
+        }
+        return mine;
+    };
+    auto counted_pass = [&](uint32_t low, uint32_t high, uint32_t& pass_no) -> uint32_t {
+        const uint32_t mine = flag_pass(low, high);
+        uint32_t before;
+        const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, mine), before);
+        ++pass_no;
+        return total;
+    };
+
+    if (blockIdx.x < rows) request_row(blockIdx.x);
+    uint32_t use = 0, pass_no = 0;
+    uint32_t guess_low = 0;
+    uint32_t window = kWideWindowF32;
+    for (uint64_t row64 = blockIdx.x; row64 < rows; row64 += gridDim.x, ++use) {
+        const uint32_t row = static_cast<uint32_t>(row64);
+        if (!__syncthreads_and(mbar_wait_bounded(&s_bar, use & 1u, 1u << 24, &s_stop) ? 1 : 0)) {
+            s_stop = 1;
+            if (threadIdx.x == 0 && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_TIMEOUT));
+            return;
+        }
+        const size_t out_base = static_cast<size_t>(row) * k;
+
+        // ---- A: bounds around the bucket of tau_i ------------------------------------------------------------
+        uint32_t low = guess_low;
+        if (low == 0) {
+            // the (k/d)-quantile of 128 samples of the first warp's columns, taken a little low, found bit by bit
+            if (warp == 0) {
+                uint32_t sample[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) sample[c] = *reinterpret_cast<const uint16_t*>(own + c * 16 + 2) & 0x7FFFu;
+                uint32_t rank = (128u * k + d - 1) / d;
+                rank += 2u * static_cast<uint32_t>(__fsqrt_rn(static_cast<float>(rank))) + 2u;
+                if (rank > 128u) rank = 128u;
+                uint32_t q = 0;
+#pragma unroll 1
+                for (int bit = 14; bit >= 0; --bit) {
+                    const uint32_t trial = q | (1u << bit);
+                    uint32_t cnt = 0;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) cnt += sample[c] >= trial ? 1u : 0u;
+                    if (__reduce_add_sync(0xFFFFFFFFu, cnt) >= rank) q = trial;
+                }
+                if (lane == 0) s_guess = q ? q : 1u;
+            }
+            __syncthreads();
+            low = s_guess;
+        }
+        if (low > 0x7F80u) low = 0x7F80u;
+
+        // ---- B: the window ---------------------------------------------------------------------------------
+        uint32_t n_low = 0, n_high = 0;
+        bool pinned = false, moved = false, bucket_zero = false;
+#pragma unroll 1
+        for (int attempt = 0; attempt < kWideRetriesF32; ++attempt) {
+            const uint32_t total = counted_pass(low, low + window, pass_no);
+            n_low = total >> 16;
+            n_high = total & 0xFFFFu;
+            if (n_high < k && k <= n_low) {
+                pinned = true;
+                break;
+            }
+            const uint32_t per_key_x16 = max(((n_low - n_high) << 4) / window, 4u);
+            moved = true;
+            if (n_low < k) {
+                if (low == 1) {                                    // fewer than k elements outside bucket 0
+                    bucket_zero = true;
+                    break;
+                }
+                const uint32_t below = max(((k - n_low) << 4) / per_key_x16 + window / 2u, window / 2u);
+                low = low > below ? low - below : 1u;
+            } else {
+                const uint32_t above = ((n_high - k + 1u) << 4) / per_key_x16 + window / 2u;
+                low = low + above < 0x7F80u ? low + above : 0x7F80u;
+            }
+        }
+
+        // ---- C: the bucket of tau_i, then tau_i inside it ----------------------------------------------------------
+        uint32_t bucket = 0, take = 0;                             // `take` members of the bucket belong to the top k
+        if (pinned) {
+            if (threadIdx.x < 64) hist[threadIdx.x] = 0;
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t m = ge_low[i] & ~ge_high[i];
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    const uint32_t col = col0 + 32u * i + 31u - q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u16 %0, [%1+2];" : "=r"(v) : "r"(row_addr + 4u * col));
+                    atomicAdd(&hist[(v & 0x7FFFu) - low], 1u);
+                }
+            }
+            __syncthreads();
+            const uint32_t drop = n_low - k;                       // window elements below the top k, from the bottom
+            const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];
+            const uint32_t own_cnt = h.x + h.y;
+            const uint32_t before = warp_inclusive_sum(own_cnt) - own_cnt;
+            uint32_t my_bucket = 0, my_take = 0;
+            bool mine = false;
+            if (before <= drop && drop < before + h.x) {
+                mine = true;
+                my_bucket = low + 2u * lane;
+                my_take = h.x - (drop - before);
+            } else if (before + h.x <= drop && drop < before + own_cnt) {
+                mine = true;
+                my_bucket = low + 2u * lane + 1u;
+                my_take = h.y - (drop - before - h.x);
+            }
+            const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
+            const int src = who ? __ffs(who) - 1 : 0;
+            bucket = __shfl_sync(0xFFFFFFFFu, my_bucket, src);
+            take = __shfl_sync(0xFFFFFFFFu, my_take, src);
+            if (moved) {
+                window = window < kWideWindowF32 ? window * 2u : kWideWindowF32;
+            } else if (n_low - n_high > 128u * W && window > 8u) {
+                window >>= 1;                                      // many window elements per lane: a narrower one next time
+            }
+            guess_low = bucket > window / 2u ? bucket - window / 2u : 1u;
+        } else {
+            // the largest bucket v with #{bucket >= v} >= k, bit by bit (known to be 0 if the window ended there)
+            uint32_t v = 0;
+            if (!bucket_zero) {
+#pragma unroll 1
+                for (int bit = 14; bit >= 0; --bit) {
+                    const uint32_t trial = v | (1u << bit);
+                    if ((counted_pass(trial, trial, pass_no) >> 16) >= k) v = trial;
+                }
+            }
+            bucket = v;
+            guess_low = 0;
+        }
+        // the members of the bucket (bucket 0: every zero, the padding behind the row included)
+        {
+            const uint32_t total = counted_pass(bucket, bucket + 1u, pass_no);
+            if (!pinned) take = k - (total & 0xFFFFu);
+        }
+        uint32_t members[kWords];
+#pragma unroll
+        for (int i = 0; i < kWords; ++i) members[i] = ge_low[i] & ~ge_high[i];
+        // t = the largest 16-bit value with #{members: lower key bits >= t} >= take
+        uint32_t t = 0;
+#pragma unroll 1
+        for (int bit = 15; bit >= 0; --bit) {
+            const uint32_t trial = t | (1u << bit);
+            uint32_t cnt = 0;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t m = members[i];
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
+                    cnt += v >= trial ? 1u : 0u;
+                }
+            }
+            uint32_t before;
+            const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, cnt), before);
+            ++pass_no;
+            if (total >= take) t = trial;
+        }
+        if (threadIdx.x == 0 && tau_out) tau_out[row] = (bucket << 16) | t;
+        // members above t are kept, and the first ties at t in column order
+        uint32_t keep[kWords];
+        {
+            uint32_t gt[kWords], eq[kWords], packed = 0;           // (#gt << 16) | #eq of this lane
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                gt[i] = eq[i] = 0;
+                uint32_t m = members[i];
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
+                    gt[i] |= v > t ? 1u << q : 0u;
+                    eq[i] |= v == t ? 1u << q : 0u;
+                }
+                packed += (__popc(gt[i]) << 16) | __popc(eq[i]);
+            }
+            const uint32_t incl = warp_inclusive_sum(packed);
+            uint32_t warps_before;
+            const uint32_t total = cta_sum(s_sum, 0, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
+            const uint32_t ties_to_take = take - (total >> 16);
+            const uint32_t ties_before = (warps_before + incl - packed) & 0xFFFFu;
+            uint32_t room = ties_before < ties_to_take ? ties_to_take - ties_before : 0u;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t z = eq[i];
+                const uint32_t n = __popc(z);
+                if (n > room) {
+                    for (uint32_t extra = n - room; extra; --extra) z &= z - 1u;   // the highest columns go (lowest bits)
+                    room = 0;
+                } else {
+                    room -= n;
+                }
+                keep[i] = ge_high[i] | gt[i] | z;
+            }
+        }
+
+        // ---- D: every lane stages its kept entries at its offset of the row's output ----------------------------
+        const uint32_t shift = static_cast<uint32_t>(out_base) & 1u;
+        {
+            uint32_t kept_mine = 0;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) kept_mine += __popc(keep[i]);
+            const uint32_t incl = warp_inclusive_sum(kept_mine);
+            uint32_t warps_before;
+            cta_sum(s_sum, 1, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
+            uint32_t at = warps_before + incl - kept_mine;
+            const uint32_t vals_addr = smem_addr(stage_vals), cols_addr = smem_addr(stage_cols) + 2u * shift;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t m = keep[i];
+                const uint32_t colb = col0 + 32u * i + 31u;
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    const uint32_t col = colb - q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(row_addr + 4u * col));
+                    asm volatile("st.shared.u32 [%0], %1;" ::"r"(vals_addr + 4u * at), "r"(v) : "memory");
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(cols_addr + 2u * at), "h"(static_cast<uint16_t>(col)) : "memory");
+                    ++at;
+                }
+            }
+        }
+        fence_proxy_async_smem();                              // this thread's reads of the row come before the next bulk copy into it
+        __syncthreads();                                       // the stage is complete, the row buffer free
+        if (row64 + gridDim.x < rows) request_row(row64 + gridDim.x);
+
+        // ---- E: the staged entries leave: values one by one, columns in pairs --------------------------------------
+        {
+            for (uint32_t p = threadIdx.x; p < k; p += W * 32u) vals_out[out_base + p] = stage_vals[p];
+            const size_t pair_base = out_base - shift;
+            const uint32_t last = shift + k;
+            for (uint32_t p = 2u * threadIdx.x; p < last; p += 2u * W * 32u) {
+                const uint32_t e = *reinterpret_cast<const uint32_t*>(stage_cols + p);
+                const bool first = p >= shift, second = p + 1u < last;
+                if (first && second) {
+                    *reinterpret_cast<uint32_t*>(cols_out + pair_base + p) = e;
+                } else if (first) {
+                    cols_out[pair_base + p] = static_cast<int16_t>(e & 0xFFFFu);
+                } else if (second) {
+                    cols_out[pair_base + p + 1u] = static_cast<int16_t>(e >> 16);
+                }
+            }
+            if (rows_out)
+                for (uint32_t p = threadIdx.x; p < k; p += W * 32u) rows_out[out_base + p] = static_cast<int32_t>(row);
+        }
+        __syncthreads();                                       // the stage has been read: the next row may fill it
+    }
+}
+
+template <int W>
+dct_status_t launch_wide_f32(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
+                             void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
+                             cudaStream_t stream) {
+    using Lay = WideLayoutF32<W>;
+    auto kernel = mp_topk_fwd_f32_wide_kernel<W>;
+    const size_t smem = Lay::cta_bytes(k);
+    static thread_local int configured_device = -1;
+    int dev = 0;
+    DCT_CUDA_TRY(cudaGetDevice(&dev));
+    if (configured_device != dev) {
+        DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        configured_device = dev;
+    }
+    int per_sm = 0;
+    DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, W * 32, smem));
+    if (per_sm < 1) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
+    const uint32_t grid = static_cast<uint32_t>(rows < max_grid ? rows : max_grid);
+    kernel<<<grid, W * 32, smem, stream>>>(static_cast<const float*>(x_act), rows, d, ld, k, cols_out,
+                                           static_cast<uint32_t*>(vals_out), rows_out, static_cast<uint32_t*>(tau_out),
+                                           result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}
+
+}  // namespace
+
+// *handled = false: the shape is not one of this path's; the caller runs the general kernel.
+dct_status_t launch_fwd_f32_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                 int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                 dct_result_t* result, cudaStream_t stream, bool* handled) {
+    *handled = false;
+    // (beyond 3/8 of the row a post-ReLU row's threshold is next to zero, where buckets are sparse and the window
+    // rarely settles: the general kernel serves those)
+    if (d <= 2048 || d > 32768 || d % 4 != 0 || k > kWideMaxKF32 || 8ull * k > 3ull * d) return DCT_OK;
+    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || !aligned_to(cols_out, 4)) return DCT_OK;
+    *handled = true;
+    // as many warps as the row has segments of 2048 columns (the last one zero-padded)
+#define DCT_WIDE_F32_WARPS(W) \
+    if (d <= 2048u * W) return launch_wide_f32<W>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+    DCT_WIDE_F32_WARPS(2);
+    DCT_WIDE_F32_WARPS(3);
+    DCT_WIDE_F32_WARPS(4);
+    DCT_WIDE_F32_WARPS(6);
+    DCT_WIDE_F32_WARPS(8);
+    DCT_WIDE_F32_WARPS(12);
+    DCT_WIDE_F32_WARPS(16);
+#undef DCT_WIDE_F32_WARPS
+    *handled = false;
+    return DCT_OK;
+}
+
+}  // namespace dct

@@ -24,8 +24,6 @@
 // A row with fewer than k non-zeros (tau_i = 0) keeps its non-zeros and fills up with its first zeros.  Rows for
 // which the window does not settle take the bit-serial slow path of mp_warp.cuh.  The result never depends on the
 // guesses.
-#include <utility>
-
 #include "common.cuh"
 #include "mp_warp.cuh"
 
@@ -57,24 +55,6 @@ template <int E8> struct SpanLayout {
     }
 };
 
-template <int kOffset> __device__ __forceinline__ uint4 lds128(uint32_t addr) {      // 128 bits at addr + kOffset
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr), "n"(kOffset));
-    return v;
-}
-// f(integral_constant<int, 0>) ... f(integral_constant<int, N - 1>): a loop whose index is a constant expression
-template <typename F, int... Is> __device__ __forceinline__ void static_for_impl(F&& f, std::integer_sequence<int, Is...>) {
-    (f(std::integral_constant<int, Is>{}), ...);
-}
-template <int N, typename F> __device__ __forceinline__ void static_for(F&& f) {
-    static_for_impl(f, std::make_integer_sequence<int, N>{});
-}
-__device__ __forceinline__ uint32_t bfind(uint32_t x) {       // position of the highest set bit
-    uint32_t d;
-    asm("bfind.u32 %0, %1;" : "=r"(d) : "r"(x));
-    return d;
-}
 // The flags key >= low and key >= high of the 8 bf16 of one 16-byte unit, element j at bit 7 - j (the walks over
 // the flags run from the highest bit down, i.e. from the first column on).  Integer compares on the keys, exact for
 // every bit pattern: per 16-bit half, bit 15 of ((x | 0x8000) - bound) is set iff key(x) >= bound, and no borrow

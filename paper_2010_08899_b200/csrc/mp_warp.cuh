@@ -2,6 +2,7 @@
 // threshold tau_i and packs the row (bf16: mp_pack.cu; fp32: mp_pack_f32.cu).
 #pragma once
 #include <type_traits>
+#include <utility>
 
 #include "common.cuh"
 
@@ -24,6 +25,24 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
 __device__ __forceinline__ int dp4a_ss(uint32_t a, uint32_t b, int c) {     // signed 8-bit dot product + c
     int d;
     asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+template <int kOffset> __device__ __forceinline__ uint4 lds128(uint32_t addr) {      // 128 bits at addr + kOffset
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4+%5];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr), "n"(kOffset));
+    return v;
+}
+// f(integral_constant<int, 0>) ... f(integral_constant<int, N - 1>): a loop whose index is a constant expression
+template <typename F, int... Is> __device__ __forceinline__ void static_for_impl(F&& f, std::integer_sequence<int, Is...>) {
+    (f(std::integral_constant<int, Is>{}), ...);
+}
+template <int N, typename F> __device__ __forceinline__ void static_for(F&& f) {
+    static_for_impl(f, std::make_integer_sequence<int, N>{});
+}
+__device__ __forceinline__ uint32_t bfind(uint32_t x) {       // position of the highest set bit
+    uint32_t d;
+    asm("bfind.u32 %0, %1;" : "=r"(d) : "r"(x));
     return d;
 }
 // bit j set iff key(element j) >= low, for the 8 bf16 of one int4; exact for every bit pattern (low <= 0x8000).
@@ -214,6 +233,10 @@ dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, 
 
 // The fp32 kernels live in their own translation unit.
 dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                 int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                 dct_result_t* result, cudaStream_t stream, bool* handled);
+// fp32 rows of 2049..32768 columns, one CTA per row (mp_pack_f32_wide.cu).
+dct_status_t launch_fwd_f32_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                  int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                  dct_result_t* result, cudaStream_t stream, bool* handled);
 

@@ -305,6 +305,34 @@ def test_mp_bf16_wide_rows(d):
         assert int(cols.max()) < d
 
 
+@pytest.mark.parametrize("d", [2052, 4096, 4100, 8192, 12000, 16384, 24580, 32768])
+def test_mp_f32_rows_wider_than_2048(d):
+    """fp32 rows of more than 2048 columns that the warp-per-row kernels leave out (every k beyond 4096 columns,
+    the denser k up to 4096) are packed by a CTA per row, each warp looking after 2048 columns: sparse and denser
+    k, rows of very different scales (the window has to move), dead rows, rows where everything ties, rows with
+    fewer than k non-zeros, rows of tiny values inside bucket 0, rows of a few distinct values (many members in one
+    bucket, ties inside it), and more rows than CTAs, so that every CTA works through several rows."""
+    rows = 900 if d <= 8192 else 400
+    x = inputs.mp_activations(rows, d, 191 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=192 + d)
+    sign = torch.where(inputs.dp_gaussian(rows * d, 193 + d, G.DEV).view(rows, d) > 0, 1.0, -1.0)
+    scale = torch.tensor([1.0, 30.0, 1e-2, 1.0, 1e3, 1.0, 1.0], device=G.DEV).repeat(rows // 7 + 1)[:rows]
+    x = x * sign * scale[:, None]
+    x[3] = 0.0
+    x[4] = -1.25
+    x[5, 300:] = 0.0
+    x[6] = inputs.quantize_mantissa(x[6], 1)
+    x[7::50] = inputs.quantize_mantissa(x[7::50], 2)
+    x[8] = 3.0e38
+    x[9] = x[9] * 1e-41                          # denormals: every key in bucket 0
+    x[10, 100:] = x[10, 100:] * 1e-42
+    x[11::50] = inputs.quantize_mantissa(x[11::50], 9)    # few distinct values inside a bucket
+    x = x.contiguous()
+    gx = inputs.mp_gradients(rows, d, 194 + d, dtype=torch.float32, device=G.DEV)
+    for k in sorted({d // 7, min(d // 4 + 1, 4095), min(3 * d // 8, 4096)} | ({1, 33, d // 20} if d > 4096 else set())):
+        cols = _compare_fwd_bwd(x, gx, d, k, want_rows=(k == 33))
+        assert int(cols.max()) < d
+
+
 @pytest.mark.parametrize("d", [8200, 12288, 16384, 20000, 32768])
 def test_mp_bf16_rows_wider_than_8192(d):
     """bf16 rows of more than 8192 columns are packed by a CTA per row (4 or 8 warps, each looking after 4096 columns):
