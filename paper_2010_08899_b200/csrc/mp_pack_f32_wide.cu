@@ -12,11 +12,12 @@
 //      The units are read in an XOR-swizzled order (no bank conflicts although the lanes' spans are 256 bytes
 //      apart); a byte permutation puts the flags back in column order.  Counts are summed over the CTA; the window
 //      moves until n_high < k <= n_low.
-//   C  the buckets of the window elements go into a 64-bin histogram, which gives the bucket of tau_i and how many of
-//      its members belong to the top k.  A second flag pass at that bucket marks the members; their lower 16 key bits
-//      are then searched bit by bit (16 counting rounds over the few members, summed over the CTA), which gives the
-//      exact 31-bit tau_i; members above it and the first ties, in column order, join the columns above the bucket.
-//   D  a scan over the kept counts gives every lane its offset in the row's output; it stages column and value.
+//   C  a radix select over the window elements: their buckets go into a 64-bin histogram, which gives the bucket of
+//      tau_i and how many of its members belong to the top k; the members' lower 16 key bits follow in digits of
+//      6, 6 and 4 bits (a round is skipped as soon as one member is left), which gives the exact 31-bit tau_i.
+//   D  kept are the columns above the bucket, the members above tau_i and the first ties in column order.  One scan
+//      over the CTA gives every lane its offset in the row's output and its share of the ties; it stages column
+//      and value.
 //   E  the staged entries leave as coalesced stores while the row buffer already receives the CTA's next row.
 // A row whose window does not settle finds its bucket bit by bit (15 counting passes) and goes on from C's second
 // half; a row with fewer than k elements outside bucket 0 starts there.  The result never depends on the guesses.
@@ -33,7 +34,7 @@ constexpr int kWideRetriesF32 = 6;
 template <int W> struct WideLayoutF32 {
     static constexpr uint32_t kSegBytes = 8192u;             // one warp's 2048 columns
     static constexpr uint32_t kRowBytes = W * kSegBytes;
-    static constexpr uint32_t kHistBytes = 256u;
+    static constexpr uint32_t kHistBytes = 1024u;            // four tables of 64 bins
     __host__ __device__ static constexpr uint32_t vals_bytes(uint32_t k) { return 4u * k; }
     __host__ __device__ static constexpr uint32_t cta_bytes(uint32_t k) {
         return (kRowBytes + kHistBytes + vals_bytes(k) + 2u * (k + 2u) + 127u) & ~127u;
@@ -171,6 +172,7 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
             return;
         }
         const size_t out_base = static_cast<size_t>(row) * k;
+        for (uint32_t b = threadIdx.x; b < Lay::kHistBytes / 4; b += W * 32u) hist[b] = 0;   // (a barrier follows in B)
 
         // ---- A: bounds around the bucket of tau_i ------------------------------------------------------------
         uint32_t low = guess_low;
@@ -227,48 +229,73 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
         }
 
         // ---- C: the bucket of tau_i, then tau_i inside it ----------------------------------------------------------
+        // A radix select over the window elements: their bucket (64 bins), then the lower 16 key bits of the members of
+        // the chosen bucket in digits of 6, 6 and 4 bits.  rank_in(h, r): the bin of h that holds the r-th largest
+        // element, how many of that bin belong to the top r, and how many the bin holds.
+        auto rank_in = [&](const uint32_t* h64, uint32_t r, uint32_t& bin_take, uint32_t& bin_count) -> uint32_t {
+            const uint2 h = reinterpret_cast<const uint2*>(h64)[31u - lane];   // lane owns bins 63 - 2 lane (h.y), 62 - 2 lane
+            const uint32_t own_cnt = h.x + h.y;
+            const uint32_t before = warp_inclusive_sum(own_cnt) - own_cnt;      // elements in higher bins
+            uint32_t my_bin = 0, my_take = 0, my_count = 0;
+            bool mine = false;
+            if (before < r && r <= before + h.y) {
+                mine = true;
+                my_bin = 63u - 2u * lane;
+                my_take = r - before;
+                my_count = h.y;
+            } else if (before + h.y < r && r <= before + own_cnt) {
+                mine = true;
+                my_bin = 62u - 2u * lane;
+                my_take = r - before - h.y;
+                my_count = h.x;
+            }
+            const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
+            const int src = who ? __ffs(who) - 1 : 0;
+            bin_take = __shfl_sync(0xFFFFFFFFu, my_take, src);
+            bin_count = __shfl_sync(0xFFFFFFFFu, my_count, src);
+            return __shfl_sync(0xFFFFFFFFu, my_bin, src);
+        };
         uint32_t bucket = 0, take = 0;                             // `take` members of the bucket belong to the top k
+        uint32_t members[kWords];
         if (pinned) {
-            if (threadIdx.x < 64) hist[threadIdx.x] = 0;
-            __syncthreads();
 #pragma unroll
             for (int i = 0; i < kWords; ++i) {
                 uint32_t m = ge_low[i] & ~ge_high[i];
                 while (m) {
                     const uint32_t q = bfind(m);
                     m ^= 1u << q;
-                    const uint32_t col = col0 + 32u * i + 31u - q;
                     uint32_t v;
-                    asm volatile("ld.shared.u16 %0, [%1+2];" : "=r"(v) : "r"(row_addr + 4u * col));
+                    asm volatile("ld.shared.u16 %0, [%1+2];" : "=r"(v) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
                     atomicAdd(&hist[(v & 0x7FFFu) - low], 1u);
                 }
             }
             __syncthreads();
-            const uint32_t drop = n_low - k;                       // window elements below the top k, from the bottom
-            const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];
-            const uint32_t own_cnt = h.x + h.y;
-            const uint32_t before = warp_inclusive_sum(own_cnt) - own_cnt;
-            uint32_t my_bucket = 0, my_take = 0;
-            bool mine = false;
-            if (before <= drop && drop < before + h.x) {
-                mine = true;
-                my_bucket = low + 2u * lane;
-                my_take = h.x - (drop - before);
-            } else if (before + h.x <= drop && drop < before + own_cnt) {
-                mine = true;
-                my_bucket = low + 2u * lane + 1u;
-                my_take = h.y - (drop - before - h.x);
-            }
-            const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
-            const int src = who ? __ffs(who) - 1 : 0;
-            bucket = __shfl_sync(0xFFFFFFFFu, my_bucket, src);
-            take = __shfl_sync(0xFFFFFFFFu, my_take, src);
+            uint32_t bucket_count;
+            bucket = low + rank_in(hist, k - n_high, take, bucket_count);
             if (moved) {
                 window = window < kWideWindowF32 ? window * 2u : kWideWindowF32;
             } else if (n_low - n_high > 128u * W && window > 8u) {
                 window >>= 1;                                      // many window elements per lane: a narrower one next time
             }
             guess_low = bucket > window / 2u ? bucket - window / 2u : 1u;
+            // window elements above the bucket join the kept columns, those inside it are its members
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t m = ge_low[i] & ~ge_high[i];
+                members[i] = 0;
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
+                    const uint32_t b = (v >> 16) & 0x7FFFu;
+                    if (b > bucket) ge_high[i] |= 1u << q;
+                    if (b == bucket) {
+                        members[i] |= 1u << q;
+                        atomicAdd(&hist[64u + ((v >> 10) & 63u)], 1u);
+                    }
+                }
+            }
         } else {
             // the largest bucket v with #{bucket >= v} >= k, bit by bit (known to be 0 if the window ended there)
             uint32_t v = 0;
@@ -281,62 +308,97 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
             }
             bucket = v;
             guess_low = 0;
-        }
-        // the members of the bucket (bucket 0: every zero, the padding behind the row included)
-        {
-            const uint32_t total = counted_pass(bucket, bucket + 1u, pass_no);
-            if (!pinned) take = k - (total & 0xFFFFu);
-        }
-        uint32_t members[kWords];
-#pragma unroll
-        for (int i = 0; i < kWords; ++i) members[i] = ge_low[i] & ~ge_high[i];
-        // t = the largest 16-bit value with #{members: lower key bits >= t} >= take
-        uint32_t t = 0;
-#pragma unroll 1
-        for (int bit = 15; bit >= 0; --bit) {
-            const uint32_t trial = t | (1u << bit);
-            uint32_t cnt = 0;
+            // the members of the bucket (bucket 0: every zero, the padding behind the row included)
+            take = k - (counted_pass(bucket, bucket + 1u, pass_no) & 0xFFFFu);
 #pragma unroll
             for (int i = 0; i < kWords; ++i) {
-                uint32_t m = members[i];
+                uint32_t m = members[i] = ge_low[i] & ~ge_high[i];
                 while (m) {
                     const uint32_t q = bfind(m);
                     m ^= 1u << q;
-                    uint32_t v;
-                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
-                    cnt += v >= trial ? 1u : 0u;
+                    uint32_t lo16;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo16) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
+                    atomicAdd(&hist[64u + (lo16 >> 10)], 1u);
                 }
             }
-            uint32_t before;
-            const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, cnt), before);
-            ++pass_no;
-            if (total >= take) t = trial;
+        }
+        __syncthreads();
+        // t = the take-th largest of the members' lower 16 key bits: up to three digits, fewer if a bin of one is met
+        uint32_t t = 0;
+        {
+            uint32_t count;
+            uint32_t prefix = rank_in(hist + 64, take, take, count);        // bits 15..10
+            int known = 6;                                                  // upper bits of t in `prefix`
+#pragma unroll 1
+            for (int round = 0; round < 2 && count > 1u; ++round) {
+                const int digit_bits = round == 0 ? 6 : 4;
+                uint32_t* h = hist + 128 + 64 * round;
+#pragma unroll
+                for (int i = 0; i < kWords; ++i) {
+                    uint32_t m = members[i];
+                    while (m) {
+                        const uint32_t q = bfind(m);
+                        m ^= 1u << q;
+                        uint32_t lo16;
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo16) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
+                        if ((lo16 >> (16 - known)) == prefix)
+                            atomicAdd(&h[(lo16 >> (16 - known - digit_bits)) & ((1u << digit_bits) - 1u)], 1u);
+                    }
+                }
+                __syncthreads();
+                prefix = (prefix << digit_bits) | rank_in(h, take, take, count);
+                known += digit_bits;
+            }
+            if (known == 16) {
+                t = prefix;
+            } else {
+                // one member left under the prefix: its owner announces it
+#pragma unroll
+                for (int i = 0; i < kWords; ++i) {
+                    uint32_t m = members[i];
+                    while (m) {
+                        const uint32_t q = bfind(m);
+                        m ^= 1u << q;
+                        uint32_t lo16;
+                        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo16) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
+                        if ((lo16 >> (16 - known)) == prefix) s_guess = lo16;
+                    }
+                }
+                __syncthreads();
+                t = s_guess;
+            }
         }
         if (threadIdx.x == 0 && tau_out) tau_out[row] = (bucket << 16) | t;
-        // members above t are kept, and the first ties at t in column order
-        uint32_t keep[kWords];
+
+        // ---- D: every lane stages its kept entries at its offset of the row's output ----------------------------
+        // kept: the columns above the bucket, the members above t, and the first ties at t in column order.  One scan
+        // of (#certain << 16 | #ties) over the CTA gives every lane both its offset and its share of the ties.
+        const uint32_t shift = static_cast<uint32_t>(out_base) & 1u;
         {
-            uint32_t gt[kWords], eq[kWords], packed = 0;           // (#gt << 16) | #eq of this lane
+            uint32_t keep[kWords], eq[kWords], packed = 0;
 #pragma unroll
             for (int i = 0; i < kWords; ++i) {
-                gt[i] = eq[i] = 0;
+                keep[i] = ge_high[i];
+                eq[i] = 0;
                 uint32_t m = members[i];
                 while (m) {
                     const uint32_t q = bfind(m);
                     m ^= 1u << q;
-                    uint32_t v;
-                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
-                    gt[i] |= v > t ? 1u << q : 0u;
-                    eq[i] |= v == t ? 1u << q : 0u;
+                    uint32_t lo16;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo16) : "r"(row_addr + 4u * (col0 + 32u * i + 31u - q)));
+                    keep[i] |= lo16 > t ? 1u << q : 0u;
+                    eq[i] |= lo16 == t ? 1u << q : 0u;
                 }
-                packed += (__popc(gt[i]) << 16) | __popc(eq[i]);
+                packed += (__popc(keep[i]) << 16) | __popc(eq[i]);
             }
             const uint32_t incl = warp_inclusive_sum(packed);
             uint32_t warps_before;
-            const uint32_t total = cta_sum(s_sum, 0, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
-            const uint32_t ties_to_take = take - (total >> 16);
-            const uint32_t ties_before = (warps_before + incl - packed) & 0xFFFFu;
+            const uint32_t total = cta_sum(s_sum, use & 1u, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
+            const uint32_t ties_to_take = k - (total >> 16);
+            const uint32_t mine_before = warps_before + incl - packed;
+            const uint32_t ties_before = mine_before & 0xFFFFu;
             uint32_t room = ties_before < ties_to_take ? ties_to_take - ties_before : 0u;
+            uint32_t at = (mine_before >> 16) + (ties_before < ties_to_take ? ties_before : ties_to_take);
 #pragma unroll
             for (int i = 0; i < kWords; ++i) {
                 uint32_t z = eq[i];
@@ -347,20 +409,8 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
                 } else {
                     room -= n;
                 }
-                keep[i] = ge_high[i] | gt[i] | z;
+                keep[i] |= z;
             }
-        }
-
-        // ---- D: every lane stages its kept entries at its offset of the row's output ----------------------------
-        const uint32_t shift = static_cast<uint32_t>(out_base) & 1u;
-        {
-            uint32_t kept_mine = 0;
-#pragma unroll
-            for (int i = 0; i < kWords; ++i) kept_mine += __popc(keep[i]);
-            const uint32_t incl = warp_inclusive_sum(kept_mine);
-            uint32_t warps_before;
-            cta_sum(s_sum, 1, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
-            uint32_t at = warps_before + incl - kept_mine;
             const uint32_t vals_addr = smem_addr(stage_vals), cols_addr = smem_addr(stage_cols) + 2u * shift;
 #pragma unroll
             for (int i = 0; i < kWords; ++i) {
