@@ -159,11 +159,11 @@ class HotPath:
             st = L.dct_mp_pack_bwd(self.gx[j].data_ptr(), 1, rows, d, d, k, cols_p, gv_p, res_b, s)
             assert st == 0, st
         rec()
-        # kernels of this library per step: the select enqueues 12 (reset, 3 sample passes, filter, decide,
-        # 3 candidate passes, 3 full passes that return at once) from n = 2^25 and 4 (reset + 3 passes) below;
+        # kernels of this library per step: the select enqueues 7 (reset, 2 sample passes, filter, 3 passes over
+        # the candidates or, as the fall-back, the vector) from n = 2^25 and 4 (reset + 3 passes) below;
         # each compress is a reset kernel + the streaming kernel; each MP iteration a forward and a backward kernel
         # (the backward pack resets its result block inside the kernel)
-        self.launches += (12 if n >= (1 << 25) else 4) + 2 * c["dp_iters"] + 2 * c["mp_iters"]
+        self.launches += (7 if n >= (1 << 25) else 4) + 2 * c["dp_iters"] + 2 * c["mp_iters"]
 
     def time_mp_parts(self, stream, reps):
         """Forward and backward pack timed on their own (after the main measurement)."""
@@ -212,6 +212,27 @@ class HotPath:
                 b.synchronize()
             ms = a.elapsed_time(b) / reps
             out[name] = {"ms": ms, "k": k, "GBps": (rows * d * 2 + rows * k * 4) / (ms * 1e-3) / 1e9}
+        return out
+
+    def time_wide_rows(self, stream, reps=10):
+        """The forward pack on rows wider than the warp-per-row kernels take (one CTA per row): 4096 x 32768 bf16 at
+        k = 1638 and 8192 x 8192 fp32 at k = 410 (5 %), each matrix (256 MiB) larger than L2."""
+        B, out = self.B, {}
+        for name, rows, d, k, dtype in (("mp_fwd_bf16_4096x32768_k1638", 4096, 32768, 1638, torch.bfloat16),
+                                        ("mp_fwd_fp32_8192x8192_k410", 8192, 8192, 410, torch.float32)):
+            x = inputs.mp_activations(rows, d, 900 + d, dtype=dtype, device=self.dev, col_scale_seed=901 + d)
+            cols = torch.empty(rows * k, dtype=torch.int16, device=self.dev)
+            vals = torch.empty(rows * k, dtype=dtype, device=self.dev)
+            for phase in range(2):
+                a = _record(stream)
+                for i in range(reps):
+                    B.dct_mp_topk_pack_fwd(x, rows, d, d, k, cols, vals, None, None, None, stream)
+                b = _record(stream)
+                b.synchronize()
+            ms = a.elapsed_time(b) / reps
+            es = x.element_size()
+            out[name] = {"ms": ms, "GBps": (rows * d * es + rows * k * (2 + es)) / (ms * 1e-3) / 1e9}
+            del x, cols, vals
         return out
 
     def time_c3(self, stream, iters=20):
@@ -699,6 +720,7 @@ def main():
     parts["beyond_the_step"] = hp.time_extras(stream)
     if args.workload == DEFAULT_WORKLOAD:
         parts["c3"] = hp.time_c3(stream)
+        parts["wide_rows"] = hp.time_wide_rows(stream)
     fwd_bytes = b0["mp_fwd"] / cfg["mp_iters"]
     roofline_mp = {
         "kernel": "mp_topk_fwd_bf16_warp_kernel<16,10>", "bound": "hbm", "achieved": parts["mp_fwd"]["GBps"], "peak": peak,
