@@ -1,16 +1,16 @@
 // dct_mp_topk_pack_fwd, fp32, rows of more than 2048 columns (up to 32768) that the warp-per-row kernels do not serve:
 // Algorithm 2 (DCT-MP), forward pass -- one CTA of W warps per row, warp w looking after the columns
-// [2048 w, 2048 w + 2048) and lane l of it after 64 of them.
+// [1024 w, 1024 w + 1024) and lane l of it after 32 of them (KW = 1; twice that with KW = 2).
 //
 // The row arrives by one bulk copy (TMA engine) into shared memory as it lies in HBM.  The steps are those of the
 // bf16 kernel for wide rows (mp_pack_span.cu), on two levels, because a key has 31 bits and the packed compares 15:
 //   A  two bounds around the *bucket* of tau_i (a bucket = the upper 15 bits of the key, the bf16 truncation of |x|):
 //      the previous row's bucket minus half a window, or a quantile of 128 samples of the row.
-//   B  one pass over the lane's sixteen 16-byte units gives two flags per column (bucket >= low, bucket >= high) as
+//   B  one pass over the lane's eight (sixteen) 16-byte units gives two flags per column (bucket >= low, bucket >= high) as
 //      bits in registers: the upper halves of the fp32 words are gathered by byte permutes, the compares are integer
 //      subtractions on the packed halves, and a byte permutation plus two dot-product instructions collect 8 flags.
-//      The units are read in an XOR-swizzled order (no bank conflicts although the lanes' spans are 256 bytes
-//      apart); a byte permutation puts the flags back in column order.  Counts are summed over the CTA; the window
+//      The units are read in an XOR-swizzled order (no bank conflicts although the lanes' spans are a multiple of
+//      128 bytes apart); a byte permutation puts the flags back in column order.  Counts are summed over the CTA; the window
 //      moves until n_high < k <= n_low.
 //   C  a radix select over the window elements: their buckets go into a 64-bin histogram, which gives the bucket of
 //      tau_i and how many of its members belong to the top k; the members' lower 16 key bits follow in digits of
@@ -31,8 +31,8 @@ constexpr uint32_t kWideWindowF32 = 64;           // widest window, in buckets (
 constexpr uint32_t kWideMaxKF32 = 4096;
 constexpr int kWideRetriesF32 = 6;
 
-template <int W> struct WideLayoutF32 {
-    static constexpr uint32_t kSegBytes = 8192u;             // one warp's 2048 columns
+template <int W, int KW> struct WideLayoutF32 {
+    static constexpr uint32_t kSegBytes = 4096u * KW;        // one warp's 1024 KW columns
     static constexpr uint32_t kRowBytes = W * kSegBytes;
     static constexpr uint32_t kHistBytes = 1024u;            // four tables of 64 bins
     __host__ __device__ static constexpr uint32_t vals_bytes(uint32_t k) { return 4u * k; }
@@ -46,19 +46,19 @@ __device__ __forceinline__ uint32_t upper_halves_set(uint32_t a, uint32_t b) {
     return prmt(a, b, 0x7632u) | 0x80008000u;
 }
 
-template <int W>
+template <int W, int KW>
 __global__ void __launch_bounds__(W * 32)
 mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                             int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
                             int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
                             dct_result_t* __restrict__ result) {
-    using Lay = WideLayoutF32<W>;
-    constexpr int kWords = 2;                                  // 64 columns per lane
-    constexpr uint32_t kLaneCols = 64u;
+    using Lay = WideLayoutF32<W, KW>;
+    constexpr int kWords = KW;                                 // 32 KW columns per lane
+    constexpr uint32_t kLaneCols = 32u * KW;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
     unsigned char* base = smem_raw;
-    const unsigned char* own = base + warp * Lay::kSegBytes + lane * 256u;
+    const unsigned char* own = base + warp * Lay::kSegBytes + lane * (4u * kLaneCols);
     uint32_t* hist = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
     uint32_t* stage_vals = hist + Lay::kHistBytes / 4;
     uint16_t* stage_cols = reinterpret_cast<uint16_t*>(stage_vals + k);
@@ -78,6 +78,7 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
     for (uint32_t b = row_bytes + threadIdx.x * 16u; b < Lay::kRowBytes; b += W * 512u)
         *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
+    chain_wait_previous();                                     // set-up done: the inputs may come from the previous kernel
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
         result->status = DCT_OK;
         result->reserved = 0;
@@ -86,7 +87,7 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
         result->n_gt = 0;
         result->n_eq = 0;
     }
-    // Step c of a pass reads the unit (swz ^ c % 8) + 8 (c / 8) of the lane's sixteen; steps 2p and 2p + 1 make up the
+    // Step c of a pass reads the unit (swz ^ c % 8) + 8 (c / 8) of the lane's 8 KW; steps 2p and 2p + 1 make up the
     // 32-byte piece (p % 4 ^ swz / 2) + 4 (p / 4), its upper half first if swz is odd.
     const uint32_t swz = lane & 7u;
     const uint32_t fix_sel = 0x3210u ^ (0x1111u * (swz >> 1));
@@ -96,7 +97,7 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
 #pragma unroll
     for (int c = 0; c < 8; ++c) unit_base[c] = smem_addr(own) ^ (16u * (swz ^ static_cast<uint32_t>(c)));
     const uint32_t row_addr = smem_addr(base);
-    const uint32_t col0 = warp * 2048u + lane * kLaneCols;     // first column of the lane's span
+    const uint32_t col0 = (warp * 32u + lane) * kLaneCols;     // first column of the lane's span
 
     auto request_row = [&](uint64_t r) {
         if (threadIdx.x == 0) {
@@ -128,7 +129,7 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
         const uint32_t low2 = low * 0x10001u, high2 = high * 0x10001u;
 #pragma unroll
         for (int i = 0; i < kWords; ++i) ge_low[i] = ge_high[i] = 0;
-        static_for<8>([&](auto p_tag) {
+        static_for<4 * KW>([&](auto p_tag) {
             constexpr int p = decltype(p_tag)::value;
             const uint4 a = lds128<128 * (p / 4)>(unit_base[(2 * p) % 8]);
             const uint4 b = lds128<128 * (p / 4)>(unit_base[(2 * p + 1) % 8]);
@@ -453,14 +454,15 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
         }
         __syncthreads();                                       // the stage has been read: the next row may fill it
     }
+    chain_release_next();
 }
 
-template <int W>
+template <int W, int KW>
 dct_status_t launch_wide_f32(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
                              void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
                              cudaStream_t stream) {
-    using Lay = WideLayoutF32<W>;
-    auto kernel = mp_topk_fwd_f32_wide_kernel<W>;
+    using Lay = WideLayoutF32<W, KW>;
+    auto kernel = mp_topk_fwd_f32_wide_kernel<W, KW>;
     const size_t smem = Lay::cta_bytes(k);
     static thread_local int configured_device = -1;
     int dev = 0;
@@ -476,10 +478,9 @@ dct_status_t launch_wide_f32(const void* x_act, uint32_t rows, uint32_t d, uint3
     if (sms <= 0) return DCT_ERR_CUDA;
     const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
     const uint32_t grid = static_cast<uint32_t>(rows < max_grid ? rows : max_grid);
-    kernel<<<grid, W * 32, smem, stream>>>(static_cast<const float*>(x_act), rows, d, ld, k, cols_out,
-                                           static_cast<uint32_t*>(vals_out), rows_out, static_cast<uint32_t*>(tau_out),
-                                           result);
-    DCT_CUDA_TRY(cudaGetLastError());
+    DCT_CUDA_TRY(launch_chained_smem(kernel, grid, static_cast<unsigned>(W * 32), smem, stream,
+                                     static_cast<const float*>(x_act), rows, d, ld, k, cols_out,
+                                     static_cast<uint32_t*>(vals_out), rows_out, static_cast<uint32_t*>(tau_out), result));
     return DCT_OK;
 }
 
@@ -495,17 +496,27 @@ dct_status_t launch_fwd_f32_wide(const void* x_act, uint32_t rows, uint32_t d, u
     if (d <= 2048 || d > 32768 || d % 4 != 0 || k > kWideMaxKF32 || 8ull * k > 3ull * d) return DCT_OK;
     if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || !aligned_to(cols_out, 4)) return DCT_OK;
     *handled = true;
-    // as many warps as the row has segments of 2048 columns (the last one zero-padded)
+    // As many warps as the row has segments of 1024 or 2048 columns (the last one zero-padded): 64 columns per lane,
+    // but 32 for rows of up to 4096 columns, which would otherwise be left with two warps (measured: 8 to 10 %
+    // faster there, 2 to 10 % slower on wider rows, where the CTA-wide steps weigh more than the lanes' own).
+    const bool narrow_spans = d <= 4096;
+    if (narrow_spans) {
 #define DCT_WIDE_F32_WARPS(W) \
-    if (d <= 2048u * W) return launch_wide_f32<W>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
-    DCT_WIDE_F32_WARPS(2);
-    DCT_WIDE_F32_WARPS(3);
-    DCT_WIDE_F32_WARPS(4);
-    DCT_WIDE_F32_WARPS(6);
-    DCT_WIDE_F32_WARPS(8);
-    DCT_WIDE_F32_WARPS(12);
-    DCT_WIDE_F32_WARPS(16);
+    if (d <= 1024u * W) return launch_wide_f32<W, 1>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+        DCT_WIDE_F32_WARPS(3);
+        DCT_WIDE_F32_WARPS(4);
 #undef DCT_WIDE_F32_WARPS
+    } else {
+#define DCT_WIDE_F32_WARPS(W) \
+    if (d <= 2048u * W) return launch_wide_f32<W, 2>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+        DCT_WIDE_F32_WARPS(3);
+        DCT_WIDE_F32_WARPS(4);
+        DCT_WIDE_F32_WARPS(6);
+        DCT_WIDE_F32_WARPS(8);
+        DCT_WIDE_F32_WARPS(12);
+        DCT_WIDE_F32_WARPS(16);
+#undef DCT_WIDE_F32_WARPS
+    }
     *handled = false;
     return DCT_OK;
 }
