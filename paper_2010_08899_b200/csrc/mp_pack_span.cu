@@ -467,23 +467,22 @@ dct_status_t launch_span(const void* x_act, uint32_t rows, uint32_t d, uint32_t 
 // ------------------------------------------------------------------------------------------
 // The same steps as above with a CTA in the place of the warp: warp w looks after the columns [4096 w, 4096 w + 4096)
 // of the row (lane l of it after 128 of them), counts and offsets are summed over the warps through shared memory, and
-// the histogram of the window elements is the CTA's.  Several CTAs share an SM, so one CTA's load overlaps another's
-// work.  A row whose window does not settle is not handed to another routine: its threshold is found bit by bit
-// (15 counting passes) and the row is then packed with a window of one key, whose elements -- all ties at tau_i --
-// are taken as bits in column order, without lists.
-constexpr uint32_t kWideListLen = 8;              // window elements a lane can take
-constexpr uint32_t kWideListStride = 9;
+// the histogram of the window elements is the CTA's.  No lists: a lane walks the window bits of its span twice, once
+// for the histogram and once, with tau_i known, to add the elements above tau_i to its kept bits and to mark the
+// ties; one scan over the CTA then gives every lane its offset in the row's output and its share of the ties.
+// Several CTAs share an SM, so one CTA's load overlaps another's work.  A row whose window does not settle is not
+// handed to another routine: its threshold is found bit by bit (15 counting passes) and the row is then packed
+// with a window of one key, whose elements all tie at tau_i.
 constexpr uint32_t kWideMaxK = 2300;
 constexpr int kWideRetries = 6;
+constexpr uint32_t kWideShrink = 3;               // window elements per lane (on average) from which the window narrows
 
 template <int W> struct WideLayout {
     static constexpr uint32_t kSegBytes = 8192u;             // one warp's 4096 columns
     static constexpr uint32_t kRowBytes = W * kSegBytes;
-    static constexpr uint32_t kHistBytes = 512u;
-    static constexpr uint32_t kListBytes = W * 32u * kWideListStride * 4u;
+    static constexpr uint32_t kHistBytes = 256u;
     __host__ __device__ static constexpr uint32_t cta_bytes(uint32_t k) {
-        const uint32_t stage = (4u * (k + 2u) + 15u) & ~15u;
-        return (kRowBytes + kHistBytes + (kListBytes > stage ? kListBytes : stage) + 127u) & ~127u;
+        return (kRowBytes + kHistBytes + 4u * (k + 2u) + 127u) & ~127u;
     }
 };
 
@@ -501,13 +500,11 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     unsigned char* base = smem_raw;
     const unsigned char* own = base + warp * Lay::kSegBytes + lane * 256u;
     uint32_t* hist = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
-    uint32_t* lists = hist + Lay::kHistBytes / 4;
-    uint32_t* stage = lists;
+    uint32_t* stage = hist + Lay::kHistBytes / 4;
     __shared__ uint64_t s_bar;
     __shared__ uint32_t s_stop;
     __shared__ uint32_t s_cnt[2][W];                           // per-warp packed counts (double-buffered across passes)
-    __shared__ uint32_t s_max[2][W];
-    __shared__ uint32_t s_sum[2][W];                           // per-warp totals for the two prefix sums of a row
+    __shared__ uint32_t s_sum[2][W];                           // per-warp totals of the row's scan (double-buffered across rows)
     __shared__ uint32_t s_guess;
 
     if (threadIdx.x == 0) {
@@ -520,6 +517,7 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     for (uint32_t b = row_bytes + threadIdx.x * 16u; b < Lay::kRowBytes; b += W * 512u)
         *reinterpret_cast<uint4*>(base + b) = make_uint4(0, 0, 0, 0);
     __syncthreads();
+    chain_wait_previous();                                     // set-up done: the inputs may come from the previous kernel
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
         result->status = DCT_OK;
         result->reserved = 0;
@@ -632,38 +630,27 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 
         // ---- B: the window ---------------------------------------------------------------------------
         uint32_t n_low = 0, n_high = 0;
-        bool pinned = false, moved = false, crowded = false;
-        uint32_t width = window;                                // of the window that is finally used (1: exact mode)
+        bool pinned = false, moved = false, tau_zero = false;
+        if (threadIdx.x < 64) hist[threadIdx.x] = 0;           // (a barrier follows in the first pass)
 #pragma unroll 1
         for (int attempt = 0; attempt < kWideRetries; ++attempt) {
             const uint32_t mine = flag_pass(low, low + window);
             uint32_t before;
             const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, mine), before);
-            const uint32_t in_window = (mine >> 16) - (mine & 0xFFFFu);
-            const uint32_t warp_max = __reduce_max_sync(0xFFFFFFFFu, in_window);
-            if (lane == 0) s_max[pass_no & 1u][warp] = warp_max;   // (read after the next barrier only if needed)
             ++pass_no;
             n_low = total >> 16;
             n_high = total & 0xFFFFu;
             if (n_high < k && k <= n_low) {
-                __syncthreads();
-                uint32_t cta_max = 0;
-#pragma unroll
-                for (int w = 0; w < W; ++w) cta_max = max(cta_max, s_max[(pass_no - 1u) & 1u][w]);
-                if (cta_max <= kWideListLen) {
-                    pinned = true;
-                    width = window;
-                    break;
-                }
-                if (window <= 4u) break;
-                window >>= 1;
-                crowded = true;
-                continue;
+                pinned = true;
+                break;
             }
             const uint32_t per_key_x16 = max(((n_low - n_high) << 4) / window, 4u);
             moved = true;
             if (n_low < k) {
-                if (low == 1) break;                               // tau_i = 0
+                if (low == 1) {                                    // fewer than k non-zeros: tau_i = 0
+                    tau_zero = true;
+                    break;
+                }
                 const uint32_t below = max(((k - n_low) << 4) / per_key_x16 + window / 2u, window / 2u);
                 low = low > below ? low - below : 1u;
             } else {
@@ -671,46 +658,104 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 low = low + above < 0x7F80u ? low + above : 0x7F80u;
             }
         }
-        uint32_t tau_key = 0, take = 0;
-        if (!pinned) {
-            // exact mode: the largest v with #{key >= v} >= k, bit by bit; then a window of one key at it
-            uint32_t v = 0;
-#pragma unroll 1
-            for (int bit = 14; bit >= 0; --bit) {
-                const uint32_t trial = v | (1u << bit);
-                const uint32_t mine = flag_pass(trial, trial);
-                uint32_t before;
-                const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, mine), before);
-                ++pass_no;
-                if ((total >> 16) >= k) v = trial;
-            }
-            tau_key = v;
-            const uint32_t mine = flag_pass(v, v + 1u);          // v = 0: every column, the padding included, is >= 0
-            uint32_t before;
-            const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, mine), before);
-            ++pass_no;
-            n_low = total >> 16;
-            n_high = total & 0xFFFFu;
-            take = k - n_high;
-            width = 1;
-            guess_low = 0;
-        }
 
-        // ---- C: tau_i and the kept columns as bits --------------------------------------------------------
-        uint32_t keep[kWords];
-        if (width == 1) {
-            // every window element ties at tau_i: the first `take` of them, in column order, are kept
-            uint32_t ties[kWords], n_ties = 0;
+        // ---- C: tau_i; the columns above it (kept for certain) and the ties at it, as bits ------------------------
+        uint32_t tau_key = 0;
+        uint32_t keep[kWords], ties[kWords];
+        if (pinned) {
 #pragma unroll
             for (int i = 0; i < kWords; ++i) {
-                ties[i] = ge_low[i] & ~ge_high[i];
-                n_ties += __popc(ties[i]);
+                uint32_t m = ge_low[i] & ~ge_high[i];
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 2u * (col0 + 32u * i + 31u - q)));
+                    atomicAdd(&hist[(v & 0x7FFFu) - low], 1u);
+                }
             }
-            const uint32_t incl = warp_inclusive_sum(n_ties);
+            __syncthreads();
+            {
+                // the (k - n_high)-th largest window element: lane l owns the bins 63 - 2 l (h.y) and 62 - 2 l
+                const uint32_t r = k - n_high;
+                const uint2 h = reinterpret_cast<const uint2*>(hist)[31u - lane];
+                const uint32_t own_cnt = h.x + h.y;
+                const uint32_t before = warp_inclusive_sum(own_cnt) - own_cnt;
+                uint32_t my_bin = 0;
+                bool mine = false;
+                if (before < r && r <= before + h.y) {
+                    mine = true;
+                    my_bin = 63u - 2u * lane;
+                } else if (before + h.y < r && r <= before + own_cnt) {
+                    mine = true;
+                    my_bin = 62u - 2u * lane;
+                }
+                const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
+                tau_key = low + __shfl_sync(0xFFFFFFFFu, my_bin, who ? __ffs(who) - 1 : 0);
+            }
+            if (moved) {
+                window = window < kSpanWindow ? window * 2u : kSpanWindow;
+            } else if (n_low - n_high > kWideShrink * 32u * W && window > 4u) {
+                window >>= 1;                                      // many window elements per lane: a narrower one next time
+            }
+            guess_low = tau_key > window / 2u ? tau_key - window / 2u : 1u;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                uint32_t m = ge_low[i] & ~ge_high[i];
+                keep[i] = ge_high[i];
+                ties[i] = 0;
+                while (m) {
+                    const uint32_t q = bfind(m);
+                    m ^= 1u << q;
+                    uint32_t v;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 2u * (col0 + 32u * i + 31u - q)));
+                    v &= 0x7FFFu;
+                    keep[i] |= v > tau_key ? 1u << q : 0u;
+                    ties[i] |= v == tau_key ? 1u << q : 0u;
+                }
+            }
+        } else {
+            // exact mode: the largest v with #{key >= v} >= k, bit by bit (0 if the window ended there); then a window
+            // of one key at it (v = 0: every column, the padding behind the row included, is >= 0)
+            uint32_t v = 0;
+            if (!tau_zero) {
+#pragma unroll 1
+                for (int bit = 14; bit >= 0; --bit) {
+                    const uint32_t trial = v | (1u << bit);
+                    const uint32_t mine = flag_pass(trial, trial);
+                    uint32_t before;
+                    const uint32_t total = cta_sum(s_cnt, pass_no & 1u, __reduce_add_sync(0xFFFFFFFFu, mine), before);
+                    ++pass_no;
+                    if ((total >> 16) >= k) v = trial;
+                }
+            }
+            tau_key = v;
+            flag_pass(v, v + 1u);
+            guess_low = 0;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) {
+                keep[i] = ge_high[i];
+                ties[i] = ge_low[i] & ~ge_high[i];
+            }
+        }
+        if (threadIdx.x == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+
+        // ---- D: every lane stages its kept entries at its offset of the row's output ----------------------------
+        // One scan of (#certain << 16 | #ties) over the CTA: the ties are taken in column order until k is reached.
+        const uint32_t shift = static_cast<uint32_t>(out_base) & 1u;
+        {
+            uint32_t packed = 0;
+#pragma unroll
+            for (int i = 0; i < kWords; ++i) packed += (__popc(keep[i]) << 16) | __popc(ties[i]);
+            const uint32_t incl = warp_inclusive_sum(packed);
             uint32_t warps_before;
-            cta_sum(s_sum, 0, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
-            const uint32_t ties_before = warps_before + incl - n_ties;
-            uint32_t room = ties_before < take ? take - ties_before : 0u;
+            const uint32_t total = cta_sum(s_sum, use & 1u, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
+            const uint32_t ties_to_take = k - (total >> 16);
+            const uint32_t mine_before = warps_before + incl - packed;
+            const uint32_t ties_before = mine_before & 0xFFFFu;
+            uint32_t room = ties_before < ties_to_take ? ties_to_take - ties_before : 0u;
+            uint32_t at = smem_addr(stage) +
+                          4u * (shift + (mine_before >> 16) + (ties_before < ties_to_take ? ties_before : ties_to_take));
 #pragma unroll
             for (int i = 0; i < kWords; ++i) {
                 uint32_t z = ties[i];
@@ -721,94 +766,7 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
                 } else {
                     room -= n;
                 }
-                keep[i] = ge_high[i] | z;
-            }
-        } else {
-            if (threadIdx.x < 64) hist[threadIdx.x] = 0;
-            __syncthreads();
-            uint32_t* my_list = lists + threadIdx.x * kWideListStride;
-            uint32_t n_list = 0;
-#pragma unroll
-            for (int i = 0; i < kWords; ++i) {
-                uint32_t m = ge_low[i] & ~ge_high[i];
-                while (m) {
-                    const uint32_t q = bfind(m);
-                    m ^= 1u << q;
-                    const uint32_t col = col0 + 32u * i + 31u - q;
-                    uint32_t v;
-                    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(v) : "r"(row_addr + 2u * col));
-                    const uint32_t key = v & 0x7FFFu;
-                    atomicAdd(&hist[key - low], 1u);
-                    my_list[n_list++] = ((32u * i + q) << 16) | key;
-                }
-            }
-            __syncthreads();
-            {
-                const uint32_t drop = n_low - k;
-                const uint2 h = reinterpret_cast<const uint2*>(hist)[lane];
-                const uint32_t own_cnt = h.x + h.y;
-                const uint32_t before = warp_inclusive_sum(own_cnt) - own_cnt;
-                uint32_t my_tau = 0, my_take = 0;
-                bool mine = false;
-                if (before <= drop && drop < before + h.x) {
-                    mine = true;
-                    my_tau = low + 2u * lane;
-                    my_take = h.x - (drop - before);
-                } else if (before + h.x <= drop && drop < before + own_cnt) {
-                    mine = true;
-                    my_tau = low + 2u * lane + 1u;
-                    my_take = h.y - (drop - before - h.x);
-                }
-                const uint32_t who = __ballot_sync(0xFFFFFFFFu, mine);
-                const int src = who ? __ffs(who) - 1 : 0;
-                tau_key = __shfl_sync(0xFFFFFFFFu, my_tau, src);
-                take = __shfl_sync(0xFFFFFFFFu, my_take, src);
-            }
-            if (crowded) {
-            } else if (moved) {
-                window = window < kSpanWindow ? window * 2u : kSpanWindow;
-            } else if (n_low - n_high > 64u * W && window > 16u) {
-                window >>= 1;
-            }
-            guess_low = tau_key > window / 2u ? tau_key - window / 2u : 1u;
-#pragma unroll
-            for (int i = 0; i < kWords; ++i) keep[i] = ge_high[i];
-            uint32_t n_ties = 0;
-            for (uint32_t j = 0; j < n_list; ++j) n_ties += (my_list[j] & 0xFFFFu) == tau_key ? 1u : 0u;
-            const uint32_t incl = warp_inclusive_sum(n_ties);
-            uint32_t warps_before;
-            cta_sum(s_sum, 0, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);
-            const uint32_t ties_before = warps_before + incl - n_ties;
-            uint32_t room = ties_before < take ? take - ties_before : 0u;
-            for (uint32_t j = 0; j < n_list; ++j) {
-                const uint32_t e = my_list[j];
-                const uint32_t key = e & 0xFFFFu;
-                bool add = key > tau_key;
-                if (key == tau_key && room > 0u) {
-                    add = true;
-                    --room;
-                }
-                const uint32_t bit = add ? 1u << ((e >> 16) & 31u) : 0u;
-                const uint32_t word = e >> 21;
-#pragma unroll
-                for (int i = 0; i < kWords; ++i) keep[i] |= word == static_cast<uint32_t>(i) ? bit : 0u;
-            }
-        }
-        if (threadIdx.x == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
-
-        // ---- D: every lane stages its kept entries at its offset of the row's output ----------------------------
-        const uint32_t shift = static_cast<uint32_t>(out_base) & 1u;
-        {
-            uint32_t kept_mine = 0;
-#pragma unroll
-            for (int i = 0; i < kWords; ++i) kept_mine += __popc(keep[i]);
-            const uint32_t incl = warp_inclusive_sum(kept_mine);
-            uint32_t warps_before;
-            cta_sum(s_sum, 1, __shfl_sync(0xFFFFFFFFu, incl, 31), warps_before);   // (the barrier inside: all lists are read)
-            uint32_t at = smem_addr(stage) + 4u * (shift + warps_before + incl - kept_mine);
-#pragma unroll
-            for (int i = 0; i < kWords; ++i) {
-                uint32_t m = keep[i];
+                uint32_t m = keep[i] | z;
                 const uint32_t colb = col0 + 32u * i + 31u;
                 while (m) {
                     const uint32_t q = bfind(m);
@@ -846,8 +804,9 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             if (rows_out)
                 for (uint32_t p = threadIdx.x; p < k; p += W * 32u) rows_out[out_base + p] = static_cast<int32_t>(row);
         }
-        __syncthreads();                                       // the stage has been read: its words may become lists again
+        __syncthreads();                                       // the stage has been read: the next row may fill it
     }
+    chain_release_next();
 }
 
 template <int W>
@@ -870,10 +829,9 @@ dct_status_t launch_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t 
     if (sms <= 0) return DCT_ERR_CUDA;
     const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
     const uint32_t grid = static_cast<uint32_t>(rows < max_grid ? rows : max_grid);
-    kernel<<<grid, W * 32, smem, stream>>>(static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out,
-                                           static_cast<uint16_t*>(vals_out), rows_out, static_cast<uint16_t*>(tau_out),
-                                           result);
-    DCT_CUDA_TRY(cudaGetLastError());
+    DCT_CUDA_TRY(launch_chained_smem(kernel, grid, static_cast<unsigned>(W * 32), smem, stream,
+                                     static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out,
+                                     static_cast<uint16_t*>(vals_out), rows_out, static_cast<uint16_t*>(tau_out), result));
     return DCT_OK;
 }
 
