@@ -305,6 +305,34 @@ def test_mp_bf16_wide_rows(d):
         assert int(cols.max()) < d
 
 
+@pytest.mark.parametrize("d,ld", [(128, 128), (256, 256), (256, 264), (384, 384), (512, 512), (512, 640)])
+def test_mp_bf16_many_short_rows(d, ld):
+    """Many short bf16 rows (the widths of the paper's recommendation-model layers), more than one round of any
+    persistent grid and not a multiple of 32: contiguous and strided rows, sparse and denser k, rows of very
+    different scales (a guess taken from a previous row fails in both directions), dead rows, rows where
+    everything ties, rows with fewer than k non-zeros, rows of a few distinct values, rows with huge values
+    (thresholds at the top of the key range)."""
+    rows = 32 * 148 * 3 + 21
+    x = inputs.mp_activations(rows, d, 291 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=292 + d, ld=ld)
+    sign = torch.where(inputs.dp_gaussian(rows * ld, 293 + d, G.DEV).view(rows, ld) > 0, 1.0, -1.0)
+    scale = torch.tensor([1.0, 30.0, 1e-2, 1.0, 1e3, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0], device=G.DEV)
+    scale = scale.repeat(rows // 11 + 1)[:rows]
+    x = x * sign * scale[:, None]
+    x[3] = 0.0
+    x[4] = -1.25
+    x[5, 9:] = 0.0
+    x[6] = inputs.quantize_mantissa(x[6], 1)
+    x[7::50] = inputs.quantize_mantissa(x[7::50], 2)
+    x[8] = 3.0e38
+    x[9, ::3] = 3.3e38
+    x[rows - 1] = 0.5
+    x = x.to(torch.bfloat16).contiguous()
+    gx = inputs.mp_gradients(rows, d, 294 + d, dtype=torch.bfloat16, device=G.DEV, ld=ld)
+    for k in sorted({1, 2, d // 20, d // 10, d // 4}):
+        cols = _compare_fwd_bwd(x, gx, d, k, want_rows=(k == 2))
+        assert int(cols.max()) < d
+
+
 @pytest.mark.parametrize("d", [2052, 4096, 4100, 8192, 12000, 16384, 24580, 32768])
 def test_mp_f32_rows_wider_than_2048(d):
     """fp32 rows of more than 2048 columns that the warp-per-row kernels leave out (every k beyond 4096 columns,
