@@ -519,6 +519,10 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
     // launched as a programmatic dependent of the kernel that resets the control block: everything above ran
     // while that kernel was still at work, nothing below may (a no-op under an ordinary launch)
     chain_wait_previous();
+    // The kernels after this one on the stream may be scheduled from here on: each of them waits for this grid to
+    // finish before it touches anything, so all they gain is that their launch latency and set-up are behind them
+    // when this grid ends (their CTAs take the places this grid's CTAs leave).
+    chain_release_next();
 
     if (warp == kLoadWarp) {
         // ================= load warp (one lane): tickets and bulk loads ====================
