@@ -1,5 +1,5 @@
 // dct_mp_topk_pack_fwd, bf16, k from about a tenth to 3/8 of the row (the 75 % sparsity level of the paper's DCT-MP
-// tables and the denser part of its 90 % level), rows of up to 8192 columns on 16-byte boundaries: Algorithm 2 (DCT-MP), forward pass -- one warp
+// tables and the denser part of its 90 % level), rows of up to 3072 columns on 16-byte boundaries: Algorithm 2 (DCT-MP), forward pass -- one warp
 // per row, every lane looking after one contiguous span of the row.
 //
 // The row arrives by one bulk copy (TMA engine) into shared memory exactly as it lies in HBM.  Lane l owns the
@@ -463,10 +463,11 @@ dct_status_t launch_span(const void* x_act, uint32_t rows, uint32_t d, uint32_t 
 
 
 // ------------------------------------------------------------------------------------------
-// rows of more than 8192 columns (up to 32768): W warps per row, one row per CTA at a time
+// rows of more than 3072 columns (up to 32768): W warps per row, one row per CTA at a time
 // ------------------------------------------------------------------------------------------
-// The same steps as above with a CTA in the place of the warp: warp w looks after the columns [4096 w, 4096 w + 4096)
-// of the row (lane l of it after 128 of them), counts and offsets are summed over the warps through shared memory, and
+// The same steps as above with a CTA in the place of the warp: lane l of warp w looks after the 32 KW columns from
+// (32 w + l) 32 KW on (KW = 2 for rows of up to 8192 columns, 4 beyond), counts and offsets are summed over the warps
+// through shared memory, and
 // the histogram of the window elements is the CTA's.  No lists: a lane walks the window bits of its span twice, once
 // for the histogram and once, with tau_i known, to add the elements above tau_i to its kept bits and to mark the
 // ties; one scan over the CTA then gives every lane its offset in the row's output and its share of the ties.
@@ -477,8 +478,8 @@ constexpr uint32_t kWideMaxK = 2300;
 constexpr int kWideRetries = 6;
 constexpr uint32_t kWideShrink = 3;               // window elements per lane (on average) from which the window narrows
 
-template <int W> struct WideLayout {
-    static constexpr uint32_t kSegBytes = 8192u;             // one warp's 4096 columns
+template <int W, int KW> struct WideLayout {             // KW: flag words (32 columns each) of a lane, 2 or 4
+    static constexpr uint32_t kSegBytes = 2048u * KW;        // one warp's 1024 KW columns
     static constexpr uint32_t kRowBytes = W * kSegBytes;
     static constexpr uint32_t kHistBytes = 256u;
     __host__ __device__ static constexpr uint32_t cta_bytes(uint32_t k) {
@@ -486,19 +487,19 @@ template <int W> struct WideLayout {
     }
 };
 
-template <int W>
+template <int W, int KW>
 __global__ void __launch_bounds__(W * 32)
 mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                              int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
                              int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
                              dct_result_t* __restrict__ result) {
-    using Lay = WideLayout<W>;
-    constexpr int kWords = 4;                                  // 128 columns per lane
-    constexpr uint32_t kLaneCols = 128u;
+    using Lay = WideLayout<W, KW>;
+    constexpr int kWords = KW;                                 // 32 KW columns per lane
+    constexpr uint32_t kLaneCols = 32u * KW;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
     unsigned char* base = smem_raw;
-    const unsigned char* own = base + warp * Lay::kSegBytes + lane * 256u;
+    const unsigned char* own = base + warp * Lay::kSegBytes + lane * (2u * kLaneCols);
     uint32_t* hist = reinterpret_cast<uint32_t*>(base + Lay::kRowBytes);
     uint32_t* stage = hist + Lay::kHistBytes / 4;
     __shared__ uint64_t s_bar;
@@ -532,7 +533,7 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 #pragma unroll
     for (int c = 0; c < 8; ++c) unit_base[c] = smem_addr(own) ^ (16u * (swz ^ static_cast<uint32_t>(c)));
     const uint32_t row_addr = smem_addr(base);
-    const uint32_t col0 = warp * 4096u + lane * kLaneCols;     // first column of the lane's span
+    const uint32_t col0 = (warp * 32u + lane) * kLaneCols;     // first column of the lane's span
 
     auto request_row = [&](uint64_t r) {
         if (threadIdx.x == 0) {
@@ -562,7 +563,7 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         const uint32_t low2 = low * 0x10001u, high2 = high * 0x10001u;
 #pragma unroll
         for (int i = 0; i < kWords; ++i) ge_low[i] = ge_high[i] = 0;
-        static_for<16>([&](auto c_tag) {
+        static_for<4 * KW>([&](auto c_tag) {
             constexpr int c = decltype(c_tag)::value;
             uint32_t f_low, f_high;
             flags8_two(lds128<128 * (c / 8)>(unit_base[c % 8]), low2, high2, f_low, f_high);
@@ -809,11 +810,11 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     chain_release_next();
 }
 
-template <int W>
+template <int W, int KW>
 dct_status_t launch_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
                          void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result, cudaStream_t stream) {
-    using Lay = WideLayout<W>;
-    auto kernel = mp_topk_fwd_bf16_wide_kernel<W>;
+    using Lay = WideLayout<W, KW>;
+    auto kernel = mp_topk_fwd_bf16_wide_kernel<W, KW>;
     const size_t smem = Lay::cta_bytes(k);
     static thread_local int configured_device = -1;
     int dev = 0;
@@ -841,23 +842,32 @@ dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, 
                                   int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                   dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
-    if (d > 8192 && d <= 32768 && d % 8 == 0 && k <= kWideMaxK && 8ull * k <= 3ull * d && aligned_to(x_act, 16) &&
+    // Rows of more than 3072 columns: one CTA per row (rows of 3073..8192 columns with 64 columns per lane, wider ones
+    // with 128).  Measured against the warp-per-row kernel below, which served rows of up to 8192 columns before:
+    // 16384x4096, k = 1024: 66.6 against 73.3 us; 8192x8192, k = 1280: 52.3 against 77.0 us; k = 2048: 69.0 against
+    // 97.8 us; and widths that kernel is not instantiated for (5120, 6144 columns in its 8192-column buffer) three
+    // times faster.  64 columns per lane on rows beyond 8192 columns: 4 to 9 % slower than 128.
+    if (d > 3072 && d <= 32768 && d % 8 == 0 && k <= kWideMaxK && 8ull * k <= 3ull * d && aligned_to(x_act, 16) &&
         (static_cast<size_t>(ld) * 2) % 16 == 0 && aligned_to(cols_out, 4) && aligned_to(vals_out, 4)) {
         *handled = true;
-        // as many warps as the row has segments of 4096 columns (the last one zero-padded)
-#define DCT_WIDE_WARPS(W) \
-    if (d <= 4096u * W) return launch_wide<W>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
-        DCT_WIDE_WARPS(3);
-        DCT_WIDE_WARPS(4);
-        DCT_WIDE_WARPS(5);
-        DCT_WIDE_WARPS(6);
-        DCT_WIDE_WARPS(7);
-        DCT_WIDE_WARPS(8);
+        // as many warps as the row has segments of 2048 (4096) columns, the last one zero-padded
+#define DCT_WIDE_WARPS(W, KW) \
+    if (d <= 1024u * KW * W)  \
+        return launch_wide<W, KW>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+        DCT_WIDE_WARPS(2, 2);
+        DCT_WIDE_WARPS(3, 2);
+        DCT_WIDE_WARPS(4, 2);
+        DCT_WIDE_WARPS(3, 4);
+        DCT_WIDE_WARPS(4, 4);
+        DCT_WIDE_WARPS(5, 4);
+        DCT_WIDE_WARPS(6, 4);
+        DCT_WIDE_WARPS(7, 4);
+        DCT_WIDE_WARPS(8, 4);
 #undef DCT_WIDE_WARPS
     }
     // (beyond 3/8 of the row a post-ReLU row's threshold is next to zero, where keys are sparse and the window
     // rarely settles: the general kernel serves those)
-    if (d > 8192 || d % 8 != 0 || k > kSpanMaxK || 8ull * k > 3ull * d) return DCT_OK;
+    if (d > 3072 || d % 8 != 0 || k > kSpanMaxK || 8ull * k > 3ull * d) return DCT_OK;
     if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0) return DCT_OK;
     if (!aligned_to(cols_out, 4) || !aligned_to(vals_out, 4)) return DCT_OK;   // the paired stores need 4-byte aligned outputs
     *handled = true;
@@ -869,8 +879,6 @@ dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, 
     DCT_SPAN_WIDTH(4);
     DCT_SPAN_WIDTH(8);
     DCT_SPAN_WIDTH(12);
-    DCT_SPAN_WIDTH(16);
-    DCT_SPAN_WIDTH(32);
 #undef DCT_SPAN_WIDTH
     *handled = false;
     return DCT_OK;

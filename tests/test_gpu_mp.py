@@ -361,12 +361,13 @@ def test_mp_f32_rows_wider_than_2048(d):
         assert int(cols.max()) < d
 
 
-@pytest.mark.parametrize("d", [8200, 12288, 16384, 20000, 32768])
-def test_mp_bf16_rows_wider_than_8192(d):
-    """bf16 rows of more than 8192 columns are packed by a CTA per row (4 or 8 warps, each looking after 4096 columns):
-    sparse and denser k, rows of very different scales (the window has to move), dead rows, rows where everything
-    ties, rows with fewer than k non-zeros, rows of a few distinct values (crowded windows and the exact mode), and
-    more rows than CTAs, so that every CTA works through several rows."""
+@pytest.mark.parametrize("d", [3080, 4096, 5120, 6152, 8192, 8200, 12288, 16384, 20000, 32768])
+def test_mp_bf16_rows_wider_than_3072(d):
+    """bf16 rows of more than 3072 columns are packed by a CTA per row (2 to 8 warps, a lane looking after 64 columns
+    up to 8192 columns, after 128 beyond) wherever the sparse warp-per-row kernel does not apply: sparse and denser
+    k, rows of very different scales (the window has to move), dead rows, rows where everything ties, rows with
+    fewer than k non-zeros, rows of a few distinct values (crowded windows and the exact mode), and more rows than
+    CTAs, so that every CTA works through several rows."""
     rows = 1500 if d <= 16384 else 700
     x = inputs.mp_activations(rows, d, 91 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=92 + d)
     sign = torch.where(inputs.dp_gaussian(rows * d, 93 + d, G.DEV).view(rows, d) > 0, 1.0, -1.0)
@@ -380,6 +381,6 @@ def test_mp_bf16_rows_wider_than_8192(d):
     x[8] = 3.0e38
     x = x.to(torch.bfloat16).contiguous()
     gx = inputs.mp_gradients(rows, d, 94 + d, dtype=torch.bfloat16, device=G.DEV)
-    for k in sorted({1, 33, d // 20, min(d // 8, 2300), min(d // 4 + 1, 2299)}):
+    for k in sorted({1, 33, d // 20, min(d // 8, 2300), min(d // 4 + 1, 2299), min(3 * d // 8, 2300)}):
         cols = _compare_fwd_bwd(x, gx, d, k, want_rows=(k == 33))
         assert int(cols.max()) < d
