@@ -175,9 +175,10 @@ DCT_API dct_status_t dct_dp_compress(
  * multiple of 16); other layouts are accepted and take a slower scalar load.
  * Every shape gives the same result; the time does depend on it.  Rows on
  * 16-byte boundaries with d*size a multiple of 16 are packed by one warp per
- * row (bf16: d <= 8192, k up to 3d/8 and 2048; fp32: d <= 4096, k up to
- * about d/10 and 441, denser k for d <= 2048) or by one CTA per row (bf16
- * rows of 8193..32768 columns with k up to 3d/8 and 2300; fp32 rows of
+ * row (bf16: d <= 8192 for k up to about d/10 and 441, d <= 3072 for k up
+ * to 3d/8 and 2048; fp32: d <= 4096, k up to about d/10 and 441, denser k for
+ * d <= 2048) or by one CTA per row (bf16 rows of 3073..32768 columns with k
+ * up to 3d/8 and 2300 where the warp kernel does not apply; fp32 rows of
  * 2049..32768 columns that the warp kernels leave out, k up to 3d/8 and
  * 4096); everything else (denser k, odd strides, cols_out not 4-byte aligned
  * for the denser and the wide cases) takes a general kernel that is several
