@@ -1003,17 +1003,16 @@ dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, u
     *handled = false;
     if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 4 != 0 || d > 4096) return DCT_OK;
     if (fwd_candidates_per_lane(d, k) == 0) {
-        // dense k (beyond the candidate registers, up to half the row): bounds + bit tables
-        // (rows of more than 2048 columns leave too few warps per SM for it: the general kernel is as fast there)
-        if (k > kDenseMaxKF32 || k > d / 2 || d > 2048) return DCT_OK;
+        // dense k (beyond the candidate registers, up to half the row) on rows of up to 512 columns: bounds + bit
+        // tables.  (From 513 columns on the CTA-per-row kernel of mp_pack_f32_wide.cu is 1.5 to 2.4 times faster up
+        // to k = 3d/8, and beyond that the general kernel is: 65536x1024, k = 512: 0.49 against 2.05 ms.)
+        if (k > kDenseMaxKF32 || k > d / 2 || d > 512) return DCT_OK;
         *handled = true;
 #define DCT_F32_DENSE(E8) \
     if (d <= 256u * E8)   \
         return launch_dense<E8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
         DCT_F32_DENSE(1);
         DCT_F32_DENSE(2);
-        DCT_F32_DENSE(4);
-        DCT_F32_DENSE(8);
 #undef DCT_F32_DENSE
         *handled = false;
         return DCT_OK;

@@ -1,4 +1,4 @@
-// dct_mp_topk_pack_fwd, fp32, rows of more than 2048 columns (up to 32768) that the warp-per-row kernels do not serve:
+// dct_mp_topk_pack_fwd, fp32, rows of more than 512 columns (up to 32768) that the warp-per-row kernels do not serve:
 // Algorithm 2 (DCT-MP), forward pass -- one CTA of W warps per row, warp w looking after the columns
 // [1024 w, 1024 w + 1024) and lane l of it after 32 of them (KW = 1; twice that with KW = 2).
 //
@@ -493,7 +493,7 @@ dct_status_t launch_fwd_f32_wide(const void* x_act, uint32_t rows, uint32_t d, u
     *handled = false;
     // (beyond 3/8 of the row a post-ReLU row's threshold is next to zero, where buckets are sparse and the window
     // rarely settles: the general kernel serves those)
-    if (d <= 2048 || d > 32768 || d % 4 != 0 || k > kWideMaxKF32 || 8ull * k > 3ull * d) return DCT_OK;
+    if (d <= 512 || d > 32768 || d % 4 != 0 || k > kWideMaxKF32 || 8ull * k > 3ull * d) return DCT_OK;
     if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || !aligned_to(cols_out, 4)) return DCT_OK;
     *handled = true;
     // As many warps as the row has segments of 1024 or 2048 columns (the last one zero-padded): 64 columns per lane,
@@ -503,6 +503,8 @@ dct_status_t launch_fwd_f32_wide(const void* x_act, uint32_t rows, uint32_t d, u
     if (narrow_spans) {
 #define DCT_WIDE_F32_WARPS(W) \
     if (d <= 1024u * W) return launch_wide_f32<W, 1>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+        DCT_WIDE_F32_WARPS(1);
+        DCT_WIDE_F32_WARPS(2);
         DCT_WIDE_F32_WARPS(3);
         DCT_WIDE_F32_WARPS(4);
 #undef DCT_WIDE_F32_WARPS

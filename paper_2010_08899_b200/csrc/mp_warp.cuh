@@ -235,7 +235,7 @@ dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, 
 dct_status_t launch_fwd_f32_warp(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                  int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                  dct_result_t* result, cudaStream_t stream, bool* handled);
-// fp32 rows of 2049..32768 columns, one CTA per row (mp_pack_f32_wide.cu).
+// fp32 rows of 513..32768 columns, one CTA per row (mp_pack_f32_wide.cu).
 dct_status_t launch_fwd_f32_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                  int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                  dct_result_t* result, cudaStream_t stream, bool* handled);

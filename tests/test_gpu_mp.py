@@ -333,13 +333,13 @@ def test_mp_bf16_many_short_rows(d, ld):
         assert int(cols.max()) < d
 
 
-@pytest.mark.parametrize("d", [2052, 4096, 4100, 8192, 12000, 16384, 24580, 32768])
-def test_mp_f32_rows_wider_than_2048(d):
-    """fp32 rows of more than 2048 columns that the warp-per-row kernels leave out (every k beyond 4096 columns,
-    the denser k up to 4096) are packed by a CTA per row, each warp looking after 2048 columns: sparse and denser
-    k, rows of very different scales (the window has to move), dead rows, rows where everything ties, rows with
-    fewer than k non-zeros, rows of tiny values inside bucket 0, rows of a few distinct values (many members in one
-    bucket, ties inside it), and more rows than CTAs, so that every CTA works through several rows."""
+@pytest.mark.parametrize("d", [516, 768, 1024, 1540, 2048, 2052, 4096, 4100, 8192, 12000, 16384, 24580, 32768])
+def test_mp_f32_rows_wider_than_512(d):
+    """fp32 rows of more than 512 columns that the sparse warp-per-row kernel leaves out (every k beyond 4096
+    columns, the denser k up to 4096) are packed by a CTA per row, a lane looking after 32 or 64 columns: sparse and
+    denser k, rows of very different scales (the window has to move), dead rows, rows where everything ties, rows
+    with fewer than k non-zeros, rows of tiny values inside bucket 0, rows of a few distinct values (many members in
+    one bucket, ties inside it), and more rows than CTAs, so that every CTA works through several rows."""
     rows = 900 if d <= 8192 else 400
     x = inputs.mp_activations(rows, d, 191 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=192 + d)
     sign = torch.where(inputs.dp_gaussian(rows * d, 193 + d, G.DEV).view(rows, d) > 0, 1.0, -1.0)
