@@ -346,15 +346,16 @@ class HotPath:
             self.grad_view(i), None, n, ks_dp, taus3, res3, ws3, s)
         calls["mp_threshold_mean_3_levels"] = lambda i: B.dct_mp_threshold_mean(
             self.x[i % len(self.x)], rows, d, d, ks_mp, mean3, tau_rows, s)
-        # the select of ONE vector range-partitioned over the ranks (every rank's vector is a shard of it): three
-        # streaming passes with one all-reduce of 2048 counts each (alone at N = 1)
+        # the select of ONE vector range-partitioned over the ranks (every rank's vector is a shard of it): the
+        # sampled rounds (one streaming pass, six all-reduces of 2048 counts) where they apply, else three passes
         import torch.distributed as dist
         world = dist.get_world_size() if dist.is_available() and dist.is_initialized() else 1
-        ws_sh = B.new_workspace(B.dct_threshold_select_shard_workspace_bytes(), self.dev)
+        ws_sh = B.new_workspace(B.dct_threshold_select_shard_sampled_workspace_bytes(n), self.dev)
         hist_sh = torch.empty(2048, dtype=torch.int64, device=self.dev)
         res_sh = B.new_result(self.dev)
         calls["threshold_select_sharded"] = lambda i: B.dct_threshold_select_sharded(
-            self.grad_view(i), None, n, c["dp_k"] * world, taus3[:1], res_sh, ws_sh, hist=hist_sh, stream=s)
+            self.grad_view(i), None, n, c["dp_k"] * world, taus3[:1], res_sh, ws_sh, hist=hist_sh, stream=s,
+            n_global=n * world)
         calls["mp_fwd_fp32"] = lambda i: B.dct_mp_topk_pack_fwd(x32[i % 2], rows, d, d, k, self.cols, vals32, None,
                                                                  None, None, s)
         for name, call in calls.items():

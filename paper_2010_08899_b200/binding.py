@@ -36,6 +36,8 @@ EXPORTED_SYMBOLS = (
     "dct_threshold_select_batched", "dct_threshold_select_batched_workspace_bytes",
     "dct_threshold_select_shard_workspace_bytes", "dct_threshold_select_shard_begin",
     "dct_threshold_select_shard_pass", "dct_threshold_select_shard_advance",
+    "dct_threshold_select_shard_sampled_workspace_bytes", "dct_threshold_select_shard_sampled_begin",
+    "dct_threshold_select_shard_sampled_pass", "dct_threshold_select_shard_sampled_advance",
 )
 
 _vp, _u64, _u32, _sz, _int = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_size_t, ctypes.c_int
@@ -121,6 +123,14 @@ def lib() -> ctypes.CDLL:
     L.dct_threshold_select_shard_pass.argtypes = [_vp, _vp, _u64, _u32, _vp, _vp, _vp]
     L.dct_threshold_select_shard_advance.restype = _int
     L.dct_threshold_select_shard_advance.argtypes = [_vp, _u32, _vp, _vp, _vp, _vp]
+    L.dct_threshold_select_shard_sampled_workspace_bytes.restype = _sz
+    L.dct_threshold_select_shard_sampled_workspace_bytes.argtypes = [_u64]
+    L.dct_threshold_select_shard_sampled_begin.restype = _int
+    L.dct_threshold_select_shard_sampled_begin.argtypes = [_u64, _u64, _u64, _vp, _sz, _vp]
+    L.dct_threshold_select_shard_sampled_pass.restype = _int
+    L.dct_threshold_select_shard_sampled_pass.argtypes = [_vp, _vp, _u64, _u32, _vp, _vp, _vp]
+    L.dct_threshold_select_shard_sampled_advance.restype = _int
+    L.dct_threshold_select_shard_sampled_advance.argtypes = [_vp, _u32, _vp, _vp, _vp, _vp]
     L.dct_debug_configure.restype = None
     L.dct_debug_configure.argtypes = [_u32, _u32]
     _lib = L
@@ -568,25 +578,36 @@ SHARD_PASSES = 3
 SHARD_BINS = 2048
 
 
-def sharded_select_rounds(local_histogram, advance, all_reduce_sum):
+def sharded_select_rounds(local_histogram, advance, all_reduce_sum, rounds=None):
     """The rounds of the range-partitioned select, free of any device code so that the exchange can be exercised on
-    CPU ranks: per pass ``local_histogram(p)`` returns this rank's 2048 digit counts, ``all_reduce_sum(h)`` returns
-    (or turns ``h`` into) their sum over the ranks, and ``advance(p, h)`` lets the rank pick the digit."""
-    for p in range(SHARD_PASSES):
+    CPU ranks: per round ``local_histogram(p)`` returns this rank's 2048 counts, ``all_reduce_sum(h)`` returns
+    (or turns ``h`` into) their sum over the ranks, and ``advance(p, h)`` lets the rank act on the sum.  Three rounds
+    (the radix passes) by default; the sampled variant has six (SHARD_SAMPLED_ROUNDS)."""
+    for p in range(SHARD_PASSES if rounds is None else rounds):
         h = local_histogram(p)
         summed = all_reduce_sum(h)
         advance(p, h if summed is None else summed)
+
+
+SHARD_SAMPLED_ROUNDS = 6
 
 
 def dct_threshold_select_shard_workspace_bytes() -> int:
     return lib().dct_threshold_select_shard_workspace_bytes()
 
 
+def dct_threshold_select_shard_sampled_workspace_bytes(n_local: int) -> int:
+    return lib().dct_threshold_select_shard_sampled_workspace_bytes(n_local)
+
+
 def dct_threshold_select_sharded(grad, residual, n_local, k_global, tau_out, result, workspace, group=None,
-                                 hist=None, stream=None) -> None:
+                                 hist=None, stream=None, n_global=None) -> bool:
     """The k_global-th largest |grad + residual| of a vector whose shards lie on the ranks of ``group`` (the default
     process group if None; a single process without a group selects over its own shard alone).  Every rank calls
-    this with its own shard; all get the same tau_out / result.  One all-reduce of 2048 int64 counts per pass."""
+    this with its own shard; all get the same tau_out / result.  Three rounds with one all-reduce of 2048 int64
+    counts each; if ``n_global`` (the total size over the ranks) is given, the vector is large enough and the
+    workspace holds dct_threshold_select_shard_sampled_workspace_bytes(n_local), the sampled variant runs instead: six
+    rounds, but one streaming pass over the shard instead of three.  Returns True if the sampled variant ran."""
     import torch.distributed as dist
     if n_local:
         _need(grad, torch.float32, "grad")
@@ -599,23 +620,45 @@ def dct_threshold_select_sharded(grad, residual, n_local, k_global, tau_out, res
         hist = torch.empty(SHARD_BINS, dtype=torch.int64, device=tau_out.device)
     _need(hist, torch.int64, "hist")
     L, s = lib(), _stream(stream)
-    _check("dct_threshold_select_shard_begin",
-           L.dct_threshold_select_shard_begin(k_global, _p(workspace), workspace.numel(), s))
     multi = dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1
-
-    def local_histogram(p):
-        _check("dct_threshold_select_shard_pass",
-               L.dct_threshold_select_shard_pass(_p(grad) if n_local else None, _p(residual), n_local, p, _p(workspace),
-                                                 _p(hist), s))
-        return hist
 
     def all_reduce_sum(h):
         if multi:
             dist.all_reduce(h, op=dist.ReduceOp.SUM, group=group)
         return None
 
+    g_ptr = _p(grad) if n_local else None
+    sampled = False
+    if n_global is not None and workspace.numel() >= L.dct_threshold_select_shard_sampled_workspace_bytes(n_local):
+        st = L.dct_threshold_select_shard_sampled_begin(k_global, n_global, n_local, _p(workspace), workspace.numel(), s)
+        if st == DCT_OK:
+            sampled = True
+        elif st != DCT_ERR_UNSUPPORTED:
+            _check("dct_threshold_select_shard_sampled_begin", st)
+    if sampled:
+        def local_counts(p):
+            _check("dct_threshold_select_shard_sampled_pass",
+                   L.dct_threshold_select_shard_sampled_pass(g_ptr, _p(residual), n_local, p, _p(workspace), _p(hist), s))
+            return hist
+
+        def act(p, h):
+            _check("dct_threshold_select_shard_sampled_advance",
+                   L.dct_threshold_select_shard_sampled_advance(_p(h), p, _p(workspace), _p(tau_out), _p(result), s))
+
+        sharded_select_rounds(local_counts, act, all_reduce_sum, rounds=SHARD_SAMPLED_ROUNDS)
+        return True
+
+    _check("dct_threshold_select_shard_begin",
+           L.dct_threshold_select_shard_begin(k_global, _p(workspace), workspace.numel(), s))
+
+    def local_histogram(p):
+        _check("dct_threshold_select_shard_pass",
+               L.dct_threshold_select_shard_pass(g_ptr, _p(residual), n_local, p, _p(workspace), _p(hist), s))
+        return hist
+
     def advance(p, h):
         _check("dct_threshold_select_shard_advance",
                L.dct_threshold_select_shard_advance(_p(h), p, _p(workspace), _p(tau_out), _p(result), s))
 
     sharded_select_rounds(local_histogram, advance, all_reduce_sum)
+    return False
