@@ -458,11 +458,11 @@ DCT_API dct_status_t dct_threshold_select_shard_advance(
  * dct_threshold_select_shard_sampled_{begin,pass,advance} -- the same select with ONE streaming pass over the shard
  * instead of three, for large vectors (the scheme of dct_threshold_select carried over to shards): a sample of the
  * vector, taken at the same rate on every rank, is radix-selected in two passes for a rank chosen six standard
- * deviations on the safe side (rounds 0 and 1), which gives a key `lo` with, almost surely, between k_global and a
+ * deviations on the safe side (stages 0 and 1), which gives a key `lo` with, almost surely, between k_global and a
  * few k_global elements of the whole vector at or above it; every rank streams its shard once and keeps its keys
- * >= lo (round 2; its message is the number of keys kept and whether they fitted); the three exact passes then run
- * over the candidates only (rounds 3, 4, 5) -- or, if the summed counts say that the candidates are fewer than
- * k_global or overflowed some rank's buffer, over the shards: every rank takes that decision alike.  Six rounds of
+ * >= lo (stage 2; its message is the number of keys kept and whether they fitted); the three exact passes then run
+ * over the candidates only (stages 3, 4, 5) -- or, if the summed counts say that the candidates are fewer than
+ * k_global or overflowed some rank's buffer, over the shards: every rank takes that decision alike.  Six stages of
  * (pass, sum of 2048 uint64 over the ranks, advance); the outputs are those of the three-pass version, bit for bit.
  *
  *   begin      returns DCT_ERR_UNSUPPORTED (nothing launched) where the scheme does not apply: n_global < 2^25, or a
@@ -472,19 +472,19 @@ DCT_API dct_status_t dct_threshold_select_shard_advance(
  *   n_global   total number of elements over all ranks; n_local this rank's (may be 0).
  *   workspace  DEVICE, >= dct_threshold_select_shard_sampled_workspace_bytes(n_local), 256-byte aligned (up to
  *              16 MiB of candidate keys).
- *   round      0 .. 5, in this order, each pass followed by its advance.
+ *   stage      0 .. 5, in this order, each pass followed by its advance.
  *   hist_out / hist_global  [2048] uint64 DEVICE, as above.
- *   tau_out, result  device; written by advance(round = 5) only.
+ *   tau_out, result  device; written by advance(stage = 5) only.
  */
 DCT_API size_t dct_threshold_select_shard_sampled_workspace_bytes(uint64_t n_local);
 DCT_API dct_status_t dct_threshold_select_shard_sampled_begin(
     uint64_t k_global, uint64_t n_global, uint64_t n_local, void* workspace, size_t workspace_bytes,
     dct_stream_t stream);
 DCT_API dct_status_t dct_threshold_select_shard_sampled_pass(
-    const float* grad, const float* residual, uint64_t n_local, uint32_t round,
+    const float* grad, const float* residual, uint64_t n_local, uint32_t stage,
     void* workspace, uint64_t* hist_out, dct_stream_t stream);
 DCT_API dct_status_t dct_threshold_select_shard_sampled_advance(
-    const uint64_t* hist_global, uint32_t round, void* workspace,
+    const uint64_t* hist_global, uint32_t stage, void* workspace,
     float* tau_out, dct_result_t* result, dct_stream_t stream);
 
 /* ------------------------------------------------------------------------- *

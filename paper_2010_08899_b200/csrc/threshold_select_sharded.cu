@@ -152,7 +152,7 @@ constexpr uint32_t kShardSampleTarget = 1u << 20;       // sampled elements of t
 constexpr uint32_t kShardGroup = 8;
 constexpr uint64_t kShardMinSampledN = 1ull << 25;
 constexpr uint32_t kShardMaxCandidates = 1u << 22;
-constexpr int kShardRounds = 6;                         // 2 sample passes, the filter, 3 exact passes
+constexpr int kShardStages = 6;                         // 2 sample passes, the filter, 3 exact passes
 
 struct SampledState {
     ShardState main;             // offset 0: the exact select (k_global)
@@ -397,7 +397,7 @@ extern "C" dct_status_t dct_threshold_select_shard_advance(const uint64_t* hist_
     return DCT_OK;
 }
 
-// ---- sampled variant: six rounds of (local pass, sum of 2048 counts over the ranks, advance) -----------------------
+// ---- sampled variant: six stages of (local pass, sum of 2048 counts over the ranks, advance) -----------------------
 extern "C" size_t dct_threshold_select_shard_sampled_workspace_bytes(uint64_t n_local) {
     if (n_local > 0x7FFFFFFFull) return 0;
     const uint64_t cap = n_local < kShardMaxCandidates ? n_local : kShardMaxCandidates;
@@ -411,7 +411,7 @@ extern "C" dct_status_t dct_threshold_select_shard_sampled_begin(uint64_t k_glob
     if (!workspace || !aligned_to(workspace, 256) ||
         workspace_bytes < dct_threshold_select_shard_sampled_workspace_bytes(n_local))
         return DCT_ERR_WORKSPACE;
-    if (n_global < kShardMinSampledN) return DCT_ERR_UNSUPPORTED;       // the plain rounds are cheaper
+    if (n_global < kShardMinSampledN) return DCT_ERR_UNSUPPORTED;       // the three-pass version is cheaper
     const uint32_t stride = shard_stride(n_global);
     if (stride < kShardGroup) return DCT_ERR_UNSUPPORTED;
     const uint64_t sample_k = shard_sample_rank(n_global, k_global, static_cast<double>(kShardGroup) / stride);
@@ -424,9 +424,9 @@ extern "C" dct_status_t dct_threshold_select_shard_sampled_begin(uint64_t k_glob
 }
 
 extern "C" dct_status_t dct_threshold_select_shard_sampled_pass(const float* grad, const float* residual,
-                                                                uint64_t n_local, uint32_t round, void* workspace,
+                                                                uint64_t n_local, uint32_t stage, void* workspace,
                                                                 uint64_t* hist_out, dct_stream_t stream_) {
-    if (!hist_out || !workspace || round >= static_cast<uint32_t>(kShardRounds) || n_local > 0x7FFFFFFFull)
+    if (!hist_out || !workspace || stage >= static_cast<uint32_t>(kShardStages) || n_local > 0x7FFFFFFFull)
         return DCT_ERR_INVALID_ARG;
     if (n_local > 0 && !grad) return DCT_ERR_INVALID_ARG;
     if (!aligned_to(grad, 4) || (residual && !aligned_to(residual, 4)) || !aligned_to(hist_out, 8) ||
@@ -444,18 +444,18 @@ extern "C" dct_status_t dct_threshold_select_shard_sampled_pass(const float* gra
     const uint64_t chunks = (n_local + kShardChunk - 1) / kShardChunk;
     const int grid = static_cast<int>(chunks < static_cast<uint64_t>(sms) * 4 ? (chunks ? chunks : 1) : sms * 4);
     const bool vec = aligned_to(grad, 16) && (!residual || aligned_to(residual, 16));
-    if (round < 2) {                                    // the sample: stride and prefix come from the state
+    if (stage < 2) {                                    // the sample: stride and prefix come from the state
         if (n_local == 0) return DCT_OK;
         // (the stride is in the state; the grid only has to cover the sample)
         const int sgrid = sms * 2;
-        if (round == 0)
+        if (stage == 0)
             sampled_hist_kernel<0><<<sgrid, kShardThreads, 0, stream>>>(grad, residual, n32, st, hist);
         else
             sampled_hist_kernel<1><<<sgrid, kShardThreads, 0, stream>>>(grad, residual, n32, st, hist);
         DCT_CUDA_TRY(cudaGetLastError());
         return DCT_OK;
     }
-    if (round == 2) {                                   // the filter, then its counts as the ranks' message
+    if (stage == 2) {                                   // the filter, then its counts as the ranks' message
         if (n_local > 0) {
             sampled_filter_kernel<<<grid, kShardThreads, 0, stream>>>(grad, residual, n32, st, cand_keys, vec);
             DCT_CUDA_TRY(cudaGetLastError());
@@ -464,8 +464,8 @@ extern "C" dct_status_t dct_threshold_select_shard_sampled_pass(const float* gra
         DCT_CUDA_TRY(cudaGetLastError());
         return DCT_OK;
     }
-    // rounds 3..5: the exact passes over the candidates or, if the summed counts said so, over the shard
-    const uint32_t pass = round - 3;
+    // stages 3..5: the exact passes over the candidates or, if the summed counts said so, over the shard
+    const uint32_t pass = stage - 3;
     if (pass == 0)
         sampled_cand_hist_kernel<0><<<sms, kShardThreads, 0, stream>>>(cand_keys, st, hist);
     else if (pass == 1)
@@ -484,28 +484,28 @@ extern "C" dct_status_t dct_threshold_select_shard_sampled_pass(const float* gra
     return DCT_OK;
 }
 
-extern "C" dct_status_t dct_threshold_select_shard_sampled_advance(const uint64_t* hist_global, uint32_t round,
+extern "C" dct_status_t dct_threshold_select_shard_sampled_advance(const uint64_t* hist_global, uint32_t stage,
                                                                    void* workspace, float* tau_out, dct_result_t* result,
                                                                    dct_stream_t stream_) {
-    if (!hist_global || !workspace || round >= static_cast<uint32_t>(kShardRounds)) return DCT_ERR_INVALID_ARG;
-    if (round == static_cast<uint32_t>(kShardRounds) - 1 && (!tau_out || !result)) return DCT_ERR_INVALID_ARG;
+    if (!hist_global || !workspace || stage >= static_cast<uint32_t>(kShardStages)) return DCT_ERR_INVALID_ARG;
+    if (stage == static_cast<uint32_t>(kShardStages) - 1 && (!tau_out || !result)) return DCT_ERR_INVALID_ARG;
     if (!aligned_to(hist_global, 8) || !aligned_to(workspace, 256) || (tau_out && !aligned_to(tau_out, 4)) ||
         (result && !aligned_to(result, 8)))
         return DCT_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const auto* hist = reinterpret_cast<const unsigned long long*>(hist_global);
     auto* st = static_cast<SampledState*>(workspace);
-    if (round == 0) {
+    if (stage == 0) {
         shard_advance_kernel<0><<<1, kShardThreads, 0, stream>>>(hist, &st->sample, nullptr, nullptr);
-    } else if (round == 1) {
+    } else if (stage == 1) {
         shard_advance_kernel<1><<<1, kShardThreads, 0, stream>>>(hist, &st->sample, nullptr, nullptr);
         DCT_CUDA_TRY(cudaGetLastError());
         sampled_lo_kernel<<<1, 1, 0, stream>>>(st);
-    } else if (round == 2) {
+    } else if (stage == 2) {
         sampled_decide_kernel<<<1, 1, 0, stream>>>(st, hist);
-    } else if (round == 3) {
+    } else if (stage == 3) {
         shard_advance_kernel<0><<<1, kShardThreads, 0, stream>>>(hist, &st->main, tau_out, result);
-    } else if (round == 4) {
+    } else if (stage == 4) {
         shard_advance_kernel<1><<<1, kShardThreads, 0, stream>>>(hist, &st->main, tau_out, result);
     } else {
         shard_advance_kernel<2><<<1, kShardThreads, 0, stream>>>(hist, &st->main, tau_out, result);
