@@ -382,12 +382,26 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         // ---- B: candidate masks (key >= low), in column order ------------------------------------------
         uint32_t masks[kMaskWords];
         uint32_t n_mine = 0, incl = 0, n_cand = 0;
-        auto build_masks = [&](uint32_t bound) {
+        auto build_masks = [&](uint32_t bound, bool probe) -> bool {
             // unit u = 32 c + lane covers columns 8 u .. 8 u + 7: its 8 flags are byte u of the mask table, which
             // therefore holds one bit per column, in column order
             unsigned char* tab8 = reinterpret_cast<unsigned char*>(mask_tab) + lane;
+            {
+                const uint32_t m0 = mask8_ge_exact(*reinterpret_cast<const uint4*>(unit0), bound);
+                tab8[0] = static_cast<unsigned char>(m0);
+                // A guessed bound is probed on the first unit of every lane (1 / E8 of the row): if that sample says
+                // that the candidates will be far too few or far too many, the rest of the pass is not worth making
+                // (rows whose scale differs from the previous row's).  Only a saving: the guess is checked exactly below.
+                if (E8 >= 8 && probe) {
+                    const uint32_t sample = __reduce_add_sync(0xFFFFFFFFu, __popc(m0)) * E8;
+                    if (8u * sample < 5u * k || 5u * sample > 8u * kRound) {
+                        n_cand = 0;
+                        return false;
+                    }
+                }
+            }
 #pragma unroll
-            for (int c = 0; c < E8; ++c)
+            for (int c = 1; c < E8; ++c)
                 tab8[c * 32] = static_cast<unsigned char>(
                     mask8_ge_exact(*reinterpret_cast<const uint4*>(unit0 + c * 512), bound));
             __syncwarp();
@@ -412,6 +426,7 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
             for (int i = 0; i < kMaskWords; ++i) n_mine += __popc(masks[i]);
             incl = warp_inclusive_sum(n_mine);
             n_cand = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            return true;
         };
 
         // Thresholds of neighbouring samples are close (the observation behind the paper's threshold
@@ -425,8 +440,8 @@ mp_topk_fwd_bf16_warp_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
 #pragma unroll 1
         while (true) {
             low = use_guess ? guess_low : exact_bound();
-            build_masks(low);
-            if (!use_guess || (n_cand >= k && n_cand <= kRound)) break;
+            const bool built = build_masks(low, use_guess);
+            if (!use_guess || (built && n_cand >= k && n_cand <= kRound)) break;
             use_guess = false;
         }
         if (!have_bound || n_cand > kRound || low == 0) {
