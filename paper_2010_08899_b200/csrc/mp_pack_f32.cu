@@ -276,11 +276,26 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
         // ---- B: candidate bits (upper key bits >= bound), in column order ------------------------------
         uint32_t masks[kMaskWords];
         uint32_t n_mine = 0, incl = 0, n_cand = 0;
-        auto build_masks = [&](uint32_t bound) {
+        auto build_masks = [&](uint32_t bound, bool probe) -> bool {
             const uint32_t low2 = bound | (bound << 16);
             unsigned char* tab8 = reinterpret_cast<unsigned char*>(mask_tab) + lane;
+            {
+                const uint4 a = *reinterpret_cast<const uint4*>(piece_first);
+                const uint4 b = *reinterpret_cast<const uint4*>(piece_second);
+                const uint32_t m0 = piece_flags(a, b, low2, w_first, w_second);
+                tab8[0] = static_cast<unsigned char>(m0);
+                // a guessed bound is probed on the first piece of every lane (1 / E8 of the row) before the rest of
+                // the pass is made for it (see the bf16 kernel, mp_pack.cu)
+                if (E8 >= 8 && probe) {
+                    const uint32_t sample = __reduce_add_sync(0xFFFFFFFFu, __popc(m0)) * E8;
+                    if (8u * sample < 5u * k || 5u * sample > 8u * kRound) {
+                        n_cand = 0;
+                        return false;
+                    }
+                }
+            }
 #pragma unroll
-            for (int c = 0; c < E8; ++c) {
+            for (int c = 1; c < E8; ++c) {
                 const uint4 a = *reinterpret_cast<const uint4*>(piece_first + c * 1024);
                 const uint4 b = *reinterpret_cast<const uint4*>(piece_second + c * 1024);
                 tab8[c * 32] = static_cast<unsigned char>(piece_flags(a, b, low2, w_first, w_second));
@@ -306,6 +321,7 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
             for (int i = 0; i < kMaskWords; ++i) n_mine += __popc(masks[i]);
             incl = warp_inclusive_sum(n_mine);
             n_cand = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            return true;
         };
 
         uint32_t low = 0;
@@ -314,8 +330,8 @@ mp_topk_fwd_f32_warp_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint3
 #pragma unroll 1
         while (true) {
             low = use_guess ? guess_low : exact_bound();
-            build_masks(low);
-            if (!use_guess || (n_cand >= k && n_cand <= kRound)) break;
+            const bool built = build_masks(low, use_guess);
+            if (!use_guess || (built && n_cand >= k && n_cand <= kRound)) break;
             use_guess = false;
         }
         if (!have_bound || n_cand > kRound || low == 0) {
