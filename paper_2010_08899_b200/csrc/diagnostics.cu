@@ -119,9 +119,26 @@ multi_pass_kernel(const float* __restrict__ grad, const float* __restrict__ resi
     const int hists = kPass == 0 ? 1 : m;
 
     for (int b = threadIdx.x; b < hists * kDiagBins; b += kDiagThreads) (&sh[0][0])[b] = 0;
+    // Ranks whose prefixes are equal so far share one histogram (that of the first of them): an element then
+    // matches at most one histogram, and a pass costs one shared-memory atomic per matching element, not one
+    // instruction per rank.  owner[q] = the rank whose histogram rank q reads; prefix[q] = 0xFFFFFFFF (matches
+    // nothing) for q >= m and for ranks that are not owners.
     uint32_t prefix[kMaxQ];
+    int owner[kMaxQ];
 #pragma unroll
-    for (int q = 0; q < kMaxQ; ++q) prefix[q] = (kPass != 0 && q < m) ? ws->rank[q].prefix : 0xFFFFFFFFu;
+    for (int q = 0; q < kMaxQ; ++q) {
+        prefix[q] = (kPass != 0 && q < m) ? ws->rank[q].prefix : 0xFFFFFFFFu;
+        owner[q] = q;
+    }
+#pragma unroll
+    for (int q = 1; q < kMaxQ; ++q) {
+#pragma unroll
+        for (int p = q - 1; p >= 0; --p)
+            if (kPass != 0 && q < m && prefix[p] == prefix[q] && owner[p] == p) owner[q] = p;
+    }
+#pragma unroll
+    for (int q = 0; q < kMaxQ; ++q)
+        if (owner[q] != q) prefix[q] = 0xFFFFFFFFu;
     __syncthreads();
 
     auto consume = [&](uint32_t key) {
@@ -130,9 +147,11 @@ multi_pass_kernel(const float* __restrict__ grad, const float* __restrict__ resi
             atomicAdd(&sh[0][digit], 1u);
         } else {
             const uint32_t upper = key >> (shift + bits);
+            int hit = -1;
 #pragma unroll
             for (int q = 0; q < kMaxQ; ++q)
-                if (upper == prefix[q]) atomicAdd(&sh[q % kHists][digit], 1u);   // prefix[q >= m] matches nothing
+                if (upper == prefix[q]) hit = q;
+            if (hit >= 0) atomicAdd(&(&sh[0][0])[(hit % kHists) * kDiagBins + digit], 1u);
         }
     };
 
@@ -162,7 +181,9 @@ multi_pass_kernel(const float* __restrict__ grad, const float* __restrict__ resi
     }
     __syncthreads();
 
-    for (int q = 0; q < hists; ++q) {
+#pragma unroll
+    for (int q = 0; q < kHists; ++q) {
+        if (q >= hists || (kPass != 0 && owner[q] != q)) continue;      // (counted in its owner's histogram)
         uint32_t* hist = ws->rank[q].hist[kPass];
         for (int b = threadIdx.x; b < kDiagBins; b += kDiagThreads) {
             const uint32_t c = sh[q][b];
@@ -175,8 +196,11 @@ multi_pass_kernel(const float* __restrict__ grad, const float* __restrict__ resi
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    for (int q = 0; q < m; ++q)
-        multi_finish<kPass>(&ws->rank[q], ws->rank[kPass == 0 ? 0 : q].hist[kPass], s_scan, tau_out + q, results + q);
+#pragma unroll
+    for (int q = 0; q < kMaxQ; ++q)
+        if (q < m)
+            multi_finish<kPass>(&ws->rank[q], ws->rank[kPass == 0 ? 0 : owner[q]].hist[kPass], s_scan, tau_out + q,
+                                results + q);
 }
 
 // ------------------------------------------------------------------------------------------------
