@@ -11,6 +11,7 @@
 // passes: the histogram of the leading digit is common to all ranks; the second and third pass keep
 // one histogram per rank, each restricted to the prefix that rank has chosen so far.
 #include "common.cuh"
+#include "mp_warp.cuh"
 #include "row_select.cuh"
 
 namespace dct {
@@ -265,6 +266,26 @@ tau_mean_kernel(const T* __restrict__ tau, uint32_t rows, double* __restrict__ m
 template <typename T>
 dct_status_t launch_threshold_mean(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, const RowRanks& ks, int m,
                                    double* mean_out, void* tau_out, cudaStream_t stream) {
+    // Where the CTA-per-row forward kernels apply to every level, they find the thresholds (one launch per level,
+    // nothing packed): 16384x4096 bf16, three levels: 0.31 -> 0.12 ms.  The general kernel below reads the row once
+    // for all levels, but selects with 8-bit radix passes.
+    {
+        bool all = true;
+        for (int q = 0; q < m && all; ++q) {
+            bool handled = false;
+            void* out = static_cast<T*>(tau_out) + static_cast<size_t>(q) * rows;
+            const dct_status_t st = sizeof(T) == 2
+                ? launch_tau_bf16_wide(x_act, rows, d, ld, ks.k[q], out, stream, &handled)
+                : launch_tau_f32_wide(x_act, rows, d, ld, ks.k[q], out, stream, &handled);
+            if (st != DCT_OK) return st;
+            all = handled;              // (q == 0 decides for shapes; a later k outside the kernels' range starts over below)
+        }
+        if (all) {
+            tau_mean_kernel<T><<<m, kMeanThreads, 0, stream>>>(static_cast<const T*>(tau_out), rows, mean_out);
+            DCT_CUDA_TRY(cudaGetLastError());
+            return DCT_OK;
+        }
+    }
     const size_t smem = ((static_cast<size_t>(d) * sizeof(T)) + 15) & ~static_cast<size_t>(15);
     auto kernel = mp_row_thresholds_kernel<T>;
     if (smem > 48 * 1024)

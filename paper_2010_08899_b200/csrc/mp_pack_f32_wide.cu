@@ -98,6 +98,7 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
     for (int c = 0; c < 8; ++c) unit_base[c] = smem_addr(own) ^ (16u * (swz ^ static_cast<uint32_t>(c)));
     const uint32_t row_addr = smem_addr(base);
     const uint32_t col0 = (warp * 32u + lane) * kLaneCols;     // first column of the lane's span
+    const bool emit = cols_out != nullptr;                     // (thresholds only, for the diagnostics, if not)
 
     auto request_row = [&](uint64_t r) {
         if (threadIdx.x == 0) {
@@ -375,7 +376,7 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
         // kept: the columns above the bucket, the members above t, and the first ties at t in column order.  One scan
         // of (#certain << 16 | #ties) over the CTA gives every lane both its offset and its share of the ties.
         const uint32_t shift = static_cast<uint32_t>(out_base) & 1u;
-        {
+        if (emit) {
             uint32_t keep[kWords], eq[kWords], packed = 0;
 #pragma unroll
             for (int i = 0; i < kWords; ++i) {
@@ -434,7 +435,7 @@ mp_topk_fwd_f32_wide_kernel(const float* __restrict__ x, uint32_t rows, uint32_t
         if (row64 + gridDim.x < rows) request_row(row64 + gridDim.x);
 
         // ---- E: the staged entries leave: values one by one, columns in pairs --------------------------------------
-        {
+        if (emit) {
             for (uint32_t p = threadIdx.x; p < k; p += W * 32u) vals_out[out_base + p] = stage_vals[p];
             const size_t pair_base = out_base - shift;
             const uint32_t last = shift + k;
@@ -485,6 +486,20 @@ dct_status_t launch_wide_f32(const void* x_act, uint32_t rows, uint32_t d, uint3
 }
 
 }  // namespace
+
+// The per-row thresholds alone (tau_out[row], nothing packed): for the threshold diagnostics.
+dct_status_t launch_tau_f32_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, void* tau_out,
+                                 cudaStream_t stream, bool* handled) {
+    bool dummy = false;
+    *handled = false;
+    if (d <= 512 || d > 32768 || d % 4 != 0 || k > kWideMaxKF32 || 8ull * k > 3ull * d || !aligned_to(x_act, 16) ||
+        (static_cast<size_t>(ld) * 4) % 16 != 0)
+        return DCT_OK;
+    const dct_status_t st = launch_fwd_f32_wide(x_act, rows, d, ld, k, nullptr, nullptr, nullptr, tau_out, nullptr, stream,
+                                                &dummy);
+    *handled = dummy;
+    return st;
+}
 
 // *handled = false: the shape is not one of this path's; the caller runs the general kernel.
 dct_status_t launch_fwd_f32_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,

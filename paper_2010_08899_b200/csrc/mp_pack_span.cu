@@ -534,6 +534,7 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
     for (int c = 0; c < 8; ++c) unit_base[c] = smem_addr(own) ^ (16u * (swz ^ static_cast<uint32_t>(c)));
     const uint32_t row_addr = smem_addr(base);
     const uint32_t col0 = (warp * 32u + lane) * kLaneCols;     // first column of the lane's span
+    const bool emit = cols_out != nullptr;                     // (thresholds only, for the diagnostics, if not)
 
     auto request_row = [&](uint64_t r) {
         if (threadIdx.x == 0) {
@@ -744,7 +745,7 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         // ---- D: every lane stages its kept entries at its offset of the row's output ----------------------------
         // One scan of (#certain << 16 | #ties) over the CTA: the ties are taken in column order until k is reached.
         const uint32_t shift = static_cast<uint32_t>(out_base) & 1u;
-        {
+        if (emit) {
             uint32_t packed = 0;
 #pragma unroll
             for (int i = 0; i < kWords; ++i) packed += (__popc(keep[i]) << 16) | __popc(ties[i]);
@@ -785,7 +786,7 @@ mp_topk_fwd_bf16_wide_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint
         if (row64 + gridDim.x < rows) request_row(row64 + gridDim.x);
 
         // ---- E: the staged entries leave in pairs ------------------------------------------------------------------
-        {
+        if (emit) {
             const size_t pair_base = out_base - shift;
             const uint32_t last = shift + k;
             for (uint32_t p = 2u * threadIdx.x; p < last; p += 2u * W * 32u) {
@@ -837,6 +838,32 @@ dct_status_t launch_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t 
 }
 
 }  // namespace
+
+// The per-row thresholds alone (tau_out[row], nothing packed), by the CTA-per-row kernel: for the threshold
+// diagnostics.  *handled = false: not a shape of this kernel.
+dct_status_t launch_tau_bf16_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, void* tau_out,
+                                  cudaStream_t stream, bool* handled) {
+    *handled = false;
+    if (d <= 3072 || d > 32768 || d % 8 != 0 || k > kWideMaxK || 8ull * k > 3ull * d || !aligned_to(x_act, 16) ||
+        (static_cast<size_t>(ld) * 2) % 16 != 0)
+        return DCT_OK;
+    *handled = true;
+#define DCT_WIDE_WARPS(W, KW) \
+    if (d <= 1024u * KW * W)  \
+        return launch_wide<W, KW>(x_act, rows, d, ld, k, nullptr, nullptr, nullptr, tau_out, nullptr, stream)
+    DCT_WIDE_WARPS(2, 2);
+    DCT_WIDE_WARPS(3, 2);
+    DCT_WIDE_WARPS(4, 2);
+    DCT_WIDE_WARPS(3, 4);
+    DCT_WIDE_WARPS(4, 4);
+    DCT_WIDE_WARPS(5, 4);
+    DCT_WIDE_WARPS(6, 4);
+    DCT_WIDE_WARPS(7, 4);
+    DCT_WIDE_WARPS(8, 4);
+#undef DCT_WIDE_WARPS
+    *handled = false;
+    return DCT_OK;
+}
 
 dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                   int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,

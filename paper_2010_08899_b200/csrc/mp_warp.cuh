@@ -240,4 +240,10 @@ dct_status_t launch_fwd_f32_wide(const void* x_act, uint32_t rows, uint32_t d, u
                                  int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                  dct_result_t* result, cudaStream_t stream, bool* handled);
 
+// The per-row thresholds alone by the CTA-per-row kernels (mp_pack_span.cu, mp_pack_f32_wide.cu).
+dct_status_t launch_tau_bf16_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, void* tau_out,
+                                  cudaStream_t stream, bool* handled);
+dct_status_t launch_tau_f32_wide(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, void* tau_out,
+                                 cudaStream_t stream, bool* handled);
+
 }  // namespace dct

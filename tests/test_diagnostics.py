@@ -162,6 +162,27 @@ def test_gpu_threshold_mean_matches_oracle(dtype, rows, d, ld):
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("ks", [[205, 2048], [2048, 205], [1500, 410, 7]])
+def test_gpu_threshold_mean_levels_inside_and_outside_the_fast_kernels(dtype, ks):
+    """Levels up to 3/8 of the row are found by the forward kernels run for their thresholds alone; a level beyond
+    that sends the whole call to the general kernel, whichever position it has in the list."""
+    B, G = _gpu()
+    rows, d = 333, 4096
+    x = inputs.mp_activations(rows, d, 43, dtype=dtype, device=G.DEV, col_scale_seed=44)
+    x[5] = 0
+    x[6, 100:] = 0
+    m = len(ks)
+    mean = torch.zeros(m, dtype=torch.float64, device=G.DEV)
+    tau = torch.zeros(m * rows, dtype=dtype, device=G.DEV)
+    B.dct_mp_threshold_mean(x, rows, d, d, ks, mean, tau)
+    want = oracle.mp_threshold_mean(G.to_oracle(x), ks, d=d)
+    got_tau = G.as_np_bits(tau).reshape(m, rows)
+    assert np.array_equal(got_tau, want.tau.view(got_tau.dtype))
+    assert np.array_equal(mean.cpu().numpy(), want.mean)
+
+
+@pytest.mark.gpu
 def test_gpu_threshold_mean_inexact_sum_stays_within_the_stated_bound():
     B, G = _gpu()
     rows, d = 4096, 64
