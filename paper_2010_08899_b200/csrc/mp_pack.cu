@@ -821,7 +821,12 @@ extern "C" dct_status_t dct_mp_topk_pack_fwd(const void* x_act, dct_dtype_t dtyp
     if ((rows_out && !aligned_to(rows_out, 4)) || (tau_out && !aligned_to(tau_out, es))) return DCT_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (dtype == DCT_F32) {
-        bool handled = false;       // the warp-per-row fp32 kernel takes the same shapes as the bf16 one below
+        bool handled = false;
+        // narrow rows (256 columns, small k): the row stays in registers, four rows per warp
+        const dct_status_t narrow = launch_fwd_f32_narrow(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
+                                                          result, stream, &handled);
+        if (narrow != DCT_OK || handled) return narrow;
+        // the warp-per-row fp32 kernel takes the same shapes as the bf16 one below
         const dct_status_t fast = launch_fwd_f32_warp(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out,
                                                       result, stream, &handled);
         if (fast != DCT_OK || handled) return fast;

@@ -38,21 +38,6 @@ template <int E8> struct RowLayoutF32 {
 
 constexpr uint32_t kMaxMembers = 64;      // bucket members ranked through the list; more take the bit-serial route
 
-// upper halves of two fp32 words in one register: (hi16(b) << 16) | hi16(a)
-__device__ __forceinline__ uint32_t upper_halves(uint32_t a, uint32_t b) { return __byte_perm(a, b, 0x7632); }
-// Flags "upper 15 key bits >= low" of the 8 fp32 of one 32-byte piece, read as two 16-byte halves `first` and `second`
-// (a lane reads the halves in either order; w_first / w_second are the dot-product weights -2^j of the four columns
-// each half holds).  Exact for every bit pattern: per 16-bit half, bit 15 of ((x | 0x8000) - low) is set iff the
-// key's upper bits are >= low; a byte permutation with sign replication and two signed dot products collect the
-// eight flags, bit j = column j of the piece (see mask8_ge_exact in mp_warp.cuh).  low2 = low in both halves.
-__device__ __forceinline__ uint32_t piece_flags(uint4 first, uint4 second, uint32_t low2, uint32_t w_first, uint32_t w_second) {
-    const uint32_t t0 = (upper_halves(first.x, first.y) | 0x80008000u) - low2;
-    const uint32_t t1 = (upper_halves(first.z, first.w) | 0x80008000u) - low2;
-    const uint32_t t2 = (upper_halves(second.x, second.y) | 0x80008000u) - low2;
-    const uint32_t t3 = (upper_halves(second.z, second.w) | 0x80008000u) - low2;
-    return static_cast<uint32_t>(dp4a_ss(prmt(t2, t3, 0xFDB9u), w_second, dp4a_ss(prmt(t0, t1, 0xFDB9u), w_first, 0)));
-}
-
 // exact key >= low on 31-bit keys, 4 elements
 __device__ __forceinline__ uint32_t mask4_ge_exact(uint4 v, uint32_t low) {
     return ((v.x & 0x7FFFFFFFu) >= low ? 1u : 0u) | ((v.y & 0x7FFFFFFFu) >= low ? 2u : 0u) |

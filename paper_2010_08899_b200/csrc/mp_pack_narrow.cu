@@ -344,6 +344,345 @@ dct_status_t launch_narrow(const void* x_act, uint32_t rows, uint32_t ld, uint32
     return DCT_OK;
 }
 
+
+// ------------------------------------------------------------------------------------------
+// fp32 rows of 256 columns: the same scheme on two levels
+// ------------------------------------------------------------------------------------------
+// The paper's recommendation model runs in fp32.  A key has 31 bits; as in the other fp32 kernels the bound, the
+// candidate bits and the windowed histogram work on its upper 15 bits (the bucket: the bf16 truncation of |x|), which
+// gives the bucket of tau_i and how many of its members belong to the top k; the members (usually one) are then
+// ranked by their lower 16 bits.  A lane holds 32 consecutive columns (eight 16-byte loads), a group of G = 8 lanes
+// a row (four rows per warp); a candidate is two list words (value, column).
+constexpr uint32_t kNarrowScratchWordsF32 = 2 * kNarrowScratchWords;
+
+// Slow path (fp32): tau_i bit by bit over the 31 key bits by counting over the row in registers, then the ordered
+// emit straight from the row.  Called by the whole warp; groups without a row run along and store nothing.
+template <int G>
+__device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ xr, bool valid, uint32_t k, size_t out_base,
+                                                  uint32_t row, int16_t* __restrict__ cols_out,
+                                                  uint32_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
+                                                  uint32_t* __restrict__ tau_out) {
+    using Gr = Group<G>;
+    constexpr uint32_t E = 32u;
+    const uint32_t gl = lane_id() & (G - 1);
+    uint32_t key[E];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(xr + gl * E) + c);
+        key[4 * c] = v.x & 0x7FFFFFFFu;
+        key[4 * c + 1] = v.y & 0x7FFFFFFFu;
+        key[4 * c + 2] = v.z & 0x7FFFFFFFu;
+        key[4 * c + 3] = v.w & 0x7FFFFFFFu;
+    }
+    uint32_t tau_key = 0;
+#pragma unroll 1
+    for (int bit = 30; bit >= 0; --bit) {
+        const uint32_t trial = tau_key | (1u << bit);
+        uint32_t cnt = 0;
+#pragma unroll
+        for (int j = 0; j < static_cast<int>(E); ++j) cnt += key[j] >= trial ? 1u : 0u;
+        if (Gr::sum(cnt) >= k) tau_key = trial;
+    }
+    uint32_t gt_mask = 0, eq_mask = 0;
+#pragma unroll
+    for (int j = 0; j < static_cast<int>(E); ++j) {
+        gt_mask |= key[j] > tau_key ? 1u << j : 0u;
+        eq_mask |= key[j] == tau_key ? 1u << j : 0u;
+    }
+    const uint32_t n_gt_mine = __popc(gt_mask), n_eq_mine = __popc(eq_mask);
+    const uint32_t incl = Gr::inclusive_sum(n_gt_mine, gl);
+    const uint32_t take = k - Gr::last(incl);       // ties to keep, lowest columns first
+    uint32_t g_at = incl - n_gt_mine;
+    uint32_t e_at = Gr::inclusive_sum(n_eq_mine, gl) - n_eq_mine;
+    uint32_t m = valid ? (gt_mask | eq_mask) : 0u;
+    while (m) {
+        const uint32_t j = __ffs(m) - 1;
+        m &= m - 1;
+        const bool is_eq = (eq_mask >> j) & 1u;
+        if (!is_eq || e_at < take) {
+            const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
+            cols_out[pos] = static_cast<int16_t>(gl * E + j);
+            vals_out[pos] = xr[gl * E + j];
+            if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
+        }
+        g_at += is_eq ? 0u : 1u;
+        e_at += is_eq ? 1u : 0u;
+    }
+    if (valid && gl == 0 && tau_out) tau_out[row] = tau_key;
+}
+
+template <int G>
+__global__ void __launch_bounds__(kNarrowWarps * 32)
+mp_topk_fwd_f32_narrow_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
+                              int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
+                              int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
+                              dct_result_t* __restrict__ result) {
+    using Gr = Group<G>;
+    constexpr int kPieces = 4;                     // 32-byte pieces (8 columns) of a lane
+    constexpr uint32_t E = 32u;                    // columns per lane; the lane's candidate bits are one word
+    constexpr uint32_t kRows = Gr::kRows;
+    constexpr uint32_t kGuessMargin = 32;          // buckets below the previous row's
+    constexpr uint32_t kShareF32 = kNarrowScratchWordsF32 / kRows;     // values, then columns: 2 x kList words
+    static_assert(kShareF32 >= 2 * Gr::kList && kShareF32 >= 64u + G, "scratch share too small");
+    __shared__ uint32_t s_scratch[kNarrowWarps][kNarrowScratchWordsF32];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    const uint32_t gl = lane & (G - 1), group = lane / G, group_base = group * G;
+    uint32_t* share = s_scratch[warp] + group * kShareF32;    // this group's list / histogram / stage, in turn
+    uint32_t* share_c = share + Gr::kList;                    // the columns of the list / stage entries
+
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+    const uint32_t warps = blockDim.x >> 5;
+    const uint64_t bundles = (static_cast<uint64_t>(rows) + kRows - 1) / kRows;
+    const uint64_t first_bundle = blockIdx.x + static_cast<uint64_t>(gridDim.x) * warp;
+    const uint64_t bundle_step = static_cast<uint64_t>(gridDim.x) * warps;
+    auto row_of = [&](uint64_t bundle) -> uint64_t {          // a group past the last row reads the last row instead
+        const uint64_t r = bundle * kRows + group;
+        return r < rows ? r : rows - 1;
+    };
+    auto load_row = [&](uint64_t r, uint4 (&v)[2 * kPieces]) {
+        const uint4* src = reinterpret_cast<const uint4*>(x + r * ld + gl * E);
+#pragma unroll
+        for (int c = 0; c < 2 * kPieces; ++c) v[c] = __ldg(src + c);
+    };
+    uint4 cur[2 * kPieces];
+
+    uint32_t guess_low = 0;                         // bucket bound guessed from the group's previous row (0: none)
+    const bool have_bound = k <= G * kPieces;       // at least k leaves in a row
+    for (uint64_t bundle = first_bundle; bundle < bundles; bundle += bundle_step) {
+        const bool valid = bundle * kRows + group < rows;
+        const uint64_t row64 = row_of(bundle);
+        const uint32_t row = static_cast<uint32_t>(row64);
+        load_row(row64, cur);       // (no prefetch of the next rows: the registers buy more warps than it gains)
+        const uint32_t* xr = x + row64 * ld;
+        const size_t out_base = static_cast<size_t>(row) * k;
+
+        // ---- B (with A): candidate bits of the lane (bucket >= bound), one word in column order ------
+        uint32_t mask = 0, incl = 0, n_cand = 0;
+        auto build_mask = [&](uint32_t bound) {
+            const uint32_t low2 = bound | (bound << 16);
+            mask = 0;
+#pragma unroll
+            for (int c = 0; c < kPieces; ++c)
+                mask |= piece_flags(cur[2 * c], cur[2 * c + 1], low2, 0xF8FCFEFFu, 0x80C0E0F0u) << (8 * c);
+            incl = Gr::inclusive_sum(__popc(mask), gl);
+            n_cand = Gr::last(incl);
+        };
+        uint32_t low = guess_low;
+        bool settled = false;
+        if (have_bound && __all_sync(0xFFFFFFFFu, guess_low != 0)) {
+            build_mask(low);
+            settled = __all_sync(0xFFFFFFFFu, n_cand >= k && n_cand <= Gr::kList);
+        }
+        if (!settled) {
+            // exact bound: the k-th largest of the row's leaf maxima (buckets), bit by bit
+            uint32_t leaf[kPieces];
+#pragma unroll
+            for (int c = 0; c < kPieces; ++c) {
+                const uint4 a = cur[2 * c], b = cur[2 * c + 1];
+                const uint32_t u0 = upper_halves(a.x, a.y) & kAbsMask2, u1 = upper_halves(a.z, a.w) & kAbsMask2;
+                const uint32_t u2 = upper_halves(b.x, b.y) & kAbsMask2, u3 = upper_halves(b.z, b.w) & kAbsMask2;
+                const uint32_t m = as_u32(__hmax2(__hmax2(as_bf162(u0), as_bf162(u1)), __hmax2(as_bf162(u2), as_bf162(u3))));
+                leaf[c] = max(m & 0xFFFFu, m >> 16);
+            }
+            low = 0;
+            if (have_bound) {
+#pragma unroll 1
+                for (int bit = 14; bit >= 0; --bit) {
+                    const uint32_t trial = low | (1u << bit);
+                    uint32_t cnt = 0;
+#pragma unroll
+                    for (int c = 0; c < kPieces; ++c) cnt += leaf[c] >= trial ? 1u : 0u;
+                    if (Gr::sum(cnt) >= k) low = trial;
+                }
+            }
+            build_mask(low);
+        }
+        if (!have_bound || __any_sync(0xFFFFFFFFu, n_cand > Gr::kList || low == 0)) {
+            narrow_slow_path_f32<G>(xr, valid, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
+            continue;
+        }
+
+        // candidates into the group's list, column order: value and column
+        __syncwarp();                                   // whatever used the scratch before is done
+        {
+            uint32_t at = incl - __popc(mask);
+            uint32_t m = mask;
+            while (m) {
+                const uint32_t col = gl * E + (__ffs(m) - 1);
+                m &= m - 1;
+                share[at] = __ldg(xr + col);
+                share_c[at] = col;
+                ++at;
+            }
+        }
+        __syncwarp();
+        uint32_t ent[kNarrowPerLane], ent_c[kNarrowPerLane];   // value 0: unused slot (its bucket 0 lies below the bound)
+        const uint32_t per_lane = (n_cand + G - 1) / G;
+#pragma unroll
+        for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+            const uint32_t r = gl * per_lane + i;
+            const bool used = static_cast<uint32_t>(i) < per_lane && r < n_cand;
+            ent[i] = used ? share[r] : 0u;
+            ent_c[i] = used ? share_c[r] : 0u;
+        }
+        __syncwarp();                                   // the list is in registers: its words become the histogram
+
+        // ---- C: the bucket of tau_i among the candidates' buckets ------------------------------------------
+        uint32_t bucket = 0, take = 0;                  // `take` members of the bucket belong to the top k
+        bool found = false;
+        {
+            // 64 bins just above the bound, G private overflow bins behind them
+            const uint32_t drop = n_cand - k;
+            for (uint32_t b = gl; b < 64u + G; b += G) share[b] = 0;
+            __syncwarp();
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+                const uint32_t rel = ((ent[i] >> 16) & 0x7FFFu) - low;
+                atomicAdd(&share[rel < 64u ? rel : 64u + gl], 1u);
+            }
+            __syncwarp();
+            uint32_t h[Gr::kBins], own = 0;             // the lane looks after bins gl kBins .. gl kBins + kBins - 1
+#pragma unroll
+            for (int j = 0; j < static_cast<int>(Gr::kBins); ++j) {
+                h[j] = share[gl * Gr::kBins + j];
+                own += h[j];
+            }
+            uint32_t before = Gr::inclusive_sum(own, gl) - own;
+            uint32_t my_bucket = 0, my_take = 0;
+            bool mine = false;
+#pragma unroll
+            for (int j = 0; j < static_cast<int>(Gr::kBins); ++j) {
+                if (before <= drop && drop < before + h[j]) {
+                    mine = true;
+                    my_bucket = low + gl * Gr::kBins + j;
+                    my_take = h[j] - (drop - before);
+                }
+                before += h[j];
+            }
+            const uint32_t who = Gr::ballot(mine, group_base);
+            const uint32_t src = who ? __ffs(who) - 1 : 0u;
+            bucket = Gr::from(my_bucket, src);
+            take = Gr::from(my_take, src);
+            found = who != 0;
+            __syncwarp();
+        }
+        if (__any_sync(0xFFFFFFFFu, !found)) {
+            // the bucket lies beyond the window for some row: the k-th largest candidate bucket, bit by bit (every
+            // group recomputes; where the window had the answer this gives the same one)
+            uint32_t t = 0;
+#pragma unroll 1
+            for (int bit = 14; bit >= 0; --bit) {
+                const uint32_t trial = t | (1u << bit);
+                uint32_t cnt = 0;
+#pragma unroll
+                for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i)
+                    cnt += ((ent[i] >> 16) & 0x7FFFu) >= trial ? 1u : 0u;
+                if (Gr::sum(cnt) >= k) t = trial;
+            }
+            uint32_t above = 0;
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) above += ((ent[i] >> 16) & 0x7FFFu) > t ? 1u : 0u;
+            bucket = t;
+            take = k - Gr::sum(above);
+        }
+        // ---- tau_i inside the bucket: the take-th largest of its members' lower 16 key bits ------------------
+        uint32_t low16 = 0;
+        {
+            uint32_t members = 0, my_min = 0xFFFFu;
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+                const bool member = ((ent[i] >> 16) & 0x7FFFu) == bucket;
+                members += member ? 1u : 0u;
+                my_min = member ? min(my_min, ent[i] & 0xFFFFu) : my_min;
+            }
+            members = Gr::sum(members);
+            if (__all_sync(0xFFFFFFFFu, members == take)) {
+                // every member is kept (the usual case: one member): tau_i is the smallest of them
+#pragma unroll
+                for (int o = G / 2; o > 0; o >>= 1) my_min = min(my_min, __shfl_xor_sync(0xFFFFFFFFu, my_min, o, G));
+                low16 = my_min;
+            } else {
+#pragma unroll 1
+                for (int bit = 15; bit >= 0; --bit) {
+                    const uint32_t trial = low16 | (1u << bit);
+                    uint32_t cnt = 0;
+#pragma unroll
+                    for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i)
+                        cnt += (((ent[i] >> 16) & 0x7FFFu) == bucket && (ent[i] & 0xFFFFu) >= trial) ? 1u : 0u;
+                    if (Gr::sum(cnt) >= take) low16 = trial;
+                }
+            }
+        }
+        const uint32_t tau_key = (bucket << 16) | low16;
+        if (valid && gl == 0 && tau_out) tau_out[row] = tau_key;
+        guess_low = bucket > kGuessMargin ? bucket - kGuessMargin : 0u;
+
+        // ---- D: ordered emit ------------------------------------------------------------------------
+        {
+            uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+                const uint32_t key = ent[i] & 0x7FFFFFFFu;
+                counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
+            }
+            const uint32_t incl_c = Gr::inclusive_sum(counts, gl);
+            const uint32_t ties = k - (Gr::last(incl_c) >> 16);     // ties to keep, lowest columns first
+            const uint32_t before = incl_c - counts;
+            uint32_t e_at = before & 0xFFFFu;
+            uint32_t pos = (before >> 16) + (e_at < ties ? e_at : ties);
+#pragma unroll
+            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
+                const uint32_t key = ent[i] & 0x7FFFFFFFu;
+                const bool is_eq = key == tau_key;
+                const bool keep = key > tau_key || (is_eq && e_at < ties);
+                if (keep) {
+                    share[pos] = ent[i];
+                    share_c[pos] = ent_c[i];
+                }
+                pos += keep ? 1u : 0u;
+                e_at += is_eq ? 1u : 0u;
+            }
+        }
+        __syncwarp();
+        if (valid) {
+            for (uint32_t p = gl; p < k; p += G) {
+                cols_out[out_base + p] = static_cast<int16_t>(share_c[p]);
+                vals_out[out_base + p] = share[p];
+                if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
+            }
+        }
+        __syncwarp();
+    }
+}
+
+template <int G>
+dct_status_t launch_narrow_f32(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+                               void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
+                               cudaStream_t stream) {
+    auto kernel = mp_topk_fwd_f32_narrow_kernel<G>;
+    int per_sm = 0;
+    DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kNarrowWarps * 32, 0));
+    if (per_sm < 1) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint64_t bundles = (static_cast<uint64_t>(rows) + Group<G>::kRows - 1) / Group<G>::kRows;
+    const uint64_t ctas_needed = (bundles + kNarrowWarps - 1) / kNarrowWarps;
+    const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
+    const uint32_t grid = static_cast<uint32_t>(ctas_needed < max_grid ? ctas_needed : max_grid);
+    kernel<<<grid, kNarrowWarps * 32, 0, stream>>>(static_cast<const uint32_t*>(x_act), rows, ld, k, cols_out,
+                                                   static_cast<uint32_t*>(vals_out), rows_out,
+                                                   static_cast<uint32_t*>(tau_out), result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}
+
 }  // namespace
 
 // *handled = false: not a shape of this path; the caller goes on to the other kernels.
@@ -364,6 +703,21 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
             break;
         default: break;
     }
+    *handled = false;
+    return DCT_OK;
+}
+
+// fp32 rows of 256 columns, sparse k (same limits as the bf16 kernel above).
+dct_status_t launch_fwd_f32_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                   int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                   dct_result_t* result, cudaStream_t stream, bool* handled) {
+    *handled = false;
+    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || k > d / 8) return DCT_OK;
+    *handled = true;
+    // (512 columns with 16 lanes per row: 0.134 ms for 131072 rows against 0.110 ms on the warp-per-row kernel, which
+    // keeps them; 256 columns: 0.157 against 0.216 ms)
+    if (d == 256 && k <= 20)
+        return launch_narrow_f32<8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     *handled = false;
     return DCT_OK;
 }

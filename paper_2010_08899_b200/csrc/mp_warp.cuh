@@ -60,6 +60,21 @@ __device__ __forceinline__ uint32_t mask8_ge_exact(uint4 v, uint32_t low) {
     return static_cast<uint32_t>(dp4a_ss(b, 0x80C0E0F0u, dp4a_ss(a, 0xF8FCFEFFu, 0)));
 }
 
+// upper halves of two fp32 words in one register: (hi16(b) << 16) | hi16(a)
+__device__ __forceinline__ uint32_t upper_halves(uint32_t a, uint32_t b) { return __byte_perm(a, b, 0x7632); }
+// Flags "upper 15 key bits >= low" of the 8 fp32 of one 32-byte piece, read as two 16-byte halves `first` and `second`
+// (a lane reads the halves in either order; w_first / w_second are the dot-product weights -2^j of the four columns
+// each half holds).  Exact for every bit pattern: per 16-bit half, bit 15 of ((x | 0x8000) - low) is set iff the
+// key's upper bits are >= low; a byte permutation with sign replication and two signed dot products collect the
+// eight flags, bit j = column j of the piece (see mask8_ge_exact in mp_warp.cuh).  low2 = low in both halves.
+__device__ __forceinline__ uint32_t piece_flags(uint4 first, uint4 second, uint32_t low2, uint32_t w_first, uint32_t w_second) {
+    const uint32_t t0 = (upper_halves(first.x, first.y) | 0x80008000u) - low2;
+    const uint32_t t1 = (upper_halves(first.z, first.w) | 0x80008000u) - low2;
+    const uint32_t t2 = (upper_halves(second.x, second.y) | 0x80008000u) - low2;
+    const uint32_t t3 = (upper_halves(second.z, second.w) | 0x80008000u) - low2;
+    return static_cast<uint32_t>(dp4a_ss(prmt(t2, t3, 0xFDB9u), w_second, dp4a_ss(prmt(t0, t1, 0xFDB9u), w_first, 0)));
+}
+
 // v = *(uint2*)shared_address if p (a predicated load: no branch)
 __device__ __forceinline__ void lds64_if(uint2& v, uint32_t shared_address, bool p) {
     asm volatile("{\n\t.reg .pred q;\n\tsetp.ne.u32 q, %3, 0;\n\t@q ld.shared.v2.u32 {%0, %1}, [%2];\n\t}"
@@ -225,6 +240,11 @@ inline int fwd_candidates_per_lane(uint32_t d, uint32_t k) {
 dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                     int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                     dct_result_t* result, cudaStream_t stream, bool* handled);
+
+// The same for fp32 rows of 256 columns.
+dct_status_t launch_fwd_f32_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                   int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                   dct_result_t* result, cudaStream_t stream, bool* handled);
 
 // bf16, every lane looking after one contiguous span of the row (mp_pack_span.cu).
 dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,

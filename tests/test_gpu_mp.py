@@ -305,13 +305,15 @@ def test_mp_bf16_wide_rows(d):
         assert int(cols.max()) < d
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("d,ld", [(128, 128), (256, 256), (256, 264), (384, 384), (512, 512), (512, 640)])
-def test_mp_bf16_many_short_rows(d, ld):
-    """Many short bf16 rows (the widths of the paper's recommendation-model layers), more than one round of any
+def test_mp_many_short_rows(dtype, d, ld):
+    """Many short rows (the widths of the paper's recommendation-model layers), more than one round of any
     persistent grid and not a multiple of 32: contiguous and strided rows, sparse and denser k, rows of very
     different scales (a guess taken from a previous row fails in both directions), dead rows, rows where
     everything ties, rows with fewer than k non-zeros, rows of a few distinct values, rows with huge values
-    (thresholds at the top of the key range)."""
+    (thresholds at the top of the key range), and in fp32 denormal rows and rows whose values differ only in
+    their lower key bits."""
     rows = 32 * 148 * 3 + 21
     x = inputs.mp_activations(rows, d, 291 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=292 + d, ld=ld)
     sign = torch.where(inputs.dp_gaussian(rows * ld, 293 + d, G.DEV).view(rows, ld) > 0, 1.0, -1.0)
@@ -325,9 +327,12 @@ def test_mp_bf16_many_short_rows(d, ld):
     x[7::50] = inputs.quantize_mantissa(x[7::50], 2)
     x[8] = 3.0e38
     x[9, ::3] = 3.3e38
+    x[10] = x[10] * 1e-41                               # fp32: denormals, every key in bucket 0 (bf16: zeros)
+    x[11::50] = inputs.quantize_mantissa(x[11::50], 9)  # fp32: several members per bucket, ties inside it
+    x[12::50] = 1.0 + torch.arange(ld, device=G.DEV) * 2.0 ** -22     # fp32: one bucket holds the whole row
     x[rows - 1] = 0.5
-    x = x.to(torch.bfloat16).contiguous()
-    gx = inputs.mp_gradients(rows, d, 294 + d, dtype=torch.bfloat16, device=G.DEV, ld=ld)
+    x = x.to(dtype).contiguous()
+    gx = inputs.mp_gradients(rows, d, 294 + d, dtype=dtype, device=G.DEV, ld=ld)
     for k in sorted({1, 2, d // 20, d // 10, d // 4}):
         cols = _compare_fwd_bwd(x, gx, d, k, want_rows=(k == 2))
         assert int(cols.max()) < d
