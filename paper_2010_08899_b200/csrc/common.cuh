@@ -55,7 +55,7 @@ __device__ __forceinline__ uint32_t lanemask_lt() {
     return m;
 }
 
-// mbarrier + bulk asynchronous copies (TMA engine, 1-D, no multicast) ---------------------------
+// mbarrier + bulk asynchronous copies (TMA engine, 1-D, plain copies) ---------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t arrivals) {

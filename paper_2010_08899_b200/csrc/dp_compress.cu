@@ -21,7 +21,7 @@
 //   * dp_compress_stream_kernel -- the fast path for 16-byte aligned vectors.
 //     Persistent CTAs with three roles.  A load warp takes tickets and streams
 //     tiles into a ring of shared-memory stages with bulk asynchronous copies
-//     (TMA engine, no multicast).  Eight compute warps threshold a stage, store
+//     (TMA engine, plain copies).  Eight compute warps threshold a stage, store
 //     the new residual with 128-bit stores, publish the tile's counts and push
 //     the tile's survivors, in index order, into a small shared-memory queue.
 //     A scan warp runs the look-back for each tile and then drains that tile's
