@@ -27,12 +27,14 @@ namespace {
 
 constexpr int kNarrowWarps = 16;                 // warps per CTA
 constexpr uint32_t kNarrowPerLane = 5;           // candidates a lane holds in registers
-constexpr uint32_t kNarrowScratchWords = 320;    // per warp; a group's share holds its list / histogram / stage
+constexpr uint32_t kNarrowScratchWords = 320;    // per warp (G >= 8); a group's share holds its list / histogram / stage
+// G = 4 (8 rows per warp): 8 shares of 64 + G words for the histogram
+template <int G> __host__ __device__ constexpr uint32_t narrow_scratch_words() { return G >= 8 ? kNarrowScratchWords : (32u / G) * (64u + G); }
 
 template <int G> struct Group {
     static constexpr uint32_t kRows = 32u / G;                       // rows a warp works on at once
     static constexpr uint32_t kList = kNarrowPerLane * G;            // candidates of a row that fit
-    static constexpr uint32_t kShare = kNarrowScratchWords / kRows;  // scratch words of one group: >= 64 + G, >= kList
+    static constexpr uint32_t kShare = narrow_scratch_words<G>() / kRows;  // scratch words of one group: >= 64 + G, >= kList
     static constexpr uint32_t kBins = 64u / G;                       // window bins a lane looks after
     static_assert(kShare >= 64u + G && kShare >= kList, "scratch share too small");
 
@@ -122,7 +124,8 @@ mp_topk_fwd_bf16_narrow_kernel(const uint16_t* __restrict__ x, uint32_t rows, ui
     constexpr uint32_t E = E8 * 8u;                // columns per lane; the lane's candidate bits are one word
     constexpr uint32_t kRows = Gr::kRows;
     constexpr uint32_t kGuessMargin = 32;
-    __shared__ uint32_t s_scratch[kNarrowWarps][kNarrowScratchWords];
+    constexpr uint32_t kScratchWords = narrow_scratch_words<G>();
+    __shared__ uint32_t s_scratch[kNarrowWarps][kScratchWords];
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
     const uint32_t gl = lane & (G - 1), group = lane / G, group_base = group * G;
     uint32_t* share = s_scratch[warp] + group * Gr::kShare;   // this group's list / histogram / stage, in turn
@@ -695,6 +698,12 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
     if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0 || k > d / 8) return DCT_OK;
     *handled = true;
     switch (d) {
+        case 64:        // (8 leaves of 8 columns: the bound needs k <= 8)
+            if (k <= 8) return launch_narrow<2, 4>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            break;
+        case 128:
+            if (k <= 13) return launch_narrow<4, 4>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+            break;
         case 256:
             if (k <= 20) return launch_narrow<4, 8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
             break;
@@ -716,6 +725,8 @@ dct_status_t launch_fwd_f32_narrow(const void* x_act, uint32_t rows, uint32_t d,
     *handled = true;
     // (512 columns with 16 lanes per row: 0.134 ms for 131072 rows against 0.110 ms on the warp-per-row kernel, which
     // keeps them; 256 columns: 0.157 against 0.216 ms)
+    if (d == 128 && k <= 13)
+        return launch_narrow_f32<4>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     if (d == 256 && k <= 20)
         return launch_narrow_f32<8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     *handled = false;

@@ -306,7 +306,8 @@ def test_mp_bf16_wide_rows(d):
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-@pytest.mark.parametrize("d,ld", [(128, 128), (256, 256), (256, 264), (384, 384), (512, 512), (512, 640)])
+@pytest.mark.parametrize("d,ld", [(64, 64), (64, 72), (128, 128), (128, 136), (256, 256), (256, 264), (384, 384),
+                                  (512, 512), (512, 640)])
 def test_mp_many_short_rows(dtype, d, ld):
     """Many short rows (the widths of the paper's recommendation-model layers), more than one round of any
     persistent grid and not a multiple of 32: contiguous and strided rows, sparse and denser k, rows of very
