@@ -184,7 +184,8 @@ cudaError_t launch_unpack(const int16_t* cols, const void* vals, uint32_t rows, 
     if (staged) {
         const size_t smem = kUnpackWarps * row_bytes;
         auto kernel = k <= 256 ? mp_unpack_staged_kernel<T, 8> : (k <= 512 ? mp_unpack_staged_kernel<T, 16> : mp_unpack_staged_kernel<T, 0>);
-        if (smem > 48 * 1024) {
+        // (static shared memory counts against the 48 KiB a kernel gets without asking: ask well below that)
+        if (smem > 32 * 1024) {
             const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                        static_cast<int>(kUnpackWarps * 16 * 1024));
             if (e != cudaSuccess) return e;

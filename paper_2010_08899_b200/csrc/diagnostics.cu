@@ -288,8 +288,8 @@ dct_status_t launch_threshold_mean(const void* x_act, uint32_t rows, uint32_t d,
     }
     const size_t smem = ((static_cast<size_t>(d) * sizeof(T)) + 15) & ~static_cast<size_t>(15);
     auto kernel = mp_row_thresholds_kernel<T>;
-    if (smem > 48 * 1024)
-        DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    // (static shared memory counts against the 48 KiB a kernel gets without asking: ask well below that)
+    if (smem > 32 * 1024) DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     const int threads = d <= 4096 ? 128 : (d <= 8192 ? 256 : (d <= 16384 ? 512 : 1024));
     int per_sm = 0;
     DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));

@@ -761,7 +761,8 @@ dct_status_t launch_fwd(const void* x_act, uint32_t rows, uint32_t d, uint32_t l
                         cudaStream_t stream) {
     const size_t smem = ((static_cast<size_t>(d) * sizeof(T)) + 15) & ~static_cast<size_t>(15);
     auto kernel = mp_topk_pack_fwd_kernel<T>;
-    if (smem > 48 * 1024) DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    // (static shared memory counts against the 48 KiB a kernel gets without asking: ask well below that)
+    if (smem > 32 * 1024) DCT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                            static_cast<int>(smem)));
     const int threads = fwd_threads_for(d);
     int per_sm = 0;

@@ -140,7 +140,8 @@ def test_gpu_select_multi_equals_single_select_with_ties_and_unaligned_input():
 
 @pytest.mark.gpu
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("rows,d,ld", [(1, 1, 1), (33, 301, 304), (2048, 1024, 1024), (700, 4096, 4096), (3, 32768, 32768)])
+@pytest.mark.parametrize("rows,d,ld", [(1, 1, 1), (33, 301, 304), (2048, 1024, 1024), (700, 4096, 4096), (3, 32768, 32768),
+                                       (5, 12287, 12288)])
 def test_gpu_threshold_mean_matches_oracle(dtype, rows, d, ld):
     B, G = _gpu()
     x = inputs.mp_activations(rows, d, 41, dtype=dtype, device=G.DEV, col_scale_seed=42, ld=ld)

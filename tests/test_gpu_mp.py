@@ -43,6 +43,17 @@ def test_mp_odd_shapes(dtype, d, ld):
         assert int(cols.max()) < d
 
 
+@pytest.mark.parametrize("dtype,d", [(torch.float32, 12288), (torch.float32, 11800), (torch.bfloat16, 24576),
+                                     (torch.bfloat16, 24000)])
+def test_mp_rows_of_just_under_48_kib_in_the_general_kernel(dtype, d):
+    """A row of 44 to 48 KiB fits the shared memory a kernel gets without asking only if the kernel had no static
+    shared memory of its own: the general kernel (k = d / 2 is beyond every fast path) must ask for more there too."""
+    rows = 9
+    x = inputs.mp_activations(rows, d, 61 + d, dtype=dtype, device=G.DEV, col_scale_seed=62 + d)
+    gx = inputs.mp_gradients(rows, d, 63 + d, dtype=dtype, device=G.DEV)
+    _compare_fwd_bwd(x, gx, d, d // 2)
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_mp_misaligned_rows(dtype):
     rows, d, ld, k = 20, 301, 303, 31
