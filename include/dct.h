@@ -178,9 +178,9 @@ DCT_API dct_status_t dct_dp_compress(
  * row (bf16: d <= 8192 for k up to about d/10 and 441, d <= 3072 for k up
  * to 3d/8 and 2048; fp32: d <= 4096, k up to about d/10 and 441, denser k for
  * d <= 512) or by one CTA per row (bf16 rows of 3073..32768 columns with k
- * up to 3d/8 and 2300 where the warp kernel does not apply; fp32 rows of
- * 513..32768 columns that the warp kernels leave out, k up to 3d/8 and
- * 4096); everything else (denser k, odd strides, cols_out not 4-byte aligned
+ * up to 3d/8 where the warp kernel does not apply; fp32 rows of
+ * 513..32768 columns that the warp kernels leave out, k up to 3d/8);
+ * everything else (denser k, odd strides, cols_out not 4-byte aligned
  * for the denser and the wide cases) takes a general kernel that is several
  * times slower.  status may also be DCT_ERR_TIMEOUT if a
  * bounded wait for an asynchronous copy gave up (not seen in practice; the

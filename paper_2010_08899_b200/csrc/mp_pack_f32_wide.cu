@@ -28,7 +28,7 @@ namespace dct {
 namespace {
 
 constexpr uint32_t kWideWindowF32 = 64;           // widest window, in buckets (= histogram bins)
-constexpr uint32_t kWideMaxKF32 = 4096;
+constexpr uint32_t kWideMaxKF32 = 12288;        // 3/8 of the widest row (staging: 6 bytes per kept entry)
 constexpr int kWideRetriesF32 = 6;
 
 template <int W, int KW> struct WideLayoutF32 {

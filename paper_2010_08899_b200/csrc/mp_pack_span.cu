@@ -474,7 +474,7 @@ dct_status_t launch_span(const void* x_act, uint32_t rows, uint32_t d, uint32_t 
 // Several CTAs share an SM, so one CTA's load overlaps another's work.  A row whose window does not settle is not
 // handed to another routine: its threshold is found bit by bit (15 counting passes) and the row is then packed
 // with a window of one key, whose elements all tie at tau_i.
-constexpr uint32_t kWideMaxK = 2300;
+constexpr uint32_t kWideMaxK = 12288;            // 3/8 of the widest row (staging: 4 bytes per kept entry)
 constexpr int kWideRetries = 6;
 constexpr uint32_t kWideShrink = 3;               // window elements per lane (on average) from which the window narrows
 
