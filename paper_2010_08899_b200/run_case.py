@@ -11,6 +11,7 @@ A small command-line driver for profiling and quick timing of a single kernel at
     python -m paper_2010_08899_b200.run_case mp_unpack --rows 16384 --d 4096 --k 205 --dtype bf16
     python -m paper_2010_08899_b200.run_case select_multi --n 268435456          (75 / 90 / 95 % sparsity)
     python -m paper_2010_08899_b200.run_case threshold_mean --rows 16384 --d 4096 --dtype bf16
+    python -m paper_2010_08899_b200.run_case mp_fwd_sweep --dtype bf16    (a table: row widths x sparsity levels)
 
 It prints the mean device time per call (CUDA events) and the algorithmic GB/s.
 """
@@ -24,10 +25,42 @@ from . import binding as B
 from . import inputs
 
 
+def mp_fwd_sweep(args, dev, stream):
+    """The forward pack over row widths and sparsity levels, about 128 MiB of activations per cell (the generator of
+    the bench: ReLU of a Gaussian with log-normal column scales), `--iters` launches back to back after a warm-up
+    round; prints the algorithmic TB/s (input + k (2 + s) bytes per row)."""
+    dt = torch.float32 if args.dtype == "f32" else torch.bfloat16
+    es = 4 if args.dtype == "f32" else 2
+    widths = [64, 128, 192, 256, 320, 384, 512, 768, 1024, 1536, 2048, 3072, 4096, 6144, 8192, 12288, 16384, 32768]
+    fracs = [0.02, 0.05, 0.10, 0.25, 0.375, 0.5]
+    print("d      " + "".join(f"{f * 100:>9.1f}%" for f in fracs) + "   TB/s algorithmic, k = fraction of d")
+    for d in widths:
+        rows = max(64, (128 << 20) // (d * es))
+        x = inputs.mp_activations(rows, d, 7 + d, dtype=dt, device=dev, col_scale_seed=8 + d)
+        k_max = max(1, int(d * max(fracs)))
+        cols = torch.empty(rows * k_max, dtype=torch.int16, device=dev)       # sized for the largest k of the row
+        vals = torch.empty(rows * k_max, dtype=dt, device=dev)
+        line = f"{d:<7d}"
+        for f in fracs:
+            k = max(1, int(d * f))
+            for phase in range(2):
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for _ in range(args.iters):
+                    B.dct_mp_topk_pack_fwd(x, rows, d, d, k, cols[: rows * k], vals[: rows * k], None, None, None, stream)
+                b.record(stream)
+                b.synchronize()
+            ms = a.elapsed_time(b) / args.iters
+            line += f"{(rows * d * es + rows * k * (2 + es)) / (ms * 1e-3) / 1e12:10.2f}"
+        print(line, flush=True)
+        del x, cols, vals
+
+
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("entry", choices=["select", "compress", "select_compress", "compress_layers", "decompress", "mp_fwd", "mp_bwd", "mp_unpack",
-                                     "select_multi", "threshold_mean"])
+                                     "select_multi", "threshold_mean", "mp_fwd_sweep"])
     ap.add_argument("--n", type=int, default=1 << 28)
     ap.add_argument("--k", type=int, default=0, help="survivor target (default: 0.01 %% of n, or 5 %% of d)")
     ap.add_argument("--rows", type=int, default=16384)
@@ -58,6 +91,8 @@ def main():
         print(f"cudaLimitMaxL2FetchGranularity <- {args.l2_fetch} B: return code {rc}, now {got.value} B")
     stream = torch.cuda.current_stream()
     reset = lambda: None
+    if args.entry == "mp_fwd_sweep":
+        return mp_fwd_sweep(args, dev, stream)
     gen = {"mixture": inputs.dp_mixture, "gaussian": inputs.dp_gaussian, "dlrm": inputs.dp_dlrm_like}[args.dist]
 
     if args.entry == "compress_layers":
