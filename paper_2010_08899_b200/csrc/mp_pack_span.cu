@@ -898,13 +898,22 @@ dct_status_t launch_fwd_bf16_span(const void* x_act, uint32_t rows, uint32_t d, 
     if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0) return DCT_OK;
     if (!aligned_to(cols_out, 4) || !aligned_to(vals_out, 4)) return DCT_OK;   // the paired stores need 4-byte aligned outputs
     *handled = true;
-    // the smallest instantiated buffer of 256 * E8 columns that holds the row
+    // The smallest buffer of 256 * E8 columns that holds the row, every E8 up to 12: a lane's span is 8 E8 columns, and
+    // a row that fills only part of the lanes crowds their lists (43690x1536, k = 576 in the 2048-column buffer: 0.98 ms,
+    // nearly every row on the slow path; in its own buffer 0.095 ms).
 #define DCT_SPAN_WIDTH(E8) \
     if (d <= 256u * E8) return launch_span<E8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
     DCT_SPAN_WIDTH(1);
     DCT_SPAN_WIDTH(2);
+    DCT_SPAN_WIDTH(3);
     DCT_SPAN_WIDTH(4);
+    DCT_SPAN_WIDTH(5);
+    DCT_SPAN_WIDTH(6);
+    DCT_SPAN_WIDTH(7);
     DCT_SPAN_WIDTH(8);
+    DCT_SPAN_WIDTH(9);
+    DCT_SPAN_WIDTH(10);
+    DCT_SPAN_WIDTH(11);
     DCT_SPAN_WIDTH(12);
 #undef DCT_SPAN_WIDTH
     *handled = false;
