@@ -64,17 +64,17 @@ template <int G, int PLN = static_cast<int>(kNarrowPerLaneFew)> struct Group {
 // memory), then the ordered emit straight from the row.  Called by the whole warp; groups without a row
 // (valid == false) run along on a row of their own that exists and store nothing.
 template <int E8, int G>
-__device__ __noinline__ void narrow_slow_path(const uint16_t* __restrict__ xr, bool valid, uint32_t k, size_t out_base,
-                                              uint32_t row, int16_t* __restrict__ cols_out,
+__device__ __noinline__ void narrow_slow_path(const uint16_t* __restrict__ xr, uint32_t d, bool valid, uint32_t k,
+                                              size_t out_base, uint32_t row, int16_t* __restrict__ cols_out,
                                               uint16_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
                                               uint16_t* __restrict__ tau_out) {
     using Gr = Group<G>;
     constexpr uint32_t E = E8 * 8u;
     const uint32_t gl = lane_id() & (G - 1);
     const uint4* mine = reinterpret_cast<const uint4*>(xr + gl * E);
-    uint4 v[E8];
+    uint4 v[E8];                                   // (a lane past the end of the row holds zeros: the last columns)
 #pragma unroll
-    for (int c = 0; c < E8; ++c) v[c] = __ldg(mine + c);
+    for (int c = 0; c < E8; ++c) v[c] = gl * E < d ? __ldg(mine + c) : make_uint4(0, 0, 0, 0);
     uint32_t tau_key = 0;
 #pragma unroll 1
     for (int bit = 14; bit >= 0; --bit) {
@@ -116,7 +116,7 @@ __device__ __noinline__ void narrow_slow_path(const uint16_t* __restrict__ xr, b
 
 template <int E8, int G, int PLN>
 __global__ void __launch_bounds__(kNarrowWarps * 32)
-mp_topk_fwd_bf16_narrow_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
+mp_topk_fwd_bf16_narrow_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
                                int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
                                dct_result_t* __restrict__ result) {
@@ -149,16 +149,19 @@ mp_topk_fwd_bf16_narrow_kernel(const uint16_t* __restrict__ x, uint32_t rows, ui
         const uint64_t r = bundle * kRows + group;
         return r < rows ? r : rows - 1;
     };
+    // A row of d <= G E columns (d a multiple of E): the lanes past its end hold zeros, which lie below every bound
+    // and, being the last columns, lose every tie.
+    const bool lane_in = gl * E < d;
     auto load_row = [&](uint64_t r, uint4 (&v)[E8]) {
         const uint4* src = reinterpret_cast<const uint4*>(x + r * ld + gl * E);
 #pragma unroll
-        for (int c = 0; c < E8; ++c) v[c] = __ldg(src + c);
+        for (int c = 0; c < E8; ++c) v[c] = lane_in ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
     };
     uint4 cur[E8], nxt[E8];
     if (first_bundle < bundles) load_row(row_of(first_bundle), nxt);
 
     uint32_t guess_low = 0;                         // bound guessed from the group's previous row (0: none)
-    const bool have_bound = k <= G * E8;            // at least k leaves in a row
+    const bool have_bound = k <= d / 8u;            // at least k leaves in a row
     for (uint64_t bundle = first_bundle; bundle < bundles; bundle += bundle_step) {
         const bool valid = bundle * kRows + group < rows;
         const uint64_t row64 = row_of(bundle);
@@ -208,7 +211,7 @@ mp_topk_fwd_bf16_narrow_kernel(const uint16_t* __restrict__ x, uint32_t rows, ui
             build_mask(low);
         }
         if (!have_bound || __any_sync(0xFFFFFFFFu, n_cand > Gr::kList || low == 0)) {
-            narrow_slow_path<E8, G>(xr, valid, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
+            narrow_slow_path<E8, G>(xr, d, valid, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
             continue;
         }
 
@@ -328,7 +331,7 @@ mp_topk_fwd_bf16_narrow_kernel(const uint16_t* __restrict__ x, uint32_t rows, ui
 }
 
 template <int E8, int G, int PLN>
-dct_status_t launch_narrow(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+dct_status_t launch_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
                            void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
                            cudaStream_t stream) {
     auto kernel = mp_topk_fwd_bf16_narrow_kernel<E8, G, PLN>;
@@ -341,7 +344,7 @@ dct_status_t launch_narrow(const void* x_act, uint32_t rows, uint32_t ld, uint32
     const uint64_t ctas_needed = (bundles + kNarrowWarps - 1) / kNarrowWarps;
     const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < max_grid ? ctas_needed : max_grid);
-    kernel<<<grid, kNarrowWarps * 32, 0, stream>>>(static_cast<const uint16_t*>(x_act), rows, ld, k, cols_out,
+    kernel<<<grid, kNarrowWarps * 32, 0, stream>>>(static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out,
                                                    static_cast<uint16_t*>(vals_out), rows_out,
                                                    static_cast<uint16_t*>(tau_out), result);
     DCT_CUDA_TRY(cudaGetLastError());
@@ -362,8 +365,8 @@ constexpr uint32_t kNarrowScratchWordsF32 = 2 * kNarrowScratchWords;
 // Slow path (fp32): tau_i bit by bit over the 31 key bits by counting over the row in registers, then the ordered
 // emit straight from the row.  Called by the whole warp; groups without a row run along and store nothing.
 template <int G>
-__device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ xr, bool valid, uint32_t k, size_t out_base,
-                                                  uint32_t row, int16_t* __restrict__ cols_out,
+__device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ xr, uint32_t d, bool valid, uint32_t k,
+                                                  size_t out_base, uint32_t row, int16_t* __restrict__ cols_out,
                                                   uint32_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
                                                   uint32_t* __restrict__ tau_out) {
     using Gr = Group<G>;
@@ -372,7 +375,7 @@ __device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ x
     uint32_t key[E];
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(xr + gl * E) + c);
+        const uint4 v = gl * E < d ? __ldg(reinterpret_cast<const uint4*>(xr + gl * E) + c) : make_uint4(0, 0, 0, 0);
         key[4 * c] = v.x & 0x7FFFFFFFu;
         key[4 * c + 1] = v.y & 0x7FFFFFFFu;
         key[4 * c + 2] = v.z & 0x7FFFFFFFu;
@@ -417,7 +420,7 @@ __device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ x
 
 template <int G, int PLN>
 __global__ void __launch_bounds__(kNarrowWarps * 32)
-mp_topk_fwd_f32_narrow_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t ld, uint32_t k,
+mp_topk_fwd_f32_narrow_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                               int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
                               int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
                               dct_result_t* __restrict__ result) {
@@ -451,15 +454,16 @@ mp_topk_fwd_f32_narrow_kernel(const uint32_t* __restrict__ x, uint32_t rows, uin
         const uint64_t r = bundle * kRows + group;
         return r < rows ? r : rows - 1;
     };
+    const bool lane_in = gl * E < d;                // (lanes past the end of the row hold zeros)
     auto load_row = [&](uint64_t r, uint4 (&v)[2 * kPieces]) {
         const uint4* src = reinterpret_cast<const uint4*>(x + r * ld + gl * E);
 #pragma unroll
-        for (int c = 0; c < 2 * kPieces; ++c) v[c] = __ldg(src + c);
+        for (int c = 0; c < 2 * kPieces; ++c) v[c] = lane_in ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
     };
     uint4 cur[2 * kPieces];
 
     uint32_t guess_low = 0;                         // bucket bound guessed from the group's previous row (0: none)
-    const bool have_bound = k <= G * kPieces;       // at least k leaves in a row
+    const bool have_bound = k <= d / 8u;            // at least k leaves in a row
     for (uint64_t bundle = first_bundle; bundle < bundles; bundle += bundle_step) {
         const bool valid = bundle * kRows + group < rows;
         const uint64_t row64 = row_of(bundle);
@@ -510,7 +514,7 @@ mp_topk_fwd_f32_narrow_kernel(const uint32_t* __restrict__ x, uint32_t rows, uin
             build_mask(low);
         }
         if (!have_bound || __any_sync(0xFFFFFFFFu, n_cand > Gr::kList || low == 0)) {
-            narrow_slow_path_f32<G>(xr, valid, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
+            narrow_slow_path_f32<G>(xr, d, valid, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
             continue;
         }
 
@@ -668,7 +672,7 @@ mp_topk_fwd_f32_narrow_kernel(const uint32_t* __restrict__ x, uint32_t rows, uin
 }
 
 template <int G, int PLN>
-dct_status_t launch_narrow_f32(const void* x_act, uint32_t rows, uint32_t ld, uint32_t k, int16_t* cols_out,
+dct_status_t launch_narrow_f32(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
                                void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
                                cudaStream_t stream) {
     auto kernel = mp_topk_fwd_f32_narrow_kernel<G, PLN>;
@@ -681,7 +685,7 @@ dct_status_t launch_narrow_f32(const void* x_act, uint32_t rows, uint32_t ld, ui
     const uint64_t ctas_needed = (bundles + kNarrowWarps - 1) / kNarrowWarps;
     const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < max_grid ? ctas_needed : max_grid);
-    kernel<<<grid, kNarrowWarps * 32, 0, stream>>>(static_cast<const uint32_t*>(x_act), rows, ld, k, cols_out,
+    kernel<<<grid, kNarrowWarps * 32, 0, stream>>>(static_cast<const uint32_t*>(x_act), rows, d, ld, k, cols_out,
                                                    static_cast<uint32_t*>(vals_out), rows_out,
                                                    static_cast<uint32_t*>(tau_out), result);
     DCT_CUDA_TRY(cudaGetLastError());
@@ -701,23 +705,19 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
     *handled = true;
     // 5 candidates per lane up to k = 2.5 lanes of the group, 8 up to 4.25 lanes (the bound leaves ~1.3 k candidates,
     // 1.45 k at the 99th percentile)
-#define DCT_NARROW(E8, G, K5, K8)                                                                                       \
-    if (k <= K5) return launch_narrow<E8, G, 5>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream); \
-    if (k <= K8) return launch_narrow<E8, G, 8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
-    switch (d) {
-        case 64:        // (8 leaves of 8 columns: the bound needs k <= 8)
-            DCT_NARROW(2, 4, 8, 8);
-            break;
-        case 128:       // (16 leaves)
-            DCT_NARROW(4, 4, 13, 16);
-            break;
-        case 256:
-            DCT_NARROW(4, 8, 20, 32);
-            break;
-        case 512:       // (k = 51 with 8 candidates per lane: 0.125 ms for 131072 rows, the warp-per-row kernel 0.104)
-            DCT_NARROW(4, 16, 40, 40);
-            break;
-        default: break;
+#define DCT_NARROW(E8, G, K5, K8)                                                                                          \
+    if (k <= K5) return launch_narrow<E8, G, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream); \
+    if (k <= K8) return launch_narrow<E8, G, 8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
+    // (k <= d / 8 was checked above: the bound needs k leaves of 8 columns; rows narrower than the group's 32 G
+    // columns, in whole lanes of 32, leave the lanes past their end empty)
+    if (d == 64) {
+        DCT_NARROW(2, 4, 8, 8);
+    } else if (d % 32 == 0 && d <= 128) {
+        DCT_NARROW(4, 4, 13, 16);
+    } else if (d % 32 == 0 && d <= 256) {
+        DCT_NARROW(4, 8, 20, 32);
+    } else if (d % 32 == 0 && d <= 512) {  // (k = 51 with 8 candidates per lane: 0.125 ms for 131072 rows of 512, the warp-per-row kernel 0.104)
+        DCT_NARROW(4, 16, 40, 40);
     }
 #undef DCT_NARROW
     *handled = false;
@@ -733,14 +733,14 @@ dct_status_t launch_fwd_f32_narrow(const void* x_act, uint32_t rows, uint32_t d,
     *handled = true;
     // (512 columns with 16 lanes per row: 0.134 ms for 131072 rows against 0.110 ms on the warp-per-row kernel, which
     // keeps them; 256 columns: 0.157 against 0.216 ms)
-    if (d == 128 && k <= 13)
-        return launch_narrow_f32<4, 5>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-    if (d == 128 && k <= 16)
-        return launch_narrow_f32<4, 8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-    if (d == 256 && k <= 20)
-        return launch_narrow_f32<8, 5>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-    if (d == 256 && k <= 32)
-        return launch_narrow_f32<8, 8>(x_act, rows, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    // (rows narrower than the group's 32 G columns, in whole lanes of 32, leave the lanes past their end empty)
+    if (d % 32 == 0 && d <= 128) {
+        if (k <= 13) return launch_narrow_f32<4, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        if (k <= 16) return launch_narrow_f32<4, 8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    } else if (d % 32 == 0 && d <= 256) {
+        if (k <= 20) return launch_narrow_f32<8, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        if (k <= 32) return launch_narrow_f32<8, 8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    }
     *handled = false;
     return DCT_OK;
 }

@@ -317,8 +317,8 @@ def test_mp_bf16_wide_rows(d):
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
-@pytest.mark.parametrize("d,ld", [(64, 64), (64, 72), (128, 128), (128, 136), (256, 256), (256, 264), (384, 384),
-                                  (512, 512), (512, 640)])
+@pytest.mark.parametrize("d,ld", [(32, 32), (64, 64), (64, 72), (96, 96), (128, 128), (128, 136), (192, 200), (256, 256),
+                                  (256, 264), (320, 320), (384, 384), (512, 512), (512, 640)])
 def test_mp_many_short_rows(dtype, d, ld):
     """Many short rows (the widths of the paper's recommendation-model layers), more than one round of any
     persistent grid and not a multiple of 32: contiguous and strided rows, sparse and denser k, rows of very
@@ -339,6 +339,7 @@ def test_mp_many_short_rows(dtype, d, ld):
     x[7::50] = inputs.quantize_mantissa(x[7::50], 2)
     x[8] = 3.0e38
     x[9, ::3] = 3.3e38
+    x[13, 1:] = 0.0                                     # one non-zero: the first zeros, never a column past the row, fill up
     x[10] = x[10] * 1e-41                               # fp32: denormals, every key in bucket 0 (bf16: zeros)
     x[11::50] = inputs.quantize_mantissa(x[11::50], 9)  # fp32: several members per bucket, ties inside it
     x[12::50] = 1.0 + torch.arange(ld, device=G.DEV) * 2.0 ** -22     # fp32: one bucket holds the whole row
