@@ -19,16 +19,16 @@
 //
 // Two kernels share the per-tile arithmetic:
 //   * dp_compress_stream_kernel -- the fast path for 16-byte aligned vectors.
-//     Persistent CTAs with three roles.  A load warp takes tickets and streams
+//     Persistent CTAs with four roles.  A load warp takes tickets and streams
 //     tiles into a ring of shared-memory stages with bulk asynchronous copies
 //     (TMA engine, plain copies).  Eight compute warps threshold a stage, store
 //     the new residual with 128-bit stores, publish the tile's counts and push
-//     the tile's survivors, in index order, into a small shared-memory queue.
-//     A scan warp runs the look-back for each tile and then drains that tile's
-//     queue to (idx, val).  Nothing on the compute warps' path waits for another
-//     CTA; a tile with more survivors than a queue slot holds is written by the
-//     compute warps themselves once its prefix is known (dense inputs: slower,
-//     same results).
+//     the tile's survivors, in index order, into a shared-memory ring that holds
+//     a whole tile's worth of entries.  A look-back warp finds each tile's output
+//     offset, starting from the tile the CTA resolved before it, and two drain
+//     warps write the tile's ring entries to (idx, val).  Nothing on the compute warps'
+//     path waits for another CTA, whatever the density of the survivors; they wait
+//     for their own drain warps only when the ring or the slot table is full.
 //   * dp_compress_tile_kernel -- one CTA per tile with plain loads and stores:
 //     the ragged last tile and vectors that are not 16-byte aligned.
 #include <mutex>
@@ -95,11 +95,18 @@ __global__ void dp_compress_init_kernel(CompressCtrl* ctrl, uint64_t* tile_state
 
 // Look-back by one warp: counts of all tiles before `tile`.  Each round examines a window of
 // 32 * kLookWide descriptors (all loads of a round are in flight together, so a round costs one
-// L2 round trip): persistent CTAs advance in step, so the nearest descriptor that already holds
-// an inclusive prefix is typically a few hundred tiles back.  Every wait is bounded.
-constexpr int kLookWide = 8;
+// L2 round trip).  The walk ends at the nearest descriptor that holds an inclusive prefix, or at
+// `anchor`: a tile whose inclusive counts the caller already knows (-1 and zeros: the empty prefix
+// before tile 0).  A persistent CTA passes the tile it resolved last, about one grid width back,
+// so its look-back needs only the other tiles' own counts, which their CTAs publish at once, and
+// never waits for another CTA's look-back.  Every wait is bounded.
+constexpr int kLookWide = 10;
+struct LookAnchor {
+    int64_t tile;
+    uint32_t gt, eq;
+};
 __device__ __forceinline__ void lookback(const uint64_t* tile_state, const CompressCtrl* ctrl,
-                                         uint32_t tile, uint32_t spin_limit,
+                                         uint32_t tile, uint32_t spin_limit, const LookAnchor& anchor,
                                          uint32_t& excl_gt, uint32_t& excl_eq, bool& timed_out) {
     const uint32_t lane = lane_id();
     uint32_t sum_gt = 0, sum_eq = 0;
@@ -110,7 +117,9 @@ __device__ __forceinline__ void lookback(const uint64_t* tile_state, const Compr
 #pragma unroll
         for (int q = 0; q < kLookWide; ++q) {            // distance from the tile: q * 32 + lane + 1
             const int64_t t = window_end - 1 - (q * 32 + static_cast<int64_t>(lane));
-            d[q] = t >= 0 ? ld_relaxed_u64(tile_state + t) : kStatusInclusive;   // before tile 0: empty prefix
+            d[q] = t > anchor.tile ? ld_relaxed_u64(tile_state + t)
+                                   : pack_counts(kStatusInclusive, t == anchor.tile ? anchor.gt : 0u,
+                                                 t == anchor.tile ? anchor.eq : 0u);
         }
         bool done = false;
 #pragma unroll
@@ -159,13 +168,14 @@ __device__ __forceinline__ bool resolve_tile_prefix(uint64_t* tile_state, Compre
                                                     uint32_t tile, uint32_t last_tile, uint32_t cta_gt,
                                                     uint32_t cta_eq, uint64_t budget, uint64_t capacity,
                                                     uint32_t spin_limit, uint32_t& excl_gt, uint32_t& excl_eq,
-                                                    bool publish_aggregate) {
+                                                    bool publish_aggregate,
+                                                    const LookAnchor& anchor = LookAnchor{-1, 0u, 0u}) {
     const uint32_t lane = lane_id();
     if (lane == 0 && publish_aggregate) publish_tile_aggregate(tile_state, tile, cta_gt, cta_eq);
     bool timed_out = false;
     excl_gt = 0;
     excl_eq = 0;
-    if (tile > 0) lookback(tile_state, ctrl, tile, spin_limit, excl_gt, excl_eq, timed_out);
+    if (tile > 0) lookback(tile_state, ctrl, tile, spin_limit, anchor, excl_gt, excl_eq, timed_out);
     if (timed_out) {
         if (lane == 0) {
             atomicExch(&ctrl->abort, 1u);
@@ -414,34 +424,56 @@ dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ resi
 }
 
 // ------------------------------------------------------------------------------------------
-// fast path: persistent CTAs; load warp + compute warps + scan warp
+// fast path: persistent CTAs; load warp + compute warps + look-back warp + drain warps
 // ------------------------------------------------------------------------------------------
-constexpr int kSlots = 8;                                // tiles a CTA may be ahead of its scan warp
-constexpr uint32_t kQueueEntries = 512;                  // survivors of one tile that fit a slot
-constexpr uint32_t kEqBit = 0x80000000u;                 // queue entry: index (31 bits) | "equal to tau"
-constexpr int kLoadWarp = kWarps, kScanWarp = kWarps + 1;
-constexpr int kStreamThreads = kThreads + 64;
+constexpr int kSlots = 16;                               // tiles a CTA may be ahead of its drain warp
+constexpr uint32_t kRingEntries = 6080;                  // survivors waiting in shared memory: any one tile fits
+constexpr uint32_t kEqBit = 0x80000000u;                 // ring entry: "equal to tau"
+constexpr uint32_t kAheadGrace = 8;                      // polls of a waiting compute warp before it counts tiles ahead
+constexpr int kDrainWarps = 2;                           // warps that share the write-out of a tile's entries
+constexpr int kLoadWarp = kWarps, kLookWarp = kWarps + 1, kDrainWarp0 = kWarps + 2;
+constexpr int kStreamThreads = kThreads + 64 + 32 * kDrainWarps;
+static_assert(kRingEntries >= kTileElems && kTileElems <= 4096, "a tile fits the ring; 12-bit fields");
 
 struct __align__(128) StreamSmem {
     float g[kStages][kTileElems];
     float e[kStages][kTileElems];
-    uint2 queue[kSlots][kQueueEntries];  // (index | kEqBit, value bits) in index order
+    // survivors of the tiles that are not written out yet, in tile order and, inside a tile, index order:
+    // x = offset inside the tile | (equal-to-tau elements of the tile before it) << 12 | kEqBit, y = value bits
+    uint2 ring[kRingEntries];
     uint64_t full[kStages];              // load -> compute: stage holds a tile (bulk loads landed)
     uint64_t empty[kStages];             // compute -> load: stage may be refilled
-    uint64_t agg_ready[kSlots];          // compute (8 warps) -> scan: counts and queue of the slot are written
-    uint64_t prefix_ready[kSlots];       // scan -> compute: exclusive prefix of the slot's tile is in prefix[]
-    uint64_t slot_free[kSlots];          // scan -> compute: the slot may be reused
+    uint64_t agg_ready[kSlots];          // compute (thread 0) -> look-back: tile and counts of the slot are written
+    uint64_t entries_ready[kSlots];      // compute (8 warps) -> drain: the tile's ring entries are written
+    uint64_t prefix_ready[kSlots];       // look-back -> drain: exclusive prefix of the slot's tile is in prefix[]
     uint32_t tile[kStages];
     uint32_t layer[kStages];             // batched calls: which vector the stage's tile belongs to
     uint32_t warp_tot[2][kWarps];
     uint32_t slot_tile[kSlots];
     uint32_t slot_layer[kSlots];
     uint32_t slot_agg[kSlots];           // (gt << 16) | eq of the tile
-    uint32_t slot_direct[kSlots];        // 1: the compute warps write this tile's output themselves
+    uint32_t slot_start[kSlots];         // ring position of the tile's first entry
+    uint32_t slot_head[kSlots];          // running count of ring entries up to and including the tile's
     uint32_t prefix[kSlots][2];
     uint32_t aborted[kSlots];
+    uint32_t ahead[4];                   // counts of a tile taken ahead of its turn: eq | gt << 13 | warps that added << 26
+    volatile uint32_t ring_tail[kDrainWarps];   // drain warp -> compute: running count of ring entries it is done with
+    volatile uint32_t drained[kDrainWarps];     // drain warp -> compute: tiles it is done with (their slots may be reused)
     volatile uint32_t stop;              // a bounded wait gave up inside this CTA
 };
+// two CTAs per SM: the SM has 228 KiB, of which each CTA costs 1 KiB on top of what it asks for
+static_assert(sizeof(StreamSmem) <= 113 * 1024, "two CTAs of the streaming kernel per SM");
+
+// Bounded wait until a counter another warp advances has reached `target` (wrapping 32-bit counts).
+__device__ __forceinline__ bool counter_wait_bounded(const volatile uint32_t* counter, uint32_t target, uint32_t limit,
+                                                     const volatile uint32_t* stop) {
+    for (uint32_t i = 0; i < limit; ++i) {
+        if (static_cast<int32_t>(*counter - target) >= 0) return true;
+        if ((i & 63u) == 63u && *stop) return false;
+        if (i >= 4) __nanosleep(100);          // leave the shared-memory pipe to the warps that are being waited for
+    }
+    return false;
+}
 
 // One vector of a call as the kernels see it (a batched call has a table of these in the workspace).
 struct LayerDesc {
@@ -507,10 +539,15 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
             mbar_init(&sm.empty[s], 1);
         }
         for (int r = 0; r < kSlots; ++r) {
-            mbar_init(&sm.agg_ready[r], kWarps);
+            mbar_init(&sm.agg_ready[r], 1);
+            mbar_init(&sm.entries_ready[r], kWarps);
             mbar_init(&sm.prefix_ready[r], 1);
-            mbar_init(&sm.slot_free[r], 1);
         }
+        for (int v = 0; v < kDrainWarps; ++v) {
+            sm.ring_tail[v] = 0;
+            sm.drained[v] = 0;
+        }
+        for (int v = 0; v < 4; ++v) sm.ahead[v] = 0;
         sm.stop = 0;
         mbar_init_fence();
         fence_proxy_async_all();
@@ -570,15 +607,56 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
         }
     }
 
-    if (warp == kScanWarp) {
-        // ================= scan warp: look-back, then drain the tile's queue ==================
+    if (warp == kLookWarp) {
+        // ================= look-back warp: the exclusive prefix of each tile, in the CTA's tile order ==========
+        TileParams P;
+        uint32_t cur_layer = 0xFFFFFFFFu;
+        if (!kBatched) P = load_params(single, tile_state_base);
+        LookAnchor anchor{-1, 0u, 0u};        // the tile this warp resolved last (same vector), with its inclusive counts
+        bool chain_ok = true;                 // false once a look-back of this CTA gave up: nothing later is sent
+        for (uint32_t it = 0;; ++it) {
+            const int r = it % kSlots;
+            const uint32_t parity = (it / kSlots) & 1u;
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&sm.agg_ready[r], parity, kMbarLimit, &sm.stop))) {
+                sm.stop = 1;
+                return;
+            }
+            const uint32_t tile = sm.slot_tile[r];
+            if (tile == kInvalidTile) {
+                if (lane == 0) mbar_arrive(&sm.prefix_ready[r]);
+                return;
+            }
+            if (kBatched && sm.slot_layer[r] != cur_layer) {
+                cur_layer = sm.slot_layer[r];
+                P = load_params(batch.layers[cur_layer], tile_state_base);
+                anchor = LookAnchor{-1, 0u, 0u};
+            }
+            const uint32_t tot = sm.slot_agg[r];
+            const uint32_t cta_gt = tot >> 16, cta_eq = tot & 0xFFFFu;
+            uint32_t excl_gt = 0, excl_eq = 0;
+            chain_ok = chain_ok && resolve_tile_prefix(P.tile_state, ctrl, P.result, tile, P.last_tile, cta_gt, cta_eq,
+                                                       P.budget, P.capacity, spin_limit, excl_gt, excl_eq, false, anchor);
+            anchor = LookAnchor{static_cast<int64_t>(tile), excl_gt + cta_gt, excl_eq + cta_eq};
+            if (lane == 0) {
+                sm.prefix[r][0] = excl_gt;
+                sm.prefix[r][1] = excl_eq;
+                sm.aborted[r] = chain_ok ? 0u : 1u;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.prefix_ready[r]);
+        }
+    }
+
+    if (warp >= kDrainWarp0) {
+        // ================= drain warps: ring entries of each tile -> (idx, val), 32 entries per warp in turn =====
+        const uint32_t dw = warp - kDrainWarp0;
         TileParams P;
         uint32_t cur_layer = 0xFFFFFFFFu;
         if (!kBatched) P = load_params(single, tile_state_base);
         for (uint32_t it = 0;; ++it) {
             const int r = it % kSlots;
             const uint32_t parity = (it / kSlots) & 1u;
-            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&sm.agg_ready[r], parity, kMbarLimit, &sm.stop))) {
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&sm.prefix_ready[r], parity, kMbarLimit, &sm.stop))) {
                 sm.stop = 1;
                 return;
             }
@@ -588,40 +666,30 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
                 cur_layer = sm.slot_layer[r];
                 P = load_params(batch.layers[cur_layer], tile_state_base);
             }
-            const uint32_t tot = sm.slot_agg[r];
-            const uint32_t cta_gt = tot >> 16, cta_eq = tot & 0xFFFFu;
-            uint32_t excl_gt, excl_eq;
-            const bool ok = resolve_tile_prefix(P.tile_state, ctrl, P.result, tile, P.last_tile, cta_gt, cta_eq,
-                                                P.budget, P.capacity, spin_limit, excl_gt, excl_eq, false);
-            if (sm.slot_direct[r]) {
-                if (lane == 0) {
-                    sm.prefix[r][0] = excl_gt;
-                    sm.prefix[r][1] = excl_eq;
-                    sm.aborted[r] = ok ? 0u : 1u;
-                }
-            } else {
-                // entries are in index order; eq entries are counted on the fly
-                const uint32_t cnt = cta_gt + cta_eq;
-                uint32_t eq_run = 0;
-                for (uint32_t base = 0; base < cnt; base += 32) {
-                    const uint32_t q = base + lane;
-                    const uint2 ent = q < cnt ? sm.queue[r][q] : make_uint2(0u, 0u);
-                    const bool is_eq = q < cnt && (ent.x & kEqBit);
-                    const uint32_t eq_bal = __ballot_sync(0xFFFFFFFFu, is_eq);
-                    if (q < cnt) {
-                        const uint32_t local_eq = eq_run + __popc(eq_bal & lanemask_lt());
-                        const uint32_t local_gt = q - local_eq;
-                        place_survivor(ent.x & ~kEqBit, __uint_as_float(ent.y), is_eq, uint64_t(excl_gt) + local_gt,
-                                       uint64_t(excl_eq) + local_eq, P.budget, P.capacity, !ok, P.idx_out, P.val_out,
-                                       P.residual);
-                    }
-                    eq_run += __popc(eq_bal);
-                }
+            if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&sm.entries_ready[r], parity, kMbarLimit, &sm.stop))) {
+                sm.stop = 1;
+                return;
             }
-            __syncwarp();
+            const uint32_t tot = sm.slot_agg[r];
+            const uint32_t cnt = (tot >> 16) + (tot & 0xFFFFu);
+            const uint32_t start = sm.slot_start[r];
+            const uint64_t excl_gt = sm.prefix[r][0], excl_eq = sm.prefix[r][1];
+            const bool aborted = sm.aborted[r] != 0;
+            const uint32_t tile_base = tile * kTileElems;
+#pragma unroll 4
+            for (uint32_t q = dw * 32u + lane; q < cnt; q += 32u * kDrainWarps) {
+                const uint32_t at = start + q;
+                const uint2 ent = sm.ring[at < kRingEntries ? at : at - kRingEntries];
+                const uint32_t local_eq = (ent.x >> 12) & 0xFFFu;
+                place_survivor(tile_base + (ent.x & 0xFFFu), __uint_as_float(ent.y), (ent.x & kEqBit) != 0,
+                               excl_gt + (q - local_eq), excl_eq + local_eq, P.budget, P.capacity, aborted, P.idx_out,
+                               P.val_out, P.residual);
+            }
+            __syncwarp();                      // every lane has read its entries: the compute warps may overwrite them
             if (lane == 0) {
-                mbar_arrive(&sm.prefix_ready[r]);
-                mbar_arrive(&sm.slot_free[r]);
+                sm.ring_tail[dw] = sm.slot_head[r];
+                __threadfence_block();
+                sm.drained[dw] = it + 1u;
             }
         }
     }
@@ -632,10 +700,12 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
     if (!kBatched) P = load_params(single, tile_state_base);
     bool healthy = true;
     uint32_t it = 0;
+    uint32_t ring_head = 0;                   // running count of ring entries written by this CTA
+    uint32_t ring_pos = 0;                    // the same modulo the size of the ring
+    uint32_t ahead_upto = 0;                  // last iteration whose tile this warp has counted ahead of its turn
     for (;; ++it) {
         const int s = it % kStages;
         const int r = it % kSlots;
-        const uint32_t slot_use = it / kSlots;
         if (!named_barrier_all(1, kThreads,
                                mbar_wait_bounded(&sm.full[s], (it / kStages) & 1u, kMbarLimit, &sm.stop) &&
                                    !sm.stop)) {
@@ -687,54 +757,122 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
             before_warp += (v < static_cast<int>(warp)) ? t : 0u;
         }
         const uint32_t cta_gt = cta_tot >> 16, cta_eq = cta_tot & 0xFFFFu;
-        const bool direct = cta_gt + cta_eq > kQueueEntries;
+        const uint32_t cnt = cta_gt + cta_eq;
         if (tid == 0) {
             mbar_arrive(&sm.empty[s]);
-            // later tiles may need these counts right now; the scan warp adds the prefix when it gets here
+            // later tiles need these counts right now; the look-back warp adds the prefix when it gets here
             publish_tile_aggregate(P.tile_state, tile, cta_gt, cta_eq);
+            sm.ahead[it & 3u] = 0;                // (whatever was counted ahead for this tile has served)
         }
-        // the slot must have been drained by the scan warp (it normally was, long ago)
+        // The slot must have been drained (it normally was, long ago); the look-back may start as soon as the slot
+        // holds the tile's counts, it does not need the ring entries.
         bool slot_ok = true;
-        if (slot_use > 0)
-            slot_ok = mbar_wait_bounded(&sm.slot_free[r], (slot_use - 1u) & 1u, kMbarLimit, &sm.stop);
-        if (!__all_sync(0xFFFFFFFFu, slot_ok)) sm.stop = 1;   // seen by everybody at the next vote
-        if (tid == 0) {
-            sm.slot_tile[r] = tile;
-            sm.slot_layer[r] = cur_layer;
-            sm.slot_agg[r] = cta_tot;
-            sm.slot_direct[r] = direct ? 1u : 0u;
+        if (warp == 0) {
+            if (lane < kDrainWarps)               // one lane per drain warp
+                slot_ok = counter_wait_bounded(&sm.drained[lane], it + 1u - kSlots, kMbarLimit, &sm.stop);
+            slot_ok = __all_sync(0xFFFFFFFFu, slot_ok);
+            if (lane == 0 && slot_ok) {
+                sm.slot_tile[r] = tile;
+                sm.slot_layer[r] = cur_layer;
+                sm.slot_agg[r] = cta_tot;
+                sm.slot_start[r] = ring_pos;
+                sm.slot_head[r] = ring_head + cnt;
+                mbar_arrive(&sm.agg_ready[r]);
+            }
         }
-        if (!direct && warp_tot != 0 && slot_ok) {
-            uint2* q = sm.queue[r];
-            for_each_flagged(gt_mask, eq_mask, warp_base, before_warp,
-                             [&](int b, uint32_t i, uint32_t local_gt, uint32_t local_eq, bool is_eq) {
-                                 q[local_gt + local_eq] = make_uint2(i | (is_eq ? kEqBit : 0u), __float_as_uint(w[b]));
+        // the tile's share of the ring must have been drained as well
+        const uint32_t need_tail = ring_head + cnt - kRingEntries;
+        bool room = true;
+        if (lane < kDrainWarps) room = static_cast<int32_t>(sm.ring_tail[lane] - need_tail) >= 0;
+        room = __all_sync(0xFFFFFFFFu, room);
+        if (!room) {
+            // This warp has to wait for the drain warps, they for the look-back, and the look-back for the counts of
+            // every earlier tile.  The CTA has taken tickets for the tiles in its other stages already; if their counts
+            // came only after this wait, the CTAs behind those tiles would stop as well, each of them holding tickets
+            // of its own, and the whole grid would advance one tile after the other.  So the warp first counts its span
+            // of the tiles the CTA has taken and the last warp to do so publishes their counts.
+            // (Only after a short while: most waits end by themselves before that.)
+            uint32_t a = 1;
+            for (uint32_t polls = 1;; ++polls) {
+                room = true;
+                if (lane < kDrainWarps) room = static_cast<int32_t>(sm.ring_tail[lane] - need_tail) >= 0;
+                room = __all_sync(0xFFFFFFFFu, room);
+                if (room || polls >= kMbarLimit || ((polls & 63u) == 63u && sm.stop)) break;
+                const uint32_t j = it + a;
+                if (polls < kAheadGrace || a > static_cast<uint32_t>(kStages)) {
+                    __nanosleep(100);          // leave the shared-memory pipe to the warps that are being waited for
+                    continue;
+                }
+                ++a;
+                if (j <= ahead_upto) continue;
+                const int sa = j % kStages;
+                if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&sm.full[sa], (j / kStages) & 1u, kMbarLimit, &sm.stop)))
+                    break;
+                const uint32_t tile_a = sm.tile[sa];
+                if (tile_a == kInvalidTile) {
+                    a = kStages + 1;           // nothing follows
+                    continue;
+                }
+                uint32_t tau_key_a = P.tau_key;
+                uint64_t* tile_state_a = P.tile_state;
+                if (kBatched && sm.layer[sa] != cur_layer) {
+                    const LayerDesc& d = batch.layers[sm.layer[sa]];
+                    tau_key_a = key_f32(*d.tau);
+                    tile_state_a = tile_state_base + d.first_desc;
+                }
+                const float4* gs = reinterpret_cast<const float4*>(sm.g[sa]) + warp * (kWarpElems / 4) + lane;
+                const float4* es = reinterpret_cast<const float4*>(sm.e[sa]) + warp * (kWarpElems / 4) + lane;
+                uint32_t mine = 0;
+#pragma unroll
+                for (int v = 0; v < kVecs; ++v) {
+                    const float4 g4 = gs[v * 32], e4 = es[v * 32];
+                    const float wa[4] = {__fadd_rn(g4.x, e4.x), __fadd_rn(g4.y, e4.y), __fadd_rn(g4.z, e4.z),
+                                         __fadd_rn(g4.w, e4.w)};
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint32_t kw = key_f32(wa[c]);
+                        mine += (kw > tau_key_a ? (1u << 13) : 0u) + (kw == tau_key_a ? 1u : 0u);
+                    }
+                }
+                mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+                if (lane == 0) {
+                    const uint32_t all = atomicAdd(&sm.ahead[j & 3u], mine + (1u << 26)) + mine + (1u << 26);
+                    if ((all >> 26) == static_cast<uint32_t>(kWarps))
+                        publish_tile_aggregate(tile_state_a, tile_a, (all >> 13) & 0x1FFFu, all & 0x1FFFu);
+                }
+                ahead_upto = j;
+            }
+        }
+        room = room && slot_ok;
+        if (!room) sm.stop = 1;                   // seen by everybody at the next vote
+        if (warp_tot != 0 && room) {
+            const uint32_t in_tile = warp * kWarpElems;
+            for_each_flagged(gt_mask, eq_mask, in_tile, before_warp,
+                             [&](int b, uint32_t off, uint32_t local_gt, uint32_t local_eq, bool is_eq) {
+                                 const uint32_t at = ring_pos + local_gt + local_eq;
+                                 sm.ring[at < kRingEntries ? at : at - kRingEntries] =
+                                     make_uint2(off | (local_eq << 12) | (is_eq ? kEqBit : 0u), __float_as_uint(w[b]));
                              });
         }
+        ring_head += cnt;
+        ring_pos += cnt;
+        ring_pos -= ring_pos >= kRingEntries ? kRingEntries : 0u;
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.agg_ready[r]);
-        if (direct) {
-            // dense tile: wait for its prefix and write the output straight from registers
-            if (!named_barrier_all(1, kThreads,
-                                   mbar_wait_bounded(&sm.prefix_ready[r], slot_use & 1u, kMbarLimit, &sm.stop))) {
-                healthy = false;
-                break;
-            }
-            if (warp_tot != 0)
-                emit_warp(w, gt_mask, eq_mask, warp_base, before_warp, sm.prefix[r][0], sm.prefix[r][1], P.budget,
-                          P.capacity, sm.aborted[r] != 0, P.idx_out, P.val_out, P.residual);
-        }
+        if (lane == 0) mbar_arrive(&sm.entries_ready[r]);
     }
     if (healthy) {
-        // tell the scan warp that no more tiles follow
+        // tell the other two warps that no more tiles follow
         const int r = it % kSlots;
-        const uint32_t slot_use = it / kSlots;
-        bool slot_ok = true;
-        if (slot_use > 0)
-            slot_ok = mbar_wait_bounded(&sm.slot_free[r], (slot_use - 1u) & 1u, kMbarLimit, &sm.stop);
-        if (tid == 0) sm.slot_tile[r] = kInvalidTile;
-        __syncwarp();
-        if (lane == 0 && slot_ok) mbar_arrive(&sm.agg_ready[r]);
+        if (warp == 0) {
+            bool slot_ok = true;
+            if (lane < kDrainWarps)
+                slot_ok = counter_wait_bounded(&sm.drained[lane], it + 1u - kSlots, kMbarLimit, &sm.stop);
+            slot_ok = __all_sync(0xFFFFFFFFu, slot_ok);
+            if (lane == 0 && slot_ok) {
+                sm.slot_tile[r] = kInvalidTile;
+                mbar_arrive(&sm.agg_ready[r]);
+            }
+        }
     } else if (tid == 0) {
         sm.stop = 1;
         atomicExch(&ctrl->abort, 1u);
@@ -855,7 +993,7 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         }
         const int sms = sm_count();
         if (sms <= 0) return DCT_ERR_CUDA;
-        const uint32_t ctas_per_sm = sizeof(StreamSmem) <= 110 * 1024 ? 2 : 1;
+        const uint32_t ctas_per_sm = 2;
         const uint32_t max_grid = static_cast<uint32_t>(sms) * ctas_per_sm;
         const uint32_t grid = num_full < max_grid ? num_full : max_grid;
         LayerDesc single{};
@@ -1040,7 +1178,7 @@ extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, ui
                                               static_cast<int>(sizeof(StreamSmem))));
             configured_device = dev;
         }
-        const uint32_t ctas_per_sm = sizeof(StreamSmem) <= 110 * 1024 ? 2 : 1;
+        const uint32_t ctas_per_sm = 2;
         const uint32_t max_grid = static_cast<uint32_t>(sms) * ctas_per_sm;
         const uint32_t grid = total_full < max_grid ? total_full : max_grid;
         DCT_CUDA_TRY(launch_chained_smem(dp_compress_stream_kernel<true>, grid, kStreamThreads, sizeof(StreamSmem), stream,

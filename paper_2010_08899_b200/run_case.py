@@ -12,6 +12,7 @@ A small command-line driver for profiling and quick timing of a single kernel at
     python -m paper_2010_08899_b200.run_case select_multi --n 268435456          (75 / 90 / 95 % sparsity)
     python -m paper_2010_08899_b200.run_case threshold_mean --rows 16384 --d 4096 --dtype bf16
     python -m paper_2010_08899_b200.run_case mp_fwd_sweep --dtype bf16    (a table: row widths x sparsity levels)
+    python -m paper_2010_08899_b200.run_case dp_sweep                     (a table: vector sizes x densities)
 
 It prints the mean device time per call (CUDA events) and the algorithmic GB/s.
 """
@@ -57,10 +58,57 @@ def mp_fwd_sweep(args, dev, stream):
         del x, cols, vals
 
 
+def dp_sweep(args, dev, stream):
+    """DCT-DP over vector sizes and densities k / n: the select, then `--iters` compress iterations with that
+    threshold (the error carried from one to the next, a fresh gradient each time from two shifted buffers), and the
+    one-call L = 1 iteration.  Prints ms per call and the algorithmic TB/s (select: 4 B per element read once;
+    compress and L = 1: 12 B per element + 8 B per survivor)."""
+    sizes = [1 << 16, 1 << 20, 1 << 22, 1 << 24, 1 << 25, 1 << 26, 1 << 28, 1 << 30]
+    densities = [1e-4, 1e-3, 1e-2, 0.05, 0.25]
+    print("n         density        k   select ms (TB/s)   compress ms (TB/s)   L=1 ms (TB/s)")
+    for n in sizes:
+        slack = 64
+        g = [inputs.dp_mixture(n + slack, 11 + j, dev) for j in range(2)]
+        e = torch.zeros(n, device=dev)
+        tau = torch.zeros(1, device=dev)
+        idx = torch.empty(n, dtype=torch.int32, device=dev)                    # capacity n: nothing is cut off
+        val = torch.empty(n, device=dev)
+        res = B.new_result(dev)
+        ws_s = B.new_workspace(B.dct_threshold_select_workspace_bytes(n), dev)
+        ws_c = B.new_workspace(B.dct_dp_compress_workspace_bytes(n), dev)
+        ws_l = B.new_workspace(B.dct_dp_select_compress_workspace_bytes(n), dev)
+        fresh = lambda i: g[i % 2][4 * (i // 2): 4 * (i // 2) + n]
+
+        def timed(call, reps):
+            for phase in range(2):
+                a = torch.cuda.Event(enable_timing=True)
+                b = torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                for i in range(reps):
+                    call(i)
+                b.record(stream)
+                b.synchronize()
+            return a.elapsed_time(b) / reps
+
+        for dens in densities:
+            k = max(1, int(n * dens))
+            ms_s = timed(lambda i: B.dct_threshold_select(fresh(i), None, n, k, tau, res, ws_s, stream), args.iters)
+            B.dct_threshold_select(fresh(0), None, n, k, tau, res, ws_s, stream)
+            e.zero_()
+            ms_c = timed(lambda i: B.dct_dp_compress(fresh(i), e, n, tau, None, idx, val, n, res, ws_c, stream), args.iters)
+            surv = B.read_result(res).count
+            e.zero_()
+            ms_l = timed(lambda i: B.dct_dp_select_compress(fresh(i), e, n, k, tau, idx, val, n, res, ws_l, stream), args.iters)
+            tb = lambda bytes_, ms: bytes_ / (ms * 1e-3) / 1e12
+            print(f"2^{n.bit_length() - 1:<3d} {dens:10.4f} {k:12d}   {ms_s:8.4f} ({tb(4 * n, ms_s):5.2f})"
+                  f"   {ms_c:8.4f} ({tb(12 * n + 8 * surv, ms_c):5.2f})   {ms_l:8.4f} ({tb(12 * n + 8 * k, ms_l):5.2f})", flush=True)
+        del g, e, idx, val, ws_s, ws_c, ws_l
+
+
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("entry", choices=["select", "compress", "select_compress", "compress_layers", "decompress", "mp_fwd", "mp_bwd", "mp_unpack",
-                                     "select_multi", "threshold_mean", "mp_fwd_sweep"])
+                                     "select_multi", "threshold_mean", "mp_fwd_sweep", "dp_sweep"])
     ap.add_argument("--n", type=int, default=1 << 28)
     ap.add_argument("--k", type=int, default=0, help="survivor target (default: 0.01 %% of n, or 5 %% of d)")
     ap.add_argument("--rows", type=int, default=16384)
@@ -93,6 +141,8 @@ def main():
     reset = lambda: None
     if args.entry == "mp_fwd_sweep":
         return mp_fwd_sweep(args, dev, stream)
+    if args.entry == "dp_sweep":
+        return dp_sweep(args, dev, stream)
     gen = {"mixture": inputs.dp_mixture, "gaussian": inputs.dp_gaussian, "dlrm": inputs.dp_dlrm_like}[args.dist]
 
     if args.entry == "compress_layers":
@@ -203,7 +253,7 @@ def main():
             nbytes = 4 * n
         else:
             e = torch.zeros(n, device=dev)
-            cap = max(n // 64, 1024)
+            cap = min(n, max(n // 64, 1024, 2 * k))      # room for every survivor of a zero residual
             idx = torch.empty(cap, dtype=torch.int32, device=dev)
             val = torch.empty(cap, device=dev)
             ws_c = B.new_workspace(B.dct_dp_compress_workspace_bytes(n), dev)
