@@ -19,6 +19,11 @@
 //   3. if the count c satisfies k <= c <= capacity, tau is the k-th largest candidate (radix select
 //      over the small buffer) and n_gt, n_eq follow from the candidates, since every element >= tau
 //      is one of them.  Otherwise -- the sample misjudged the vector -- the three full passes run.
+// When k is too large for all elements >= lo to fit the candidate buffer (k of a few per cent of n and
+// more), the sample also gives an upper bound `hi`, chosen the same way on the other side of tau: the
+// streaming pass counts the keys above hi and keeps the keys in [lo, hi] -- a band around tau that holds
+// a fraction of a per cent of the vector whatever k is -- and tau is the (k - count above hi)-th largest
+// of those.
 // Every decision is taken on the device; all kernels are enqueued up front and the ones that are
 // not needed return at once.  The result is exact in every case.
 #include "common.cuh"
@@ -34,7 +39,7 @@ constexpr int kBins = 2048;
 constexpr int kPasses = 3;
 constexpr uint32_t kSampleSize = 1u << 20;                   // elements in the sample
 constexpr uint32_t kSampleGroup = 8;                         // consecutive elements taken at each sample position
-constexpr uint32_t kMaxCandidates = 1u << 22;                // candidate buffer: at most 16 MiB
+constexpr uint32_t kMaxCandidates = 1u << 23;                // candidate buffer: at most 32 MiB
 constexpr uint32_t kMinSampledN = 1u << 25;                  // below this the three plain passes are cheaper
 
 __host__ __device__ constexpr int pass_shift(int p) { return p == 0 ? 20 : (p == 1 ? 10 : 0); }
@@ -54,13 +59,16 @@ struct SelectState {
     uint32_t hist[kPasses * kBins];
 };
 
-// Workspace layout: three select states (whole vector, sample, candidates), the candidate counter,
-// the candidate keys.
+// Workspace layout: the select states (whole vector, sample for the lower bound, candidates, sample for the
+// upper bound), the counters of the filter pass, the candidate keys.
 struct SelectWorkspace {
-    SelectState full, sample, cand;
-    uint32_t cand_count;      // keys >= lo met by the filter pass (may exceed the capacity)
+    SelectState full, sample, cand, sample_hi;
+    uint32_t cand_count;      // keys in [lo, hi] met by the filter pass (may exceed the capacity)
     uint32_t cand_capacity;
-    uint32_t pad[62];
+    uint32_t above_count;     // keys above hi met by the filter pass (0 without an upper bound)
+    uint32_t filter_done;     // CTAs of the filter pass that have finished
+    uint32_t k_total;         // the rank the call asks for
+    uint32_t pad[59];
 };
 
 constexpr int kInitThreads = 1024;
@@ -80,7 +88,7 @@ __device__ __forceinline__ void reset_state(SelectState* st, uint32_t k, uint32_
 }
 
 __global__ void select_init_kernel(SelectWorkspace* ws, uint32_t n, uint32_t k, uint32_t sample_n, uint32_t sample_k,
-                                   uint32_t cand_capacity, dct_result_t* result) {
+                                   uint32_t cand_capacity, dct_result_t* result, uint32_t sample_k_hi = 0) {
     chain_release_next();
     const uint32_t i = threadIdx.x;
     const bool sampled = sample_n != 0;
@@ -88,9 +96,14 @@ __global__ void select_init_kernel(SelectWorkspace* ws, uint32_t n, uint32_t k, 
     // the sample only has to give a lower bound of its rank-th key: two passes (21 of the 31 key bits) do
     reset_state(&ws->sample, sample_k, sample_n, sampled ? 1u : 0u, i, kInitThreads, 1u);
     reset_state(&ws->cand, k, 0u, 0u, i, kInitThreads);
+    // the upper bound, where the call uses one: the select rounds down, the filter adds the bits it left out
+    reset_state(&ws->sample_hi, sample_k_hi, sample_n, sampled && sample_k_hi ? 1u : 0u, i, kInitThreads, 1u);
     if (i == 0) {
         ws->cand_count = 0;
         ws->cand_capacity = cand_capacity;
+        ws->above_count = 0;
+        ws->filter_done = 0;
+        ws->k_total = k;
         result->status = DCT_OK;
         result->reserved = 0;
         result->count = 0;
@@ -267,7 +280,8 @@ select_pass_kernel(Source src, SelectState* st, float* __restrict__ tau_out, dct
 // misjudged the vector, the plain one over the whole vector -- one launch instead of two, of which one would return
 // at once.  Which one: with k_decide == 0 the enabled flags of the two states say (a kernel before this one set
 // them); otherwise every CTA of every pass decides for itself from the candidate count that the filter left, the
-// same way each time: the candidates if they are at least k_decide and all fitted into their buffer.
+// same way each time: the candidates if rank k_decide lies among them (fewer than k_decide keys above them, at least
+// k_decide together with those) and all fitted into their buffer.
 template <int kPass, typename CandSource, bool kVectorised>
 __global__ void __launch_bounds__(kSelThreads)
 select_pass_either_kernel(CandSource cand_src, VectorSource full_src, SelectWorkspace* ws, uint32_t k_decide,
@@ -281,7 +295,8 @@ select_pass_either_kernel(CandSource cand_src, VectorSource full_src, SelectWork
     uint32_t cand_n;
     if (k_decide) {
         cand_n = ws->cand_count;
-        use_cand = cand_n >= k_decide && cand_n <= ws->cand_capacity;
+        const uint32_t above = ws->above_count;       // (the filter has set the candidates' rank to k_decide - above)
+        use_cand = above < k_decide && k_decide - above <= cand_n && cand_n <= ws->cand_capacity;
         use_full = !use_cand;
     } else {
         cand_n = ws->cand.n;
@@ -295,14 +310,18 @@ select_pass_either_kernel(CandSource cand_src, VectorSource full_src, SelectWork
                                                            s_last);
 }
 
-// The single streaming pass of the sampled path: every key >= key(lo) goes to the candidate buffer.
-template <bool kVectorised>
+// The single streaming pass of the sampled path: every key in [lo, hi] goes to the candidate buffer and the keys
+// above hi are counted (without an upper bound hi is the largest key: nothing is above it).  The last CTA to finish
+// hands the candidate select its rank: k less the keys above hi.
+template <bool kVectorised, bool kBand>
 __global__ void __launch_bounds__(kSelThreads)
 select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t* __restrict__ cand_keys) {
     chain_wait_previous();
     if (!ws->sample.enabled) return;
     const uint32_t lo = ws->sample.key_out;
+    const uint32_t hi = kBand ? (ws->sample_hi.key_out | ((1u << pass_shift(1)) - 1u)) : 0xFFFFFFFFu;
     const uint32_t capacity = ws->cand_capacity;
+    uint32_t above = 0;                             // keys above hi seen by this thread
     // Each warp collects its survivors in a small shared-memory buffer and moves them to the candidate
     // buffer 64 or more at a time, so the global counter sees one atomic per flush, not one per survivor.
     constexpr uint32_t kWarpBuf = 96, kFlushAt = 64;
@@ -344,12 +363,15 @@ select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t
                 const uint32_t k1 = key_f32(add ? __fadd_rn(g4[j].y, e4[j].y) : g4[j].y);
                 const uint32_t k2 = key_f32(add ? __fadd_rn(g4[j].z, e4[j].z) : g4[j].z);
                 const uint32_t k3 = key_f32(add ? __fadd_rn(g4[j].w, e4[j].w) : g4[j].w);
+                if (kBand) above += (k0 > hi ? 1u : 0u) + (k1 > hi ? 1u : 0u) + (k2 > hi ? 1u : 0u) + (k3 > hi ? 1u : 0u);
+                const bool in0 = k0 >= lo && (!kBand || k0 <= hi), in1 = k1 >= lo && (!kBand || k1 <= hi);
+                const bool in2 = k2 >= lo && (!kBand || k2 <= hi), in3 = k3 >= lo && (!kBand || k3 <= hi);
                 const uint32_t top = max(max(k0, k1), max(k2, k3));
-                if (__any_sync(0xFFFFFFFFu, top >= lo)) {
-                    keep(k0 >= lo, k0);
-                    keep(k1 >= lo, k1);
-                    keep(k2 >= lo, k2);
-                    keep(k3 >= lo, k3);
+                if (__any_sync(0xFFFFFFFFu, kBand ? (in0 || in1 || in2 || in3) : top >= lo)) {
+                    keep(in0, k0);
+                    keep(in1, k1);
+                    keep(in2, k2);
+                    keep(in3, k3);
                 }
             }
         } else {
@@ -358,12 +380,23 @@ select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t
                 const uint32_t i = i0 + lane_id();
                 const bool in = i < n && i < base + kSelChunk;
                 const uint32_t key = in ? key_at(src, i) : 0u;
-                keep(in && key >= lo, key);
+                above += in && key > hi ? 1u : 0u;
+                keep(in && key >= lo && key <= hi, key);
             }
         }
     }
     chain_release_next();
     if (held) flush();
+    above = __reduce_add_sync(0xFFFFFFFFu, above);
+    if (lane_id() == 0 && above) atomicAdd(&ws->above_count, above);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0 && atomicAdd(&ws->filter_done, 1u) == gridDim.x - 1) {
+        __threadfence();
+        const uint32_t all_above = ld_relaxed_u32(&ws->above_count), k = ws->k_total;
+        ws->cand.k_rem = all_above < k ? k - all_above : k;     // (not below k: the candidates are not used then)
+        ws->cand.n_gt = all_above;
+    }
 }
 
 template <typename Source, bool kVectorised>
@@ -410,6 +443,25 @@ uint32_t sample_rank(uint64_t n, uint64_t k, uint32_t sample_n, uint32_t capacit
     const double expected_max = (r + 6.0 * __builtin_sqrt(r)) * static_cast<double>(n) / sample_n;
     if (r >= sample_n / 4.0 || expected_max > capacity) return 0;
     return static_cast<uint32_t>(r);
+}
+
+// The same for k too large for that: two ranks, one on either side of tau's expected rank in the sample, so that
+// rank k lies, six standard deviations out, between the two sampled values, and the vector elements between them
+// fit the candidate buffer.  Returns false if there is no such pair.
+bool sample_band(uint64_t n, uint64_t k, uint32_t sample_n, uint32_t capacity, uint32_t* rank_lo, uint32_t* rank_hi) {
+    const double m = static_cast<double>(k) * sample_n / static_cast<double>(n);
+    const double margin = 6.0 * __builtin_sqrt(m + 1.0) + 20.0;
+    const double lo = m + margin, hi = m - margin;
+    if (hi < 1.0 || lo >= sample_n / 2.0) return false;
+    const double between = lo - hi;
+    const double per_sample = static_cast<double>(n) / sample_n;
+    // the elements between the two sampled values, six standard deviations out, and those the two-pass sample
+    // selects add by rounding their values to 21 bits
+    const double expected_max = (between + 6.0 * __builtin_sqrt(between)) * per_sample + static_cast<double>(n) / 2048.0;
+    if (expected_max > capacity) return false;
+    *rank_lo = static_cast<uint32_t>(lo);
+    *rank_hi = static_cast<uint32_t>(hi);
+    return true;
 }
 
 uint32_t candidate_capacity(uint64_t n) {
@@ -532,25 +584,27 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
     const VectorSource vsrc{grad, residual};
 
     // sampled single-pass path?
-    uint32_t sample_n = 0, sample_k = 0, stride = 0, capacity = 0;
+    uint32_t sample_n = 0, sample_k = 0, sample_k_hi = 0, stride = 0, capacity = 0;
     if (n >= kMinSampledN) {
         capacity = candidate_capacity(n);
         stride = (n32 / (kSampleSize / kSampleGroup)) & ~(kSampleGroup - 1u);   // groups start on 32-byte boundaries
         sample_n = kSampleSize;
         sample_k = sample_rank(n, k, sample_n, capacity);
-        if (sample_k == 0) sample_n = 0;
+        if (sample_k == 0 && !sample_band(n, k, sample_n, capacity, &sample_k, &sample_k_hi)) sample_n = 0;
     }
 
-    select_init_kernel<<<1, kInitThreads, 0, stream>>>(ws, n32, k32, sample_n, sample_k, capacity, result);
+    select_init_kernel<<<1, kInitThreads, 0, stream>>>(ws, n32, k32, sample_n, sample_k, capacity, result, sample_k_hi);
     DCT_CUDA_TRY(cudaGetLastError());
     if (sample_n) {
         const StridedSource ssrc{grad, residual, stride};
         DCT_CUDA_TRY((launch_three_passes<StridedSource, false>(grid_for(sample_n), stream, ssrc, &ws->sample, nullptr,
                                                                 result, kSamplePasses)));
-        if (vec)
-            DCT_CUDA_TRY(launch_chained(select_filter_kernel<true>, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
-        else
-            DCT_CUDA_TRY(launch_chained(select_filter_kernel<false>, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
+        if (sample_k_hi)
+            DCT_CUDA_TRY((launch_three_passes<StridedSource, false>(grid_for(sample_n), stream, ssrc, &ws->sample_hi,
+                                                                    nullptr, result, kSamplePasses)));
+        auto* filter = vec ? (sample_k_hi ? select_filter_kernel<true, true> : select_filter_kernel<true, false>)
+                           : (sample_k_hi ? select_filter_kernel<false, true> : select_filter_kernel<false, false>);
+        DCT_CUDA_TRY(launch_chained(filter, grid_for(n), kSelThreads, stream, vsrc, n32, ws, cand_keys));
         // the exact select over the candidates (their count is only known on the device) or, should the sample
         // have misjudged the vector, over the vector itself: the same three launches serve either
         const KeySource ksrc{cand_keys};

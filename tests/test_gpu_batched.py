@@ -13,7 +13,7 @@ from tests._util import bits32
 pytestmark = pytest.mark.gpu
 
 
-def _make_layers(sizes, seed, misalign=()):
+def _make_layers(sizes, seed, misalign=(), dense=False):
     layers = []
     for j, n in enumerate(sizes):
         g = inputs.dp_gaussian(n, seed + 3 * j, G.DEV) * (0.1 + j % 5)
@@ -21,6 +21,8 @@ def _make_layers(sizes, seed, misalign=()):
         if j in misalign:
             g, e = G.offset_copy(g, 1), G.offset_copy(e, 3)
         k = max(1, n // (20 + 7 * (j % 4)))
+        if dense:
+            k = max(1, n // (1 + j % 5))                      # all, a half, a third, ... of the elements pass
         tau, sel = G.select(g, e, k)
         cap = n if j % 3 else max(1, k // 2)                 # every third layer overflows its capacity
         budget = None if j % 2 else torch.tensor([k - sel.n_gt], dtype=torch.int64, device=G.DEV)
@@ -54,6 +56,27 @@ def test_batched_equals_per_layer_oracle(sizes, misalign):
         assert np.array_equal(a["idx_out"][:r.count].cpu().numpy(), w.idx)
         assert np.array_equal(bits32(a["val_out"][:r.count].cpu().numpy()), bits32(w.val))
         assert bool((a["idx_out"][r.count:] == -7).all()) and bool((a["val_out"][r.count:] == -7.0).all())
+        assert np.array_equal(bits32(a["residual"].cpu().numpy()), bits32(e_want))
+
+
+def test_batched_dense_layers_many_tiles_per_cta():
+    """Layers of up to a thousand tiles in which a fifth to all of the elements pass: the ring of the streaming
+    kernel fills up and the tiles a waiting CTA counts ahead of their turn belong to the next layer now and then."""
+    sizes = [(1 << 21) + 5, 1 << 22, 4096 * 700, (1 << 20) + 4096, 4096 * 3, 4096 * 333 + 1, 1 << 21]
+    layers = _make_layers(sizes, 77, dense=True)
+    ws = B.new_workspace(B.dct_dp_compress_batched_workspace_bytes(sizes))
+    want = []
+    for a in layers:
+        e = a["residual"].cpu().numpy().copy()
+        bud = None if a["tie_budget"] is None else int(a["tie_budget"].item())
+        want.append((oracle.dp_compress(a["grad"].cpu().numpy(), e, a["tau"].cpu().numpy()[0], bud, a["capacity"]), e))
+    B.dct_dp_compress_batched(layers, ws)
+    for a, (w, e_want) in zip(layers, want):
+        r = B.read_result(a["result"])
+        assert (r.count, r.needed) == (w.count, w.needed)
+        assert r.status == (B.DCT_ERR_CAPACITY if w.needed > a["capacity"] else B.DCT_OK)
+        assert np.array_equal(a["idx_out"][:r.count].cpu().numpy(), w.idx)
+        assert np.array_equal(bits32(a["val_out"][:r.count].cpu().numpy()), bits32(w.val))
         assert np.array_equal(bits32(a["residual"].cpu().numpy()), bits32(e_want))
 
 

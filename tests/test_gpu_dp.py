@@ -80,6 +80,57 @@ def test_heavy_ties_and_exact_k():
         _compare_compress(g_dev, ee, tau_dev, 0, n)            # budget 0: strictly-greater only
 
 
+@pytest.mark.parametrize("kind", ["gaussian", "dense_and_sparse_stretches", "ties"])
+def test_dense_survivors_many_tiles_per_cta(kind):
+    """Every persistent CTA takes a dozen tiles and most tiles have hundreds to thousands of survivors: the
+    shared-memory ring wraps, fills up (the compute warps wait for their drain warps and count the tiles they
+    hold ahead of their turn) and carries tiles of every density up to all 4096 elements."""
+    n = (1 << 24) + 4096 + 3
+    g_dev = inputs.dp_gaussian(n, 31, G.DEV)
+    if kind == "dense_and_sparse_stretches":                   # stretches of 1..40 tiles, alternately scaled up and down
+        gen = torch.Generator().manual_seed(5)
+        edges = torch.cumsum(torch.randint(1, 41, (2000,), generator=gen) * 4096, 0)
+        scale = torch.ones(n)
+        lo = 0
+        for j, hi in enumerate(edges.tolist()):
+            if lo >= n:
+                break
+            scale[lo:hi] = 8.0 if j % 2 else 0.05
+            lo = hi
+        g_dev = g_dev * scale.to(G.DEV)
+    if kind == "ties":
+        g_dev = inputs.quantize_mantissa(g_dev, 1)
+    e0 = inputs.dp_gaussian(n, 32, G.DEV) * 0.3
+    if kind == "ties":
+        e0 = torch.zeros(n, device=G.DEV)
+    g = g_dev.cpu().numpy()
+    for k in (n // 8, n // 4, n // 2, n):
+        tau_dev, r = G.select(g_dev, e0, k)
+        want = oracle.dp_select(g, e0.cpu().numpy(), k)
+        assert bits32(tau_dev.cpu().numpy())[0] == bits32(want.tau)[0] and (r.n_gt, r.n_eq) == (want.n_gt, want.n_eq)
+        _compare_compress(g_dev, e0.clone(), tau_dev, None, n)
+        if kind == "ties":
+            rr = _compare_compress(g_dev, e0.clone(), tau_dev, k - r.n_gt, n)
+            assert rr.count == k
+    # an output that is too small: the survivors past the capacity go back into the residual, by the million
+    tau_dev, r = G.select(g_dev, e0, n // 4)
+    rr = _compare_compress(g_dev, e0.clone(), tau_dev, None, n // 16)
+    assert rr.status == B.DCT_ERR_CAPACITY and rr.count == n // 16
+
+
+def test_dense_survivors_with_error_feedback_over_iterations():
+    """A threshold of 5 % kept over eight iterations: the residual fills up and about 15 % of the elements pass."""
+    n = (1 << 23) + 100
+    g0 = inputs.dp_gaussian(n, 40, G.DEV)
+    tau_dev, _ = G.select(g0, None, n // 20)
+    e_dev = torch.zeros(n, device=G.DEV)
+    counts = []
+    for t in range(8):
+        g_dev = inputs.dp_gaussian(n, 41 + t, G.DEV)
+        counts.append(_compare_compress(g_dev, e_dev, tau_dev, None, n).count)
+    assert counts[0] == pytest.approx(n / 20, rel=0.05) and counts[-1] > 2.5 * counts[0]
+
+
 def test_degenerate_vectors():
     n = 10_000
     cases = {
@@ -201,7 +252,7 @@ def test_host_buffer_entry_point():
 def test_select_sampled_path_and_its_fallbacks():
     """From 2^25 elements the select reads the vector once, guided by a sample of 2^17 groups of 8
     neighbours.  The sample only steers: when it misjudges the vector (too few or far too many
-    candidates) or cannot be used (dense k), the plain passes must give the same exact answer."""
+    candidates, a band that misses rank k) or cannot be used, the plain passes must give the same exact answer."""
     n = (1 << 25) + 999
     stride = (n // (1 << 17)) & ~7
     sampled = (torch.arange(1 << 17, device=G.DEV)[:, None] * stride + torch.arange(8, device=G.DEV)[None, :]).reshape(-1)
@@ -209,13 +260,23 @@ def test_select_sampled_path_and_its_fallbacks():
     base = inputs.dp_mixture(n, 90, G.DEV)
     cases = {}
     cases["iid, sparse k"] = (base, 3356)
-    cases["dense k: no sample"] = (base, n // 4)
+    cases["dense k: bounds on both sides of tau"] = (base, n // 4)
+    cases["dense k, 5 %"] = (base, n // 20)
+    cases["dense k, 1.5 %"] = (base, n // 64)
+    cases["dense k, ties around tau"] = (inputs.quantize_mantissa(base, 3), n // 10)
+    cases["k of half the vector: no sample"] = (base, n // 2 + 1)
     big_at_sampled = inputs.dp_gaussian(n, 91, G.DEV)
     big_at_sampled[sampled] = 1000.0 + inputs.dp_gaussian(sampled.numel(), 92, G.DEV)
     cases["sample overestimates: too few candidates"] = (big_at_sampled, 10_000)
     zero_at_sampled = inputs.dp_gaussian(n, 93, G.DEV)
     zero_at_sampled[sampled] = 0.0
     cases["sample underestimates: candidates overflow"] = (zero_at_sampled, 5_000)
+    # dense k with a sample that says nothing about the rest: the band misses rank k on one side or the other
+    cases["dense k, sample too large: rank k lies below the band"] = (big_at_sampled, n // 10)
+    cases["dense k, sample too small: rank k lies above the band"] = (zero_at_sampled, n // 10)
+    shifted = inputs.dp_gaussian(n, 94, G.DEV)
+    shifted[sampled] *= 1.02                                   # the band sits a little too high: part of it is used
+    cases["dense k, sample slightly off"] = (shifted, n // 10)
     for name, (g, k) in cases.items():
         tau_dev, r = G.select(g, None, k)
         want = oracle.dp_select(g.cpu().numpy(), None, k)
