@@ -235,6 +235,49 @@ class HotPath:
             del x, cols, vals
         return out
 
+    def time_dp_dense(self, stream, iters=12):
+        """DCT-DP at the paper's 95 % sparsity level: N = 2^28 gradients, k = 5 % of N; the select, then `iters`
+        iterations with that threshold and the error carried over (the survivors settle near 15 % of N), fresh
+        values every iteration from two shifted buffers."""
+        B = self.B
+        n, dev = 1 << 28, self.dev
+        k = n // 20
+        slack = 1 << 10
+        g_raw = [inputs.dp_mixture(n + slack, 700 + j, dev) for j in range(2)]
+        fresh = lambda i: g_raw[i % 2][4 * (i // 2): 4 * (i // 2) + n]
+        e = torch.zeros(n, device=dev)
+        tau = torch.zeros(1, device=dev)
+        cap = n // 2
+        idx = torch.empty(cap, dtype=torch.int32, device=dev)
+        val = torch.empty(cap, device=dev)
+        res = torch.zeros(iters, 5, dtype=torch.int64, device=dev)
+        res_s = B.new_result(dev)
+        ws_s = B.new_workspace(B.dct_threshold_select_workspace_bytes(n), dev)
+        ws_c = B.new_workspace(B.dct_dp_compress_workspace_bytes(n), dev)
+        out = {"n": n, "k": k}
+        for phase in range(2):
+            a = _record(stream)
+            for i in range(4):
+                B.dct_threshold_select(fresh(i), None, n, k, tau, res_s, ws_s, stream)
+            b = _record(stream)
+            b.synchronize()
+        ms = a.elapsed_time(b) / 4
+        out["select"] = {"ms": ms, "GBps_at_4B_per_elem": 4 * n / (ms * 1e-3) / 1e9}
+        B.dct_threshold_select(fresh(0), None, n, k, tau, res_s, ws_s, stream)
+        for phase in range(2):
+            e.zero_()
+            a = _record(stream)
+            for i in range(iters):
+                B.dct_dp_compress(fresh(i), e, n, tau, None, idx, val, cap, res[i], ws_c, stream)
+            b = _record(stream)
+            b.synchronize()
+        ms = a.elapsed_time(b) / iters
+        counts = [int(c) for c in res[:, 1].cpu().tolist()]
+        assert all(int(st) == B.DCT_OK for st in res[:, 0].cpu().tolist())
+        nbytes = sum(12 * n + 8 * c for c in counts) / iters
+        out["compress"] = {"ms": ms, "GBps": nbytes / (ms * 1e-3) / 1e9, "survivors_first_last": [counts[0], counts[-1]]}
+        return out
+
     def time_c3(self, stream, iters=20):
         """DCT-DP at DLRM-like MLP scale (64 Mi gradients as concatenated dense-layer blocks, Student-t values,
         density 0.1 %): the select, the fixed-threshold iterations (mean of `iters`, error starting at zero), and
@@ -722,6 +765,7 @@ def main():
     if args.workload == DEFAULT_WORKLOAD:
         parts["c3"] = hp.time_c3(stream)
         parts["wide_rows"] = hp.time_wide_rows(stream)
+        parts["dp_dense"] = hp.time_dp_dense(stream)
     fwd_bytes = b0["mp_fwd"] / cfg["mp_iters"]
     roofline_mp = {
         "kernel": "mp_topk_fwd_bf16_warp_kernel<16,10>", "bound": "hbm", "achieved": parts["mp_fwd"]["GBps"], "peak": peak,

@@ -85,7 +85,9 @@ DCT_API const char* dct_last_cuda_error(void);
 
 /* Bytes of device workspace the calls below need for a vector of n elements.
  * The workspace must be 256-byte aligned; its contents need not be preserved
- * between calls and two calls that may overlap on the GPU need separate ones. */
+ * between calls and two calls that may overlap on the GPU need separate ones.
+ * (Select: about 100 KB, from 2^25 elements on plus 4 B per element up to 32 MiB;
+ * compress: 256 B plus 8 B per 4096 elements.) */
 DCT_API size_t dct_threshold_select_workspace_bytes(uint64_t n);
 DCT_API size_t dct_dp_compress_workspace_bytes(uint64_t n);
 

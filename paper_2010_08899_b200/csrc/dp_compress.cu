@@ -427,7 +427,7 @@ dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ resi
 // fast path: persistent CTAs; load warp + compute warps + look-back warp + drain warps
 // ------------------------------------------------------------------------------------------
 constexpr int kSlots = 16;                               // tiles a CTA may be ahead of its drain warp
-constexpr uint32_t kRingEntries = 6080;                  // survivors waiting in shared memory: any one tile fits
+constexpr uint32_t kRingEntries = 6016;                  // survivors waiting in shared memory: any one tile fits
 constexpr uint32_t kEqBit = 0x80000000u;                 // ring entry: "equal to tau"
 constexpr uint32_t kAheadGrace = 8;                      // polls of a waiting compute warp before it counts tiles ahead
 constexpr int kDrainWarps = 2;                           // warps that share the write-out of a tile's entries
@@ -456,6 +456,13 @@ struct __align__(128) StreamSmem {
     uint32_t slot_head[kSlots];          // running count of ring entries up to and including the tile's
     uint32_t prefix[kSlots][2];
     uint32_t aborted[kSlots];
+    // batched calls: what the drain warps need to know about the slot's vector, from the look-back warp, which has
+    // read the vector's description anyway
+    int32_t* slot_idx_out[kSlots];
+    float* slot_val_out[kSlots];
+    float* slot_residual[kSlots];
+    uint64_t slot_budget[kSlots];
+    uint64_t slot_capacity[kSlots];
     uint32_t ahead[4];                   // counts of a tile taken ahead of its turn: eq | gt << 13 | warps that added << 26
     volatile uint32_t ring_tail[kDrainWarps];   // drain warp -> compute: running count of ring entries it is done with
     volatile uint32_t drained[kDrainWarps];     // drain warp -> compute: tiles it is done with (their slots may be reused)
@@ -533,22 +540,20 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
     StreamSmem& sm = *reinterpret_cast<StreamSmem*>(smem_raw);
     const uint32_t tid = threadIdx.x, lane = lane_id(), warp = tid >> 5;
 
-    if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm.full[s], 1);
-            mbar_init(&sm.empty[s], 1);
+    if (tid < static_cast<uint32_t>(kSlots)) {
+        mbar_init(&sm.agg_ready[tid], 1);
+        mbar_init(&sm.entries_ready[tid], kWarps);
+        mbar_init(&sm.prefix_ready[tid], 1);
+        if (tid < static_cast<uint32_t>(kStages)) {
+            mbar_init(&sm.full[tid], 1);
+            mbar_init(&sm.empty[tid], 1);
         }
-        for (int r = 0; r < kSlots; ++r) {
-            mbar_init(&sm.agg_ready[r], 1);
-            mbar_init(&sm.entries_ready[r], kWarps);
-            mbar_init(&sm.prefix_ready[r], 1);
+        if (tid < static_cast<uint32_t>(kDrainWarps)) {
+            sm.ring_tail[tid] = 0;
+            sm.drained[tid] = 0;
         }
-        for (int v = 0; v < kDrainWarps; ++v) {
-            sm.ring_tail[v] = 0;
-            sm.drained[v] = 0;
-        }
-        for (int v = 0; v < 4; ++v) sm.ahead[v] = 0;
-        sm.stop = 0;
+        if (tid < 4) sm.ahead[tid] = 0;
+        if (tid == 0) sm.stop = 0;
         mbar_init_fence();
         fence_proxy_async_all();
     }
@@ -641,6 +646,13 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
                 sm.prefix[r][0] = excl_gt;
                 sm.prefix[r][1] = excl_eq;
                 sm.aborted[r] = chain_ok ? 0u : 1u;
+                if (kBatched) {
+                    sm.slot_idx_out[r] = P.idx_out;
+                    sm.slot_val_out[r] = P.val_out;
+                    sm.slot_residual[r] = P.residual;
+                    sm.slot_budget[r] = P.budget;
+                    sm.slot_capacity[r] = P.capacity;
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.prefix_ready[r]);
@@ -651,7 +663,6 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
         // ================= drain warps: ring entries of each tile -> (idx, val), 32 entries per warp in turn =====
         const uint32_t dw = warp - kDrainWarp0;
         TileParams P;
-        uint32_t cur_layer = 0xFFFFFFFFu;
         if (!kBatched) P = load_params(single, tile_state_base);
         for (uint32_t it = 0;; ++it) {
             const int r = it % kSlots;
@@ -662,9 +673,12 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
             }
             const uint32_t tile = sm.slot_tile[r];
             if (tile == kInvalidTile) return;
-            if (kBatched && sm.slot_layer[r] != cur_layer) {
-                cur_layer = sm.slot_layer[r];
-                P = load_params(batch.layers[cur_layer], tile_state_base);
+            if (kBatched) {
+                P.idx_out = sm.slot_idx_out[r];
+                P.val_out = sm.slot_val_out[r];
+                P.residual = sm.slot_residual[r];
+                P.budget = sm.slot_budget[r];
+                P.capacity = sm.slot_capacity[r];
             }
             if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&sm.entries_ready[r], parity, kMbarLimit, &sm.stop))) {
                 sm.stop = 1;
@@ -703,6 +717,7 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
     uint32_t ring_head = 0;                   // running count of ring entries written by this CTA
     uint32_t ring_pos = 0;                    // the same modulo the size of the ring
     uint32_t ahead_upto = 0;                  // last iteration whose tile this warp has counted ahead of its turn
+    uint32_t drained_seen = 0, tail_seen = 0; // what this warp last read of the drain warps' counters (they only grow)
     for (;; ++it) {
         const int s = it % kStages;
         const int r = it % kSlots;
@@ -768,9 +783,16 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
         // holds the tile's counts, it does not need the ring entries.
         bool slot_ok = true;
         if (warp == 0) {
-            if (lane < kDrainWarps)               // one lane per drain warp
-                slot_ok = counter_wait_bounded(&sm.drained[lane], it + 1u - kSlots, kMbarLimit, &sm.stop);
-            slot_ok = __all_sync(0xFFFFFFFFu, slot_ok);
+            const uint32_t need_drained = it + 1u - kSlots;
+            if (static_cast<int32_t>(drained_seen - need_drained) < 0) {     // (else: seen to be free earlier)
+                int32_t lead = 0x7FFFFFFF;
+                if (lane < kDrainWarps) {         // one lane per drain warp
+                    slot_ok = counter_wait_bounded(&sm.drained[lane], need_drained, kMbarLimit, &sm.stop);
+                    lead = static_cast<int32_t>(sm.drained[lane] - need_drained);
+                }
+                slot_ok = __all_sync(0xFFFFFFFFu, slot_ok);
+                drained_seen = need_drained + static_cast<uint32_t>(__reduce_min_sync(0xFFFFFFFFu, lead));
+            }
             if (lane == 0 && slot_ok) {
                 sm.slot_tile[r] = tile;
                 sm.slot_layer[r] = cur_layer;
@@ -782,9 +804,15 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
         }
         // the tile's share of the ring must have been drained as well
         const uint32_t need_tail = ring_head + cnt - kRingEntries;
-        bool room = true;
-        if (lane < kDrainWarps) room = static_cast<int32_t>(sm.ring_tail[lane] - need_tail) >= 0;
-        room = __all_sync(0xFFFFFFFFu, room);
+        auto least_tail = [&]() -> uint32_t {     // the least of the drain warps' counts (one lane per drain warp)
+            const int32_t lead = lane < kDrainWarps ? static_cast<int32_t>(sm.ring_tail[lane] - need_tail) : 0x7FFFFFFF;
+            return need_tail + static_cast<uint32_t>(__reduce_min_sync(0xFFFFFFFFu, lead));
+        };
+        bool room = static_cast<int32_t>(tail_seen - need_tail) >= 0;     // (seen to be free earlier)
+        if (!room) {
+            tail_seen = least_tail();
+            room = static_cast<int32_t>(tail_seen - need_tail) >= 0;
+        }
         if (!room) {
             // This warp has to wait for the drain warps, they for the look-back, and the look-back for the counts of
             // every earlier tile.  The CTA has taken tickets for the tiles in its other stages already; if their counts
@@ -794,9 +822,8 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
             // (Only after a short while: most waits end by themselves before that.)
             uint32_t a = 1;
             for (uint32_t polls = 1;; ++polls) {
-                room = true;
-                if (lane < kDrainWarps) room = static_cast<int32_t>(sm.ring_tail[lane] - need_tail) >= 0;
-                room = __all_sync(0xFFFFFFFFu, room);
+                tail_seen = least_tail();
+                room = static_cast<int32_t>(tail_seen - need_tail) >= 0;
                 if (room || polls >= kMbarLimit || ((polls & 63u) == 63u && sm.stop)) break;
                 const uint32_t j = it + a;
                 if (polls < kAheadGrace || a > static_cast<uint32_t>(kStages)) {

@@ -41,6 +41,7 @@ constexpr uint32_t kSampleSize = 1u << 20;                   // elements in the 
 constexpr uint32_t kSampleGroup = 8;                         // consecutive elements taken at each sample position
 constexpr uint32_t kMaxCandidates = 1u << 23;                // candidate buffer: at most 32 MiB
 constexpr uint32_t kMinSampledN = 1u << 25;                  // below this the three plain passes are cheaper
+constexpr uint64_t kBandFromK = 1u << 21;                    // from this k on the filter keeps a band around tau, if it can
 
 __host__ __device__ constexpr int pass_shift(int p) { return p == 0 ? 20 : (p == 1 ? 10 : 0); }
 __host__ __device__ constexpr int pass_bits(int p) { return p == 0 ? 11 : 10; }
@@ -589,8 +590,12 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
         capacity = candidate_capacity(n);
         stride = (n32 / (kSampleSize / kSampleGroup)) & ~(kSampleGroup - 1u);   // groups start on 32-byte boundaries
         sample_n = kSampleSize;
-        sample_k = sample_rank(n, k, sample_n, capacity);
-        if (sample_k == 0 && !sample_band(n, k, sample_n, capacity, &sample_k, &sample_k_hi)) sample_n = 0;
+        // millions of elements above tau: the band around tau is the shorter candidate list, where there is one
+        const bool band = k >= kBandFromK && sample_band(n, k, sample_n, capacity, &sample_k, &sample_k_hi);
+        if (!band) {
+            sample_k = sample_rank(n, k, sample_n, capacity);
+            if (sample_k == 0 && !sample_band(n, k, sample_n, capacity, &sample_k, &sample_k_hi)) sample_n = 0;
+        }
     }
 
     select_init_kernel<<<1, kInitThreads, 0, stream>>>(ws, n32, k32, sample_n, sample_k, capacity, result, sample_k_hi);
