@@ -264,6 +264,39 @@ __device__ __forceinline__ void for_each_flagged(uint32_t gt_mask, uint32_t eq_m
     }
 }
 
+// The same for a span without elements equal to tau (the usual case: one packed scan, no second kind to carry):
+//   visit(b, j * 128 + c, local_gt)      with the element at warp_base + lane * 4 + j * 128 + c
+template <typename Visit>
+__device__ __forceinline__ void for_each_above(uint32_t gt_mask, uint32_t before, Visit&& visit) {
+    const uint32_t lane = lane_id();
+    uint32_t pg = 0;
+#pragma unroll
+    for (int j = 0; j < kVecs; ++j) pg |= static_cast<uint32_t>(__popc((gt_mask >> (4 * j)) & 0xFu)) << (8 * j);
+    uint32_t ig = pg;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t tg = __shfl_up_sync(0xFFFFFFFFu, ig, o);
+        if (lane >= static_cast<uint32_t>(o)) ig += tg;
+    }
+    const uint32_t tot_g = __shfl_sync(0xFFFFFFFFu, ig, 31);
+    const uint32_t ex_g = ig - pg;
+    if (gt_mask == 0) return;
+    uint32_t base_g = before;
+#pragma unroll
+    for (int j = 0; j < kVecs; ++j) {
+        uint32_t g0 = base_g + ((ex_g >> (8 * j)) & 0xFFu);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const int b = 4 * j + c;
+            if ((gt_mask >> b) & 1u) {
+                visit(b, static_cast<uint32_t>(j * 128 + c), g0);
+                ++g0;
+            }
+        }
+        base_g += (tot_g >> (8 * j)) & 0xFFu;
+    }
+}
+
 // One flagged element whose global counts of preceding flagged elements are known: it is either
 // written to the output or, if it is not sent after all, put back into the residual.
 __device__ __forceinline__ void place_survivor(uint32_t i, float w, bool is_eq, uint64_t gt_before,
@@ -872,7 +905,21 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
         }
         room = room && slot_ok;
         if (!room) sm.stop = 1;                   // seen by everybody at the next vote
-        if (warp_tot != 0 && room) {
+        if (warp_tot != 0 && room && cta_eq == 0) {
+            // no element of the tile equals tau (the usual case): one kind of entry, nothing to count before it
+            const uint32_t first_off = warp * kWarpElems + lane * 4u;
+            if (ring_pos + cnt <= kRingEntries) {
+                uint2* ring = sm.ring + ring_pos;
+                for_each_above(gt_mask, before_warp >> 16, [&](int b, uint32_t off, uint32_t local_gt) {
+                    ring[local_gt] = make_uint2(first_off + off, __float_as_uint(w[b]));
+                });
+            } else {
+                for_each_above(gt_mask, before_warp >> 16, [&](int b, uint32_t off, uint32_t local_gt) {
+                    const uint32_t at = ring_pos + local_gt;
+                    sm.ring[at < kRingEntries ? at : at - kRingEntries] = make_uint2(first_off + off, __float_as_uint(w[b]));
+                });
+            }
+        } else if (warp_tot != 0 && room) {
             const uint32_t in_tile = warp * kWarpElems;
             for_each_flagged(gt_mask, eq_mask, in_tile, before_warp,
                              [&](int b, uint32_t off, uint32_t local_gt, uint32_t local_eq, bool is_eq) {
