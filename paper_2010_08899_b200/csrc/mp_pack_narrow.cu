@@ -1,5 +1,11 @@
-// dct_mp_topk_pack_fwd, bf16 rows of 256 or 512 columns: Algorithm 2 (DCT-MP) with the row held in
-// registers and several samples per warp.
+// dct_mp_topk_pack_fwd, rows of up to 512 bf16 or 256 fp32 columns: Algorithm 2 (DCT-MP) with the row held in
+// registers and several samples per warp.  Two schemes:
+//   * the count over the row in registers (narrow_slow_path, narrow_bisect_f32): tau_i bit by bit, every round a
+//     count of the row's keys against a trial value by the G lanes that hold the row, then the ordered emit.  It
+//     serves every k on bf16 rows of up to 128 columns and fp32 rows of up to 256, the denser k (more than an eighth
+//     of the row) on bf16 rows of up to 256 columns, and the rows the second scheme gives up on;
+//   * bound and candidates (mp_topk_fwd_bf16_narrow_kernel, bf16 rows of 129 to 512 columns, k up to an eighth of
+//     the row), described next.
 //
 // For narrow rows the fixed cost per row of the shared-memory kernel (mp_pack.cu: bulk copy, barrier, bit
 // table, bisection, linked walk) outweighs the work on the row itself, and so do the warp scans and votes
@@ -31,6 +37,7 @@ constexpr uint32_t kNarrowScratchWords = 320;    // per warp (G >= 8); a group's
 // G = 4 (8 rows per warp): 8 shares of 64 + G words for the histogram
 template <int G> __host__ __device__ constexpr uint32_t narrow_scratch_words() { return G >= 8 ? kNarrowScratchWords : (32u / G) * (64u + G); }
 
+#pragma nv_diag_suppress 177   // (members that one instantiation or another does not use)
 template <int G, int PLN = static_cast<int>(kNarrowPerLaneFew)> struct Group {
     static constexpr uint32_t kRows = 32u / G;                       // rows a warp works on at once
     static constexpr uint32_t kList = PLN * G;                       // candidates of a row that fit
@@ -351,21 +358,71 @@ dct_status_t launch_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_
     return DCT_OK;
 }
 
+// Denser k (more than an eighth of the row: no leaf bound applies): every row takes the bit-by-bit count over the
+// row in registers, 15 rounds for a bf16 key, and the ordered emit from the row.  The warp kernels and the general
+// kernel pay their fixed cost per row for these short rows; here a warp serves 32 / G rows at once.
+template <int E8, int G>
+__global__ void __launch_bounds__(kNarrowWarps * 32)
+mp_topk_fwd_bf16_narrow_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                     int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
+                                     int32_t* __restrict__ rows_out, uint16_t* __restrict__ tau_out,
+                                     dct_result_t* __restrict__ result) {
+    constexpr uint32_t kRows = 32u / G;
+    const uint32_t warp = threadIdx.x >> 5, group = lane_id() / G;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->reserved = 0;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+    }
+    const uint64_t bundles = (static_cast<uint64_t>(rows) + kRows - 1) / kRows;
+    const uint64_t bundle_step = static_cast<uint64_t>(gridDim.x) * (blockDim.x >> 5);
+    for (uint64_t bundle = blockIdx.x + static_cast<uint64_t>(gridDim.x) * warp; bundle < bundles; bundle += bundle_step) {
+        const uint64_t r = bundle * kRows + group;
+        const bool valid = r < rows;
+        const uint64_t row64 = valid ? r : rows - 1;     // a group past the last row runs along on the last row
+        narrow_slow_path<E8, G>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
+                                cols_out, vals_out, rows_out, tau_out);
+    }
+}
+
+template <int E8, int G>
+dct_status_t launch_narrow_dense(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
+                                 void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
+                                 cudaStream_t stream) {
+    auto kernel = mp_topk_fwd_bf16_narrow_dense_kernel<E8, G>;
+    int per_sm = 0;
+    DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kNarrowWarps * 32, 0));
+    if (per_sm < 1) return DCT_ERR_UNSUPPORTED;
+    const int sms = sm_count();
+    if (sms <= 0) return DCT_ERR_CUDA;
+    const uint64_t bundles = (static_cast<uint64_t>(rows) + (32u / G) - 1) / (32u / G);
+    const uint64_t ctas_needed = (bundles + kNarrowWarps - 1) / kNarrowWarps;
+    const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
+    const uint32_t grid = static_cast<uint32_t>(ctas_needed < max_grid ? ctas_needed : max_grid);
+    kernel<<<grid, kNarrowWarps * 32, 0, stream>>>(static_cast<const uint16_t*>(x_act), rows, d, ld, k, cols_out,
+                                                   static_cast<uint16_t*>(vals_out), rows_out,
+                                                   static_cast<uint16_t*>(tau_out), result);
+    DCT_CUDA_TRY(cudaGetLastError());
+    return DCT_OK;
+}
 
 // ------------------------------------------------------------------------------------------
-// fp32 rows of 256 columns: the same scheme on two levels
+// fp32 rows of up to 256 columns: the count over the row in registers, on two levels
 // ------------------------------------------------------------------------------------------
-// The paper's recommendation model runs in fp32.  A key has 31 bits; as in the other fp32 kernels the bound, the
-// candidate bits and the windowed histogram work on its upper 15 bits (the bucket: the bf16 truncation of |x|), which
-// gives the bucket of tau_i and how many of its members belong to the top k; the members (usually one) are then
-// ranked by their lower 16 bits.  A lane holds 32 consecutive columns (eight 16-byte loads), a group of G = 8 lanes
-// a row (four rows per warp); a candidate is two list words (value, column).
-constexpr uint32_t kNarrowScratchWordsF32 = 2 * kNarrowScratchWords;
-
-// Slow path (fp32): tau_i bit by bit over the 31 key bits by counting over the row in registers, then the ordered
-// emit straight from the row.  Called by the whole warp; groups without a row run along and store nothing.
+// The paper's recommendation model runs in fp32.  A key has 31 bits; as in the other fp32 kernels the first level
+// works on its upper 15 bits (the bucket: the bf16 truncation of |x|), which gives the bucket of tau_i and how many
+// of its members belong to the top k; the members (usually one) are then ranked by their lower 16 bits.  A lane
+// holds 32 consecutive columns (eight 16-byte loads), a group of G = 2, 4 or 8 lanes a row.
+// tau_i bit by bit by counting over the row in registers, then the ordered emit straight from the
+// row.  The upper 15 key bits (the bucket) take 15 rounds on the packed upper halves, eight columns per exact flag
+// step as in the bf16 kernels; the lower 16 bits come from the bucket's members: the smallest of them if all are
+// needed (the usual case: one member), the largest if one is, else 16 more rounds over the row's keys.  Called by the
+// whole warp; groups without a row run along and store nothing.
 template <int G>
-__device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ xr, uint32_t d, bool valid, uint32_t k,
+__device__ __forceinline__ void narrow_bisect_f32(const uint32_t* __restrict__ xr, uint32_t d, bool valid, uint32_t k,
                                                   size_t out_base, uint32_t row, int16_t* __restrict__ cols_out,
                                                   uint32_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
                                                   uint32_t* __restrict__ tau_out) {
@@ -373,6 +430,7 @@ __device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ x
     constexpr uint32_t E = 32u;
     const uint32_t gl = lane_id() & (G - 1);
     uint32_t key[E];
+    uint4 up[4];                                   // upper halves of the lane's 32 columns, eight to a register quad
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
         const uint4 v = gl * E < d ? __ldg(reinterpret_cast<const uint4*>(xr + gl * E) + c) : make_uint4(0, 0, 0, 0);
@@ -380,15 +438,57 @@ __device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ x
         key[4 * c + 1] = v.y & 0x7FFFFFFFu;
         key[4 * c + 2] = v.z & 0x7FFFFFFFu;
         key[4 * c + 3] = v.w & 0x7FFFFFFFu;
+        if (c & 1) {
+            up[c / 2].z = upper_halves(v.x, v.y);
+            up[c / 2].w = upper_halves(v.z, v.w);
+        } else {
+            up[c / 2].x = upper_halves(v.x, v.y);
+            up[c / 2].y = upper_halves(v.z, v.w);
+        }
     }
-    uint32_t tau_key = 0;
+    uint32_t bucket = 0;
 #pragma unroll 1
-    for (int bit = 30; bit >= 0; --bit) {
-        const uint32_t trial = tau_key | (1u << bit);
+    for (int bit = 14; bit >= 0; --bit) {
+        const uint32_t trial = bucket | (1u << bit);
         uint32_t cnt = 0;
 #pragma unroll
-        for (int j = 0; j < static_cast<int>(E); ++j) cnt += key[j] >= trial ? 1u : 0u;
-        if (Gr::sum(cnt) >= k) tau_key = trial;
+        for (int c = 0; c < 4; ++c) cnt += __popc(mask8_ge_exact(up[c], trial));
+        if (Gr::sum(cnt) >= k) bucket = trial;
+    }
+    uint32_t above = 0, members = 0;               // columns of the lane above the bucket / inside it
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint32_t gt = mask8_ge_exact(up[c], bucket + 1u);
+        above |= gt << (8 * c);
+        members |= (mask8_ge_exact(up[c], bucket) & ~gt) << (8 * c);
+    }
+    const uint32_t need = k - Gr::sum(__popc(above));      // members of the bucket that belong to the top k: >= 1
+    const uint32_t in_bucket = Gr::sum(__popc(members));
+    uint32_t tau_key = bucket << 16;
+    if (__all_sync(0xFFFFFFFFu, need == in_bucket || need == 1u)) {
+        uint32_t lo = 0xFFFFFFFFu, hi = 0;
+        for (uint32_t m = members; m; m &= m - 1) {
+            // (a lane past the end of the row holds zeros: nothing of its own to read)
+            const uint32_t v = gl * E < d ? xr[gl * E + __ffs(m) - 1] & 0x7FFFFFFFu : 0u;
+            lo = v < lo ? v : lo;
+            hi = v > hi ? v : hi;
+        }
+#pragma unroll
+        for (int o = G / 2; o > 0; o >>= 1) {
+            const uint32_t a = __shfl_xor_sync(0xFFFFFFFFu, lo, o, G), b = __shfl_xor_sync(0xFFFFFFFFu, hi, o, G);
+            lo = a < lo ? a : lo;
+            hi = b > hi ? b : hi;
+        }
+        tau_key = need == in_bucket ? lo : hi;
+    } else {
+#pragma unroll 1
+        for (int bit = 15; bit >= 0; --bit) {
+            const uint32_t trial = tau_key | (1u << bit);
+            uint32_t cnt = 0;
+#pragma unroll
+            for (int j = 0; j < static_cast<int>(E); ++j) cnt += key[j] >= trial ? 1u : 0u;
+            if (Gr::sum(cnt) >= k) tau_key = trial;
+        }
     }
     uint32_t gt_mask = 0, eq_mask = 0;
 #pragma unroll
@@ -418,26 +518,15 @@ __device__ __noinline__ void narrow_slow_path_f32(const uint32_t* __restrict__ x
     if (valid && gl == 0 && tau_out) tau_out[row] = tau_key;
 }
 
-template <int G, int PLN>
+// Denser k, fp32: the two-level bit-by-bit count over the row in registers (narrow_bisect_f32), for every row.
+template <int G>
 __global__ void __launch_bounds__(kNarrowWarps * 32)
-mp_topk_fwd_f32_narrow_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
-                              int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
-                              int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
-                              dct_result_t* __restrict__ result) {
-    using Gr = Group<G, PLN>;
-    constexpr uint32_t kNarrowPerLane = PLN;       // candidates a lane holds in registers
-    constexpr int kPieces = 4;                     // 32-byte pieces (8 columns) of a lane
-    constexpr uint32_t E = 32u;                    // columns per lane; the lane's candidate bits are one word
-    constexpr uint32_t kRows = Gr::kRows;
-    constexpr uint32_t kGuessMargin = 32;          // buckets below the previous row's
-    constexpr uint32_t kShareF32 = kNarrowScratchWordsF32 / kRows;     // values, then columns: 2 x kList words
-    static_assert(kShareF32 >= 2 * Gr::kList && kShareF32 >= 64u + G, "scratch share too small");
-    __shared__ uint32_t s_scratch[kNarrowWarps][kNarrowScratchWordsF32];
-    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
-    const uint32_t gl = lane & (G - 1), group = lane / G, group_base = group * G;
-    uint32_t* share = s_scratch[warp] + group * kShareF32;    // this group's list / histogram / stage, in turn
-    uint32_t* share_c = share + Gr::kList;                    // the columns of the list / stage entries
-
+mp_topk_fwd_f32_narrow_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                    int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
+                                    int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
+                                    dct_result_t* __restrict__ result) {
+    constexpr uint32_t kRows = 32u / G;
+    const uint32_t warp = threadIdx.x >> 5, group = lane_id() / G;
     if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
         result->status = DCT_OK;
         result->reserved = 0;
@@ -446,242 +535,28 @@ mp_topk_fwd_f32_narrow_kernel(const uint32_t* __restrict__ x, uint32_t rows, uin
         result->n_gt = 0;
         result->n_eq = 0;
     }
-    const uint32_t warps = blockDim.x >> 5;
     const uint64_t bundles = (static_cast<uint64_t>(rows) + kRows - 1) / kRows;
-    const uint64_t first_bundle = blockIdx.x + static_cast<uint64_t>(gridDim.x) * warp;
-    const uint64_t bundle_step = static_cast<uint64_t>(gridDim.x) * warps;
-    auto row_of = [&](uint64_t bundle) -> uint64_t {          // a group past the last row reads the last row instead
+    const uint64_t bundle_step = static_cast<uint64_t>(gridDim.x) * (blockDim.x >> 5);
+    for (uint64_t bundle = blockIdx.x + static_cast<uint64_t>(gridDim.x) * warp; bundle < bundles; bundle += bundle_step) {
         const uint64_t r = bundle * kRows + group;
-        return r < rows ? r : rows - 1;
-    };
-    const bool lane_in = gl * E < d;                // (lanes past the end of the row hold zeros)
-    auto load_row = [&](uint64_t r, uint4 (&v)[2 * kPieces]) {
-        const uint4* src = reinterpret_cast<const uint4*>(x + r * ld + gl * E);
-#pragma unroll
-        for (int c = 0; c < 2 * kPieces; ++c) v[c] = lane_in ? __ldg(src + c) : make_uint4(0, 0, 0, 0);
-    };
-    uint4 cur[2 * kPieces];
-
-    uint32_t guess_low = 0;                         // bucket bound guessed from the group's previous row (0: none)
-    const bool have_bound = k <= d / 8u;            // at least k leaves in a row
-    for (uint64_t bundle = first_bundle; bundle < bundles; bundle += bundle_step) {
-        const bool valid = bundle * kRows + group < rows;
-        const uint64_t row64 = row_of(bundle);
-        const uint32_t row = static_cast<uint32_t>(row64);
-        load_row(row64, cur);       // (no prefetch of the next rows: the registers buy more warps than it gains)
-        const uint32_t* xr = x + row64 * ld;
-        const size_t out_base = static_cast<size_t>(row) * k;
-
-        // ---- B (with A): candidate bits of the lane (bucket >= bound), one word in column order ------
-        uint32_t mask = 0, incl = 0, n_cand = 0;
-        auto build_mask = [&](uint32_t bound) {
-            const uint32_t low2 = bound | (bound << 16);
-            mask = 0;
-#pragma unroll
-            for (int c = 0; c < kPieces; ++c)
-                mask |= piece_flags(cur[2 * c], cur[2 * c + 1], low2, 0xF8FCFEFFu, 0x80C0E0F0u) << (8 * c);
-            incl = Gr::inclusive_sum(__popc(mask), gl);
-            n_cand = Gr::last(incl);
-        };
-        uint32_t low = guess_low;
-        bool settled = false;
-        if (have_bound && __all_sync(0xFFFFFFFFu, guess_low != 0)) {
-            build_mask(low);
-            settled = __all_sync(0xFFFFFFFFu, n_cand >= k && n_cand <= Gr::kList);
-        }
-        if (!settled) {
-            // exact bound: the k-th largest of the row's leaf maxima (buckets), bit by bit
-            uint32_t leaf[kPieces];
-#pragma unroll
-            for (int c = 0; c < kPieces; ++c) {
-                const uint4 a = cur[2 * c], b = cur[2 * c + 1];
-                const uint32_t u0 = upper_halves(a.x, a.y) & kAbsMask2, u1 = upper_halves(a.z, a.w) & kAbsMask2;
-                const uint32_t u2 = upper_halves(b.x, b.y) & kAbsMask2, u3 = upper_halves(b.z, b.w) & kAbsMask2;
-                const uint32_t m = as_u32(__hmax2(__hmax2(as_bf162(u0), as_bf162(u1)), __hmax2(as_bf162(u2), as_bf162(u3))));
-                leaf[c] = max(m & 0xFFFFu, m >> 16);
-            }
-            low = 0;
-            if (have_bound) {
-#pragma unroll 1
-                for (int bit = 14; bit >= 0; --bit) {
-                    const uint32_t trial = low | (1u << bit);
-                    uint32_t cnt = 0;
-#pragma unroll
-                    for (int c = 0; c < kPieces; ++c) cnt += leaf[c] >= trial ? 1u : 0u;
-                    if (Gr::sum(cnt) >= k) low = trial;
-                }
-            }
-            build_mask(low);
-        }
-        if (!have_bound || __any_sync(0xFFFFFFFFu, n_cand > Gr::kList || low == 0)) {
-            narrow_slow_path_f32<G>(xr, d, valid, k, out_base, row, cols_out, vals_out, rows_out, tau_out);
-            continue;
-        }
-
-        // candidates into the group's list, column order: value and column
-        __syncwarp();                                   // whatever used the scratch before is done
-        {
-            uint32_t at = incl - __popc(mask);
-            uint32_t m = mask;
-            while (m) {
-                const uint32_t col = gl * E + (__ffs(m) - 1);
-                m &= m - 1;
-                share[at] = __ldg(xr + col);
-                share_c[at] = col;
-                ++at;
-            }
-        }
-        __syncwarp();
-        uint32_t ent[kNarrowPerLane], ent_c[kNarrowPerLane];   // value 0: unused slot (its bucket 0 lies below the bound)
-        const uint32_t per_lane = (n_cand + G - 1) / G;
-#pragma unroll
-        for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
-            const uint32_t r = gl * per_lane + i;
-            const bool used = static_cast<uint32_t>(i) < per_lane && r < n_cand;
-            ent[i] = used ? share[r] : 0u;
-            ent_c[i] = used ? share_c[r] : 0u;
-        }
-        __syncwarp();                                   // the list is in registers: its words become the histogram
-
-        // ---- C: the bucket of tau_i among the candidates' buckets ------------------------------------------
-        uint32_t bucket = 0, take = 0;                  // `take` members of the bucket belong to the top k
-        bool found = false;
-        {
-            // 64 bins just above the bound, G private overflow bins behind them
-            const uint32_t drop = n_cand - k;
-            for (uint32_t b = gl; b < 64u + G; b += G) share[b] = 0;
-            __syncwarp();
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
-                const uint32_t rel = ((ent[i] >> 16) & 0x7FFFu) - low;
-                atomicAdd(&share[rel < 64u ? rel : 64u + gl], 1u);
-            }
-            __syncwarp();
-            uint32_t h[Gr::kBins], own = 0;             // the lane looks after bins gl kBins .. gl kBins + kBins - 1
-#pragma unroll
-            for (int j = 0; j < static_cast<int>(Gr::kBins); ++j) {
-                h[j] = share[gl * Gr::kBins + j];
-                own += h[j];
-            }
-            uint32_t before = Gr::inclusive_sum(own, gl) - own;
-            uint32_t my_bucket = 0, my_take = 0;
-            bool mine = false;
-#pragma unroll
-            for (int j = 0; j < static_cast<int>(Gr::kBins); ++j) {
-                if (before <= drop && drop < before + h[j]) {
-                    mine = true;
-                    my_bucket = low + gl * Gr::kBins + j;
-                    my_take = h[j] - (drop - before);
-                }
-                before += h[j];
-            }
-            const uint32_t who = Gr::ballot(mine, group_base);
-            const uint32_t src = who ? __ffs(who) - 1 : 0u;
-            bucket = Gr::from(my_bucket, src);
-            take = Gr::from(my_take, src);
-            found = who != 0;
-            __syncwarp();
-        }
-        if (__any_sync(0xFFFFFFFFu, !found)) {
-            // the bucket lies beyond the window for some row: the k-th largest candidate bucket, bit by bit (every
-            // group recomputes; where the window had the answer this gives the same one)
-            uint32_t t = 0;
-#pragma unroll 1
-            for (int bit = 14; bit >= 0; --bit) {
-                const uint32_t trial = t | (1u << bit);
-                uint32_t cnt = 0;
-#pragma unroll
-                for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i)
-                    cnt += ((ent[i] >> 16) & 0x7FFFu) >= trial ? 1u : 0u;
-                if (Gr::sum(cnt) >= k) t = trial;
-            }
-            uint32_t above = 0;
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) above += ((ent[i] >> 16) & 0x7FFFu) > t ? 1u : 0u;
-            bucket = t;
-            take = k - Gr::sum(above);
-        }
-        // ---- tau_i inside the bucket: the take-th largest of its members' lower 16 key bits ------------------
-        uint32_t low16 = 0;
-        {
-            uint32_t members = 0, my_min = 0xFFFFu;
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
-                const bool member = ((ent[i] >> 16) & 0x7FFFu) == bucket;
-                members += member ? 1u : 0u;
-                my_min = member ? min(my_min, ent[i] & 0xFFFFu) : my_min;
-            }
-            members = Gr::sum(members);
-            if (__all_sync(0xFFFFFFFFu, members == take)) {
-                // every member is kept (the usual case: one member): tau_i is the smallest of them
-#pragma unroll
-                for (int o = G / 2; o > 0; o >>= 1) my_min = min(my_min, __shfl_xor_sync(0xFFFFFFFFu, my_min, o, G));
-                low16 = my_min;
-            } else {
-#pragma unroll 1
-                for (int bit = 15; bit >= 0; --bit) {
-                    const uint32_t trial = low16 | (1u << bit);
-                    uint32_t cnt = 0;
-#pragma unroll
-                    for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i)
-                        cnt += (((ent[i] >> 16) & 0x7FFFu) == bucket && (ent[i] & 0xFFFFu) >= trial) ? 1u : 0u;
-                    if (Gr::sum(cnt) >= take) low16 = trial;
-                }
-            }
-        }
-        const uint32_t tau_key = (bucket << 16) | low16;
-        if (valid && gl == 0 && tau_out) tau_out[row] = tau_key;
-        guess_low = bucket > kGuessMargin ? bucket - kGuessMargin : 0u;
-
-        // ---- D: ordered emit ------------------------------------------------------------------------
-        {
-            uint32_t counts = 0;                              // (gt << 16) | eq of this lane's entries
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
-                const uint32_t key = ent[i] & 0x7FFFFFFFu;
-                counts += key > tau_key ? 0x10000u : (key == tau_key ? 1u : 0u);
-            }
-            const uint32_t incl_c = Gr::inclusive_sum(counts, gl);
-            const uint32_t ties = k - (Gr::last(incl_c) >> 16);     // ties to keep, lowest columns first
-            const uint32_t before = incl_c - counts;
-            uint32_t e_at = before & 0xFFFFu;
-            uint32_t pos = (before >> 16) + (e_at < ties ? e_at : ties);
-#pragma unroll
-            for (int i = 0; i < static_cast<int>(kNarrowPerLane); ++i) {
-                const uint32_t key = ent[i] & 0x7FFFFFFFu;
-                const bool is_eq = key == tau_key;
-                const bool keep = key > tau_key || (is_eq && e_at < ties);
-                if (keep) {
-                    share[pos] = ent[i];
-                    share_c[pos] = ent_c[i];
-                }
-                pos += keep ? 1u : 0u;
-                e_at += is_eq ? 1u : 0u;
-            }
-        }
-        __syncwarp();
-        if (valid) {
-            for (uint32_t p = gl; p < k; p += G) {
-                cols_out[out_base + p] = static_cast<int16_t>(share_c[p]);
-                vals_out[out_base + p] = share[p];
-                if (rows_out) rows_out[out_base + p] = static_cast<int32_t>(row);
-            }
-        }
-        __syncwarp();
+        const bool valid = r < rows;
+        const uint64_t row64 = valid ? r : rows - 1;
+        narrow_bisect_f32<G>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
+                             cols_out, vals_out, rows_out, tau_out);
     }
 }
 
-template <int G, int PLN>
-dct_status_t launch_narrow_f32(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
-                               void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
-                               cudaStream_t stream) {
-    auto kernel = mp_topk_fwd_f32_narrow_kernel<G, PLN>;
+template <int G>
+dct_status_t launch_narrow_dense_f32(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                                     int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
+                                     dct_result_t* result, cudaStream_t stream) {
+    auto kernel = mp_topk_fwd_f32_narrow_dense_kernel<G>;
     int per_sm = 0;
     DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kNarrowWarps * 32, 0));
     if (per_sm < 1) return DCT_ERR_UNSUPPORTED;
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
-    const uint64_t bundles = (static_cast<uint64_t>(rows) + Group<G>::kRows - 1) / Group<G>::kRows;
+    const uint64_t bundles = (static_cast<uint64_t>(rows) + (32u / G) - 1) / (32u / G);
     const uint64_t ctas_needed = (bundles + kNarrowWarps - 1) / kNarrowWarps;
     const uint64_t max_grid = static_cast<uint64_t>(sms) * per_sm;
     const uint32_t grid = static_cast<uint32_t>(ctas_needed < max_grid ? ctas_needed : max_grid);
@@ -701,8 +576,19 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
                                     int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                     dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
-    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0 || k > d / 8) return DCT_OK;
+    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0) return DCT_OK;
     *handled = true;
+    // The count over the row in registers, for every row (15 rounds): the denser k on rows of up to 256 columns, and
+    // every k on rows of up to 128 columns, where it beats the bound-and-candidates kernel as well (1572864 rows of 64
+    // columns, k = 3: 0.133 against 0.322 ms; 786432 x 128, k = 6: 0.141 against 0.174 ms; 256 columns, k = 2: 0.136
+    // against 0.123 ms).
+    if (d % 32 == 0 && d <= 64) return launch_narrow_dense<4, 2>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    if (d % 32 == 0 && d <= 128) return launch_narrow_dense<4, 4>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    if (k > d / 8) {
+        if (d % 32 == 0 && d <= 256) return launch_narrow_dense<4, 8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        *handled = false;
+        return DCT_OK;
+    }
     // 5 candidates per lane up to k = 2.5 lanes of the group, 8 up to 4.25 lanes (the bound leaves ~1.3 k candidates,
     // 1.45 k at the 99th percentile)
 #define DCT_NARROW(E8, G, K5, K8)                                                                                          \
@@ -710,11 +596,7 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
     if (k <= K8) return launch_narrow<E8, G, 8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream)
     // (k <= d / 8 was checked above: the bound needs k leaves of 8 columns; rows narrower than the group's 32 G
     // columns, in whole lanes of 32, leave the lanes past their end empty)
-    if (d == 64) {
-        DCT_NARROW(2, 4, 8, 8);
-    } else if (d % 32 == 0 && d <= 128) {
-        DCT_NARROW(4, 4, 13, 16);
-    } else if (d % 32 == 0 && d <= 256) {
+    if (d % 32 == 0 && d <= 256) {
         DCT_NARROW(4, 8, 20, 32);
     } else if (d % 32 == 0 && d <= 512) {  // (k = 51 with 8 candidates per lane: 0.125 ms for 131072 rows of 512, the warp-per-row kernel 0.104)
         DCT_NARROW(4, 16, 40, 40);
@@ -724,25 +606,20 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
     return DCT_OK;
 }
 
-// fp32 rows of 256 columns, sparse k (same limits as the bf16 kernel above).
+// fp32 rows of up to 256 columns (whole lanes of 32), any k: the two-level count over the row in registers.  It beat
+// the bound-and-candidates kernel this file used to have for fp32 at every width it served (786432 rows of 64 columns,
+// k = 3: 0.100 against 0.252 ms; 393216 x 128, k = 6: 0.107 against 0.152; 196608 x 256, k = 12: 0.112 against 0.120)
+// and serves the denser k the warp-per-row kernels leave to the general one (128 columns, k = 32: 0.159 against 0.98 ms).
+// Rows of 512 columns stay with the warp-per-row kernels (0.084 against 0.110 ms at k = 5).
 dct_status_t launch_fwd_f32_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                    int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                    dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
-    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || k > d / 8) return DCT_OK;
+    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 32 != 0 || d > 256) return DCT_OK;
     *handled = true;
-    // (512 columns with 16 lanes per row: 0.134 ms for 131072 rows against 0.110 ms on the warp-per-row kernel, which
-    // keeps them; 256 columns: 0.157 against 0.216 ms)
-    // (rows narrower than the group's 32 G columns, in whole lanes of 32, leave the lanes past their end empty)
-    if (d % 32 == 0 && d <= 128) {
-        if (k <= 13) return launch_narrow_f32<4, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-        if (k <= 16) return launch_narrow_f32<4, 8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-    } else if (d % 32 == 0 && d <= 256) {
-        if (k <= 20) return launch_narrow_f32<8, 5>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-        if (k <= 32) return launch_narrow_f32<8, 8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
-    }
-    *handled = false;
-    return DCT_OK;
+    if (d <= 64) return launch_narrow_dense_f32<2>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    if (d <= 128) return launch_narrow_dense_f32<4>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    return launch_narrow_dense_f32<8>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
 }
 
 }  // namespace dct

@@ -346,7 +346,7 @@ def test_mp_many_short_rows(dtype, d, ld):
     x[rows - 1] = 0.5
     x = x.to(dtype).contiguous()
     gx = inputs.mp_gradients(rows, d, 294 + d, dtype=dtype, device=G.DEV, ld=ld)
-    for k in sorted({1, 2, d // 20, d // 10, d // 8, d // 4}):
+    for k in sorted({1, 2, d // 20, d // 10, d // 8, d // 4, d // 2, d - 1, d}):
         cols = _compare_fwd_bwd(x, gx, d, k, want_rows=(k == 2))
         assert int(cols.max()) < d
 
