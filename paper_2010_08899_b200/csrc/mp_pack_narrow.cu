@@ -615,7 +615,14 @@ dct_status_t launch_fwd_f32_narrow(const void* x_act, uint32_t rows, uint32_t d,
                                    int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                    dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
-    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 32 != 0 || d > 256) return DCT_OK;
+    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 32 != 0) return DCT_OK;
+    // 288 to 480 columns, the denser k: 16 lanes per row (the bounds-and-bit-tables kernel of the 512-column buffer
+    // is crowded by rows that fill only part of it: 320 columns, k = 80: 0.47 TB/s)
+    if (d > 256 && d < 512 && fwd_candidates_per_lane(d, k) == 0) {
+        *handled = true;
+        return launch_narrow_dense_f32<16>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    }
+    if (d > 256) return DCT_OK;
     *handled = true;
     if (d <= 64) return launch_narrow_dense_f32<2>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
     if (d <= 128) return launch_narrow_dense_f32<4>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
