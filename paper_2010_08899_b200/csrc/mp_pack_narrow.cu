@@ -358,6 +358,89 @@ dct_status_t launch_narrow(const void* x_act, uint32_t rows, uint32_t d, uint32_
     return DCT_OK;
 }
 
+// The largest 15-bit value t with "at least k of the row's keys are >= t", by counting (count_ge(t): the lane's keys
+// >= t; the G lanes of the group are summed here).  With a guess (the value the group found for its previous row;
+// 0: none) the search first tries the 256 values around it: two counts to see that the answer lies among them, then
+// 8 halvings; otherwise, or if a group of the warp finds its guess off, 15 rounds bit by bit.  The control flow is
+// the warp's (the sums are shuffles of all 32 lanes), so one group with a bad guess takes the others along.
+template <int G, typename CountGe>
+__device__ __forceinline__ uint32_t narrow_search15(CountGe&& count_ge, uint32_t k, uint32_t guess) {
+    using Gr = Group<G>;
+    constexpr uint32_t kHalf = 128;                  // one binade of bf16 keys on either side
+    uint32_t lo = guess > kHalf ? guess - kHalf : 0u, hi = guess + kHalf < 0x8000u ? guess + kHalf : 0x8000u;
+    bool ok = guess != 0;
+    if (__any_sync(0xFFFFFFFFu, ok)) {               // (no group has a guess: skip the two counts)
+        const uint32_t at_lo = Gr::sum(count_ge(lo)), at_hi = Gr::sum(count_ge(hi));   // (nothing is >= 0x8000)
+        ok = ok && at_lo >= k && at_hi < k;
+    }
+    if (__all_sync(0xFFFFFFFFu, ok)) {
+#pragma unroll 1
+        for (int round = 0; round < 8; ++round) {    // hi - lo <= 256: 8 halvings leave one value
+            const uint32_t mid = lo + ((hi - lo) >> 1);
+            if (Gr::sum(count_ge(mid)) >= k) lo = mid; else hi = mid;
+        }
+        return lo;
+    }
+    uint32_t key = 0;
+#pragma unroll 1
+    for (int bit = 14; bit >= 0; --bit) {
+        const uint32_t trial = key | (1u << bit);
+        if (Gr::sum(count_ge(trial)) >= k) key = trial;
+    }
+    return key;
+}
+
+// One bf16 row of a group by the count over the row in registers: narrow_slow_path with the search started from the
+// group's previous tau_i (`guess`, updated).
+template <int E8, int G>
+__device__ __forceinline__ void narrow_count_path(const uint16_t* __restrict__ xr, uint32_t d, bool valid, uint32_t k,
+                                                  size_t out_base, uint32_t row, int16_t* __restrict__ cols_out,
+                                                  uint16_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
+                                                  uint16_t* __restrict__ tau_out, uint32_t& guess) {
+    using Gr = Group<G>;
+    constexpr uint32_t E = E8 * 8u;
+    const uint32_t gl = lane_id() & (G - 1);
+    const uint4* mine = reinterpret_cast<const uint4*>(xr + gl * E);
+    uint4 v[E8];                                   // (a lane past the end of the row holds zeros: the last columns)
+#pragma unroll
+    for (int c = 0; c < E8; ++c) v[c] = gl * E < d ? __ldg(mine + c) : make_uint4(0, 0, 0, 0);
+    const uint32_t tau_key = narrow_search15<G>([&](uint32_t t) {
+        uint32_t cnt = 0;
+#pragma unroll
+        for (int c = 0; c < E8; ++c) cnt += __popc(mask8_ge_exact(v[c], t));
+        return cnt;
+    }, k, guess);
+    guess = tau_key;
+    uint32_t gt_mask = 0, eq_mask = 0;
+#pragma unroll
+    for (int c = 0; c < E8; ++c) {
+        const uint32_t gt = mask8_ge_exact(v[c], tau_key + 1u);
+        const uint32_t eq = mask8_ge_exact(v[c], tau_key) & ~gt;
+        gt_mask |= gt << (8 * c);
+        eq_mask |= eq << (8 * c);
+    }
+    const uint32_t n_gt_mine = __popc(gt_mask), n_eq_mine = __popc(eq_mask);
+    const uint32_t incl = Gr::inclusive_sum(n_gt_mine, gl);
+    const uint32_t take = k - Gr::last(incl);       // ties to keep, lowest columns first
+    uint32_t g_at = incl - n_gt_mine;
+    uint32_t e_at = Gr::inclusive_sum(n_eq_mine, gl) - n_eq_mine;
+    uint32_t m = valid ? (gt_mask | eq_mask) : 0u;
+    while (m) {
+        const uint32_t j = __ffs(m) - 1;
+        m &= m - 1;
+        const bool is_eq = (eq_mask >> j) & 1u;
+        if (!is_eq || e_at < take) {
+            const size_t pos = out_base + g_at + (e_at < take ? e_at : take);
+            cols_out[pos] = static_cast<int16_t>(gl * E + j);
+            vals_out[pos] = xr[gl * E + j];
+            if (rows_out) rows_out[pos] = static_cast<int32_t>(row);
+        }
+        g_at += is_eq ? 0u : 1u;
+        e_at += is_eq ? 1u : 0u;
+    }
+    if (valid && gl == 0 && tau_out) tau_out[row] = static_cast<uint16_t>(tau_key);
+}
+
 // Denser k (more than an eighth of the row: no leaf bound applies): every row takes the bit-by-bit count over the
 // row in registers, 15 rounds for a bf16 key, and the ordered emit from the row.  The warp kernels and the general
 // kernel pay their fixed cost per row for these short rows; here a warp serves 32 / G rows at once.
@@ -379,12 +462,13 @@ mp_topk_fwd_bf16_narrow_dense_kernel(const uint16_t* __restrict__ x, uint32_t ro
     }
     const uint64_t bundles = (static_cast<uint64_t>(rows) + kRows - 1) / kRows;
     const uint64_t bundle_step = static_cast<uint64_t>(gridDim.x) * (blockDim.x >> 5);
+    uint32_t guess = 0;                              // tau_i of the group's previous row
     for (uint64_t bundle = blockIdx.x + static_cast<uint64_t>(gridDim.x) * warp; bundle < bundles; bundle += bundle_step) {
         const uint64_t r = bundle * kRows + group;
         const bool valid = r < rows;
         const uint64_t row64 = valid ? r : rows - 1;     // a group past the last row runs along on the last row
-        narrow_slow_path<E8, G>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
-                                cols_out, vals_out, rows_out, tau_out);
+        narrow_count_path<E8, G>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
+                                 cols_out, vals_out, rows_out, tau_out, guess);
     }
 }
 
@@ -425,7 +509,7 @@ template <int G>
 __device__ __forceinline__ void narrow_bisect_f32(const uint32_t* __restrict__ xr, uint32_t d, bool valid, uint32_t k,
                                                   size_t out_base, uint32_t row, int16_t* __restrict__ cols_out,
                                                   uint32_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
-                                                  uint32_t* __restrict__ tau_out) {
+                                                  uint32_t* __restrict__ tau_out, uint32_t& guess) {
     using Gr = Group<G>;
     constexpr uint32_t E = 32u;
     const uint32_t gl = lane_id() & (G - 1);
@@ -446,15 +530,13 @@ __device__ __forceinline__ void narrow_bisect_f32(const uint32_t* __restrict__ x
             up[c / 2].y = upper_halves(v.z, v.w);
         }
     }
-    uint32_t bucket = 0;
-#pragma unroll 1
-    for (int bit = 14; bit >= 0; --bit) {
-        const uint32_t trial = bucket | (1u << bit);
+    const uint32_t bucket = narrow_search15<G>([&](uint32_t t) {
         uint32_t cnt = 0;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) cnt += __popc(mask8_ge_exact(up[c], trial));
-        if (Gr::sum(cnt) >= k) bucket = trial;
-    }
+        for (int c = 0; c < 4; ++c) cnt += __popc(mask8_ge_exact(up[c], t));
+        return cnt;
+    }, k, guess);
+    guess = bucket;                                // (the group's next row starts its search around this bucket)
     uint32_t above = 0, members = 0;               // columns of the lane above the bucket / inside it
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
@@ -537,12 +619,13 @@ mp_topk_fwd_f32_narrow_dense_kernel(const uint32_t* __restrict__ x, uint32_t row
     }
     const uint64_t bundles = (static_cast<uint64_t>(rows) + kRows - 1) / kRows;
     const uint64_t bundle_step = static_cast<uint64_t>(gridDim.x) * (blockDim.x >> 5);
+    uint32_t guess = 0;                              // bucket of tau_i of the group's previous row
     for (uint64_t bundle = blockIdx.x + static_cast<uint64_t>(gridDim.x) * warp; bundle < bundles; bundle += bundle_step) {
         const uint64_t r = bundle * kRows + group;
         const bool valid = r < rows;
         const uint64_t row64 = valid ? r : rows - 1;
         narrow_bisect_f32<G>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
-                             cols_out, vals_out, rows_out, tau_out);
+                             cols_out, vals_out, rows_out, tau_out, guess);
     }
 }
 
