@@ -292,13 +292,81 @@ mp_unpack_staged_kernel(const int16_t* __restrict__ cols, const T* __restrict__ 
     if (bad && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
 }
 
+// (a thread walks all k columns of its row, so the work per row is units * k: beyond ~250 the warp-per-row kernel with
+// its shared-memory row wins again -- 393216 rows of 256 bf16 columns, k = 12: 0.231 against 0.094 ms)
+constexpr uint32_t kUnpackFlatMaxWork = 256;
+// Short rows with few kept columns (the paper's layer widths): one THREAD per 16-byte unit of the dense matrix.  The
+// thread reads the k columns of its row (the threads of a row sit in the same warp or the next: the loads are
+// broadcasts or L1 hits), puts the values that fall into its unit into four registers and stores the unit; nothing
+// goes through shared memory, every lane works, HBM sees full sequential 16-byte writes.  (With a warp per row a row
+// of 128 bytes uses 8 of 32 lanes per store: 1572864 rows of 64 bf16 columns, k = 3: 0.354 ms.)  Row and unit advance
+// by fixed steps from one of a thread's units to the next, so only the first costs a division.
+template <typename T>
+__global__ void __launch_bounds__(256)
+mp_unpack_flat_kernel(const int16_t* __restrict__ cols, const T* __restrict__ vals, uint32_t rows, uint32_t d,
+                      uint32_t ld, uint32_t k, T* __restrict__ dense, dct_result_t* __restrict__ result) {
+    constexpr uint32_t per16 = 16 / sizeof(T);
+    const uint32_t units = d / per16;                  // 16-byte units of a row
+    const uint64_t total = static_cast<uint64_t>(rows) * units;
+    const uint64_t round = static_cast<uint64_t>(gridDim.x) * blockDim.x;
+    const uint64_t round_q = round / units;
+    const uint32_t round_r = static_cast<uint32_t>(round % units);
+    uint64_t e = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    uint64_t row = e / units;
+    uint32_t unit = static_cast<uint32_t>(e - row * units);
+    bool bad = false;
+    for (; e < total; e += round) {
+        const int16_t* cr = cols + row * k;
+        const T* vr = vals + row * k;
+        uint32_t w0 = 0, w1 = 0, w2 = 0, w3 = 0;
+        for (uint32_t s = 0; s < k; ++s) {
+            const uint32_t c = static_cast<uint16_t>(__ldg(cr + s));
+            if (c >= d) {
+                bad = true;
+                continue;
+            }
+            if (c / per16 != unit) continue;
+            const uint32_t p = c % per16;
+            if constexpr (sizeof(T) == 2) {
+                const uint32_t sh = (p & 1u) * 16u, keep = ~(0xFFFFu << sh);
+                const uint32_t v = static_cast<uint32_t>(__ldg(reinterpret_cast<const uint16_t*>(vr) + s)) << sh;
+                const uint32_t word = p >> 1;
+                w0 = word == 0 ? (w0 & keep) | v : w0;
+                w1 = word == 1 ? (w1 & keep) | v : w1;
+                w2 = word == 2 ? (w2 & keep) | v : w2;
+                w3 = word == 3 ? (w3 & keep) | v : w3;
+            } else {
+                const uint32_t v = __ldg(reinterpret_cast<const uint32_t*>(vr) + s);
+                w0 = p == 0 ? v : w0;
+                w1 = p == 1 ? v : w1;
+                w2 = p == 2 ? v : w2;
+                w3 = p == 3 ? v : w3;
+            }
+        }
+        __stcs(reinterpret_cast<uint4*>(dense + row * ld + static_cast<size_t>(unit) * per16), make_uint4(w0, w1, w2, w3));
+        row += round_q;
+        unit += round_r;
+        if (unit >= units) {
+            unit -= units;
+            ++row;
+        }
+    }
+    if (bad && result) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
+}
+
 template <typename T>
 cudaError_t launch_unpack(const int16_t* cols, const void* vals, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                           void* dense_out, dct_result_t* result, int sms, cudaStream_t stream) {
     const size_t row_bytes = static_cast<size_t>(d) * sizeof(T);
     const bool staged = aligned_to(dense_out, 16) && (static_cast<size_t>(ld) * sizeof(T)) % 16 == 0 &&
                         row_bytes % 16 == 0 && row_bytes <= 16 * 1024;
-    if (staged) {
+    if (staged && (row_bytes / 16) * k <= kUnpackFlatMaxWork) {
+        const uint64_t total = static_cast<uint64_t>(rows) * (row_bytes / 16);
+        const uint64_t need = (total + 255) / 256;
+        const uint64_t cap = static_cast<uint64_t>(sms) * 32;
+        mp_unpack_flat_kernel<T><<<static_cast<unsigned>(need < cap ? need : cap), 256, 0, stream>>>(
+            cols, static_cast<const T*>(vals), rows, d, ld, k, static_cast<T*>(dense_out), result);
+    } else if (staged) {
         const size_t smem = kUnpackWarps * row_bytes;
         auto kernel = k <= 256 ? mp_unpack_staged_kernel<T, 8> : (k <= 512 ? mp_unpack_staged_kernel<T, 16> : mp_unpack_staged_kernel<T, 0>);
         // (static shared memory counts against the 48 KiB a kernel gets without asking: ask well below that)

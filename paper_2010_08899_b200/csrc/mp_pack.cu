@@ -185,6 +185,79 @@ mp_pack_bwd_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t
     }
 }
 
+// The same for small k (fewer kept columns than lanes): one THREAD per kept entry, the rows' entries taken as one list
+// of rows * k -- with a warp per row only k of 32 lanes work (1572864 rows of 64 columns, k = 3: 0.215 ms).  A thread
+// takes four entries blockDim apart per round; row and position inside the row advance by fixed steps, so only the first
+// entry of a thread costs a division.
+template <typename T>
+__global__ void __launch_bounds__(256)
+mp_pack_bwd_flat_kernel(const T* __restrict__ gx, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
+                        const int16_t* __restrict__ cols, T* __restrict__ gvals, dct_result_t* __restrict__ result,
+                        uint32_t ticket) {
+    bool bad = false;
+    if (blockIdx.x == 0 && threadIdx.x == 0 && result) {
+        result->status = DCT_OK;
+        result->count = 0;
+        result->needed = 0;
+        result->n_gt = 0;
+        result->n_eq = 0;
+        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(&result->reserved), "r"(ticket) : "memory");
+    }
+    const uint64_t total = static_cast<uint64_t>(rows) * k;
+    const uint32_t step_q = blockDim.x / k, step_r = blockDim.x % k;                        // one step of blockDim entries
+    const uint64_t round = static_cast<uint64_t>(gridDim.x) * blockDim.x * 4u;              // one round of the grid
+    const uint64_t round_q = round / k;
+    const uint32_t round_r = static_cast<uint32_t>(round % k);
+    uint64_t e0 = static_cast<uint64_t>(blockIdx.x) * blockDim.x * 4u + threadIdx.x;
+    uint64_t row0 = e0 / k;
+    uint32_t s0 = static_cast<uint32_t>(e0 - row0 * k);
+    for (; e0 < total; e0 += round) {
+        uint32_t c[4];
+        uint64_t row[4];
+        uint64_t r = row0;
+        uint32_t s = s0;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint64_t e = e0 + static_cast<uint64_t>(u) * blockDim.x;
+            row[u] = r;
+            c[u] = e < total ? static_cast<uint16_t>(__ldg(cols + e)) : 0u;
+            r += step_q;
+            s += step_r;
+            if (s >= k) {
+                s -= k;
+                ++r;
+            }
+        }
+        T v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint64_t e = e0 + static_cast<uint64_t>(u) * blockDim.x;
+            const bool ok = c[u] < d;
+            if (e < total && !ok) bad = true;
+            v[u] = (e < total && ok) ? gather_load(gx + row[u] * ld + c[u]) : T(0);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint64_t e = e0 + static_cast<uint64_t>(u) * blockDim.x;
+            if (e < total) gvals[e] = v[u];
+        }
+        row0 += round_q;
+        s0 += round_r;
+        if (s0 >= k) {
+            s0 -= k;
+            ++row0;
+        }
+    }
+    if (bad && result) {
+        for (uint32_t spin = 0; spin < (1u << 20); ++spin) {          // CTA 0 is dispatched first: normally no wait at all
+            uint32_t seen;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&result->reserved) : "memory");
+            if (seen == ticket) break;
+        }
+        atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // bf16 fast path: one warp per row, d <= 8192 a multiple of 8 (held in a buffer of 256 * E8 columns), rows on 16-byte boundaries
 // ------------------------------------------------------------------------------------------
@@ -785,6 +858,15 @@ dct_status_t launch_bwd(const void* x_grad, uint32_t rows, uint32_t d, uint32_t 
                         void* gvals_out, dct_result_t* result, cudaStream_t stream) {
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
+    if (k <= 24) {                // fewer kept columns than lanes: a thread per entry
+        const uint64_t total = static_cast<uint64_t>(rows) * k;
+        const uint64_t need = (total + 1023) / 1024;
+        const uint64_t cap = static_cast<uint64_t>(sms) * 16;
+        mp_pack_bwd_flat_kernel<T><<<static_cast<unsigned>(need < cap ? need : cap), 256, 0, stream>>>(
+            static_cast<const T*>(x_grad), rows, d, ld, k, cols, static_cast<T*>(gvals_out), result, next_launch_ticket());
+        DCT_CUDA_TRY(cudaGetLastError());
+        return DCT_OK;
+    }
     const uint64_t ctas_needed = (static_cast<uint64_t>(rows) + 7) / 8;
     // one row per warp up to 256 rows per SM: CTAs then start as others finish, which evens out the last round
     // (a grid of 8 resident CTAs per SM with a stride loop gives a warp 1 or 2 rows: 4 % slower at 16384 rows)
