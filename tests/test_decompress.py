@@ -153,7 +153,12 @@ def test_gpu_dp_decompress_reports_bad_indices_without_touching_anything_else():
 @pytest.mark.gpu
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("rows,d,ld,k", [(1, 1, 1, 1), (37, 33, 40, 5), (64, 1000, 1000, 50), (300, 4096, 4096, 205),
-                                         (9, 4097, 4101, 400)])
+                                         (9, 4097, 4101, 400),
+                                         # short rows with few kept columns: a thread per 16-byte unit
+                                         (70001, 64, 64, 3), (5003, 64, 72, 16), (3001, 128, 136, 6), (2000, 256, 256, 2),
+                                         (999, 32, 32, 32), (777, 8, 8, 1),
+                                         # just beyond that kernel's reach
+                                         (3000, 128, 128, 32), (1000, 512, 512, 25)])
 def test_gpu_mp_unpack_matches_oracle_and_round_trips(dtype, rows, d, ld, k):
     from paper_2010_08899_b200 import binding as B
     from tests import _gpu as G
@@ -203,6 +208,27 @@ def test_gpu_dp_decompress_checks_the_whole_index_list(bad_idx, accumulate):
     res2 = B.new_result()
     B.dct_dp_decompress(idx2, val[:len(ok)].contiguous(), packed2, len(ok), buf[:n], n, accumulate, res2)
     assert B.read_result(res2).status == B.DCT_OK
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_gpu_mp_unpack_of_short_rows_rejects_out_of_range_and_takes_any_order(dtype):
+    """The thread-per-unit kernel for short rows: a column past the row is skipped and reported, the other entries of
+    the row are placed, and the columns of a row need not be ascending."""
+    from paper_2010_08899_b200 import binding as B
+    rows, d, k = 4, 64, 3
+    cols = torch.tensor([[0, 1, 2], [3, 64, 5], [63, 7, 8], [-1, 10, 9]], dtype=torch.int16, device="cuda")
+    vals = torch.arange(1, rows * k + 1, dtype=torch.float32, device="cuda").view(rows, k).to(dtype)
+    dense = torch.full((rows, d), 2.0, dtype=dtype, device="cuda")
+    res = B.new_result()
+    B.dct_mp_unpack(cols, vals, rows, d, d, k, dense, res)
+    assert B.read_result(res).status == B.DCT_ERR_BAD_MASK
+    want = torch.zeros(rows, d, device="cuda")
+    want[0, 0], want[0, 1], want[0, 2] = 1, 2, 3
+    want[1, 3], want[1, 5] = 4, 6
+    want[2, 63], want[2, 7], want[2, 8] = 7, 8, 9
+    want[3, 10], want[3, 9] = 11, 12
+    assert torch.equal(dense.float(), want)
 
 
 @pytest.mark.gpu
