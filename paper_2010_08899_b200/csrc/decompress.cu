@@ -217,6 +217,9 @@ mp_unpack_kernel(const int16_t* __restrict__ cols, const T* __restrict__ vals, u
 // row in shared memory (clear, scatter the k kept values) and writes it out with 128-bit streaming stores, so HBM only
 // sees full, sequential 16-byte-aligned writes.
 constexpr int kUnpackWarps = 8;
+// kSlots > 0: the row's entries (k <= 32 kSlots) in registers, fetched one row ahead; kSlots == 0: any k, the entries
+// read as they are scattered; kSlots == -1: the same for the denser k, where zeroing the whole row buffer again (one
+// 128-bit store per 16 bytes) is cheaper than clearing the k positions one by one.
 template <typename T, int kSlots>
 __global__ void __launch_bounds__(kUnpackWarps * 32)
 mp_unpack_staged_kernel(const int16_t* __restrict__ cols, const T* __restrict__ vals, uint32_t rows, uint32_t d,
@@ -276,16 +279,31 @@ mp_unpack_staged_kernel(const int16_t* __restrict__ cols, const T* __restrict__ 
             const int16_t* cr = cols + row * k;
             const T* vr = vals + row * k;
             __syncwarp();
-            for (uint32_t s = lane; s < k; s += 32) {
-                const uint32_t c = static_cast<uint16_t>(__ldg(cr + s));
-                if (c < d) buf[c] = __ldg(vr + s); else bad = true;
+            for (uint32_t s0 = lane; s0 < k; s0 += 128) {          // four entries of a lane in flight
+                uint32_t c[4];
+                T v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint32_t s = s0 + 32u * u;
+                    c[u] = s < k ? static_cast<uint16_t>(__ldg(cr + s)) : 0xFFFFFFFFu;
+                    if (s < k) v[u] = __ldg(vr + s);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (c[u] < d) buf[c[u]] = v[u];
+                    else if (c[u] != 0xFFFFFFFFu) bad = true;
+                }
             }
             __syncwarp();
             write_out(row);
             __syncwarp();
-            for (uint32_t s = lane; s < k; s += 32) {              // (L1 still holds the columns)
-                const uint32_t c = static_cast<uint16_t>(__ldg(cr + s));
-                if (c < d) buf[c] = T(0);
+            if (kSlots < 0) {
+                for (uint32_t v = lane; v < row_bytes / 16; v += 32) b16[v] = make_uint4(0, 0, 0, 0);
+            } else {
+                for (uint32_t s = lane; s < k; s += 32) {          // (L1 still holds the columns)
+                    const uint32_t c = static_cast<uint16_t>(__ldg(cr + s));
+                    if (c < d) buf[c] = T(0);
+                }
             }
         }
     }
@@ -368,7 +386,11 @@ cudaError_t launch_unpack(const int16_t* cols, const void* vals, uint32_t rows, 
             cols, static_cast<const T*>(vals), rows, d, ld, k, static_cast<T*>(dense_out), result);
     } else if (staged) {
         const size_t smem = kUnpackWarps * row_bytes;
-        auto kernel = k <= 256 ? mp_unpack_staged_kernel<T, 8> : (k <= 512 ? mp_unpack_staged_kernel<T, 16> : mp_unpack_staged_kernel<T, 0>);
+        // (the denser k, more than an eighth of the row: zero the whole buffer instead of the k positions)
+        const bool zero_all = static_cast<size_t>(k) * (sizeof(T) == 2 ? 16 : 32) > row_bytes;     // k > d / 8
+        auto kernel = zero_all ? mp_unpack_staged_kernel<T, -1>
+                               : (k <= 256 ? mp_unpack_staged_kernel<T, 8>
+                                           : (k <= 512 ? mp_unpack_staged_kernel<T, 16> : mp_unpack_staged_kernel<T, 0>));
         // (static shared memory counts against the 48 KiB a kernel gets without asking: ask well below that)
         if (smem > 32 * 1024) {
             const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
