@@ -858,7 +858,10 @@ dct_status_t launch_bwd(const void* x_grad, uint32_t rows, uint32_t d, uint32_t 
                         void* gvals_out, dct_result_t* result, cudaStream_t stream) {
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
-    if (k <= 24) {                // fewer kept columns than lanes: a thread per entry
+    // A thread per entry: fewer kept columns than lanes, and the widest rows, where it is as fast or faster at every k
+    // (3072 rows of 32768 bf16 columns, k = 8192: 0.129 -> 0.073 ms; fp32: 0.127 -> 0.043 ms); on rows of up to 4096 bf16
+    // columns the warp per row is 10 to 15 % faster at the denser k and equal otherwise.
+    if (k <= 24 || d >= 8192 || (sizeof(T) == 4 && d >= 4096)) {
         const uint64_t total = static_cast<uint64_t>(rows) * k;
         const uint64_t need = (total + 1023) / 1024;
         const uint64_t cap = static_cast<uint64_t>(sms) * 16;

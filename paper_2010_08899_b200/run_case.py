@@ -13,6 +13,7 @@ A small command-line driver for profiling and quick timing of a single kernel at
     python -m paper_2010_08899_b200.run_case threshold_mean --rows 16384 --d 4096 --dtype bf16
     python -m paper_2010_08899_b200.run_case mp_fwd_sweep --dtype bf16    (a table: row widths x sparsity levels)
     python -m paper_2010_08899_b200.run_case dp_sweep                     (a table: vector sizes x densities)
+    python -m paper_2010_08899_b200.run_case receiver_sweep               (backward pack, unpack, decompress over shapes)
 
 It prints the mean device time per call (CUDA events) and the algorithmic GB/s.
 """
@@ -105,10 +106,69 @@ def dp_sweep(args, dev, stream):
         del g, e, idx, val, ws_s, ws_c, ws_l
 
 
+def receiver_sweep(args, dev, stream):
+    """The backward pack and the receiver side over shapes: `dct_mp_pack_bwd` and `dct_mp_unpack` for both dtypes, row
+    widths from 64 to 32768 columns and k = 1 %, 5 % and 25 % of the row (192 MiB of matrix per cell; the forward pack
+    beside them), then `dct_dp_decompress` (overwriting and accumulating) at N = 2^28 over survivor densities.  ms per
+    call and TB/s: forward and unpack count the dense matrix + the packed entries, the backward pack the dense matrix
+    (what reaches DRAM), decompress 4 B (accumulating: 8 B) per element + 8 B per survivor."""
+    def timed(call, reps):
+        for phase in range(2):
+            a = torch.cuda.Event(enable_timing=True)
+            b = torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(reps):
+                call(i)
+            b.record(stream)
+            b.synchronize()
+        return a.elapsed_time(b) / reps
+    print("dtype      d     k     rows |  fwd ms (TB/s) |  bwd ms (TB/s) | unpack ms (TB/s)")
+    for dt, es in ((torch.bfloat16, 2), (torch.float32, 4)):
+        for d in (64, 128, 256, 512, 1024, 2048, 4096, 8192, 16384, 32768):
+            rows = max(256, (192 << 20) // (d * es))
+            kmax = max(1, d // 4)
+            x = [inputs.mp_activations(rows, d, 410 + j, dtype=dt, device=dev, col_scale_seed=400) for j in range(2)]
+            gx = [inputs.mp_gradients(rows, d, 420 + j, dtype=dt, device=dev) for j in range(2)]
+            cols = torch.empty(rows * kmax, dtype=torch.int16, device=dev)
+            vals = torch.empty(rows * kmax, dtype=dt, device=dev)
+            gv = torch.empty(rows * kmax, dtype=dt, device=dev)
+            dense = [torch.empty(rows, d, dtype=dt, device=dev) for _ in range(2)]
+            for k in sorted({max(1, d // 100), max(1, d // 20), max(1, d // 4)}):
+                f = timed(lambda i: B.dct_mp_topk_pack_fwd(x[i % 2], rows, d, d, k, cols, vals, None, None, None, stream), args.iters)
+                B.dct_mp_topk_pack_fwd(x[0], rows, d, d, k, cols, vals, None, None, None, stream)
+                bw = timed(lambda i: B.dct_mp_pack_bwd(gx[i % 2], rows, d, d, k, cols, gv, None, stream), args.iters)
+                u = timed(lambda i: B.dct_mp_unpack(cols, vals, rows, d, d, k, dense[i % 2], None, stream), args.iters)
+                nb, pk = rows * d * es, rows * k * (2 + es)
+                print(f"{'bf16' if es == 2 else 'f32 '} {d:6d} {k:5d} {rows:8d} | {f:7.4f} ({(nb + pk) / f / 1e9:5.2f}) | "
+                      f"{bw:7.4f} ({nb / bw / 1e9:5.2f}) | {u:7.4f} ({(nb + pk) / u / 1e9:5.2f})", flush=True)
+            del x, gx, cols, vals, gv, dense
+    n = 1 << 28
+    print(f"decompress, N = 2^28: survivors | overwrite ms (TB/s) | accumulate ms (TB/s)")
+    g = inputs.dp_mixture(n, 7, dev)
+    e = torch.zeros(n, device=dev)
+    tau, res, res2 = torch.zeros(1, device=dev), B.new_result(dev), B.new_result(dev)
+    ws_s = B.new_workspace(B.dct_threshold_select_workspace_bytes(n), dev)
+    ws_c = B.new_workspace(B.dct_dp_compress_workspace_bytes(n), dev)
+    cap = n // 4 + 1024
+    idx = torch.empty(cap, dtype=torch.int32, device=dev)
+    val = torch.empty(cap, device=dev)
+    dense = torch.empty(n, device=dev)
+    for dens in (1e-4, 1e-3, 1e-2, 0.05, 0.25):
+        B.dct_threshold_select(g, None, n, int(n * dens), tau, res, ws_s, stream)
+        e.zero_()
+        B.dct_dp_compress(g, e, n, tau, None, idx, val, cap, res, ws_c, stream)
+        cnt = B.read_result(res).count
+        packed = res.clone()
+        ms = timed(lambda i: B.dct_dp_decompress(idx, val, packed, cap, dense, n, False, res2, stream), args.iters)
+        ms_a = timed(lambda i: B.dct_dp_decompress(idx, val, packed, cap, dense, n, True, res2, stream), args.iters)
+        print(f"{cnt:10d} ({100 * dens:g} %) | {ms:7.4f} ({(4 * n + 8 * cnt) / ms / 1e9:5.2f}) | "
+              f"{ms_a:7.4f} ({(8 * n + 8 * cnt) / ms_a / 1e9:5.2f})", flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser(description=__doc__, formatter_class=argparse.RawDescriptionHelpFormatter)
     ap.add_argument("entry", choices=["select", "compress", "select_compress", "compress_layers", "decompress", "mp_fwd", "mp_bwd", "mp_unpack",
-                                     "select_multi", "threshold_mean", "mp_fwd_sweep", "dp_sweep"])
+                                     "select_multi", "threshold_mean", "mp_fwd_sweep", "dp_sweep", "receiver_sweep"])
     ap.add_argument("--n", type=int, default=1 << 28)
     ap.add_argument("--k", type=int, default=0, help="survivor target (default: 0.01 %% of n, or 5 %% of d)")
     ap.add_argument("--rows", type=int, default=16384)
@@ -143,6 +203,8 @@ def main():
         return mp_fwd_sweep(args, dev, stream)
     if args.entry == "dp_sweep":
         return dp_sweep(args, dev, stream)
+    if args.entry == "receiver_sweep":
+        return receiver_sweep(args, dev, stream)
     gen = {"mixture": inputs.dp_mixture, "gaussian": inputs.dp_gaussian, "dlrm": inputs.dp_dlrm_like}[args.dist]
 
     if args.entry == "compress_layers":
