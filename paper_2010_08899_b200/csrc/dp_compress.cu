@@ -615,12 +615,25 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
             const int s = it % kStages;
             uint32_t tile = ticket < total_work ? ticket : kInvalidTile;
             if (kBatched && tile != kInvalidTile) {
-                if (tile >= work_hi) {                                 // tickets only grow: walk forward
-                    do {
-                        ++cur_layer;
-                        work_lo = work_hi;
-                        work_hi = batch.full_prefix[cur_layer + 1];
-                    } while (tile >= work_hi);
+                if (tile >= work_hi) {
+                    // Tickets only grow: the first later vector whose tiles reach beyond this one.  With large vectors it
+                    // is the next one or two; with thousands of small ones a CTA's next ticket lies hundreds of vectors
+                    // on, and stepping through them one dependent load at a time held the whole CTA up.  So: steps of
+                    // 1, 2, 4, ... vectors (the first probes share a cache line), then bisection inside the last step.
+                    const uint32_t last = batch.num_layers - 1;
+                    uint32_t lo = cur_layer + 1, hi = lo, step = 1;
+                    while (hi < last && batch.full_prefix[hi + 1] <= tile) {
+                        lo = hi + 1;
+                        hi = last - hi > step ? hi + step : last;
+                        step <<= 1;
+                    }
+                    while (lo < hi) {
+                        const uint32_t mid = (lo + hi) >> 1;
+                        if (batch.full_prefix[mid + 1] > tile) hi = mid; else lo = mid + 1;
+                    }
+                    cur_layer = lo;
+                    work_lo = batch.full_prefix[lo];
+                    work_hi = batch.full_prefix[lo + 1];
                     grad = batch.layers[cur_layer].grad;
                     residual = batch.layers[cur_layer].residual;
                 }
