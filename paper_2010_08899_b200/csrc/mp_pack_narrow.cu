@@ -602,7 +602,7 @@ __device__ __forceinline__ void narrow_bisect_f32(const uint32_t* __restrict__ x
 
 // Denser k, fp32: the two-level bit-by-bit count over the row in registers (narrow_bisect_f32), for every row.
 template <int G>
-__global__ void __launch_bounds__(kNarrowWarps * 32)
+__global__ void __launch_bounds__(kNarrowWarps * 32, 2)
 mp_topk_fwd_f32_narrow_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                     int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
                                     int32_t* __restrict__ rows_out, uint32_t* __restrict__ tau_out,
