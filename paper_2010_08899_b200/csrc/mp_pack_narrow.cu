@@ -371,6 +371,7 @@ __device__ __forceinline__ uint32_t narrow_search15(CountGe&& count_ge, uint32_t
     bool ok = guess != 0;
     if (__any_sync(0xFFFFFFFFu, ok)) {               // (no group has a guess: skip the two counts)
         const uint32_t at_lo = Gr::sum(count_ge(lo)), at_hi = Gr::sum(count_ge(hi));   // (nothing is >= 0x8000)
+        // (the sums are shuffles of all 32 lanes: they stay outside every condition that a lane can fail)
         ok = ok && at_lo >= k && at_hi < k;
     }
     if (__all_sync(0xFFFFFFFFu, ok)) {
