@@ -393,7 +393,9 @@ __device__ __forceinline__ uint32_t narrow_search15(CountGe&& count_ge, uint32_t
 
 // One bf16 row of a group by the count over the row in registers: narrow_slow_path with the search started from the
 // group's previous tau_i (`guess`, updated).
-template <int E8, int G>
+// kAligned == false: rows of any width up to 32 G columns at any address (16-bit loads, columns past the end read as
+// zeros, which lie below every bound and, being the last columns, lose every tie).
+template <int E8, int G, bool kAligned = true>
 __device__ __forceinline__ void narrow_count_path(const uint16_t* __restrict__ xr, uint32_t d, bool valid, uint32_t k,
                                                   size_t out_base, uint32_t row, int16_t* __restrict__ cols_out,
                                                   uint16_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
@@ -401,10 +403,22 @@ __device__ __forceinline__ void narrow_count_path(const uint16_t* __restrict__ x
     using Gr = Group<G>;
     constexpr uint32_t E = E8 * 8u;
     const uint32_t gl = lane_id() & (G - 1);
-    const uint4* mine = reinterpret_cast<const uint4*>(xr + gl * E);
     uint4 v[E8];                                   // (a lane past the end of the row holds zeros: the last columns)
+    if constexpr (kAligned) {
+        const uint4* mine = reinterpret_cast<const uint4*>(xr + gl * E);
 #pragma unroll
-    for (int c = 0; c < E8; ++c) v[c] = gl * E < d ? __ldg(mine + c) : make_uint4(0, 0, 0, 0);
+        for (int c = 0; c < E8; ++c) v[c] = gl * E < d ? __ldg(mine + c) : make_uint4(0, 0, 0, 0);
+    } else {
+        auto pair = [&](uint32_t col) -> uint32_t {
+            const uint32_t a = col < d ? __ldg(xr + col) : 0u, b = col + 1 < d ? __ldg(xr + col + 1) : 0u;
+            return a | (b << 16);
+        };
+#pragma unroll
+        for (int c = 0; c < E8; ++c) {
+            const uint32_t col = gl * E + 8u * c;
+            v[c] = make_uint4(pair(col), pair(col + 2), pair(col + 4), pair(col + 6));
+        }
+    }
     const uint32_t tau_key = narrow_search15<G>([&](uint32_t t) {
         uint32_t cnt = 0;
 #pragma unroll
@@ -445,7 +459,7 @@ __device__ __forceinline__ void narrow_count_path(const uint16_t* __restrict__ x
 // Denser k (more than an eighth of the row: no leaf bound applies): every row takes the bit-by-bit count over the
 // row in registers, 15 rounds for a bf16 key, and the ordered emit from the row.  The warp kernels and the general
 // kernel pay their fixed cost per row for these short rows; here a warp serves 32 / G rows at once.
-template <int E8, int G>
+template <int E8, int G, bool kAligned>
 __global__ void __launch_bounds__(kNarrowWarps * 32)
 mp_topk_fwd_bf16_narrow_dense_kernel(const uint16_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                      int16_t* __restrict__ cols_out, uint16_t* __restrict__ vals_out,
@@ -468,16 +482,16 @@ mp_topk_fwd_bf16_narrow_dense_kernel(const uint16_t* __restrict__ x, uint32_t ro
         const uint64_t r = bundle * kRows + group;
         const bool valid = r < rows;
         const uint64_t row64 = valid ? r : rows - 1;     // a group past the last row runs along on the last row
-        narrow_count_path<E8, G>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
+        narrow_count_path<E8, G, kAligned>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
                                  cols_out, vals_out, rows_out, tau_out, guess);
     }
 }
 
-template <int E8, int G>
+template <int E8, int G, bool kAligned = true>
 dct_status_t launch_narrow_dense(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k, int16_t* cols_out,
                                  void* vals_out, int32_t* rows_out, void* tau_out, dct_result_t* result,
                                  cudaStream_t stream) {
-    auto kernel = mp_topk_fwd_bf16_narrow_dense_kernel<E8, G>;
+    auto kernel = mp_topk_fwd_bf16_narrow_dense_kernel<E8, G, kAligned>;
     int per_sm = 0;
     DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kNarrowWarps * 32, 0));
     if (per_sm < 1) return DCT_ERR_UNSUPPORTED;
@@ -506,7 +520,7 @@ dct_status_t launch_narrow_dense(const void* x_act, uint32_t rows, uint32_t d, u
 // step as in the bf16 kernels; the lower 16 bits come from the bucket's members: the smallest of them if all are
 // needed (the usual case: one member), the largest if one is, else 16 more rounds over the row's keys.  Called by the
 // whole warp; groups without a row run along and store nothing.
-template <int G>
+template <int G, bool kAligned = true>
 __device__ __forceinline__ void narrow_bisect_f32(const uint32_t* __restrict__ xr, uint32_t d, bool valid, uint32_t k,
                                                   size_t out_base, uint32_t row, int16_t* __restrict__ cols_out,
                                                   uint32_t* __restrict__ vals_out, int32_t* __restrict__ rows_out,
@@ -518,7 +532,16 @@ __device__ __forceinline__ void narrow_bisect_f32(const uint32_t* __restrict__ x
     uint4 up[4];                                   // upper halves of the lane's 32 columns, eight to a register quad
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-        const uint4 v = gl * E < d ? __ldg(reinterpret_cast<const uint4*>(xr + gl * E) + c) : make_uint4(0, 0, 0, 0);
+        uint4 v;
+        if constexpr (kAligned) {
+            v = gl * E < d ? __ldg(reinterpret_cast<const uint4*>(xr + gl * E) + c) : make_uint4(0, 0, 0, 0);
+        } else {                               // any width, any address: columns past the end read as zeros
+            const uint32_t col = gl * E + 4u * c;
+            v.x = col < d ? __ldg(xr + col) : 0u;
+            v.y = col + 1 < d ? __ldg(xr + col + 1) : 0u;
+            v.z = col + 2 < d ? __ldg(xr + col + 2) : 0u;
+            v.w = col + 3 < d ? __ldg(xr + col + 3) : 0u;
+        }
         key[4 * c] = v.x & 0x7FFFFFFFu;
         key[4 * c + 1] = v.y & 0x7FFFFFFFu;
         key[4 * c + 2] = v.z & 0x7FFFFFFFu;
@@ -552,7 +575,8 @@ __device__ __forceinline__ void narrow_bisect_f32(const uint32_t* __restrict__ x
         uint32_t lo = 0xFFFFFFFFu, hi = 0;
         for (uint32_t m = members; m; m &= m - 1) {
             // (a lane past the end of the row holds zeros: nothing of its own to read)
-            const uint32_t v = gl * E < d ? xr[gl * E + __ffs(m) - 1] & 0x7FFFFFFFu : 0u;
+            const uint32_t col = gl * E + __ffs(m) - 1;
+            const uint32_t v = col < d ? xr[col] & 0x7FFFFFFFu : 0u;
             lo = v < lo ? v : lo;
             hi = v > hi ? v : hi;
         }
@@ -602,7 +626,7 @@ __device__ __forceinline__ void narrow_bisect_f32(const uint32_t* __restrict__ x
 }
 
 // Denser k, fp32: the two-level bit-by-bit count over the row in registers (narrow_bisect_f32), for every row.
-template <int G>
+template <int G, bool kAligned>
 __global__ void __launch_bounds__(kNarrowWarps * 32, 2)
 mp_topk_fwd_f32_narrow_dense_kernel(const uint32_t* __restrict__ x, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                     int16_t* __restrict__ cols_out, uint32_t* __restrict__ vals_out,
@@ -625,16 +649,16 @@ mp_topk_fwd_f32_narrow_dense_kernel(const uint32_t* __restrict__ x, uint32_t row
         const uint64_t r = bundle * kRows + group;
         const bool valid = r < rows;
         const uint64_t row64 = valid ? r : rows - 1;
-        narrow_bisect_f32<G>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
+        narrow_bisect_f32<G, kAligned>(x + row64 * ld, d, valid, k, static_cast<size_t>(row64) * k, static_cast<uint32_t>(row64),
                              cols_out, vals_out, rows_out, tau_out, guess);
     }
 }
 
-template <int G>
+template <int G, bool kAligned = true>
 dct_status_t launch_narrow_dense_f32(const void* x_act, uint32_t rows, uint32_t d, uint32_t ld, uint32_t k,
                                      int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                      dct_result_t* result, cudaStream_t stream) {
-    auto kernel = mp_topk_fwd_f32_narrow_dense_kernel<G>;
+    auto kernel = mp_topk_fwd_f32_narrow_dense_kernel<G, kAligned>;
     int per_sm = 0;
     DCT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kNarrowWarps * 32, 0));
     if (per_sm < 1) return DCT_ERR_UNSUPPORTED;
@@ -660,7 +684,19 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
                                     int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                     dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
-    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0) return DCT_OK;
+    const bool odd = !aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0 || d % 8 != 0;
+    if (odd || (d <= 256 && d % 32 != 0)) {
+        // Rows the 16-byte loads of every other fast kernel cannot take (odd widths, odd strides, odd addresses): up to
+        // 512 columns they take the count over the row with 16-bit loads, for every k (the general kernel: 0.1 to 0.2
+        // TB/s).  So do short rows that are not whole lanes of 32 columns (100, 200 columns: the warp-per-row kernels
+        // spend a warp on a few hundred bytes).
+        if (d > 512) return DCT_OK;
+        *handled = true;
+        if (d <= 64) return launch_narrow_dense<4, 2, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        if (d <= 128) return launch_narrow_dense<4, 4, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        if (d <= 256) return launch_narrow_dense<4, 8, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        return launch_narrow_dense<4, 16, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    }
     *handled = true;
     // The count over the row in registers, for every row (15 rounds): the denser k on rows of up to 256 columns, and
     // every k on rows of up to 128 columns, where it beats the bound-and-candidates kernel as well (1572864 rows of 64
@@ -699,7 +735,18 @@ dct_status_t launch_fwd_f32_narrow(const void* x_act, uint32_t rows, uint32_t d,
                                    int16_t* cols_out, void* vals_out, int32_t* rows_out, void* tau_out,
                                    dct_result_t* result, cudaStream_t stream, bool* handled) {
     *handled = false;
-    if (!aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 32 != 0) return DCT_OK;
+    const bool odd = !aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 4 != 0;
+    if (odd || (d <= 256 && d % 32 != 0)) {
+        // rows the 16-byte loads cannot take: up to 512 columns, the count over the row with 32-bit loads, for every k;
+        // so do short rows that are not whole lanes of 32 columns
+        if (d > 512) return DCT_OK;
+        *handled = true;
+        if (d <= 64) return launch_narrow_dense_f32<2, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        if (d <= 128) return launch_narrow_dense_f32<4, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        if (d <= 256) return launch_narrow_dense_f32<8, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+        return launch_narrow_dense_f32<16, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
+    }
+    if (d % 32 != 0) return DCT_OK;
     // 288 to 480 columns, the denser k: 16 lanes per row (the bounds-and-bit-tables kernel of the 512-column buffer
     // is crowded by rows that fill only part of it: 320 columns, k = 80: 0.47 TB/s)
     if (d > 256 && d < 512 && fwd_candidates_per_lane(d, k) == 0) {

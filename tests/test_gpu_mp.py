@@ -351,6 +351,33 @@ def test_mp_many_short_rows(dtype, d, ld):
         assert int(cols.max()) < d
 
 
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
+@pytest.mark.parametrize("d,ld,shift", [(1, 1, 0), (7, 7, 0), (33, 40, 0), (64, 64, 1), (100, 100, 0), (127, 131, 0),
+                                        (128, 128, 3), (250, 250, 0), (256, 260, 0), (257, 257, 1), (500, 500, 0),
+                                        (512, 516, 0), (512, 512, 1)])
+def test_mp_short_rows_at_any_width_stride_and_address(dtype, d, ld, shift):
+    """Rows of up to 512 columns that do not start on 16-byte boundaries or are not whole 16-byte units (odd widths, odd
+    strides, a matrix that starts `shift` elements into its buffer): every k, rows of different scales, dead rows,
+    ties, fewer than k non-zeros; the columns past the end of a row are never read as part of it."""
+    rows = 16 * 148 * 2 + 5
+    buf = torch.full((rows * ld + shift + 8,), 7.0e30, dtype=torch.float32, device=G.DEV)   # huge values around the rows
+    x = inputs.mp_activations(rows, d, 391 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=392 + d, ld=ld)
+    sign = torch.where(inputs.dp_gaussian(rows * ld, 393 + d, G.DEV).view(rows, ld) > 0, 1.0, -1.0)
+    scale = torch.tensor([1.0, 30.0, 1e-2, 1.0, 1e3, 1.0, 1.0], device=G.DEV).repeat(rows // 7 + 1)[:rows]
+    x = x * sign * scale[:, None]
+    x[3] = 0.0
+    x[4] = -1.25
+    x[5, 2:] = 0.0
+    x[6] = inputs.quantize_mantissa(x[6], 1)
+    x[:, d:] = 7.0e30                                  # the padding between rows must never win
+    buf[shift:shift + rows * ld] = x.reshape(-1)
+    xs = buf.to(dtype)[shift:shift + rows * ld].view(rows, ld)
+    gx = inputs.mp_gradients(rows, d, 394 + d, dtype=dtype, device=G.DEV, ld=ld)
+    for k in sorted({1, max(1, d // 20), max(1, d // 4), max(1, d // 2), d}):
+        cols = _compare_fwd_bwd(xs, gx, d, k)
+        assert int(cols.max()) < d
+
+
 @pytest.mark.parametrize("d", [516, 768, 1024, 1540, 2048, 2052, 4096, 4100, 8192, 12000, 16384, 24580, 32768])
 def test_mp_f32_rows_wider_than_512(d):
     """fp32 rows of more than 512 columns that the sparse warp-per-row kernel leaves out (every k beyond 4096
