@@ -182,9 +182,12 @@ DCT_API dct_status_t dct_dp_compress(
  * d <= 512) or by one CTA per row (bf16 rows of 3073..32768 columns with k
  * up to 3d/8 where the warp kernel does not apply; fp32 rows of
  * 513..32768 columns that the warp kernels leave out, k up to 3d/8);
- * everything else (denser k, odd strides, cols_out not 4-byte aligned
- * for the denser and the wide cases) takes a general kernel that is several
- * times slower.  status may also be DCT_ERR_TIMEOUT if a
+ * short rows are held in registers, several rows to a warp (bf16 up to 128
+ * columns and fp32 up to 256: every k; bf16 up to 512 columns: k up to d/8;
+ * rows of up to 512 columns at any width, stride and address: every k).
+ * Everything else (denser k on longer rows, longer rows at odd strides,
+ * cols_out not 4-byte aligned for the denser and the wide cases) takes a
+ * general kernel that is several times slower.  status may also be DCT_ERR_TIMEOUT if a
  * bounded wait for an asynchronous copy gave up (not seen in practice; the
  * outputs are then incomplete).
  */
