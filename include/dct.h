@@ -184,7 +184,7 @@ DCT_API dct_status_t dct_dp_compress(
  * 513..32768 columns that the warp kernels leave out, k up to 3d/8);
  * short rows are held in registers, several rows to a warp (bf16 up to 128
  * columns and fp32 up to 256: every k; bf16 up to 512 columns: k up to d/8;
- * rows of up to 512 columns at any width, stride and address: every k).
+ * rows of up to 1024 columns at any width, stride and address: every k).
  * Everything else (denser k on longer rows, longer rows at odd strides,
  * cols_out not 4-byte aligned for the denser and the wide cases) takes a
  * general kernel that is several times slower.  status may also be DCT_ERR_TIMEOUT if a

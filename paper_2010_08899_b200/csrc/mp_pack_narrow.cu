@@ -687,11 +687,12 @@ dct_status_t launch_fwd_bf16_narrow(const void* x_act, uint32_t rows, uint32_t d
     const bool odd = !aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 2) % 16 != 0 || d % 8 != 0;
     if (odd || (d <= 256 && d % 32 != 0)) {
         // Rows the 16-byte loads of every other fast kernel cannot take (odd widths, odd strides, odd addresses): up to
-        // 512 columns they take the count over the row with 16-bit loads, for every k (the general kernel: 0.1 to 0.2
+        // 1024 columns they take the count over the row with 16-bit loads, for every k (the general kernel: 0.1 to 0.4
         // TB/s).  So do short rows that are not whole lanes of 32 columns (100, 200 columns: the warp-per-row kernels
         // spend a warp on a few hundred bytes).
-        if (d > 512) return DCT_OK;
+        if (d > 1024) return DCT_OK;
         *handled = true;
+        if (d > 512) return launch_narrow_dense<4, 32, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
         if (d <= 64) return launch_narrow_dense<4, 2, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
         if (d <= 128) return launch_narrow_dense<4, 4, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
         if (d <= 256) return launch_narrow_dense<4, 8, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
@@ -737,10 +738,11 @@ dct_status_t launch_fwd_f32_narrow(const void* x_act, uint32_t rows, uint32_t d,
     *handled = false;
     const bool odd = !aligned_to(x_act, 16) || (static_cast<size_t>(ld) * 4) % 16 != 0 || d % 4 != 0;
     if (odd || (d <= 256 && d % 32 != 0)) {
-        // rows the 16-byte loads cannot take: up to 512 columns, the count over the row with 32-bit loads, for every k;
+        // rows the 16-byte loads cannot take: up to 1024 columns, the count over the row with 32-bit loads, for every k;
         // so do short rows that are not whole lanes of 32 columns
-        if (d > 512) return DCT_OK;
+        if (d > 1024) return DCT_OK;
         *handled = true;
+        if (d > 512) return launch_narrow_dense_f32<32, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
         if (d <= 64) return launch_narrow_dense_f32<2, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
         if (d <= 128) return launch_narrow_dense_f32<4, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);
         if (d <= 256) return launch_narrow_dense_f32<8, false>(x_act, rows, d, ld, k, cols_out, vals_out, rows_out, tau_out, result, stream);

@@ -354,12 +354,13 @@ def test_mp_many_short_rows(dtype, d, ld):
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float32])
 @pytest.mark.parametrize("d,ld,shift", [(1, 1, 0), (7, 7, 0), (33, 40, 0), (64, 64, 1), (100, 100, 0), (127, 131, 0),
                                         (128, 128, 3), (250, 250, 0), (256, 260, 0), (257, 257, 1), (500, 500, 0),
-                                        (512, 516, 0), (512, 512, 1)])
+                                        (512, 516, 0), (512, 512, 1), (513, 513, 0), (1000, 1004, 0), (1001, 1001, 0),
+                                        (1024, 1024, 1)])
 def test_mp_short_rows_at_any_width_stride_and_address(dtype, d, ld, shift):
-    """Rows of up to 512 columns that do not start on 16-byte boundaries or are not whole 16-byte units (odd widths, odd
+    """Rows of up to 1024 columns that do not start on 16-byte boundaries or are not whole 16-byte units (odd widths, odd
     strides, a matrix that starts `shift` elements into its buffer): every k, rows of different scales, dead rows,
     ties, fewer than k non-zeros; the columns past the end of a row are never read as part of it."""
-    rows = 16 * 148 * 2 + 5
+    rows = (16 * 148 * 2 if d <= 512 else 16 * 148) + 5
     buf = torch.full((rows * ld + shift + 8,), 7.0e30, dtype=torch.float32, device=G.DEV)   # huge values around the rows
     x = inputs.mp_activations(rows, d, 391 + d, dtype=torch.float32, device=G.DEV, col_scale_seed=392 + d, ld=ld)
     sign = torch.where(inputs.dp_gaussian(rows * ld, 393 + d, G.DEV).view(rows, ld) > 0, 1.0, -1.0)
