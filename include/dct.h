@@ -402,7 +402,7 @@ DCT_API dct_status_t dct_mp_pack_host(
  * a gradient hook that runs inside a framework whose caching allocator already owns the whole GPU
  * (a raw cudaMalloc there can fail outright, and it stalls every stream of the device while it
  * runs), or a plug-in that is only ever handed the tensors it must transform.  For them the tile
- * descriptors live in an array that is part of the library image itself: 262,400 bytes of device
+ * descriptors live in an array that is part of the library image itself: 262,656 bytes of device
  * memory on every GPU that loads the library, held until the process exits.  The call allocates
  * nothing -- no cudaMalloc, no cudaFree, no library routine that allocates.
  *

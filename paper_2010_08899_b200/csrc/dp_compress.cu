@@ -338,7 +338,11 @@ __device__ __forceinline__ void compress_tile_body(const float* __restrict__ gra
                                                    int32_t* __restrict__ idx_out, float* __restrict__ val_out,
                                                    uint64_t capacity, dct_result_t* __restrict__ result,
                                                    CompressCtrl* ctrl, uint64_t* __restrict__ tile_state,
-                                                   uint32_t num_tiles, uint32_t tile, uint32_t spin_limit) {
+                                                   uint32_t num_tiles, uint32_t tile, uint32_t spin_limit,
+                                                   uint32_t first_valid = 0) {
+    // first_valid != 0: grad and residual point first_valid (1 to 3) elements BEFORE the vector, on the 16-byte boundary
+    // below it, and n counts from there.  Those elements are read (they share the vector's first 16 bytes) but belong to
+    // somebody else: never flagged, never written; the indices that go out count from the vector's own first element.
     __shared__ uint32_t s_warp_tot[kWarps];   // (gt << 16) | eq of each warp, each <= 512
     __shared__ uint32_t s_excl[2];
     __shared__ uint32_t s_abort;
@@ -352,7 +356,7 @@ __device__ __forceinline__ void compress_tile_body(const float* __restrict__ gra
 
     float w[kVecs * 4];
     uint32_t valid_mask = 0xFFFFu;
-    const bool full_tile = kVectorised && (tile_base + kTileElems <= n);
+    const bool full_tile = kVectorised && (tile_base + kTileElems <= n) && tile_base >= first_valid;
     if (full_tile) {
         float4 g4[kVecs], e4[kVecs];
 #pragma unroll
@@ -373,7 +377,7 @@ __device__ __forceinline__ void compress_tile_body(const float* __restrict__ gra
 #pragma unroll
         for (int b = 0; b < kVecs * 4; ++b) {
             const uint32_t i = warp_base + (b >> 2) * 128 + lane * 4 + (b & 3);
-            const bool valid = i < n;
+            const bool valid = i < n && i >= first_valid;
             w[b] = valid ? (grad ? __fadd_rn(grad[i], residual[i]) : residual[i]) : 0.0f;
             valid_mask |= valid ? (1u << b) : 0u;
         }
@@ -427,8 +431,8 @@ __device__ __forceinline__ void compress_tile_body(const float* __restrict__ gra
     if (cta_tot != 0) {                        // (nothing flagged in this tile: no output, no rewrite)
         __syncthreads();
         if (warp_tot != 0)
-            emit_warp(w, gt_mask, eq_mask, warp_base, before_warp, s_excl[0], s_excl[1], budget, capacity, s_abort != 0,
-                      idx_out, val_out, residual);
+            emit_warp(w, gt_mask, eq_mask, warp_base - first_valid, before_warp, s_excl[0], s_excl[1], budget, capacity,
+                      s_abort != 0, idx_out, val_out, residual + first_valid);
     }
 }
 
@@ -439,7 +443,7 @@ dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ resi
                         int32_t* __restrict__ idx_out, float* __restrict__ val_out, uint64_t capacity,
                         dct_result_t* __restrict__ result, CompressCtrl* ctrl,
                         uint64_t* __restrict__ tile_state, uint32_t num_tiles, uint32_t fixed_tile,
-                        uint32_t spin_limit, const uint32_t* __restrict__ enabled = nullptr) {
+                        uint32_t spin_limit, const uint32_t* __restrict__ enabled = nullptr, uint32_t first_valid = 0) {
     __shared__ uint32_t s_tile;
     if (enabled && *enabled == 0) return;     // a conditional call that is not needed
     // A CTA works through tickets until none is left (the grid need not be as large as the number of tiles).  Tiles
@@ -450,7 +454,7 @@ dp_compress_tile_kernel(const float* __restrict__ grad, float* __restrict__ resi
         const uint32_t tile = s_tile;
         if (tile >= num_tiles) return;
         compress_tile_body<kVectorised>(grad, residual, n, tau_p, budget_p, idx_out, val_out, capacity, result, ctrl,
-                                        tile_state, num_tiles, tile, spin_limit);
+                                        tile_state, num_tiles, tile, spin_limit, first_valid);
         if (fixed_tile != kInvalidTile) return;
         __syncthreads();                      // the tile's shared-memory words are free for the next one
     }
@@ -529,6 +533,7 @@ struct LayerDesc {
     uint32_t first_desc;   // index of the vector's first tile descriptor
     uint32_t num_full;     // full tiles handled by the streaming kernel (0 for an unaligned vector)
     uint32_t num_tiles;    // all tiles, a ragged last one included
+    uint32_t idx_bias;     // grad and residual point this many elements before the vector (see compress_tile_body)
 };
 struct BatchTable {
     const LayerDesc* layers;
@@ -545,7 +550,7 @@ struct TileParams {
     dct_result_t* result;
     uint64_t* tile_state;          // descriptors of this vector: look-back never leaves them
     uint64_t capacity, budget;
-    uint32_t tau_key, last_tile;
+    uint32_t tau_key, last_tile, idx_bias;
 };
 __device__ __forceinline__ TileParams load_params(const LayerDesc& d, uint64_t* tile_state_base) {
     TileParams p;
@@ -559,6 +564,7 @@ __device__ __forceinline__ TileParams load_params(const LayerDesc& d, uint64_t* 
     p.budget = d.tie_budget ? *d.tie_budget : ~0ull;
     p.tau_key = key_f32(*d.tau);
     p.last_tile = d.num_tiles - 1;
+    p.idx_bias = d.idx_bias;
     return p;
 }
 
@@ -735,7 +741,9 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
             const uint32_t start = sm.slot_start[r];
             const uint64_t excl_gt = sm.prefix[r][0], excl_eq = sm.prefix[r][1];
             const bool aborted = sm.aborted[r] != 0;
-            const uint32_t tile_base = tile * kTileElems;
+            // (indices count from the vector's own first element; the residual pointer moves with them)
+            const uint32_t tile_base = tile * kTileElems - (kBatched ? 0u : P.idx_bias);
+            float* const residual_own = kBatched ? P.residual : P.residual + P.idx_bias;
 #pragma unroll 4
             for (uint32_t q = dw * 32u + lane; q < cnt; q += 32u * kDrainWarps) {
                 const uint32_t at = start + q;
@@ -743,7 +751,7 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
                 const uint32_t local_eq = (ent.x >> 12) & 0xFFFu;
                 place_survivor(tile_base + (ent.x & 0xFFFu), __uint_as_float(ent.y), (ent.x & kEqBit) != 0,
                                excl_gt + (q - local_eq), excl_eq + local_eq, P.budget, P.capacity, aborted, P.idx_out,
-                               P.val_out, P.residual);
+                               P.val_out, residual_own);
             }
             __syncwarp();                      // every lane has read its entries: the compute warps may overwrite them
             if (lane == 0) {
@@ -1024,7 +1032,8 @@ using namespace dct;
 
 extern "C" size_t dct_dp_compress_workspace_bytes(uint64_t n) {
     if (n == 0 || n > 0x7FFFFFFFull) return 0;
-    const size_t bytes = kCtrlBytes + sizeof(uint64_t) * static_cast<size_t>(dp_compress_num_tiles(n));
+    // (+ 3: a vector that starts 4, 8 or 12 bytes past a 16-byte boundary is worked on from that boundary)
+    const size_t bytes = kCtrlBytes + sizeof(uint64_t) * static_cast<size_t>(dp_compress_num_tiles(n + 3));
     return (bytes + 255) & ~static_cast<size_t>(255);
 }
 
@@ -1050,13 +1059,23 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     auto* ctrl = static_cast<CompressCtrl*>(workspace);
     auto* tile_state = reinterpret_cast<uint64_t*>(static_cast<char*>(workspace) + kCtrlBytes);
-    const uint32_t n32 = static_cast<uint32_t>(n);
-    const uint32_t num_tiles = dp_compress_num_tiles(n);
+    // A gradient and a residual that sit the same 4, 8 or 12 bytes past a 16-byte boundary (views at the same offset
+    // into two flat buffers) are worked on from that boundary: the `lead` elements before them lie in the same 16 bytes
+    // of the same allocation, are read and never written, and the fast kernel's 16-byte accesses apply to all tiles but
+    // the first.  (Any other misalignment: one CTA per tile with plain loads, about a quarter of the rate.)
+    uint32_t lead = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(grad) & 15u) / 4u);
+    if (lead != (reinterpret_cast<uintptr_t>(residual) & 15u) / 4u || n + lead > 0x7FFFFFFFull) lead = 0;
+    grad -= lead;
+    residual -= lead;
+    const uint32_t n32 = static_cast<uint32_t>(n) + lead;
+    const uint32_t num_tiles = dp_compress_num_tiles(n32);
     const uint32_t num_full = n32 / kTileElems;
+    const uint32_t first_full = lead ? 1u : 0u;       // the first tile holds elements that are not the vector's
     const DebugConfig& dbg = debug_config();
 
     DCT_CUDA_TRY(launch_chained(dp_compress_init_kernel, (num_tiles + 1023) / 1024, 1024, stream, ctrl, tile_state, num_tiles,
-                                result, dbg.first_ticket, static_cast<const uint32_t*>(nullptr)));
+                                result, dbg.first_ticket > first_full ? dbg.first_ticket : first_full,
+                                static_cast<const uint32_t*>(nullptr)));
     const bool vec = aligned_to(grad, 16) && aligned_to(residual, 16);
     if (!vec) {
         const int sms_t = sm_count();
@@ -1068,7 +1087,13 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         DCT_CUDA_TRY(cudaGetLastError());
         return DCT_OK;
     }
-    if (num_full > 0) {
+    if (lead && num_full > 0) {   // the first tile, before the kernel whose tiles wait for its counts
+        dp_compress_tile_kernel<true><<<1, kThreads, 0, stream>>>(
+            grad, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles, 0u,
+            dbg.spin_limit, static_cast<const uint32_t*>(nullptr), lead);
+        DCT_CUDA_TRY(cudaGetLastError());
+    }
+    if (num_full > first_full) {
         static thread_local int configured_device = -1;
         int dev = 0;
         DCT_CUDA_TRY(cudaGetDevice(&dev));
@@ -1082,7 +1107,7 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         if (sms <= 0) return DCT_ERR_CUDA;
         const uint32_t ctas_per_sm = 2;
         const uint32_t max_grid = static_cast<uint32_t>(sms) * ctas_per_sm;
-        const uint32_t grid = num_full < max_grid ? num_full : max_grid;
+        const uint32_t grid = num_full - first_full < max_grid ? num_full - first_full : max_grid;
         LayerDesc single{};
         single.grad = grad;
         single.residual = residual;
@@ -1096,13 +1121,14 @@ extern "C" dct_status_t dct_dp_compress(const float* grad, float* residual, uint
         single.first_desc = 0;
         single.num_full = num_full;
         single.num_tiles = num_tiles;
+        single.idx_bias = lead;
         DCT_CUDA_TRY(launch_chained_smem(dp_compress_stream_kernel<false>, grid, kStreamThreads, sizeof(StreamSmem), stream,
                                          single, BatchTable{}, num_full, ctrl, tile_state, dbg.spin_limit));
     }
     if (num_tiles > num_full) {   // ragged last tile
         dp_compress_tile_kernel<true><<<1, kThreads, 0, stream>>>(
             grad, residual, n32, tau, tie_budget, idx_out, val_out, capacity, result, ctrl, tile_state, num_tiles,
-            num_full, dbg.spin_limit);
+            num_full, dbg.spin_limit, static_cast<const uint32_t*>(nullptr), lead);
         DCT_CUDA_TRY(cudaGetLastError());
     }
     return DCT_OK;
@@ -1283,13 +1309,14 @@ extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, ui
 // dct_dp_compress_static: the same operator for callers that cannot hand over a workspace
 // ------------------------------------------------------------------------------------------
 // The tile descriptors and the ticket live in this file-scope device array instead of a caller
-// buffer.  Every GPU that loads the library carries these 256.25 KiB until the process exits.
+// buffer.  Every GPU that loads the library carries these 256.5 KiB until the process exits.
 // In host code the array's name is only a stand-in: the device address is fetched once per device
 // with cudaGetSymbolAddress (that device being current) and handed to the kernels like any workspace.
 namespace {
 
 constexpr uint64_t kStaticMaxElems = DCT_DP_COMPRESS_STATIC_MAX_N;
-constexpr size_t kStaticScratchBytes = kCtrlBytes + sizeof(uint64_t) * (kStaticMaxElems / kTileElems);
+// (one descriptor more than whole tiles: a vector that starts past a 16-byte boundary is worked on from that boundary)
+constexpr size_t kStaticScratchBytes = (kCtrlBytes + sizeof(uint64_t) * (kStaticMaxElems / kTileElems + 1) + 255) / 256 * 256;
 static_assert(kStaticMaxElems % kTileElems == 0, "the static scratch is sized in whole tiles");
 
 static __device__ __align__(256) unsigned char dct_static_scratch[kStaticScratchBytes];

@@ -61,6 +61,30 @@ def test_misaligned_pointers(offset):
     _compare_compress(g_dev, e_dev, tau_dev, None, n)
 
 
+@pytest.mark.parametrize("offset", [1, 2, 3])
+@pytest.mark.parametrize("n", [3, 4093, 4096, 20_001, 3 * 4096 - 2, (1 << 21) + 7])
+def test_gradient_and_residual_at_the_same_odd_offset(offset, n):
+    """Views at the same element offset into two flat buffers: both vectors sit 4, 8 or 12 bytes past a 16-byte
+    boundary.  The elements next to them in the buffers (before the first, after the last) are left alone, the
+    indices count from the vector's own first element, ties and a capacity that cuts the list off work as ever."""
+    gbuf = inputs.dp_gaussian(n + 8, 15 + n % 7, G.DEV)
+    ebuf = inputs.dp_gaussian(n + 8, 16 + n % 5, G.DEV) * 0.5
+    if n > 1000:
+        gbuf = inputs.quantize_mantissa(gbuf, 4)
+        ebuf = torch.zeros_like(ebuf)
+    g_dev, e_view = gbuf[offset:offset + n], ebuf[offset:offset + n]
+    assert g_dev.data_ptr() % 16 == 4 * offset and e_view.data_ptr() % 16 == 4 * offset
+    around = ebuf.clone()
+    for k in sorted({1, max(1, n // 50), n}):
+        tau_dev, r = G.select(g_dev, e_view, k)
+        want = oracle.dp_select(g_dev.cpu().numpy(), e_view.cpu().numpy(), k)
+        assert bits32(tau_dev.cpu().numpy())[0] == bits32(want.tau)[0] and (r.n_gt, r.n_eq) == (want.n_gt, want.n_eq)
+        for budget, cap in ((None, n), (k - r.n_gt, n), (None, max(1, k // 2))):
+            ebuf.copy_(around)
+            _compare_compress(g_dev, e_view, tau_dev, budget, cap)
+            assert torch.equal(ebuf[:offset], around[:offset]) and torch.equal(ebuf[offset + n:], around[offset + n:])
+
+
 def test_heavy_ties_and_exact_k():
     n = 300_000
     g_dev = inputs.quantize_mantissa(inputs.dp_gaussian(n, 77, G.DEV), 2)
