@@ -144,8 +144,11 @@ DCT_API dct_status_t dct_threshold_select(
  *              DCT_ERR_CAPACITY or DCT_ERR_TIMEOUT) are written.
  *   workspace  >= dct_dp_compress_workspace_bytes(n), 256-byte aligned.
  *
- * grad and residual should be 16-byte aligned; other alignments are accepted
- * and take a slower scalar path.
+ * grad and residual should be 16-byte aligned, or sit the same 4, 8 or 12
+ * bytes past a 16-byte boundary (views at one element offset into two flat
+ * buffers; the up to three elements before them in their 16-byte unit are
+ * then read, never written); other alignments are accepted and take a slower
+ * scalar path.
  */
 DCT_API dct_status_t dct_dp_compress(
     const float* grad, float* residual, uint64_t n,
