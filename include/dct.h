@@ -108,6 +108,10 @@ DCT_API size_t dct_dp_compress_workspace_bytes(uint64_t n);
  *   result    device block; n_gt, n_eq and status are written.
  *   workspace >= dct_threshold_select_workspace_bytes(n), 256-byte aligned.
  *
+ * grad (and residual) should be 16-byte aligned or sit the same 4, 8 or 12
+ * bytes past a 16-byte boundary (the up to three elements before them in
+ * their 16-byte unit are then read); other alignments take scalar loads.
+ *
  * Returns DCT_OK after enqueueing; DCT_ERR_INVALID_ARG / DCT_ERR_WORKSPACE /
  * DCT_ERR_CUDA without having launched anything.
  */

@@ -115,10 +115,14 @@ __global__ void select_init_kernel(SelectWorkspace* ws, uint32_t n, uint32_t k, 
 }
 
 // Where a pass reads its keys from.
-struct VectorSource {        // key(fl32(grad[i] + residual[i])), i < n
+struct VectorSource {        // key(fl32(grad[i] + residual[i])), skip <= i < n
     const float* grad;
     const float* residual;   // may be null
+    uint32_t skip = 0;       // leading elements that are not the vector's (a vector that starts 4, 8 or 12 bytes past a
+                             // 16-byte boundary is read from that boundary, so that the 16-byte loads apply)
 };
+template <typename Source> __device__ __forceinline__ uint32_t skip_of(const Source&) { return 0u; }
+__device__ __forceinline__ uint32_t skip_of(const VectorSource& s) { return s.skip; }
 struct StridedSource {       // the same at (i / 8) * stride + i % 8: groups of 8 neighbours, `stride` elements apart
     const float* grad;
     const float* residual;
@@ -210,7 +214,7 @@ __device__ __forceinline__ void select_pass_body(const Source& src, SelectState*
         const uint32_t base = chunk * kSelChunk;
         bool done = false;
         if constexpr (kVectorised) {      // VectorSource with 16-byte aligned pointers
-            if (base + kSelChunk <= n) {
+            if (base + kSelChunk <= n && base >= skip_of(src)) {
                 float4 g4[kSelVecs], e4[kSelVecs];
 #pragma unroll
                 for (int j = 0; j < kSelVecs; ++j) {
@@ -242,7 +246,7 @@ __device__ __forceinline__ void select_pass_body(const Source& src, SelectState*
                 }
 #pragma unroll
                 for (int u = 0; u < kBatch; ++u)
-                    if (i0 + u * kSelThreads < lim) consume(key[u]);
+                    if (i0 + u * kSelThreads < lim && i0 + u * kSelThreads >= skip_of(src)) consume(key[u]);
             }
         }
     }
@@ -349,7 +353,7 @@ select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t
     const uint32_t num_chunks = (n + kSelChunk - 1) / kSelChunk;
     for (uint32_t chunk = blockIdx.x; chunk < num_chunks; chunk += gridDim.x) {
         const uint32_t base = chunk * kSelChunk;
-        if (kVectorised && base + kSelChunk <= n) {
+        if (kVectorised && base + kSelChunk <= n && base >= src.skip) {
             float4 g4[kSelVecs], e4[kSelVecs];
 #pragma unroll
             for (int j = 0; j < kSelVecs; ++j) {
@@ -379,7 +383,7 @@ select_filter_kernel(VectorSource src, uint32_t n, SelectWorkspace* ws, uint32_t
             // whole warps stay together so that the ballots above see every lane
             for (uint32_t i0 = base + (threadIdx.x & ~31u); i0 < n && i0 < base + kSelChunk; i0 += kSelThreads) {
                 const uint32_t i = i0 + lane_id();
-                const bool in = i < n && i < base + kSelChunk;
+                const bool in = i < n && i < base + kSelChunk && i >= src.skip;
                 const uint32_t key = in ? key_at(src, i) : 0u;
                 above += in && key > hi ? 1u : 0u;
                 keep(in && key >= lo && key <= hi, key);
@@ -574,6 +578,14 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     auto* ws = static_cast<SelectWorkspace*>(workspace);
     auto* cand_keys = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + sizeof(SelectWorkspace));
+    // A vector 4, 8 or 12 bytes past a 16-byte boundary (and a residual, if any, at the same offset) is read from that
+    // boundary: the 1 to 3 elements before it share its first 16 bytes, are loaded and not counted.
+    uint32_t lead = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(grad) & 15u) / 4u);
+    if ((residual && lead != (reinterpret_cast<uintptr_t>(residual) & 15u) / 4u) || n + lead > 0x7FFFFFFFull) lead = 0;
+    grad -= lead;
+    if (residual) residual -= lead;
+    const uint64_t n_own = n;                       // (the workspace was sized for this many elements)
+    n += lead;
     const uint32_t n32 = static_cast<uint32_t>(n), k32 = static_cast<uint32_t>(k);
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
@@ -582,12 +594,12 @@ extern "C" dct_status_t dct_threshold_select(const float* grad, const float* res
         return static_cast<int>(chunks < static_cast<uint64_t>(sms) * 4 ? (chunks ? chunks : 1) : sms * 4);
     };
     const bool vec = aligned_to(grad, 16) && (!residual || aligned_to(residual, 16));
-    const VectorSource vsrc{grad, residual};
+    const VectorSource vsrc{grad, residual, lead};
 
     // sampled single-pass path?
     uint32_t sample_n = 0, sample_k = 0, sample_k_hi = 0, stride = 0, capacity = 0;
-    if (n >= kMinSampledN) {
-        capacity = candidate_capacity(n);
+    if (n_own >= kMinSampledN) {
+        capacity = candidate_capacity(n_own);
         stride = (n32 / (kSampleSize / kSampleGroup)) & ~(kSampleGroup - 1u);   // groups start on 32-byte boundaries
         sample_n = kSampleSize;
         // millions of elements above tau: the band around tau is the shorter candidate list, where there is one
