@@ -500,6 +500,7 @@ struct __align__(128) StreamSmem {
     float* slot_residual[kSlots];
     uint64_t slot_budget[kSlots];
     uint64_t slot_capacity[kSlots];
+    uint32_t slot_bias[kSlots];
     uint32_t ahead[4];                   // counts of a tile taken ahead of its turn: eq | gt << 13 | warps that added << 26
     volatile uint32_t ring_tail[kDrainWarps];   // drain warp -> compute: running count of ring entries it is done with
     volatile uint32_t drained[kDrainWarps];     // drain warp -> compute: tiles it is done with (their slots may be reused)
@@ -539,6 +540,7 @@ struct BatchTable {
     const LayerDesc* layers;
     const uint32_t* full_prefix;   // [num_layers + 1] running count of streaming-kernel tiles
     const uint32_t* slow_prefix;   // [num_layers + 1] running count of tile-kernel tiles
+    const uint32_t* head_layers;   // vectors whose first tile goes to the tile kernel ahead of the streaming kernel
     uint32_t num_layers;
 };
 // What a role needs to know about the vector it is working on, held in registers.
@@ -611,10 +613,12 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
         const float* grad = single.grad;
         const float* residual = single.residual;
         uint32_t cur_layer = 0, work_lo = 0, work_hi = total_work;     // work items of the current vector
+        uint32_t first_full = 0;             // batched: the vector's first tile of this kernel (1 if its tile 0 is a head)
         if (kBatched) {
             work_hi = batch.full_prefix[1];
             grad = batch.layers[0].grad;
             residual = batch.layers[0].residual;
+            first_full = batch.layers[0].idx_bias ? 1u : 0u;
         }
         uint32_t ticket = atomicAdd(&ctrl->ticket, 1u);
         for (uint32_t it = 0;; ++it) {
@@ -642,8 +646,9 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
                     work_hi = batch.full_prefix[lo + 1];
                     grad = batch.layers[cur_layer].grad;
                     residual = batch.layers[cur_layer].residual;
+                    first_full = batch.layers[cur_layer].idx_bias ? 1u : 0u;
                 }
-                tile -= work_lo;                                       // tile index inside its vector
+                tile = tile - work_lo + first_full;                    // tile index inside its vector
             }
             // the next ticket is requested now; its latency overlaps the wait below
             if (tile != kInvalidTile) ticket = atomicAdd(&ctrl->ticket, 1u);
@@ -701,9 +706,10 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
                 if (kBatched) {
                     sm.slot_idx_out[r] = P.idx_out;
                     sm.slot_val_out[r] = P.val_out;
-                    sm.slot_residual[r] = P.residual;
+                    sm.slot_residual[r] = P.residual + P.idx_bias;        // (the vector's own first element)
                     sm.slot_budget[r] = P.budget;
                     sm.slot_capacity[r] = P.capacity;
+                    sm.slot_bias[r] = P.idx_bias;
                 }
             }
             __syncwarp();
@@ -731,6 +737,7 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
                 P.residual = sm.slot_residual[r];
                 P.budget = sm.slot_budget[r];
                 P.capacity = sm.slot_capacity[r];
+                P.idx_bias = sm.slot_bias[r];
             }
             if (!__all_sync(0xFFFFFFFFu, mbar_wait_bounded(&sm.entries_ready[r], parity, kMbarLimit, &sm.stop))) {
                 sm.stop = 1;
@@ -742,8 +749,8 @@ dp_compress_stream_kernel(const LayerDesc single, const BatchTable batch, uint32
             const uint64_t excl_gt = sm.prefix[r][0], excl_eq = sm.prefix[r][1];
             const bool aborted = sm.aborted[r] != 0;
             // (indices count from the vector's own first element; the residual pointer moves with them)
-            const uint32_t tile_base = tile * kTileElems - (kBatched ? 0u : P.idx_bias);
-            float* const residual_own = kBatched ? P.residual : P.residual + P.idx_bias;
+            const uint32_t tile_base = tile * kTileElems - P.idx_bias;
+            float* const residual_own = kBatched ? P.residual : P.residual + P.idx_bias;   // (batched: moved already)
 #pragma unroll 4
             for (uint32_t q = dw * 32u + lane; q < cnt; q += 32u * kDrainWarps) {
                 const uint32_t at = start + q;
@@ -1019,7 +1026,18 @@ dp_compress_tile_batched_kernel(const BatchTable batch, uint32_t total_slow, Com
     // an aligned vector contributes only its last tile; an unaligned one all of them
     const uint32_t tile = d.num_full + (work - batch.slow_prefix[lo]);
     compress_tile_body<false>(d.grad, d.residual, d.n, d.tau, d.tie_budget, d.idx_out, d.val_out, d.capacity,
-                              d.result, ctrl, tile_state_base + d.first_desc, d.num_tiles, tile, spin_limit);
+                              d.result, ctrl, tile_state_base + d.first_desc, d.num_tiles, tile, spin_limit, d.idx_bias);
+}
+
+// The first tiles of the vectors that are worked on from the 16-byte boundary below them (LayerDesc::idx_bias != 0):
+// they hold elements that are not the vector's, so the tile kernel's per-element path takes them -- before the streaming
+// kernel, whose tiles of these vectors wait for their counts.  One CTA per such vector.
+__global__ void __launch_bounds__(kThreads, kTileKernelMinBlocks)
+dp_compress_heads_batched_kernel(const BatchTable batch, CompressCtrl* ctrl, uint64_t* __restrict__ tile_state_base,
+                                 uint32_t spin_limit) {
+    const LayerDesc& d = batch.layers[batch.head_layers[blockIdx.x]];
+    compress_tile_body<false>(d.grad, d.residual, d.n, d.tau, d.tie_budget, d.idx_out, d.val_out, d.capacity,
+                              d.result, ctrl, tile_state_base + d.first_desc, d.num_tiles, 0u, spin_limit, d.idx_bias);
 }
 
 }  // namespace
@@ -1172,13 +1190,14 @@ dct_status_t dct::compress_presummed_if(const uint32_t* enabled, float* residual
 namespace {
 
 struct BatchLayout {
-    size_t layers_off, full_off, slow_off, state_off, bytes;
+    size_t layers_off, full_off, slow_off, head_off, state_off, bytes;
     uint64_t total_tiles;
 };
 BatchLayout batch_layout(const uint64_t* n, uint32_t num_layers) {
     BatchLayout L{};
     uint64_t tiles = 0;
-    for (uint32_t l = 0; l < num_layers; ++l) tiles += dp_compress_num_tiles(n[l]);
+    // (+ 3: a vector that starts 4, 8 or 12 bytes past a 16-byte boundary is worked on from that boundary)
+    for (uint32_t l = 0; l < num_layers; ++l) tiles += dp_compress_num_tiles(n[l] + 3);
     L.total_tiles = tiles;
     size_t off = kCtrlBytes;
     L.layers_off = off;
@@ -1188,6 +1207,8 @@ BatchLayout batch_layout(const uint64_t* n, uint32_t num_layers) {
     off += sizeof(uint32_t) * (num_layers + 1);
     L.slow_off = off;
     off += sizeof(uint32_t) * (num_layers + 1);
+    L.head_off = off;
+    off += sizeof(uint32_t) * num_layers;
     off = (off + 255) & ~static_cast<size_t>(255);
     L.state_off = off;
     off += sizeof(uint64_t) * tiles;
@@ -1231,14 +1252,20 @@ extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, ui
     auto* descs = reinterpret_cast<LayerDesc*>(table.data());
     auto* full_prefix = reinterpret_cast<uint32_t*>(table.data() + (L.full_off - L.layers_off));
     auto* slow_prefix = reinterpret_cast<uint32_t*>(table.data() + (L.slow_off - L.layers_off));
-    uint32_t first_desc = 0, total_full = 0, total_slow = 0;
+    auto* head_layers = reinterpret_cast<uint32_t*>(table.data() + (L.head_off - L.layers_off));
+    uint32_t first_desc = 0, total_full = 0, total_slow = 0, num_heads = 0;
     for (uint32_t l = 0; l < num_layers; ++l) {
         const dct_dp_layer_t& a = layers[l];
         LayerDesc& d = descs[l];
-        const uint32_t n32 = static_cast<uint32_t>(a.n);
-        const bool vec = aligned_to(a.grad, 16) && aligned_to(a.residual, 16);
-        d.grad = a.grad;
-        d.residual = a.residual;
+        // a gradient and a residual the same 4, 8 or 12 bytes past a 16-byte boundary (the usual state of a layer
+        // inside two flat buffers) are worked on from that boundary: see dct_dp_compress
+        uint32_t lead = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(a.grad) & 15u) / 4u);
+        if (lead != (reinterpret_cast<uintptr_t>(a.residual) & 15u) / 4u || a.n + lead > 0x7FFFFFFFull) lead = 0;
+        const uint32_t n32 = static_cast<uint32_t>(a.n) + lead;
+        const bool vec = aligned_to(a.grad - lead, 16) && aligned_to(a.residual - lead, 16);
+        d.grad = a.grad - lead;
+        d.residual = a.residual - lead;
+        d.idx_bias = lead;
         d.tau = a.tau;
         d.tie_budget = a.tie_budget;
         d.idx_out = a.idx_out;
@@ -1247,11 +1274,14 @@ extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, ui
         d.capacity = a.capacity;
         d.n = n32;
         d.first_desc = first_desc;
-        d.num_tiles = dp_compress_num_tiles(a.n);
+        d.num_tiles = dp_compress_num_tiles(n32);
         d.num_full = vec ? n32 / kTileElems : 0;
+        // the first tile of a vector with leading elements goes to the tile kernel ahead of the streaming kernel
+        const uint32_t head = lead && d.num_full > 0 ? 1u : 0u;
+        if (head) head_layers[num_heads++] = l;
         full_prefix[l] = total_full;
         slow_prefix[l] = total_slow;
-        total_full += d.num_full;
+        total_full += d.num_full - head;
         total_slow += d.num_tiles - d.num_full;
         first_desc += d.num_tiles;
     }
@@ -1268,6 +1298,7 @@ extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, ui
     batch.layers = reinterpret_cast<const LayerDesc*>(ws + L.layers_off);
     batch.full_prefix = reinterpret_cast<const uint32_t*>(ws + L.full_off);
     batch.slow_prefix = reinterpret_cast<const uint32_t*>(ws + L.slow_off);
+    batch.head_layers = reinterpret_cast<const uint32_t*>(ws + L.head_off);
     batch.num_layers = num_layers;
     const int sms = sm_count();
     if (sms <= 0) return DCT_ERR_CUDA;
@@ -1279,6 +1310,10 @@ extern "C" dct_status_t dct_dp_compress_batched(const dct_dp_layer_t* layers, ui
         dp_compress_batched_init_kernel<<<grid, 1024, 0, stream>>>(ctrl, tile_state,
                                                                    static_cast<uint32_t>(L.total_tiles), batch.layers,
                                                                    num_layers);
+        DCT_CUDA_TRY(cudaGetLastError());
+    }
+    if (num_heads > 0) {
+        dp_compress_heads_batched_kernel<<<num_heads, kThreads, 0, stream>>>(batch, ctrl, tile_state, dbg.spin_limit);
         DCT_CUDA_TRY(cudaGetLastError());
     }
     if (total_full > 0) {

@@ -80,6 +80,52 @@ def test_batched_dense_layers_many_tiles_per_cta():
         assert np.array_equal(bits32(a["residual"].cpu().numpy()), bits32(e_want))
 
 
+@pytest.mark.parametrize("dense", [False, True])
+def test_batched_layers_inside_two_flat_buffers(dense):
+    """The layers of a model as views into one flat gradient buffer and one flat residual buffer: an odd-sized tensor
+    shifts every layer behind it off the 16-byte boundaries, gradient and residual alike.  Every layer must come out as
+    the oracle's, and what lies between the layers (and before the first, after the last) must be left alone."""
+    sizes = [4096 * 3 + 1, 250, 1 << 20, 7, 65536 + 3, 4096, 100_000, 4095, 4096 * 2 + 2, (1 << 21) + 5, 33]
+    gaps = [0, 1, 0, 0, 2, 0, 0, 3, 0, 0, 0]            # unused elements behind a layer (another tensor's, say)
+    total = sum(sizes) + sum(gaps) + 8
+    g_flat = inputs.dp_gaussian(total, 501, G.DEV)
+    e_flat = inputs.dp_gaussian(total, 502, G.DEV) * 0.2
+    e_before = e_flat.clone()
+    layers, spans, off = [], [], 1                      # the first layer starts one element into the buffers
+    for j, (n, gap) in enumerate(zip(sizes, gaps)):
+        g, e = g_flat[off:off + n], e_flat[off:off + n]
+        assert g.data_ptr() % 16 == e.data_ptr() % 16
+        k = max(1, n // (3 if dense else 40))
+        tau, sel = G.select(g, e, k)
+        cap = n if j % 3 else max(1, k // 2)
+        budget = None if j % 2 else torch.tensor([k - sel.n_gt], dtype=torch.int64, device=G.DEV)
+        layers.append(dict(grad=g, residual=e, n=n, tau=tau.clone(), tie_budget=budget, capacity=cap,
+                           idx_out=torch.full((cap + 8,), -7, dtype=torch.int32, device=G.DEV),
+                           val_out=torch.full((cap + 8,), -7.0, device=G.DEV), result=B.new_result()))
+        spans.append((off, off + n))
+        off += n + gap
+    want = []
+    for a in layers:
+        e = a["residual"].cpu().numpy().copy()
+        bud = None if a["tie_budget"] is None else int(a["tie_budget"].item())
+        want.append((oracle.dp_compress(a["grad"].cpu().numpy(), e, a["tau"].cpu().numpy()[0], bud, a["capacity"]), e))
+    ws = B.new_workspace(B.dct_dp_compress_batched_workspace_bytes(sizes))
+    ws.fill_(0xCD)
+    B.dct_dp_compress_batched(layers, ws)
+    for a, (w, e_want) in zip(layers, want):
+        r = B.read_result(a["result"])
+        assert (r.count, r.needed) == (w.count, w.needed)
+        assert r.status == (B.DCT_ERR_CAPACITY if w.needed > a["capacity"] else B.DCT_OK)
+        assert np.array_equal(a["idx_out"][:r.count].cpu().numpy(), w.idx)
+        assert np.array_equal(bits32(a["val_out"][:r.count].cpu().numpy()), bits32(w.val))
+        assert bool((a["idx_out"][r.count:] == -7).all())
+        assert np.array_equal(bits32(a["residual"].cpu().numpy()), bits32(e_want))
+    outside = torch.ones(total, dtype=torch.bool, device=G.DEV)
+    for lo, hi in spans:
+        outside[lo:hi] = False
+    assert torch.equal(e_flat[outside], e_before[outside])
+
+
 def test_batched_rejects_bad_layers_on_the_host():
     layers = _make_layers([5000, 6000], 7)
     ws = B.new_workspace(B.dct_dp_compress_batched_workspace_bytes([5000, 6000]))
