@@ -33,6 +33,8 @@ struct LayerState {                 // device copy of a layer's description + it
     uint64_t n_gt;                  // elements known to be above the prefix bucket
     uint32_t n, k;
     uint32_t prefix, k_rem;
+    uint32_t skip;                  // leading elements that are not the layer's (see LayerHead::skip)
+    uint32_t pad;
     uint32_t hist[kPasses][kBins];
 };
 
@@ -47,8 +49,9 @@ struct LayerHead {
     uint64_t first_chunk;
     uint64_t n_gt;
     uint32_t n, k;
-};
-static_assert(sizeof(LayerHead) <= offsetof(LayerState, prefix), "head must not reach into the select state");
+    uint32_t skip;                  // a layer 4, 8 or 12 bytes past a 16-byte boundary (and its residual with it) is read
+    uint32_t pad;                   // from that boundary: grad, residual and n count from there, the first `skip`
+};                                  // elements are loaded and not counted
 
 // chunk -> layer: the last layer whose first chunk is <= chunk
 __device__ __forceinline__ uint32_t layer_of_chunk(const LayerState* layers, uint32_t num_layers, uint64_t chunk) {
@@ -76,6 +79,7 @@ __global__ void batched_init_kernel(LayerState* layers, const LayerHead* heads, 
             st->first_chunk = hd.first_chunk;
             st->n = hd.n;
             st->k = hd.k;
+            st->skip = hd.skip;
             st->n_gt = 0;
             st->prefix = 0;
             st->k_rem = hd.k;
@@ -138,7 +142,8 @@ batched_pass_kernel(LayerState* layers, uint32_t num_layers, uint64_t total_chun
         };
         const bool vec = (reinterpret_cast<uintptr_t>(grad) & 15u) == 0 &&
                          (residual == nullptr || (reinterpret_cast<uintptr_t>(residual) & 15u) == 0);
-        if (vec && base + kChunk <= n) {
+        const uint32_t skip = st.skip;
+        if (vec && base + kChunk <= n && base >= skip) {
             float4 g4[kVecs], e4[kVecs];
 #pragma unroll
             for (int j = 0; j < kVecs; ++j) {
@@ -156,7 +161,7 @@ batched_pass_kernel(LayerState* layers, uint32_t num_layers, uint64_t total_chun
             }
         } else {
             for (uint32_t i = base + threadIdx.x; i < n && i < base + kChunk; i += kThreads)
-                consume(key_f32(residual ? __fadd_rn(grad[i], residual[i]) : grad[i]));
+                if (i >= skip) consume(key_f32(residual ? __fadd_rn(grad[i], residual[i]) : grad[i]));
         }
     }
     chain_release_next();
@@ -251,9 +256,13 @@ extern "C" dct_status_t dct_threshold_select_batched(const dct_select_layer_t* l
     std::vector<LayerHead> heads(num_layers);
     for (uint32_t l = 0; l < num_layers; ++l) {
         const dct_select_layer_t& a = layers[l];
-        heads[l] = LayerHead{a.grad, a.residual, a.tau_out, a.result, total_chunks, 0, static_cast<uint32_t>(a.n),
-                             static_cast<uint32_t>(a.k)};
-        total_chunks += (a.n + kChunk - 1) / kChunk;
+        uint32_t lead = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(a.grad) & 15u) / 4u);
+        if ((a.residual && lead != (reinterpret_cast<uintptr_t>(a.residual) & 15u) / 4u) || a.n + lead > 0x7FFFFFFFull)
+            lead = 0;
+        const uint64_t n_view = a.n + lead;
+        heads[l] = LayerHead{a.grad - lead, a.residual ? a.residual - lead : nullptr, a.tau_out, a.result, total_chunks, 0,
+                             static_cast<uint32_t>(n_view), static_cast<uint32_t>(a.k), lead, 0};
+        total_chunks += (n_view + kChunk - 1) / kChunk;
     }
     // pageable source: the runtime has staged the bytes by the time the call returns, so `heads` may go away
     DCT_CUDA_TRY(cudaMemcpyAsync(dev_heads, heads.data(), sizeof(LayerHead) * num_layers, cudaMemcpyHostToDevice, stream));

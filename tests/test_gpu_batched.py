@@ -104,6 +104,15 @@ def test_batched_layers_inside_two_flat_buffers(dense):
                            val_out=torch.full((cap + 8,), -7.0, device=G.DEV), result=B.new_result()))
         spans.append((off, off + n))
         off += n + gap
+    # the thresholds of all layers in one batched select, from the same views
+    sel_layers = [dict(grad=a["grad"], residual=a["residual"], n=a["n"], k=max(1, a["n"] // (3 if dense else 40)),
+                       tau_out=torch.zeros(1, device=G.DEV), result=B.new_result()) for a in layers]
+    ws_sel = B.new_workspace(B.dct_threshold_select_batched_workspace_bytes(len(sizes)))
+    B.dct_threshold_select_batched(sel_layers, ws_sel)
+    for a, sl in zip(layers, sel_layers):
+        w = oracle.dp_select(a["grad"].cpu().numpy(), a["residual"].cpu().numpy(), sl["k"])
+        r = B.read_result(sl["result"])
+        assert bits32(sl["tau_out"].cpu().numpy())[0] == bits32(w.tau)[0] and (r.n_gt, r.n_eq) == (w.n_gt, w.n_eq)
     want = []
     for a in layers:
         e = a["residual"].cpu().numpy().copy()
