@@ -90,10 +90,15 @@ __device__ __forceinline__ uint32_t cta_lower_bound(const int32_t* __restrict__ 
     }
     return a;
 }
+template <bool kShifted>
 __global__ void __launch_bounds__(256)
 dp_decompress_tiled_kernel(const int32_t* __restrict__ idx, const float* __restrict__ val,
                            const dct_result_t* __restrict__ packed, uint64_t capacity, float* __restrict__ dense,
-                           uint32_t n, int accumulate, dct_result_t* __restrict__ result) {
+                           uint32_t n, int accumulate, dct_result_t* __restrict__ result, uint32_t lead_arg) {
+    const uint32_t lead = kShifted ? lead_arg : 0u;          // (the aligned instance carries no checks for it)
+    // lead != 0: the dense vector starts 4, 8 or 12 bytes past a 16-byte boundary; `dense` points to that boundary, n
+    // counts from there and an index i of the list means position i + lead.  The `lead` elements before the vector share
+    // its first 16 bytes: they are read when accumulating, never written.
     __shared__ __align__(16) float tile[kDecompTile];
     __shared__ uint32_t s_taken[2];     // entries the tile took, and
     __shared__ uint32_t s_first[2];     // the index of the first entry after them (two rounds in turn)
@@ -107,15 +112,29 @@ dp_decompress_tiled_kernel(const int32_t* __restrict__ idx, const float* __restr
         const uint32_t hi = (n - lo > per) ? lo + per : n;
         // the entries of this CTA's range: idx[a, end) (idx ascending; malformed input only costs misplaced work,
         // never a fault)
-        uint32_t a = cta_lower_bound(idx, count, lo);
-        const uint32_t end = hi < n ? cta_lower_bound(idx, count, hi) : count;
+        const uint32_t n_own = n - lead;
+        auto place_of = [&](uint32_t i) -> uint32_t { return i < n_own ? i + lead : 0xFFFFFFFFu; };   // (past the end: nowhere)
+        uint32_t a = cta_lower_bound(idx, count, lo > lead ? lo - lead : 0u);
+        const uint32_t end = hi < n ? cta_lower_bound(idx, count, hi - lead) : count;
+        auto before_vector = [&](uint32_t at) -> bool {     // a position that is not the vector's
+            if constexpr (kShifted) return at < lead; else return false;
+        };
+        auto store4 = [&](uint32_t at, float4 v) {     // 16 bytes at position `at`, but never the elements before the vector
+            if (!before_vector(at)) {
+                st_stream_f4(dense + at, v);
+            } else {
+                if (lead <= 1) dense[1] = v.y;
+                if (lead <= 2) dense[2] = v.z;
+                dense[3] = v.w;
+            }
+        };
         if (threadIdx.x < 2) {
             s_taken[threadIdx.x] = 0;
             s_first[threadIdx.x] = 0xFFFFFFFFu;
         }
         // index of the first entry that is not placed yet (none: past every tile); after a tile it is what the thread
         // that ran into it saw, so only this one is a load of its own
-        uint32_t first = a < end ? static_cast<uint32_t>(idx[a]) : 0xFFFFFFFFu;
+        uint32_t first = a < end ? place_of(static_cast<uint32_t>(idx[a])) : 0xFFFFFFFFu;
         uint32_t round = 0;
         for (uint32_t t_lo = lo; t_lo < hi; t_lo += kDecompTile) {
             const uint32_t t_hi = hi - t_lo > kDecompTile ? t_lo + kDecompTile : hi;
@@ -125,8 +144,9 @@ dp_decompress_tiled_kernel(const int32_t* __restrict__ idx, const float* __restr
             if (first >= t_hi) {
                 if (!accumulate) {
                     for (uint32_t i = threadIdx.x * 4; i < len4; i += blockDim.x * 4)
-                        st_stream_f4(dense + t_lo + i, make_float4(0.f, 0.f, 0.f, 0.f));
-                    for (uint32_t i = len4 + threadIdx.x; i < len; i += blockDim.x) dense[t_lo + i] = 0.0f;
+                        store4(t_lo + i, make_float4(0.f, 0.f, 0.f, 0.f));
+                    for (uint32_t i = len4 + threadIdx.x; i < len; i += blockDim.x)
+                        if (!before_vector(t_lo + i)) dense[t_lo + i] = 0.0f;
                 }
                 continue;
             }
@@ -146,7 +166,7 @@ dp_decompress_tiled_kernel(const int32_t* __restrict__ idx, const float* __restr
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {     // four entries in flight (the values on the chance that they are needed)
                     const uint32_t j = j0 + u * blockDim.x;
-                    i4[u] = j < end ? static_cast<uint32_t>(idx[j]) : 0xFFFFFFFFu;
+                    i4[u] = j < end ? place_of(static_cast<uint32_t>(idx[j])) : 0xFFFFFFFFu;
                     v4[u] = j < end ? val[j] : 0.0f;
                 }
 #pragma unroll
@@ -165,8 +185,9 @@ dp_decompress_tiled_kernel(const int32_t* __restrict__ idx, const float* __restr
             if (seen != 0xFFFFFFFFu) atomicMin(&s_first[round & 1u], seen);
             __syncthreads();      // every entry of the tile is in place
             for (uint32_t i = threadIdx.x * 4; i < len4; i += blockDim.x * 4)
-                st_stream_f4(dense + t_lo + i, *reinterpret_cast<const float4*>(tile + i));
-            for (uint32_t i = len4 + threadIdx.x; i < len; i += blockDim.x) dense[t_lo + i] = tile[i];
+                store4(t_lo + i, *reinterpret_cast<const float4*>(tile + i));
+            for (uint32_t i = len4 + threadIdx.x; i < len; i += blockDim.x)
+                if (!before_vector(t_lo + i)) dense[t_lo + i] = tile[i];
             a += s_taken[round & 1u];
             first = s_first[round & 1u];
             ++round;
@@ -177,7 +198,7 @@ dp_decompress_tiled_kernel(const int32_t* __restrict__ idx, const float* __restr
     for (uint64_t j = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; j < count;
          j += static_cast<uint64_t>(gridDim.x) * blockDim.x) {
         const int32_t i = idx[j];
-        if (static_cast<uint32_t>(i) >= n || (j > 0 && i <= idx[j - 1])) bad = true;
+        if (static_cast<uint32_t>(i) >= n - lead || (j > 0 && i <= idx[j - 1])) bad = true;
     }
     if (bad) atomicMax(&result->status, static_cast<uint32_t>(DCT_ERR_BAD_MASK));
 }
@@ -441,9 +462,15 @@ extern "C" dct_status_t dct_dp_decompress(const int32_t* idx, const float* val, 
     // streams spread over the whole vector (2^30 elements: 0.749 -> 0.620 ms; ranges of 8192 or 32768 are slower)
     const uint64_t by_range = (n + 16383) / 16384;
     if (grid < by_range) grid = by_range;
-    if (aligned_to(dense, 16))
-        dp_decompress_tiled_kernel<<<static_cast<unsigned>(grid), 256, 0, stream>>>(idx, val, packed, capacity, dense,
-                                                                                   static_cast<uint32_t>(n), accumulate, result);
+    // (a dense vector 4, 8 or 12 bytes past a 16-byte boundary is written from that boundary on, its neighbours before it
+    // left alone)
+    const uint32_t lead = static_cast<uint32_t>((reinterpret_cast<uintptr_t>(dense) & 15u) / 4u);
+    if (lead == 0)
+        dp_decompress_tiled_kernel<false><<<static_cast<unsigned>(grid), 256, 0, stream>>>(
+            idx, val, packed, capacity, dense, static_cast<uint32_t>(n), accumulate, result, 0u);
+    else if (n + lead <= 0x7FFFFFFFull)
+        dp_decompress_tiled_kernel<true><<<static_cast<unsigned>(grid), 256, 0, stream>>>(
+            idx, val, packed, capacity, dense - lead, static_cast<uint32_t>(n) + lead, accumulate, result, lead);
     else
         dp_decompress_kernel<<<static_cast<unsigned>(grid), 256, 0, stream>>>(idx, val, packed, capacity, dense,
                                                                              static_cast<uint32_t>(n), accumulate, result);
